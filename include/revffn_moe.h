@@ -1,0 +1,205 @@
+/*
+ * revffn_moe.h -- C ABI of the B200 (sm_100a) library for the MoE coupling
+ * branch of a RevFFN block.
+ *
+ * The block (paper Sec. 3.1) splits the hidden state H = [X1, X2] into two
+ * streams of width h = d/2 and updates them in a coupled way.  This library
+ * implements the second update (Eq. 2) and what reversible back-propagation
+ * needs from it:
+ *
+ *   forward   Y2 = X2 + MLP(Norm(Y1))                         (Eq. 2)
+ *   inverse   X2 = Y2 - MLP(Norm(Y1))                         (Sec. 3.1, inverse pass)
+ *   backward  dY1 += J^T dY2 and the weight gradients, with the intermediates
+ *             recomputed from Y1 instead of cached            (Sec. 2, Sec. 3.1)
+ *
+ * with  MLP(y) = P_down( MLP_pt( P_up(y) ) )                  (Sec. 3.2)
+ * where P_up: R^h -> R^d and P_down: R^d -> R^h are bias-free linear adapters
+ * and MLP_pt is the base model's sparse MoE block evaluated in the d-wide
+ * space: a linear router, top-k selection (ties to the lower expert index),
+ * softmax over the k selected logits, routed SwiGLU experts, and an optional
+ * SwiGLU shared expert scaled by sigmoid(<w_sgate, u>).  Norm is RMSNorm over
+ * the h-wide stream with a learnable scale.
+ *
+ * Conventions
+ *   - T tokens (batch*seq flattened), d = d_model, h = d/2, E experts, k = top_k,
+ *     I = d_expert, I_s = d_shared.
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".
+ *   - Matrices are row-major [out, in], contiguous, 16-byte aligned.  Streams
+ *     (y1, x2, y2, dy2, dy1) are fp32 [T, h] with row stride ld_stream elements
+ *     (h for packed streams, d for views into an interleaved [X1, X2] tensor).
+ *   - The caller owns every buffer including the workspace.  The library
+ *     allocates no device memory, creates no streams and never synchronises,
+ *     except revffn_moe_status, which synchronises the given stream.
+ *   - All kernels are enqueued on the caller's CUDA stream (cudaStream_t passed
+ *     as void*).  Calls that share a workspace must be ordered on one stream.
+ *   - Return value: REVFFN_OK (0) or a negative revffn_error.  On an error
+ *     return nothing has been launched.  Device-side problems (a bounded wait
+ *     that expired) set a sticky status word in the workspace; read it with
+ *     revffn_moe_status.
+ */
+#ifndef REVFFN_MOE_H_
+#define REVFFN_MOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  REVFFN_OK = 0,
+  REVFFN_ERR_NULL = -1,         /* a required pointer is NULL                       */
+  REVFFN_ERR_SHAPE = -2,        /* descriptor violates a stated shape constraint    */
+  REVFFN_ERR_ALIGN = -3,        /* a pointer or stride is not 16-byte aligned       */
+  REVFFN_ERR_WORKSPACE = -4,    /* workspace smaller than revffn_moe_workspace_size */
+  REVFFN_ERR_ARCH = -5,         /* current device is not compute capability 10.x    */
+  REVFFN_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed                */
+  REVFFN_ERR_DEVICE_WAIT = -7,  /* status word: a bounded device-side wait expired  */
+  REVFFN_ERR_UNSUPPORTED = -8   /* valid request that this build does not implement */
+} revffn_error;
+
+enum { REVFFN_F32 = 0, REVFFN_BF16 = 1 };          /* weight_dtype                    */
+enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                       */
+
+/* flags */
+#define REVFFN_FLAG_FORCE_SIMT 1u  /* run bf16 GEMMs on the plain CUDA-core kernels (cross-check) */
+
+/*
+ * Block descriptor.  Shape constraints (else REVFFN_ERR_SHAPE):
+ *   tokens >= 0; d_model even; 1 <= top_k <= 8; top_k <= n_experts <= 256;
+ *   d_shared >= 0 (0 = no shared expert).
+ *   weight_dtype REVFFN_F32 : every width (h, d, I, I_s) a multiple of 4.
+ *   weight_dtype REVFFN_BF16: every width a multiple of 128 (TMA / tcgen05 tiles).
+ * With REVFFN_F32 all weights are float and every intermediate is fp32; with
+ * REVFFN_BF16 weights are bfloat16, GEMM operands are bf16 with fp32
+ * accumulation, and routing is still decided in higher precision from the
+ * fp32 stream.
+ */
+typedef struct {
+  int32_t tokens, d_model, n_experts, top_k, d_expert, d_shared;
+  int32_t weight_dtype;
+  int32_t norm_kind;
+  float norm_eps;
+  int64_t ld_stream;
+  uint32_t flags;
+} revffn_moe_desc;
+
+/* Weights of one block (Sec. 3.2 adapters; MLP_pt of the base model). */
+typedef struct {
+  const float* norm_gamma; /* [h] fp32 RMSNorm scale, NULL = ones                       */
+  const void* w_up;        /* [d, h]   P_up                                              */
+  const void* w_down;      /* [h, d]   P_down                                            */
+  const void* w_router;    /* [E, d]                                                     */
+  const float* b_router;   /* [E] fp32 router bias or NULL                               */
+  const void* w_gate;      /* [E, I, d] expert gate projections                          */
+  const void* w_upx;       /* [E, I, d] expert up projections                            */
+  const void* w_downx;     /* [E, d, I] expert down projections                          */
+  const void* ws_gate;     /* [I_s, d] shared expert (all four NULL iff d_shared == 0)   */
+  const void* ws_up;       /* [I_s, d]                                                   */
+  const void* ws_down;     /* [d, I_s]                                                   */
+  const void* ws_sgate;    /* [d]      shared-expert sigmoid gate                        */
+} revffn_moe_weights;
+
+/*
+ * Weight-gradient outputs, fp32, same shapes as the weights.  Any member may be
+ * NULL: that gradient is skipped (Sec. 3.3: stage 1 trains only the adapters,
+ * stage 2 the experts and adapters, the router stays frozen).  accumulate != 0
+ * adds to the buffers' contents instead of overwriting them.
+ */
+typedef struct {
+  float *norm_gamma, *w_up, *w_down, *w_router, *b_router, *w_gate, *w_upx, *w_downx,
+        *ws_gate, *ws_up, *ws_down, *ws_sgate;
+  int32_t accumulate;
+} revffn_moe_grads;
+
+/* Bytes of workspace forward/inverse (fwd_bytes) and backward (bwd_bytes) need.
+ * Both out-pointers are host pointers and may be NULL.  (Planner; no paper counterpart.) */
+int revffn_moe_workspace_size(const revffn_moe_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes);
+
+/*
+ * Eq. 2:  y2[t] = x2[t] + MLP(Norm(y1[t])).
+ *   y1, x2  in   fp32 [T, h] (stride ld_stream);  y2 out, may alias x2.
+ *   topk_idx_out  optional int32 [T, k]: selected experts per token in
+ *                 descending-logit order.
+ *   ws / ws_bytes workspace of at least fwd_bytes, 256-byte aligned.
+ */
+int revffn_moe_forward(const revffn_moe_desc* desc, const revffn_moe_weights* w,
+                       const float* y1, const float* x2, float* y2,
+                       int32_t* topk_idx_out, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Sec. 3.1 inverse pass:  x2[t] = y2[t] - MLP(Norm(y1[t])).  The branch is
+ * recomputed with the same kernels and reduction orders as the forward pass, so
+ * the subtracted term is bit-identical to the one that was added.
+ *   topk_idx_in   optional int32 [T, k]: reuse these expert sets instead of
+ *                 re-selecting them (gate weights are still recomputed).
+ *   x2 out, may alias y2.
+ */
+int revffn_moe_inverse(const revffn_moe_desc* desc, const revffn_moe_weights* w,
+                       const float* y1, const float* y2, float* x2,
+                       const int32_t* topk_idx_in, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Backward of Eq. 2 by recomputation (Sec. 2 "Reversible Networks", Sec. 3.1):
+ * given y1 and dy2 = dL/dY2, recompute the branch's intermediates, then
+ *   dy1_inout[t] += J^T dy2[t]      (fp32 [T, h], stride ld_stream)
+ *   grads->X (+)= dL/dX             for every non-NULL member.
+ * dL/dX2 equals dy2 and is not written.  The router may be frozen (its
+ * gradient pointers NULL) but the gradient through the gate values still
+ * reaches dy1.  ws must hold at least bwd_bytes.
+ */
+int revffn_moe_backward(const revffn_moe_desc* desc, const revffn_moe_weights* w,
+                        const float* y1, const float* dy2, float* dy1_inout,
+                        const revffn_moe_grads* grads, const int32_t* topk_idx_in,
+                        void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Synchronise the stream and copy the workspace's sticky device status word to
+ * *device_status (host pointer): 0 or a negative revffn_error.  (No paper counterpart.) */
+int revffn_moe_status(const void* ws, void* cuda_stream, int32_t* device_status);
+
+/* Text for an error code; static storage. */
+const char* revffn_strerror(int code);
+
+/*
+ * Introspection for tests: byte offset and size inside the backward workspace
+ * layout of a named intermediate ("n", "u", "gates", "sgate", "tok_row",
+ * "row_tok", "expert_off", "up", "hmid", "o", "hs", "s", "z", "ab", ...).
+ * The forward layout is a prefix of the backward layout.  Returns
+ * REVFFN_ERR_UNSUPPORTED for unknown names.  (No paper counterpart.)
+ */
+int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* offset, size_t* bytes);
+
+/*
+ * One C = A * B^T problem on either GEMM backend; used by the tests to check
+ * the tcgen05 kernels against the CUDA-core kernels.  See revffn_gemm_problem
+ * in the library source for field meanings.  (No paper counterpart.)
+ */
+typedef struct {
+  int32_t M, N, K;
+  int32_t a_mn_major, b_mn_major;  /* 0: [rows, K] K contiguous; 1: [K, rows] rows contiguous */
+  int32_t concat;                  /* 0 none, 1 N-concat (SwiGLU pair), 2 K-concat            */
+  int32_t epilogue;                /* 0 store, 1 swiglu, 2 rowscale, 3 couple, 4 dswiglu, 5 wgrad */
+  int32_t out_f32;                 /* store epilogue: fp32 instead of bf16 output             */
+  int32_t accumulate;
+  int32_t use_simt;
+  const void *A, *B0, *B1;         /* bf16                                                    */
+  int64_t lda, ldb;
+  void *C, *C1;
+  int64_t ldc, ldc1;
+  const float* rowscale;
+  const float* resid; int64_t ld_resid; float resid_sign;
+  void* ab; int64_t ld_ab;         /* dswiglu: [M, 2N] bf16 a|b in, da|db out                  */
+  float* dg_part; int32_t dg_ld;
+  /* grouping: 0 none, 1 rows grouped (group_off, tile_group, rows_total), 2 K grouped */
+  int32_t group_mode, n_groups;
+  const int32_t *group_off, *tile_group, *rows_total;
+  int64_t b_group_stride, c_group_stride;
+  int32_t a_col0, b_col0;
+} revffn_dbg_gemm_args;
+int revffn_dbg_gemm(const revffn_dbg_gemm_args* args, int32_t* status_word_dev, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REVFFN_MOE_H_ */

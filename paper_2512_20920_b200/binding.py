@@ -1,0 +1,200 @@
+"""ctypes binding of librevffn_moe.so: the same entry points as
+include/revffn_moe.h, taking torch tensors for device memory and the current
+torch CUDA stream.  Argument marshalling only; no arithmetic happens here, and
+there is no fallback: a missing library is an ImportError."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "librevffn_moe.so")
+
+F32, BF16 = 0, 1
+NORM_RMS, NORM_NONE = 0, 1
+FLAG_FORCE_SIMT = 1
+
+WEIGHT_NAMES = ("norm_gamma", "w_up", "w_down", "w_router", "b_router", "w_gate", "w_upx", "w_downx",
+                "ws_gate", "ws_up", "ws_down", "ws_sgate")
+_F32_ALWAYS = ("norm_gamma", "b_router")
+
+
+class RevffnError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where}: {revffn_strerror(code)} ({code})")
+        self.code = code
+
+
+class Desc(C.Structure):
+    _fields_ = [("tokens", C.c_int32), ("d_model", C.c_int32), ("n_experts", C.c_int32), ("top_k", C.c_int32),
+                ("d_expert", C.c_int32), ("d_shared", C.c_int32), ("weight_dtype", C.c_int32),
+                ("norm_kind", C.c_int32), ("norm_eps", C.c_float), ("ld_stream", C.c_int64), ("flags", C.c_uint32)]
+
+
+class Weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
+
+
+class Grads(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES] + [("accumulate", C.c_int32)]
+
+
+class DbgGemmArgs(C.Structure):
+    _fields_ = [("M", C.c_int32), ("N", C.c_int32), ("K", C.c_int32), ("a_mn_major", C.c_int32),
+                ("b_mn_major", C.c_int32), ("concat", C.c_int32), ("epilogue", C.c_int32), ("out_f32", C.c_int32),
+                ("accumulate", C.c_int32), ("use_simt", C.c_int32), ("A", C.c_void_p), ("B0", C.c_void_p),
+                ("B1", C.c_void_p), ("lda", C.c_int64), ("ldb", C.c_int64), ("C", C.c_void_p), ("C1", C.c_void_p),
+                ("ldc", C.c_int64), ("ldc1", C.c_int64), ("rowscale", C.c_void_p), ("resid", C.c_void_p),
+                ("ld_resid", C.c_int64), ("resid_sign", C.c_float), ("ab", C.c_void_p), ("ld_ab", C.c_int64),
+                ("dg_part", C.c_void_p), ("dg_ld", C.c_int32), ("group_mode", C.c_int32), ("n_groups", C.c_int32),
+                ("group_off", C.c_void_p), ("tile_group", C.c_void_p), ("rows_total", C.c_void_p),
+                ("b_group_stride", C.c_int64), ("c_group_stride", C.c_int64), ("a_col0", C.c_int32),
+                ("b_col0", C.c_int32)]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2512_20920_b200.build` "
+                          "(there is no fallback path)")
+    lib = C.CDLL(_LIB_PATH)
+    vp, sz = C.c_void_p, C.c_size_t
+    lib.revffn_moe_workspace_size.argtypes = [C.POINTER(Desc), C.POINTER(sz), C.POINTER(sz)]
+    lib.revffn_moe_forward.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, vp, vp, sz, vp]
+    lib.revffn_moe_inverse.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, vp, vp, sz, vp]
+    lib.revffn_moe_backward.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, C.POINTER(Grads), vp, vp,
+                                        sz, vp]
+    lib.revffn_moe_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
+    lib.revffn_strerror.argtypes = [C.c_int]
+    lib.revffn_strerror.restype = C.c_char_p
+    lib.revffn_moe_ws_lookup.argtypes = [C.POINTER(Desc), C.c_char_p, C.POINTER(sz), C.POINTER(sz)]
+    lib.revffn_dbg_gemm.argtypes = [C.POINTER(DbgGemmArgs), vp, vp]
+    for f in ("revffn_moe_workspace_size", "revffn_moe_forward", "revffn_moe_inverse", "revffn_moe_backward",
+              "revffn_moe_status", "revffn_moe_ws_lookup", "revffn_dbg_gemm"):
+        getattr(lib, f).restype = C.c_int
+    return lib
+
+
+lib = _load()
+
+
+def revffn_strerror(code: int) -> str:
+    return lib.revffn_strerror(int(code)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise RevffnError(code, where)
+
+
+def revffn_moe_workspace_size(desc: Desc):
+    f, b = C.c_size_t(0), C.c_size_t(0)
+    _check(lib.revffn_moe_workspace_size(C.byref(desc), C.byref(f), C.byref(b)), "revffn_moe_workspace_size")
+    return f.value, b.value
+
+
+def revffn_moe_forward(desc: Desc, w: Weights, y1, x2, y2, topk_idx_out, ws, stream: Optional[int] = None):
+    _check(lib.revffn_moe_forward(C.byref(desc), C.byref(w), _ptr(y1), _ptr(x2), _ptr(y2), _ptr(topk_idx_out),
+                                  _ptr(ws), ws.numel() * ws.element_size(), stream if stream is not None else _stream()),
+           "revffn_moe_forward")
+
+
+def revffn_moe_inverse(desc: Desc, w: Weights, y1, y2, x2, topk_idx_in, ws, stream: Optional[int] = None):
+    _check(lib.revffn_moe_inverse(C.byref(desc), C.byref(w), _ptr(y1), _ptr(y2), _ptr(x2), _ptr(topk_idx_in),
+                                  _ptr(ws), ws.numel() * ws.element_size(), stream if stream is not None else _stream()),
+           "revffn_moe_inverse")
+
+
+def revffn_moe_backward(desc: Desc, w: Weights, y1, dy2, dy1_inout, grads: Grads, topk_idx_in, ws,
+                        stream: Optional[int] = None):
+    _check(lib.revffn_moe_backward(C.byref(desc), C.byref(w), _ptr(y1), _ptr(dy2), _ptr(dy1_inout), C.byref(grads),
+                                   _ptr(topk_idx_in), _ptr(ws), ws.numel() * ws.element_size(),
+                                   stream if stream is not None else _stream()),
+           "revffn_moe_backward")
+
+
+def revffn_moe_status(ws, stream: Optional[int] = None) -> int:
+    out = C.c_int32(0)
+    _check(lib.revffn_moe_status(_ptr(ws), stream if stream is not None else _stream(), C.byref(out)),
+           "revffn_moe_status")
+    return out.value
+
+
+def ws_lookup(desc: Desc, name: str):
+    off, nbytes = C.c_size_t(0), C.c_size_t(0)
+    _check(lib.revffn_moe_ws_lookup(C.byref(desc), name.encode(), C.byref(off), C.byref(nbytes)), "revffn_moe_ws_lookup")
+    return off.value, nbytes.value
+
+
+class Block:
+    """One block's descriptor, device weights and workspace, with the three
+    passes as methods.  Pure marshalling around the C entry points."""
+
+    def __init__(self, *, tokens: int, d_model: int, n_experts: int, top_k: int, d_expert: int, d_shared: int,
+                 weight_dtype: int, weights: Dict[str, torch.Tensor], norm_kind: int = NORM_RMS,
+                 norm_eps: float = 1e-6, ld_stream: Optional[int] = None, flags: int = 0,
+                 workspace: Optional[torch.Tensor] = None, backward: bool = True):
+        self.desc = Desc(tokens, d_model, n_experts, top_k, d_expert, d_shared, weight_dtype, norm_kind, norm_eps,
+                         ld_stream if ld_stream is not None else d_model // 2, flags)
+        wdt = torch.bfloat16 if weight_dtype == BF16 else torch.float32
+        self.weights = {}
+        for name in WEIGHT_NAMES:
+            t = weights.get(name)
+            if t is None:
+                continue
+            want = torch.float32 if name in _F32_ALWAYS else wdt
+            if t.dtype != want or not t.is_cuda or not t.is_contiguous():
+                raise ValueError(f"weight {name}: need a contiguous CUDA tensor of {want}")
+            self.weights[name] = t
+        self.w = Weights(**{n: _ptr(self.weights.get(n)) for n in WEIGHT_NAMES})
+        self.fwd_bytes, self.bwd_bytes = revffn_moe_workspace_size(self.desc)
+        need = self.bwd_bytes if backward else self.fwd_bytes
+        if workspace is None:
+            workspace = torch.empty(need, dtype=torch.uint8, device="cuda")
+        if workspace.numel() * workspace.element_size() < need:
+            raise ValueError("workspace too small")
+        self.ws = workspace
+
+    @property
+    def tokens(self) -> int:
+        return self.desc.tokens
+
+    def forward(self, y1, x2, y2=None, topk_idx_out=None):
+        if y2 is None:
+            y2 = torch.empty_like(x2)
+        revffn_moe_forward(self.desc, self.w, y1, x2, y2, topk_idx_out, self.ws)
+        return y2
+
+    def inverse(self, y1, y2, x2=None, topk_idx_in=None):
+        if x2 is None:
+            x2 = torch.empty_like(y2)
+        revffn_moe_inverse(self.desc, self.w, y1, y2, x2, topk_idx_in, self.ws)
+        return x2
+
+    def backward(self, y1, dy2, dy1_inout, grads: Optional[Dict[str, torch.Tensor]] = None, accumulate: bool = False,
+                 topk_idx_in=None):
+        grads = grads or {}
+        for n, t in grads.items():
+            if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+                raise ValueError(f"gradient {n}: need a contiguous fp32 CUDA tensor")
+        g = Grads(**{n: _ptr(grads.get(n)) for n in WEIGHT_NAMES}, accumulate=1 if accumulate else 0)
+        revffn_moe_backward(self.desc, self.w, y1, dy2, dy1_inout, g, topk_idx_in, self.ws)
+        return dy1_inout
+
+    def status(self) -> int:
+        return revffn_moe_status(self.ws)
+
+    def buffer(self, name: str, dtype: torch.dtype) -> torch.Tensor:
+        """A named intermediate inside the workspace (tests only)."""
+        off, nbytes = ws_lookup(self.desc, name)
+        return self.ws[off:off + nbytes].view(dtype)

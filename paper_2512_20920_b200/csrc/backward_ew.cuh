@@ -1,0 +1,204 @@
+// Element-wise and reduction kernels of the backward pass (everything that is
+// not a matrix product).  Notation follows the forward pass: u = P_up(n),
+// z = sum_s g_s f_s(u) + sgate * S, F = P_down(z).
+#pragma once
+
+#include "common.cuh"
+
+namespace revffn {
+
+// Gb = T(G): the upstream gradient as a GEMM operand.
+template <typename T>
+__global__ void cast_stream_kernel(const float* __restrict__ g, int64_t ld, int tokens, int h, T* __restrict__ out) {
+  int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= (int64_t)tokens * h) return;
+  int t = (int)(i / h), c = (int)(i % h);
+  float4 v = *reinterpret_cast<const float4*>(g + (int64_t)t * ld + c);
+  T* o = out + i;
+  o[0] = from_f32<T>(v.x); o[1] = from_f32<T>(v.y); o[2] = from_f32<T>(v.z); o[3] = from_f32<T>(v.w);
+}
+
+// Shared-expert gate:  z += sgate * S.
+//   dsg[t] = <dZ_t, S_t>;  dS[t] = sgate_t * dZ_t;  dl[t] = dsg * sgate (1 - sgate)
+// One block per token.
+template <typename T>
+__global__ void shared_gate_bwd_kernel(const T* __restrict__ dZ, const T* __restrict__ S,
+                                       const float* __restrict__ sgate, int width, T* __restrict__ dS,
+                                       float* __restrict__ dl) {
+  __shared__ float red[32];
+  int t = blockIdx.x;
+  float sg = sgate[t];
+  float dot = 0.f;
+  for (int c = threadIdx.x * 8; c < width; c += blockDim.x * 8) {
+    Vec8<T> a, b;
+    float fa[8], fb[8];
+    a.load(dZ + (int64_t)t * width + c); a.get(fa);
+    b.load(S + (int64_t)t * width + c); b.get(fb);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { dot += fa[i] * fb[i]; fa[i] *= sg; }
+    a.set(fa);
+    a.store(dS + (int64_t)t * width + c);
+  }
+  dot = block_sum(dot, red);
+  if (threadIdx.x == 0) dl[t] = dot * sg * (1.f - sg);
+}
+
+// Gate backward (softmax over the selected logits):
+//   dg[t,s]  = sum_j dg_part[row(t,s), j]              (fixed order)
+//   dsel[t,s] = g[t,s] * (dg[t,s] - sum_s' g[t,s'] dg[t,s'])
+// written per (token, slot) and per padded row.
+__global__ void router_bwd_kernel(const float* __restrict__ dg_part, int dg_ld, int n_part,
+                                  const float* __restrict__ gate, const int32_t* __restrict__ tok_row,
+                                  int tokens, int k, float* __restrict__ tok_dl, float* __restrict__ row_dl) {
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= tokens) return;
+  float dg[8], g[8], mix = 0.f;
+  for (int s = 0; s < k; ++s) {
+    int row = tok_row[(int64_t)t * k + s];
+    float acc = 0.f;
+    for (int j = 0; j < n_part; ++j) acc += dg_part[(int64_t)row * dg_ld + j];
+    dg[s] = acc;
+    g[s] = gate[(int64_t)t * k + s];
+    mix += g[s] * acc;
+  }
+  for (int s = 0; s < k; ++s) {
+    float v = g[s] * (dg[s] - mix);
+    tok_dl[(int64_t)t * k + s] = v;
+    row_dl[tok_row[(int64_t)t * k + s]] = v;
+  }
+}
+
+// Router weight gradient from the permuted layout:
+//   dW_r[e, c] (+)= sum_{rows of e} row_dl[row] * Up[row, c];  db_r[e] (+)= sum row_dl[row]
+// grid (ceil(d / blockDim), E); each thread owns one column.
+template <typename T>
+__global__ void router_wgrad_kernel(const T* __restrict__ Up, const float* __restrict__ row_dl,
+                                    const int32_t* __restrict__ expert_off, const int32_t* __restrict__ expert_cnt,
+                                    int d, int accumulate, float* __restrict__ dWr, float* __restrict__ dbr) {
+  int e = blockIdx.y;
+  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  int r0 = expert_off[e], n = expert_cnt[e];
+  if (c < d && dWr) {
+    float acc = 0.f;
+    for (int r = r0; r < r0 + n; ++r) acc += row_dl[r] * to_f32(Up[(int64_t)r * d + c]);
+    float* o = dWr + (int64_t)e * d + c;
+    *o = (accumulate ? *o : 0.f) + acc;
+  }
+  if (c == 0 && dbr) {
+    float acc = 0.f;
+    for (int r = r0; r < r0 + n; ++r) acc += row_dl[r];
+    dbr[e] = (accumulate ? dbr[e] : 0.f) + acc;
+  }
+}
+
+// Column reduction with a per-row weight, two passes (deterministic):
+//   part[b, c] = sum_{t in strip b} w[t] * X[t, c]      (colsum_partial)
+//   out[c] (+)= sum_b part[b, c]                        (colsum_final)
+// Used for d w_sgate = sum_t dl[t] u_t.
+template <typename T>
+__global__ void colsum_partial_kernel(const T* __restrict__ X, int64_t ldx, const float* __restrict__ w,
+                                      int rows, int cols, int strip, float* __restrict__ part) {
+  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  int b = blockIdx.y;
+  if (c >= cols) return;
+  int t0 = b * strip, t1 = min(rows, t0 + strip);
+  float acc = 0.f;
+  for (int t = t0; t < t1; ++t) acc += w[t] * to_f32(X[(int64_t)t * ldx + c]);
+  part[(int64_t)b * cols + c] = acc;
+}
+
+__global__ void colsum_final_kernel(const float* __restrict__ part, int n_strips, int cols, int accumulate,
+                                    float* __restrict__ out) {
+  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols) return;
+  float acc = 0.f;
+  for (int b = 0; b < n_strips; ++b) acc += part[(int64_t)b * cols + c];
+  out[c] = (accumulate ? out[c] : 0.f) + acc;
+}
+
+// dU[t, :] = sum_s dUp[tok_row[t,s], :] + dUsh[t, :] + sum_s tok_dl[t,s] * W_r[idx[t,s], :]
+//            + dl[t] * w_sgate[:]
+// One block per token, fp32 sums in a fixed order.
+template <typename T>
+__global__ void du_reduce_kernel(const T* __restrict__ dUp, const int32_t* __restrict__ tok_row,
+                                 const int32_t* __restrict__ idx, const float* __restrict__ tok_dl, int k,
+                                 const T* __restrict__ dUsh, const T* __restrict__ w_router,
+                                 const float* __restrict__ dl, const T* __restrict__ w_sgate, int width,
+                                 T* __restrict__ dU) {
+  int t = blockIdx.x;
+  int rows[8], ex[8];
+  float dls[8];
+  for (int s = 0; s < k; ++s) {
+    rows[s] = tok_row[(int64_t)t * k + s];
+    ex[s] = idx[(int64_t)t * k + s];
+    dls[s] = tok_dl[(int64_t)t * k + s];
+  }
+  float dlt = dUsh ? dl[t] : 0.f;
+  for (int c = threadIdx.x * 8; c < width; c += blockDim.x * 8) {
+    float acc[8], f[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    Vec8<T> v;
+    for (int s = 0; s < k; ++s) {
+      v.load(dUp + (int64_t)rows[s] * width + c); v.get(f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] += f[i];
+    }
+    if (dUsh) {
+      v.load(dUsh + (int64_t)t * width + c); v.get(f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] += f[i];
+      v.load(w_sgate + c); v.get(f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] += dlt * f[i];
+    }
+    for (int s = 0; s < k; ++s) {
+      v.load(w_router + (int64_t)ex[s] * width + c); v.get(f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] += dls[s] * f[i];
+    }
+    v.set(acc);
+    v.store(dU + (int64_t)t * width + c);
+  }
+}
+
+// RMSNorm backward, rows:  q = gamma * dn;  dy = r q - y r^3 <q, y> / h;  dY1 += dy.
+// One warp per token.  norm NONE: dY1 += dn.
+__global__ void rmsnorm_bwd_rows_kernel(const float* __restrict__ dn, const float* __restrict__ y, int64_t ld,
+                                        const float* __restrict__ gamma, const float* __restrict__ r,
+                                        int norm_none, int tokens, int h, float* __restrict__ dy1, int64_t ld_dy) {
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  int lane = threadIdx.x & 31;
+  if (warp >= tokens) return;
+  const float* dn_row = dn + (int64_t)warp * h;
+  const float* y_row = y + (int64_t)warp * ld;
+  float* o = dy1 + (int64_t)warp * ld_dy;
+  if (norm_none) {
+    for (int i = lane; i < h; i += 32) o[i] += dn_row[i];
+    return;
+  }
+  float dot = 0.f;
+  for (int i = lane; i < h; i += 32) dot += (gamma ? gamma[i] : 1.f) * dn_row[i] * y_row[i];
+  dot = warp_sum(dot);
+  float rt = r[warp];
+  float coef = rt * rt * rt * dot / (float)h;
+  for (int i = lane; i < h; i += 32) {
+    float q = (gamma ? gamma[i] : 1.f) * dn_row[i];
+    o[i] += rt * q - y_row[i] * coef;
+  }
+}
+
+// dgamma partials: part[b, c] = sum_{t in strip b} dn[t, c] * y[t, c] * r[t]
+__global__ void dgamma_partial_kernel(const float* __restrict__ dn, const float* __restrict__ y, int64_t ld,
+                                      const float* __restrict__ r, int tokens, int h, int strip,
+                                      float* __restrict__ part) {
+  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  int b = blockIdx.y;
+  if (c >= h) return;
+  int t0 = b * strip, t1 = min(tokens, t0 + strip);
+  float acc = 0.f;
+  for (int t = t0; t < t1; ++t) acc += dn[(int64_t)t * h + c] * y[(int64_t)t * ld + c] * r[t];
+  part[(int64_t)b * h + c] = acc;
+}
+
+}  // namespace revffn

@@ -1,0 +1,244 @@
+// One description of every matrix product on the path, the per-element
+// epilogue arithmetic shared by both back ends, and the plain CUDA-core
+// back end (used for fp32 weights and as the on-device cross-check of the
+// tcgen05 back end).
+//
+//   C[m, n] = sum_k A(m, k) * B(n, k)
+//
+// Operand storage
+//   a_mn_major = 0: A is [M, K] row-major (K contiguous), lda = row stride
+//   a_mn_major = 1: A is [K, M] row-major (M contiguous), lda = row stride,
+//                   columns a_col0 .. a_col0+M-1 of that buffer
+//   b_mn_major likewise for B ([N, K] or [K, N], column offset b_col0).
+// B concatenation
+//   CONCAT_N: two products with the same A: acc0 against B0, acc1 against B1
+//             (gate and up projections of a SwiGLU pair)
+//   CONCAT_K: K = 2*Kh; k < Kh multiplies B0(n, k), k >= Kh multiplies B1(n, k-Kh)
+// Grouping
+//   GROUP_M: rows of A/C live in the padded expert-major row space; the 128-row
+//            tile i belongs to expert tile_group[i]; B/C1 are offset by
+//            expert * b_group_stride; rows >= *rows_total are not touched.
+//   GROUP_K: one product per expert e over the rows group_off[e]..group_off[e+1]
+//            as the K range (weight gradients); output offset e * c_group_stride.
+#pragma once
+
+#include "common.cuh"
+
+namespace revffn {
+
+enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_ROWSCALE = 2, EPI_COUPLE = 3, EPI_DSWIGLU = 4, EPI_WGRAD = 5 };
+enum { CONCAT_NONE = 0, CONCAT_N = 1, CONCAT_K = 2 };
+enum { GROUP_NONE = 0, GROUP_M = 1, GROUP_K = 2 };
+
+struct GemmProblem {
+  int M, N, K;
+  int a_mn_major, b_mn_major;
+  int concat;
+  int epilogue;
+  int out_f32;        // EPI_STORE: write fp32 instead of T
+  int accumulate;     // EPI_WGRAD: add to C
+  const void* A; const void* B0; const void* B1;
+  int64_t lda, ldb;
+  void* C; void* C1;  // C1: SWIGLU -> optional [M, 2N] pre-activations a|b; DSWIGLU -> optional g*H
+  int64_t ldc, ldc1;
+  const float* rowscale;                       // ROWSCALE / DSWIGLU (NULL = 1)
+  const float* resid; int64_t ld_resid; float resid_sign;   // COUPLE: C = resid + sign * acc (fp32)
+  void* ab; int64_t ld_ab;                     // DSWIGLU: [M, 2N] a|b in, da|db out (in place)
+  float* dg_part; int dg_ld;                   // DSWIGLU: per (row, n-tile) partial of <acc, H>
+  int group_mode, n_groups;
+  const int32_t* group_off; const int32_t* tile_group; const int32_t* rows_total;
+  int64_t b_group_stride, c_group_stride;
+  int a_col0, b_col0;
+  int* status;
+};
+
+// --------------------------------------------------------------------------
+// Epilogue arithmetic (fp32), shared by both back ends.
+// --------------------------------------------------------------------------
+__device__ __forceinline__ float swiglu_f(float a, float b) { return a * sigmoid_f(a) * b; }
+
+// SwiGLU backward for one element.  dh = dL/dH; returns H and writes da, db.
+__device__ __forceinline__ float dswiglu_f(float a, float b, float dh, float& da, float& db) {
+  float s = sigmoid_f(a);
+  float si = a * s;
+  da = dh * b * (s * (1.f + a * (1.f - s)));
+  db = dh * si;
+  return si * b;
+}
+
+// --------------------------------------------------------------------------
+// CUDA-core back end: 64x64 tile, 256 threads, 4x4 outputs per thread, BK = 16.
+// Element loads go through generic accessors, bounds-checked; slow but plain.
+// --------------------------------------------------------------------------
+constexpr int SIMT_BM = 64, SIMT_BN = 64, SIMT_BK = 16;
+
+template <typename T>
+__device__ __forceinline__ float simt_load_a(const GemmProblem& p, int m, int64_t k, int m_lim, int64_t k_lim) {
+  if (m >= m_lim || k >= k_lim) return 0.f;
+  const T* A = reinterpret_cast<const T*>(p.A);
+  return p.a_mn_major ? to_f32(A[k * p.lda + p.a_col0 + m]) : to_f32(A[(int64_t)m * p.lda + k]);
+}
+
+template <typename T>
+__device__ __forceinline__ float simt_load_b(const GemmProblem& p, const T* B, int n, int64_t k, int64_t k_lim) {
+  if (n >= p.N || k >= k_lim) return 0.f;
+  return p.b_mn_major ? to_f32(B[k * p.ldb + p.b_col0 + n]) : to_f32(B[(int64_t)n * p.ldb + k]);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmProblem p) {
+  __shared__ float As[SIMT_BK][SIMT_BM + 1];
+  __shared__ float Bs0[SIMT_BK][SIMT_BN + 1];
+  __shared__ float Bs1[SIMT_BK][SIMT_BN + 1];
+  __shared__ float red[SIMT_BM][17];
+
+  const int tid = threadIdx.x;
+  const int tx = tid & 15, ty = tid >> 4;
+  const int n0 = blockIdx.x * SIMT_BN;
+  int m0 = blockIdx.y * SIMT_BM;
+  int group = 0;
+  int m_lim = p.M;
+  int64_t k_begin = 0, k_end = p.K;
+  if (p.group_mode == GROUP_M) {
+    int total = *p.rows_total;
+    if (m0 >= total) return;
+    group = p.tile_group[m0 / ROW_PAD];
+    m_lim = total;
+  } else if (p.group_mode == GROUP_K) {
+    group = blockIdx.z;
+    k_begin = p.group_off[group];
+    k_end = p.group_off[group + 1];
+  }
+  const T* B0 = reinterpret_cast<const T*>(p.B0);
+  const T* B1 = reinterpret_cast<const T*>(p.B1);
+  if (p.group_mode == GROUP_M) {
+    B0 += (int64_t)group * p.b_group_stride;
+    if (B1) B1 += (int64_t)group * p.b_group_stride;
+  }
+  const int64_t k_half = (p.concat == CONCAT_K) ? (k_end / 2) : k_end;
+  const bool dual = (p.concat == CONCAT_N);
+
+  float acc0[4][4], acc1[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { acc0[i][j] = 0.f; acc1[i][j] = 0.f; }
+
+  for (int64_t k0 = k_begin; k0 < k_end; k0 += SIMT_BK) {
+    for (int i = tid; i < SIMT_BK * SIMT_BM; i += 256) {
+      int kk, mm;
+      if (p.a_mn_major) { kk = i / SIMT_BM; mm = i % SIMT_BM; } else { mm = i / SIMT_BK; kk = i % SIMT_BK; }
+      As[kk][mm] = simt_load_a<T>(p, m0 + mm, k0 + kk, m_lim, k_end);
+    }
+    for (int i = tid; i < SIMT_BK * SIMT_BN; i += 256) {
+      int kk, nn;
+      if (p.b_mn_major) { kk = i / SIMT_BN; nn = i % SIMT_BN; } else { nn = i / SIMT_BK; kk = i % SIMT_BK; }
+      int64_t k = k0 + kk;
+      float v0, v1 = 0.f;
+      if (p.concat == CONCAT_K) {
+        v0 = (k < k_half) ? simt_load_b<T>(p, B0, n0 + nn, k, k_half)
+                          : simt_load_b<T>(p, B1, n0 + nn, k - k_half, k_half);
+      } else {
+        v0 = simt_load_b<T>(p, B0, n0 + nn, k, k_end);
+        if (dual) v1 = simt_load_b<T>(p, B1, n0 + nn, k, k_end);
+      }
+      Bs0[kk][nn] = v0;
+      Bs1[kk][nn] = v1;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < SIMT_BK; ++kk) {
+      float a[4], b0[4], b1[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { b0[j] = Bs0[kk][tx * 4 + j]; b1[j] = Bs1[kk][tx * 4 + j]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc0[i][j] += a[i] * b0[j];
+          if (dual) acc1[i][j] += a[i] * b1[j];
+        }
+    }
+    __syncthreads();
+  }
+
+  // epilogue
+  float dg_local[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    int m = m0 + ty * 4 + i;
+    bool m_ok = m < m_lim;
+    float rs = (p.rowscale && m_ok) ? p.rowscale[m] : 1.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int n = n0 + tx * 4 + j;
+      if (!m_ok || n >= p.N) continue;
+      float v = acc0[i][j];
+      switch (p.epilogue) {
+        case EPI_STORE:
+          if (p.out_f32) reinterpret_cast<float*>(p.C)[(int64_t)m * p.ldc + n] = v;
+          else reinterpret_cast<T*>(p.C)[(int64_t)m * p.ldc + n] = from_f32<T>(v);
+          break;
+        case EPI_SWIGLU: {
+          float w = acc1[i][j];
+          reinterpret_cast<T*>(p.C)[(int64_t)m * p.ldc + n] = from_f32<T>(swiglu_f(v, w));
+          if (p.C1) {
+            T* ab = reinterpret_cast<T*>(p.C1) + (int64_t)m * p.ldc1;
+            ab[n] = from_f32<T>(v);
+            ab[p.N + n] = from_f32<T>(w);
+          }
+        } break;
+        case EPI_ROWSCALE:
+          reinterpret_cast<T*>(p.C)[(int64_t)m * p.ldc + n] = from_f32<T>(rs * v);
+          break;
+        case EPI_COUPLE:
+          reinterpret_cast<float*>(p.C)[(int64_t)m * p.ldc + n] =
+              p.resid[(int64_t)m * p.ld_resid + n] + p.resid_sign * v;
+          break;
+        case EPI_DSWIGLU: {
+          T* ab = reinterpret_cast<T*>(p.ab) + (int64_t)m * p.ld_ab;
+          float a = to_f32(ab[n]), b = to_f32(ab[p.N + n]);
+          float da, db;
+          float H = dswiglu_f(a, b, rs * v, da, db);
+          ab[n] = from_f32<T>(da);
+          ab[p.N + n] = from_f32<T>(db);
+          if (p.C1) reinterpret_cast<T*>(p.C1)[(int64_t)m * p.ldc1 + n] = from_f32<T>(rs * H);
+          dg_local[i] += v * H;
+        } break;
+        case EPI_WGRAD: {
+          float* o = reinterpret_cast<float*>(p.C) + (int64_t)group * p.c_group_stride + (int64_t)m * p.ldc + n;
+          *o = (p.accumulate ? *o : 0.f) + v;
+        } break;
+      }
+    }
+  }
+  if (p.epilogue == EPI_DSWIGLU && p.dg_part) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) red[ty * 4 + i][tx] = dg_local[i];
+    __syncthreads();
+    if (tid < SIMT_BM) {
+      int m = m0 + tid;
+      if (m < m_lim) {
+        float s = 0.f;
+        for (int j = 0; j < 16; ++j) s += red[tid][j];
+        p.dg_part[(int64_t)m * p.dg_ld + blockIdx.x] = s;
+      }
+    }
+  }
+}
+
+// Number of per-row dg partials the SIMT back end writes for N columns.
+inline int simt_dg_parts(int N) { return (int)ceil_div(N, SIMT_BN); }
+
+template <typename T>
+inline cudaError_t launch_gemm_simt(const GemmProblem& p, cudaStream_t stream) {
+  if (p.M <= 0 || p.N <= 0) return cudaSuccess;
+  dim3 grid((unsigned)ceil_div(p.N, SIMT_BN), (unsigned)ceil_div(p.M, SIMT_BM),
+            p.group_mode == GROUP_K ? (unsigned)p.n_groups : 1u);
+  gemm_simt_kernel<T><<<grid, 256, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace revffn

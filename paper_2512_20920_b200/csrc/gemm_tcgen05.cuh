@@ -1,0 +1,603 @@
+// tcgen05 / TMEM / TMA back end for every bf16 matrix product on the path.
+//
+// One persistent, warp-specialised kernel (1 CTA per SM, 192 threads):
+//   warp 0      TMA producer: cp.async.bulk.tensor 2D loads (128-byte swizzle) of
+//               A and B tiles into a ring of shared-memory stages, completion on
+//               mbarriers (no cluster multicast anywhere).
+//   warp 1      MMA issuer: owns the TMEM allocation (two accumulators, so the
+//               epilogue of tile i overlaps the main loop of tile i+1); one
+//               elected lane issues tcgen05.mma kind::f16 (bf16 x bf16 -> fp32),
+//               M = 128, N = 128 or 256, K = 16 per instruction; tcgen05.commit
+//               releases stages and publishes finished accumulators.
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (lane = tile row), apply the
+//               fused epilogue (SwiGLU, gate scale, coupling add/sub, SwiGLU
+//               backward, fp32 weight-gradient store) and write global memory.
+// Tile = 128 rows x MMA_N columns, K step 64 (one 128-byte swizzle atom of bf16).
+// Both operands may be K-major or MN-major; MN-major tiles are fetched as
+// 64x64 boxes and described to the tensor core with leading/stride offsets.
+// Every wait is bounded; on expiry the kernel sets the status word and leaves.
+#pragma once
+
+#include <cuda.h>
+#include <type_traits>
+
+#include "common.cuh"
+#include "gemm.cuh"
+
+namespace revffn {
+
+constexpr int TC_BM = 128;
+constexpr int TC_BK = 64;
+constexpr int TC_THREADS = 192;
+constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
+constexpr long long TC_WAIT_CYCLES = 4000000000LL;       // ~2 s: bound on any single wait
+
+template <int MMA_N> struct TcCfg {
+  static constexpr int B_BYTES = MMA_N * TC_BK * 2;
+  static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
+  static constexpr int STAGES = (MMA_N == 256) ? 4 : 6;
+  static constexpr int TMEM_COLS = 2 * MMA_N;           // 512 or 256: power of two >= 32
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+};
+
+struct TcParams {
+  GemmProblem p;
+  int tiles_m, tiles_n;      // GROUP_M: tiles_m is an upper bound, the device value comes from rows_total
+  int tile_n;                // logical output columns per tile
+  int k_blocks;              // dense / GROUP_M
+  uint32_t idesc;
+};
+
+// ---------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the wait was abandoned (this or another
+// role ran out of time); the caller then leaves its loop.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  long long t0 = clock64();
+  int spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (((++spins) & 63) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > TC_WAIT_CYCLES) {
+        *abort_flag = 1;
+        set_status(status, REVFFN_ERR_DEVICE_WAIT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+
+// 32 consecutive accumulator columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, tile base 1024-byte aligned.
+//   K-major : rows of 128 bytes, 8-row groups 1024 bytes apart (SBO); LBO unused (1)
+//   MN-major: 64-element chunks along M/N are lbo bytes apart, 8-k-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;      // descriptor version of this architecture
+  d |= 2ull << 61;      // 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  uint4 u;
+  __nv_bfloat162 h;
+  h = __floats2bfloat162_rn(f[0], f[1]); u.x = *reinterpret_cast<uint32_t*>(&h);
+  h = __floats2bfloat162_rn(f[2], f[3]); u.y = *reinterpret_cast<uint32_t*>(&h);
+  h = __floats2bfloat162_rn(f[4], f[5]); u.z = *reinterpret_cast<uint32_t*>(&h);
+  h = __floats2bfloat162_rn(f[6], f[7]); u.w = *reinterpret_cast<uint32_t*>(&h);
+  return u;
+}
+__device__ __forceinline__ void unpack8(uint4 u, float* f) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+}
+// store 32 floats as 32 bf16 (64 contiguous bytes)
+__device__ __forceinline__ void store32_bf16(bf16* dst, const float* f) {
+  uint4* o = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) o[i] = pack8(f + 8 * i);
+}
+__device__ __forceinline__ void load32_bf16(const bf16* src, float* f) {
+  const uint4* s = reinterpret_cast<const uint4*>(src);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) unpack8(s[i], f + 8 * i);
+}
+
+// Tile coordinates shared by the three roles.
+struct TcTile {
+  int m0, n0, group, k_blocks, krow0;
+  bool valid;
+};
+
+__device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_dev) {
+  TcTile t;
+  const GemmProblem& p = P.p;
+  int per_group = tiles_m_dev * P.tiles_n;
+  t.group = 0;
+  t.krow0 = 0;
+  t.k_blocks = P.k_blocks;
+  int total = (p.group_mode == GROUP_K) ? per_group * p.n_groups : per_group;
+  t.valid = w < total;
+  if (!t.valid) { t.m0 = t.n0 = 0; return t; }
+  int r = w;
+  if (p.group_mode == GROUP_K) {
+    t.group = w / per_group;
+    r = w - t.group * per_group;
+    int k0 = p.group_off[t.group], k1 = p.group_off[t.group + 1];
+    t.krow0 = k0;
+    t.k_blocks = (k1 - k0) / TC_BK;
+  }
+  int tm = r / P.tiles_n, tn = r - tm * P.tiles_n;
+  t.m0 = tm * TC_BM;
+  t.n0 = tn * P.tile_n;
+  if (p.group_mode == GROUP_M) t.group = p.tile_group[tm];
+  return t;
+}
+
+// ---------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------
+template <int MMA_N, int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUtensorMap map_a,
+               const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1) {
+  using Cfg = TcCfg<MMA_N>;
+  extern __shared__ uint8_t smem_raw[];
+  const GemmProblem& p = P.p;
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;                 // stage ring, 1024-byte aligned
+  uint8_t* gen_base = smem_raw + (base - raw);
+  const uint32_t bars = base + Cfg::STAGES * Cfg::STAGE_BYTES;  // barrier block
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (Cfg::STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + 2 + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + Cfg::STAGES * Cfg::STAGE_BYTES + 8 * (2 * Cfg::STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* issued = reinterpret_cast<int*>(tmem_slot + 2);   // [STAGES] parity+1 of the last load issued per stage
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); issued[s] = 0; }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  int tiles_m_dev = P.tiles_m;
+  if (p.group_mode == GROUP_M) tiles_m_dev = min(P.tiles_m, *p.rows_total / TC_BM);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; ok; w += gridDim.x) {
+        TcTile t = tc_tile(P, w, tiles_m_dev);
+        if (!t.valid) break;
+        const int k_half = t.k_blocks / 2;
+        for (int kb = 0; kb < t.k_blocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
+          const uint32_t sb = sa + TC_A_BYTES;
+          const uint32_t fb = full_bar(stage);
+          mbar_expect_tx(fb, Cfg::STAGE_BYTES);
+          issued[stage] = (int)phase + 1;
+          // A tile
+          if (!p.a_mn_major) {
+            tma_load_2d(sa, &map_a, kb * TC_BK, t.m0, fb);
+          } else {
+            int krow = t.krow0 + kb * TC_BK;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) tma_load_2d(sa + j * 8192, &map_a, p.a_col0 + t.m0 + 64 * j, krow, fb);
+          }
+          // B tile
+          const CUtensorMap* mb = &map_b0;
+          int kb_b = kb;
+          if (p.concat == CONCAT_K && kb >= k_half) { mb = &map_b1; kb_b = kb - k_half; }
+          if (!p.b_mn_major) {
+            // rows of the flattened [groups * N, K] weight tensor
+            int row0 = (p.group_mode == GROUP_M ? t.group * p.N : 0) + t.n0;
+            if (p.concat == CONCAT_N) {
+              tma_load_2d(sb, &map_b0, kb_b * TC_BK, row0, fb);
+              tma_load_2d(sb + 16384, &map_b1, kb_b * TC_BK, row0, fb);
+            } else {
+#pragma unroll
+              for (int j = 0; j < MMA_N / 128; ++j) tma_load_2d(sb + j * 16384, mb, kb_b * TC_BK, row0 + 128 * j, fb);
+            }
+          } else {
+            // rows of the flattened [groups * Kdim, N] weight tensor, or token rows (GROUP_K / dense wgrad)
+            int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
+            int krow = (p.group_mode == GROUP_M ? t.group * kdim : t.krow0) + kb_b * TC_BK;
+#pragma unroll
+            for (int j = 0; j < MMA_N / 64; ++j) tma_load_2d(sb + j * 8192, mb, p.b_col0 + t.n0 + 64 * j, krow, fb);
+          }
+          if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      int it = 0;
+      for (int w = blockIdx.x; ok; w += gridDim.x, ++it) {
+        TcTile t = tc_tile(P, w, tiles_m_dev);
+        if (!t.valid) break;
+        const int acc = it & 1;
+        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MMA_N);
+        for (int kb = 0; kb < t.k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
+          const uint32_t sb = sa + TC_A_BYTES;
+          const uint64_t a_desc = p.a_mn_major ? make_smem_desc(sa, 8192, 1024) : make_smem_desc(sa, 16, 1024);
+          const uint64_t b_desc = p.b_mn_major ? make_smem_desc(sb, 8192, 1024) : make_smem_desc(sb, 16, 1024);
+          const uint32_t a_step = p.a_mn_major ? (2048u >> 4) : (32u >> 4);   // 16 k-elements per instruction
+          const uint32_t b_step = p.b_mn_major ? (2048u >> 4) : (32u >> 4);
+#pragma unroll
+          for (int ks = 0; ks < TC_BK / 16; ++ks) {
+            tc_mma(d_tmem, a_desc + (uint64_t)(a_step * ks), b_desc + (uint64_t)(b_step * ks), P.idesc,
+                   (kb | ks) != 0 ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));          // stage reusable once these MMAs have read it
+          if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));              // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;                      // TMEM lane quadrant this warp may access
+    const int row_in_tile = q * 32 + lane;
+    bool ok = true;
+    int it = 0;
+    for (int w = blockIdx.x; ok; w += gridDim.x, ++it) {
+      TcTile t = tc_tile(P, w, tiles_m_dev);
+      if (!t.valid) break;
+      const int acc = it & 1;
+      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * MMA_N);
+      const int m = t.m0 + row_in_tile;
+      const int m_lim = (p.group_mode == GROUP_M) ? tiles_m_dev * TC_BM : p.M;
+      const bool m_ok = m < m_lim;
+      const bool have_acc = t.k_blocks > 0;      // an empty K range leaves the accumulator undefined: use zeros
+      uint32_t r0[32];
+      float f[32];
+
+      if constexpr (EPI == EPI_STORE || EPI == EPI_ROWSCALE || EPI == EPI_COUPLE || EPI == EPI_WGRAD) {
+        float rs = 1.f;
+        if (EPI == EPI_ROWSCALE && m_ok) rs = p.rowscale[m];
+#pragma unroll 1
+        for (int c = 0; c < MMA_N; c += 32) {
+          if (have_acc) { tmem_ld32(taddr + c, r0); tmem_ld_wait(); }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) f[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
+          const int n = t.n0 + c;
+          if (!m_ok || n >= p.N) continue;
+          if constexpr (EPI == EPI_STORE) {
+            if (p.out_f32) {
+              float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (int64_t)m * p.ldc + n);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) o[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+            } else {
+              store32_bf16(reinterpret_cast<bf16*>(p.C) + (int64_t)m * p.ldc + n, f);
+            }
+          } else if constexpr (EPI == EPI_ROWSCALE) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) f[i] *= rs;
+            store32_bf16(reinterpret_cast<bf16*>(p.C) + (int64_t)m * p.ldc + n, f);
+          } else if constexpr (EPI == EPI_COUPLE) {
+            const float4* x = reinterpret_cast<const float4*>(p.resid + (int64_t)m * p.ld_resid + n);
+            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (int64_t)m * p.ldc + n);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              float4 xv = x[i];
+              o[i] = make_float4(xv.x + p.resid_sign * f[4 * i], xv.y + p.resid_sign * f[4 * i + 1],
+                                 xv.z + p.resid_sign * f[4 * i + 2], xv.w + p.resid_sign * f[4 * i + 3]);
+            }
+          } else {   // EPI_WGRAD
+            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (int64_t)t.group * p.c_group_stride +
+                                                  (int64_t)m * p.ldc + n);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              float4 v = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+              if (p.accumulate) { float4 old = o[i]; v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w; }
+              o[i] = v;
+            }
+          }
+        }
+      } else if constexpr (EPI == EPI_SWIGLU) {
+        // columns [0, MMA_N/2) hold the gate projection, [MMA_N/2, MMA_N) the up projection
+        uint32_t r1[32];
+        float g[32];
+#pragma unroll 1
+        for (int c = 0; c < MMA_N / 2; c += 32) {
+          tmem_ld32(taddr + c, r0);
+          tmem_ld32(taddr + MMA_N / 2 + c, r1);
+          tmem_ld_wait();
+          const int n = t.n0 + c;
+          if (!m_ok || n >= p.N) continue;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            f[i] = __uint_as_float(r0[i]);
+            g[i] = __uint_as_float(r1[i]);
+          }
+          if (p.C1) {
+            bf16* ab = reinterpret_cast<bf16*>(p.C1) + (int64_t)m * p.ldc1;
+            store32_bf16(ab + n, f);
+            store32_bf16(ab + p.N + n, g);
+          }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) f[i] = swiglu_f(f[i], g[i]);
+          store32_bf16(reinterpret_cast<bf16*>(p.C) + (int64_t)m * p.ldc + n, f);
+        }
+      } else {   // EPI_DSWIGLU
+        float rs = (p.rowscale && m_ok) ? p.rowscale[m] : 1.f;
+        float dg = 0.f;
+        float a[32], b[32];
+#pragma unroll 1
+        for (int c = 0; c < MMA_N; c += 32) {
+          tmem_ld32(taddr + c, r0);
+          tmem_ld_wait();
+          const int n = t.n0 + c;
+          if (!m_ok || n >= p.N) continue;
+          bf16* ab = reinterpret_cast<bf16*>(p.ab) + (int64_t)m * p.ld_ab;
+          load32_bf16(ab + n, a);
+          load32_bf16(ab + p.N + n, b);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            float v = __uint_as_float(r0[i]);
+            float da, db;
+            float H = dswiglu_f(a[i], b[i], rs * v, da, db);
+            dg += v * H;
+            a[i] = da; b[i] = db; f[i] = rs * H;
+          }
+          store32_bf16(ab + n, a);
+          store32_bf16(ab + p.N + n, b);
+          if (p.C1) store32_bf16(reinterpret_cast<bf16*>(p.C1) + (int64_t)m * p.ldc1 + n, f);
+        }
+        if (p.dg_part && m_ok) p.dg_part[(int64_t)m * p.dg_ld + t.n0 / P.tile_n] = dg;
+      }
+      // accumulator may be overwritten by the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) {
+    // loads already issued into this CTA's shared memory must land before the CTA exits
+    for (int s = 0; s < Cfg::STAGES; ++s) {
+      if (issued[s] == 0) continue;
+      long long t0 = clock64();
+      while (!mbar_try_wait(full_bar(s), (uint32_t)(issued[s] - 1)) && clock64() - t0 < TC_WAIT_CYCLES) {}
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
+                 : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcState {
+  EncodeTiledFn encode = nullptr;
+  int n_sms = 0;
+  bool ready = false;
+};
+inline TcState& tc_state() { static TcState s; return s; }
+
+template <int MMA_N, int EPI>
+inline cudaError_t tc_set_attr() {
+  return cudaFuncSetAttribute(gemm_tc_kernel<MMA_N, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TcCfg<MMA_N>::SMEM_BYTES);
+}
+
+// Once per process: driver entry point for tensor-map encoding, SM count, shared-memory opt-in.
+inline int tc_prepare() {
+  TcState& s = tc_state();
+  if (s.ready) return REVFFN_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
+    return REVFFN_ERR_CUDA;
+  s.encode = reinterpret_cast<EncodeTiledFn>(fn);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return REVFFN_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&s.n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return REVFFN_ERR_CUDA;
+  cudaError_t e = cudaSuccess;
+  if (e == cudaSuccess) e = tc_set_attr<256, EPI_STORE>();
+  if (e == cudaSuccess) e = tc_set_attr<128, EPI_STORE>();
+  if (e == cudaSuccess) e = tc_set_attr<256, EPI_SWIGLU>();
+  if (e == cudaSuccess) e = tc_set_attr<256, EPI_ROWSCALE>();
+  if (e == cudaSuccess) e = tc_set_attr<128, EPI_ROWSCALE>();
+  if (e == cudaSuccess) e = tc_set_attr<256, EPI_COUPLE>();
+  if (e == cudaSuccess) e = tc_set_attr<128, EPI_COUPLE>();
+  if (e == cudaSuccess) e = tc_set_attr<128, EPI_DSWIGLU>();
+  if (e == cudaSuccess) e = tc_set_attr<256, EPI_WGRAD>();
+  if (e == cudaSuccess) e = tc_set_attr<128, EPI_WGRAD>();
+  if (e != cudaSuccess) return REVFFN_ERR_CUDA;
+  s.ready = true;
+  return REVFFN_OK;
+}
+
+// 2D bf16 tensor map: `inner` contiguous elements per row, `outer` rows of stride ld elements.
+inline int tc_make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer, uint64_t ld,
+                       uint32_t box_inner, uint32_t box_outer) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = tc_state().encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
+                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? REVFFN_OK : REVFFN_ERR_CUDA;
+}
+
+inline int tc_pick_n(const GemmProblem& p) {
+  if (p.epilogue == EPI_SWIGLU) return 256;          // 128 gate + 128 up columns
+  if (p.epilogue == EPI_DSWIGLU) return 128;
+  return (p.N % 256 == 0) ? 256 : 128;
+}
+inline int tc_dg_parts(int N) { return (int)ceil_div(N, 128); }
+
+template <int MMA_N, int EPI>
+inline int tc_launch(const TcParams& P, const CUtensorMap& ma, const CUtensorMap& mb0, const CUtensorMap& mb1,
+                     int grid, cudaStream_t st) {
+  gemm_tc_kernel<MMA_N, EPI><<<grid, TC_THREADS, TcCfg<MMA_N>::SMEM_BYTES, st>>>(P, ma, mb0, mb1);
+  return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
+}
+
+inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
+  TcState& s = tc_state();
+  if (!s.ready) return REVFFN_ERR_CUDA;
+  if (p.M <= 0 || p.N <= 0) return REVFFN_OK;
+  const int mma_n = tc_pick_n(p);
+  TcParams P;
+  P.p = p;
+  P.tile_n = (p.concat == CONCAT_N) ? mma_n / 2 : mma_n;
+  P.tiles_m = (int)ceil_div(p.M, TC_BM);
+  P.tiles_n = (int)ceil_div(p.N, P.tile_n);
+  P.k_blocks = (int)ceil_div(p.K, TC_BK);
+  if (p.N % 128 != 0) return REVFFN_ERR_SHAPE;
+  if (p.group_mode != GROUP_K && p.K % TC_BK != 0 && !(p.a_mn_major && p.b_mn_major)) return REVFFN_ERR_SHAPE;
+  if (p.concat == CONCAT_K && (P.k_blocks & 1)) return REVFFN_ERR_SHAPE;
+  P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.a_mn_major ? 1 : 0) << 15) |
+            ((uint32_t)(p.b_mn_major ? 1 : 0) << 16) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+
+  const int groups = p.n_groups > 0 ? p.n_groups : 1;
+  CUtensorMap ma, mb0, mb1;
+  // A
+  if (!p.a_mn_major) {
+    // [rows, K]: dense M rows, or the padded row space for GROUP_M
+    int r = tc_make_map(&ma, p.A, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.lda, 64, 128);
+    if (r) return r;
+  } else {
+    // [K rows, lda columns]; K rows = tokens (dense) or the bound on padded rows (GROUP_K)
+    int r = tc_make_map(&ma, p.A, (uint64_t)p.lda, (uint64_t)p.K, (uint64_t)p.lda, 64, 64);
+    if (r) return r;
+  }
+  // B
+  const int k_half = (p.concat == CONCAT_K) ? p.K / 2 : p.K;
+  if (!p.b_mn_major) {
+    uint64_t rows = (p.group_mode == GROUP_M) ? (uint64_t)groups * p.N : (uint64_t)p.N;
+    int r = tc_make_map(&mb0, p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, 64, 128);
+    if (r) return r;
+    r = tc_make_map(&mb1, p.B1 ? p.B1 : p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, 64, 128);
+    if (r) return r;
+  } else {
+    uint64_t rows = (p.group_mode == GROUP_M) ? (uint64_t)groups * k_half : (uint64_t)p.K;
+    int r = tc_make_map(&mb0, p.B0, (uint64_t)p.ldb, rows, (uint64_t)p.ldb, 64, 64);
+    if (r) return r;
+    r = tc_make_map(&mb1, p.B1 ? p.B1 : p.B0, (uint64_t)p.ldb, rows, (uint64_t)p.ldb, 64, 64);
+    if (r) return r;
+  }
+  int64_t total = (int64_t)P.tiles_m * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
+  int grid = (int)(total < s.n_sms ? total : s.n_sms);
+  if (grid <= 0) return REVFFN_OK;
+
+#define TC_CASE(N_, E_) \
+  if (mma_n == N_ && p.epilogue == E_) return tc_launch<N_, E_>(P, ma, mb0, mb1, grid, st);
+  TC_CASE(256, EPI_STORE) TC_CASE(128, EPI_STORE)
+  TC_CASE(256, EPI_SWIGLU)
+  TC_CASE(256, EPI_ROWSCALE) TC_CASE(128, EPI_ROWSCALE)
+  TC_CASE(256, EPI_COUPLE) TC_CASE(128, EPI_COUPLE)
+  TC_CASE(128, EPI_DSWIGLU)
+  TC_CASE(256, EPI_WGRAD) TC_CASE(128, EPI_WGRAD)
+#undef TC_CASE
+  return REVFFN_ERR_UNSUPPORTED;
+}
+
+}  // namespace revffn

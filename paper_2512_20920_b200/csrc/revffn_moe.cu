@@ -1,0 +1,626 @@
+// C ABI, workspace planner and launch sequences of the RevFFN MoE coupling branch.
+// See include/revffn_moe.h for the contract of every entry point.
+
+#include <cstdio>
+#include <cstring>
+#include <type_traits>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "routing.cuh"
+#include "backward_ew.cuh"
+#include "gemm.cuh"
+#include "gemm_tcgen05.cuh"
+
+namespace revffn {
+
+// ---------------------------------------------------------------------------
+// Workspace layout
+// ---------------------------------------------------------------------------
+struct Buf { size_t off = 0, bytes = 0; };
+
+struct WsLayout {
+  // forward / inverse
+  Buf status, rows_total, w_rc, n, r, idx, gates, sgate, local_rank, chunk_cnt, chunk_base, expert_cnt,
+      expert_off, tile_group, tok_row, row_tok, row_gate, u, up, hmid, o, hs, s, z;
+  size_t fwd_bytes = 0;
+  // backward only
+  Buf ab, abs, gb, dz, ds, dl, dop, dg_part, tok_dl, row_dl, dup, dush, du, dn, part;
+  size_t bwd_bytes = 0;
+  int64_t rows_pad = 0;   // upper bound on padded rows
+  int n_chunks = 0, max_tiles = 0, dg_ld = 0, strips = 0;
+};
+
+constexpr int STRIP = 256;   // tokens per strip in two-pass column reductions
+
+static WsLayout plan_workspace(const revffn_moe_desc& D) {
+  WsLayout L;
+  const size_t ts = D.weight_dtype == REVFFN_BF16 ? 2 : 4;
+  const int64_t T = D.tokens, d = D.d_model, h = d / 2, E = D.n_experts, k = D.top_k, I = D.d_expert,
+                Is = D.d_shared;
+  L.rows_pad = max_padded_rows(T, (int)k, (int)E);
+  L.n_chunks = (int)ceil_div(T > 0 ? T : 1, MAP_CHUNK);
+  L.max_tiles = (int)(L.rows_pad / ROW_PAD);
+  L.dg_ld = (int)ceil_div(I, SIMT_BN);
+  L.strips = (int)ceil_div(T > 0 ? T : 1, STRIP);
+  const int64_t Rp = L.rows_pad;
+  size_t off = 0;
+  auto take = [&](Buf& b, size_t bytes) {
+    b.off = off; b.bytes = bytes;
+    off += (size_t)round_up((int64_t)(bytes > 0 ? bytes : 1), 256);
+  };
+  take(L.status, 256);
+  take(L.rows_total, 256);
+  take(L.w_rc, (size_t)(E + 1) * h * 8);
+  take(L.n, (size_t)T * h * ts);
+  take(L.r, (size_t)T * 4);
+  take(L.idx, (size_t)T * k * 4);
+  take(L.gates, (size_t)T * k * 4);
+  take(L.sgate, (size_t)T * 4);
+  take(L.local_rank, (size_t)T * k * 4);
+  take(L.chunk_cnt, (size_t)L.n_chunks * E * 4);
+  take(L.chunk_base, (size_t)L.n_chunks * E * 4);
+  take(L.expert_cnt, (size_t)E * 4);
+  take(L.expert_off, (size_t)(E + 1) * 4);
+  take(L.tile_group, (size_t)L.max_tiles * 4);
+  take(L.tok_row, (size_t)T * k * 4);
+  take(L.row_tok, (size_t)Rp * 4);
+  take(L.row_gate, (size_t)Rp * 4);
+  take(L.u, (size_t)T * d * ts);
+  take(L.up, (size_t)Rp * d * ts);
+  take(L.hmid, (size_t)Rp * I * ts);
+  take(L.o, (size_t)Rp * d * ts);
+  take(L.hs, (size_t)T * Is * ts);
+  take(L.s, (size_t)T * d * ts);
+  take(L.z, (size_t)T * d * ts);
+  L.fwd_bytes = off;
+  take(L.ab, (size_t)Rp * 2 * I * ts);
+  take(L.abs, (size_t)T * 2 * Is * ts);
+  take(L.gb, (size_t)T * h * ts);
+  take(L.dz, (size_t)T * d * ts);
+  take(L.ds, (size_t)T * d * ts);
+  take(L.dl, (size_t)T * 4);
+  take(L.dop, (size_t)Rp * d * ts);
+  take(L.dg_part, (size_t)Rp * L.dg_ld * 4);
+  take(L.tok_dl, (size_t)T * k * 4);
+  take(L.row_dl, (size_t)Rp * 4);
+  take(L.dup, (size_t)Rp * d * ts);
+  take(L.dush, (size_t)T * d * ts);
+  take(L.du, (size_t)T * d * ts);
+  take(L.dn, (size_t)T * h * 4);
+  take(L.part, (size_t)L.strips * d * 4);
+  L.bwd_bytes = off;
+  return L;
+}
+
+static int validate_desc(const revffn_moe_desc* D) {
+  if (!D) return REVFFN_ERR_NULL;
+  if (D->tokens < 0 || D->d_model <= 0 || (D->d_model & 1)) return REVFFN_ERR_SHAPE;
+  if (D->top_k < 1 || D->top_k > 8 || D->n_experts < D->top_k || D->n_experts > 256) return REVFFN_ERR_SHAPE;
+  if (D->d_expert <= 0 || D->d_shared < 0) return REVFFN_ERR_SHAPE;
+  if (D->weight_dtype != REVFFN_F32 && D->weight_dtype != REVFFN_BF16) return REVFFN_ERR_SHAPE;
+  if (D->norm_kind != REVFFN_NORM_RMS && D->norm_kind != REVFFN_NORM_NONE) return REVFFN_ERR_SHAPE;
+  const int h = D->d_model / 2;
+  const int mult = D->weight_dtype == REVFFN_BF16 ? 128 : 8;
+  if (h % mult || D->d_model % mult || D->d_expert % mult || D->d_shared % mult) return REVFFN_ERR_SHAPE;
+  if (D->ld_stream < h || (D->ld_stream % 4)) return REVFFN_ERR_ALIGN;
+  if ((int64_t)D->tokens * D->top_k > (int64_t)1 << 28) return REVFFN_ERR_SHAPE;
+  return REVFFN_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int validate_weights(const revffn_moe_desc& D, const revffn_moe_weights* w) {
+  if (!w) return REVFFN_ERR_NULL;
+  if (!w->w_up || !w->w_down || !w->w_router || !w->w_gate || !w->w_upx || !w->w_downx) return REVFFN_ERR_NULL;
+  if (D.d_shared > 0 && (!w->ws_gate || !w->ws_up || !w->ws_down || !w->ws_sgate)) return REVFFN_ERR_NULL;
+  const void* ps[] = {w->norm_gamma, w->w_up, w->w_down, w->w_router, w->b_router, w->w_gate, w->w_upx,
+                      w->w_downx, w->ws_gate, w->ws_up, w->ws_down, w->ws_sgate};
+  for (const void* p : ps)
+    if (p && !aligned16(p)) return REVFFN_ERR_ALIGN;
+  return REVFFN_OK;
+}
+
+static int check_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return REVFFN_ERR_CUDA;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return REVFFN_ERR_CUDA;
+  return major == 10 ? REVFFN_OK : REVFFN_ERR_ARCH;
+}
+
+#define CK(expr)                                   \
+  do {                                             \
+    cudaError_t e_ = (expr);                       \
+    if (e_ != cudaSuccess) return REVFFN_ERR_CUDA; \
+  } while (0)
+#define CKR(expr)                  \
+  do {                             \
+    int r_ = (expr);               \
+    if (r_ != REVFFN_OK) return r_; \
+  } while (0)
+
+// ---------------------------------------------------------------------------
+// Launch context
+// ---------------------------------------------------------------------------
+template <typename T>
+struct Ctx {
+  revffn_moe_desc D;
+  revffn_moe_weights W;
+  WsLayout L;
+  char* ws;
+  cudaStream_t st;
+  bool tc;   // tcgen05 back end for the matrix products
+  template <typename U> U* p(const Buf& b) const { return reinterpret_cast<U*>(ws + b.off); }
+  int T_() const { return D.tokens; }
+};
+
+template <typename T>
+static int run_gemm(const Ctx<T>& c, GemmProblem p) {
+  p.status = c.template p<int>(c.L.status);
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (c.tc) return launch_gemm_tc(p, c.st);
+  }
+  return launch_gemm_simt<T>(p, c.st) == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
+}
+
+template <typename T>
+static int dg_parts(const Ctx<T>& c, int N) {
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (c.tc) return tc_dg_parts(N);
+  }
+  return simt_dg_parts(N);
+}
+
+static GemmProblem blank_problem() {
+  GemmProblem p;
+  memset(&p, 0, sizeof(p));
+  p.resid_sign = 1.f;
+  return p;
+}
+
+// ---------------------------------------------------------------------------
+// F = MLP(Norm(Y1)) up to z (the input of P_down).  save_ab keeps the SwiGLU
+// pre-activations for the backward pass.
+// ---------------------------------------------------------------------------
+template <typename T>
+static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, int32_t* idx_user, bool save_ab) {
+  const revffn_moe_desc& D = c.D;
+  const WsLayout& L = c.L;
+  const int Tn = D.tokens, d = D.d_model, h = d / 2, E = D.n_experts, k = D.top_k, I = D.d_expert, Is = D.d_shared;
+  const int norm_none = D.norm_kind == REVFFN_NORM_NONE;
+  cudaStream_t st = c.st;
+  const T* w_up = reinterpret_cast<const T*>(c.W.w_up);
+
+  // Norm
+  rmsnorm_fwd_kernel<T><<<(unsigned)ceil_div((int64_t)Tn * 32, 128), 128, 0, st>>>(
+      y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, Tn, h, c.template p<T>(L.n), c.template p<float>(L.r));
+  CK(cudaGetLastError());
+
+  // Router: fold through P_up, logits, top-k, gates
+  {
+    dim3 grid((unsigned)ceil_div(h, 128), (unsigned)(E + 1));
+    fold_router_kernel<T><<<grid, 128, 0, st>>>(reinterpret_cast<const T*>(c.W.w_router),
+                                                 reinterpret_cast<const T*>(c.W.ws_sgate), w_up, E, d, h,
+                                                 c.template p<double>(L.w_rc));
+    CK(cudaGetLastError());
+    size_t smem = router_smem_bytes(E);
+    router_topk_kernel<<<(unsigned)ceil_div(Tn, RT_TOK), 256, smem, st>>>(
+        y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, c.template p<double>(L.w_rc), c.W.b_router, Tn, h,
+        E, k, Is > 0 ? 1 : 0, idx_in, c.template p<int32_t>(L.idx), c.template p<float>(L.gates),
+        c.template p<float>(L.sgate), idx_user);
+    CK(cudaGetLastError());
+  }
+
+  // Permutation maps
+  CK(cudaMemsetAsync(c.ws + L.row_tok.off, 0xFF, L.row_tok.bytes, st));
+  CK(cudaMemsetAsync(c.ws + L.row_gate.off, 0, L.row_gate.bytes, st));
+  map_rank_kernel<<<L.n_chunks, 256, (size_t)MAP_CHUNK * k * 4, st>>>(
+      c.template p<int32_t>(L.idx), Tn, k, E, c.template p<int32_t>(L.local_rank), c.template p<int32_t>(L.chunk_cnt));
+  CK(cudaGetLastError());
+  map_scan_kernel<<<1, 256, (size_t)(E + 1) * 4, st>>>(
+      c.template p<int32_t>(L.chunk_cnt), L.n_chunks, E, c.template p<int32_t>(L.chunk_base),
+      c.template p<int32_t>(L.expert_cnt), c.template p<int32_t>(L.expert_off), c.template p<int32_t>(L.tile_group),
+      c.template p<int32_t>(L.rows_total), L.max_tiles);
+  CK(cudaGetLastError());
+  map_assign_kernel<<<(unsigned)ceil_div((int64_t)Tn * k, 256), 256, 0, st>>>(
+      c.template p<int32_t>(L.idx), c.template p<float>(L.gates), c.template p<int32_t>(L.local_rank),
+      c.template p<int32_t>(L.chunk_base), c.template p<int32_t>(L.expert_off), Tn, k, E,
+      c.template p<int32_t>(L.tok_row), c.template p<int32_t>(L.row_tok), c.template p<float>(L.row_gate));
+  CK(cudaGetLastError());
+
+  // P_up: U = N W_up^T
+  {
+    GemmProblem p = blank_problem();
+    p.M = Tn; p.N = d; p.K = h;
+    p.A = c.template p<T>(L.n); p.lda = h;
+    p.B0 = w_up; p.ldb = h;
+    p.epilogue = EPI_STORE; p.C = c.template p<T>(L.u); p.ldc = d;
+    CKR(run_gemm(c, p));
+  }
+
+  // Permute: Up[row] = U[token(row)]
+  gather_rows_kernel<T><<<(unsigned)L.rows_pad, 256, 0, st>>>(c.template p<T>(L.u), d, c.template p<int32_t>(L.row_tok),
+                                                              c.template p<int32_t>(L.rows_total), d,
+                                                              c.template p<T>(L.up));
+  CK(cudaGetLastError());
+
+  // Routed experts: H = silu(Up Wg^T) * (Up Wu^T);  O = g * (H Wd^T)
+  {
+    GemmProblem p = blank_problem();
+    p.M = (int)L.rows_pad; p.N = I; p.K = d;
+    p.A = c.template p<T>(L.up); p.lda = d;
+    p.B0 = c.W.w_gate; p.B1 = c.W.w_upx; p.ldb = d; p.concat = CONCAT_N;
+    p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)I * d;
+    p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
+    p.rows_total = c.template p<int32_t>(L.rows_total);
+    p.epilogue = EPI_SWIGLU; p.C = c.template p<T>(L.hmid); p.ldc = I;
+    if (save_ab) { p.C1 = c.template p<T>(L.ab); p.ldc1 = 2 * (int64_t)I; }
+    CKR(run_gemm(c, p));
+  }
+  {
+    GemmProblem p = blank_problem();
+    p.M = (int)L.rows_pad; p.N = d; p.K = I;
+    p.A = c.template p<T>(L.hmid); p.lda = I;
+    p.B0 = c.W.w_downx; p.ldb = I;
+    p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)d * I;
+    p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
+    p.rows_total = c.template p<int32_t>(L.rows_total);
+    p.epilogue = EPI_ROWSCALE; p.rowscale = c.template p<float>(L.row_gate);
+    p.C = c.template p<T>(L.o); p.ldc = d;
+    CKR(run_gemm(c, p));
+  }
+
+  // Shared expert: S = (silu(U Wsg^T) * (U Wsu^T)) Wsd^T
+  if (Is > 0) {
+    GemmProblem p = blank_problem();
+    p.M = Tn; p.N = Is; p.K = d;
+    p.A = c.template p<T>(L.u); p.lda = d;
+    p.B0 = c.W.ws_gate; p.B1 = c.W.ws_up; p.ldb = d; p.concat = CONCAT_N;
+    p.epilogue = EPI_SWIGLU; p.C = c.template p<T>(L.hs); p.ldc = Is;
+    if (save_ab) { p.C1 = c.template p<T>(L.abs); p.ldc1 = 2 * (int64_t)Is; }
+    CKR(run_gemm(c, p));
+    GemmProblem q = blank_problem();
+    q.M = Tn; q.N = d; q.K = Is;
+    q.A = c.template p<T>(L.hs); q.lda = Is;
+    q.B0 = c.W.ws_down; q.ldb = Is;
+    q.epilogue = EPI_STORE; q.C = c.template p<T>(L.s); q.ldc = d;
+    CKR(run_gemm(c, q));
+  }
+
+  // Combine: Z[t] = sum_s O[row(t,s)] + sgate_t S[t]
+  if (Tn > 0) {
+    combine_rows_kernel<T><<<Tn, 256, 0, st>>>(c.template p<T>(L.o), c.template p<int32_t>(L.tok_row), k,
+                                               Is > 0 ? c.template p<T>(L.s) : nullptr, c.template p<float>(L.sgate),
+                                               d, c.template p<T>(L.z));
+    CK(cudaGetLastError());
+  }
+  return REVFFN_OK;
+}
+
+// P_down fused with the coupling: out = resid + sign * (Z W_down^T)
+template <typename T>
+static int run_couple(const Ctx<T>& c, const float* resid, float sign, float* out) {
+  const int d = c.D.d_model, h = d / 2;
+  GemmProblem p = blank_problem();
+  p.M = c.D.tokens; p.N = h; p.K = d;
+  p.A = c.template p<T>(c.L.z); p.lda = d;
+  p.B0 = c.W.w_down; p.ldb = d;
+  p.epilogue = EPI_COUPLE; p.resid = resid; p.ld_resid = c.D.ld_stream; p.resid_sign = sign;
+  p.C = out; p.ldc = c.D.ld_stream;
+  return run_gemm(c, p);
+}
+
+template <typename T>
+static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, float* dy1, const revffn_moe_grads& G,
+                        const int32_t* idx_in) {
+  const revffn_moe_desc& D = c.D;
+  const WsLayout& L = c.L;
+  const int Tn = D.tokens, d = D.d_model, h = d / 2, E = D.n_experts, k = D.top_k, I = D.d_expert, Is = D.d_shared;
+  const int norm_none = D.norm_kind == REVFFN_NORM_NONE;
+  const int acc = G.accumulate ? 1 : 0;
+  cudaStream_t st = c.st;
+  const int Rp = (int)L.rows_pad;
+
+  CKR(run_branch(c, y1, idx_in, nullptr, true));
+
+  auto wgrad = [&](float* out, int M, int N, const void* A, int64_t lda, int a_col0, const void* B, int64_t ldb,
+                   bool grouped, int64_t cstride) -> int {
+    GemmProblem p = blank_problem();
+    p.M = M; p.N = N; p.K = grouped ? Rp : Tn;   // grouped: bound on rows, the range comes from group_off
+    p.a_mn_major = 1; p.b_mn_major = 1;
+    p.A = A; p.lda = lda; p.a_col0 = a_col0;
+    p.B0 = B; p.ldb = ldb;
+    p.epilogue = EPI_WGRAD; p.accumulate = acc;
+    p.C = out; p.ldc = N; p.c_group_stride = cstride;
+    if (grouped) {
+      p.group_mode = GROUP_K; p.n_groups = E;
+      p.group_off = c.template p<int32_t>(L.expert_off);
+    }
+    return run_gemm(c, p);
+  };
+
+  // P_down backward: dZ = G W_down;  dW_down = G^T Z
+  cast_stream_kernel<T><<<(unsigned)ceil_div((int64_t)Tn * h, 4 * 256), 256, 0, st>>>(dy2, D.ld_stream, Tn, h,
+                                                                                      c.template p<T>(L.gb));
+  CK(cudaGetLastError());
+  {
+    GemmProblem p = blank_problem();
+    p.M = Tn; p.N = d; p.K = h;
+    p.A = c.template p<T>(L.gb); p.lda = h;
+    p.B0 = c.W.w_down; p.ldb = d; p.b_mn_major = 1;
+    p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dz); p.ldc = d;
+    CKR(run_gemm(c, p));
+  }
+  if (G.w_down) CKR(wgrad(G.w_down, h, d, c.template p<T>(L.gb), h, 0, c.template p<T>(L.z), d, false, 0));
+
+  // Shared expert backward
+  if (Is > 0) {
+    shared_gate_bwd_kernel<T><<<Tn, 256, 0, st>>>(c.template p<T>(L.dz), c.template p<T>(L.s),
+                                                  c.template p<float>(L.sgate), d, c.template p<T>(L.ds),
+                                                  c.template p<float>(L.dl));
+    CK(cudaGetLastError());
+    {
+      GemmProblem p = blank_problem();   // dH_s = dS Ws_d, then SwiGLU backward in place on a|b
+      p.M = Tn; p.N = Is; p.K = d;
+      p.A = c.template p<T>(L.ds); p.lda = d;
+      p.B0 = c.W.ws_down; p.ldb = Is; p.b_mn_major = 1;
+      p.epilogue = EPI_DSWIGLU; p.ab = c.template p<T>(L.abs); p.ld_ab = 2 * (int64_t)Is;
+      CKR(run_gemm(c, p));
+    }
+    if (G.ws_down) CKR(wgrad(G.ws_down, d, Is, c.template p<T>(L.ds), d, 0, c.template p<T>(L.hs), Is, false, 0));
+    {
+      GemmProblem p = blank_problem();   // dU_sh = da Ws_g + db Ws_u
+      p.M = Tn; p.N = d; p.K = 2 * Is;
+      p.A = c.template p<T>(L.abs); p.lda = 2 * (int64_t)Is;
+      p.B0 = c.W.ws_gate; p.B1 = c.W.ws_up; p.ldb = d; p.b_mn_major = 1; p.concat = CONCAT_K;
+      p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dush); p.ldc = d;
+      CKR(run_gemm(c, p));
+    }
+    if (G.ws_gate) CKR(wgrad(G.ws_gate, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, 0, c.template p<T>(L.u), d, false, 0));
+    if (G.ws_up) CKR(wgrad(G.ws_up, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, Is, c.template p<T>(L.u), d, false, 0));
+    if (G.ws_sgate) {
+      dim3 grid((unsigned)ceil_div(d, 256), (unsigned)L.strips);
+      colsum_partial_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.u), d, c.template p<float>(L.dl), Tn, d, STRIP,
+                                                     c.template p<float>(L.part));
+      CK(cudaGetLastError());
+      colsum_final_kernel<<<(unsigned)ceil_div(d, 256), 256, 0, st>>>(c.template p<float>(L.part), L.strips, d, acc,
+                                                                      G.ws_sgate);
+      CK(cudaGetLastError());
+    }
+  }
+
+  // Routed experts backward
+  gather_rows_kernel<T><<<(unsigned)Rp, 256, 0, st>>>(c.template p<T>(L.dz), d, c.template p<int32_t>(L.row_tok),
+                                                      c.template p<int32_t>(L.rows_total), d, c.template p<T>(L.dop));
+  CK(cudaGetLastError());
+  const int n_part = dg_parts(c, I);
+  {
+    GemmProblem p = blank_problem();   // dH' = dO Wd; SwiGLU backward; dg partials; hmid <- g * H
+    p.M = Rp; p.N = I; p.K = d;
+    p.A = c.template p<T>(L.dop); p.lda = d;
+    p.B0 = c.W.w_downx; p.ldb = I; p.b_mn_major = 1;
+    p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)d * I;
+    p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
+    p.rows_total = c.template p<int32_t>(L.rows_total);
+    p.epilogue = EPI_DSWIGLU; p.ab = c.template p<T>(L.ab); p.ld_ab = 2 * (int64_t)I;
+    p.rowscale = c.template p<float>(L.row_gate);
+    p.C1 = c.template p<T>(L.hmid); p.ldc1 = I;
+    p.dg_part = c.template p<float>(L.dg_part); p.dg_ld = L.dg_ld;
+    CKR(run_gemm(c, p));
+  }
+  {
+    GemmProblem p = blank_problem();   // dUp = da Wg + db Wu
+    p.M = Rp; p.N = d; p.K = 2 * I;
+    p.A = c.template p<T>(L.ab); p.lda = 2 * (int64_t)I;
+    p.B0 = c.W.w_gate; p.B1 = c.W.w_upx; p.ldb = d; p.b_mn_major = 1; p.concat = CONCAT_K;
+    p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)I * d;
+    p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
+    p.rows_total = c.template p<int32_t>(L.rows_total);
+    p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dup); p.ldc = d;
+    CKR(run_gemm(c, p));
+  }
+  if (G.w_downx) CKR(wgrad(G.w_downx, d, I, c.template p<T>(L.dop), d, 0, c.template p<T>(L.hmid), I, true, (int64_t)d * I));
+  if (G.w_gate) CKR(wgrad(G.w_gate, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, 0, c.template p<T>(L.up), d, true, (int64_t)I * d));
+  if (G.w_upx) CKR(wgrad(G.w_upx, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, I, c.template p<T>(L.up), d, true, (int64_t)I * d));
+
+  // Gate / router backward
+  router_bwd_kernel<<<(unsigned)ceil_div(Tn, 128), 128, 0, st>>>(
+      c.template p<float>(L.dg_part), L.dg_ld, n_part, c.template p<float>(L.gates), c.template p<int32_t>(L.tok_row),
+      Tn, k, c.template p<float>(L.tok_dl), c.template p<float>(L.row_dl));
+  CK(cudaGetLastError());
+  if (G.w_router || G.b_router) {
+    dim3 grid((unsigned)ceil_div(d, 256), (unsigned)E);
+    router_wgrad_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.up), c.template p<float>(L.row_dl),
+                                                 c.template p<int32_t>(L.expert_off), c.template p<int32_t>(L.expert_cnt),
+                                                 d, acc, G.w_router, G.b_router);
+    CK(cudaGetLastError());
+  }
+
+  // dU, then P_up backward and the norm
+  du_reduce_kernel<T><<<Tn, 256, 0, st>>>(c.template p<T>(L.dup), c.template p<int32_t>(L.tok_row),
+                                          c.template p<int32_t>(L.idx), c.template p<float>(L.tok_dl), k,
+                                          Is > 0 ? c.template p<T>(L.dush) : nullptr,
+                                          reinterpret_cast<const T*>(c.W.w_router), c.template p<float>(L.dl),
+                                          reinterpret_cast<const T*>(c.W.ws_sgate), d, c.template p<T>(L.du));
+  CK(cudaGetLastError());
+  {
+    GemmProblem p = blank_problem();   // dN = dU W_up  (fp32 out)
+    p.M = Tn; p.N = h; p.K = d;
+    p.A = c.template p<T>(L.du); p.lda = d;
+    p.B0 = c.W.w_up; p.ldb = h; p.b_mn_major = 1;
+    p.epilogue = EPI_STORE; p.out_f32 = 1; p.C = c.template p<float>(L.dn); p.ldc = h;
+    CKR(run_gemm(c, p));
+  }
+  if (G.w_up) CKR(wgrad(G.w_up, d, h, c.template p<T>(L.du), d, 0, c.template p<T>(L.n), h, false, 0));
+  rmsnorm_bwd_rows_kernel<<<(unsigned)ceil_div((int64_t)Tn * 32, 128), 128, 0, st>>>(
+      c.template p<float>(L.dn), y1, D.ld_stream, c.W.norm_gamma, c.template p<float>(L.r), norm_none, Tn, h, dy1,
+      D.ld_stream);
+  CK(cudaGetLastError());
+  if (G.norm_gamma) {
+    if (norm_none) {
+      if (!acc) CK(cudaMemsetAsync(G.norm_gamma, 0, (size_t)h * 4, st));
+    } else {
+      dim3 grid((unsigned)ceil_div(h, 256), (unsigned)L.strips);
+      dgamma_partial_kernel<<<grid, 256, 0, st>>>(c.template p<float>(L.dn), y1, D.ld_stream, c.template p<float>(L.r),
+                                                  Tn, h, STRIP, c.template p<float>(L.part));
+      CK(cudaGetLastError());
+      colsum_final_kernel<<<(unsigned)ceil_div(h, 256), 256, 0, st>>>(c.template p<float>(L.part), L.strips, h, acc,
+                                                                      G.norm_gamma);
+      CK(cudaGetLastError());
+    }
+  }
+  return REVFFN_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Entry-point plumbing
+// ---------------------------------------------------------------------------
+enum Pass { PASS_FWD, PASS_INV, PASS_BWD };
+
+template <typename T>
+static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weights& W, const WsLayout& L, void* ws,
+                    cudaStream_t st, const float* y1, const float* in2, float* out, const revffn_moe_grads* G,
+                    const int32_t* idx_in, int32_t* idx_out) {
+  Ctx<T> c;
+  c.D = D; c.W = W; c.L = L; c.ws = reinterpret_cast<char*>(ws); c.st = st;
+  c.tc = std::is_same<T, bf16>::value && !(D.flags & REVFFN_FLAG_FORCE_SIMT);
+  if (c.tc) CKR(tc_prepare());
+  CK(cudaMemsetAsync(c.ws + L.status.off, 0, L.status.bytes, st));
+  if (D.tokens == 0) return REVFFN_OK;   // empty batch: nothing to compute, gradients untouched
+  if (pass == PASS_BWD) return run_backward(c, y1, in2, out, *G, idx_in);
+  CKR(run_branch(c, y1, idx_in, idx_out, false));
+  return run_couple(c, in2, pass == PASS_FWD ? 1.f : -1.f, out);
+}
+
+static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1,
+                 const float* in2, float* out, const revffn_moe_grads* grads, const int32_t* idx_in,
+                 int32_t* idx_out, void* ws, size_t ws_bytes, void* cuda_stream) {
+  CKR(validate_desc(desc));
+  CKR(validate_weights(*desc, w));
+  if (!ws) return REVFFN_ERR_NULL;
+  if (pass == PASS_BWD && !grads) return REVFFN_ERR_NULL;
+  if (desc->tokens > 0 && (!y1 || !in2 || !out)) return REVFFN_ERR_NULL;
+  if (!aligned16(y1) || !aligned16(in2) || !aligned16(out) || (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return REVFFN_ERR_ALIGN;
+  if (idx_in && !aligned16(idx_in)) return REVFFN_ERR_ALIGN;
+  if (grads) {
+    const float* gs[] = {grads->norm_gamma, grads->w_up, grads->w_down, grads->w_router, grads->b_router,
+                         grads->w_gate, grads->w_upx, grads->w_downx, grads->ws_gate, grads->ws_up,
+                         grads->ws_down, grads->ws_sgate};
+    for (const float* g : gs)
+      if (g && !aligned16(g)) return REVFFN_ERR_ALIGN;
+  }
+  WsLayout L = plan_workspace(*desc);
+  if (ws_bytes < (pass == PASS_BWD ? L.bwd_bytes : L.fwd_bytes)) return REVFFN_ERR_WORKSPACE;
+  CKR(check_device());
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (desc->weight_dtype == REVFFN_BF16)
+    return dispatch<bf16>(pass, *desc, *w, L, ws, st, y1, in2, out, grads, idx_in, idx_out);
+  return dispatch<float>(pass, *desc, *w, L, ws, st, y1, in2, out, grads, idx_in, idx_out);
+}
+
+}  // namespace revffn
+
+using namespace revffn;
+
+extern "C" {
+
+int revffn_moe_workspace_size(const revffn_moe_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  WsLayout L = plan_workspace(*desc);
+  if (fwd_bytes) *fwd_bytes = L.fwd_bytes;
+  if (bwd_bytes) *bwd_bytes = L.bwd_bytes;
+  return REVFFN_OK;
+}
+
+int revffn_moe_forward(const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1, const float* x2,
+                       float* y2, int32_t* topk_idx_out, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return entry(PASS_FWD, desc, w, y1, x2, y2, nullptr, nullptr, topk_idx_out, ws, ws_bytes, cuda_stream);
+}
+
+int revffn_moe_inverse(const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1, const float* y2,
+                       float* x2, const int32_t* topk_idx_in, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return entry(PASS_INV, desc, w, y1, y2, x2, nullptr, topk_idx_in, nullptr, ws, ws_bytes, cuda_stream);
+}
+
+int revffn_moe_backward(const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1, const float* dy2,
+                        float* dy1_inout, const revffn_moe_grads* grads, const int32_t* topk_idx_in, void* ws,
+                        size_t ws_bytes, void* cuda_stream) {
+  return entry(PASS_BWD, desc, w, y1, dy2, dy1_inout, grads, topk_idx_in, nullptr, ws, ws_bytes, cuda_stream);
+}
+
+int revffn_moe_status(const void* ws, void* cuda_stream, int32_t* device_status) {
+  if (!ws || !device_status) return REVFFN_ERR_NULL;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(device_status, ws, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return REVFFN_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return REVFFN_ERR_CUDA;
+  return REVFFN_OK;
+}
+
+const char* revffn_strerror(int code) {
+  switch (code) {
+    case REVFFN_OK: return "ok";
+    case REVFFN_ERR_NULL: return "a required pointer is NULL";
+    case REVFFN_ERR_SHAPE: return "descriptor violates a shape constraint";
+    case REVFFN_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
+    case REVFFN_ERR_WORKSPACE: return "workspace too small";
+    case REVFFN_ERR_ARCH: return "device is not compute capability 10.x (sm_100a)";
+    case REVFFN_ERR_CUDA: return "CUDA call failed";
+    case REVFFN_ERR_DEVICE_WAIT: return "a bounded device-side wait expired";
+    case REVFFN_ERR_UNSUPPORTED: return "not supported";
+    default: return "unknown error";
+  }
+}
+
+int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* offset, size_t* bytes) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  if (!name) return REVFFN_ERR_NULL;
+  WsLayout L = plan_workspace(*desc);
+  struct { const char* n; const Buf* b; } tab[] = {
+      {"status", &L.status}, {"rows_total", &L.rows_total}, {"w_rc", &L.w_rc}, {"n", &L.n}, {"r", &L.r},
+      {"idx", &L.idx}, {"gates", &L.gates}, {"sgate", &L.sgate}, {"expert_cnt", &L.expert_cnt},
+      {"expert_off", &L.expert_off}, {"tile_group", &L.tile_group}, {"tok_row", &L.tok_row},
+      {"row_tok", &L.row_tok}, {"row_gate", &L.row_gate}, {"u", &L.u}, {"up", &L.up}, {"hmid", &L.hmid},
+      {"o", &L.o}, {"hs", &L.hs}, {"s", &L.s}, {"z", &L.z}, {"ab", &L.ab}, {"abs", &L.abs}, {"gb", &L.gb},
+      {"dz", &L.dz}, {"ds", &L.ds}, {"dl", &L.dl}, {"dop", &L.dop}, {"dg_part", &L.dg_part},
+      {"tok_dl", &L.tok_dl}, {"row_dl", &L.row_dl}, {"dup", &L.dup}, {"dush", &L.dush}, {"du", &L.du},
+      {"dn", &L.dn}};
+  for (auto& t : tab)
+    if (strcmp(t.n, name) == 0) {
+      if (offset) *offset = t.b->off;
+      if (bytes) *bytes = t.b->bytes;
+      return REVFFN_OK;
+    }
+  return REVFFN_ERR_UNSUPPORTED;
+}
+
+int revffn_dbg_gemm(const revffn_dbg_gemm_args* a, int32_t* status_word_dev, void* cuda_stream) {
+  if (!a) return REVFFN_ERR_NULL;
+  int r = check_device();
+  if (r != REVFFN_OK) return r;
+  GemmProblem p = blank_problem();
+  p.M = a->M; p.N = a->N; p.K = a->K;
+  p.a_mn_major = a->a_mn_major; p.b_mn_major = a->b_mn_major;
+  p.concat = a->concat; p.epilogue = a->epilogue; p.out_f32 = a->out_f32; p.accumulate = a->accumulate;
+  p.A = a->A; p.B0 = a->B0; p.B1 = a->B1; p.lda = a->lda; p.ldb = a->ldb;
+  p.C = a->C; p.C1 = a->C1; p.ldc = a->ldc; p.ldc1 = a->ldc1;
+  p.rowscale = a->rowscale; p.resid = a->resid; p.ld_resid = a->ld_resid; p.resid_sign = a->resid_sign;
+  p.ab = a->ab; p.ld_ab = a->ld_ab; p.dg_part = a->dg_part; p.dg_ld = a->dg_ld;
+  p.group_mode = a->group_mode; p.n_groups = a->n_groups;
+  p.group_off = a->group_off; p.tile_group = a->tile_group; p.rows_total = a->rows_total;
+  p.b_group_stride = a->b_group_stride; p.c_group_stride = a->c_group_stride;
+  p.a_col0 = a->a_col0; p.b_col0 = a->b_col0;
+  p.status = status_word_dev;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (a->use_simt) return launch_gemm_simt<bf16>(p, st) == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
+  r = tc_prepare();
+  if (r != REVFFN_OK) return r;
+  return launch_gemm_tc(p, st);
+}
+
+}  // extern "C"

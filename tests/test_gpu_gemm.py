@@ -1,0 +1,206 @@
+"""Unit tests of the two GEMM back ends (tcgen05 and CUDA-core) through the
+debug entry point, against a plain torch fp32 evaluation of the same problem.
+Covers every operand layout, concatenation, grouping and epilogue the three
+passes use, at sizes that span several tiles and a ragged tail."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+EPI = dict(store=0, swiglu=1, rowscale=2, couple=3, dswiglu=4, wgrad=5)
+
+
+@pytest.fixture(scope="module")
+def rv():
+    import paper_2512_20920_b200 as rv
+    return rv
+
+
+def _bf(shape, seed, scale=1.0):
+    g = torch.Generator("cuda").manual_seed(seed)
+    return (torch.randn(*shape, device="cuda", generator=g) * scale).to(torch.bfloat16)
+
+
+def _call(rv, use_simt, **kw):
+    from paper_2512_20920_b200.binding import DbgGemmArgs
+    a = DbgGemmArgs()
+    a.resid_sign = 1.0
+    keep = []
+    for k, v in kw.items():
+        if isinstance(v, torch.Tensor):
+            keep.append(v)
+            v = v.data_ptr()
+        setattr(a, k, v)
+    a.use_simt = 1 if use_simt else 0
+    status = torch.zeros(64, dtype=torch.int32, device="cuda")
+    code = rv.lib.revffn_dbg_gemm(C.byref(a), status.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    assert code == 0, rv.revffn_strerror(code)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    return keep
+
+
+def _close(a, b, tol=1e-2):
+    a = a.float().cpu().numpy().astype(np.float64)
+    b = b.float().cpu().numpy().astype(np.float64)
+    err = np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30)
+    assert err <= tol, err
+
+
+BACKENDS = [pytest.param(True, id="simt"), pytest.param(False, id="tcgen05")]
+
+
+@pytest.mark.parametrize("simt", BACKENDS)
+@pytest.mark.parametrize("M,N,K", [(300, 256, 192), (128, 128, 64), (77, 384, 1024), (1000, 512, 128)])
+def test_store_k_major(rv, simt, M, N, K):
+    A, B = _bf((M, K), 1), _bf((N, K), 2)
+    Cb = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
+    _call(rv, simt, M=M, N=N, K=K, A=A, B0=B, lda=K, ldb=K, C=Cb, ldc=N, epilogue=EPI["store"])
+    _close(Cb, A.float() @ B.float().T)
+    Cf = torch.full((M, N), float("nan"), device="cuda", dtype=torch.float32)
+    _call(rv, simt, M=M, N=N, K=K, A=A, B0=B, lda=K, ldb=K, C=Cf, ldc=N, epilogue=EPI["store"], out_f32=1)
+    _close(Cf, A.float() @ B.float().T, 1e-5)
+
+
+@pytest.mark.parametrize("simt", BACKENDS)
+def test_store_b_mn_major(rv, simt):
+    M, N, K = 300, 384, 256
+    A, B = _bf((M, K), 3), _bf((K, N), 4)            # B stored [K, N]
+    Cf = torch.full((M, N), float("nan"), device="cuda", dtype=torch.float32)
+    _call(rv, simt, M=M, N=N, K=K, A=A, B0=B, lda=K, ldb=N, b_mn_major=1, C=Cf, ldc=N, epilogue=EPI["store"], out_f32=1)
+    _close(Cf, A.float() @ B.float(), 1e-5)
+
+
+@pytest.mark.parametrize("simt", BACKENDS)
+@pytest.mark.parametrize("K", [300, 64, 1000])
+def test_wgrad_both_mn_major_ragged_k(rv, simt, K):
+    M, N = 256, 384
+    A, B = _bf((K, M + 128), 5), _bf((K, N + 128), 6)   # operands are column windows of wider buffers
+    ref = A[:, 128:].float().T @ B[:, 128:].float()
+    Cf = torch.full((M, N), float("nan"), device="cuda", dtype=torch.float32)
+    _call(rv, simt, M=M, N=N, K=K, A=A, B0=B, lda=M + 128, ldb=N + 128, a_mn_major=1, b_mn_major=1, a_col0=128,
+          b_col0=128, C=Cf, ldc=N, epilogue=EPI["wgrad"])
+    _close(Cf, ref, 1e-5)
+    _call(rv, simt, M=M, N=N, K=K, A=A, B0=B, lda=M + 128, ldb=N + 128, a_mn_major=1, b_mn_major=1, a_col0=128,
+          b_col0=128, C=Cf, ldc=N, epilogue=EPI["wgrad"], accumulate=1)
+    _close(Cf, 2 * ref, 1e-5)
+
+
+@pytest.mark.parametrize("simt", BACKENDS)
+def test_swiglu_n_concat(rv, simt):
+    M, N, K = 260, 384, 256
+    A, Bg, Bu = _bf((M, K), 7), _bf((N, K), 8, 0.2), _bf((N, K), 9, 0.2)
+    H = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
+    AB = torch.full((M, 2 * N), float("nan"), device="cuda", dtype=torch.bfloat16)
+    _call(rv, simt, M=M, N=N, K=K, A=A, B0=Bg, B1=Bu, lda=K, ldb=K, concat=1, C=H, ldc=N, C1=AB, ldc1=2 * N,
+          epilogue=EPI["swiglu"])
+    a, b = A.float() @ Bg.float().T, A.float() @ Bu.float().T
+    _close(H, torch.nn.functional.silu(a) * b)
+    _close(AB[:, :N], a)
+    _close(AB[:, N:], b)
+
+
+@pytest.mark.parametrize("simt", BACKENDS)
+def test_k_concat_b_mn_major(rv, simt):
+    M, N, Kh = 200, 256, 384
+    A, B0, B1 = _bf((M, 2 * Kh), 10), _bf((Kh, N), 11), _bf((Kh, N), 12)
+    Cb = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
+    _call(rv, simt, M=M, N=N, K=2 * Kh, A=A, B0=B0, B1=B1, lda=2 * Kh, ldb=N, b_mn_major=1, concat=2, C=Cb, ldc=N,
+          epilogue=EPI["store"])
+    _close(Cb, A[:, :Kh].float() @ B0.float() + A[:, Kh:].float() @ B1.float())
+
+
+@pytest.mark.parametrize("simt", BACKENDS)
+def test_rowscale_and_couple(rv, simt):
+    M, N, K = 300, 256, 128
+    A, B = _bf((M, K), 13), _bf((N, K), 14)
+    rs = torch.rand(M, device="cuda")
+    Cb = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
+    _call(rv, simt, M=M, N=N, K=K, A=A, B0=B, lda=K, ldb=K, C=Cb, ldc=N, rowscale=rs, epilogue=EPI["rowscale"])
+    ref = A.float() @ B.float().T
+    _close(Cb, rs[:, None] * ref)
+    # coupling epilogue on strided fp32 streams
+    X = torch.randn(M, 2 * N, device="cuda")
+    Y = torch.full((M, 2 * N), float("nan"), device="cuda")
+    for sign in (1.0, -1.0):
+        _call(rv, simt, M=M, N=N, K=K, A=A, B0=B, lda=K, ldb=K, C=Y, ldc=2 * N, resid=X, ld_resid=2 * N,
+              resid_sign=sign, epilogue=EPI["couple"])
+        _close(Y[:, :N], X[:, :N] + sign * ref, 1e-5)
+        assert torch.isnan(Y[:, N:]).all()
+
+
+@pytest.mark.parametrize("simt", BACKENDS)
+def test_dswiglu(rv, simt):
+    M, N, K = 300, 256, 128
+    A, B = _bf((M, K), 15), _bf((K, N), 16, 0.3)
+    AB = _bf((M, 2 * N), 17)
+    AB0 = AB.clone()
+    rs = torch.rand(M, device="cuda") + 0.1
+    Hg = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
+    parts = N // (64 if simt else 128)
+    dg = torch.full((M, parts), float("nan"), device="cuda")
+    _call(rv, simt, M=M, N=N, K=K, A=A, B0=B, lda=K, ldb=N, b_mn_major=1, ab=AB, ld_ab=2 * N, rowscale=rs, C1=Hg,
+          ldc1=N, dg_part=dg, dg_ld=parts, epilogue=EPI["dswiglu"])
+    acc = A.float() @ B.float()
+    a, b = AB0[:, :N].float(), AB0[:, N:].float()
+    s = torch.sigmoid(a)
+    H = a * s * b
+    dH = rs[:, None] * acc
+    _close(AB[:, :N], dH * b * (s * (1 + a * (1 - s))))
+    _close(AB[:, N:], dH * a * s)
+    _close(Hg, rs[:, None] * H)
+    _close(dg.sum(1), (acc * H).sum(1), 1e-3)
+
+
+def _groups(counts):
+    off = [0]
+    for c in counts:
+        off.append(off[-1] + ((c + 127) // 128) * 128)
+    tile_group = []
+    for e in range(len(counts)):
+        tile_group += [e] * ((off[e + 1] - off[e]) // 128)
+    return off, tile_group
+
+
+@pytest.mark.parametrize("simt", BACKENDS)
+def test_grouped_rows_and_grouped_k(rv, simt):
+    counts = [130, 0, 5, 256, 1]
+    E = len(counts)
+    off, tile_group = _groups(counts)
+    rows = off[-1]
+    rows_cap = rows + 256                              # buffers are sized for an upper bound
+    N, K = 256, 128
+    A = torch.zeros(rows_cap, K, device="cuda", dtype=torch.bfloat16)
+    for e, c in enumerate(counts):
+        A[off[e]: off[e] + c] = _bf((c, K), 20 + e)
+    A[rows:] = float("nan")                            # never read
+    W = _bf((E, N, K), 30)
+    g_off = torch.tensor(off, dtype=torch.int32, device="cuda")
+    g_tile = torch.tensor(tile_group + [0] * 8, dtype=torch.int32, device="cuda")
+    g_total = torch.tensor([rows], dtype=torch.int32, device="cuda")
+    Cb = torch.full((rows_cap, N), 7.0, device="cuda", dtype=torch.bfloat16)
+    _call(rv, simt, M=rows_cap, N=N, K=K, A=A, B0=W, lda=K, ldb=K, C=Cb, ldc=N, epilogue=EPI["store"], group_mode=1,
+          n_groups=E, group_off=g_off, tile_group=g_tile, rows_total=g_total, b_group_stride=N * K)
+    for e, c in enumerate(counts):
+        if c:
+            _close(Cb[off[e]: off[e] + c], A[off[e]: off[e] + c].float() @ W[e].float().T)
+        assert (Cb[off[e] + c: off[e + 1]] == 0).all()                    # padding rows come out as zeros
+    assert (Cb[rows:] == 7.0).all()                                       # rows past the total are untouched
+    # grouped K: per-expert weight gradient  dW[e] = A_e^T B_e
+    Bm = torch.zeros(rows_cap, N, device="cuda", dtype=torch.bfloat16)
+    Bm[:rows] = _bf((rows, N), 40)
+    for e, c in enumerate(counts):
+        Bm[off[e] + c: off[e + 1]] = 0
+    Am = A.clone(); Am[rows:] = 0
+    dW = torch.full((E, K, N), float("nan"), device="cuda")
+    _call(rv, simt, M=K, N=N, K=rows_cap, A=Am, B0=Bm, lda=K, ldb=N, a_mn_major=1, b_mn_major=1, C=dW, ldc=N,
+          epilogue=EPI["wgrad"], group_mode=2, n_groups=E, group_off=g_off, c_group_stride=K * N)
+    for e, c in enumerate(counts):
+        ref = Am[off[e]: off[e + 1]].float().T @ Bm[off[e]: off[e + 1]].float()
+        if c == 0:
+            assert (dW[e] == 0).all()
+        else:
+            _close(dW[e], ref, 1e-5)
