@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the RevFFN MoE coupling branch on B200.
+
+One step = forward (Eq. 2) + inverse reconstruction + backward by recomputation
+of one Qwen1.5-MoE-A2.7B-shaped block over one batch of synthetic tokens
+(configuration C1: 8192 tokens).  Prints ONE JSON line.
+
+    python bench.py --gpus 1 --steps 10 --warmup 3
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   (independent replicas)
+    python bench.py --impl reference        (the CPU oracle on the host cores, bounded sample per step)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "RevFFN MoE block fwd+inverse+bwd tokens/s; % of B200 bf16 tensor peak"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic per launch (bytes) of the dominant kernels from one ncu capture each
+# (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def gemm_flops(cfg, routed_rows):
+    """Algorithmic flops per launch of every matrix product, by profiler slot name
+    (rows actually routed, not the padded row space)."""
+    T, d, h, I, Is = cfg.tokens, cfg.d_model, cfg.h, cfg.d_expert, cfg.d_shared
+    R = routed_rows
+    return {
+        "gemm_p_up": 2 * T * h * d, "gemm_expert_gate_up_swiglu": 2 * R * d * 2 * I,
+        "gemm_expert_down_scale": 2 * R * I * d, "gemm_shared_gate_up_swiglu": 2 * T * d * 2 * Is,
+        "gemm_shared_down": 2 * T * Is * d, "gemm_p_down_couple": 2 * T * d * h, "gemm_dz": 2 * T * h * d,
+        "wgrad_p_down": 2 * T * h * d, "gemm_shared_dh_dswiglu": 2 * T * d * Is, "wgrad_shared_down": 2 * T * d * Is,
+        "gemm_shared_du": 2 * T * 2 * Is * d, "wgrad_shared_gate": 2 * T * Is * d, "wgrad_shared_up": 2 * T * Is * d,
+        "gemm_expert_dh_dswiglu": 2 * R * d * I, "gemm_expert_du": 2 * R * 2 * I * d,
+        "wgrad_expert_down": 2 * R * d * I, "wgrad_expert_gate": 2 * R * I * d, "wgrad_expert_up": 2 * R * I * d,
+        "gemm_dn": 2 * T * d * h, "wgrad_p_up": 2 * T * d * h,
+    }
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clocks and throttle reasons during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "50"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = [r.strip().split(", ") for r in open(self.tmp.name).read().strip().splitlines() if r.strip()]
+        os.unlink(self.tmp.name)
+        clocks, power, reasons, mx = [], [], set(), None
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                clocks.append(float(r[1])); mx = float(r[2]); power.append(float(r[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.strip().lower() == "active":
+                    reasons.add(name)
+        if clocks:
+            # under load = samples drawing real power (idle samples at the edges are dropped)
+            busy = [c for c, p in zip(clocks, power) if p >= 0.5 * max(power)] or clocks
+            out.update(sm_mhz=float(np.median(busy)), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(clocks),
+                       power_w_max=max(power))
+        return out
+
+
+def oracle_step(orc, w, s, cfg, n_tok):
+    """forward + inverse + backward of the oracle on the first n_tok tokens."""
+    y1, x2, dy2 = s["y1"][:n_tok], s["x2"][:n_tok], s["dy2"][:n_tok]
+    y2, _ = orc.forward(w, y1, x2, cfg.top_k, cfg.norm_eps)
+    orc.inverse(w, y1, y2, cfg.top_k, cfg.norm_eps)
+    orc.backward(w, y1, dy2, cfg.top_k, cfg.norm_eps)
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, cfg):
+    """The CPU oracle, as it stands, on the host cores; each step a bounded token sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import revffn_oracle as orc
+    from workloads import make_streams, make_weights
+    w = make_weights(cfg, args.seed)
+    s = make_streams(cfg, args.seed)
+    n_tok = args.cpu_sample_tokens
+    for _ in range(args.warmup):
+        oracle_step(orc, w, s, cfg, n_tok)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(orc, w, s, cfg, n_tok)
+    dt = time.perf_counter() - t0
+    value = n_tok * args.steps / dt
+    cores = blas_threads()
+    sample = f"first {n_tok} of {cfg.tokens} tokens per step, full weights, fp64 numpy"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: {cfg.tokens} tokens, d={cfg.d_model}, E={cfg.n_experts}, k={cfg.top_k}, "
+                               f"I={cfg.d_expert}, I_s={cfg.d_shared}", "sample_tokens": n_tok},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+    import paper_2512_20920_b200 as rv
+    from workloads import make_streams, make_weights
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank is an independent replica with its own tokens (seed + rank); weights are the same
+    w_host = make_weights(cfg, args.seed)
+    s_host = make_streams(cfg, args.seed + rank)
+    wdt = torch.bfloat16 if cfg.weight_dtype == "bf16" else torch.float32
+    w_dev = {n: torch.from_numpy(v).cuda().to(torch.float32 if n in ("norm_gamma", "b_router") else wdt).contiguous()
+             for n, v in w_host.items()}
+    blk = rv.Block(tokens=cfg.tokens, d_model=cfg.d_model, n_experts=cfg.n_experts, top_k=cfg.top_k,
+                   d_expert=cfg.d_expert, d_shared=cfg.d_shared,
+                   weight_dtype=rv.BF16 if cfg.weight_dtype == "bf16" else rv.F32, weights=w_dev,
+                   norm_eps=cfg.norm_eps)
+    y1, x2, dy2 = (torch.from_numpy(s_host[n]).cuda() for n in ("y1", "x2", "dy2"))
+    y2, x2r, dy1 = torch.empty_like(x2), torch.empty_like(x2), torch.zeros_like(y1)
+    # routers stay frozen (Sec. 3.3 of the paper); every other weight gets its fp32 gradient
+    grads = {n: torch.empty(v.shape, dtype=torch.float32, device="cuda") for n, v in w_dev.items()
+             if n not in ("w_router", "b_router")}
+
+    def step():
+        blk.forward(y1, x2, y2)
+        blk.inverse(y1, y2, x2r)
+        blk.backward(y1, dy2, dy1, grads)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    assert blk.status() == 0, "device status word set during warm-up"
+    routed_rows = cfg.tokens * cfg.top_k
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = rv.revffn_prof_launches()
+    rv.revffn_prof_enable(True)
+    barrier()
+    if sampler:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms_total = e0.elapsed_time(e1)
+    prof = rv.revffn_prof_collect()
+    rv.revffn_prof_enable(False)
+    launches = rv.revffn_prof_launches() - launches0
+    assert blk.status() == 0, "device status word set during the timed region"
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * cfg.tokens * args.steps / (ms_total * 1e-3)
+
+    # end to end: host-resident streams, H2D and D2H copies inside the timed region
+    pin = lambda a: torch.from_numpy(a).pin_memory()
+    hy1, hx2, hdy2 = pin(s_host["y1"]), pin(s_host["x2"]), pin(s_host["dy2"])
+    hy2, hx2r, hdy1 = (torch.empty_like(hy1).pin_memory() for _ in range(3))
+    slot = ((hy1.numel() * 4 + 255) // 256) * 256
+    staging = torch.empty(6 * slot, dtype=torch.uint8, device="cuda")
+    g_struct = blk.grads_struct(grads)
+    host_step = lambda: rv.revffn_moe_step_host(blk.desc, blk.w, g_struct, hy1, hx2, hdy2, hy2, hx2r, hdy1, staging, blk.ws)
+    for _ in range(2):
+        host_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        host_step()
+        torch.cuda.synchronize()     # the step's results are read on the host
+    dt = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([dt], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+    e2e_value = world * cfg.tokens * args.steps / dt
+    bytes_dir = 3 * hy1.numel() * 4
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    flops = gemm_flops(cfg, routed_rows)
+    # per-pass and per-kernel accounting
+    passes = {"fwd": 0.0, "inv": 0.0, "bwd": 0.0}
+    kernels = []
+    for name, (ms, cnt) in prof.items():
+        ps, kn = name.split("/")
+        passes[ps] += ms / args.steps
+        kernels.append((ms, cnt, name, kn))
+    kernels.sort(reverse=True)
+    step_flops = {"fwd": 0.0, "inv": 0.0, "bwd": 0.0}
+    for ms, cnt, name, kn in kernels:
+        if kn in flops:
+            step_flops[name.split("/")[0]] += flops[kn] * cnt / args.steps
+    total_flops = sum(step_flops.values())
+    # dominant kernel = the matrix product with the largest share of the step
+    dom = next(((ms, cnt, name, kn) for ms, cnt, name, kn in kernels if kn in flops), None)
+    roofline = None
+    if dom:
+        ms, cnt, name, kn = dom
+        achieved = flops[kn] / (ms / cnt * 1e-3) / 1e12
+        peak = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
+        roofline = {"bound": "tensor", "kernel": name, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "peak_source": f"{peak_kind} (sustained bf16 cuBLAS figure)",
+                    "traffic": NCU_TRAFFIC_BYTES.get(kn), "launch_ms": ms / cnt,
+                    "share_of_step": ms / (ms_step * args.steps)}
+    grouped = [k for k in kernels if k[3] in ("gemm_expert_gate_up_swiglu", "gemm_expert_down_scale",
+                                              "gemm_expert_dh_dswiglu", "gemm_expert_du", "wgrad_expert_down",
+                                              "wgrad_expert_gate", "wgrad_expert_up")]
+    g_fl = sum(flops[k[3]] * k[1] for k in grouped)
+    g_ms = sum(k[0] for k in grouped)
+    top = [{"kernel": name, "ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps,
+            "tflops": (flops[kn] * cnt / (ms * 1e-3) / 1e12) if kn in flops and ms > 0 else None}
+           for ms, cnt, name, kn in kernels]
+
+    # CPU baseline: the oracle as it stands on a bounded sample of the same workload (rank 0, N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import revffn_oracle as orc
+        n_tok = args.cpu_sample_tokens
+        oracle_step(orc, w_host, s_host, cfg, n_tok)      # first call pays for first-touch of its gradient arrays
+        t0 = time.perf_counter()
+        oracle_step(orc, w_host, s_host, cfg, n_tok)
+        cdt = time.perf_counter() - t0
+        cpu = {"value": n_tok / cdt, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+               "sample": f"second of two fwd+inverse+bwd passes over the first {n_tok} of {cfg.tokens} tokens, "
+                         f"full weights, fp64 numpy, {cdt:.1f} s"}
+
+    peak_t = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
+    out = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: one Qwen1.5-MoE-A2.7B-shaped block, {cfg.tokens} tokens per GPU, "
+                               f"d={cfg.d_model}, E={cfg.n_experts}, top-{cfg.top_k}, I={cfg.d_expert}, "
+                               f"I_s={cfg.d_shared}; step = forward + inverse + backward (all weight gradients "
+                               f"in fp32 except the frozen router)",
+                   "l2": "per-step working set (1.1 GB weights + >2 GB activations) exceeds the 126 MB L2",
+                   "parallelism": "independent replicas" if world > 1 else "single GPU"},
+        "pct_bf16_tensor_peak": 100.0 * total_flops / (ms_step * 1e-3) / 1e12 / peak_t,
+        "step_tflops": total_flops / (ms_step * 1e-3) / 1e12,
+        "passes_ms": passes,
+        "passes_tokens_per_s": {k: (cfg.tokens / (v * 1e-3) if v > 0 else None) for k, v in passes.items()},
+        "grouped_expert_gemms": {"tflops": g_fl / (g_ms * 1e-3) / 1e12 if g_ms > 0 else None,
+                                 "frac_of_peak": (g_fl / (g_ms * 1e-3) / 1e12 / peak_t) if g_ms > 0 else None,
+                                 "ms_per_step": g_ms / args.steps},
+        "kernels": top,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": bytes_dir,
+                "d2h_bytes_per_step": bytes_dir, "ms_per_step": 1e3 * dt / args.steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "peak_device_bytes": int(torch.cuda.max_memory_allocated()),
+        "workspace_bytes": {"fwd": blk.fwd_bytes, "bwd": blk.bwd_bytes},
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="C1")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--cpu-sample-tokens", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from workloads import CONFIGS
+    cfg = CONFIGS[args.config]
+    if args.cpu_sample_tokens is None:
+        args.cpu_sample_tokens = min(cfg.tokens, 128 if args.impl == "ours" else 64)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

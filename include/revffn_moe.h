@@ -69,7 +69,7 @@ enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                
  * Block descriptor.  Shape constraints (else REVFFN_ERR_SHAPE):
  *   tokens >= 0; d_model even; 1 <= top_k <= 8; top_k <= n_experts <= 256;
  *   d_shared >= 0 (0 = no shared expert).
- *   weight_dtype REVFFN_F32 : every width (h, d, I, I_s) a multiple of 4.
+ *   weight_dtype REVFFN_F32 : every width (h, d, I, I_s) a multiple of 8.
  *   weight_dtype REVFFN_BF16: every width a multiple of 128 (TMA / tcgen05 tiles).
  * With REVFFN_F32 all weights are float and every intermediate is fp32; with
  * REVFFN_BF16 weights are bfloat16, GEMM operands are bf16 with fp32
@@ -160,6 +160,38 @@ int revffn_moe_status(const void* ws, void* cuda_stream, int32_t* device_status)
 
 /* Text for an error code; static storage. */
 const char* revffn_strerror(int code);
+
+/*
+ * One whole step of the path with HOST-resident streams: copies y1, x2 and dy2
+ * (host, [T, h] packed, ideally pinned) to the device, runs forward (Eq. 2),
+ * inverse (Sec. 3.1) and backward (dy1 starting from zero), and copies y2, the
+ * reconstructed x2 and dy1 back to the host buffers.  `staging` is caller-owned
+ * device memory of at least 6 * round_up(T*h*4, 256) bytes, 256-byte aligned;
+ * requires ld_stream == h.  Asynchronous on the stream like the other entry
+ * points: synchronise the stream before reading the host outputs.
+ * (Convenience for end-to-end timing; no paper counterpart.)
+ */
+int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* w, const revffn_moe_grads* grads,
+                         const float* y1_host, const float* x2_host, const float* dy2_host, float* y2_host,
+                         float* x2_rec_host, float* dy1_host, void* staging, size_t staging_bytes, void* ws,
+                         size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Launch accounting and optional per-kernel timing.  (No paper counterpart.)
+ * revffn_prof_enable(1) makes every later kernel launch of this library record
+ * a CUDA event before and after itself on the caller's stream;
+ * revffn_prof_collect waits for those events and returns, per slot, the summed
+ * device milliseconds and the number of launches (host arrays of
+ * revffn_prof_num_slots() entries), then forgets them.  Slots are named
+ * "<pass>/<kernel>", pass in {fwd, inv, bwd}.  revffn_prof_launches counts
+ * every kernel this library has launched since it was loaded, enabled or not.
+ * Not thread-safe.
+ */
+int revffn_prof_enable(int on);
+long long revffn_prof_launches(void);
+int revffn_prof_num_slots(void);
+const char* revffn_prof_slot_name(int slot);
+int revffn_prof_collect(float* ms, int32_t* count, int n_slots);
 
 /*
  * Introspection for tests: byte offset and size inside the backward workspace

@@ -71,6 +71,17 @@ def _load() -> C.CDLL:
     lib.revffn_strerror.restype = C.c_char_p
     lib.revffn_moe_ws_lookup.argtypes = [C.POINTER(Desc), C.c_char_p, C.POINTER(sz), C.POINTER(sz)]
     lib.revffn_dbg_gemm.argtypes = [C.POINTER(DbgGemmArgs), vp, vp]
+    lib.revffn_moe_step_host.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.POINTER(Grads), vp, vp, vp, vp, vp, vp,
+                                         vp, sz, vp, sz, vp]
+    lib.revffn_prof_enable.argtypes = [C.c_int]
+    lib.revffn_prof_launches.argtypes = []
+    lib.revffn_prof_launches.restype = C.c_longlong
+    lib.revffn_prof_num_slots.argtypes = []
+    lib.revffn_prof_slot_name.argtypes = [C.c_int]
+    lib.revffn_prof_slot_name.restype = C.c_char_p
+    lib.revffn_prof_collect.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int32), C.c_int]
+    for f in ("revffn_moe_step_host", "revffn_prof_enable", "revffn_prof_num_slots", "revffn_prof_collect"):
+        getattr(lib, f).restype = C.c_int
     for f in ("revffn_moe_workspace_size", "revffn_moe_forward", "revffn_moe_inverse", "revffn_moe_backward",
               "revffn_moe_status", "revffn_moe_ws_lookup", "revffn_dbg_gemm"):
         getattr(lib, f).restype = C.c_int
@@ -128,6 +139,33 @@ def revffn_moe_status(ws, stream: Optional[int] = None) -> int:
     _check(lib.revffn_moe_status(_ptr(ws), stream if stream is not None else _stream(), C.byref(out)),
            "revffn_moe_status")
     return out.value
+
+
+def revffn_moe_step_host(desc: Desc, w: Weights, grads: Grads, y1_host, x2_host, dy2_host, y2_host, x2_rec_host,
+                         dy1_host, staging, ws, stream: Optional[int] = None):
+    """Host-resident streams (pinned CPU tensors) in and out; see the header."""
+    _check(lib.revffn_moe_step_host(C.byref(desc), C.byref(w), C.byref(grads), _ptr(y1_host), _ptr(x2_host),
+                                    _ptr(dy2_host), _ptr(y2_host), _ptr(x2_rec_host), _ptr(dy1_host), _ptr(staging),
+                                    staging.numel() * staging.element_size(), _ptr(ws),
+                                    ws.numel() * ws.element_size(), stream if stream is not None else _stream()),
+           "revffn_moe_step_host")
+
+
+def revffn_prof_enable(on: bool) -> bool:
+    return bool(lib.revffn_prof_enable(1 if on else 0))
+
+
+def revffn_prof_launches() -> int:
+    return int(lib.revffn_prof_launches())
+
+
+def revffn_prof_collect() -> Dict[str, tuple]:
+    """{slot name: (total device ms, launches)} since profiling was enabled or last collected."""
+    n = lib.revffn_prof_num_slots()
+    ms = (C.c_float * n)()
+    cnt = (C.c_int32 * n)()
+    _check(lib.revffn_prof_collect(ms, cnt, n), "revffn_prof_collect")
+    return {lib.revffn_prof_slot_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i] > 0}
 
 
 def ws_lookup(desc: Desc, name: str):
@@ -190,6 +228,10 @@ class Block:
         g = Grads(**{n: _ptr(grads.get(n)) for n in WEIGHT_NAMES}, accumulate=1 if accumulate else 0)
         revffn_moe_backward(self.desc, self.w, y1, dy2, dy1_inout, g, topk_idx_in, self.ws)
         return dy1_inout
+
+    def grads_struct(self, grads: Optional[Dict[str, torch.Tensor]] = None, accumulate: bool = False) -> Grads:
+        grads = grads or {}
+        return Grads(**{n: _ptr(grads.get(n)) for n in WEIGHT_NAMES}, accumulate=1 if accumulate else 0)
 
     def status(self) -> int:
         return revffn_moe_status(self.ws)

@@ -15,6 +15,59 @@
 
 namespace revffn {
 
+
+// ---------------------------------------------------------------------------
+// Launch accounting and optional per-kernel timing (CUDA events on the caller's
+// stream around each launch).  Off by default; revffn_prof_enable switches it.
+// ---------------------------------------------------------------------------
+enum Tag {
+  TG_NORM, TG_FOLD, TG_ROUTER, TG_MAP, TG_PUP, TG_GATHER, TG_EXP_GATEUP, TG_EXP_DOWN, TG_SH_GATEUP, TG_SH_DOWN,
+  TG_COMBINE, TG_PDOWN, TG_CAST, TG_DZ, TG_WG_PDOWN, TG_SHGATE_BWD, TG_SH_DH, TG_WG_SH_DOWN, TG_SH_DU,
+  TG_WG_SH_GATE, TG_WG_SH_UP, TG_WG_SGATE, TG_GATHER_DZ, TG_EXP_DH, TG_EXP_DU, TG_WG_EXP_DOWN, TG_WG_EXP_GATE,
+  TG_WG_EXP_UP, TG_ROUTER_BWD, TG_WG_ROUTER, TG_DU_REDUCE, TG_DN, TG_WG_PUP, TG_NORM_BWD, TG_DGAMMA, TG_COUNT
+};
+static const char* kTagNames[TG_COUNT] = {
+    "rmsnorm_fwd", "fold_router", "router_topk", "permute_maps", "gemm_p_up", "gather_u", "gemm_expert_gate_up_swiglu",
+    "gemm_expert_down_scale", "gemm_shared_gate_up_swiglu", "gemm_shared_down", "combine", "gemm_p_down_couple",
+    "cast_dy2", "gemm_dz", "wgrad_p_down", "shared_gate_bwd", "gemm_shared_dh_dswiglu", "wgrad_shared_down",
+    "gemm_shared_du", "wgrad_shared_gate", "wgrad_shared_up", "wgrad_shared_sgate", "gather_dz",
+    "gemm_expert_dh_dswiglu", "gemm_expert_du", "wgrad_expert_down", "wgrad_expert_gate", "wgrad_expert_up",
+    "router_bwd", "wgrad_router", "du_reduce", "gemm_dn", "wgrad_p_up", "rmsnorm_bwd", "dgamma"};
+static const char* kPassNames[3] = {"fwd", "inv", "bwd"};
+
+struct Profiler {
+  bool on = false;
+  int pass = 0;
+  std::vector<cudaEvent_t> pool;
+  size_t used = 0;
+  struct Rec { int slot; size_t e; };
+  std::vector<Rec> recs;
+  long long launches = 0;
+};
+static Profiler g_prof;
+
+struct ProfScope {
+  cudaStream_t st;
+  bool active;
+  ProfScope(int tag, cudaStream_t s) : st(s), active(false) {
+    ++g_prof.launches;
+    if (!g_prof.on) return;
+    while (g_prof.pool.size() < g_prof.used + 2) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      g_prof.pool.push_back(e);
+    }
+    cudaEventRecord(g_prof.pool[g_prof.used], st);
+    g_prof.recs.push_back({g_prof.pass * TG_COUNT + tag, g_prof.used});
+    active = true;
+  }
+  ~ProfScope() {
+    if (!active) return;
+    cudaEventRecord(g_prof.pool[g_prof.used + 1], st);
+    g_prof.used += 2;
+  }
+};
+
 // ---------------------------------------------------------------------------
 // Workspace layout
 // ---------------------------------------------------------------------------
@@ -157,8 +210,9 @@ struct Ctx {
 };
 
 template <typename T>
-static int run_gemm(const Ctx<T>& c, GemmProblem p) {
+static int run_gemm(const Ctx<T>& c, GemmProblem p, int tag) {
   p.status = c.template p<int>(c.L.status);
+  ProfScope ps(tag, c.st);
   if constexpr (std::is_same<T, bf16>::value) {
     if (c.tc) return launch_gemm_tc(p, c.st);
   }
@@ -194,40 +248,52 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
   const T* w_up = reinterpret_cast<const T*>(c.W.w_up);
 
   // Norm
+  { ProfScope ps(TG_NORM, st);
   rmsnorm_fwd_kernel<T><<<(unsigned)ceil_div((int64_t)Tn * 32, 128), 128, 0, st>>>(
       y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, Tn, h, c.template p<T>(L.n), c.template p<float>(L.r));
+  }
   CK(cudaGetLastError());
 
   // Router: fold through P_up, logits, top-k, gates
   {
     dim3 grid((unsigned)ceil_div(h, 128), (unsigned)(E + 1));
+    { ProfScope ps(TG_FOLD, st);
     fold_router_kernel<T><<<grid, 128, 0, st>>>(reinterpret_cast<const T*>(c.W.w_router),
                                                  reinterpret_cast<const T*>(c.W.ws_sgate), w_up, E, d, h,
                                                  c.template p<double>(L.w_rc));
+    }
     CK(cudaGetLastError());
     size_t smem = router_smem_bytes(E);
+    { ProfScope ps(TG_ROUTER, st);
     router_topk_kernel<<<(unsigned)ceil_div(Tn, RT_TOK), 256, smem, st>>>(
         y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, c.template p<double>(L.w_rc), c.W.b_router, Tn, h,
         E, k, Is > 0 ? 1 : 0, idx_in, c.template p<int32_t>(L.idx), c.template p<float>(L.gates),
         c.template p<float>(L.sgate), idx_user);
+    }
     CK(cudaGetLastError());
   }
 
   // Permutation maps
   CK(cudaMemsetAsync(c.ws + L.row_tok.off, 0xFF, L.row_tok.bytes, st));
   CK(cudaMemsetAsync(c.ws + L.row_gate.off, 0, L.row_gate.bytes, st));
+  { ProfScope ps(TG_MAP, st);
   map_rank_kernel<<<L.n_chunks, 256, (size_t)MAP_CHUNK * k * 4, st>>>(
       c.template p<int32_t>(L.idx), Tn, k, E, c.template p<int32_t>(L.local_rank), c.template p<int32_t>(L.chunk_cnt));
+  }
   CK(cudaGetLastError());
+  { ProfScope ps(TG_MAP, st);
   map_scan_kernel<<<1, 256, (size_t)(E + 1) * 4, st>>>(
       c.template p<int32_t>(L.chunk_cnt), L.n_chunks, E, c.template p<int32_t>(L.chunk_base),
       c.template p<int32_t>(L.expert_cnt), c.template p<int32_t>(L.expert_off), c.template p<int32_t>(L.tile_group),
       c.template p<int32_t>(L.rows_total), L.max_tiles);
+  }
   CK(cudaGetLastError());
+  { ProfScope ps(TG_MAP, st);
   map_assign_kernel<<<(unsigned)ceil_div((int64_t)Tn * k, 256), 256, 0, st>>>(
       c.template p<int32_t>(L.idx), c.template p<float>(L.gates), c.template p<int32_t>(L.local_rank),
       c.template p<int32_t>(L.chunk_base), c.template p<int32_t>(L.expert_off), Tn, k, E,
       c.template p<int32_t>(L.tok_row), c.template p<int32_t>(L.row_tok), c.template p<float>(L.row_gate));
+  }
   CK(cudaGetLastError());
 
   // P_up: U = N W_up^T
@@ -237,13 +303,15 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     p.A = c.template p<T>(L.n); p.lda = h;
     p.B0 = w_up; p.ldb = h;
     p.epilogue = EPI_STORE; p.C = c.template p<T>(L.u); p.ldc = d;
-    CKR(run_gemm(c, p));
+    CKR(run_gemm(c, p, TG_PUP));
   }
 
   // Permute: Up[row] = U[token(row)]
+  { ProfScope ps(TG_GATHER, st);
   gather_rows_kernel<T><<<(unsigned)L.rows_pad, 256, 0, st>>>(c.template p<T>(L.u), d, c.template p<int32_t>(L.row_tok),
                                                               c.template p<int32_t>(L.rows_total), d,
                                                               c.template p<T>(L.up));
+  }
   CK(cudaGetLastError());
 
   // Routed experts: H = silu(Up Wg^T) * (Up Wu^T);  O = g * (H Wd^T)
@@ -257,7 +325,7 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     p.rows_total = c.template p<int32_t>(L.rows_total);
     p.epilogue = EPI_SWIGLU; p.C = c.template p<T>(L.hmid); p.ldc = I;
     if (save_ab) { p.C1 = c.template p<T>(L.ab); p.ldc1 = 2 * (int64_t)I; }
-    CKR(run_gemm(c, p));
+    CKR(run_gemm(c, p, TG_EXP_GATEUP));
   }
   {
     GemmProblem p = blank_problem();
@@ -269,7 +337,7 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     p.rows_total = c.template p<int32_t>(L.rows_total);
     p.epilogue = EPI_ROWSCALE; p.rowscale = c.template p<float>(L.row_gate);
     p.C = c.template p<T>(L.o); p.ldc = d;
-    CKR(run_gemm(c, p));
+    CKR(run_gemm(c, p, TG_EXP_DOWN));
   }
 
   // Shared expert: S = (silu(U Wsg^T) * (U Wsu^T)) Wsd^T
@@ -280,20 +348,22 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     p.B0 = c.W.ws_gate; p.B1 = c.W.ws_up; p.ldb = d; p.concat = CONCAT_N;
     p.epilogue = EPI_SWIGLU; p.C = c.template p<T>(L.hs); p.ldc = Is;
     if (save_ab) { p.C1 = c.template p<T>(L.abs); p.ldc1 = 2 * (int64_t)Is; }
-    CKR(run_gemm(c, p));
+    CKR(run_gemm(c, p, TG_SH_GATEUP));
     GemmProblem q = blank_problem();
     q.M = Tn; q.N = d; q.K = Is;
     q.A = c.template p<T>(L.hs); q.lda = Is;
     q.B0 = c.W.ws_down; q.ldb = Is;
     q.epilogue = EPI_STORE; q.C = c.template p<T>(L.s); q.ldc = d;
-    CKR(run_gemm(c, q));
+    CKR(run_gemm(c, q, TG_SH_DOWN));
   }
 
   // Combine: Z[t] = sum_s O[row(t,s)] + sgate_t S[t]
   if (Tn > 0) {
+    { ProfScope ps(TG_COMBINE, st);
     combine_rows_kernel<T><<<Tn, 256, 0, st>>>(c.template p<T>(L.o), c.template p<int32_t>(L.tok_row), k,
                                                Is > 0 ? c.template p<T>(L.s) : nullptr, c.template p<float>(L.sgate),
                                                d, c.template p<T>(L.z));
+    }
     CK(cudaGetLastError());
   }
   return REVFFN_OK;
@@ -309,7 +379,7 @@ static int run_couple(const Ctx<T>& c, const float* resid, float sign, float* ou
   p.B0 = c.W.w_down; p.ldb = d;
   p.epilogue = EPI_COUPLE; p.resid = resid; p.ld_resid = c.D.ld_stream; p.resid_sign = sign;
   p.C = out; p.ldc = c.D.ld_stream;
-  return run_gemm(c, p);
+  return run_gemm(c, p, TG_PDOWN);
 }
 
 template <typename T>
@@ -325,7 +395,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
 
   CKR(run_branch(c, y1, idx_in, nullptr, true));
 
-  auto wgrad = [&](float* out, int M, int N, const void* A, int64_t lda, int a_col0, const void* B, int64_t ldb,
+  auto wgrad = [&](int tag, float* out, int M, int N, const void* A, int64_t lda, int a_col0, const void* B, int64_t ldb,
                    bool grouped, int64_t cstride) -> int {
     GemmProblem p = blank_problem();
     p.M = M; p.N = N; p.K = grouped ? Rp : Tn;   // grouped: bound on rows, the range comes from group_off
@@ -338,12 +408,14 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       p.group_mode = GROUP_K; p.n_groups = E;
       p.group_off = c.template p<int32_t>(L.expert_off);
     }
-    return run_gemm(c, p);
+    return run_gemm(c, p, tag);
   };
 
   // P_down backward: dZ = G W_down;  dW_down = G^T Z
+  { ProfScope ps(TG_CAST, st);
   cast_stream_kernel<T><<<(unsigned)ceil_div((int64_t)Tn * h, 4 * 256), 256, 0, st>>>(dy2, D.ld_stream, Tn, h,
                                                                                       c.template p<T>(L.gb));
+  }
   CK(cudaGetLastError());
   {
     GemmProblem p = blank_problem();
@@ -351,15 +423,17 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.A = c.template p<T>(L.gb); p.lda = h;
     p.B0 = c.W.w_down; p.ldb = d; p.b_mn_major = 1;
     p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dz); p.ldc = d;
-    CKR(run_gemm(c, p));
+    CKR(run_gemm(c, p, TG_DZ));
   }
-  if (G.w_down) CKR(wgrad(G.w_down, h, d, c.template p<T>(L.gb), h, 0, c.template p<T>(L.z), d, false, 0));
+  if (G.w_down) CKR(wgrad(TG_WG_PDOWN, G.w_down, h, d, c.template p<T>(L.gb), h, 0, c.template p<T>(L.z), d, false, 0));
 
   // Shared expert backward
   if (Is > 0) {
+    { ProfScope ps(TG_SHGATE_BWD, st);
     shared_gate_bwd_kernel<T><<<Tn, 256, 0, st>>>(c.template p<T>(L.dz), c.template p<T>(L.s),
                                                   c.template p<float>(L.sgate), d, c.template p<T>(L.ds),
                                                   c.template p<float>(L.dl));
+    }
     CK(cudaGetLastError());
     {
       GemmProblem p = blank_problem();   // dH_s = dS Ws_d, then SwiGLU backward in place on a|b
@@ -367,33 +441,39 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       p.A = c.template p<T>(L.ds); p.lda = d;
       p.B0 = c.W.ws_down; p.ldb = Is; p.b_mn_major = 1;
       p.epilogue = EPI_DSWIGLU; p.ab = c.template p<T>(L.abs); p.ld_ab = 2 * (int64_t)Is;
-      CKR(run_gemm(c, p));
+      CKR(run_gemm(c, p, TG_SH_DH));
     }
-    if (G.ws_down) CKR(wgrad(G.ws_down, d, Is, c.template p<T>(L.ds), d, 0, c.template p<T>(L.hs), Is, false, 0));
+    if (G.ws_down) CKR(wgrad(TG_WG_SH_DOWN, G.ws_down, d, Is, c.template p<T>(L.ds), d, 0, c.template p<T>(L.hs), Is, false, 0));
     {
       GemmProblem p = blank_problem();   // dU_sh = da Ws_g + db Ws_u
       p.M = Tn; p.N = d; p.K = 2 * Is;
       p.A = c.template p<T>(L.abs); p.lda = 2 * (int64_t)Is;
       p.B0 = c.W.ws_gate; p.B1 = c.W.ws_up; p.ldb = d; p.b_mn_major = 1; p.concat = CONCAT_K;
       p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dush); p.ldc = d;
-      CKR(run_gemm(c, p));
+      CKR(run_gemm(c, p, TG_SH_DU));
     }
-    if (G.ws_gate) CKR(wgrad(G.ws_gate, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, 0, c.template p<T>(L.u), d, false, 0));
-    if (G.ws_up) CKR(wgrad(G.ws_up, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, Is, c.template p<T>(L.u), d, false, 0));
+    if (G.ws_gate) CKR(wgrad(TG_WG_SH_GATE, G.ws_gate, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, 0, c.template p<T>(L.u), d, false, 0));
+    if (G.ws_up) CKR(wgrad(TG_WG_SH_UP, G.ws_up, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, Is, c.template p<T>(L.u), d, false, 0));
     if (G.ws_sgate) {
       dim3 grid((unsigned)ceil_div(d, 256), (unsigned)L.strips);
+      { ProfScope ps(TG_WG_SGATE, st);
       colsum_partial_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.u), d, c.template p<float>(L.dl), Tn, d, STRIP,
                                                      c.template p<float>(L.part));
+      }
       CK(cudaGetLastError());
+      { ProfScope ps(TG_WG_SGATE, st);
       colsum_final_kernel<<<(unsigned)ceil_div(d, 256), 256, 0, st>>>(c.template p<float>(L.part), L.strips, d, acc,
                                                                       G.ws_sgate);
+      }
       CK(cudaGetLastError());
     }
   }
 
   // Routed experts backward
+  { ProfScope ps(TG_GATHER_DZ, st);
   gather_rows_kernel<T><<<(unsigned)Rp, 256, 0, st>>>(c.template p<T>(L.dz), d, c.template p<int32_t>(L.row_tok),
                                                       c.template p<int32_t>(L.rows_total), d, c.template p<T>(L.dop));
+  }
   CK(cudaGetLastError());
   const int n_part = dg_parts(c, I);
   {
@@ -408,7 +488,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.rowscale = c.template p<float>(L.row_gate);
     p.C1 = c.template p<T>(L.hmid); p.ldc1 = I;
     p.dg_part = c.template p<float>(L.dg_part); p.dg_ld = L.dg_ld;
-    CKR(run_gemm(c, p));
+    CKR(run_gemm(c, p, TG_EXP_DH));
   }
   {
     GemmProblem p = blank_problem();   // dUp = da Wg + db Wu
@@ -419,31 +499,37 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
     p.rows_total = c.template p<int32_t>(L.rows_total);
     p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dup); p.ldc = d;
-    CKR(run_gemm(c, p));
+    CKR(run_gemm(c, p, TG_EXP_DU));
   }
-  if (G.w_downx) CKR(wgrad(G.w_downx, d, I, c.template p<T>(L.dop), d, 0, c.template p<T>(L.hmid), I, true, (int64_t)d * I));
-  if (G.w_gate) CKR(wgrad(G.w_gate, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, 0, c.template p<T>(L.up), d, true, (int64_t)I * d));
-  if (G.w_upx) CKR(wgrad(G.w_upx, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, I, c.template p<T>(L.up), d, true, (int64_t)I * d));
+  if (G.w_downx) CKR(wgrad(TG_WG_EXP_DOWN, G.w_downx, d, I, c.template p<T>(L.dop), d, 0, c.template p<T>(L.hmid), I, true, (int64_t)d * I));
+  if (G.w_gate) CKR(wgrad(TG_WG_EXP_GATE, G.w_gate, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, 0, c.template p<T>(L.up), d, true, (int64_t)I * d));
+  if (G.w_upx) CKR(wgrad(TG_WG_EXP_UP, G.w_upx, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, I, c.template p<T>(L.up), d, true, (int64_t)I * d));
 
   // Gate / router backward
+  { ProfScope ps(TG_ROUTER_BWD, st);
   router_bwd_kernel<<<(unsigned)ceil_div(Tn, 128), 128, 0, st>>>(
       c.template p<float>(L.dg_part), L.dg_ld, n_part, c.template p<float>(L.gates), c.template p<int32_t>(L.tok_row),
       Tn, k, c.template p<float>(L.tok_dl), c.template p<float>(L.row_dl));
+  }
   CK(cudaGetLastError());
   if (G.w_router || G.b_router) {
     dim3 grid((unsigned)ceil_div(d, 256), (unsigned)E);
+    { ProfScope ps(TG_WG_ROUTER, st);
     router_wgrad_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.up), c.template p<float>(L.row_dl),
                                                  c.template p<int32_t>(L.expert_off), c.template p<int32_t>(L.expert_cnt),
                                                  d, acc, G.w_router, G.b_router);
+    }
     CK(cudaGetLastError());
   }
 
   // dU, then P_up backward and the norm
+  { ProfScope ps(TG_DU_REDUCE, st);
   du_reduce_kernel<T><<<Tn, 256, 0, st>>>(c.template p<T>(L.dup), c.template p<int32_t>(L.tok_row),
                                           c.template p<int32_t>(L.idx), c.template p<float>(L.tok_dl), k,
                                           Is > 0 ? c.template p<T>(L.dush) : nullptr,
                                           reinterpret_cast<const T*>(c.W.w_router), c.template p<float>(L.dl),
                                           reinterpret_cast<const T*>(c.W.ws_sgate), d, c.template p<T>(L.du));
+  }
   CK(cudaGetLastError());
   {
     GemmProblem p = blank_problem();   // dN = dU W_up  (fp32 out)
@@ -451,23 +537,29 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.A = c.template p<T>(L.du); p.lda = d;
     p.B0 = c.W.w_up; p.ldb = h; p.b_mn_major = 1;
     p.epilogue = EPI_STORE; p.out_f32 = 1; p.C = c.template p<float>(L.dn); p.ldc = h;
-    CKR(run_gemm(c, p));
+    CKR(run_gemm(c, p, TG_DN));
   }
-  if (G.w_up) CKR(wgrad(G.w_up, d, h, c.template p<T>(L.du), d, 0, c.template p<T>(L.n), h, false, 0));
+  if (G.w_up) CKR(wgrad(TG_WG_PUP, G.w_up, d, h, c.template p<T>(L.du), d, 0, c.template p<T>(L.n), h, false, 0));
+  { ProfScope ps(TG_NORM_BWD, st);
   rmsnorm_bwd_rows_kernel<<<(unsigned)ceil_div((int64_t)Tn * 32, 128), 128, 0, st>>>(
       c.template p<float>(L.dn), y1, D.ld_stream, c.W.norm_gamma, c.template p<float>(L.r), norm_none, Tn, h, dy1,
       D.ld_stream);
+  }
   CK(cudaGetLastError());
   if (G.norm_gamma) {
     if (norm_none) {
       if (!acc) CK(cudaMemsetAsync(G.norm_gamma, 0, (size_t)h * 4, st));
     } else {
       dim3 grid((unsigned)ceil_div(h, 256), (unsigned)L.strips);
+      { ProfScope ps(TG_DGAMMA, st);
       dgamma_partial_kernel<<<grid, 256, 0, st>>>(c.template p<float>(L.dn), y1, D.ld_stream, c.template p<float>(L.r),
                                                   Tn, h, STRIP, c.template p<float>(L.part));
+      }
       CK(cudaGetLastError());
+      { ProfScope ps(TG_DGAMMA, st);
       colsum_final_kernel<<<(unsigned)ceil_div(h, 256), 256, 0, st>>>(c.template p<float>(L.part), L.strips, h, acc,
                                                                       G.norm_gamma);
+      }
       CK(cudaGetLastError());
     }
   }
@@ -485,6 +577,7 @@ static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weight
                     const int32_t* idx_in, int32_t* idx_out) {
   Ctx<T> c;
   c.D = D; c.W = W; c.L = L; c.ws = reinterpret_cast<char*>(ws); c.st = st;
+  g_prof.pass = (int)pass;
   c.tc = std::is_same<T, bf16>::value && !(D.flags & REVFFN_FLAG_FORCE_SIMT);
   if (c.tc) CKR(tc_prepare());
   CK(cudaMemsetAsync(c.ws + L.status.off, 0, L.status.bytes, st));
@@ -597,6 +690,77 @@ int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* 
       return REVFFN_OK;
     }
   return REVFFN_ERR_UNSUPPORTED;
+}
+
+int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* w, const revffn_moe_grads* grads,
+                         const float* y1_host, const float* x2_host, const float* dy2_host, float* y2_host,
+                         float* x2_rec_host, float* dy1_host, void* staging, size_t staging_bytes, void* ws,
+                         size_t ws_bytes, void* cuda_stream) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  if (!y1_host || !x2_host || !dy2_host || !y2_host || !x2_rec_host || !dy1_host || !staging) return REVFFN_ERR_NULL;
+  const int h = desc->d_model / 2;
+  if (desc->ld_stream != h) return REVFFN_ERR_SHAPE;
+  const size_t n = (size_t)desc->tokens * h * sizeof(float);
+  const size_t slot = (size_t)round_up((int64_t)(n > 0 ? n : 1), 256);
+  if (staging_bytes < 6 * slot || (reinterpret_cast<uintptr_t>(staging) & 255u)) return REVFFN_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* sp = reinterpret_cast<char*>(staging);
+  float* y1 = reinterpret_cast<float*>(sp);
+  float* x2 = reinterpret_cast<float*>(sp + slot);
+  float* dy2 = reinterpret_cast<float*>(sp + 2 * slot);
+  float* y2 = reinterpret_cast<float*>(sp + 3 * slot);
+  float* x2r = reinterpret_cast<float*>(sp + 4 * slot);
+  float* dy1 = reinterpret_cast<float*>(sp + 5 * slot);
+  if (n > 0) {
+    CK(cudaMemcpyAsync(y1, y1_host, n, cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(x2, x2_host, n, cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(dy2, dy2_host, n, cudaMemcpyHostToDevice, st));
+    CK(cudaMemsetAsync(dy1, 0, n, st));
+  }
+  CKR(revffn_moe_forward(desc, w, y1, x2, y2, nullptr, ws, ws_bytes, cuda_stream));
+  CKR(revffn_moe_inverse(desc, w, y1, y2, x2r, nullptr, ws, ws_bytes, cuda_stream));
+  CKR(revffn_moe_backward(desc, w, y1, dy2, dy1, grads, nullptr, ws, ws_bytes, cuda_stream));
+  if (n > 0) {
+    CK(cudaMemcpyAsync(y2_host, y2, n, cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(x2_rec_host, x2r, n, cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(dy1_host, dy1, n, cudaMemcpyDeviceToHost, st));
+  }
+  return REVFFN_OK;
+}
+
+int revffn_prof_enable(int on) {
+  int prev = g_prof.on ? 1 : 0;
+  g_prof.on = on != 0;
+  g_prof.recs.clear();
+  g_prof.used = 0;
+  return prev;
+}
+
+long long revffn_prof_launches(void) { return g_prof.launches; }
+
+int revffn_prof_num_slots(void) { return 3 * TG_COUNT; }
+
+const char* revffn_prof_slot_name(int slot) {
+  static char buf[3 * TG_COUNT][64];
+  if (slot < 0 || slot >= 3 * TG_COUNT) return "";
+  snprintf(buf[slot], sizeof(buf[slot]), "%s/%s", kPassNames[slot / TG_COUNT], kTagNames[slot % TG_COUNT]);
+  return buf[slot];
+}
+
+int revffn_prof_collect(float* ms, int32_t* count, int n_slots) {
+  if (!ms || !count) return REVFFN_ERR_NULL;
+  for (int i = 0; i < n_slots; ++i) { ms[i] = 0.f; count[i] = 0; }
+  for (const auto& rec : g_prof.recs) {
+    if (rec.e + 1 >= g_prof.pool.size()) continue;
+    if (cudaEventSynchronize(g_prof.pool[rec.e + 1]) != cudaSuccess) return REVFFN_ERR_CUDA;
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, g_prof.pool[rec.e], g_prof.pool[rec.e + 1]) != cudaSuccess) return REVFFN_ERR_CUDA;
+    if (rec.slot >= 0 && rec.slot < n_slots) { ms[rec.slot] += t; count[rec.slot] += 1; }
+  }
+  g_prof.recs.clear();
+  g_prof.used = 0;
+  return REVFFN_OK;
 }
 
 int revffn_dbg_gemm(const revffn_dbg_gemm_args* a, int32_t* status_word_dev, void* cuda_stream) {
