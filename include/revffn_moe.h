@@ -34,8 +34,9 @@
  *     as void*).  Calls that share a workspace must be ordered on one stream.
  *   - Return value: REVFFN_OK (0) or a negative revffn_error.  On an error
  *     return nothing has been launched.  Device-side problems (a bounded wait
- *     that expired) set a sticky status word in the workspace; read it with
- *     revffn_moe_status.
+ *     that expired) set a status word in the workspace, first error wins; each
+ *     forward/inverse/backward call clears it when it starts, so
+ *     revffn_moe_status reports the most recent call.
  */
 #ifndef REVFFN_MOE_H_
 #define REVFFN_MOE_H_
@@ -154,7 +155,7 @@ int revffn_moe_backward(const revffn_moe_desc* desc, const revffn_moe_weights* w
                         const revffn_moe_grads* grads, const int32_t* topk_idx_in,
                         void* ws, size_t ws_bytes, void* cuda_stream);
 
-/* Synchronise the stream and copy the workspace's sticky device status word to
+/* Synchronise the stream and copy the workspace's device status word to
  * *device_status (host pointer): 0 or a negative revffn_error.  (No paper counterpart.) */
 int revffn_moe_status(const void* ws, void* cuda_stream, int32_t* device_status);
 
