@@ -57,7 +57,8 @@ typedef enum {
   REVFFN_ERR_ARCH = -5,         /* current device is not compute capability 10.x    */
   REVFFN_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed                */
   REVFFN_ERR_DEVICE_WAIT = -7,  /* status word: a bounded device-side wait expired  */
-  REVFFN_ERR_UNSUPPORTED = -8   /* valid request that this build does not implement */
+  REVFFN_ERR_UNSUPPORTED = -8,  /* valid request that this build does not implement */
+  REVFFN_ERR_NOALLOC_LIMIT = -9 /* revffn_moe_route_noalloc: problem exceeds its fixed scratch */
 } revffn_error;
 
 enum { REVFFN_F32 = 0, REVFFN_BF16 = 1 };          /* weight_dtype                    */
@@ -176,6 +177,39 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
                          const float* y1_host, const float* x2_host, const float* dy2_host, float* y2_host,
                          float* x2_rec_host, float* dy1_host, void* staging, size_t staging_bytes, void* ws,
                          size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Routing only, for callers that must not allocate.  (The paper has no
+ * counterpart: this is a packaging of the router step of MLP_pt.)
+ *
+ * Some callers cannot provide a workspace because they cannot call cudaMalloc
+ * at the point where they need the routing decision: code running inside a
+ * stream-ordered region that forbids allocation, a plug-in whose host gives it
+ * only its input and output tensors, or a process that has handed all device
+ * memory to another allocator.  For them this entry point computes
+ *   topk_idx_out [T, k] int32   selected experts per token, descending logit
+ *   gates_out    [T, k] fp32    softmax over the selected logits
+ *   sgate_out    [T]    fp32    shared-expert sigmoid gate (0 without one)
+ * from y1 ([T, h] fp32, stride ld_stream) exactly as revffn_moe_forward does,
+ * but keeps its one piece of scratch -- the router folded through P_up,
+ * (E + 1) * h doubles -- in a fixed array inside the library's device image
+ * rather than in a workspace.  It calls no cudaMalloc, cudaFree or other
+ * allocating routine.
+ *
+ * Limits and sharing
+ *   - (E + 1) * h <= REVFFN_ROUTE_NOALLOC_MAX_ELEMS (512 KB of scratch, held by
+ *     every device that loads the library until the process exits) and
+ *     n_experts small enough for 48 KB of shared memory (E <= 100 or so);
+ *     otherwise REVFFN_ERR_NOALLOC_LIMIT and nothing is launched.
+ *   - The first call on a device looks up the array's device address; make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call rewrites the part
+ *     it uses before reading it, so nothing has to be cleared, but two calls
+ *     that overlap on the GPU (different streams) race: order them.
+ */
+#define REVFFN_ROUTE_NOALLOC_MAX_ELEMS 65536
+int revffn_moe_route_noalloc(const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1,
+                             int32_t* topk_idx_out, float* gates_out, float* sgate_out, void* cuda_stream);
 
 /*
  * Launch accounting and optional per-kernel timing.  (No paper counterpart.)

@@ -1,12 +1,20 @@
 """B200 (sm_100a) library for the MoE coupling branch of a RevFFN block:
 forward Y2 = X2 + MLP(Norm(Y1)), its inverse, and its backward by
 recomputation.  All arithmetic runs in the CUDA library behind the C ABI in
-include/revffn_moe.h; this package only marshals arguments."""
-from .binding import (revffn_moe_step_host, revffn_prof_enable, revffn_prof_launches, revffn_prof_collect,
-                      Block, Desc, Grads, Weights, lib, revffn_moe_backward, revffn_moe_forward,
-                      revffn_moe_inverse, revffn_moe_status, revffn_moe_workspace_size, revffn_strerror,
-                      RevffnError, BF16, F32, NORM_RMS, NORM_NONE, FLAG_FORCE_SIMT)
+include/revffn_moe.h; this package only marshals arguments.
 
-__all__ = ["revffn_moe_step_host", "revffn_prof_enable", "revffn_prof_launches", "revffn_prof_collect", "Block", "Desc", "Grads", "Weights", "lib", "revffn_moe_backward", "revffn_moe_forward",
+Names are resolved from `binding` on first use, so that `build` can be imported
+before the shared library exists.  There is no fallback: using anything here
+without the built library raises ImportError."""
+import importlib
+
+__all__ = ["Block", "Desc", "Grads", "Weights", "lib", "revffn_moe_backward", "revffn_moe_forward",
            "revffn_moe_inverse", "revffn_moe_status", "revffn_moe_workspace_size", "revffn_strerror",
-           "RevffnError", "BF16", "F32", "NORM_RMS", "NORM_NONE", "FLAG_FORCE_SIMT"]
+           "revffn_moe_step_host", "revffn_moe_route_noalloc", "revffn_prof_enable", "revffn_prof_launches",
+           "revffn_prof_collect", "RevffnError", "BF16", "F32", "NORM_RMS", "NORM_NONE", "FLAG_FORCE_SIMT"]
+
+
+def __getattr__(name):
+    if name in __all__:
+        return getattr(importlib.import_module(".binding", __name__), name)
+    raise AttributeError(f"module {__name__!r} has no attribute {name!r}")

@@ -73,6 +73,8 @@ def _load() -> C.CDLL:
     lib.revffn_dbg_gemm.argtypes = [C.POINTER(DbgGemmArgs), vp, vp]
     lib.revffn_moe_step_host.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.POINTER(Grads), vp, vp, vp, vp, vp, vp,
                                          vp, sz, vp, sz, vp]
+    lib.revffn_moe_route_noalloc.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, vp, vp]
+    lib.revffn_moe_route_noalloc.restype = C.c_int
     lib.revffn_prof_enable.argtypes = [C.c_int]
     lib.revffn_prof_launches.argtypes = []
     lib.revffn_prof_launches.restype = C.c_longlong
@@ -149,6 +151,15 @@ def revffn_moe_step_host(desc: Desc, w: Weights, grads: Grads, y1_host, x2_host,
                                     staging.numel() * staging.element_size(), _ptr(ws),
                                     ws.numel() * ws.element_size(), stream if stream is not None else _stream()),
            "revffn_moe_step_host")
+
+
+def revffn_moe_route_noalloc(desc: Desc, w: Weights, y1, topk_idx_out, gates_out, sgate_out,
+                             stream: Optional[int] = None):
+    """Routing (expert indices, gate weights, shared gate) with the library's own fixed scratch: for callers
+    that cannot allocate a workspace.  Calls on one device must not overlap; see the header."""
+    _check(lib.revffn_moe_route_noalloc(C.byref(desc), C.byref(w), _ptr(y1), _ptr(topk_idx_out), _ptr(gates_out),
+                                        _ptr(sgate_out), stream if stream is not None else _stream()),
+           "revffn_moe_route_noalloc")
 
 
 def revffn_prof_enable(on: bool) -> bool:

@@ -614,6 +614,46 @@ static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weight
   return dispatch<float>(pass, *desc, *w, L, ws, st, y1, in2, out, grads, idx_in, idx_out);
 }
 
+// ---------------------------------------------------------------------------
+// Routing without any allocation.  The folded router matrix, which the regular
+// entry points keep in the caller's workspace, lives in a fixed array inside
+// the library's own device image instead.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) double g_route_scratch[REVFFN_ROUTE_NOALLOC_MAX_ELEMS];
+
+// Device address of g_route_scratch, looked up once per device.  In host code the
+// symbol itself is only a handle, not something a kernel may dereference.
+static double* route_scratch_ptr(int* err) {
+  static double* ptr[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = REVFFN_ERR_CUDA; return nullptr; }
+  if (!ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_route_scratch) != cudaSuccess || !p) { *err = REVFFN_ERR_CUDA; return nullptr; }
+    ptr[dev] = reinterpret_cast<double*>(p);
+  }
+  *err = REVFFN_OK;
+  return ptr[dev];
+}
+
+template <typename T>
+static int route_noalloc_launch(const revffn_moe_desc& D, const revffn_moe_weights& W, const float* y1,
+                                double* w_rc, int32_t* idx, float* gates, float* sgate, cudaStream_t st) {
+  const int d = D.d_model, h = d / 2, E = D.n_experts;
+  const int norm_none = D.norm_kind == REVFFN_NORM_NONE;
+  dim3 grid((unsigned)ceil_div(h, 128), (unsigned)(E + 1));
+  fold_router_kernel<T><<<grid, 128, 0, st>>>(reinterpret_cast<const T*>(W.w_router),
+                                               reinterpret_cast<const T*>(W.ws_sgate),
+                                               reinterpret_cast<const T*>(W.w_up), E, d, h, w_rc);
+  CK(cudaGetLastError());
+  router_topk_kernel<<<(unsigned)ceil_div(D.tokens, RT_TOK), 256, router_smem_bytes(E), st>>>(
+      y1, D.ld_stream, W.norm_gamma, D.norm_eps, norm_none, w_rc, W.b_router, D.tokens, h, E, D.top_k,
+      D.d_shared > 0 ? 1 : 0, nullptr, idx, gates, sgate, nullptr);
+  CK(cudaGetLastError());
+  g_prof.launches += 2;
+  return REVFFN_OK;
+}
+
 }  // namespace revffn
 
 using namespace revffn;
@@ -665,6 +705,7 @@ const char* revffn_strerror(int code) {
     case REVFFN_ERR_CUDA: return "CUDA call failed";
     case REVFFN_ERR_DEVICE_WAIT: return "a bounded device-side wait expired";
     case REVFFN_ERR_UNSUPPORTED: return "not supported";
+    case REVFFN_ERR_NOALLOC_LIMIT: return "problem exceeds the fixed scratch of the no-allocation entry point";
     default: return "unknown error";
   }
 }
@@ -727,6 +768,28 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
     CK(cudaMemcpyAsync(dy1_host, dy1, n, cudaMemcpyDeviceToHost, st));
   }
   return REVFFN_OK;
+}
+
+int revffn_moe_route_noalloc(const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1,
+                             int32_t* topk_idx_out, float* gates_out, float* sgate_out, void* cuda_stream) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  r = validate_weights(*desc, w);
+  if (r != REVFFN_OK) return r;
+  if (desc->tokens > 0 && (!y1 || !topk_idx_out || !gates_out || !sgate_out)) return REVFFN_ERR_NULL;
+  if (!aligned16(y1) || !aligned16(topk_idx_out)) return REVFFN_ERR_ALIGN;
+  const int64_t need = (int64_t)(desc->n_experts + 1) * (desc->d_model / 2);
+  if (need > REVFFN_ROUTE_NOALLOC_MAX_ELEMS || router_smem_bytes(desc->n_experts) > 48 * 1024)
+    return REVFFN_ERR_NOALLOC_LIMIT;
+  r = check_device();
+  if (r != REVFFN_OK) return r;
+  if (desc->tokens == 0) return REVFFN_OK;
+  double* scratch = route_scratch_ptr(&r);     // first call on a device resolves the array's address
+  if (r != REVFFN_OK) return r;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (desc->weight_dtype == REVFFN_BF16)
+    return route_noalloc_launch<bf16>(*desc, *w, y1, scratch, topk_idx_out, gates_out, sgate_out, st);
+  return route_noalloc_launch<float>(*desc, *w, y1, scratch, topk_idx_out, gates_out, sgate_out, st);
 }
 
 int revffn_prof_enable(int on) {
