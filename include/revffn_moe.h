@@ -66,6 +66,21 @@ enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                
 
 /* flags */
 #define REVFFN_FLAG_FORCE_SIMT 1u  /* run bf16 GEMMs on the plain CUDA-core kernels (cross-check) */
+/* Sharing one evaluation of the branch between two passes.  In a reversible stack the
+ * backward sweep visits a block twice with the same y1: first the inverse pass (Sec. 3.1)
+ * to recover x2, then the gradient pass, which by the method recomputes the branch's
+ * intermediates.  Both evaluate MLP(Norm(y1)); with these two flags the second call reads
+ * what the first one left in the workspace instead of computing it again.  The same pair
+ * of flags gives the activation-caching variant that the reversible design is compared
+ * against: forward with SAVE into a workspace kept per block, backward with REUSE.
+ *   SAVE_ACTIVATIONS   forward / inverse: ws must hold bwd_bytes; the SwiGLU
+ *                      pre-activations are kept next to the other intermediates.
+ *   REUSE_ACTIVATIONS  backward: ws still holds everything a forward / inverse call with
+ *                      SAVE_ACTIVATIONS wrote for the same y1, weights and descriptor; the
+ *                      recomputation is skipped.  The backward pass overwrites some of it,
+ *                      so one saved evaluation serves one backward call.               */
+#define REVFFN_FLAG_SAVE_ACTIVATIONS 2u
+#define REVFFN_FLAG_REUSE_ACTIVATIONS 4u
 
 /*
  * Block descriptor.  Shape constraints (else REVFFN_ERR_SHAPE):
@@ -166,8 +181,9 @@ const char* revffn_strerror(int code);
 /*
  * One whole step of the path with HOST-resident streams: copies y1, x2 and dy2
  * (host, [T, h] packed, ideally pinned) to the device, runs forward (Eq. 2),
- * inverse (Sec. 3.1) and backward (dy1 starting from zero), and copies y2, the
- * reconstructed x2 and dy1 back to the host buffers.  `staging` is caller-owned
+ * inverse (Sec. 3.1) and backward (dy1 starting from zero; it reuses the branch
+ * evaluation of the inverse pass, REVFFN_FLAG_SAVE/REUSE_ACTIVATIONS), and copies y2,
+ * the reconstructed x2 and dy1 back to the host buffers.  `staging` is caller-owned
  * device memory of at least 6 * round_up(T*h*4, 256) bytes, 256-byte aligned;
  * requires ld_stream == h.  Asynchronous on the stream like the other entry
  * points: synchronise the stream before reading the host outputs.

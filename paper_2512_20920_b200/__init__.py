@@ -11,7 +11,8 @@ import importlib
 __all__ = ["Block", "Desc", "Grads", "Weights", "lib", "revffn_moe_backward", "revffn_moe_forward",
            "revffn_moe_inverse", "revffn_moe_status", "revffn_moe_workspace_size", "revffn_strerror",
            "revffn_moe_step_host", "revffn_moe_route_noalloc", "revffn_prof_enable", "revffn_prof_launches",
-           "revffn_prof_collect", "RevffnError", "BF16", "F32", "NORM_RMS", "NORM_NONE", "FLAG_FORCE_SIMT"]
+           "revffn_prof_collect", "RevffnError", "BF16", "F32", "NORM_RMS", "NORM_NONE", "FLAG_FORCE_SIMT",
+           "FLAG_SAVE_ACTIVATIONS", "FLAG_REUSE_ACTIVATIONS"]
 
 
 def __getattr__(name):

@@ -16,6 +16,8 @@ _LIB_PATH = os.path.join(_HERE, "librevffn_moe.so")
 F32, BF16 = 0, 1
 NORM_RMS, NORM_NONE = 0, 1
 FLAG_FORCE_SIMT = 1
+FLAG_SAVE_ACTIVATIONS = 2
+FLAG_REUSE_ACTIVATIONS = 4
 
 WEIGHT_NAMES = ("norm_gamma", "w_up", "w_down", "w_router", "b_router", "w_gate", "w_upx", "w_downx",
                 "ws_gate", "ws_up", "ws_down", "ws_sgate")
@@ -218,26 +220,39 @@ class Block:
     def tokens(self) -> int:
         return self.desc.tokens
 
-    def forward(self, y1, x2, y2=None, topk_idx_out=None):
+    def _desc(self, extra_flags: int) -> Desc:
+        if not extra_flags:
+            return self.desc
+        d = Desc()
+        C.memmove(C.byref(d), C.byref(self.desc), C.sizeof(Desc))
+        d.flags = self.desc.flags | extra_flags
+        return d
+
+    def forward(self, y1, x2, y2=None, topk_idx_out=None, save: bool = False, ws=None):
+        """save=True keeps the branch's intermediates for a later backward(reuse=True)."""
         if y2 is None:
             y2 = torch.empty_like(x2)
-        revffn_moe_forward(self.desc, self.w, y1, x2, y2, topk_idx_out, self.ws)
+        revffn_moe_forward(self._desc(FLAG_SAVE_ACTIVATIONS if save else 0), self.w, y1, x2, y2, topk_idx_out,
+                           self.ws if ws is None else ws)
         return y2
 
-    def inverse(self, y1, y2, x2=None, topk_idx_in=None):
+    def inverse(self, y1, y2, x2=None, topk_idx_in=None, save: bool = False, ws=None):
         if x2 is None:
             x2 = torch.empty_like(y2)
-        revffn_moe_inverse(self.desc, self.w, y1, y2, x2, topk_idx_in, self.ws)
+        revffn_moe_inverse(self._desc(FLAG_SAVE_ACTIVATIONS if save else 0), self.w, y1, y2, x2, topk_idx_in,
+                           self.ws if ws is None else ws)
         return x2
 
     def backward(self, y1, dy2, dy1_inout, grads: Optional[Dict[str, torch.Tensor]] = None, accumulate: bool = False,
-                 topk_idx_in=None):
+                 topk_idx_in=None, reuse: bool = False, ws=None):
+        """reuse=True: the workspace still holds what forward/inverse(save=True) left for this y1."""
         grads = grads or {}
         for n, t in grads.items():
             if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
                 raise ValueError(f"gradient {n}: need a contiguous fp32 CUDA tensor")
         g = Grads(**{n: _ptr(grads.get(n)) for n in WEIGHT_NAMES}, accumulate=1 if accumulate else 0)
-        revffn_moe_backward(self.desc, self.w, y1, dy2, dy1_inout, g, topk_idx_in, self.ws)
+        revffn_moe_backward(self._desc(FLAG_REUSE_ACTIVATIONS if reuse else 0), self.w, y1, dy2, dy1_inout, g,
+                            topk_idx_in, self.ws if ws is None else ws)
         return dy1_inout
 
     def grads_struct(self, grads: Optional[Dict[str, torch.Tensor]] = None, accumulate: bool = False) -> Grads:

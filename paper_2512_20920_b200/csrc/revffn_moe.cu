@@ -256,21 +256,15 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
 
   // Router: fold through P_up, logits, top-k, gates
   {
-    dim3 grid((unsigned)ceil_div(h, 128), (unsigned)(E + 1));
     { ProfScope ps(TG_FOLD, st);
-    fold_router_kernel<T><<<grid, 128, 0, st>>>(reinterpret_cast<const T*>(c.W.w_router),
-                                                 reinterpret_cast<const T*>(c.W.ws_sgate), w_up, E, d, h,
-                                                 c.template p<double>(L.w_rc));
+    CK(launch_fold_router<T>(reinterpret_cast<const T*>(c.W.w_router), reinterpret_cast<const T*>(c.W.ws_sgate), w_up, E,
+                             d, h, c.template p<double>(L.w_rc), st));
     }
-    CK(cudaGetLastError());
-    size_t smem = router_smem_bytes(E);
     { ProfScope ps(TG_ROUTER, st);
-    router_topk_kernel<<<(unsigned)ceil_div(Tn, RT_TOK), 256, smem, st>>>(
-        y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, c.template p<double>(L.w_rc), c.W.b_router, Tn, h,
-        E, k, Is > 0 ? 1 : 0, idx_in, c.template p<int32_t>(L.idx), c.template p<float>(L.gates),
-        c.template p<float>(L.sgate), idx_user);
+    CK(launch_router_topk(y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, c.template p<double>(L.w_rc),
+                          c.W.b_router, Tn, h, E, k, Is > 0 ? 1 : 0, idx_in, c.template p<int32_t>(L.idx),
+                          c.template p<float>(L.gates), c.template p<float>(L.sgate), idx_user, st));
     }
-    CK(cudaGetLastError());
   }
 
   // Permutation maps
@@ -393,7 +387,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
   cudaStream_t st = c.st;
   const int Rp = (int)L.rows_pad;
 
-  CKR(run_branch(c, y1, idx_in, nullptr, true));
+  if (!(D.flags & REVFFN_FLAG_REUSE_ACTIVATIONS)) CKR(run_branch(c, y1, idx_in, nullptr, true));
 
   auto wgrad = [&](int tag, float* out, int M, int N, const void* A, int64_t lda, int a_col0, const void* B, int64_t ldb,
                    bool grouped, int64_t cstride) -> int {
@@ -583,7 +577,7 @@ static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weight
   CK(cudaMemsetAsync(c.ws + L.status.off, 0, L.status.bytes, st));
   if (D.tokens == 0) return REVFFN_OK;   // empty batch: nothing to compute, gradients untouched
   if (pass == PASS_BWD) return run_backward(c, y1, in2, out, *G, idx_in);
-  CKR(run_branch(c, y1, idx_in, idx_out, false));
+  CKR(run_branch(c, y1, idx_in, idx_out, (D.flags & REVFFN_FLAG_SAVE_ACTIVATIONS) != 0));
   return run_couple(c, in2, pass == PASS_FWD ? 1.f : -1.f, out);
 }
 
@@ -606,7 +600,8 @@ static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weight
       if (g && !aligned16(g)) return REVFFN_ERR_ALIGN;
   }
   WsLayout L = plan_workspace(*desc);
-  if (ws_bytes < (pass == PASS_BWD ? L.bwd_bytes : L.fwd_bytes)) return REVFFN_ERR_WORKSPACE;
+  const bool big_ws = pass == PASS_BWD || (desc->flags & REVFFN_FLAG_SAVE_ACTIVATIONS);
+  if (ws_bytes < (big_ws ? L.bwd_bytes : L.fwd_bytes)) return REVFFN_ERR_WORKSPACE;
   CKR(check_device());
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (desc->weight_dtype == REVFFN_BF16)
@@ -641,15 +636,10 @@ static int route_noalloc_launch(const revffn_moe_desc& D, const revffn_moe_weigh
                                 double* w_rc, int32_t* idx, float* gates, float* sgate, cudaStream_t st) {
   const int d = D.d_model, h = d / 2, E = D.n_experts;
   const int norm_none = D.norm_kind == REVFFN_NORM_NONE;
-  dim3 grid((unsigned)ceil_div(h, 128), (unsigned)(E + 1));
-  fold_router_kernel<T><<<grid, 128, 0, st>>>(reinterpret_cast<const T*>(W.w_router),
-                                               reinterpret_cast<const T*>(W.ws_sgate),
-                                               reinterpret_cast<const T*>(W.w_up), E, d, h, w_rc);
-  CK(cudaGetLastError());
-  router_topk_kernel<<<(unsigned)ceil_div(D.tokens, RT_TOK), 256, router_smem_bytes(E), st>>>(
-      y1, D.ld_stream, W.norm_gamma, D.norm_eps, norm_none, w_rc, W.b_router, D.tokens, h, E, D.top_k,
-      D.d_shared > 0 ? 1 : 0, nullptr, idx, gates, sgate, nullptr);
-  CK(cudaGetLastError());
+  CK(launch_fold_router<T>(reinterpret_cast<const T*>(W.w_router), reinterpret_cast<const T*>(W.ws_sgate),
+                           reinterpret_cast<const T*>(W.w_up), E, d, h, w_rc, st));
+  CK(launch_router_topk(y1, D.ld_stream, W.norm_gamma, D.norm_eps, norm_none, w_rc, W.b_router, D.tokens, h, E,
+                        D.top_k, D.d_shared > 0 ? 1 : 0, nullptr, idx, gates, sgate, nullptr, st));
   g_prof.launches += 2;
   return REVFFN_OK;
 }
@@ -759,9 +749,13 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
     CK(cudaMemcpyAsync(dy2, dy2_host, n, cudaMemcpyHostToDevice, st));
     CK(cudaMemsetAsync(dy1, 0, n, st));
   }
+  // the inverse and the gradient pass share one evaluation of the branch
+  revffn_moe_desc d_inv = *desc, d_bwd = *desc;
+  d_inv.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS;
+  d_bwd.flags |= REVFFN_FLAG_REUSE_ACTIVATIONS;
   CKR(revffn_moe_forward(desc, w, y1, x2, y2, nullptr, ws, ws_bytes, cuda_stream));
-  CKR(revffn_moe_inverse(desc, w, y1, y2, x2r, nullptr, ws, ws_bytes, cuda_stream));
-  CKR(revffn_moe_backward(desc, w, y1, dy2, dy1, grads, nullptr, ws, ws_bytes, cuda_stream));
+  CKR(revffn_moe_inverse(&d_inv, w, y1, y2, x2r, nullptr, ws, ws_bytes, cuda_stream));
+  CKR(revffn_moe_backward(&d_bwd, w, y1, dy2, dy1, grads, nullptr, ws, ws_bytes, cuda_stream));
   if (n > 0) {
     CK(cudaMemcpyAsync(y2_host, y2, n, cudaMemcpyDeviceToHost, st));
     CK(cudaMemcpyAsync(x2_rec_host, x2r, n, cudaMemcpyDeviceToHost, st));
@@ -779,7 +773,7 @@ int revffn_moe_route_noalloc(const revffn_moe_desc* desc, const revffn_moe_weigh
   if (desc->tokens > 0 && (!y1 || !topk_idx_out || !gates_out || !sgate_out)) return REVFFN_ERR_NULL;
   if (!aligned16(y1) || !aligned16(topk_idx_out)) return REVFFN_ERR_ALIGN;
   const int64_t need = (int64_t)(desc->n_experts + 1) * (desc->d_model / 2);
-  if (need > REVFFN_ROUTE_NOALLOC_MAX_ELEMS || router_smem_bytes(desc->n_experts) > 48 * 1024)
+  if (need > REVFFN_ROUTE_NOALLOC_MAX_ELEMS || router_smem_bytes(desc->n_experts) > 200 * 1024)
     return REVFFN_ERR_NOALLOC_LIMIT;
   r = check_device();
   if (r != REVFFN_OK) return r;

@@ -54,34 +54,121 @@ __global__ void rmsnorm_fwd_kernel(const float* __restrict__ y, int64_t ld, cons
 // fp64 accumulation and output, so that logits = W_rc * n differ from the
 // two-step definition only by fp64 rounding and the routing decision is
 // reproducible against a higher-precision reference.
+// Block = FD_I columns i x FD_E rows e x FD_S slices of j (512 threads).  W_up is staged
+// through shared memory in chunks of FD_J rows (16-byte loads, the next chunk in flight
+// while the current one is summed); the rows' weights are staged as doubles.  A thread
+// owns one column, one slice (FD_J / FD_S consecutive j of every chunk) and FD_E
+// accumulators; the slices are added in ascending order at the end (fixed order).
 // ---------------------------------------------------------------------------
+constexpr int FD_E = 4;     // rows of W_r' per block
+constexpr int FD_J = 64;    // j-chunk staged per iteration
+constexpr int FD_I = 128;   // columns per block
+constexpr int FD_S = 4;     // j-slices per chunk
+constexpr int FD_THREADS = FD_I * FD_S;
+
 template <typename T>
-__global__ void fold_router_kernel(const T* __restrict__ w_router, const T* __restrict__ w_sgate,
-                                   const T* __restrict__ w_up, int E, int d, int h,
-                                   double* __restrict__ w_rc) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  int e = blockIdx.y;
-  if (i >= h) return;
-  const T* wr = (e < E) ? (w_router + (int64_t)e * d) : w_sgate;
-  double acc = 0.0;
-  if (wr != nullptr) {
-    for (int j = 0; j < d; ++j) acc += (double)to_f32(wr[j]) * (double)to_f32(w_up[(int64_t)j * h + i]);
+__global__ void __launch_bounds__(FD_THREADS)
+fold_router_kernel(const T* __restrict__ w_router, const T* __restrict__ w_sgate,
+                   const T* __restrict__ w_up, int E, int d, int h, double* __restrict__ w_rc) {
+  constexpr int PER16 = 16 / (int)sizeof(T);                  // elements per 16-byte piece
+  constexpr int ROW_PIECES = FD_I / PER16;                    // pieces per staged row
+  constexpr int N_PIECES = FD_J * ROW_PIECES / FD_THREADS;    // pieces per thread and chunk
+  constexpr int SL = FD_J / FD_S;                             // rows per slice
+  __shared__ __align__(16) double wr_s[FD_J][FD_E];
+  __shared__ __align__(16) T up_s[FD_J][FD_I];
+  static_assert(sizeof(T) * FD_J * FD_I >= sizeof(double) * FD_S * FD_E * FD_I, "slice sums reuse the W_up stage");
+  double (*red)[FD_E][FD_I] = reinterpret_cast<double (*)[FD_E][FD_I]>(&up_s[0][0]);   // used after the last chunk
+  const int tid = threadIdx.x;
+  const int col = tid % FD_I, sl = tid / FD_I;
+  const int i0 = blockIdx.x * FD_I;
+  const int e0 = blockIdx.y * FD_E;
+  double acc[FD_E];
+#pragma unroll
+  for (int a = 0; a < FD_E; ++a) acc[a] = 0.0;
+
+  uint4 pre[N_PIECES];
+  float pre_w = 0.f;
+  auto prefetch = [&](int j0) {
+#pragma unroll
+    for (int q = 0; q < N_PIECES; ++q) {
+      int piece = tid + q * FD_THREADS;
+      int jj = piece / ROW_PIECES, c = (piece % ROW_PIECES) * PER16;
+      pre[q] = make_uint4(0u, 0u, 0u, 0u);
+      if (j0 + jj < d && i0 + c < h)      // h is a multiple of 8: a piece never straddles the edge
+        pre[q] = *reinterpret_cast<const uint4*>(w_up + (int64_t)(j0 + jj) * h + i0 + c);
+    }
+    if (tid < FD_E * FD_J) {
+      int ee = tid / FD_J, jj = tid % FD_J;
+      int e = e0 + ee, j = j0 + jj;
+      const T* src = (e < E) ? (w_router + (int64_t)e * d) : (e == E ? w_sgate : nullptr);
+      pre_w = (src != nullptr && j < d) ? to_f32(src[j]) : 0.f;
+    }
+  };
+  prefetch(0);
+  for (int j0 = 0; j0 < d; j0 += FD_J) {
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < N_PIECES; ++q) {
+      int piece = tid + q * FD_THREADS;
+      int jj = piece / ROW_PIECES, c = (piece % ROW_PIECES) * PER16;
+      *reinterpret_cast<uint4*>(&up_s[jj][c]) = pre[q];
+    }
+    if (tid < FD_E * FD_J) wr_s[tid % FD_J][tid / FD_J] = (double)pre_w;
+    __syncthreads();
+    if (j0 + FD_J < d) prefetch(j0 + FD_J);
+#pragma unroll
+    for (int q = 0; q < SL; ++q) {      // rows past d were staged as zeros
+      const int jj = sl * SL + q;
+      double b = (double)to_f32(up_s[jj][col]);
+      const double2* w2 = reinterpret_cast<const double2*>(wr_s[jj]);
+#pragma unroll
+      for (int a = 0; a < FD_E / 2; ++a) {
+        double2 w = w2[a];
+        acc[2 * a] += w.x * b;
+        acc[2 * a + 1] += w.y * b;
+      }
+    }
   }
-  w_rc[(int64_t)e * h + i] = acc;
+  __syncthreads();      // every slice has finished reading the stage
+#pragma unroll
+  for (int a = 0; a < FD_E; ++a) red[sl][a][col] = acc[a];
+  __syncthreads();
+  if (sl == 0 && i0 + col < h) {
+#pragma unroll
+    for (int a = 0; a < FD_E; ++a) {
+      double v = red[0][a][col];
+#pragma unroll
+      for (int q = 1; q < FD_S; ++q) v += red[q][a][col];
+      if (e0 + a <= E) w_rc[(int64_t)(e0 + a) * h + i0 + col] = v;
+    }
+  }
+}
+
+template <typename T>
+inline cudaError_t launch_fold_router(const T* w_router, const T* w_sgate, const T* w_up, int E, int d, int h,
+                                      double* w_rc, cudaStream_t st) {
+  dim3 grid((unsigned)ceil_div(h, FD_I), (unsigned)ceil_div(E + 1, FD_E));
+  fold_router_kernel<T><<<grid, FD_THREADS, 0, st>>>(w_router, w_sgate, w_up, E, d, h, w_rc);
+  return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------
 // Router: logits in fp64 from the fp32 stream, top-k by warp shuffles, gates.
 //   block = 256 threads, RT_TOK tokens per block.
-//   phase 1: r per token (fp64) and n = y*r*gamma (fp64) staged chunk-wise
-//   phase 2: L[t, e] = <W_rc[e], n_t> (+ b_r[e]) for e < E; row E is the shared gate
-//   phase 3: per token, k rounds of warp arg-max (ties -> lowest index), softmax
+//   phase 1: L[t, e] = r_t <W_rc[e], y_t * gamma> (+ b_r[e]) for e < E; row E is the
+//            shared gate.  y*gamma (fp64) and W_rc are staged chunk-wise, k-major, so
+//            that a thread reads its 4 tokens and 4 experts with 16-byte loads; every
+//            thread owns a 4 x 4 block of dot products and sums over i in ascending
+//            order.  The staging threads also sum y^2 (fp64), which gives
+//            r_t = (mean(y_t^2)+eps)^-1/2; the scale is applied to the finished sums.
+//   phase 2: per token, k rounds of warp arg-max (ties -> lowest index), softmax
 //            over the k selected logits, sigmoid of the shared-gate logit.
 // idx_in != NULL: expert sets are taken from it (gates are still recomputed).
 // ---------------------------------------------------------------------------
-constexpr int RT_TOK = 32;   // tokens per block
+constexpr int RT_TOK = 64;   // tokens per block
 constexpr int RT_KC = 32;    // k-chunk
 constexpr int RT_EC = 64;    // experts per pass
+constexpr int RT_LD = RT_TOK + 2;   // row stride (doubles) of the staged chunks: even, and not a multiple of 32 banks
 
 __global__ void __launch_bounds__(256)
 router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restrict__ gamma, float eps,
@@ -89,84 +176,118 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
                    int tokens, int h, int E, int k, int has_shared, const int32_t* __restrict__ idx_in,
                    int32_t* __restrict__ idx_out, float* __restrict__ gate_out, float* __restrict__ sgate_out,
                    int32_t* __restrict__ idx_user) {
-  extern __shared__ double smem_d[];
+  extern __shared__ __align__(16) double smem_d[];
   const int EP = E + 1;                       // logits per token incl. the shared-gate row
-  double* Ls = smem_d;                        // [RT_TOK][EP]
-  double* ns = Ls + RT_TOK * EP;              // [RT_TOK][RT_KC + 1]
-  double* ws = ns + RT_TOK * (RT_KC + 1);     // [RT_EC][RT_KC + 1]
-  double* rs = ws + RT_EC * (RT_KC + 1);      // [RT_TOK]
+  double* ns = smem_d;                        // [RT_KC][RT_LD]   n chunk, k-major
+  double* ws = ns + RT_KC * RT_LD;            // [RT_KC][RT_LD]   W_rc chunk, k-major (RT_EC == RT_TOK)
+  double* rs = ws + RT_KC * RT_LD;            // [RT_TOK]
+  double* Ls = rs + RT_TOK;                   // [RT_TOK][EP]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t0 = blockIdx.x * RT_TOK;
 
-  // phase 1: r per token
-  for (int tt = warp; tt < RT_TOK; tt += 8) {
-    int t = t0 + tt;
-    double r = 1.0;
-    if (t < tokens && !norm_none) {
-      const float* row = y + (int64_t)t * ld;
-      double ss = 0.0;
-      for (int i = lane; i < h; i += 32) { double v = (double)row[i]; ss += v * v; }
-      ss = warp_sum(ss);
-      r = 1.0 / sqrt(ss / (double)h + (double)eps);
-    }
-    if (lane == 0) rs[tt] = r;
-  }
-  __syncthreads();
-
-  // phase 2: logits
-  const int tx = tid & 15, ty = tid >> 4;     // 16 x 16 threads: 2 tokens x 4 experts each
+  // phase 1: logits.  16 x 16 threads, each 4 tokens x 4 experts; a warp spans 4 expert
+  // groups x 8 token groups, which keeps its shared-memory reads within few wavefronts.
+  const int tx = (warp & 3) * 4 + (lane & 3);       // expert group: experts e0 + 4 tx .. + 3
+  const int ty = (warp >> 2) * 8 + (lane >> 2);     // token group: tokens 4 ty .. + 3
   for (int e0 = 0; e0 < EP; e0 += RT_EC) {
-    double acc[2][4];
+    double acc[4][4];
 #pragma unroll
-    for (int a = 0; a < 2; ++a)
+    for (int a = 0; a < 4; ++a)
 #pragma unroll
       for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
-    for (int k0 = 0; k0 < h; k0 += RT_KC) {
-      // stage n chunk: RT_TOK x RT_KC
-      for (int idx = tid; idx < RT_TOK * RT_KC; idx += 256) {
-        int tt = idx / RT_KC, kk = idx % RT_KC;
-        int t = t0 + tt, i = k0 + kk;
-        double v = 0.0;
-        if (t < tokens && i < h) {
-          v = (double)y[(int64_t)t * ld + i] * rs[tt];
-          if (gamma && !norm_none) v *= (double)gamma[i];
-        }
-        ns[tt * (RT_KC + 1) + kk] = v;
+    // Register prefetch: the global loads of chunk c+1 are in flight while chunk c is summed.
+    //   y:    RT_TOK x RT_KC floats  = 2 float4 per thread  (token tt, 4 consecutive i)
+    //   W_rc: RT_EC x RT_KC doubles  = 4 double2 per thread (expert ee, 2 consecutive i)
+    float4 py[2];
+    double2 pw[4];
+    double ss[2] = {0.0, 0.0};      // sum of y^2 over this thread's 4-column strip of its two tokens
+    auto prefetch = [&](int k0) {
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        int idx = tid + q * 256;
+        int tt = idx / (RT_KC / 4), kq = (idx % (RT_KC / 4)) * 4;
+        int t = t0 + tt, i = k0 + kq;
+        py[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (t < tokens && i < h) py[q] = *reinterpret_cast<const float4*>(y + (int64_t)t * ld + i);   // h % 4 == 0
       }
-      for (int idx = tid; idx < RT_EC * RT_KC; idx += 256) {
-        int ee = idx / RT_KC, kk = idx % RT_KC;
-        int e = e0 + ee, i = k0 + kk;
-        ws[ee * (RT_KC + 1) + kk] = (e < EP && i < h) ? w_rc[(int64_t)e * h + i] : 0.0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        int idx = tid + q * 256;
+        int ee = idx / (RT_KC / 2), kq = (idx % (RT_KC / 2)) * 2;
+        int e = e0 + ee, i = k0 + kq;
+        pw[q] = make_double2(0.0, 0.0);
+        if (e < EP && i < h) pw[q] = *reinterpret_cast<const double2*>(w_rc + (int64_t)e * h + i);   // h % 2 == 0
+      }
+    };
+    prefetch(0);
+    for (int k0 = 0; k0 < h; k0 += RT_KC) {
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        int idx = tid + q * 256;
+        int tt = idx / (RT_KC / 4), kq = (idx % (RT_KC / 4)) * 4;
+        int i = k0 + kq;
+        float4 g = make_float4(1.f, 1.f, 1.f, 1.f);
+        if (gamma && !norm_none && i < h) g = *reinterpret_cast<const float4*>(gamma + i);
+        const double v0 = (double)py[q].x, v1 = (double)py[q].y, v2 = (double)py[q].z, v3 = (double)py[q].w;
+        ss[q] += v0 * v0; ss[q] += v1 * v1; ss[q] += v2 * v2; ss[q] += v3 * v3;
+        ns[(kq + 0) * RT_LD + tt] = v0 * (double)g.x;
+        ns[(kq + 1) * RT_LD + tt] = v1 * (double)g.y;
+        ns[(kq + 2) * RT_LD + tt] = v2 * (double)g.z;
+        ns[(kq + 3) * RT_LD + tt] = v3 * (double)g.w;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        int idx = tid + q * 256;
+        int ee = idx / (RT_KC / 2), kq = (idx % (RT_KC / 2)) * 2;
+        ws[(kq + 0) * RT_LD + ee] = pw[q].x;
+        ws[(kq + 1) * RT_LD + ee] = pw[q].y;
       }
       __syncthreads();
-#pragma unroll 4
-      for (int kk = 0; kk < RT_KC; ++kk) {
-        double nv0 = ns[(ty * 2 + 0) * (RT_KC + 1) + kk];
-        double nv1 = ns[(ty * 2 + 1) * (RT_KC + 1) + kk];
+      if (k0 + RT_KC < h) prefetch(k0 + RT_KC);
+      // operands of step kk+1 are read from shared memory before the sums of step kk are issued
+      const double2* n2 = reinterpret_cast<const double2*>(ns + ty * 4);
+      const double2* w2 = reinterpret_cast<const double2*>(ws + tx * 4);
+      double2 n01 = n2[0], n23 = n2[1], w01 = w2[0], w23 = w2[1];
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          double wv = ws[(tx * 4 + b) * (RT_KC + 1) + kk];
-          acc[0][b] += nv0 * wv;
-          acc[1][b] += nv1 * wv;
+      for (int kk = 0; kk < RT_KC; ++kk) {
+        const double nv[4] = {n01.x, n01.y, n23.x, n23.y};
+        const double wv[4] = {w01.x, w01.y, w23.x, w23.y};
+        if (kk + 1 < RT_KC) {
+          n01 = n2[(kk + 1) * (RT_LD / 2)]; n23 = n2[(kk + 1) * (RT_LD / 2) + 1];
+          w01 = w2[(kk + 1) * (RT_LD / 2)]; w23 = w2[(kk + 1) * (RT_LD / 2) + 1];
         }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int b = 0; b < 4; ++b) acc[a][b] += nv[a] * wv[b];
       }
       __syncthreads();
     }
+    // r per token: the 8 threads that staged one token hold its strips (lanes 8m .. 8m+7)
 #pragma unroll
-    for (int a = 0; a < 2; ++a)
+    for (int q = 0; q < 2; ++q) {
+      double v = ss[q];
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      v += __shfl_xor_sync(0xffffffffu, v, 2);
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      if ((tid & 7) == 0) rs[tid / 8 + q * 32] = norm_none ? 1.0 : 1.0 / sqrt(v / (double)h + (double)eps);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
         int e = e0 + tx * 4 + b;
         if (e < EP) {
-          double v = acc[a][b];
+          double v = acc[a][b] * rs[ty * 4 + a];
           if (e < E && b_router) v += (double)b_router[e];
-          Ls[(ty * 2 + a) * EP + e] = v;
+          Ls[(ty * 4 + a) * EP + e] = v;
         }
       }
   }
   __syncthreads();
 
-  // phase 3: top-k and gates; one warp per token, 4 tokens per warp
+  // phase 2: top-k and gates; one warp per token, 8 tokens per warp
   for (int tt = warp; tt < RT_TOK; tt += 8) {
     int t = t0 + tt;
     if (t >= tokens) continue;
@@ -215,7 +336,32 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
 }
 
 inline size_t router_smem_bytes(int E) {
-  return sizeof(double) * ((size_t)RT_TOK * (E + 1) + RT_TOK * (RT_KC + 1) + RT_EC * (RT_KC + 1) + RT_TOK);
+  return sizeof(double) * ((size_t)2 * RT_KC * RT_LD + RT_TOK + (size_t)RT_TOK * (E + 1));
+}
+
+// Raises the kernel's dynamic shared-memory limit when the logits of a block do not
+// fit the default 48 KB (once per device), then launches.
+inline cudaError_t launch_router_topk(const float* y, int64_t ld, const float* gamma, float eps, int norm_none,
+                                      const double* w_rc, const float* b_router, int tokens, int h, int E, int k,
+                                      int has_shared, const int32_t* idx_in, int32_t* idx_out, float* gate_out,
+                                      float* sgate_out, int32_t* idx_user, cudaStream_t st) {
+  static size_t raised[64] = {0};
+  const size_t smem = router_smem_bytes(E);
+  if (smem > 48 * 1024) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (raised[dev] < smem) {
+      e = cudaFuncSetAttribute(router_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      raised[dev] = smem;
+    }
+  }
+  router_topk_kernel<<<(unsigned)ceil_div(tokens, RT_TOK), 256, smem, st>>>(
+      y, ld, gamma, eps, norm_none, w_rc, b_router, tokens, h, E, k, has_shared, idx_in, idx_out, gate_out,
+      sgate_out, idx_user);
+  return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------

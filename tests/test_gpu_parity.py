@@ -217,3 +217,33 @@ def test_tensor_core_and_cuda_core_backends_agree(rv):
         if n == "y2":
             a, b = a - s["x2"], b - s["x2"]
         assert rel_l2(a, b) <= 5e-3, n
+
+
+@pytest.mark.parametrize("simt", [True, False])
+def test_backward_reuses_a_saved_evaluation(rv, simt):
+    """A backward pass that reads the intermediates a forward or inverse call left in the
+    workspace gives bit for bit what the recomputing backward pass gives."""
+    cfg = small_cfg(tokens=333, n_experts=8, top_k=3)
+    w, s = scaled_weights(cfg, 7, 4.0), make_streams(cfg, 7)
+    blk = make_block(cfg, w, flags=rv.FLAG_FORCE_SIMT if simt else 0)
+    y1, x2, dy2 = dev(s["y1"]), dev(s["x2"]), dev(s["dy2"])
+    y2 = blk.forward(y1, x2)
+    x2_plain = blk.inverse(y1, y2)
+    dy1_plain, g_plain = torch.zeros_like(y1), grad_buffers(cfg, w)
+    blk.backward(y1, dy2, dy1_plain, g_plain)
+    for first in ("inverse", "forward"):
+        if first == "inverse":
+            x2_rec = blk.inverse(y1, y2, save=True)
+            assert torch.equal(x2_rec, x2_plain)
+        else:
+            assert torch.equal(blk.forward(y1, x2, save=True), y2)
+        dy1, g = torch.zeros_like(y1), grad_buffers(cfg, w)
+        blk.backward(y1, dy2, dy1, g, reuse=True)
+        assert blk.status() == 0
+        assert torch.equal(dy1, dy1_plain), first
+        for n in g:
+            assert torch.equal(g[n], g_plain[n]), (first, n)
+    # a workspace of forward size is refused when the intermediates are to be kept
+    small = torch.empty(blk.fwd_bytes, dtype=torch.uint8, device="cuda")
+    with pytest.raises(rv.RevffnError):
+        blk.forward(y1, x2, save=True, ws=small)
