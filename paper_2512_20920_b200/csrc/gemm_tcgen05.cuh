@@ -11,7 +11,10 @@
 //               releases stages and publishes finished accumulators.
 //   warps 2..5  epilogue: tcgen05.ld the accumulator (lane = tile row), apply the
 //               fused epilogue (SwiGLU, gate scale, coupling add/sub, SwiGLU
-//               backward, fp32 weight-gradient store) and write global memory.
+//               backward, fp32 weight-gradient store), stage 32 x 32 output blocks in
+//               swizzled shared memory and hand them to TMA bulk tensor stores
+//               (reduce-add when a gradient is accumulated), so that global
+//               writes are whole lines whatever the row stride.
 // Tile = 128 rows x MMA_N columns, K step 64 (one 128-byte swizzle atom of bf16).
 // Both operands may be K-major or MN-major; MN-major tiles are fetched as
 // 64x64 boxes and described to the tensor core with leading/stride offsets.
@@ -19,6 +22,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <cstring>
 #include <type_traits>
 
 #include "common.cuh"
@@ -32,12 +36,19 @@ constexpr int TC_THREADS = 192;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
 constexpr long long TC_WAIT_CYCLES = 4000000000LL;       // ~2 s: bound on any single wait
 
+constexpr int TC_EPI_WARP_BYTES = 8192;                  // output staging per epilogue warp
+constexpr int TC_EPI_BYTES = 4 * TC_EPI_WARP_BYTES;
+
 template <int MMA_N> struct TcCfg {
   static constexpr int B_BYTES = MMA_N * TC_BK * 2;
   static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
   static constexpr int STAGES = (MMA_N == 256) ? 4 : 6;
   static constexpr int TMEM_COLS = 2 * MMA_N;           // 512 or 256: power of two >= 32
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+  // stage ring | epilogue staging | barriers; the ring starts 1024-byte aligned and
+  // every stage is a multiple of 1024 bytes, so the staging area is aligned too
+  static constexpr int EPI_OFF = STAGES * STAGE_BYTES;
+  static constexpr int BAR_OFF = EPI_OFF + TC_EPI_BYTES;
+  static constexpr int SMEM_BYTES = BAR_OFF + 1024 /*align*/ + 256 /*barriers*/;
 };
 
 struct TcParams {
@@ -95,6 +106,25 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+
+// Shared -> global bulk tensor store of one box (the box and the swizzle come from the map).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(src) : "memory");
+}
+// Same box added element-wise (fp32) to what global memory holds.
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Wait until at most N of this thread's bulk groups still read their shared-memory source.
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Orders this thread's shared-memory writes before later async-proxy (TMA) reads of them.
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -164,6 +194,23 @@ __device__ __forceinline__ void load32_bf16(const bf16* src, float* f) {
   for (int i = 0; i < 4; ++i) unpack8(s[i], f + 8 * i);
 }
 
+// Output staging.  A warp stages a 32-row x 32-column block, one row per lane, in the
+// layout the store's tensor map expects: rows of 128 bytes (fp32) under the 128-byte
+// swizzle, rows of 64 bytes (bf16) under the 64-byte swizzle.  `buf` is aligned to the
+// swizzle period, so the 16-byte piece j of row r lands at piece j ^ (r & 7), or
+// j ^ ((r >> 1) & 3); lanes of one store instruction then hit distinct banks.
+__device__ __forceinline__ void stage32_f32(uint8_t* buf, int r, const float* f) {
+  uint8_t* row = buf + r * 128;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    *reinterpret_cast<float4*>(row + ((j ^ (r & 7)) << 4)) = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+}
+__device__ __forceinline__ void stage32_bf16(uint8_t* buf, int r, const float* f) {
+  uint8_t* row = buf + r * 64;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(row + ((j ^ ((r >> 1) & 3)) << 4)) = pack8(f + 8 * j);
+}
+
 // Tile coordinates shared by the three roles.
 struct TcTile {
   int m0, n0, group, k_blocks, krow0;
@@ -201,19 +248,20 @@ __device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_
 template <int MMA_N, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUtensorMap map_a,
-               const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1) {
+               const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
+               const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c1) {
   using Cfg = TcCfg<MMA_N>;
   extern __shared__ uint8_t smem_raw[];
   const GemmProblem& p = P.p;
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;                 // stage ring, 1024-byte aligned
   uint8_t* gen_base = smem_raw + (base - raw);
-  const uint32_t bars = base + Cfg::STAGES * Cfg::STAGE_BYTES;  // barrier block
+  const uint32_t bars = base + Cfg::BAR_OFF;                    // barrier block
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (Cfg::STAGES + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + 2 + a); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + Cfg::STAGES * Cfg::STAGE_BYTES + 8 * (2 * Cfg::STAGES + 4));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + Cfg::BAR_OFF + 8 * (2 * Cfg::STAGES + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* issued = reinterpret_cast<int*>(tmem_slot + 2);   // [STAGES] parity+1 of the last load issued per stage
 
@@ -329,8 +377,11 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int q = warp & 3;                      // TMEM lane quadrant this warp may access
     const int row_in_tile = q * 32 + lane;
+    uint8_t* stg = gen_base + Cfg::EPI_OFF + q * TC_EPI_WARP_BYTES;   // this warp's staging area
+    const uint32_t stg_u32 = base + Cfg::EPI_OFF + q * TC_EPI_WARP_BYTES;
     bool ok = true;
     int it = 0;
+    uint32_t n_grp = 0;                          // bulk groups committed so far (same in every lane)
     for (int w = blockIdx.x; ok; w += gridDim.x, ++it) {
       TcTile t = tc_tile(P, w, tiles_m_dev);
       if (!t.valid) break;
@@ -342,6 +393,9 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       const int m = t.m0 + row_in_tile;
       const int m_lim = (p.group_mode == GROUP_M) ? tiles_m_dev * TC_BM : p.M;
       const bool m_ok = m < m_lim;
+      const bool slab_ok = t.m0 + q * 32 < m_lim;             // this warp's 32 rows hold at least one real row
+      // row coordinate of the slab in the output tensor map (rows past its extent are clipped by the store)
+      const int y0 = (p.group_mode == GROUP_K ? t.group * p.M : 0) + t.m0 + q * 32;
       const bool have_acc = t.k_blocks > 0;      // an empty K range leaves the accumulator undefined: use zeros
       uint32_t r0[32];
       float f[32];
@@ -349,69 +403,82 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       if constexpr (EPI == EPI_STORE || EPI == EPI_ROWSCALE || EPI == EPI_COUPLE || EPI == EPI_WGRAD) {
         float rs = 1.f;
         if (EPI == EPI_ROWSCALE && m_ok) rs = p.rowscale[m];
+        const bool f32_out = (EPI == EPI_COUPLE) || (EPI == EPI_WGRAD) || (EPI == EPI_STORE && p.out_f32);
 #pragma unroll 1
         for (int c = 0; c < MMA_N; c += 32) {
+          const int n = t.n0 + c;
+          if (!slab_ok || n >= p.N) continue;      // warp-uniform
           if (have_acc) { tmem_ld32(taddr + c, r0); tmem_ld_wait(); }
 #pragma unroll
           for (int i = 0; i < 32; ++i) f[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
-          const int n = t.n0 + c;
-          if (!m_ok || n >= p.N) continue;
-          if constexpr (EPI == EPI_STORE) {
-            if (p.out_f32) {
-              float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (int64_t)m * p.ldc + n);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) o[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
-            } else {
-              store32_bf16(reinterpret_cast<bf16*>(p.C) + (int64_t)m * p.ldc + n, f);
-            }
-          } else if constexpr (EPI == EPI_ROWSCALE) {
+          if constexpr (EPI == EPI_ROWSCALE) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) f[i] *= rs;
-            store32_bf16(reinterpret_cast<bf16*>(p.C) + (int64_t)m * p.ldc + n, f);
           } else if constexpr (EPI == EPI_COUPLE) {
-            const float4* x = reinterpret_cast<const float4*>(p.resid + (int64_t)m * p.ld_resid + n);
-            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (int64_t)m * p.ldc + n);
+            if (m_ok) {
+              const float4* x = reinterpret_cast<const float4*>(p.resid + (int64_t)m * p.ld_resid + n);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              float4 xv = x[i];
-              o[i] = make_float4(xv.x + p.resid_sign * f[4 * i], xv.y + p.resid_sign * f[4 * i + 1],
-                                 xv.z + p.resid_sign * f[4 * i + 2], xv.w + p.resid_sign * f[4 * i + 3]);
-            }
-          } else {   // EPI_WGRAD
-            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (int64_t)t.group * p.c_group_stride +
-                                                  (int64_t)m * p.ldc + n);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              float4 v = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
-              if (p.accumulate) { float4 old = o[i]; v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w; }
-              o[i] = v;
+              for (int i = 0; i < 8; ++i) {
+                float4 xv = x[i];
+                f[4 * i] = xv.x + p.resid_sign * f[4 * i];
+                f[4 * i + 1] = xv.y + p.resid_sign * f[4 * i + 1];
+                f[4 * i + 2] = xv.z + p.resid_sign * f[4 * i + 2];
+                f[4 * i + 3] = xv.w + p.resid_sign * f[4 * i + 3];
+              }
             }
           }
+          // two staging buffers: the store issued two blocks ago must have read its buffer
+          uint8_t* buf = stg + (n_grp & 1u) * 4096;
+          if (lane == 0) bulk_wait_read<1>();
+          __syncwarp();
+          if (f32_out) stage32_f32(buf, lane, f); else stage32_bf16(buf, lane, f);
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t src = stg_u32 + (n_grp & 1u) * 4096;
+            if (EPI == EPI_WGRAD && p.accumulate) tma_reduce_add_2d(&map_c, src, n, y0);
+            else tma_store_2d(&map_c, src, n, y0);
+            bulk_commit();
+          }
+          ++n_grp;
         }
       } else if constexpr (EPI == EPI_SWIGLU) {
-        // columns [0, MMA_N/2) hold the gate projection, [MMA_N/2, MMA_N) the up projection
+        // columns [0, MMA_N/2) hold the gate projection, [MMA_N/2, MMA_N) the up projection.
+        // staging: H in two alternating 2 KB buffers; the optional a|b block in one 4 KB buffer
         uint32_t r1[32];
         float g[32];
 #pragma unroll 1
         for (int c = 0; c < MMA_N / 2; c += 32) {
+          const int n = t.n0 + c;
+          if (!slab_ok || n >= p.N) continue;      // warp-uniform
           tmem_ld32(taddr + c, r0);
           tmem_ld32(taddr + MMA_N / 2 + c, r1);
           tmem_ld_wait();
-          const int n = t.n0 + c;
-          if (!m_ok || n >= p.N) continue;
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             f[i] = __uint_as_float(r0[i]);
             g[i] = __uint_as_float(r1[i]);
           }
+          if (lane == 0) { if (p.C1) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
+          __syncwarp();
           if (p.C1) {
-            bf16* ab = reinterpret_cast<bf16*>(p.C1) + (int64_t)m * p.ldc1;
-            store32_bf16(ab + n, f);
-            store32_bf16(ab + p.N + n, g);
+            stage32_bf16(stg + 4096, lane, f);
+            stage32_bf16(stg + 6144, lane, g);
           }
 #pragma unroll
           for (int i = 0; i < 32; ++i) f[i] = swiglu_f(f[i], g[i]);
-          store32_bf16(reinterpret_cast<bf16*>(p.C) + (int64_t)m * p.ldc + n, f);
+          stage32_bf16(stg + (n_grp & 1u) * 2048, lane, f);
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&map_c, stg_u32 + (n_grp & 1u) * 2048, n, y0);
+            if (p.C1) {
+              tma_store_2d(&map_c1, stg_u32 + 4096, n, y0);
+              tma_store_2d(&map_c1, stg_u32 + 6144, p.N + n, y0);
+            }
+            bulk_commit();
+          }
+          ++n_grp;
         }
       } else {   // EPI_DSWIGLU
         float rs = (p.rowscale && m_ok) ? p.rowscale[m] : 1.f;
@@ -445,6 +512,8 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
     }
+    // this lane's stores must be complete (shared memory read, global memory written) before the CTA exits
+    if (lane == 0) bulk_wait_all();
   }
 
   // ------------------------------------------------------------------ teardown
@@ -526,6 +595,20 @@ inline int tc_make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64
   return r == CUDA_SUCCESS ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
 
+// Tensor map of an epilogue output: boxes of 32 rows x 32 columns, fp32 (128-byte rows,
+// 128-byte swizzle) or bf16 (64-byte rows, 64-byte swizzle).
+inline int tc_make_out_map(CUtensorMap* map, const void* ptr, bool f32, uint64_t inner, uint64_t outer, uint64_t ld) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld * (f32 ? 4u : 2u)};
+  cuuint32_t box[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = tc_state().encode(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                                 const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 f32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? REVFFN_OK : REVFFN_ERR_CUDA;
+}
+
 inline int tc_pick_n(const GemmProblem& p) {
   if (p.epilogue == EPI_SWIGLU) return 256;          // 128 gate + 128 up columns
   if (p.epilogue == EPI_DSWIGLU) return 128;
@@ -535,8 +618,8 @@ inline int tc_dg_parts(int N) { return (int)ceil_div(N, 128); }
 
 template <int MMA_N, int EPI>
 inline int tc_launch(const TcParams& P, const CUtensorMap& ma, const CUtensorMap& mb0, const CUtensorMap& mb1,
-                     int grid, cudaStream_t st) {
-  gemm_tc_kernel<MMA_N, EPI><<<grid, TC_THREADS, TcCfg<MMA_N>::SMEM_BYTES, st>>>(P, ma, mb0, mb1);
+                     const CUtensorMap& mc, const CUtensorMap& mc1, int grid, cudaStream_t st) {
+  gemm_tc_kernel<MMA_N, EPI><<<grid, TC_THREADS, TcCfg<MMA_N>::SMEM_BYTES, st>>>(P, ma, mb0, mb1, mc, mc1);
   return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
 
@@ -584,12 +667,33 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
     r = tc_make_map(&mb1, p.B1 ? p.B1 : p.B0, (uint64_t)p.ldb, rows, (uint64_t)p.ldb, 64, 64);
     if (r) return r;
   }
+  // epilogue outputs written through TMA stores
+  CUtensorMap mc, mc1;
+  memset(&mc, 0, sizeof(mc));
+  memset(&mc1, 0, sizeof(mc1));
+  if (p.epilogue != EPI_DSWIGLU) {
+    const bool f32_out = p.epilogue == EPI_COUPLE || p.epilogue == EPI_WGRAD || (p.epilogue == EPI_STORE && p.out_f32);
+    uint64_t rows = (uint64_t)p.M;
+    if (p.group_mode == GROUP_K) {
+      // group g's block must start g * M rows further down one 2D tensor
+      if (p.M % TC_BM != 0 || p.c_group_stride != (int64_t)p.M * p.ldc) return REVFFN_ERR_SHAPE;
+      rows = (uint64_t)groups * p.M;
+    }
+    if ((reinterpret_cast<uintptr_t>(p.C) & 15u) || (p.ldc * (f32_out ? 4 : 2)) % 16 != 0) return REVFFN_ERR_ALIGN;
+    int r = tc_make_out_map(&mc, p.C, f32_out, (uint64_t)p.N, rows, (uint64_t)p.ldc);
+    if (r) return r;
+    if (p.epilogue == EPI_SWIGLU && p.C1) {
+      if ((reinterpret_cast<uintptr_t>(p.C1) & 15u) || (p.ldc1 * 2) % 16 != 0) return REVFFN_ERR_ALIGN;
+      r = tc_make_out_map(&mc1, p.C1, false, (uint64_t)2 * p.N, (uint64_t)p.M, (uint64_t)p.ldc1);
+      if (r) return r;
+    }
+  }
   int64_t total = (int64_t)P.tiles_m * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
   int grid = (int)(total < s.n_sms ? total : s.n_sms);
   if (grid <= 0) return REVFFN_OK;
 
 #define TC_CASE(N_, E_) \
-  if (mma_n == N_ && p.epilogue == E_) return tc_launch<N_, E_>(P, ma, mb0, mb1, grid, st);
+  if (mma_n == N_ && p.epilogue == E_) return tc_launch<N_, E_>(P, ma, mb0, mb1, mc, mc1, grid, st);
   TC_CASE(256, EPI_STORE) TC_CASE(128, EPI_STORE)
   TC_CASE(256, EPI_SWIGLU)
   TC_CASE(256, EPI_ROWSCALE) TC_CASE(128, EPI_ROWSCALE)
