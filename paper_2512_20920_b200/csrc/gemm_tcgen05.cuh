@@ -1,6 +1,6 @@
 // tcgen05 / TMEM / TMA back end for every bf16 matrix product on the path.
 //
-// One persistent, warp-specialised kernel (1 CTA per SM, 192 threads):
+// One persistent, warp-specialised kernel (1 CTA per SM, 320 threads):
 //   warp 0      TMA producer: cp.async.bulk.tensor 2D loads (128-byte swizzle) of
 //               A and B tiles into a ring of shared-memory stages, completion on
 //               mbarriers (no cluster multicast anywhere).
@@ -9,13 +9,15 @@
 //               elected lane issues tcgen05.mma kind::f16 (bf16 x bf16 -> fp32),
 //               M = 128, N = 128 or 256, K = 16 per instruction; tcgen05.commit
 //               releases stages and publishes finished accumulators.
-//   warps 2..5  epilogue: tcgen05.ld the accumulator (lane = tile row), apply the
+//   warps 2..9  epilogue (two warps per TMEM lane quadrant, alternating 32-column blocks):
+//               tcgen05.ld the accumulator (lane = tile row), apply the
 //               fused epilogue (SwiGLU, gate scale, coupling add/sub, SwiGLU
 //               backward, fp32 weight-gradient store), stage 32 x 32 output blocks in
 //               swizzled shared memory and hand them to TMA bulk tensor stores
 //               (reduce-add when a gradient is accumulated), so that global
 //               writes are whole lines whatever the row stride.
-// Tile = 128 rows x MMA_N columns, K step 64 (one 128-byte swizzle atom of bf16).
+// Tile = 128 rows x 256 columns (the last column tile of a row may be 128 wide: N only has
+// to be a multiple of 128), K step 64 (one 128-byte swizzle atom of bf16).
 // Both operands may be K-major or MN-major; MN-major tiles are fetched as
 // 64x64 boxes and described to the tensor core with leading/stride offsets.
 // Every wait is bounded; on expiry the kernel sets the status word and leaves.
@@ -32,23 +34,24 @@ namespace revffn {
 
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;
+constexpr int TC_EPI_WARPS = 8;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
 constexpr long long TC_WAIT_CYCLES = 4000000000LL;       // ~2 s: bound on any single wait
 
-constexpr int TC_EPI_WARP_BYTES = 8192;                  // output staging per epilogue warp
-constexpr int TC_EPI_BYTES = 4 * TC_EPI_WARP_BYTES;
-
-template <int MMA_N> struct TcCfg {
+template <int MMA_N, int EPI> struct TcCfg {
   static constexpr int B_BYTES = MMA_N * TC_BK * 2;
   static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
-  static constexpr int STAGES = (MMA_N == 256) ? 4 : 6;
-  static constexpr int TMEM_COLS = 2 * MMA_N;           // 512 or 256: power of two >= 32
+  // The SwiGLU-backward epilogue streams its a|b operands through shared memory as well
+  // and gets a larger staging area at the price of one pipeline stage.
+  static constexpr int STAGES = (EPI == EPI_DSWIGLU) ? 3 : 4;
+  static constexpr int EPI_WARP_BYTES = (EPI == EPI_DSWIGLU) ? 10240 : 4096;   // staging per epilogue warp
+  static constexpr int TMEM_COLS = 2 * MMA_N;           // two accumulators; a power of two >= 32
   // stage ring | epilogue staging | barriers; the ring starts 1024-byte aligned and
   // every stage is a multiple of 1024 bytes, so the staging area is aligned too
   static constexpr int EPI_OFF = STAGES * STAGE_BYTES;
-  static constexpr int BAR_OFF = EPI_OFF + TC_EPI_BYTES;
-  static constexpr int SMEM_BYTES = BAR_OFF + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr int BAR_OFF = EPI_OFF + TC_EPI_WARPS * EPI_WARP_BYTES;
+  static constexpr int SMEM_BYTES = BAR_OFF + 1024 /*align*/ + 512 /*barriers*/;
 };
 
 struct TcParams {
@@ -214,6 +217,7 @@ __device__ __forceinline__ void stage32_bf16(uint8_t* buf, int r, const float* f
 // Tile coordinates shared by the three roles.
 struct TcTile {
   int m0, n0, group, k_blocks, krow0;
+  int ncols;      // accumulator columns in use: 256, or 128 in the last column tile of an odd multiple of 128
   bool valid;
 };
 
@@ -226,6 +230,7 @@ __device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_
   t.k_blocks = P.k_blocks;
   int total = (p.group_mode == GROUP_K) ? per_group * p.n_groups : per_group;
   t.valid = w < total;
+  t.ncols = 0;
   if (!t.valid) { t.m0 = t.n0 = 0; return t; }
   int r = w;
   if (p.group_mode == GROUP_K) {
@@ -238,6 +243,7 @@ __device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_
   int tm = r / P.tiles_n, tn = r - tm * P.tiles_n;
   t.m0 = tm * TC_BM;
   t.n0 = tn * P.tile_n;
+  t.ncols = (p.concat == CONCAT_N) ? 2 * P.tile_n : min(P.tile_n, p.N - t.n0);
   if (p.group_mode == GROUP_M) t.group = p.tile_group[tm];
   return t;
 }
@@ -250,7 +256,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUtensorMap map_a,
                const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c1) {
-  using Cfg = TcCfg<MMA_N>;
+  using Cfg = TcCfg<MMA_N, EPI>;
   extern __shared__ uint8_t smem_raw[];
   const GemmProblem& p = P.p;
   const uint32_t raw = smem_u32(smem_raw);
@@ -261,7 +267,8 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   auto empty_bar = [&](int s) { return bars + 8u * (Cfg::STAGES + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + 2 + a); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + Cfg::BAR_OFF + 8 * (2 * Cfg::STAGES + 4));
+  auto epi_bar = [&](int ew, int s) { return bars + 128u + 8u * (ew * 2 + s); };   // SwiGLU backward: operand loads
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + Cfg::BAR_OFF + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* issued = reinterpret_cast<int*>(tmem_slot + 2);   // [STAGES] parity+1 of the last load issued per stage
 
@@ -269,7 +276,8 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); issued[s] = 0; }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), TC_EPI_WARPS); }
+    for (int a = 0; a < 2 * TC_EPI_WARPS; ++a) mbar_init(epi_bar(a / 2, a % 2), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -302,7 +310,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
           const uint32_t sb = sa + TC_A_BYTES;
           const uint32_t fb = full_bar(stage);
-          mbar_expect_tx(fb, Cfg::STAGE_BYTES);
+          mbar_expect_tx(fb, TC_A_BYTES + t.ncols * TC_BK * 2);
           issued[stage] = (int)phase + 1;
           // A tile
           if (!p.a_mn_major) {
@@ -324,14 +332,16 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
               tma_load_2d(sb + 16384, &map_b1, kb_b * TC_BK, row0, fb);
             } else {
 #pragma unroll
-              for (int j = 0; j < MMA_N / 128; ++j) tma_load_2d(sb + j * 16384, mb, kb_b * TC_BK, row0 + 128 * j, fb);
+              for (int j = 0; j < MMA_N / 128; ++j)
+                if (128 * j < t.ncols) tma_load_2d(sb + j * 16384, mb, kb_b * TC_BK, row0 + 128 * j, fb);
             }
           } else {
             // rows of the flattened [groups * Kdim, N] weight tensor, or token rows (GROUP_K / dense wgrad)
             int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
             int krow = (p.group_mode == GROUP_M ? t.group * kdim : t.krow0) + kb_b * TC_BK;
 #pragma unroll
-            for (int j = 0; j < MMA_N / 64; ++j) tma_load_2d(sb + j * 8192, mb, p.b_col0 + t.n0 + 64 * j, krow, fb);
+            for (int j = 0; j < MMA_N / 64; ++j)
+              if (64 * j < t.ncols) tma_load_2d(sb + j * 8192, mb, p.b_col0 + t.n0 + 64 * j, krow, fb);
           }
           if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -352,6 +362,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MMA_N);
+        const uint32_t idesc = (P.idesc & ~(0x3Fu << 17)) | ((uint32_t)(t.ncols >> 3) << 17);   // N of this tile
         for (int kb = 0; kb < t.k_blocks; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
@@ -363,7 +374,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           const uint32_t b_step = p.b_mn_major ? (2048u >> 4) : (32u >> 4);
 #pragma unroll
           for (int ks = 0; ks < TC_BK / 16; ++ks) {
-            tc_mma(d_tmem, a_desc + (uint64_t)(a_step * ks), b_desc + (uint64_t)(b_step * ks), P.idesc,
+            tc_mma(d_tmem, a_desc + (uint64_t)(a_step * ks), b_desc + (uint64_t)(b_step * ks), idesc,
                    (kb | ks) != 0 ? 1u : 0u);
           }
           tc_commit(empty_bar(stage));          // stage reusable once these MMAs have read it
@@ -374,14 +385,48 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
     const int q = warp & 3;                      // TMEM lane quadrant this warp may access
+    const int ew = warp - 2;                     // epilogue warp index
+    const int half = ew >> 2;                    // this warp takes the 32-column blocks half, half+2, ...
     const int row_in_tile = q * 32 + lane;
-    uint8_t* stg = gen_base + Cfg::EPI_OFF + q * TC_EPI_WARP_BYTES;   // this warp's staging area
-    const uint32_t stg_u32 = base + Cfg::EPI_OFF + q * TC_EPI_WARP_BYTES;
+    uint8_t* stg = gen_base + Cfg::EPI_OFF + ew * Cfg::EPI_WARP_BYTES;   // this warp's staging area
+    const uint32_t stg_u32 = base + Cfg::EPI_OFF + ew * Cfg::EPI_WARP_BYTES;
     bool ok = true;
     int it = 0;
     uint32_t n_grp = 0;                          // bulk groups committed so far (same in every lane)
+    // SwiGLU backward: a|b blocks arrive by TMA in one of two 4 KB sets [a 2 KB | b 2 KB]; the
+    // prefetch cursor runs one block ahead of the consumer, across tile boundaries.
+    constexpr int DS_SET = 4096;
+    auto ds_chunks = [&](const TcTile& t) -> int {   // blocks of this warp in tile t
+      if (!t.valid) return 0;
+      const int lim = (p.group_mode == GROUP_M) ? tiles_m_dev * TC_BM : p.M;
+      return (t.m0 + q * 32 < lim) ? (t.ncols / 32 - half + 1) / 2 : 0;
+    };
+    uint32_t ds_g = 0, ds_pf_g = 0;              // blocks consumed / loads issued
+    int ds_pf_w = blockIdx.x, ds_pf_c = 0;
+    TcTile ds_pf_t;
+    ds_pf_t.valid = false;
+    auto ds_prefetch = [&]() {
+      while (ds_pf_t.valid && ds_pf_c >= ds_chunks(ds_pf_t)) {
+        ds_pf_w += gridDim.x; ds_pf_c = 0;
+        ds_pf_t = tc_tile(P, ds_pf_w, tiles_m_dev);
+      }
+      if (!ds_pf_t.valid) return;
+      const int s2 = (int)(ds_pf_g & 1u);
+      if (lane == 0) {
+        const int n = ds_pf_t.n0 + (half + 2 * ds_pf_c) * 32, y = ds_pf_t.m0 + q * 32;
+        const uint32_t dst = stg_u32 + s2 * DS_SET, bar = epi_bar(ew, s2);
+        mbar_expect_tx(bar, 4096);
+        tma_load_2d(dst, &map_c, n, y, bar);
+        tma_load_2d(dst + 2048, &map_c, p.N + n, y, bar);
+      }
+      ++ds_pf_c; ++ds_pf_g;
+    };
+    if constexpr (EPI == EPI_DSWIGLU) {
+      ds_pf_t = tc_tile(P, ds_pf_w, tiles_m_dev);
+      ds_prefetch();
+    }
     for (int w = blockIdx.x; ok; w += gridDim.x, ++it) {
       TcTile t = tc_tile(P, w, tiles_m_dev);
       if (!t.valid) break;
@@ -405,9 +450,9 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         if (EPI == EPI_ROWSCALE && m_ok) rs = p.rowscale[m];
         const bool f32_out = (EPI == EPI_COUPLE) || (EPI == EPI_WGRAD) || (EPI == EPI_STORE && p.out_f32);
 #pragma unroll 1
-        for (int c = 0; c < MMA_N; c += 32) {
+        for (int c = half * 32; c < t.ncols; c += 64) {
           const int n = t.n0 + c;
-          if (!slab_ok || n >= p.N) continue;      // warp-uniform
+          if (!slab_ok) continue;      // warp-uniform
           if (have_acc) { tmem_ld32(taddr + c, r0); tmem_ld_wait(); }
 #pragma unroll
           for (int i = 0; i < 32; ++i) f[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
@@ -427,30 +472,31 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
               }
             }
           }
-          // two staging buffers: the store issued two blocks ago must have read its buffer
-          uint8_t* buf = stg + (n_grp & 1u) * 4096;
-          if (lane == 0) bulk_wait_read<1>();
+          // fp32 blocks fill the staging area (4 KB): the previous store must have read it;
+          // bf16 blocks (2 KB) alternate between its halves
+          const uint32_t off = f32_out ? 0u : (n_grp & 1u) * 2048u;
+          if (lane == 0) { if (f32_out) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
           __syncwarp();
-          if (f32_out) stage32_f32(buf, lane, f); else stage32_bf16(buf, lane, f);
+          if (f32_out) stage32_f32(stg + off, lane, f); else stage32_bf16(stg + off, lane, f);
           fence_async_smem();
           __syncwarp();
           if (lane == 0) {
-            const uint32_t src = stg_u32 + (n_grp & 1u) * 4096;
-            if (EPI == EPI_WGRAD && p.accumulate) tma_reduce_add_2d(&map_c, src, n, y0);
-            else tma_store_2d(&map_c, src, n, y0);
+            if (EPI == EPI_WGRAD && p.accumulate) tma_reduce_add_2d(&map_c, stg_u32 + off, n, y0);
+            else tma_store_2d(&map_c, stg_u32 + off, n, y0);
             bulk_commit();
           }
           ++n_grp;
         }
       } else if constexpr (EPI == EPI_SWIGLU) {
         // columns [0, MMA_N/2) hold the gate projection, [MMA_N/2, MMA_N) the up projection.
-        // staging: H in two alternating 2 KB buffers; the optional a|b block in one 4 KB buffer
+        // H goes out through two alternating 2 KB staging buffers; the optional a|b copy is
+        // written straight from registers (64 contiguous bytes per row and operand).
         uint32_t r1[32];
         float g[32];
 #pragma unroll 1
-        for (int c = 0; c < MMA_N / 2; c += 32) {
+        for (int c = half * 32; c < MMA_N / 2; c += 64) {
           const int n = t.n0 + c;
-          if (!slab_ok || n >= p.N) continue;      // warp-uniform
+          if (!slab_ok) continue;      // warp-uniform
           tmem_ld32(taddr + c, r0);
           tmem_ld32(taddr + MMA_N / 2 + c, r1);
           tmem_ld_wait();
@@ -459,58 +505,97 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             f[i] = __uint_as_float(r0[i]);
             g[i] = __uint_as_float(r1[i]);
           }
-          if (lane == 0) { if (p.C1) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
-          __syncwarp();
-          if (p.C1) {
-            stage32_bf16(stg + 4096, lane, f);
-            stage32_bf16(stg + 6144, lane, g);
+          if (p.C1 && m_ok) {
+            bf16* ab = reinterpret_cast<bf16*>(p.C1) + (int64_t)m * p.ldc1;
+            store32_bf16(ab + n, f);
+            store32_bf16(ab + p.N + n, g);
           }
 #pragma unroll
           for (int i = 0; i < 32; ++i) f[i] = swiglu_f(f[i], g[i]);
-          stage32_bf16(stg + (n_grp & 1u) * 2048, lane, f);
+          const uint32_t off = (n_grp & 1u) * 2048u;
+          if (lane == 0) bulk_wait_read<1>();
+          __syncwarp();
+          stage32_bf16(stg + off, lane, f);
           fence_async_smem();
           __syncwarp();
           if (lane == 0) {
-            tma_store_2d(&map_c, stg_u32 + (n_grp & 1u) * 2048, n, y0);
-            if (p.C1) {
-              tma_store_2d(&map_c1, stg_u32 + 4096, n, y0);
-              tma_store_2d(&map_c1, stg_u32 + 6144, p.N + n, y0);
-            }
+            tma_store_2d(&map_c, stg_u32 + off, n, y0);
             bulk_commit();
           }
           ++n_grp;
         }
       } else {   // EPI_DSWIGLU
+        // Per 32-column block: a|b arrive by TMA in a set [a 2 KB | b 2 KB] of this warp's staging
+        // area, da|db are written over them, g*H into a buffer of its own, and three TMA stores
+        // take them back to global memory.  Two sets alternate; the load of the warp's next block
+        // is issued as soon as the stores of its previous block have read their set.
         float rs = (p.rowscale && m_ok) ? p.rowscale[m] : 1.f;
         float dg = 0.f;
         float a[32], b[32];
+        const int nch = ds_chunks(t);
 #pragma unroll 1
-        for (int c = 0; c < MMA_N; c += 32) {
-          tmem_ld32(taddr + c, r0);
-          tmem_ld_wait();
+        for (int ci = 0; ci < nch && ok; ++ci, ++ds_g) {
+          const int s2 = (int)(ds_g & 1u);
+          const uint32_t par = (ds_g >> 1) & 1u;
+          const int c = (half + 2 * ci) * 32;
           const int n = t.n0 + c;
-          if (!m_ok || n >= p.N) continue;
-          bf16* ab = reinterpret_cast<bf16*>(p.ab) + (int64_t)m * p.ld_ab;
-          load32_bf16(ab + n, a);
-          load32_bf16(ab + p.N + n, b);
+          tmem_ld32(taddr + c, r0);
+          if (!mbar_wait(epi_bar(ew, s2), par, abort_flag, p.status)) { ok = false; tmem_ld_wait(); break; }
+          tmem_ld_wait();
+          uint8_t* set = stg + s2 * DS_SET;
+          uint8_t* row_a = set + lane * 64;
+          uint8_t* row_b = set + 2048 + lane * 64;
+          uint8_t* row_h = stg + 2 * DS_SET + lane * 64;
+          const int sw = (lane >> 1) & 3;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            unpack8(*reinterpret_cast<const uint4*>(row_a + ((j ^ sw) << 4)), a + 8 * j);
+            unpack8(*reinterpret_cast<const uint4*>(row_b + ((j ^ sw) << 4)), b + 8 * j);
+          }
+          // the previous block's stores have read their sources: its set is free for the next load,
+          // and the single g*H buffer may be rewritten
+          if (lane == 0) bulk_wait_read<0>();
+          __syncwarp();
+          ds_prefetch();
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             float v = __uint_as_float(r0[i]);
             float da, db;
             float H = dswiglu_f(a[i], b[i], rs * v, da, db);
-            dg += v * H;
+            if (m_ok) dg += v * H;
             a[i] = da; b[i] = db; f[i] = rs * H;
           }
-          store32_bf16(ab + n, a);
-          store32_bf16(ab + p.N + n, b);
-          if (p.C1) store32_bf16(reinterpret_cast<bf16*>(p.C1) + (int64_t)m * p.ldc1 + n, f);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            *reinterpret_cast<uint4*>(row_a + ((j ^ sw) << 4)) = pack8(a + 8 * j);
+            *reinterpret_cast<uint4*>(row_b + ((j ^ sw) << 4)) = pack8(b + 8 * j);
+            *reinterpret_cast<uint4*>(row_h + ((j ^ sw) << 4)) = pack8(f + 8 * j);
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t src = stg_u32 + s2 * DS_SET;
+            tma_store_2d(&map_c, src, n, y0);
+            tma_store_2d(&map_c, src + 2048, p.N + n, y0);
+            if (p.C1) tma_store_2d(&map_c1, stg_u32 + 2 * DS_SET, n, y0);
+            bulk_commit();
+          }
         }
-        if (p.dg_part && m_ok) p.dg_part[(int64_t)m * p.dg_ld + t.n0 / P.tile_n] = dg;
+        if (p.dg_part && m_ok) p.dg_part[(int64_t)m * p.dg_ld + 2 * (t.n0 / P.tile_n) + half] = dg;
       }
       // accumulator may be overwritten by the MMA warp
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
+    }
+    if constexpr (EPI == EPI_DSWIGLU) {
+      // operand loads issued but not consumed (only after an abandoned wait) must land before the CTA exits
+      if (lane == 0) {
+        for (uint32_t g = ds_g; g < ds_pf_g; ++g) {
+          long long t0 = clock64();
+          while (!mbar_try_wait(epi_bar(ew, (int)(g & 1u)), (g >> 1) & 1u) && clock64() - t0 < TC_WAIT_CYCLES) {}
+        }
+      }
     }
     // this lane's stores must be complete (shared memory read, global memory written) before the CTA exits
     if (lane == 0) bulk_wait_all();
@@ -551,7 +636,7 @@ inline TcState& tc_state() { static TcState s; return s; }
 template <int MMA_N, int EPI>
 inline cudaError_t tc_set_attr() {
   return cudaFuncSetAttribute(gemm_tc_kernel<MMA_N, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              TcCfg<MMA_N>::SMEM_BYTES);
+                              TcCfg<MMA_N, EPI>::SMEM_BYTES);
 }
 
 // Once per process: driver entry point for tensor-map encoding, SM count, shared-memory opt-in.
@@ -568,15 +653,11 @@ inline int tc_prepare() {
   if (cudaDeviceGetAttribute(&s.n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return REVFFN_ERR_CUDA;
   cudaError_t e = cudaSuccess;
   if (e == cudaSuccess) e = tc_set_attr<256, EPI_STORE>();
-  if (e == cudaSuccess) e = tc_set_attr<128, EPI_STORE>();
   if (e == cudaSuccess) e = tc_set_attr<256, EPI_SWIGLU>();
   if (e == cudaSuccess) e = tc_set_attr<256, EPI_ROWSCALE>();
-  if (e == cudaSuccess) e = tc_set_attr<128, EPI_ROWSCALE>();
   if (e == cudaSuccess) e = tc_set_attr<256, EPI_COUPLE>();
-  if (e == cudaSuccess) e = tc_set_attr<128, EPI_COUPLE>();
-  if (e == cudaSuccess) e = tc_set_attr<128, EPI_DSWIGLU>();
+  if (e == cudaSuccess) e = tc_set_attr<256, EPI_DSWIGLU>();
   if (e == cudaSuccess) e = tc_set_attr<256, EPI_WGRAD>();
-  if (e == cudaSuccess) e = tc_set_attr<128, EPI_WGRAD>();
   if (e != cudaSuccess) return REVFFN_ERR_CUDA;
   s.ready = true;
   return REVFFN_OK;
@@ -609,17 +690,12 @@ inline int tc_make_out_map(CUtensorMap* map, const void* ptr, bool f32, uint64_t
   return r == CUDA_SUCCESS ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
 
-inline int tc_pick_n(const GemmProblem& p) {
-  if (p.epilogue == EPI_SWIGLU) return 256;          // 128 gate + 128 up columns
-  if (p.epilogue == EPI_DSWIGLU) return 128;
-  return (p.N % 256 == 0) ? 256 : 128;
-}
-inline int tc_dg_parts(int N) { return (int)ceil_div(N, 128); }
+inline int tc_dg_parts(int N) { return 2 * (int)ceil_div(N, 256); }   // two epilogue warps per row and column tile
 
 template <int MMA_N, int EPI>
 inline int tc_launch(const TcParams& P, const CUtensorMap& ma, const CUtensorMap& mb0, const CUtensorMap& mb1,
                      const CUtensorMap& mc, const CUtensorMap& mc1, int grid, cudaStream_t st) {
-  gemm_tc_kernel<MMA_N, EPI><<<grid, TC_THREADS, TcCfg<MMA_N>::SMEM_BYTES, st>>>(P, ma, mb0, mb1, mc, mc1);
+  gemm_tc_kernel<MMA_N, EPI><<<grid, TC_THREADS, TcCfg<MMA_N, EPI>::SMEM_BYTES, st>>>(P, ma, mb0, mb1, mc, mc1);
   return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
 
@@ -627,7 +703,7 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   TcState& s = tc_state();
   if (!s.ready) return REVFFN_ERR_CUDA;
   if (p.M <= 0 || p.N <= 0) return REVFFN_OK;
-  const int mma_n = tc_pick_n(p);
+  const int mma_n = 256;
   TcParams P;
   P.p = p;
   P.tile_n = (p.concat == CONCAT_N) ? mma_n / 2 : mma_n;
@@ -671,7 +747,17 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   CUtensorMap mc, mc1;
   memset(&mc, 0, sizeof(mc));
   memset(&mc1, 0, sizeof(mc1));
-  if (p.epilogue != EPI_DSWIGLU) {
+  if (p.epilogue == EPI_DSWIGLU) {
+    // a|b are loaded and written back in place through one map; g*H (optional) through the other
+    if ((reinterpret_cast<uintptr_t>(p.ab) & 15u) || (p.ld_ab * 2) % 16 != 0) return REVFFN_ERR_ALIGN;
+    int r = tc_make_out_map(&mc, p.ab, false, (uint64_t)2 * p.N, (uint64_t)p.M, (uint64_t)p.ld_ab);
+    if (r) return r;
+    if (p.C1) {
+      if ((reinterpret_cast<uintptr_t>(p.C1) & 15u) || (p.ldc1 * 2) % 16 != 0) return REVFFN_ERR_ALIGN;
+      r = tc_make_out_map(&mc1, p.C1, false, (uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.ldc1);
+      if (r) return r;
+    }
+  } else {
     const bool f32_out = p.epilogue == EPI_COUPLE || p.epilogue == EPI_WGRAD || (p.epilogue == EPI_STORE && p.out_f32);
     uint64_t rows = (uint64_t)p.M;
     if (p.group_mode == GROUP_K) {
@@ -682,11 +768,8 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
     if ((reinterpret_cast<uintptr_t>(p.C) & 15u) || (p.ldc * (f32_out ? 4 : 2)) % 16 != 0) return REVFFN_ERR_ALIGN;
     int r = tc_make_out_map(&mc, p.C, f32_out, (uint64_t)p.N, rows, (uint64_t)p.ldc);
     if (r) return r;
-    if (p.epilogue == EPI_SWIGLU && p.C1) {
-      if ((reinterpret_cast<uintptr_t>(p.C1) & 15u) || (p.ldc1 * 2) % 16 != 0) return REVFFN_ERR_ALIGN;
-      r = tc_make_out_map(&mc1, p.C1, false, (uint64_t)2 * p.N, (uint64_t)p.M, (uint64_t)p.ldc1);
-      if (r) return r;
-    }
+    if (p.epilogue == EPI_SWIGLU && p.C1 && ((reinterpret_cast<uintptr_t>(p.C1) & 15u) || (p.ldc1 * 2) % 16 != 0))
+      return REVFFN_ERR_ALIGN;
   }
   int64_t total = (int64_t)P.tiles_m * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
   int grid = (int)(total < s.n_sms ? total : s.n_sms);
@@ -694,12 +777,8 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
 
 #define TC_CASE(N_, E_) \
   if (mma_n == N_ && p.epilogue == E_) return tc_launch<N_, E_>(P, ma, mb0, mb1, mc, mc1, grid, st);
-  TC_CASE(256, EPI_STORE) TC_CASE(128, EPI_STORE)
-  TC_CASE(256, EPI_SWIGLU)
-  TC_CASE(256, EPI_ROWSCALE) TC_CASE(128, EPI_ROWSCALE)
-  TC_CASE(256, EPI_COUPLE) TC_CASE(128, EPI_COUPLE)
-  TC_CASE(128, EPI_DSWIGLU)
-  TC_CASE(256, EPI_WGRAD) TC_CASE(128, EPI_WGRAD)
+  TC_CASE(256, EPI_STORE) TC_CASE(256, EPI_SWIGLU) TC_CASE(256, EPI_ROWSCALE) TC_CASE(256, EPI_COUPLE)
+  TC_CASE(256, EPI_DSWIGLU) TC_CASE(256, EPI_WGRAD)
 #undef TC_CASE
   return REVFFN_ERR_UNSUPPORTED;
 }

@@ -140,7 +140,7 @@ def test_dswiglu(rv, simt):
     AB0 = AB.clone()
     rs = torch.rand(M, device="cuda") + 0.1
     Hg = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16)
-    parts = N // (64 if simt else 128)
+    parts = N // 64 if simt else 2 * ((N + 255) // 256)      # partials per row
     dg = torch.full((M, parts), float("nan"), device="cuda")
     _call(rv, simt, M=M, N=N, K=K, A=A, B0=B, lda=K, ldb=N, b_mn_major=1, ab=AB, ld_ab=2 * N, rowscale=rs, C1=Hg,
           ldc1=N, dg_part=dg, dg_ld=parts, epilogue=EPI["dswiglu"])
