@@ -274,3 +274,73 @@ def backward(p, Y1, dY2, k: int, eps: float = 1e-6, norm: str = "rms", route_ove
         out["dy1"] = r[:, None] * q - Y1 * (r ** 3 * np.sum(q * Y1, axis=1) / h)[:, None]
         out["norm_gamma"] = np.sum(dn * Y1 * r[:, None], axis=0)
     return out
+
+
+# --------------------------------------------------------------------------- #
+# A stack of coupling branches (Sec. 3.1: the two output streams of a layer are
+# the input of the next one; Sec. 2: inputs are rebuilt layer by layer from the
+# outputs during back-propagation, nothing is cached).
+#
+# Only the MoE branch of each block is modelled, so the streams swap roles from
+# one layer to the next: layer l reads stream P_l and updates stream R_l,
+# (P_l, R_l) = (A, B) for even l and (B, A) for odd l.  Both streams are
+# therefore rewritten every two layers and reconstruction error compounds
+# through both, as it does in the full block.
+# --------------------------------------------------------------------------- #
+def stack_forward(blocks, A, B, k: int, eps: float = 1e-6, norm: str = "rms", route_overrides=None):
+    """R_l <- R_l + MLP_l(Norm(P_l)) for l = 0 .. L-1 (Eq. 2 per layer).
+    Returns (A, B, infos); infos[l] is the layer's `forward` info."""
+    A = np.array(A, dtype=F64)
+    B = np.array(B, dtype=F64)
+    infos = []
+    for l, p in enumerate(blocks):
+        ro = None if route_overrides is None else route_overrides[l]
+        if l % 2 == 0:
+            B, info = forward(p, A, B, k, eps, norm, ro)
+        else:
+            A, info = forward(p, B, A, k, eps, norm, ro)
+        infos.append(info)
+    return A, B, infos
+
+
+def stack_inverse(blocks, A, B, k: int, eps: float = 1e-6, norm: str = "rms", route_overrides=None):
+    """Undo `stack_forward` from its outputs: R_l <- R_l - MLP_l(Norm(P_l)) for
+    l = L-1 .. 0 (inverse pass of Sec. 3.1 per layer).  Returns (A, B)."""
+    A = np.array(A, dtype=F64)
+    B = np.array(B, dtype=F64)
+    for l in reversed(range(len(blocks))):
+        ro = None if route_overrides is None else route_overrides[l]
+        if l % 2 == 0:
+            B, _ = inverse(blocks[l], A, B, k, eps, norm, ro)
+        else:
+            A, _ = inverse(blocks[l], B, A, k, eps, norm, ro)
+    return A, B
+
+
+def stack_backward(blocks, A_out, B_out, gA, gB, k: int, eps: float = 1e-6, norm: str = "rms",
+                   route_overrides=None):
+    """Reversible back-propagation through the stack: for l = L-1 .. 0 rebuild
+    the layer's input from its output, then push the gradient through the
+    layer (dP += J^T dR, dR passes through unchanged).
+
+    A_out, B_out: outputs of `stack_forward`; gA, gB: dLoss/dA_out, dLoss/dB_out.
+    Returns (A_in, B_in, dA_in, dB_in, grads); grads[l] holds layer l's weight
+    gradients (the dict `backward` returns)."""
+    A = np.array(A_out, dtype=F64)
+    B = np.array(B_out, dtype=F64)
+    gA = np.array(gA, dtype=F64)
+    gB = np.array(gB, dtype=F64)
+    grads = [None] * len(blocks)
+    for l in reversed(range(len(blocks))):
+        ro = None if route_overrides is None else route_overrides[l]
+        p = blocks[l]
+        if l % 2 == 0:
+            B, _ = inverse(p, A, B, k, eps, norm, ro)
+            g = backward(p, A, gB, k, eps, norm, ro)
+            gA = gA + g["dy1"]
+        else:
+            A, _ = inverse(p, B, A, k, eps, norm, ro)
+            g = backward(p, B, gA, k, eps, norm, ro)
+            gB = gB + g["dy1"]
+        grads[l] = g
+    return A, B, gA, gB, grads
