@@ -8,6 +8,9 @@ of one Qwen1.5-MoE-A2.7B-shaped block over one batch of synthetic tokens
     python bench.py --gpus 1 --steps 10 --warmup 3
     python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   (independent replicas)
     python bench.py --impl reference        (the CPU oracle on the host cores, bounded sample per step)
+    python bench.py --config C3             (24-block reversible stack: tokens/s, peak memory against the
+                                             activation-caching variant, reconstruction drift per layer)
+    python bench.py --config C4             (token-count sweep 512 .. 65536 on the same block shape)
 """
 from __future__ import annotations
 
@@ -155,30 +158,52 @@ def run_reference(args, cfg):
     }))
 
 
-def run_ours(args, cfg):
+def dist_setup():
     import torch
     import torch.distributed as dist
-    import paper_2512_20920_b200 as rv
-    from workloads import make_streams, make_weights
-
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
-    if world > 1:
+    if world > 1 and not dist.is_initialized():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
+    return rank, world, local, barrier
+
+
+def run_ours(args, cfg):
+    out = measure_block(args, cfg, e2e=True, cpu=not args.no_cpu_baseline)
+    if out is not None:
+        print(json.dumps(out))
+    finish()
+
+
+def finish():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.destroy_process_group()
+
+
+def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
+    """One block at cfg.tokens tokens per GPU; returns the JSON record (rank 0) or None."""
+    import torch
+    import torch.distributed as dist
+    import paper_2512_20920_b200 as rv
+    from workloads import make_streams, make_weights
+
+    rank, world, local, barrier = dist_setup()
 
     # every rank is an independent replica with its own tokens (seed + rank); weights are the same
-    w_host = make_weights(cfg, args.seed)
+    if w_dev is None:
+        w_host = make_weights(cfg, args.seed)
+        wdt = torch.bfloat16 if cfg.weight_dtype == "bf16" else torch.float32
+        w_dev = {n: torch.from_numpy(v).cuda().to(torch.float32 if n in ("norm_gamma", "b_router") else wdt).contiguous()
+                 for n, v in w_host.items()}
     s_host = make_streams(cfg, args.seed + rank)
-    wdt = torch.bfloat16 if cfg.weight_dtype == "bf16" else torch.float32
-    w_dev = {n: torch.from_numpy(v).cuda().to(torch.float32 if n in ("norm_gamma", "b_router") else wdt).contiguous()
-             for n, v in w_host.items()}
     blk = rv.Block(tokens=cfg.tokens, d_model=cfg.d_model, n_experts=cfg.n_experts, top_k=cfg.top_k,
                    d_expert=cfg.d_expert, d_shared=cfg.d_shared,
                    weight_dtype=rv.BF16 if cfg.weight_dtype == "bf16" else rv.F32, weights=w_dev,
@@ -246,33 +271,33 @@ def run_ours(args, cfg):
     ms_prof_step = ms_prof_total / args.steps
     value = world * cfg.tokens * args.steps / (ms_total * 1e-3)
 
-    # end to end: host-resident streams, H2D and D2H copies inside the timed region
-    pin = lambda a: torch.from_numpy(a).pin_memory()
-    hy1, hx2, hdy2 = pin(s_host["y1"]), pin(s_host["x2"]), pin(s_host["dy2"])
-    hy2, hx2r, hdy1 = (torch.empty_like(hy1).pin_memory() for _ in range(3))
-    slot = ((hy1.numel() * 4 + 255) // 256) * 256
-    staging = torch.empty(6 * slot, dtype=torch.uint8, device="cuda")
-    g_struct = blk.grads_struct(grads)
-    host_step = lambda: rv.revffn_moe_step_host(blk.desc, blk.w, g_struct, hy1, hx2, hdy2, hy2, hx2r, hdy1, staging, blk.ws)
-    for _ in range(2):
-        host_step()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        host_step()
-        torch.cuda.synchronize()     # the step's results are read on the host
-    dt = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([dt], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dt = float(t.item())
-    e2e_value = world * cfg.tokens * args.steps / dt
-    bytes_dir = 3 * hy1.numel() * 4
+    e2e_value, dt, bytes_dir = None, 0.0, 0
+    if e2e:
+        # end to end: host-resident streams, H2D and D2H copies inside the timed region
+        pin = lambda a: torch.from_numpy(a).pin_memory()
+        hy1, hx2, hdy2 = pin(s_host["y1"]), pin(s_host["x2"]), pin(s_host["dy2"])
+        hy2, hx2r, hdy1 = (torch.empty_like(hy1).pin_memory() for _ in range(3))
+        slot = ((hy1.numel() * 4 + 255) // 256) * 256
+        staging = torch.empty(6 * slot, dtype=torch.uint8, device="cuda")
+        g_struct = blk.grads_struct(grads)
+        host_step = lambda: rv.revffn_moe_step_host(blk.desc, blk.w, g_struct, hy1, hx2, hdy2, hy2, hx2r, hdy1, staging, blk.ws)
+        for _ in range(2):
+            host_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            host_step()
+            torch.cuda.synchronize()     # the step's results are read on the host
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e_value = world * cfg.tokens * args.steps / dt
+        bytes_dir = 3 * hy1.numel() * 4
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+        return None
 
     peaks, peak_kind = load_peaks()
     flops = gemm_flops(cfg, routed_rows)
@@ -312,15 +337,15 @@ def run_ours(args, cfg):
            for ms, cnt, name, kn in kernels]
 
     # CPU baseline: the oracle as it stands on a bounded sample of the same workload (rank 0, N = 1 only)
-    cpu = None
-    if world == 1 and not args.no_cpu_baseline:
+    cpu_rec = None
+    if world == 1 and cpu and w_host is not None:
         from oracle import revffn_oracle as orc
         n_tok = args.cpu_sample_tokens
         oracle_step(orc, w_host, s_host, cfg, n_tok)      # first call pays for first-touch of its gradient arrays
         t0 = time.perf_counter()
         oracle_step(orc, w_host, s_host, cfg, n_tok)
         cdt = time.perf_counter() - t0
-        cpu = {"value": n_tok / cdt, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+        cpu_rec = {"value": n_tok / cdt, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
                "sample": f"second of two fwd+inverse+bwd passes over the first {n_tok} of {cfg.tokens} tokens, "
                          f"full weights, fp64 numpy, {cdt:.1f} s"}
 
@@ -347,17 +372,183 @@ def run_ours(args, cfg):
                                  "ms_per_step": g_ms / args.steps},
         "kernels": top,
         "roofline": roofline,
-        "cpu_baseline": cpu,
-        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": bytes_dir,
-                "d2h_bytes_per_step": bytes_dir, "ms_per_step": 1e3 * dt / args.steps},
+        "cpu_baseline": cpu_rec,
+        "e2e": ({"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": bytes_dir,
+                 "d2h_bytes_per_step": bytes_dir, "ms_per_step": 1e3 * dt / args.steps} if e2e else None),
         "gpu_launches": int(launches),
         "clocks": clocks,
         "peak_device_bytes": int(torch.cuda.max_memory_allocated()),
         "workspace_bytes": {"fwd": blk.fwd_bytes, "bwd": blk.bwd_bytes},
     }
-    print(json.dumps(out))
-    if world > 1:
-        dist.destroy_process_group()
+    # achieved GB/s of the copy-like kernels (algorithmic bytes: rows read + rows written)
+    T, d, k_ = cfg.tokens, cfg.d_model, cfg.top_k
+    hbm_bytes = {"gather_u": 2 * routed_rows * d * 2, "gather_dz": 2 * routed_rows * d * 2,
+                 "combine": (k_ + 2) * T * d * 2, "du_reduce": (k_ + 2) * T * d * 2}
+    out["hbm_kernels"] = {name: {"gbs": hbm_bytes[kn] * cnt / (ms * 1e-3) / 1e9,
+                                 "frac_of_peak": hbm_bytes[kn] * cnt / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                          for ms, cnt, name, kn in kernels if kn in hbm_bytes and ms > 0}
+    return out
+
+
+def run_sweep(args):
+    """C4: the C1 block shape at 512 .. 65536 tokens; one record per size in one JSON line."""
+    import torch
+    from workloads import CONFIGS, make_weights
+    rank, world, local, barrier = dist_setup()
+    base = CONFIGS["C1"]
+    w_host = make_weights(base, args.seed)
+    w_dev = {n: torch.from_numpy(v).cuda().to(torch.float32 if n in ("norm_gamma", "b_router") else torch.bfloat16)
+             .contiguous() for n, v in w_host.items()}
+    del w_host
+    recs = []
+    for t in (512, 2048, 8192, 32768, 65536):
+        cfg = CONFIGS[f"C4-{t}"]
+        a = argparse.Namespace(**vars(args))
+        a.steps = max(5, min(args.steps, int(args.steps * 8192 / t)))      # about the same timed work per size
+        r = measure_block(a, cfg, e2e=False, cpu=False, w_dev=w_dev)
+        torch.cuda.empty_cache()
+        if r is None:
+            continue
+        bwd_gemm = [k for k in r["kernels"] if k["tflops"]]
+        recs.append({"tokens": t, "steps": a.steps, "ms_per_step": r["ms_per_step"], "tokens_per_s": r["value"],
+                     "passes_tokens_per_s": r["passes_tokens_per_s"], "step_tflops": r["step_tflops"],
+                     "pct_bf16_tensor_peak": r["pct_bf16_tensor_peak"],
+                     "grouped_expert_gemms_frac_of_peak": r["grouped_expert_gemms"]["frac_of_peak"],
+                     "hbm_kernels": r["hbm_kernels"], "clocks": r["clocks"],
+                     "slowest_gemm": min(bwd_gemm, key=lambda k: k["tflops"])["kernel"] if bwd_gemm else None})
+    if rank == 0:
+        mid = next(x for x in recs if x["tokens"] == 8192)
+        peaks, kind = load_peaks()
+        print(json.dumps({
+            "metric": METRIC, "value": mid["tokens_per_s"], "unit": "tokens/s", "n_gpus": world, "steps": mid["steps"],
+            "warmup": max(args.warmup, 3), "ms_per_step": mid["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "C4: token-count sweep on the C1 block shape; value is the 8192-token point",
+                       "l2": "working set exceeds the 126 MB L2 at every size (1.1 GB of weights per pass)"},
+            "peak": {"bf16_tflops_sustained": peaks.get("bf16_tflops_sustained"), "hbm_gbs": peaks.get("hbm_gbs"),
+                     "source": kind},
+            "sweep": recs}))
+    finish()
+
+
+def run_stack(args, cfg):
+    """C3: n_blocks coupling branches; step = forward through the stack + reversible backward."""
+    import torch
+    import paper_2512_20920_b200 as rv
+    from workloads import make_streams, make_weights_device, weight_shapes
+    rank, world, local, barrier = dist_setup()
+    L = args.blocks or cfg.n_blocks
+    weights = [make_weights_device(cfg, args.seed, block=l) for l in range(L)]
+    w_bytes = sum(t.numel() * t.element_size() for w in weights for t in w.values())
+    s_host = make_streams(cfg, args.seed + rank)
+    a0, b0 = torch.from_numpy(s_host["y1"]).cuda(), torch.from_numpy(s_host["x2"]).cuda()
+    g0 = torch.from_numpy(s_host["dy2"]).cuda()
+    # one fp32 gradient buffer per tensor, reused by every layer (an optimiser would consume it layer by layer);
+    # the router stays frozen
+    gbuf = {n: torch.empty(shp, dtype=torch.float32, device="cuda") for n, shp in weight_shapes(cfg).items()
+            if n not in ("w_router", "b_router")}
+    a, b, ga, gb = (torch.empty_like(a0) for _ in range(4))
+    kw = dict(tokens=cfg.tokens, d_model=cfg.d_model, n_experts=cfg.n_experts, top_k=cfg.top_k, d_expert=cfg.d_expert,
+              d_shared=cfg.d_shared, weight_dtype=rv.BF16, weights=weights, norm_eps=cfg.norm_eps)
+
+    def timed_variant(caching):
+        torch.cuda.synchronize()
+        base_alloc = torch.cuda.memory_allocated()
+        torch.cuda.reset_peak_memory_stats()
+        stk = rv.Stack(caching=caching, **kw)
+        garr = stk.grads_array([gbuf] * L)
+
+        def step():
+            a.copy_(a0); b.copy_(b0); ga.copy_(g0); gb.copy_(g0)
+            stk.forward(a, b)
+            stk.backward(a, b, ga, gb, garr)
+
+        for _ in range(max(args.warmup, 3)):
+            step()
+        torch.cuda.synchronize()
+        assert stk.status() == 0
+        l0 = rv.revffn_prof_launches()
+        barrier()
+        sampler = ClockSampler(local) if rank == 0 else None
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        barrier()
+        clocks = sampler.stop() if sampler else None
+        ms = e0.elapsed_time(e1) / args.steps
+        assert stk.status() == 0
+        rec = {"ms_per_step": ms, "tokens_per_s": cfg.tokens / (ms * 1e-3), "launches": rv.revffn_prof_launches() - l0,
+               "activation_bytes": int(torch.cuda.max_memory_allocated() - base_alloc),
+               "peak_device_bytes": int(torch.cuda.max_memory_allocated()), "clocks": clocks,
+               "workspace_bytes": stk.bwd_bytes, "cache_bytes": 0 if stk.cache is None else stk.cache.numel(),
+               "saved_bytes_per_layer": stk.saved_bytes}
+        rec["recon_rel_l2"] = [float((a - a0).norm() / a0.norm()), float((b - b0).norm() / b0.norm())] if not caching else None
+        del stk, garr
+        torch.cuda.empty_cache()
+        return rec
+
+    rev = timed_variant(False)
+    cac = timed_variant(True)
+
+    # reconstruction drift and routing flips per layer (diagnostic pass, not timed): layer by layer through
+    # the single-layer entry points, keeping every layer's streams and expert sets from the forward sweep
+    drift = None
+    if not args.no_drift and rank == 0:
+        mk = lambda w, ws: rv.Block(tokens=cfg.tokens, d_model=cfg.d_model, n_experts=cfg.n_experts, top_k=cfg.top_k,
+                                    d_expert=cfg.d_expert, d_shared=cfg.d_shared, weight_dtype=rv.BF16, weights=w,
+                                    norm_eps=cfg.norm_eps, workspace=ws, backward=False)
+        first = mk(weights[0], None)
+        blks = [first] + [mk(w, first.ws) for w in weights[1:]]      # one workspace for all layers
+        drift = {}
+        for mode in ("recomputed_routing", "remembered_routing"):
+            s = [a0.clone(), b0.clone()]
+            kept, idxs = [], []
+            for l, blk in enumerate(blks):
+                P, R = (s[0], s[1]) if l % 2 == 0 else (s[1], s[0])
+                kept.append(R.clone())
+                idx = torch.empty(cfg.tokens, cfg.top_k, dtype=torch.int32, device="cuda")
+                blk.forward(P, R, R, topk_idx_out=idx)
+                idxs.append(idx)
+            per_layer = []
+            for l in reversed(range(L)):
+                blk = blks[l]
+                P, R = (s[0], s[1]) if l % 2 == 0 else (s[1], s[0])
+                blk.inverse(P, R, R, topk_idx_in=idxs[l] if mode == "remembered_routing" else None)
+                idx_now = blk.buffer("idx", torch.int32)[: cfg.tokens * cfg.top_k].view(cfg.tokens, cfg.top_k)
+                flips = int((idx_now.sort(dim=1).values != idxs[l].sort(dim=1).values).any(dim=1).sum())
+                per_layer.append({"layer": l, "rel_l2": float((R - kept[l]).norm() / kept[l].norm()),
+                                  "max_abs": float((R - kept[l]).abs().max()), "routing_flips": flips})
+            drift[mode] = per_layer[::-1]
+        del blks, kept, idxs
+
+    if rank != 0:
+        finish()
+        return
+    print(json.dumps({
+        "metric": METRIC, "value": world * rev["tokens_per_s"], "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": rev["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"C3: {L}-block reversible stack of the C1 block, {cfg.tokens} tokens per GPU; step = "
+                               f"forward through all layers + backward by layer-wise inverse reconstruction (no "
+                               f"cached activations); streams swap roles between layers (only the MoE branch of "
+                               f"each block exists here); weights drawn on the device",
+                   "l2": "per-layer working set exceeds the 126 MB L2", "blocks": L},
+        "gpu_launches": int(rev["launches"]), "clocks": rev["clocks"],
+        "reversible": rev, "caching": cac,
+        "memory": {"weights_bytes": w_bytes,
+                   "reversible_activation_bytes": rev["activation_bytes"],
+                   "caching_activation_bytes": cac["activation_bytes"],
+                   "caching_saved_bytes_minimum": L * (cac["saved_bytes_per_layer"] + a0.numel() * 4),
+                   "note": "activation bytes = peak allocation above weights, streams and the shared gradient "
+                           "buffers while the variant ran; the caching variant allocates a full workspace per "
+                           "layer, of which saved_bytes_per_layer (+ the layer's input stream) must be kept"},
+        "speed_ratio_reversible_over_caching": cac["ms_per_step"] / rev["ms_per_step"],
+        "drift": drift}))
+    finish()
 
 
 def main():
@@ -370,13 +561,22 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-sample-tokens", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--blocks", type=int, default=0, help="C3: number of layers (default: the configuration's 24)")
+    ap.add_argument("--no-drift", action="store_true", help="C3: skip the per-layer drift pass")
     args = ap.parse_args()
     from workloads import CONFIGS
+    if args.config == "C4":
+        if args.impl == "reference":
+            args.config = "C1"
+        else:
+            return run_sweep(args)
     cfg = CONFIGS[args.config]
     if args.cpu_sample_tokens is None:
         args.cpu_sample_tokens = min(cfg.tokens, 128 if args.impl == "ours" else 64)
     if args.impl == "reference":
         run_reference(args, cfg)
+    elif cfg.n_blocks > 1:
+        run_stack(args, cfg)
     else:
         run_ours(args, cfg)
 

@@ -179,6 +179,51 @@ int revffn_moe_status(const void* ws, void* cuda_stream, int32_t* device_status)
 const char* revffn_strerror(int code);
 
 /*
+ * A stack of n_blocks coupling branches (Sec. 3.1: a layer's two output streams are the
+ * next layer's input; Sec. 2: during back-propagation each layer's input is rebuilt from
+ * its output, so no activation outlives its layer).  Only the MoE branch of each block is
+ * in this library, so the streams swap roles between layers: layer l reads stream P_l and
+ * updates stream R_l in place, (P_l, R_l) = (stream_a, stream_b) for even l and
+ * (stream_b, stream_a) for odd l.
+ *
+ *   weights, grads   HOST arrays of n_blocks structs (device pointers inside); several
+ *                    layers may name the same gradient buffers.
+ *   stream_a/b       fp32 [T, h], stride ld_stream, updated in place.
+ *   ws               one workspace of bwd_bytes shared by all layers.
+ *   cache            NULL: reversible operation, nothing is kept between layers.
+ *                    non-NULL: the activation-caching variant the reversible design is
+ *                    measured against: n_blocks slots of revffn_moe_stack_cache_stride
+ *                    bytes (256-byte aligned); forward keeps every layer's input stream
+ *                    and intermediates there, backward reads them and runs no inverse.
+ *
+ * revffn_moe_stack_forward: for l = 0 .. n_blocks-1:  R_l += MLP_l(Norm(P_l))   (Eq. 2).
+ *   topk_idx  optional int32 [n_blocks, T, k], the expert sets of every layer.
+ * revffn_moe_stack_backward: for l = n_blocks-1 .. 0:  R_l -= MLP_l(Norm(P_l)) (the inverse
+ *   pass), then dP_l += J_l^T dR_l and layer l's weight gradients; the gradient pass reuses
+ *   the branch evaluation of the inverse pass.  On entry stream_a/b hold the stack's
+ *   outputs and grad_a/b the loss gradients w.r.t. them; on return stream_a/b hold the
+ *   reconstructed inputs (reversible operation only) and grad_a/b the gradients w.r.t.
+ *   the inputs.
+ *   topk_idx  optional: reuse these expert sets instead of re-selecting them from the
+ *             reconstructed streams (a reconstructed stream differs from the original by
+ *             rounding, which can flip a near-tie).
+ * Same ownership, stream and error conventions as the single-layer entry points.
+ */
+int revffn_moe_stack_cache_stride(const revffn_moe_desc* desc, size_t* bytes);
+int revffn_moe_stack_forward(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                             float* stream_a, float* stream_b, int32_t* topk_idx, void* cache, size_t cache_bytes,
+                             void* ws, size_t ws_bytes, void* cuda_stream);
+int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                              float* stream_a, float* stream_b, float* grad_a, float* grad_b,
+                              const revffn_moe_grads* grads, const int32_t* topk_idx, void* cache,
+                              size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Bytes at the start of a workspace that hold what REVFFN_FLAG_SAVE_ACTIVATIONS keeps for
+ * the gradient pass (the rest of bwd_bytes is scratch of the gradient pass itself).
+ * (Planner; no paper counterpart.) */
+int revffn_moe_saved_size(const revffn_moe_desc* desc, size_t* bytes);
+
+/*
  * One whole step of the path with HOST-resident streams: copies y1, x2 and dy2
  * (host, [T, h] packed, ideally pinned) to the device, runs forward (Eq. 2),
  * inverse (Sec. 3.1) and backward (dy1 starting from zero; it reuses the branch

@@ -8,7 +8,8 @@ before the shared library exists.  There is no fallback: using anything here
 without the built library raises ImportError."""
 import importlib
 
-__all__ = ["Block", "Desc", "Grads", "Weights", "lib", "revffn_moe_backward", "revffn_moe_forward",
+__all__ = ["Block", "Stack", "revffn_moe_saved_size", "revffn_moe_stack_cache_stride",
+           "revffn_moe_stack_forward", "revffn_moe_stack_backward", "Desc", "Grads", "Weights", "lib", "revffn_moe_backward", "revffn_moe_forward",
            "revffn_moe_inverse", "revffn_moe_status", "revffn_moe_workspace_size", "revffn_strerror",
            "revffn_moe_step_host", "revffn_moe_route_noalloc", "revffn_prof_enable", "revffn_prof_launches",
            "revffn_prof_collect", "RevffnError", "BF16", "F32", "NORM_RMS", "NORM_NONE", "FLAG_FORCE_SIMT",

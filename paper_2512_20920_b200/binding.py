@@ -75,6 +75,14 @@ def _load() -> C.CDLL:
     lib.revffn_dbg_gemm.argtypes = [C.POINTER(DbgGemmArgs), vp, vp]
     lib.revffn_moe_step_host.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.POINTER(Grads), vp, vp, vp, vp, vp, vp,
                                          vp, sz, vp, sz, vp]
+    lib.revffn_moe_saved_size.argtypes = [C.POINTER(Desc), C.POINTER(sz)]
+    lib.revffn_moe_stack_cache_stride.argtypes = [C.POINTER(Desc), C.POINTER(sz)]
+    lib.revffn_moe_stack_forward.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp, sz, vp, sz, vp]
+    lib.revffn_moe_stack_backward.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp,
+                                              C.POINTER(Grads), vp, vp, sz, vp, sz, vp]
+    for f in ("revffn_moe_saved_size", "revffn_moe_stack_cache_stride", "revffn_moe_stack_forward",
+              "revffn_moe_stack_backward"):
+        getattr(lib, f).restype = C.c_int
     lib.revffn_moe_route_noalloc.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, vp, vp]
     lib.revffn_moe_route_noalloc.restype = C.c_int
     lib.revffn_prof_enable.argtypes = [C.c_int]
@@ -162,6 +170,39 @@ def revffn_moe_route_noalloc(desc: Desc, w: Weights, y1, topk_idx_out, gates_out
     _check(lib.revffn_moe_route_noalloc(C.byref(desc), C.byref(w), _ptr(y1), _ptr(topk_idx_out), _ptr(gates_out),
                                         _ptr(sgate_out), stream if stream is not None else _stream()),
            "revffn_moe_route_noalloc")
+
+
+def revffn_moe_saved_size(desc: Desc) -> int:
+    n = C.c_size_t(0)
+    _check(lib.revffn_moe_saved_size(C.byref(desc), C.byref(n)), "revffn_moe_saved_size")
+    return n.value
+
+
+def revffn_moe_stack_cache_stride(desc: Desc) -> int:
+    n = C.c_size_t(0)
+    _check(lib.revffn_moe_stack_cache_stride(C.byref(desc), C.byref(n)), "revffn_moe_stack_cache_stride")
+    return n.value
+
+
+def _nbytes(t: Optional[torch.Tensor]) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def revffn_moe_stack_forward(desc: Desc, weights, n_blocks: int, stream_a, stream_b, topk_idx, cache, ws,
+                             stream: Optional[int] = None):
+    """`weights` is a ctypes array of n_blocks Weights structs."""
+    _check(lib.revffn_moe_stack_forward(C.byref(desc), weights, n_blocks, _ptr(stream_a), _ptr(stream_b),
+                                        _ptr(topk_idx), _ptr(cache), _nbytes(cache), _ptr(ws), _nbytes(ws),
+                                        stream if stream is not None else _stream()), "revffn_moe_stack_forward")
+
+
+def revffn_moe_stack_backward(desc: Desc, weights, n_blocks: int, stream_a, stream_b, grad_a, grad_b, grads,
+                              topk_idx, cache, ws, stream: Optional[int] = None):
+    """`weights` / `grads`: ctypes arrays of n_blocks Weights / Grads structs."""
+    _check(lib.revffn_moe_stack_backward(C.byref(desc), weights, n_blocks, _ptr(stream_a), _ptr(stream_b),
+                                         _ptr(grad_a), _ptr(grad_b), grads, _ptr(topk_idx), _ptr(cache),
+                                         _nbytes(cache), _ptr(ws), _nbytes(ws),
+                                         stream if stream is not None else _stream()), "revffn_moe_stack_backward")
 
 
 def revffn_prof_enable(on: bool) -> bool:
@@ -266,3 +307,66 @@ class Block:
         """A named intermediate inside the workspace (tests only)."""
         off, nbytes = ws_lookup(self.desc, name)
         return self.ws[off:off + nbytes].view(dtype)
+
+
+class Stack:
+    """n_blocks coupling branches with alternating stream roles: descriptor, per-layer device
+    weights, one shared workspace and, for the activation-caching variant, the per-layer cache.
+    Pure marshalling around revffn_moe_stack_forward / revffn_moe_stack_backward."""
+
+    def __init__(self, *, tokens: int, d_model: int, n_experts: int, top_k: int, d_expert: int, d_shared: int,
+                 weight_dtype: int, weights, norm_kind: int = NORM_RMS, norm_eps: float = 1e-6,
+                 ld_stream: Optional[int] = None, flags: int = 0, caching: bool = False):
+        self.n_blocks = len(weights)
+        self.desc = Desc(tokens, d_model, n_experts, top_k, d_expert, d_shared, weight_dtype, norm_kind, norm_eps,
+                         ld_stream if ld_stream is not None else d_model // 2, flags)
+        wdt = torch.bfloat16 if weight_dtype == BF16 else torch.float32
+        self.weights = []
+        for w in weights:
+            kept = {}
+            for name in WEIGHT_NAMES:
+                t = w.get(name)
+                if t is None:
+                    continue
+                want = torch.float32 if name in _F32_ALWAYS else wdt
+                if t.dtype != want or not t.is_cuda or not t.is_contiguous():
+                    raise ValueError(f"weight {name}: need a contiguous CUDA tensor of {want}")
+                kept[name] = t
+            self.weights.append(kept)
+        self.w = (Weights * max(self.n_blocks, 1))(*[Weights(**{n: _ptr(w.get(n)) for n in WEIGHT_NAMES})
+                                                     for w in self.weights])
+        self.fwd_bytes, self.bwd_bytes = revffn_moe_workspace_size(self.desc)
+        self.saved_bytes = revffn_moe_saved_size(self.desc)
+        self.cache_stride = revffn_moe_stack_cache_stride(self.desc)
+        self.ws = torch.empty(self.bwd_bytes, dtype=torch.uint8, device="cuda")
+        self.cache = torch.empty(self.cache_stride * self.n_blocks, dtype=torch.uint8, device="cuda") if caching else None
+
+    def grads_array(self, grads, accumulate: bool = False):
+        """ctypes array of n_blocks Grads structs from a list of {name: fp32 CUDA tensor} (one dict per layer;
+        the same dict may be given for several layers)."""
+        if len(grads) != self.n_blocks:
+            raise ValueError("one gradient dict per layer")
+        for g in grads:
+            for n, t in g.items():
+                if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+                    raise ValueError(f"gradient {n}: need a contiguous fp32 CUDA tensor")
+        return (Grads * max(self.n_blocks, 1))(*[Grads(**{n: _ptr(g.get(n)) for n in WEIGHT_NAMES},
+                                                       accumulate=1 if accumulate else 0) for g in grads])
+
+    def forward(self, stream_a, stream_b, topk_idx=None):
+        revffn_moe_stack_forward(self.desc, self.w, self.n_blocks, stream_a, stream_b, topk_idx, self.cache, self.ws)
+
+    def backward(self, stream_a, stream_b, grad_a, grad_b, grads_array, topk_idx=None):
+        revffn_moe_stack_backward(self.desc, self.w, self.n_blocks, stream_a, stream_b, grad_a, grad_b, grads_array,
+                                  topk_idx, self.cache, self.ws)
+
+    def status(self) -> int:
+        """First non-zero device status word of the shared workspace and of every cache slot."""
+        st = revffn_moe_status(self.ws)
+        if st == 0 and self.cache is not None:
+            slot = self.cache_stride - self.bwd_bytes
+            for l in range(self.n_blocks):
+                st = revffn_moe_status(self.cache[l * self.cache_stride + slot:])
+                if st != 0:
+                    break
+        return st

@@ -78,6 +78,7 @@ struct WsLayout {
   Buf status, rows_total, w_rc, n, r, idx, gates, sgate, local_rank, chunk_cnt, chunk_base, expert_cnt,
       expert_off, tile_group, tok_row, row_tok, row_gate, u, up, hmid, o, hs, s, z;
   size_t fwd_bytes = 0;
+  size_t saved_bytes = 0;   // fwd region + SwiGLU pre-activations: what a saved evaluation consists of
   // backward only
   Buf ab, abs, gb, dz, ds, dl, dop, dg_part, tok_dl, row_dl, dup, dush, du, dn, part;
   size_t bwd_bytes = 0;
@@ -130,6 +131,7 @@ static WsLayout plan_workspace(const revffn_moe_desc& D) {
   L.fwd_bytes = off;
   take(L.ab, (size_t)Rp * 2 * I * ts);
   take(L.abs, (size_t)T * 2 * Is * ts);
+  L.saved_bytes = off;
   take(L.gb, (size_t)T * h * ts);
   take(L.dz, (size_t)T * d * ts);
   take(L.ds, (size_t)T * d * ts);
@@ -591,7 +593,7 @@ static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weight
   if (desc->tokens > 0 && (!y1 || !in2 || !out)) return REVFFN_ERR_NULL;
   if (!aligned16(y1) || !aligned16(in2) || !aligned16(out) || (reinterpret_cast<uintptr_t>(ws) & 255u))
     return REVFFN_ERR_ALIGN;
-  if (idx_in && !aligned16(idx_in)) return REVFFN_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(idx_in) | reinterpret_cast<uintptr_t>(idx_out)) & 3u) return REVFFN_ERR_ALIGN;
   if (grads) {
     const float* gs[] = {grads->norm_gamma, grads->w_up, grads->w_down, grads->w_router, grads->b_router,
                          grads->w_gate, grads->w_upx, grads->w_downx, grads->ws_gate, grads->ws_up,
@@ -760,6 +762,103 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
     CK(cudaMemcpyAsync(y2_host, y2, n, cudaMemcpyDeviceToHost, st));
     CK(cudaMemcpyAsync(x2_rec_host, x2r, n, cudaMemcpyDeviceToHost, st));
     CK(cudaMemcpyAsync(dy1_host, dy1, n, cudaMemcpyDeviceToHost, st));
+  }
+  return REVFFN_OK;
+}
+
+int revffn_moe_saved_size(const revffn_moe_desc* desc, size_t* bytes) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  if (!bytes) return REVFFN_ERR_NULL;
+  *bytes = plan_workspace(*desc).saved_bytes;
+  return REVFFN_OK;
+}
+
+// One cache slot of the activation-caching stack: the layer's input stream (rows of
+// ld_stream floats, as in the caller's buffer) followed by a full workspace.
+static size_t stack_stream_slot(const revffn_moe_desc& D) {
+  return (size_t)round_up((int64_t)(D.tokens > 0 ? D.tokens : 1) * D.ld_stream * (int64_t)sizeof(float), 256);
+}
+
+int revffn_moe_stack_cache_stride(const revffn_moe_desc* desc, size_t* bytes) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  if (!bytes) return REVFFN_ERR_NULL;
+  *bytes = stack_stream_slot(*desc) + plan_workspace(*desc).bwd_bytes;
+  return REVFFN_OK;
+}
+
+int revffn_moe_stack_forward(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                             float* stream_a, float* stream_b, int32_t* topk_idx, void* cache, size_t cache_bytes,
+                             void* ws, size_t ws_bytes, void* cuda_stream) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  if (n_blocks < 0) return REVFFN_ERR_SHAPE;
+  if (n_blocks > 0 && !weights) return REVFFN_ERR_NULL;
+  size_t stride = 0;
+  revffn_moe_stack_cache_stride(desc, &stride);
+  if (cache && (cache_bytes < stride * (size_t)n_blocks || (reinterpret_cast<uintptr_t>(cache) & 255u)))
+    return REVFFN_ERR_WORKSPACE;
+  const size_t slot = stack_stream_slot(*desc);
+  const size_t idx_stride = (size_t)desc->tokens * desc->top_k;
+  const size_t ws_need = plan_workspace(*desc).bwd_bytes;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  revffn_moe_desc d = *desc;
+  if (cache) d.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS;
+  // with a cache every layer runs in its own slot: the shared workspace still reports "no error"
+  if (cache && ws && ws_bytes >= 256) CK(cudaMemsetAsync(ws, 0, 256, st));
+  for (int l = 0; l < n_blocks; ++l) {
+    float* P = (l & 1) ? stream_b : stream_a;
+    float* R = (l & 1) ? stream_a : stream_b;
+    void* lws = ws;
+    size_t lws_bytes = ws_bytes;
+    if (cache) {
+      char* c = reinterpret_cast<char*>(cache) + (size_t)l * stride;
+      if (desc->tokens > 0)   // the layer's input stream is overwritten two layers later: keep a copy
+        CK(cudaMemcpy2DAsync(c, (size_t)desc->ld_stream * 4, P, (size_t)desc->ld_stream * 4,
+                             (size_t)(desc->d_model / 2) * 4, (size_t)desc->tokens, cudaMemcpyDeviceToDevice, st));
+      lws = c + slot;
+      lws_bytes = ws_need;
+    }
+    CKR(revffn_moe_forward(&d, &weights[l], P, R, R, topk_idx ? topk_idx + (size_t)l * idx_stride : nullptr, lws,
+                           lws_bytes, cuda_stream));
+  }
+  return REVFFN_OK;
+}
+
+int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                              float* stream_a, float* stream_b, float* grad_a, float* grad_b,
+                              const revffn_moe_grads* grads, const int32_t* topk_idx, void* cache,
+                              size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  if (n_blocks < 0) return REVFFN_ERR_SHAPE;
+  if (n_blocks > 0 && (!weights || !grads)) return REVFFN_ERR_NULL;
+  size_t stride = 0;
+  revffn_moe_stack_cache_stride(desc, &stride);
+  if (cache && (cache_bytes < stride * (size_t)n_blocks || (reinterpret_cast<uintptr_t>(cache) & 255u)))
+    return REVFFN_ERR_WORKSPACE;
+  const size_t slot = stack_stream_slot(*desc);
+  const size_t idx_stride = (size_t)desc->tokens * desc->top_k;
+  const size_t ws_need = plan_workspace(*desc).bwd_bytes;
+  revffn_moe_desc d_inv = *desc, d_bwd = *desc;
+  d_inv.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS;
+  d_bwd.flags |= REVFFN_FLAG_REUSE_ACTIVATIONS;
+  if (cache && ws && ws_bytes >= 256) CK(cudaMemsetAsync(ws, 0, 256, reinterpret_cast<cudaStream_t>(cuda_stream)));
+  for (int l = n_blocks - 1; l >= 0; --l) {
+    float* P = (l & 1) ? stream_b : stream_a;
+    float* R = (l & 1) ? stream_a : stream_b;
+    float* gP = (l & 1) ? grad_b : grad_a;
+    float* gR = (l & 1) ? grad_a : grad_b;
+    const int32_t* idx = topk_idx ? topk_idx + (size_t)l * idx_stride : nullptr;
+    if (cache) {
+      char* c = reinterpret_cast<char*>(cache) + (size_t)l * stride;
+      CKR(revffn_moe_backward(&d_bwd, &weights[l], reinterpret_cast<const float*>(c), gR, gP, &grads[l], idx,
+                              c + slot, ws_need, cuda_stream));
+    } else {
+      CKR(revffn_moe_inverse(&d_inv, &weights[l], P, R, R, idx, ws, ws_bytes, cuda_stream));
+      CKR(revffn_moe_backward(&d_bwd, &weights[l], P, gR, gP, &grads[l], idx, ws, ws_bytes, cuda_stream));
+    }
   }
   return REVFFN_OK;
 }

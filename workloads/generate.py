@@ -143,3 +143,30 @@ def make_streams(cfg: BlockConfig, seed: int = 0) -> Dict[str, np.ndarray]:
     T, h = cfg.tokens, cfg.h
     return {name: _normal((T, h), 1.0, 0.0, seed, 0, name, False)
             for name in ("y1", "x2", "dy2")}
+
+
+def make_weights_device(cfg: BlockConfig, seed: int = 0, block: int = 0, device: str = "cuda") -> Dict[str, torch.Tensor]:
+    """Weights of one block drawn on `device` in their final dtypes (bf16 or fp32 matrices,
+    fp32 norm scale and router bias): same shapes and distributions as `make_weights`, its own
+    seeded streams.  For stacks whose weights are too large to draw on the host in reasonable
+    time; a CPU reference reads the same bytes back with `.cpu()`."""
+    wdt = torch.bfloat16 if cfg.weight_dtype == "bf16" else torch.float32
+    out = {}
+    for name, shape in weight_shapes(cfg).items():
+        g = torch.Generator(device=device)
+        g.manual_seed((int(seed) * 1_000_003 + int(block) * 7919) * 64 + _TENSOR_IDS[name] + (1 << 40))
+        if name == "b_router":
+            out[name] = torch.from_numpy(zipf_router_bias(cfg.n_experts, cfg.zipf_s, seed, block)).to(device)
+            continue
+        n = int(np.prod(shape))
+        # drawn in slices to bound the fp32 scratch of a large tensor
+        t = torch.empty(n, dtype=torch.float32 if name == "norm_gamma" else wdt, device=device)
+        step = 1 << 27
+        for i in range(0, n, step):
+            m = min(step, n - i)
+            v = torch.randn(m, generator=g, device=device, dtype=torch.float32) * 0.02
+            if name == "norm_gamma":
+                v = v + 1.0
+            t[i:i + m] = v.to(t.dtype)
+        out[name] = t.view(shape)
+    return out
