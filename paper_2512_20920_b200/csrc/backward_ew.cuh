@@ -103,6 +103,7 @@ __global__ void colsum_partial_kernel(const T* __restrict__ X, int64_t ldx, cons
   if (c >= cols) return;
   int t0 = b * strip, t1 = min(rows, t0 + strip);
   float acc = 0.f;
+#pragma unroll 8
   for (int t = t0; t < t1; ++t) acc += w[t] * to_f32(X[(int64_t)t * ldx + c]);
   part[(int64_t)b * cols + c] = acc;
 }
@@ -197,6 +198,7 @@ __global__ void dgamma_partial_kernel(const float* __restrict__ dn, const float*
   if (c >= h) return;
   int t0 = b * strip, t1 = min(tokens, t0 + strip);
   float acc = 0.f;
+#pragma unroll 8
   for (int t = t0; t < t1; ++t) acc += dn[(int64_t)t * h + c] * y[(int64_t)t * ld + c] * r[t];
   part[(int64_t)b * h + c] = acc;
 }

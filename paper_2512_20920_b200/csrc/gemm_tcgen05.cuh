@@ -489,8 +489,8 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         }
       } else if constexpr (EPI == EPI_SWIGLU) {
         // columns [0, MMA_N/2) hold the gate projection, [MMA_N/2, MMA_N) the up projection.
-        // H goes out through two alternating 2 KB staging buffers; the optional a|b copy is
-        // written straight from registers (64 contiguous bytes per row and operand).
+        // H goes out through two alternating 2 KB staging buffers; when the a|b copy is wanted too,
+        // a|b and H take turns in the staging area.
         uint32_t r1[32];
         float g[32];
 #pragma unroll 1
@@ -505,15 +505,24 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             f[i] = __uint_as_float(r0[i]);
             g[i] = __uint_as_float(r1[i]);
           }
-          if (p.C1 && m_ok) {
-            bf16* ab = reinterpret_cast<bf16*>(p.C1) + (int64_t)m * p.ldc1;
-            store32_bf16(ab + n, f);
-            store32_bf16(ab + p.N + n, g);
+          if (p.C1) {
+            // the a|b copy goes first, through the whole staging area; H follows once that store has read it
+            if (lane == 0) bulk_wait_read<0>();
+            __syncwarp();
+            stage32_bf16(stg, lane, f);
+            stage32_bf16(stg + 2048, lane, g);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&map_c1, stg_u32, n, y0);
+              tma_store_2d(&map_c1, stg_u32 + 2048, p.N + n, y0);
+              bulk_commit();
+            }
           }
 #pragma unroll
           for (int i = 0; i < 32; ++i) f[i] = swiglu_f(f[i], g[i]);
-          const uint32_t off = (n_grp & 1u) * 2048u;
-          if (lane == 0) bulk_wait_read<1>();
+          const uint32_t off = p.C1 ? 0u : (n_grp & 1u) * 2048u;
+          if (lane == 0) { if (p.C1) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
           __syncwarp();
           stage32_bf16(stg + off, lane, f);
           fence_async_smem();
@@ -768,8 +777,11 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
     if ((reinterpret_cast<uintptr_t>(p.C) & 15u) || (p.ldc * (f32_out ? 4 : 2)) % 16 != 0) return REVFFN_ERR_ALIGN;
     int r = tc_make_out_map(&mc, p.C, f32_out, (uint64_t)p.N, rows, (uint64_t)p.ldc);
     if (r) return r;
-    if (p.epilogue == EPI_SWIGLU && p.C1 && ((reinterpret_cast<uintptr_t>(p.C1) & 15u) || (p.ldc1 * 2) % 16 != 0))
-      return REVFFN_ERR_ALIGN;
+    if (p.epilogue == EPI_SWIGLU && p.C1) {
+      if ((reinterpret_cast<uintptr_t>(p.C1) & 15u) || (p.ldc1 * 2) % 16 != 0) return REVFFN_ERR_ALIGN;
+      r = tc_make_out_map(&mc1, p.C1, false, (uint64_t)2 * p.N, (uint64_t)p.M, (uint64_t)p.ldc1);
+      if (r) return r;
+    }
   }
   int64_t total = (int64_t)P.tiles_m * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
   int grid = (int)(total < s.n_sms ? total : s.n_sms);

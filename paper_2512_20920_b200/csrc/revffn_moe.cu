@@ -86,7 +86,7 @@ struct WsLayout {
   int n_chunks = 0, max_tiles = 0, dg_ld = 0, strips = 0;
 };
 
-constexpr int STRIP = 256;   // tokens per strip in two-pass column reductions
+constexpr int STRIP = 32;    // tokens per strip in two-pass column reductions
 
 static WsLayout plan_workspace(const revffn_moe_desc& D) {
   WsLayout L;
