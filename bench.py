@@ -31,9 +31,13 @@ if ROOT not in sys.path:
 METRIC = "RevFFN MoE block fwd+inverse+bwd tokens/s; % of B200 bf16 tensor peak"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM traffic per launch (bytes) of the dominant kernels from one ncu capture each
-# (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None = not captured.
-NCU_TRAFFIC_BYTES = {}
+# DRAM traffic per launch (bytes) at C1 from one single-pass ncu capture at full size
+# (dram__bytes_read.sum + dram__bytes_write.sum; profiles/traffic_gemm_expert_gate_up_C1.md).
+# Keyed by pass/kernel; anything else, or any other workload, reports null.
+NCU_TRAFFIC_BYTES = {
+    "fwd/gemm_expert_gate_up_swiglu": 937_933_824, "inv/gemm_expert_gate_up_swiglu": 1_127_639_808,
+    "fwd/gemm_shared_gate_up_swiglu": 171_396_864, "inv/gemm_shared_gate_up_swiglu": 476_753_664,
+}
 
 
 def load_peaks():
@@ -323,7 +327,7 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
         peak = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
         roofline = {"bound": "tensor", "kernel": name, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                     "frac": achieved / peak, "peak_source": f"{peak_kind} (sustained bf16 cuBLAS figure)",
-                    "traffic": NCU_TRAFFIC_BYTES.get(kn), "launch_ms": ms / cnt,
+                    "traffic": NCU_TRAFFIC_BYTES.get(name) if cfg.name == "C1" else None, "launch_ms": ms / cnt,
                     "share_of_step": ms / (ms_prof_step * args.steps),
                     "timed_over": f"a second pass of the same {args.steps} steps with a CUDA-event pair around "
                                   f"every launch ({ms_prof_step:.3f} ms per step against {ms_step:.3f} without)"}
