@@ -156,10 +156,13 @@ inline cudaError_t launch_fold_router(const T* w_router, const T* w_sgate, const
 // Router: logits in fp64 from the fp32 stream, top-k by warp shuffles, gates.
 //   block = 256 threads, RT_TOK tokens per block.
 //   phase 1: L[t, e] = r_t <W_rc[e], y_t * gamma> (+ b_r[e]) for e < E; row E is the
-//            shared gate.  y*gamma (fp64) and W_rc are staged chunk-wise, k-major, so
-//            that a thread reads its 4 tokens and 4 experts with 16-byte loads; every
-//            thread owns a 4 x 4 block of dot products and sums over i in ascending
-//            order.  The staging threads also sum y^2 (fp64), which gives
+//            shared gate.  The product runs on the fp64 tensor-core path
+//            (mma.sync m8n8k4): y*gamma (fp64, [token][i]) and W_rc ([expert][i]) are
+//            staged chunk-wise in shared memory, each warp owns a 16-token x 32-expert
+//            block of the 64 x 64 tile as 2 x 4 fragments, and reads 6 operand values
+//            per 8 instructions.  (A register-tiled DFMA version of the same product
+//            spent its time on shared-memory operand reads: 8 values per 16 FMAs.)
+//            The staging threads also sum y^2 (fp64), which gives
 //            r_t = (mean(y_t^2)+eps)^-1/2; the scale is applied to the finished sums.
 //   phase 2: per token, k rounds of warp arg-max (ties -> lowest index), softmax
 //            over the k selected logits, sigmoid of the shared-gate logit.
@@ -168,7 +171,15 @@ inline cudaError_t launch_fold_router(const T* w_router, const T* w_sgate, const
 constexpr int RT_TOK = 64;   // tokens per block
 constexpr int RT_KC = 32;    // k-chunk
 constexpr int RT_EC = 64;    // experts per pass
-constexpr int RT_LD = RT_TOK + 2;   // row stride (doubles) of the staged chunks: even, and not a multiple of 32 banks
+constexpr int RT_LD = RT_KC + 4;    // row stride (doubles) of both staged chunks: rows 4 doubles apart modulo 16 banks,
+                                    // so the 8 rows x 4 columns a fragment load touches fall on distinct banks
+
+// D (8x8) += A (8x4, row-major fragment) * B (4x8, column-major fragment), fp64.
+// Lane l holds A[l/4][l%4], B[l%4][l/4] and D[l/4][2*(l%4) + {0,1}].
+__device__ __forceinline__ void dmma_8x8x4(double& d0, double& d1, double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d0), "+d"(d1) : "d"(a), "d"(b));
+}
 
 __global__ void __launch_bounds__(256)
 router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restrict__ gamma, float eps,
@@ -178,23 +189,22 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
                    int32_t* __restrict__ idx_user) {
   extern __shared__ __align__(16) double smem_d[];
   const int EP = E + 1;                       // logits per token incl. the shared-gate row
-  double* ns = smem_d;                        // [RT_KC][RT_LD]   n chunk, k-major
-  double* ws = ns + RT_KC * RT_LD;            // [RT_KC][RT_LD]   W_rc chunk, k-major (RT_EC == RT_TOK)
-  double* rs = ws + RT_KC * RT_LD;            // [RT_TOK]
+  double* ns = smem_d;                        // [RT_TOK][RT_LD]  stream chunk, one row per token
+  double* ws = ns + RT_TOK * RT_LD;           // [RT_EC][RT_LD]   W_rc chunk, one row per expert
+  double* rs = ws + RT_EC * RT_LD;            // [RT_TOK]
   double* Ls = rs + RT_TOK;                   // [RT_TOK][EP]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t0 = blockIdx.x * RT_TOK;
 
-  // phase 1: logits.  16 x 16 threads, each 4 tokens x 4 experts; a warp spans 4 expert
-  // groups x 8 token groups, which keeps its shared-memory reads within few wavefronts.
-  const int tx = (warp & 3) * 4 + (lane & 3);       // expert group: experts e0 + 4 tx .. + 3
-  const int ty = (warp >> 2) * 8 + (lane >> 2);     // token group: tokens 4 ty .. + 3
+  // phase 1: logits.  Warp (wm, wn) owns tokens 16 wm .. +15 and experts e0 + 32 wn .. +31.
+  const int wm = warp >> 1, wn = warp & 1;
+  const int fr = lane >> 2, fc = lane & 3;          // fragment row / column of this lane
   for (int e0 = 0; e0 < EP; e0 += RT_EC) {
-    double acc[4][4];
+    double acc[2][4][2];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int a = 0; a < 2; ++a)
 #pragma unroll
-      for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+      for (int b = 0; b < 4; ++b) { acc[a][b][0] = 0.0; acc[a][b][1] = 0.0; }
     // Register prefetch: the global loads of chunk c+1 are in flight while chunk c is summed.
     //   y:    RT_TOK x RT_KC floats  = 2 float4 per thread  (token tt, 4 consecutive i)
     //   W_rc: RT_EC x RT_KC doubles  = 4 double2 per thread (expert ee, 2 consecutive i)
@@ -230,36 +240,31 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
         if (gamma && !norm_none && i < h) g = *reinterpret_cast<const float4*>(gamma + i);
         const double v0 = (double)py[q].x, v1 = (double)py[q].y, v2 = (double)py[q].z, v3 = (double)py[q].w;
         ss[q] += v0 * v0; ss[q] += v1 * v1; ss[q] += v2 * v2; ss[q] += v3 * v3;
-        ns[(kq + 0) * RT_LD + tt] = v0 * (double)g.x;
-        ns[(kq + 1) * RT_LD + tt] = v1 * (double)g.y;
-        ns[(kq + 2) * RT_LD + tt] = v2 * (double)g.z;
-        ns[(kq + 3) * RT_LD + tt] = v3 * (double)g.w;
+        double2* dst = reinterpret_cast<double2*>(ns + tt * RT_LD + kq);
+        dst[0] = make_double2(v0 * (double)g.x, v1 * (double)g.y);
+        dst[1] = make_double2(v2 * (double)g.z, v3 * (double)g.w);
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         int idx = tid + q * 256;
         int ee = idx / (RT_KC / 2), kq = (idx % (RT_KC / 2)) * 2;
-        ws[(kq + 0) * RT_LD + ee] = pw[q].x;
-        ws[(kq + 1) * RT_LD + ee] = pw[q].y;
+        *reinterpret_cast<double2*>(ws + ee * RT_LD + kq) = pw[q];
       }
       __syncthreads();
       if (k0 + RT_KC < h) prefetch(k0 + RT_KC);
-      // operands of step kk+1 are read from shared memory before the sums of step kk are issued
-      const double2* n2 = reinterpret_cast<const double2*>(ns + ty * 4);
-      const double2* w2 = reinterpret_cast<const double2*>(ws + tx * 4);
-      double2 n01 = n2[0], n23 = n2[1], w01 = w2[0], w23 = w2[1];
+      const double* ap = ns + (wm * 16 + fr) * RT_LD + fc;
+      const double* bp = ws + (wn * 32 + fr) * RT_LD + fc;
 #pragma unroll
-      for (int kk = 0; kk < RT_KC; ++kk) {
-        const double nv[4] = {n01.x, n01.y, n23.x, n23.y};
-        const double wv[4] = {w01.x, w01.y, w23.x, w23.y};
-        if (kk + 1 < RT_KC) {
-          n01 = n2[(kk + 1) * (RT_LD / 2)]; n23 = n2[(kk + 1) * (RT_LD / 2) + 1];
-          w01 = w2[(kk + 1) * (RT_LD / 2)]; w23 = w2[(kk + 1) * (RT_LD / 2) + 1];
-        }
+      for (int kk = 0; kk < RT_KC; kk += 4) {
+        double af[2], bf[4];
 #pragma unroll
-        for (int a = 0; a < 4; ++a)
+        for (int a = 0; a < 2; ++a) af[a] = ap[a * 8 * RT_LD + kk];
 #pragma unroll
-          for (int b = 0; b < 4; ++b) acc[a][b] += nv[a] * wv[b];
+        for (int b = 0; b < 4; ++b) bf[b] = bp[b * 8 * RT_LD + kk];
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+          for (int b = 0; b < 4; ++b) dmma_8x8x4(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
       }
       __syncthreads();
     }
@@ -274,20 +279,23 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
     }
     __syncthreads();
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int a = 0; a < 2; ++a)
 #pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        int e = e0 + tx * 4 + b;
-        if (e < EP) {
-          double v = acc[a][b] * rs[ty * 4 + a];
-          if (e < E && b_router) v += (double)b_router[e];
-          Ls[(ty * 4 + a) * EP + e] = v;
+      for (int b = 0; b < 4; ++b)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const int tt = wm * 16 + a * 8 + fr;
+          const int e = e0 + wn * 32 + b * 8 + 2 * fc + c;
+          if (e < EP) {
+            double v = acc[a][b][c] * rs[tt];
+            if (e < E && b_router) v += (double)b_router[e];
+            Ls[tt * EP + e] = v;
+          }
         }
-      }
   }
   __syncthreads();
 
-  // phase 2: top-k and gates; one warp per token, 8 tokens per warp
+  // phase 2: top-k and gates; one warp per token
   for (int tt = warp; tt < RT_TOK; tt += 8) {
     int t = t0 + tt;
     if (t >= tokens) continue;
@@ -295,11 +303,15 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
     double sel[8];
     int seli[8];
     if (idx_in) {
-      for (int s = 0; s < k; ++s) { seli[s] = idx_in[(int64_t)t * k + s]; sel[s] = L[seli[s]]; }
+#pragma unroll
+      for (int s = 0; s < 8; ++s)
+        if (s < k) { seli[s] = idx_in[(int64_t)t * k + s]; sel[s] = L[seli[s]]; }
     } else {
       // candidates of this lane: e = lane + 32 j
       unsigned taken = 0u;                    // bit j set: candidate j already selected
-      for (int s = 0; s < k; ++s) {
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        if (s >= k) break;
         double best = __longlong_as_double(0xfff0000000000000LL);   // -inf
         int besti = 0x7fffffff;
         for (int j = 0; lane + 32 * j < E; ++j) {
@@ -320,23 +332,37 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
         if ((besti & 31) == lane) taken |= 1u << (besti >> 5);
       }
     }
-    if (lane == 0) {
-      double m = sel[0];
-      for (int s = 1; s < k; ++s) m = fmax(m, sel[s]);
-      double den = 0.0, ex[8];
-      for (int s = 0; s < k; ++s) { ex[s] = exp(sel[s] - m); den += ex[s]; }
-      for (int s = 0; s < k; ++s) {
-        idx_out[(int64_t)t * k + s] = seli[s];
-        if (idx_user) idx_user[(int64_t)t * k + s] = seli[s];
-        gate_out[(int64_t)t * k + s] = (float)(ex[s] / den);
+    // gates: lane s < k takes slot s, lane k the shared gate.  The softmax runs in fp32 on the fp64
+    // differences to the largest selected logit (the decision above is fp64; the weights are fp32 outputs).
+    double m = sel[0], mine = sel[0];
+    int mine_i = seli[0];
+#pragma unroll
+    for (int s = 1; s < 8; ++s) {
+      if (s < k) {
+        m = fmax(m, sel[s]);
+        if (lane == s) { mine = sel[s]; mine_i = seli[s]; }
       }
-      sgate_out[t] = has_shared ? (float)(1.0 / (1.0 + exp(-L[E]))) : 0.f;
+    }
+    float x = 0.f;
+    if (lane < k) x = (float)(mine - m);
+    else if (lane == k) x = (float)(-L[E]);
+    const float ev = expf(x);
+    float den = (lane < k) ? ev : 0.f;
+    den += __shfl_xor_sync(0xffffffffu, den, 1);
+    den += __shfl_xor_sync(0xffffffffu, den, 2);
+    den += __shfl_xor_sync(0xffffffffu, den, 4);      // k <= 8: lanes 0..7 hold the sum
+    if (lane < k) {
+      idx_out[(int64_t)t * k + lane] = mine_i;
+      if (idx_user) idx_user[(int64_t)t * k + lane] = mine_i;
+      gate_out[(int64_t)t * k + lane] = ev / den;
+    } else if (lane == k) {
+      sgate_out[t] = has_shared ? 1.f / (1.f + ev) : 0.f;
     }
   }
 }
 
 inline size_t router_smem_bytes(int E) {
-  return sizeof(double) * ((size_t)2 * RT_KC * RT_LD + RT_TOK + (size_t)RT_TOK * (E + 1));
+  return sizeof(double) * ((size_t)(RT_TOK + RT_EC) * RT_LD + RT_TOK + (size_t)RT_TOK * (E + 1));
 }
 
 // Raises the kernel's dynamic shared-memory limit when the logits of a block do not
