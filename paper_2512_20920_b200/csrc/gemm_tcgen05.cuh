@@ -197,17 +197,10 @@ __device__ __forceinline__ void load32_bf16(const bf16* src, float* f) {
   for (int i = 0; i < 4; ++i) unpack8(s[i], f + 8 * i);
 }
 
-// Output staging.  A warp stages a 32-row x 32-column block, one row per lane, in the
-// layout the store's tensor map expects: rows of 128 bytes (fp32) under the 128-byte
-// swizzle, rows of 64 bytes (bf16) under the 64-byte swizzle.  `buf` is aligned to the
-// swizzle period, so the 16-byte piece j of row r lands at piece j ^ (r & 7), or
-// j ^ ((r >> 1) & 3); lanes of one store instruction then hit distinct banks.
-__device__ __forceinline__ void stage32_f32(uint8_t* buf, int r, const float* f) {
-  uint8_t* row = buf + r * 128;
-#pragma unroll
-  for (int j = 0; j < 8; ++j)
-    *reinterpret_cast<float4*>(row + ((j ^ (r & 7)) << 4)) = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
-}
+// Output staging.  A warp stages a 32-row x 32-column bf16 block, one row per lane, in the layout
+// the store's tensor map expects: rows of 64 bytes under the 64-byte swizzle.  `buf` is aligned to
+// the swizzle period, so the 16-byte piece j of row r lands at piece j ^ ((r >> 1) & 3); lanes of
+// one store instruction then hit distinct banks.
 __device__ __forceinline__ void stage32_bf16(uint8_t* buf, int r, const float* f) {
   uint8_t* row = buf + r * 64;
 #pragma unroll
@@ -472,20 +465,54 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
               }
             }
           }
-          // fp32 blocks fill the staging area (4 KB): the previous store must have read it;
-          // bf16 blocks (2 KB) alternate between its halves
-          const uint32_t off = f32_out ? 0u : (n_grp & 1u) * 2048u;
-          if (lane == 0) { if (f32_out) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
-          __syncwarp();
-          if (f32_out) stage32_f32(stg + off, lane, f); else stage32_bf16(stg + off, lane, f);
-          fence_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-            if (EPI == EPI_WGRAD && p.accumulate) tma_reduce_add_2d(&map_c, stg_u32 + off, n, y0);
-            else tma_store_2d(&map_c, stg_u32 + off, n, y0);
-            bulk_commit();
+          // bf16 blocks (32 x 32, 2 KB) leave through two alternating staging buffers and TMA stores.
+          // fp32 blocks (32 x 32, 4 KB) are transposed through the staging area and written with plain
+          // 16-byte stores, 4 rows x 128 bytes per instruction: whole lines, and nothing to wait for
+          // before the area is reused.  (A TMA store of such a block sat behind the producer's operand
+          // loads in the copy engine; with the short K of a weight gradient that wait set the pace.)
+          if (f32_out) {
+            if (lane == 0) bulk_wait_read<0>();     // no bulk store of this warp reads the area any more
+            __syncwarp();
+            {
+              uint8_t* row = stg + lane * 128;
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<float4*>(row + ((j ^ (lane & 7)) << 4)) =
+                    make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+            }
+            __syncwarp();
+            const int piece = lane & 7;
+            const int64_t y_lim = (p.group_mode == GROUP_K) ? (int64_t)(t.group + 1) * p.M
+                                                            : (p.group_mode == GROUP_M ? (int64_t)m_lim : (int64_t)p.M);
+            float* cbase = reinterpret_cast<float*>(p.C) + n + piece * 4;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r = i * 4 + (lane >> 3);
+              const float4 v = *reinterpret_cast<const float4*>(stg + r * 128 + ((piece ^ (r & 7)) << 4));
+              if ((int64_t)y0 + r < y_lim) {
+                float4* o = reinterpret_cast<float4*>(cbase + ((int64_t)y0 + r) * p.ldc);
+                if (EPI == EPI_WGRAD && p.accumulate) {
+                  float4 old = *o;
+                  *o = make_float4(old.x + v.x, old.y + v.y, old.z + v.z, old.w + v.w);
+                } else {
+                  *o = v;
+                }
+              }
+            }
+            __syncwarp();
+          } else {
+            const uint32_t off = (n_grp & 1u) * 2048u;
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+            stage32_bf16(stg + off, lane, f);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&map_c, stg_u32 + off, n, y0);
+              bulk_commit();
+            }
+            ++n_grp;
           }
-          ++n_grp;
         }
       } else if constexpr (EPI == EPI_SWIGLU) {
         // columns [0, MMA_N/2) hold the gate projection, [MMA_N/2, MMA_N) the up projection.
@@ -685,16 +712,16 @@ inline int tc_make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64
   return r == CUDA_SUCCESS ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
 
-// Tensor map of an epilogue output: boxes of 32 rows x 32 columns, fp32 (128-byte rows,
-// 128-byte swizzle) or bf16 (64-byte rows, 64-byte swizzle).
+// Tensor map of an epilogue output: boxes of 32 rows x 64 bytes (32 bf16 or 16 fp32 columns),
+// 64-byte swizzle.
 inline int tc_make_out_map(CUtensorMap* map, const void* ptr, bool f32, uint64_t inner, uint64_t outer, uint64_t ld) {
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {ld * (f32 ? 4u : 2u)};
-  cuuint32_t box[2] = {32, 32};
+  cuuint32_t box[2] = {f32 ? 16u : 32u, 32};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = tc_state().encode(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                                  const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                 f32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                                 CU_TENSOR_MAP_SWIZZLE_64B,
                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
