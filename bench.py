@@ -284,7 +284,9 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
         slot = ((hy1.numel() * 4 + 255) // 256) * 256
         staging = torch.empty(6 * slot, dtype=torch.uint8, device="cuda")
         g_struct = blk.grads_struct(grads)
-        host_step = lambda: rv.revffn_moe_step_host(blk.desc, blk.w, g_struct, hy1, hx2, hdy2, hy2, hx2r, hdy1, staging, blk.ws)
+        copy_stream = torch.cuda.Stream()
+        host_step = lambda: rv.revffn_moe_step_host(blk.desc, blk.w, g_struct, hy1, hx2, hdy2, hy2, hx2r, hdy1, staging,
+                                                    blk.ws, copy_stream=copy_stream.cuda_stream)
         for _ in range(2):
             host_step()
         barrier()

@@ -231,13 +231,18 @@ int revffn_moe_saved_size(const revffn_moe_desc* desc, size_t* bytes);
  * the reconstructed x2 and dy1 back to the host buffers.  `staging` is caller-owned
  * device memory of at least 6 * round_up(T*h*4, 256) bytes, 256-byte aligned;
  * requires ld_stream == h.  Asynchronous on the stream like the other entry
- * points: synchronise the stream before reading the host outputs.
- * (Convenience for end-to-end timing; no paper counterpart.)
+ * points: synchronise cuda_stream before reading the host outputs.
+ * copy_stream: NULL, or a second stream of the caller's on which the transfers that a
+ * pass does not need at once run beside the passes (dy2 in during forward and inverse,
+ * y2 out during the inverse pass, the reconstructed x2 out during backward).  The call
+ * orders the two streams with events (five per device, created on its first use); when it
+ * returns, work queued on cuda_stream afterwards follows everything of this step.
+ * (Convenience for end-to-end use; no paper counterpart.)
  */
 int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* w, const revffn_moe_grads* grads,
                          const float* y1_host, const float* x2_host, const float* dy2_host, float* y2_host,
                          float* x2_rec_host, float* dy1_host, void* staging, size_t staging_bytes, void* ws,
-                         size_t ws_bytes, void* cuda_stream);
+                         size_t ws_bytes, void* cuda_stream, void* copy_stream);
 
 /*
  * Routing only, for callers that must not allocate.  (The paper has no

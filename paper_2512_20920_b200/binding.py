@@ -74,7 +74,7 @@ def _load() -> C.CDLL:
     lib.revffn_moe_ws_lookup.argtypes = [C.POINTER(Desc), C.c_char_p, C.POINTER(sz), C.POINTER(sz)]
     lib.revffn_dbg_gemm.argtypes = [C.POINTER(DbgGemmArgs), vp, vp]
     lib.revffn_moe_step_host.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.POINTER(Grads), vp, vp, vp, vp, vp, vp,
-                                         vp, sz, vp, sz, vp]
+                                         vp, sz, vp, sz, vp, vp]
     lib.revffn_moe_saved_size.argtypes = [C.POINTER(Desc), C.POINTER(sz)]
     lib.revffn_moe_stack_cache_stride.argtypes = [C.POINTER(Desc), C.POINTER(sz)]
     lib.revffn_moe_stack_forward.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp, sz, vp, sz, vp]
@@ -154,12 +154,14 @@ def revffn_moe_status(ws, stream: Optional[int] = None) -> int:
 
 
 def revffn_moe_step_host(desc: Desc, w: Weights, grads: Grads, y1_host, x2_host, dy2_host, y2_host, x2_rec_host,
-                         dy1_host, staging, ws, stream: Optional[int] = None):
-    """Host-resident streams (pinned CPU tensors) in and out; see the header."""
+                         dy1_host, staging, ws, stream: Optional[int] = None, copy_stream: Optional[int] = None):
+    """Host-resident streams (pinned CPU tensors) in and out; see the header.  copy_stream: raw handle of a
+    second CUDA stream for the transfers that can run beside the passes, or None."""
     _check(lib.revffn_moe_step_host(C.byref(desc), C.byref(w), C.byref(grads), _ptr(y1_host), _ptr(x2_host),
                                     _ptr(dy2_host), _ptr(y2_host), _ptr(x2_rec_host), _ptr(dy1_host), _ptr(staging),
                                     staging.numel() * staging.element_size(), _ptr(ws),
-                                    ws.numel() * ws.element_size(), stream if stream is not None else _stream()),
+                                    ws.numel() * ws.element_size(), stream if stream is not None else _stream(),
+                                    copy_stream),
            "revffn_moe_step_host")
 
 

@@ -725,10 +725,26 @@ int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* 
   return REVFFN_ERR_UNSUPPORTED;
 }
 
+// Events that order the copy stream against the compute stream in revffn_moe_step_host
+// (created on first use, per device; no timing).
+static cudaEvent_t* step_events(int* err) {
+  static cudaEvent_t ev[64][5];
+  static bool made[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = REVFFN_ERR_CUDA; return nullptr; }
+  if (!made[dev]) {
+    for (int i = 0; i < 5; ++i)
+      if (cudaEventCreateWithFlags(&ev[dev][i], cudaEventDisableTiming) != cudaSuccess) { *err = REVFFN_ERR_CUDA; return nullptr; }
+    made[dev] = true;
+  }
+  *err = REVFFN_OK;
+  return ev[dev];
+}
+
 int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* w, const revffn_moe_grads* grads,
                          const float* y1_host, const float* x2_host, const float* dy2_host, float* y2_host,
                          float* x2_rec_host, float* dy1_host, void* staging, size_t staging_bytes, void* ws,
-                         size_t ws_bytes, void* cuda_stream) {
+                         size_t ws_bytes, void* cuda_stream, void* copy_stream) {
   int r = validate_desc(desc);
   if (r != REVFFN_OK) return r;
   if (!y1_host || !x2_host || !dy2_host || !y2_host || !x2_rec_host || !dy1_host || !staging) return REVFFN_ERR_NULL;
@@ -738,6 +754,14 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
   const size_t slot = (size_t)round_up((int64_t)(n > 0 ? n : 1), 256);
   if (staging_bytes < 6 * slot || (reinterpret_cast<uintptr_t>(staging) & 255u)) return REVFFN_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(copy_stream);
+  const bool two = copy_stream != nullptr && cs != st;
+  if (!two) cs = st;
+  cudaEvent_t* ev = nullptr;
+  if (two) {
+    ev = step_events(&r);
+    if (r != REVFFN_OK) return r;
+  }
   char* sp = reinterpret_cast<char*>(staging);
   float* y1 = reinterpret_cast<float*>(sp);
   float* x2 = reinterpret_cast<float*>(sp + slot);
@@ -745,23 +769,41 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
   float* y2 = reinterpret_cast<float*>(sp + 3 * slot);
   float* x2r = reinterpret_cast<float*>(sp + 4 * slot);
   float* dy1 = reinterpret_cast<float*>(sp + 5 * slot);
-  if (n > 0) {
-    CK(cudaMemcpyAsync(y1, y1_host, n, cudaMemcpyHostToDevice, st));
-    CK(cudaMemcpyAsync(x2, x2_host, n, cudaMemcpyHostToDevice, st));
-    CK(cudaMemcpyAsync(dy2, dy2_host, n, cudaMemcpyHostToDevice, st));
-    CK(cudaMemsetAsync(dy1, 0, n, st));
-  }
   // the inverse and the gradient pass share one evaluation of the branch
   revffn_moe_desc d_inv = *desc, d_bwd = *desc;
   d_inv.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS;
   d_bwd.flags |= REVFFN_FLAG_REUSE_ACTIVATIONS;
-  CKR(revffn_moe_forward(desc, w, y1, x2, y2, nullptr, ws, ws_bytes, cuda_stream));
-  CKR(revffn_moe_inverse(&d_inv, w, y1, y2, x2r, nullptr, ws, ws_bytes, cuda_stream));
-  CKR(revffn_moe_backward(&d_bwd, w, y1, dy2, dy1, grads, nullptr, ws, ws_bytes, cuda_stream));
+  // With a copy stream, what a pass does not need right away travels beside the passes: dy2 comes in
+  // during forward and inverse, y2 goes out during the inverse pass, the reconstructed x2 during backward.
+  if (two) {
+    CK(cudaEventRecord(ev[0], st));            // everything queued on the compute stream so far (earlier steps
+    CK(cudaStreamWaitEvent(cs, ev[0], 0));     // may still use the staging buffers)
+  }
   if (n > 0) {
-    CK(cudaMemcpyAsync(y2_host, y2, n, cudaMemcpyDeviceToHost, st));
-    CK(cudaMemcpyAsync(x2_rec_host, x2r, n, cudaMemcpyDeviceToHost, st));
-    CK(cudaMemcpyAsync(dy1_host, dy1, n, cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(y1, y1_host, n, cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(x2, x2_host, n, cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(dy2, dy2_host, n, cudaMemcpyHostToDevice, cs));
+    CK(cudaMemsetAsync(dy1, 0, n, st));
+  }
+  if (two) CK(cudaEventRecord(ev[1], cs));     // dy2 is on the device
+  CKR(revffn_moe_forward(desc, w, y1, x2, y2, nullptr, ws, ws_bytes, cuda_stream));
+  if (two) {
+    CK(cudaEventRecord(ev[2], st));
+    CK(cudaStreamWaitEvent(cs, ev[2], 0));
+  }
+  if (n > 0) CK(cudaMemcpyAsync(y2_host, y2, n, cudaMemcpyDeviceToHost, cs));
+  CKR(revffn_moe_inverse(&d_inv, w, y1, y2, x2r, nullptr, ws, ws_bytes, cuda_stream));
+  if (two) {
+    CK(cudaEventRecord(ev[3], st));
+    CK(cudaStreamWaitEvent(cs, ev[3], 0));
+  }
+  if (n > 0) CK(cudaMemcpyAsync(x2_rec_host, x2r, n, cudaMemcpyDeviceToHost, cs));
+  if (two) CK(cudaStreamWaitEvent(st, ev[1], 0));
+  CKR(revffn_moe_backward(&d_bwd, w, y1, dy2, dy1, grads, nullptr, ws, ws_bytes, cuda_stream));
+  if (n > 0) CK(cudaMemcpyAsync(dy1_host, dy1, n, cudaMemcpyDeviceToHost, st));
+  if (two) {
+    CK(cudaEventRecord(ev[4], cs));            // the compute stream's completion covers the copy stream's work
+    CK(cudaStreamWaitEvent(st, ev[4], 0));
   }
   return REVFFN_OK;
 }

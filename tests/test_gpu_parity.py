@@ -247,3 +247,32 @@ def test_backward_reuses_a_saved_evaluation(rv, simt):
     small = torch.empty(blk.fwd_bytes, dtype=torch.uint8, device="cuda")
     with pytest.raises(rv.RevffnError):
         blk.forward(y1, x2, save=True, ws=small)
+
+
+@pytest.mark.parametrize("two_streams", [False, True])
+def test_host_step_matches_the_device_entry_points(rv, two_streams):
+    """The host-buffer step (copies in, three passes, copies out; optionally with a second stream for the
+    transfers) returns exactly what the three device entry points return."""
+    cfg = small_cfg(tokens=500)
+    w, s = scaled_weights(cfg, 8, 4.0), make_streams(cfg, 8)
+    blk = make_block(cfg, w)
+    y1, x2, dy2 = dev(s["y1"]), dev(s["x2"]), dev(s["dy2"])
+    y2 = blk.forward(y1, x2)
+    x2r = blk.inverse(y1, y2)
+    dy1, g_ref = torch.zeros_like(y1), grad_buffers(cfg, w)
+    blk.backward(y1, dy2, dy1, g_ref)
+    pin = lambda a: torch.from_numpy(a).pin_memory()
+    hy1, hx2, hdy2 = pin(s["y1"]), pin(s["x2"]), pin(s["dy2"])
+    hy2, hx2r, hdy1 = (torch.empty_like(hy1).pin_memory() for _ in range(3))
+    slot = ((hy1.numel() * 4 + 255) // 256) * 256
+    staging = torch.empty(6 * slot, dtype=torch.uint8, device="cuda")
+    g = grad_buffers(cfg, w)
+    cs = torch.cuda.Stream() if two_streams else None
+    for _ in range(2):      # twice: the second step starts while the first one's copies may still be in flight
+        rv.revffn_moe_step_host(blk.desc, blk.w, blk.grads_struct(g), hy1, hx2, hdy2, hy2, hx2r, hdy1, staging, blk.ws,
+                                copy_stream=cs.cuda_stream if cs is not None else None)
+    torch.cuda.synchronize()
+    assert blk.status() == 0
+    assert torch.equal(hy2, y2.cpu()) and torch.equal(hx2r, x2r.cpu()) and torch.equal(hdy1, dy1.cpu())
+    for n in g:
+        assert torch.equal(g[n], g_ref[n]), n
