@@ -49,6 +49,7 @@ struct GemmProblem {
   const int32_t* group_off; const int32_t* tile_group; const int32_t* rows_total;
   int64_t b_group_stride, c_group_stride;
   int a_col0, b_col0;
+  int no_pair;        // tcgen05 back end: never pair CTAs for this product
   int* status;
 };
 

@@ -21,6 +21,14 @@
 // Both operands may be K-major or MN-major; MN-major tiles are fetched as
 // 64x64 boxes and described to the tensor core with leading/stride offsets.
 // Every wait is bounded; on expiry the kernel sets the status word and leaves.
+//
+// Pair mode (template flag PAIR; dense and K-grouped problems whose N is a multiple of 256):
+// the grid is launched as clusters of two CTAs that work one 256 x 256 tile together with
+// tcgen05.mma.cta_group::2.  Each CTA loads its own 128 rows of A and ITS HALF of B's columns
+// (the tensor core reads both halves across the pair), so a K step costs a CTA 32 KB of operand
+// traffic instead of 48 KB and six stages fit.  The even CTA issues the MMAs; its commits
+// arrive on the barriers of both CTAs, both CTAs' loads complete on its "full" barriers, and
+// both CTAs' epilogue warps release its accumulator barriers.
 #pragma once
 
 #include <cuda.h>
@@ -39,12 +47,12 @@ constexpr int TC_EPI_WARPS = 8;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
 constexpr long long TC_WAIT_CYCLES = 4000000000LL;       // ~2 s: bound on any single wait
 
-template <int MMA_N, int EPI> struct TcCfg {
-  static constexpr int B_BYTES = MMA_N * TC_BK * 2;
+template <int MMA_N, int EPI, bool PAIR> struct TcCfg {
+  static constexpr int B_BYTES = (PAIR ? MMA_N / 2 : MMA_N) * TC_BK * 2;
   static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
   // The SwiGLU-backward epilogue streams its a|b operands through shared memory as well
-  // and gets a larger staging area at the price of one pipeline stage.
-  static constexpr int STAGES = (EPI == EPI_DSWIGLU) ? 3 : 4;
+  // and gets a larger staging area at the price of pipeline stages.
+  static constexpr int STAGES = PAIR ? ((EPI == EPI_DSWIGLU) ? 4 : 6) : ((EPI == EPI_DSWIGLU) ? 3 : 4);
   static constexpr int EPI_WARP_BYTES = (EPI == EPI_DSWIGLU) ? 10240 : 4096;   // staging per epilogue warp
   static constexpr int TMEM_COLS = 2 * MMA_N;           // two accumulators; a power of two >= 32
   // stage ring | epilogue staging | barriers; the ring starts 1024-byte aligned and
@@ -128,6 +136,44 @@ template <int N> __device__ __forceinline__ void bulk_wait_read() {
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Orders this thread's shared-memory writes before later async-proxy (TMA) reads of them.
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Pair mode: the same load, completing on a barrier that may live in the partner CTA (cluster address).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Cluster-wide address of the location `addr` (own shared window) in the CTA of rank `rank`.
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+// All threads of both CTAs of the pair.
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Pair mode: arrive on the barrier at this shared-memory offset in both CTAs once the MMAs issued so far are done.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -214,9 +260,12 @@ struct TcTile {
   bool valid;
 };
 
-__device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_dev) {
+// pair_rank < 0: one CTA per 128-row tile.  pair_rank 0 / 1: w counts 256-row tiles worked by two CTAs,
+// this CTA takes rows 128 * pair_rank .. + 127 of it (rows past M are loaded as zeros and never stored).
+__device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_dev, int pair_rank = -1) {
   TcTile t;
   const GemmProblem& p = P.p;
+  if (pair_rank >= 0) tiles_m_dev = (tiles_m_dev + 1) / 2;
   int per_group = tiles_m_dev * P.tiles_n;
   t.group = 0;
   t.krow0 = 0;
@@ -234,7 +283,7 @@ __device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_
     t.k_blocks = (k1 - k0) / TC_BK;
   }
   int tm = r / P.tiles_n, tn = r - tm * P.tiles_n;
-  t.m0 = tm * TC_BM;
+  t.m0 = (pair_rank >= 0) ? tm * 2 * TC_BM + pair_rank * TC_BM : tm * TC_BM;
   t.n0 = tn * P.tile_n;
   t.ncols = (p.concat == CONCAT_N) ? 2 * P.tile_n : min(P.tile_n, p.N - t.n0);
   if (p.group_mode == GROUP_M) t.group = p.tile_group[tm];
@@ -244,12 +293,12 @@ __device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_
 // ---------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------
-template <int MMA_N, int EPI>
+template <int MMA_N, int EPI, bool PAIR>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUtensorMap map_a,
                const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_c1) {
-  using Cfg = TcCfg<MMA_N, EPI>;
+  using Cfg = TcCfg<MMA_N, EPI, PAIR>;
   extern __shared__ uint8_t smem_raw[];
   const GemmProblem& p = P.p;
   const uint32_t raw = smem_u32(smem_raw);
@@ -266,22 +315,33 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   int* issued = reinterpret_cast<int*>(tmem_slot + 2);   // [STAGES] parity+1 of the last load issued per stage
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int crank = PAIR ? (int)cluster_ctarank() : 0;     // rank in the pair; rank 0 issues the MMAs
+  const int prank = PAIR ? crank : -1;
+  const int w0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // first tile and tile stride of this CTA / pair
+  const int wstride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); issued[s] = 0; }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), TC_EPI_WARPS); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), PAIR ? 2 * TC_EPI_WARPS : TC_EPI_WARPS); }
     for (int a = 0; a < 2 * TC_EPI_WARPS; ++a) mbar_init(epi_bar(a / 2, a % 2), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (PAIR) {      // the same warp of both CTAs, the same shared-memory offset
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();      // the partner's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -294,14 +354,44 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int w = blockIdx.x; ok; w += gridDim.x) {
-        TcTile t = tc_tile(P, w, tiles_m_dev);
+      for (int w = w0; ok; w += wstride) {
+        TcTile t = tc_tile(P, w, tiles_m_dev, prank);
         if (!t.valid) break;
         const int k_half = t.k_blocks / 2;
         for (int kb = 0; kb < t.k_blocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
           const uint32_t sb = sa + TC_A_BYTES;
+          if constexpr (PAIR) {
+            // both CTAs' loads complete on the even CTA's barrier, which expects the bytes of both
+            const uint32_t fbc = mapa_u32(full_bar(stage), 0);
+            if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
+            if (!p.a_mn_major) {
+              tma_load_2d_pair(sa, &map_a, kb * TC_BK, t.m0, fbc);
+            } else {
+              const int krow = t.krow0 + kb * TC_BK;
+#pragma unroll
+              for (int j = 0; j < 2; ++j) tma_load_2d_pair(sa + j * 8192, &map_a, p.a_col0 + t.m0 + 64 * j, krow, fbc);
+            }
+            const CUtensorMap* mbp = &map_b0;
+            int kbp = kb;
+            if (p.concat == CONCAT_K && kb >= k_half) { mbp = &map_b1; kbp = kb - k_half; }
+            if (!p.b_mn_major) {
+              // this CTA's 128 of the 256 accumulator columns: gate rows (rank 0) or up rows (rank 1) of a
+              // SwiGLU pair, else rows n0 + 128 rank .. + 127 of B
+              if (p.concat == CONCAT_N) tma_load_2d_pair(sb, crank == 0 ? &map_b0 : &map_b1, kbp * TC_BK, t.n0, fbc);
+              else tma_load_2d_pair(sb, mbp, kbp * TC_BK, t.n0 + 128 * crank, fbc);
+            } else {
+              const int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
+              (void)kdim;
+              const int krow = t.krow0 + kbp * TC_BK;
+#pragma unroll
+              for (int j = 0; j < 2; ++j)
+                tma_load_2d_pair(sb + j * 8192, mbp, p.b_col0 + t.n0 + 128 * crank + 64 * j, krow, fbc);
+            }
+            if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           const uint32_t fb = full_bar(stage);
           mbar_expect_tx(fb, TC_A_BYTES + t.ncols * TC_BK * 2);
           issued[stage] = (int)phase + 1;
@@ -347,8 +437,8 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       uint32_t phase = 0;
       bool ok = true;
       int it = 0;
-      for (int w = blockIdx.x; ok; w += gridDim.x, ++it) {
-        TcTile t = tc_tile(P, w, tiles_m_dev);
+      for (int w = w0; ok && crank == 0; w += wstride, ++it) {
+        TcTile t = tc_tile(P, w, tiles_m_dev, prank);
         if (!t.valid) break;
         const int acc = it & 1;
         const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
@@ -367,14 +457,19 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           const uint32_t b_step = p.b_mn_major ? (2048u >> 4) : (32u >> 4);
 #pragma unroll
           for (int ks = 0; ks < TC_BK / 16; ++ks) {
-            tc_mma(d_tmem, a_desc + (uint64_t)(a_step * ks), b_desc + (uint64_t)(b_step * ks), idesc,
-                   (kb | ks) != 0 ? 1u : 0u);
+            if constexpr (PAIR)
+              tc_mma_pair(d_tmem, a_desc + (uint64_t)(a_step * ks), b_desc + (uint64_t)(b_step * ks), idesc,
+                          (kb | ks) != 0 ? 1u : 0u);
+            else
+              tc_mma(d_tmem, a_desc + (uint64_t)(a_step * ks), b_desc + (uint64_t)(b_step * ks), idesc,
+                     (kb | ks) != 0 ? 1u : 0u);
           }
-          tc_commit(empty_bar(stage));          // stage reusable once these MMAs have read it
+          // stage reusable once these MMAs have read it (in both CTAs of a pair)
+          if constexpr (PAIR) tc_commit_pair(empty_bar(stage)); else tc_commit(empty_bar(stage));
           if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        tc_commit(tfull_bar(acc));              // accumulator complete
+        if constexpr (PAIR) tc_commit_pair(tfull_bar(acc)); else tc_commit(tfull_bar(acc));   // accumulator complete
       }
     }
   } else {
@@ -397,13 +492,13 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       return (t.m0 + q * 32 < lim) ? (t.ncols / 32 - half + 1) / 2 : 0;
     };
     uint32_t ds_g = 0, ds_pf_g = 0;              // blocks consumed / loads issued
-    int ds_pf_w = blockIdx.x, ds_pf_c = 0;
+    int ds_pf_w = w0, ds_pf_c = 0;
     TcTile ds_pf_t;
     ds_pf_t.valid = false;
     auto ds_prefetch = [&]() {
       while (ds_pf_t.valid && ds_pf_c >= ds_chunks(ds_pf_t)) {
-        ds_pf_w += gridDim.x; ds_pf_c = 0;
-        ds_pf_t = tc_tile(P, ds_pf_w, tiles_m_dev);
+        ds_pf_w += wstride; ds_pf_c = 0;
+        ds_pf_t = tc_tile(P, ds_pf_w, tiles_m_dev, prank);
       }
       if (!ds_pf_t.valid) return;
       const int s2 = (int)(ds_pf_g & 1u);
@@ -417,11 +512,11 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       ++ds_pf_c; ++ds_pf_g;
     };
     if constexpr (EPI == EPI_DSWIGLU) {
-      ds_pf_t = tc_tile(P, ds_pf_w, tiles_m_dev);
+      ds_pf_t = tc_tile(P, ds_pf_w, tiles_m_dev, prank);
       ds_prefetch();
     }
-    for (int w = blockIdx.x; ok; w += gridDim.x, ++it) {
-      TcTile t = tc_tile(P, w, tiles_m_dev);
+    for (int w = w0; ok; w += wstride, ++it) {
+      TcTile t = tc_tile(P, w, tiles_m_dev, prank);
       if (!t.valid) break;
       const int acc = it & 1;
       const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
@@ -622,7 +717,10 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       // accumulator may be overwritten by the MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) {
+        if constexpr (PAIR) mbar_arrive_cluster(mapa_u32(tempty_bar(acc), 0));   // the even CTA's MMA warp waits for both
+        else mbar_arrive(tempty_bar(acc));
+      }
     }
     if constexpr (EPI == EPI_DSWIGLU) {
       // operand loads issued but not consumed (only after an abandoned wait) must land before the CTA exits
@@ -648,10 +746,20 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
     }
   }
   __syncthreads();
+  if constexpr (PAIR) {
+    // neither CTA frees tensor memory or leaves while the other may still signal its barriers or
+    // have MMAs in flight that write its accumulators
+    tc_fence_before();
+    cluster_sync_all();
+  }
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
-                 : "memory");
+    if constexpr (PAIR)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS)
+                   : "memory");
   }
 }
 
@@ -671,8 +779,11 @@ inline TcState& tc_state() { static TcState s; return s; }
 
 template <int MMA_N, int EPI>
 inline cudaError_t tc_set_attr() {
-  return cudaFuncSetAttribute(gemm_tc_kernel<MMA_N, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              TcCfg<MMA_N, EPI>::SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MMA_N, EPI, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       TcCfg<MMA_N, EPI, false>::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_tc_kernel<MMA_N, EPI, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TcCfg<MMA_N, EPI, true>::SMEM_BYTES);
 }
 
 // Once per process: driver entry point for tensor-map encoding, SM count, shared-memory opt-in.
@@ -730,9 +841,26 @@ inline int tc_dg_parts(int N) { return 2 * (int)ceil_div(N, 256); }   // two epi
 
 template <int MMA_N, int EPI>
 inline int tc_launch(const TcParams& P, const CUtensorMap& ma, const CUtensorMap& mb0, const CUtensorMap& mb1,
-                     const CUtensorMap& mc, const CUtensorMap& mc1, int grid, cudaStream_t st) {
-  gemm_tc_kernel<MMA_N, EPI><<<grid, TC_THREADS, TcCfg<MMA_N, EPI>::SMEM_BYTES, st>>>(P, ma, mb0, mb1, mc, mc1);
-  return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
+                     const CUtensorMap& mc, const CUtensorMap& mc1, int grid, bool pair, cudaStream_t st) {
+  if (!pair) {
+    gemm_tc_kernel<MMA_N, EPI, false><<<grid, TC_THREADS, TcCfg<MMA_N, EPI, false>::SMEM_BYTES, st>>>(P, ma, mb0, mb1, mc, mc1);
+    return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = TcCfg<MMA_N, EPI, true>::SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<MMA_N, EPI, true>, P, ma, mb0, mb1, mc, mc1) == cudaSuccess
+             ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
 
 inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
@@ -810,12 +938,20 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
       if (r) return r;
     }
   }
+  // Pair mode wherever a 256-row tile cannot straddle two experts and every column tile is 256 wide.
+  const bool pair = p.group_mode != GROUP_M && p.N % 256 == 0 && !p.no_pair;
   int64_t total = (int64_t)P.tiles_m * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
   int grid = (int)(total < s.n_sms ? total : s.n_sms);
+  if (pair) {
+    total = (int64_t)((P.tiles_m + 1) / 2) * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
+    const int64_t pairs = total < s.n_sms / 2 ? total : s.n_sms / 2;
+    grid = (int)(2 * pairs);
+    P.idesc = (P.idesc & ~(0x1Fu << 24)) | ((uint32_t)(2 * TC_BM >> 4) << 24);   // M = 256 across the pair
+  }
   if (grid <= 0) return REVFFN_OK;
 
 #define TC_CASE(N_, E_) \
-  if (mma_n == N_ && p.epilogue == E_) return tc_launch<N_, E_>(P, ma, mb0, mb1, mc, mc1, grid, st);
+  if (mma_n == N_ && p.epilogue == E_) return tc_launch<N_, E_>(P, ma, mb0, mb1, mc, mc1, grid, pair, st);
   TC_CASE(256, EPI_STORE) TC_CASE(256, EPI_SWIGLU) TC_CASE(256, EPI_ROWSCALE) TC_CASE(256, EPI_COUPLE)
   TC_CASE(256, EPI_DSWIGLU) TC_CASE(256, EPI_WGRAD)
 #undef TC_CASE
