@@ -22,7 +22,8 @@
 // 64x64 boxes and described to the tensor core with leading/stride offsets.
 // Every wait is bounded; on expiry the kernel sets the status word and leaves.
 //
-// Pair mode (template flag PAIR; dense and K-grouped problems whose N is a multiple of 256):
+// Pair mode (template flag PAIR; dense and K-grouped problems whose N is a multiple of 256, or of 128
+// when B is stored [K, N]):
 // the grid is launched as clusters of two CTAs that work one 256 x 256 tile together with
 // tcgen05.mma.cta_group::2.  Each CTA loads its own 128 rows of A and ITS HALF of B's columns
 // (the tensor core reads both halves across the pair), so a K step costs a CTA 32 KB of operand
@@ -365,7 +366,8 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           if constexpr (PAIR) {
             // both CTAs' loads complete on the even CTA's barrier, which expects the bytes of both
             const uint32_t fbc = mapa_u32(full_bar(stage), 0);
-            if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
+            const int nhalf = t.ncols / 2;       // this CTA's share of the tile's columns: 128, or 64 in a ragged last tile
+            if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * (TC_A_BYTES + nhalf * TC_BK * 2));
             if (!p.a_mn_major) {
               tma_load_2d_pair(sa, &map_a, kb * TC_BK, t.m0, fbc);
             } else {
@@ -387,7 +389,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
               const int krow = t.krow0 + kbp * TC_BK;
 #pragma unroll
               for (int j = 0; j < 2; ++j)
-                tma_load_2d_pair(sb + j * 8192, mbp, p.b_col0 + t.n0 + 128 * crank + 64 * j, krow, fbc);
+                if (64 * j < nhalf) tma_load_2d_pair(sb + j * 8192, mbp, p.b_col0 + t.n0 + nhalf * crank + 64 * j, krow, fbc);
             }
             if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
             continue;
@@ -939,7 +941,8 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
     }
   }
   // Pair mode wherever a 256-row tile cannot straddle two experts and every column tile is 256 wide.
-  const bool pair = p.group_mode != GROUP_M && p.N % 256 == 0 && !p.no_pair;
+  // (a ragged 128-wide last tile splits into 64-column halves, which only the [K, N] storage of B can load)
+  const bool pair = p.group_mode != GROUP_M && (p.N % 256 == 0 || p.b_mn_major) && !p.no_pair;
   int64_t total = (int64_t)P.tiles_m * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
   int grid = (int)(total < s.n_sms ? total : s.n_sms);
   if (pair) {
