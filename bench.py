@@ -35,8 +35,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # (dram__bytes_read.sum + dram__bytes_write.sum; profiles/traffic_gemm_expert_gate_up_C1.md).
 # Keyed by pass/kernel; anything else, or any other workload, reports null.
 NCU_TRAFFIC_BYTES = {
-    "fwd/gemm_expert_gate_up_swiglu": 937_933_824, "inv/gemm_expert_gate_up_swiglu": 1_127_639_808,
-    "fwd/gemm_shared_gate_up_swiglu": 171_396_864, "inv/gemm_shared_gate_up_swiglu": 476_753_664,
+    "fwd/gemm_expert_gate_up_swiglu": 937_895_936, "inv/gemm_expert_gate_up_swiglu": 1_126_080_512,
+    "fwd/gemm_shared_gate_up_swiglu": 189_896_960, "inv/gemm_shared_gate_up_swiglu": 414_986_240,
 }
 
 
