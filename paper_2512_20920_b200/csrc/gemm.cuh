@@ -20,6 +20,8 @@
 //            expert * b_group_stride; rows >= *rows_total are not touched.
 //   GROUP_K: one product per expert e over the rows group_off[e]..group_off[e+1]
 //            as the K range (weight gradients); output offset e * c_group_stride.
+//            With group_cnt the range may stop at the first 64-row boundary past the
+//            expert's real rows: what follows is zero padding.
 #pragma once
 
 #include "common.cuh"
@@ -47,6 +49,7 @@ struct GemmProblem {
   float* dg_part; int dg_ld;                   // DSWIGLU: per (row, n-tile) partial of <acc, H>
   int group_mode, n_groups;
   const int32_t* group_off; const int32_t* tile_group; const int32_t* rows_total;
+  const int32_t* group_cnt;                    // GROUP_K, optional: real rows per group (the rest up to the next offset is zero padding)
   int64_t b_group_stride, c_group_stride;
   int a_col0, b_col0;
   int no_pair;        // tcgen05 back end: never pair CTAs for this product

@@ -282,6 +282,7 @@ __device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_
     int k0 = p.group_off[t.group], k1 = p.group_off[t.group + 1];
     t.krow0 = k0;
     t.k_blocks = (k1 - k0) / TC_BK;
+    if (p.group_cnt) t.k_blocks = min(t.k_blocks, (p.group_cnt[t.group] + TC_BK - 1) / TC_BK);   // skip all-zero K blocks
   }
   int tm = r / P.tiles_n, tn = r - tm * P.tiles_n;
   t.m0 = (pair_rank >= 0) ? tm * 2 * TC_BM + pair_rank * TC_BM : tm * TC_BM;

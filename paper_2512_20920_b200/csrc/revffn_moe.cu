@@ -403,6 +403,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     if (grouped) {
       p.group_mode = GROUP_K; p.n_groups = E;
       p.group_off = c.template p<int32_t>(L.expert_off);
+      p.group_cnt = c.template p<int32_t>(L.expert_cnt);
     }
     return run_gemm(c, p, tag);
   };
