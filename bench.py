@@ -171,6 +171,27 @@ def run_reference(args, cfg):
     }))
 
 
+def max_over_ranks(values, world, device="cuda"):
+    """Element-wise maximum of a list of floats over all ranks (the slowest replica sets the job's time)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def job_tokens_per_s(world, tokens_per_rank, steps, ms_total):
+    """Whole-job throughput of `world` independent replicas that each ran `steps` steps in ms_total."""
+    return world * tokens_per_rank * steps / (ms_total * 1e-3)
+
+
+def replica_seed(seed, rank):
+    """Every replica draws its own tokens; the weights are the same on all of them."""
+    return seed + rank
+
+
 def dist_setup():
     import torch
     import torch.distributed as dist
@@ -216,7 +237,7 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
         wdt = torch.bfloat16 if cfg.weight_dtype == "bf16" else torch.float32
         w_dev = {n: torch.from_numpy(v).cuda().to(torch.float32 if n in ("norm_gamma", "b_router") else wdt).contiguous()
                  for n, v in w_host.items()}
-    s_host = make_streams(cfg, args.seed + rank)
+    s_host = make_streams(cfg, replica_seed(args.seed, rank))
     blk = rv.Block(tokens=cfg.tokens, d_model=cfg.d_model, n_experts=cfg.n_experts, top_k=cfg.top_k,
                    d_expert=cfg.d_expert, d_shared=cfg.d_shared,
                    weight_dtype=rv.BF16 if cfg.weight_dtype == "bf16" else rv.F32, weights=w_dev,
@@ -276,13 +297,10 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
     step_unshared()
     barrier()
     ms_unshared = timed(step_unshared, n_un) / n_un
-    if world > 1:
-        t = torch.tensor([ms_total, ms_unshared], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_unshared = float(t[0].item()), float(t[1].item())
+    ms_total, ms_unshared = max_over_ranks([ms_total, ms_unshared], world)
     ms_step = ms_total / args.steps
     ms_prof_step = ms_prof_total / args.steps
-    value = world * cfg.tokens * args.steps / (ms_total * 1e-3)
+    value = job_tokens_per_s(world, cfg.tokens, args.steps, ms_total)
 
     e2e_value, dt, bytes_dir = None, 0.0, 0
     if e2e:
@@ -304,11 +322,8 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
             host_step()
             torch.cuda.synchronize()     # the step's results are read on the host
         dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
-        e2e_value = world * cfg.tokens * args.steps / dt
+        dt = max_over_ranks([dt], world)[0]
+        e2e_value = job_tokens_per_s(world, cfg.tokens, args.steps, dt * 1e3)
         bytes_dir = 3 * hy1.numel() * 4
 
     if rank != 0:
@@ -455,7 +470,7 @@ def run_stack(args, cfg):
     L = args.blocks or cfg.n_blocks
     weights = [make_weights_device(cfg, args.seed, block=l) for l in range(L)]
     w_bytes = sum(t.numel() * t.element_size() for w in weights for t in w.values())
-    s_host = make_streams(cfg, args.seed + rank)
+    s_host = make_streams(cfg, replica_seed(args.seed, rank))
     a0, b0 = torch.from_numpy(s_host["y1"]).cuda(), torch.from_numpy(s_host["x2"]).cuda()
     g0 = torch.from_numpy(s_host["dy2"]).cuda()
     # one fp32 gradient buffer per tensor, reused by every layer (an optimiser would consume it layer by layer);
@@ -494,7 +509,7 @@ def run_stack(args, cfg):
         e1.record()
         barrier()
         clocks = sampler.stop() if sampler else None
-        ms = e0.elapsed_time(e1) / args.steps
+        ms = max_over_ranks([e0.elapsed_time(e1)], world)[0] / args.steps
         assert stk.status() == 0
         rec = {"ms_per_step": ms, "tokens_per_s": cfg.tokens / (ms * 1e-3), "launches": rv.revffn_prof_launches() - l0,
                "activation_bytes": int(torch.cuda.max_memory_allocated() - base_alloc),
