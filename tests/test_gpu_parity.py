@@ -276,3 +276,13 @@ def test_host_step_matches_the_device_entry_points(rv, two_streams):
     assert torch.equal(hy2, y2.cpu()) and torch.equal(hx2r, x2r.cpu()) and torch.equal(hdy1, dy1.cpu())
     for n in g:
         assert torch.equal(g[n], g_ref[n]), n
+
+
+@pytest.mark.parametrize("kw", [dict(n_experts=64, top_k=8, tokens=150), dict(n_experts=130, top_k=3, tokens=97),
+                                dict(n_experts=256, top_k=8, tokens=70, d_shared=0)])
+def test_many_experts(rv, kw):
+    """More experts than one pass of the router's logit tile holds (64 incl. the shared-gate row), up to the
+    largest supported count, and the largest top-k."""
+    cfg = small_cfg(**kw)
+    w, s = scaled_weights(cfg, 9, 4.0), make_streams(cfg, 9)
+    run_all_passes(rv, cfg, w, s, TOL_BF16, check_grads=False)
