@@ -14,7 +14,9 @@ What it follows
     intro and Sec. 3.2 "Advantages").  The benchmark configurations fix it: a
     linear router, top-k selection, softmax over the k selected logits (gate
     weights sum to 1), routed SwiGLU experts, and a SwiGLU shared expert scaled
-    by a sigmoid gate.  No token dropping, no biases in the experts.
+    by a sigmoid gate.  No token dropping, no biases in the experts.  A second gating
+    mode ("softmax_all") takes the selected probabilities of a softmax over all E
+    logits without renormalising them.
   * Norm: RMSNorm over the d/2-wide stream (the base model family's norm) with a
     learnable scale; "none" is available for tests.
   * Backward (Sec. 2 "Reversible Networks", Sec. 3.1): the transpose-Jacobian of
@@ -97,19 +99,31 @@ def topk_margin(L: np.ndarray, k: int) -> np.ndarray:
     return s[..., k - 1] - s[..., k]
 
 
-def gate_weights(L: np.ndarray, idx: np.ndarray) -> np.ndarray:
-    """softmax over the selected logits only, so the k gate weights sum to 1."""
+GATINGS = ("renorm", "softmax_all")
+
+
+def gate_weights(L: np.ndarray, idx: np.ndarray, gating: str = "renorm") -> np.ndarray:
+    """Gate weights of the selected experts.
+      "renorm":      softmax over the selected logits only, so the k weights sum to 1
+                     (what the benchmark definition asks for);
+      "softmax_all": softmax over all E logits, the selected probabilities taken as
+                     they are (they sum to less than 1 unless k == E): the variant in
+                     which the top-k probabilities are not renormalised."""
+    assert gating in GATINGS
     sel = np.take_along_axis(L, idx, axis=-1)
-    m = sel.max(axis=-1, keepdims=True)
-    ex = np.exp(sel - m)
-    return ex / ex.sum(axis=-1, keepdims=True)
+    if gating == "renorm":
+        m = sel.max(axis=-1, keepdims=True)
+        ex = np.exp(sel - m)
+        return ex / ex.sum(axis=-1, keepdims=True)
+    m = L.max(axis=-1, keepdims=True)
+    return np.exp(sel - m) / np.exp(L - m).sum(axis=-1, keepdims=True)
 
 
 # --------------------------------------------------------------------------- #
 # One token, written out step by step (the definition)
 # --------------------------------------------------------------------------- #
 def branch_token(p, y: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
-                 idx_override: Optional[np.ndarray] = None):
+                 idx_override: Optional[np.ndarray] = None, gating: str = "renorm"):
     """F = P_down(MLP_pt(P_up(Norm(y)))) for one token y (length h).
 
     Returns (F, idx, gates, margin).  idx_override forces the expert set (used
@@ -118,7 +132,7 @@ def branch_token(p, y: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
     u = _w(p, "w_up") @ n                                   # P_up, Sec. 3.2
     L = router_logits(u[None, :], p)[0]                     # router
     idx = topk_indices(L, k) if idx_override is None else np.asarray(idx_override)
-    g = gate_weights(L[None, :], idx[None, :])[0]
+    g = gate_weights(L[None, :], idx[None, :], gating)[0]
     z = np.zeros_like(u)
     for s, e in enumerate(idx):                             # routed SwiGLU experts
         a = _w(p, "w_gate", e) @ u
@@ -137,7 +151,7 @@ def branch_token(p, y: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
 # All tokens (same arithmetic, tokens grouped per expert so matmul can be used)
 # --------------------------------------------------------------------------- #
 def branch(p, Y1: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
-           route_override: Optional[np.ndarray] = None, keep: bool = False):
+           route_override: Optional[np.ndarray] = None, keep: bool = False, gating: str = "renorm"):
     """F[T,h] = MLP(Norm(Y1)) for all tokens.  Returns (F, info); info holds the
     routing (idx, gates, margin, logits) and, with keep=True, the intermediates
     the backward pass needs."""
@@ -147,7 +161,7 @@ def branch(p, Y1: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
     u = n @ _w(p, "w_up").T
     L = router_logits(u, p)
     idx = topk_indices(L, k) if route_override is None else np.asarray(route_override)
-    g = gate_weights(L, idx)
+    g = gate_weights(L, idx, gating)
     E = p["w_router"].shape[0]
     d = u.shape[1]
     z = np.zeros((T, d), dtype=F64)
@@ -181,16 +195,16 @@ def branch(p, Y1: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
     return F, info
 
 
-def forward(p, Y1, X2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None):
+def forward(p, Y1, X2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None, gating: str = "renorm"):
     """Eq. 2: Y2 = X2 + MLP(Norm(Y1)).  Returns (Y2, info)."""
-    F, info = branch(p, Y1, k, eps, norm, route_override)
+    F, info = branch(p, Y1, k, eps, norm, route_override, gating=gating)
     info["F"] = F
     return np.asarray(X2, dtype=F64) + F, info
 
 
-def inverse(p, Y1, Y2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None):
+def inverse(p, Y1, Y2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None, gating: str = "renorm"):
     """Inverse pass of Sec. 3.1: X2 = Y2 - MLP(Norm(Y1)).  Returns (X2, info)."""
-    F, info = branch(p, Y1, k, eps, norm, route_override)
+    F, info = branch(p, Y1, k, eps, norm, route_override, gating=gating)
     info["F"] = F
     return np.asarray(Y2, dtype=F64) - F, info
 
@@ -198,7 +212,8 @@ def inverse(p, Y1, Y2, k: int, eps: float = 1e-6, norm: str = "rms", route_overr
 # --------------------------------------------------------------------------- #
 # Backward: J^T dY2 for the stream Y1 and every weight
 # --------------------------------------------------------------------------- #
-def backward(p, Y1, dY2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None):
+def backward(p, Y1, dY2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None,
+             gating: str = "renorm"):
     """Gradients of <dY2, Y2> through Eq. 2 with Y1 as the only kept input
     (intermediates are recomputed, as reversible back-propagation does).
 
@@ -206,7 +221,7 @@ def backward(p, Y1, dY2, k: int, eps: float = 1e-6, norm: str = "rms", route_ove
     gradient Y1 already carries), dx2 (= dY2) and one entry per weight."""
     Y1 = np.asarray(Y1, dtype=F64)
     G = np.asarray(dY2, dtype=F64)
-    F, c = branch(p, Y1, k, eps, norm, route_override, keep=True)
+    F, c = branch(p, Y1, k, eps, norm, route_override, keep=True, gating=gating)
     idx, g, u, n, r, z = c["idx"], c["gates"], c["u"], c["n"], c["r"], c["z"]
     T, h = Y1.shape
     E = p["w_router"].shape[0]
@@ -252,10 +267,21 @@ def backward(p, Y1, dY2, k: int, eps: float = 1e-6, norm: str = "rms", route_ove
         out["w_gate"][e] = da.T @ u[toks]
         out["w_upx"][e] = db.T @ u[toks]
 
-    # gates: softmax over the selected logits; selection itself has zero gradient
-    dsel = g * (dgate - np.sum(g * dgate, axis=1, keepdims=True))
-    dL = np.zeros((T, E), dtype=F64)
-    np.put_along_axis(dL, idx, dsel, axis=1)
+    # gates; the selection itself has zero gradient
+    if gating == "renorm":
+        # softmax over the selected logits: only those logits receive a gradient
+        dsel = g * (dgate - np.sum(g * dgate, axis=1, keepdims=True))
+        dL = np.zeros((T, E), dtype=F64)
+        np.put_along_axis(dL, idx, dsel, axis=1)
+    else:
+        # softmax over all logits, g_s = p_s for the selected s:
+        # dL_j = p_j ([j selected] dg_j - sum_s p_s dg_s) for every j
+        L = c["logits"]
+        prob = np.exp(L - L.max(axis=1, keepdims=True))
+        prob = prob / prob.sum(axis=1, keepdims=True)
+        dfull = np.zeros((T, E), dtype=F64)
+        np.put_along_axis(dfull, idx, dgate, axis=1)
+        dL = prob * (dfull - np.sum(g * dgate, axis=1, keepdims=True))
     out["w_router"] = dL.T @ u
     out["b_router"] = dL.sum(axis=0)
     du += dL @ _w(p, "w_router")
@@ -287,7 +313,8 @@ def backward(p, Y1, dY2, k: int, eps: float = 1e-6, norm: str = "rms", route_ove
 # therefore rewritten every two layers and reconstruction error compounds
 # through both, as it does in the full block.
 # --------------------------------------------------------------------------- #
-def stack_forward(blocks, A, B, k: int, eps: float = 1e-6, norm: str = "rms", route_overrides=None):
+def stack_forward(blocks, A, B, k: int, eps: float = 1e-6, norm: str = "rms", route_overrides=None,
+                  gating: str = "renorm"):
     """R_l <- R_l + MLP_l(Norm(P_l)) for l = 0 .. L-1 (Eq. 2 per layer).
     Returns (A, B, infos); infos[l] is the layer's `forward` info."""
     A = np.array(A, dtype=F64)
@@ -296,14 +323,15 @@ def stack_forward(blocks, A, B, k: int, eps: float = 1e-6, norm: str = "rms", ro
     for l, p in enumerate(blocks):
         ro = None if route_overrides is None else route_overrides[l]
         if l % 2 == 0:
-            B, info = forward(p, A, B, k, eps, norm, ro)
+            B, info = forward(p, A, B, k, eps, norm, ro, gating)
         else:
-            A, info = forward(p, B, A, k, eps, norm, ro)
+            A, info = forward(p, B, A, k, eps, norm, ro, gating)
         infos.append(info)
     return A, B, infos
 
 
-def stack_inverse(blocks, A, B, k: int, eps: float = 1e-6, norm: str = "rms", route_overrides=None):
+def stack_inverse(blocks, A, B, k: int, eps: float = 1e-6, norm: str = "rms", route_overrides=None,
+                  gating: str = "renorm"):
     """Undo `stack_forward` from its outputs: R_l <- R_l - MLP_l(Norm(P_l)) for
     l = L-1 .. 0 (inverse pass of Sec. 3.1 per layer).  Returns (A, B)."""
     A = np.array(A, dtype=F64)
@@ -311,14 +339,14 @@ def stack_inverse(blocks, A, B, k: int, eps: float = 1e-6, norm: str = "rms", ro
     for l in reversed(range(len(blocks))):
         ro = None if route_overrides is None else route_overrides[l]
         if l % 2 == 0:
-            B, _ = inverse(blocks[l], A, B, k, eps, norm, ro)
+            B, _ = inverse(blocks[l], A, B, k, eps, norm, ro, gating)
         else:
-            A, _ = inverse(blocks[l], B, A, k, eps, norm, ro)
+            A, _ = inverse(blocks[l], B, A, k, eps, norm, ro, gating)
     return A, B
 
 
 def stack_backward(blocks, A_out, B_out, gA, gB, k: int, eps: float = 1e-6, norm: str = "rms",
-                   route_overrides=None):
+                   route_overrides=None, gating: str = "renorm"):
     """Reversible back-propagation through the stack: for l = L-1 .. 0 rebuild
     the layer's input from its output, then push the gradient through the
     layer (dP += J^T dR, dR passes through unchanged).
@@ -335,12 +363,12 @@ def stack_backward(blocks, A_out, B_out, gA, gB, k: int, eps: float = 1e-6, norm
         ro = None if route_overrides is None else route_overrides[l]
         p = blocks[l]
         if l % 2 == 0:
-            B, _ = inverse(p, A, B, k, eps, norm, ro)
-            g = backward(p, A, gB, k, eps, norm, ro)
+            B, _ = inverse(p, A, B, k, eps, norm, ro, gating)
+            g = backward(p, A, gB, k, eps, norm, ro, gating)
             gA = gA + g["dy1"]
         else:
-            A, _ = inverse(p, B, A, k, eps, norm, ro)
-            g = backward(p, B, gA, k, eps, norm, ro)
+            A, _ = inverse(p, B, A, k, eps, norm, ro, gating)
+            g = backward(p, B, gA, k, eps, norm, ro, gating)
             gB = gB + g["dy1"]
         grads[l] = g
     return A, B, gA, gB, grads

@@ -304,14 +304,15 @@ def test_route_override_changes_only_selection():
 
 
 # ------------------------------------------------------------------ library cross-check of MLP_pt
-def test_mlp_pt_matches_transformers_qwen2_moe_block():
+@pytest.mark.parametrize("gating,norm_topk", [("renorm", True), ("softmax_all", False)])
+def test_mlp_pt_matches_transformers_qwen2_moe_block(gating, norm_topk):
     m = pytest.importorskip("transformers.models.qwen2_moe.modeling_qwen2_moe")
     cfg, p, s = _tiny(14, d_model=32, n_experts=6, top_k=3, d_expert=16, d_shared=24)
     try:
         hf_cfg = m.Qwen2MoeConfig(hidden_size=cfg.d_model, moe_intermediate_size=cfg.d_expert,
                                   shared_expert_intermediate_size=cfg.d_shared,
                                   num_experts=cfg.n_experts, num_experts_per_tok=cfg.top_k,
-                                  norm_topk_prob=True)
+                                  norm_topk_prob=norm_topk)
         blk = m.Qwen2MoeSparseMoeBlock(hf_cfg).double()
         sd = blk.state_dict()
         T = lambda a: torch.tensor(np.asarray(a, dtype=np.float64))
@@ -333,10 +334,73 @@ def test_mlp_pt_matches_transformers_qwen2_moe_block():
     q = dict(p)
     q["w_up"] = np.eye(cfg.d_model); q["w_down"] = np.eye(cfg.d_model); q["norm_gamma"] = None
     u = np.random.default_rng(3).standard_normal((9, cfg.d_model))
-    F, info = orc.branch(q, u, cfg.top_k, norm="none")
+    F, info = orc.branch(q, u, cfg.top_k, norm="none", gating=gating)
     with torch.no_grad():
         ref = blk(torch.tensor(u)[None])
     ref = ref[0] if isinstance(ref, tuple) else ref
     # the library evaluates its gate softmax in fp32, hence the tolerance; a swapped
     # operand or a different normalisation is off by orders of magnitude more
     assert np.allclose(F, ref.reshape(9, cfg.d_model).numpy(), rtol=1e-6, atol=1e-7)
+
+
+# ------------------------------------------------------------------ gating without renormalisation
+def test_softmax_all_gates_are_the_renormalised_gates_times_the_selected_mass():
+    cfg, p, s = _tiny(21)
+    _, a = orc.forward(p, s["y1"], s["x2"], cfg.top_k, gating="softmax_all")
+    _, r = orc.forward(p, s["y1"], s["x2"], cfg.top_k, gating="renorm")
+    assert np.array_equal(a["idx"], r["idx"])                       # the same experts are selected
+    L = a["logits"]
+    prob = np.exp(L) / np.exp(L).sum(axis=1, keepdims=True)         # textbook softmax over all experts
+    mass = np.take_along_axis(prob, a["idx"], axis=1).sum(axis=1)
+    assert (mass < 1).all() and (mass > 0).all()
+    assert np.allclose(a["gates"].sum(axis=1), mass, rtol=1e-13)
+    assert np.allclose(a["gates"], r["gates"] * mass[:, None], rtol=1e-13)
+    assert np.allclose(a["gates"], np.take_along_axis(prob, a["idx"], axis=1), rtol=1e-13)
+
+
+def test_softmax_all_equals_renorm_when_every_expert_is_selected():
+    cfg, p, s = _tiny(22, top_k=5)
+    Fa, _ = orc.branch(p, s["y1"], cfg.top_k, gating="softmax_all")
+    Fr, _ = orc.branch(p, s["y1"], cfg.top_k, gating="renorm")
+    assert np.allclose(Fa, Fr, rtol=1e-12, atol=1e-14)
+    ga = orc.backward(p, s["y1"], s["dy2"], cfg.top_k, gating="softmax_all")
+    gr = orc.backward(p, s["y1"], s["dy2"], cfg.top_k, gating="renorm")
+    for n in ("dy1", "w_router", "w_gate", "w_up", "ws_sgate"):
+        assert np.allclose(ga[n], gr[n], rtol=1e-10, atol=1e-13), n
+
+
+@pytest.mark.parametrize("seed", [23, 24])
+def test_softmax_all_backward_matches_central_differences(seed):
+    """Here the unselected logits carry gradient too (through the softmax denominator)."""
+    cfg, p, s = _tiny(seed)
+    for n in p:
+        p[n] = p[n].astype(np.float64)
+    y1, dy2 = s["y1"].astype(np.float64), s["dy2"].astype(np.float64)
+    _, info = orc.branch(p, y1, cfg.top_k, gating="softmax_all")
+    assert info["margin"].min() > 1e-3
+    g = orc.backward(p, y1, dy2, cfg.top_k, gating="softmax_all")
+    loss = lambda: float(np.sum(dy2 * orc.branch(p, y1, cfg.top_k, gating="softmax_all")[0]))
+    rng = np.random.default_rng(seed)
+    eps = 1e-6
+    for _ in range(6):
+        t, i = int(rng.integers(cfg.tokens)), int(rng.integers(cfg.h))
+        old = y1[t, i]
+        y1[t, i] = old + eps; lp = loss()
+        y1[t, i] = old - eps; lm = loss()
+        y1[t, i] = old
+        fd = (lp - lm) / (2 * eps)
+        assert abs(fd - g["dy1"][t, i]) <= 1e-6 * max(1.0, abs(fd)), (t, i, fd, g["dy1"][t, i])
+    for name in ("w_router", "w_up", "w_downx", "ws_gate"):
+        W = p[name]
+        for _ in range(3):
+            pos = tuple(int(rng.integers(n)) for n in W.shape)
+            old = W[pos]
+            W[pos] = old + eps; lp = loss()
+            W[pos] = old - eps; lm = loss()
+            W[pos] = old
+            fd = (lp - lm) / (2 * eps)
+            assert abs(fd - g[name][pos]) <= 2e-6 * max(1.0, abs(fd)), (name, pos, fd, g[name][pos])
+    # the router gradient is dense now: experts that were never selected still get one
+    never = np.setdiff1d(np.arange(cfg.n_experts), np.unique(info["idx"]))
+    if never.size:
+        assert np.abs(g["w_router"][never]).max() > 0
