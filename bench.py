@@ -241,7 +241,7 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
     blk = rv.Block(tokens=cfg.tokens, d_model=cfg.d_model, n_experts=cfg.n_experts, top_k=cfg.top_k,
                    d_expert=cfg.d_expert, d_shared=cfg.d_shared,
                    weight_dtype=rv.BF16 if cfg.weight_dtype == "bf16" else rv.F32, weights=w_dev,
-                   norm_eps=cfg.norm_eps)
+                   norm_eps=cfg.norm_eps, flags=rv.FLAG_GATE_SOFTMAX_ALL if args.gating == "softmax_all" else 0)
     y1, x2, dy2 = (torch.from_numpy(s_host[n]).cuda() for n in ("y1", "x2", "dy2"))
     y2, x2r, dy1 = torch.empty_like(x2), torch.empty_like(x2), torch.zeros_like(y1)
     # routers stay frozen (Sec. 3.3 of the paper); every other weight gets its fp32 gradient
@@ -388,7 +388,7 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
                                f"d={cfg.d_model}, E={cfg.n_experts}, top-{cfg.top_k}, I={cfg.d_expert}, "
                                f"I_s={cfg.d_shared}; step = forward + inverse + backward (all weight gradients "
                                f"in fp32 except the frozen router); the backward pass reuses the branch "
-                               f"evaluation of the inverse pass",
+                               f"evaluation of the inverse pass" + ("; gates not renormalised" if args.gating != "renorm" else ""),
                    "l2": "per-step working set (1.1 GB weights + >2 GB activations) exceeds the 126 MB L2",
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},
         "pct_bf16_tensor_peak": 100.0 * total_flops / (ms_step * 1e-3) / 1e12 / peak_t,
@@ -593,6 +593,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--blocks", type=int, default=0, help="C3: number of layers (default: the configuration's 24)")
     ap.add_argument("--no-drift", action="store_true", help="C3: skip the per-layer drift pass")
+    ap.add_argument("--gating", default="renorm", choices=["renorm", "softmax_all"],
+                    help="single-block runs: gate weights renormalised over the top-k (default, the benchmark's "
+                         "definition) or taken from the softmax over all experts")
     args = ap.parse_args()
     from workloads import CONFIGS
     if args.config == "C4":

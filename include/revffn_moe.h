@@ -81,6 +81,12 @@ enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                
  *                      so one saved evaluation serves one backward call.               */
 #define REVFFN_FLAG_SAVE_ACTIVATIONS 2u
 #define REVFFN_FLAG_REUSE_ACTIVATIONS 4u
+/* Gate weights without renormalisation: g_e = softmax(L over all E experts)_e for the k selected
+ * experts (they sum to less than 1 unless k == E), instead of the softmax over the k selected
+ * logits.  The same experts are selected.  In the backward pass every logit then receives a
+ * gradient (through the softmax denominator), not only the selected ones.  Set the flag on every
+ * pass of a block alike. */
+#define REVFFN_FLAG_GATE_SOFTMAX_ALL 8u
 
 /*
  * Block descriptor.  Shape constraints (else REVFFN_ERR_SHAPE):

@@ -18,6 +18,7 @@ NORM_RMS, NORM_NONE = 0, 1
 FLAG_FORCE_SIMT = 1
 FLAG_SAVE_ACTIVATIONS = 2
 FLAG_REUSE_ACTIVATIONS = 4
+FLAG_GATE_SOFTMAX_ALL = 8
 
 WEIGHT_NAMES = ("norm_gamma", "w_up", "w_down", "w_router", "b_router", "w_gate", "w_upx", "w_downx",
                 "ws_gate", "ws_up", "ws_down", "ws_sgate")

@@ -68,6 +68,41 @@ __global__ void router_bwd_kernel(const float* __restrict__ dg_part, int dg_ld, 
   }
 }
 
+// Gate backward when the gates are entries of the softmax over all experts (no renormalisation):
+//   dg[t,s] as above;  c = sum_s p[t, e_s] dg[t,s];  dL[t,j] = p[t,j] * ([j = e_s] dg[t,s] - c) for every j.
+// dL is written as a GEMM operand [T, ld_dl] (columns E .. ld_dl-1 zero).
+template <typename T>
+__global__ void router_bwd_dense_kernel(const float* __restrict__ dg_part, int dg_ld, int n_part,
+                                        const float* __restrict__ prob, const int32_t* __restrict__ idx,
+                                        const int32_t* __restrict__ tok_row, int tokens, int k, int E, int ld_dl,
+                                        T* __restrict__ dl_out) {
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= tokens) return;
+  float dg[8];
+  int ex[8];
+  const float* p = prob + (int64_t)t * E;
+  float c = 0.f;
+  for (int s = 0; s < k; ++s) {
+    int row = tok_row[(int64_t)t * k + s];
+    float acc = 0.f;
+    for (int j = 0; j < n_part; ++j) acc += dg_part[(int64_t)row * dg_ld + j];
+    dg[s] = acc;
+    ex[s] = idx[(int64_t)t * k + s];
+    c += p[ex[s]] * acc;
+  }
+  T* o = dl_out + (int64_t)t * ld_dl;
+  for (int j = 0; j < ld_dl; ++j) {
+    float v = 0.f;
+    if (j < E) {
+      float sel = 0.f;
+      for (int s = 0; s < k; ++s)
+        if (ex[s] == j) sel = dg[s];
+      v = p[j] * (sel - c);
+    }
+    o[j] = from_f32<T>(v);
+  }
+}
+
 // Router weight gradient from the permuted layout:
 //   dW_r[e, c] (+)= sum_{rows of e} row_dl[row] * Up[row, c];  db_r[e] (+)= sum row_dl[row]
 // grid (ceil(d / blockDim), E); each thread owns one column.
@@ -94,7 +129,7 @@ __global__ void router_wgrad_kernel(const T* __restrict__ Up, const float* __res
 // Column reduction with a per-row weight, two passes (deterministic):
 //   part[b, c] = sum_{t in strip b} w[t] * X[t, c]      (colsum_partial)
 //   out[c] (+)= sum_b part[b, c]                        (colsum_final)
-// Used for d w_sgate = sum_t dl[t] u_t.
+// Used for d w_sgate = sum_t dl[t] u_t (and, with w == NULL meaning all ones, for plain column sums).
 template <typename T>
 __global__ void colsum_partial_kernel(const T* __restrict__ X, int64_t ldx, const float* __restrict__ w,
                                       int rows, int cols, int strip, float* __restrict__ part) {
@@ -104,7 +139,7 @@ __global__ void colsum_partial_kernel(const T* __restrict__ X, int64_t ldx, cons
   int t0 = b * strip, t1 = min(rows, t0 + strip);
   float acc = 0.f;
 #pragma unroll 8
-  for (int t = t0; t < t1; ++t) acc += w[t] * to_f32(X[(int64_t)t * ldx + c]);
+  for (int t = t0; t < t1; ++t) acc += (w ? w[t] : 1.f) * to_f32(X[(int64_t)t * ldx + c]);
   part[(int64_t)b * cols + c] = acc;
 }
 
@@ -124,15 +159,15 @@ template <typename T>
 __global__ void du_reduce_kernel(const T* __restrict__ dUp, const int32_t* __restrict__ tok_row,
                                  const int32_t* __restrict__ idx, const float* __restrict__ tok_dl, int k,
                                  const T* __restrict__ dUsh, const T* __restrict__ w_router,
-                                 const float* __restrict__ dl, const T* __restrict__ w_sgate, int width,
-                                 T* __restrict__ dU) {
+                                 const float* __restrict__ dl, const T* __restrict__ w_sgate,
+                                 const T* __restrict__ dUr, int width, T* __restrict__ dU) {
   int t = blockIdx.x;
   int rows[8], ex[8];
   float dls[8];
   for (int s = 0; s < k; ++s) {
     rows[s] = tok_row[(int64_t)t * k + s];
     ex[s] = idx[(int64_t)t * k + s];
-    dls[s] = tok_dl[(int64_t)t * k + s];
+    dls[s] = dUr ? 0.f : tok_dl[(int64_t)t * k + s];
   }
   float dlt = dUsh ? dl[t] : 0.f;
   for (int c = threadIdx.x * 8; c < width; c += blockDim.x * 8) {
@@ -153,10 +188,16 @@ __global__ void du_reduce_kernel(const T* __restrict__ dUp, const int32_t* __res
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[i] += dlt * f[i];
     }
-    for (int s = 0; s < k; ++s) {
-      v.load(w_router + (int64_t)ex[s] * width + c); v.get(f);
+    if (dUr) {        // the router term arrives as one row, dL[t, :] W_r, computed as a matrix product
+      v.load(dUr + (int64_t)t * width + c); v.get(f);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] += dls[s] * f[i];
+      for (int i = 0; i < 8; ++i) acc[i] += f[i];
+    } else {
+      for (int s = 0; s < k; ++s) {
+        v.load(w_router + (int64_t)ex[s] * width + c); v.get(f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] += dls[s] * f[i];
+      }
     }
     v.set(acc);
     v.store(dU + (int64_t)t * width + c);

@@ -878,7 +878,8 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   P.tiles_n = (int)ceil_div(p.N, P.tile_n);
   P.k_blocks = (int)ceil_div(p.K, TC_BK);
   if (p.N % 128 != 0) return REVFFN_ERR_SHAPE;
-  if (p.group_mode != GROUP_K && p.K % TC_BK != 0 && !(p.a_mn_major && p.b_mn_major)) return REVFFN_ERR_SHAPE;
+  // K need not be a multiple of the 64-wide K step: the tensor maps end at K, so the rest of the last
+  // step is loaded as zeros (K-major rows must still start on 16-byte boundaries: lda, ldb)
   if (p.concat == CONCAT_K && (P.k_blocks & 1)) return REVFFN_ERR_SHAPE;
   P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.a_mn_major ? 1 : 0) << 15) |
             ((uint32_t)(p.b_mn_major ? 1 : 0) << 16) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);

@@ -75,12 +75,13 @@ struct Buf { size_t off = 0, bytes = 0; };
 
 struct WsLayout {
   // forward / inverse
-  Buf status, rows_total, w_rc, n, r, idx, gates, sgate, local_rank, chunk_cnt, chunk_base, expert_cnt,
+  Buf status, rows_total, w_rc, n, r, idx, gates, sgate, prob, local_rank, chunk_cnt, chunk_base, expert_cnt,
       expert_off, tile_group, tok_row, row_tok, row_gate, u, up, hmid, o, hs, s, z;
   size_t fwd_bytes = 0;
   size_t saved_bytes = 0;   // fwd region + SwiGLU pre-activations: what a saved evaluation consists of
   // backward only
-  Buf ab, abs, gb, dz, ds, dl, dop, dg_part, tok_dl, row_dl, dup, dush, du, dn, part;
+  Buf ab, abs, gb, dz, ds, dl, dop, dg_part, tok_dl, row_dl, dlf, dur, dup, dush, du, dn, part;
+  int ld_dlf = 0;
   size_t bwd_bytes = 0;
   int64_t rows_pad = 0;   // upper bound on padded rows
   int n_chunks = 0, max_tiles = 0, dg_ld = 0, strips = 0;
@@ -112,6 +113,7 @@ static WsLayout plan_workspace(const revffn_moe_desc& D) {
   take(L.idx, (size_t)T * k * 4);
   take(L.gates, (size_t)T * k * 4);
   take(L.sgate, (size_t)T * 4);
+  take(L.prob, (D.flags & REVFFN_FLAG_GATE_SOFTMAX_ALL) ? (size_t)T * E * 4 : 0);
   take(L.local_rank, (size_t)T * k * 4);
   take(L.chunk_cnt, (size_t)L.n_chunks * E * 4);
   take(L.chunk_base, (size_t)L.n_chunks * E * 4);
@@ -140,6 +142,10 @@ static WsLayout plan_workspace(const revffn_moe_desc& D) {
   take(L.dg_part, (size_t)Rp * L.dg_ld * 4);
   take(L.tok_dl, (size_t)T * k * 4);
   take(L.row_dl, (size_t)Rp * 4);
+  L.ld_dlf = (int)round_up(E, 64);
+  const bool dense_gate = (D.flags & REVFFN_FLAG_GATE_SOFTMAX_ALL) != 0;
+  take(L.dlf, dense_gate ? (size_t)T * L.ld_dlf * ts : 0);
+  take(L.dur, dense_gate ? (size_t)T * d * ts : 0);
   take(L.dup, (size_t)Rp * d * ts);
   take(L.dush, (size_t)T * d * ts);
   take(L.du, (size_t)T * d * ts);
@@ -265,7 +271,8 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     { ProfScope ps(TG_ROUTER, st);
     CK(launch_router_topk(y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, c.template p<double>(L.w_rc),
                           c.W.b_router, Tn, h, E, k, Is > 0 ? 1 : 0, idx_in, c.template p<int32_t>(L.idx),
-                          c.template p<float>(L.gates), c.template p<float>(L.sgate), idx_user, st));
+                          c.template p<float>(L.gates), c.template p<float>(L.sgate), idx_user,
+                          (D.flags & REVFFN_FLAG_GATE_SOFTMAX_ALL) ? c.template p<float>(L.prob) : nullptr, st));
     }
   }
 
@@ -503,20 +510,54 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
   if (G.w_upx) CKR(wgrad(TG_WG_EXP_UP, G.w_upx, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, I, c.template p<T>(L.up), d, true, (int64_t)I * d));
 
   // Gate / router backward
-  { ProfScope ps(TG_ROUTER_BWD, st);
-  router_bwd_kernel<<<(unsigned)ceil_div(Tn, 128), 128, 0, st>>>(
-      c.template p<float>(L.dg_part), L.dg_ld, n_part, c.template p<float>(L.gates), c.template p<int32_t>(L.tok_row),
-      Tn, k, c.template p<float>(L.tok_dl), c.template p<float>(L.row_dl));
-  }
-  CK(cudaGetLastError());
-  if (G.w_router || G.b_router) {
-    dim3 grid((unsigned)ceil_div(d, 256), (unsigned)E);
-    { ProfScope ps(TG_WG_ROUTER, st);
-    router_wgrad_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.up), c.template p<float>(L.row_dl),
-                                                 c.template p<int32_t>(L.expert_off), c.template p<int32_t>(L.expert_cnt),
-                                                 d, acc, G.w_router, G.b_router);
+  const bool dense_gate = (D.flags & REVFFN_FLAG_GATE_SOFTMAX_ALL) != 0;
+  if (!dense_gate) {
+    { ProfScope ps(TG_ROUTER_BWD, st);
+    router_bwd_kernel<<<(unsigned)ceil_div(Tn, 128), 128, 0, st>>>(
+        c.template p<float>(L.dg_part), L.dg_ld, n_part, c.template p<float>(L.gates), c.template p<int32_t>(L.tok_row),
+        Tn, k, c.template p<float>(L.tok_dl), c.template p<float>(L.row_dl));
     }
     CK(cudaGetLastError());
+    if (G.w_router || G.b_router) {
+      dim3 grid((unsigned)ceil_div(d, 256), (unsigned)E);
+      { ProfScope ps(TG_WG_ROUTER, st);
+      router_wgrad_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.up), c.template p<float>(L.row_dl),
+                                                   c.template p<int32_t>(L.expert_off), c.template p<int32_t>(L.expert_cnt),
+                                                   d, acc, G.w_router, G.b_router);
+      }
+      CK(cudaGetLastError());
+    }
+  } else {
+    // every logit carries a gradient: dL is a dense [T, E] matrix and its products are matrix products
+    { ProfScope ps(TG_ROUTER_BWD, st);
+    router_bwd_dense_kernel<T><<<(unsigned)ceil_div(Tn, 128), 128, 0, st>>>(
+        c.template p<float>(L.dg_part), L.dg_ld, n_part, c.template p<float>(L.prob), c.template p<int32_t>(L.idx),
+        c.template p<int32_t>(L.tok_row), Tn, k, E, L.ld_dlf, c.template p<T>(L.dlf));
+    }
+    CK(cudaGetLastError());
+    {
+      GemmProblem p = blank_problem();   // dU_r = dL W_r
+      p.M = Tn; p.N = d; p.K = E;
+      p.A = c.template p<T>(L.dlf); p.lda = L.ld_dlf;
+      p.B0 = c.W.w_router; p.ldb = d; p.b_mn_major = 1;
+      p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dur); p.ldc = d;
+      CKR(run_gemm(c, p, TG_ROUTER_BWD));
+    }
+    if (G.w_router)
+      CKR(wgrad(TG_WG_ROUTER, G.w_router, E, d, c.template p<T>(L.dlf), L.ld_dlf, 0, c.template p<T>(L.u), d, false, 0));
+    if (G.b_router) {
+      dim3 grid((unsigned)ceil_div(E, 256), (unsigned)L.strips);
+      { ProfScope ps(TG_WG_ROUTER, st);
+      colsum_partial_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.dlf), L.ld_dlf, nullptr, Tn, E, STRIP,
+                                                     c.template p<float>(L.part));
+      }
+      CK(cudaGetLastError());
+      { ProfScope ps(TG_WG_ROUTER, st);
+      colsum_final_kernel<<<(unsigned)ceil_div(E, 256), 256, 0, st>>>(c.template p<float>(L.part), L.strips, E, acc,
+                                                                      G.b_router);
+      }
+      CK(cudaGetLastError());
+    }
   }
 
   // dU, then P_up backward and the norm
@@ -525,7 +566,8 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
                                           c.template p<int32_t>(L.idx), c.template p<float>(L.tok_dl), k,
                                           Is > 0 ? c.template p<T>(L.dush) : nullptr,
                                           reinterpret_cast<const T*>(c.W.w_router), c.template p<float>(L.dl),
-                                          reinterpret_cast<const T*>(c.W.ws_sgate), d, c.template p<T>(L.du));
+                                          reinterpret_cast<const T*>(c.W.ws_sgate),
+                                          dense_gate ? c.template p<T>(L.dur) : nullptr, d, c.template p<T>(L.du));
   }
   CK(cudaGetLastError());
   {
@@ -642,7 +684,7 @@ static int route_noalloc_launch(const revffn_moe_desc& D, const revffn_moe_weigh
   CK(launch_fold_router<T>(reinterpret_cast<const T*>(W.w_router), reinterpret_cast<const T*>(W.ws_sgate),
                            reinterpret_cast<const T*>(W.w_up), E, d, h, w_rc, st));
   CK(launch_router_topk(y1, D.ld_stream, W.norm_gamma, D.norm_eps, norm_none, w_rc, W.b_router, D.tokens, h, E,
-                        D.top_k, D.d_shared > 0 ? 1 : 0, nullptr, idx, gates, sgate, nullptr, st));
+                        D.top_k, D.d_shared > 0 ? 1 : 0, nullptr, idx, gates, sgate, nullptr, nullptr, st));
   g_prof.launches += 2;
   return REVFFN_OK;
 }
@@ -715,7 +757,7 @@ int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* 
       {"row_tok", &L.row_tok}, {"row_gate", &L.row_gate}, {"u", &L.u}, {"up", &L.up}, {"hmid", &L.hmid},
       {"o", &L.o}, {"hs", &L.hs}, {"s", &L.s}, {"z", &L.z}, {"ab", &L.ab}, {"abs", &L.abs}, {"gb", &L.gb},
       {"dz", &L.dz}, {"ds", &L.ds}, {"dl", &L.dl}, {"dop", &L.dop}, {"dg_part", &L.dg_part},
-      {"tok_dl", &L.tok_dl}, {"row_dl", &L.row_dl}, {"dup", &L.dup}, {"dush", &L.dush}, {"du", &L.du},
+      {"tok_dl", &L.tok_dl}, {"row_dl", &L.row_dl}, {"prob", &L.prob}, {"dlf", &L.dlf}, {"dup", &L.dup}, {"dush", &L.dush}, {"du", &L.du},
       {"dn", &L.dn}};
   for (auto& t : tab)
     if (strcmp(t.n, name) == 0) {

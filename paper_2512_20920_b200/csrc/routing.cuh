@@ -167,6 +167,8 @@ inline cudaError_t launch_fold_router(const T* w_router, const T* w_sgate, const
 //   phase 2: per token, k rounds of warp arg-max (ties -> lowest index), softmax
 //            over the k selected logits, sigmoid of the shared-gate logit.
 // idx_in != NULL: expert sets are taken from it (gates are still recomputed).
+// prob_out != NULL: gates are the selected entries of the softmax over ALL experts (not
+// renormalised), and that softmax is written to prob_out[T, E].
 // ---------------------------------------------------------------------------
 constexpr int RT_TOK = 64;   // tokens per block
 constexpr int RT_KC = 32;    // k-chunk
@@ -186,7 +188,7 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
                    int norm_none, const double* __restrict__ w_rc, const float* __restrict__ b_router,
                    int tokens, int h, int E, int k, int has_shared, const int32_t* __restrict__ idx_in,
                    int32_t* __restrict__ idx_out, float* __restrict__ gate_out, float* __restrict__ sgate_out,
-                   int32_t* __restrict__ idx_user) {
+                   int32_t* __restrict__ idx_user, float* __restrict__ prob_out) {
   extern __shared__ __align__(16) double smem_d[];
   const int EP = E + 1;                       // logits per token incl. the shared-gate row
   double* ns = smem_d;                        // [RT_TOK][RT_LD]  stream chunk, one row per token
@@ -343,14 +345,30 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
         if (lane == s) { mine = sel[s]; mine_i = seli[s]; }
       }
     }
+    float den;
+    if (prob_out) {
+      // softmax over all E logits (no renormalisation of the selected ones): largest logit and the sum of
+      // exponentials over every expert; the probabilities are kept for the backward pass
+      double ma = __longlong_as_double(0xfff0000000000000LL);
+      for (int e = lane; e < E; e += 32) ma = fmax(ma, L[e]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ma = fmax(ma, __shfl_xor_sync(0xffffffffu, ma, o));
+      m = ma;
+      float sa = 0.f;
+      for (int e = lane; e < E; e += 32) sa += expf((float)(L[e] - ma));
+      den = warp_sum(sa);
+      for (int e = lane; e < E; e += 32) prob_out[(int64_t)t * E + e] = expf((float)(L[e] - ma)) / den;
+    }
     float x = 0.f;
     if (lane < k) x = (float)(mine - m);
     else if (lane == k) x = (float)(-L[E]);
     const float ev = expf(x);
-    float den = (lane < k) ? ev : 0.f;
-    den += __shfl_xor_sync(0xffffffffu, den, 1);
-    den += __shfl_xor_sync(0xffffffffu, den, 2);
-    den += __shfl_xor_sync(0xffffffffu, den, 4);      // k <= 8: lanes 0..7 hold the sum
+    if (!prob_out) {
+      den = (lane < k) ? ev : 0.f;
+      den += __shfl_xor_sync(0xffffffffu, den, 1);
+      den += __shfl_xor_sync(0xffffffffu, den, 2);
+      den += __shfl_xor_sync(0xffffffffu, den, 4);      // k <= 8: lanes 0..7 hold the sum
+    }
     if (lane < k) {
       idx_out[(int64_t)t * k + lane] = mine_i;
       if (idx_user) idx_user[(int64_t)t * k + lane] = mine_i;
@@ -370,7 +388,7 @@ inline size_t router_smem_bytes(int E) {
 inline cudaError_t launch_router_topk(const float* y, int64_t ld, const float* gamma, float eps, int norm_none,
                                       const double* w_rc, const float* b_router, int tokens, int h, int E, int k,
                                       int has_shared, const int32_t* idx_in, int32_t* idx_out, float* gate_out,
-                                      float* sgate_out, int32_t* idx_user, cudaStream_t st) {
+                                      float* sgate_out, int32_t* idx_user, float* prob_out, cudaStream_t st) {
   static size_t raised[64] = {0};
   const size_t smem = router_smem_bytes(E);
   if (smem > 48 * 1024) {
@@ -386,7 +404,7 @@ inline cudaError_t launch_router_topk(const float* y, int64_t ld, const float* g
   }
   router_topk_kernel<<<(unsigned)ceil_div(tokens, RT_TOK), 256, smem, st>>>(
       y, ld, gamma, eps, norm_none, w_rc, b_router, tokens, h, E, k, has_shared, idx_in, idx_out, gate_out,
-      sgate_out, idx_user);
+      sgate_out, idx_user, prob_out);
   return cudaGetLastError();
 }
 

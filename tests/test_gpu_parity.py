@@ -59,21 +59,26 @@ def check_routing(idx_gpu, info, k):
     return idx_gpu if (~same).any() else None
 
 
-def run_all_passes(rv, cfg, w, s, tol, flags=0, norm_none=False, check_grads=True):
+def run_all_passes(rv, cfg, w, s, tol, flags=0, norm_none=False, check_grads=True, gating="renorm"):
+    if gating == "softmax_all":
+        flags |= rv.FLAG_GATE_SOFTMAX_ALL
     blk = make_block(cfg, w, flags=flags, norm_none=norm_none)
     norm = "none" if norm_none else "rms"
     y1, x2, dy2 = dev(s["y1"]), dev(s["x2"]), dev(s["dy2"])
     idx = torch.empty(cfg.tokens, cfg.top_k, dtype=torch.int32, device="cuda")
     y2 = blk.forward(y1, x2, topk_idx_out=idx)
     assert blk.status() == 0
-    y2_ref, info = orc.forward(w, s["y1"], s["x2"], cfg.top_k, cfg.norm_eps, norm)
+    y2_ref, info = orc.forward(w, s["y1"], s["x2"], cfg.top_k, cfg.norm_eps, norm, gating=gating)
     override = check_routing(idx.cpu().numpy(), info, cfg.top_k)
     if override is not None:
-        y2_ref, info = orc.forward(w, s["y1"], s["x2"], cfg.top_k, cfg.norm_eps, norm, route_override=override)
+        y2_ref, info = orc.forward(w, s["y1"], s["x2"], cfg.top_k, cfg.norm_eps, norm, route_override=override, gating=gating)
     # slot order too, where margins are clear
     clear = info["margin"] >= MARGIN
     gates = blk.buffer("gates", torch.float32)[: cfg.tokens * cfg.top_k].view(cfg.tokens, cfg.top_k).cpu().numpy()
-    assert np.allclose(gates.sum(axis=1), 1.0, atol=1e-6)
+    if gating == "renorm":
+        assert np.allclose(gates.sum(axis=1), 1.0, atol=1e-6)
+    else:
+        assert (gates.sum(axis=1) < 1.0).all() or cfg.top_k == cfg.n_experts
     assert np.allclose(gates[clear], info["gates"][clear], atol=1e-5)
     # the branch output itself (X2 = 0), so that the pass-through term does not mask its error
     zero = torch.zeros_like(x2)
@@ -86,7 +91,7 @@ def run_all_passes(rv, cfg, w, s, tol, flags=0, norm_none=False, check_grads=Tru
     x2_rec = blk.inverse(y1, y2)
     assert blk.status() == 0
     assert rel_l2(x2_rec.cpu().numpy(), s["x2"]) <= TOL_RECON
-    x2_ref, _ = orc.inverse(w, s["y1"], y2.cpu().numpy(), cfg.top_k, cfg.norm_eps, norm, route_override=override)
+    x2_ref, _ = orc.inverse(w, s["y1"], y2.cpu().numpy(), cfg.top_k, cfg.norm_eps, norm, route_override=override, gating=gating)
     assert rel_l2(x2_rec.cpu().numpy(), x2_ref) <= tol
 
     # the subtracted branch is bit-identical to the added one
@@ -98,7 +103,7 @@ def run_all_passes(rv, cfg, w, s, tol, flags=0, norm_none=False, check_grads=Tru
     grads = grad_buffers(cfg, w) if check_grads else {}
     blk.backward(y1, dy2, dy1, grads)
     assert blk.status() == 0
-    ref = orc.backward(w, s["y1"], s["dy2"], cfg.top_k, cfg.norm_eps, norm, route_override=override)
+    ref = orc.backward(w, s["y1"], s["dy2"], cfg.top_k, cfg.norm_eps, norm, route_override=override, gating=gating)
     err = rel_l2(dy1.cpu().numpy(), ref["dy1"])
     assert err <= tol, f"dY1 rel-L2 {err}"
     errs = {}
@@ -286,3 +291,19 @@ def test_many_experts(rv, kw):
     cfg = small_cfg(**kw)
     w, s = scaled_weights(cfg, 9, 4.0), make_streams(cfg, 9)
     run_all_passes(rv, cfg, w, s, TOL_BF16, check_grads=False)
+
+
+@pytest.mark.parametrize("simt", [True, False])
+@pytest.mark.parametrize("kw", [dict(), dict(n_experts=40, top_k=4, tokens=130), dict(d_shared=0, tokens=257)])
+def test_gating_without_renormalisation(rv, simt, kw):
+    """Gates taken from the softmax over all experts: forward, inverse and backward (where every
+    logit, selected or not, now carries a gradient) against the oracle in the same mode."""
+    cfg = small_cfg(**kw)
+    w, s = scaled_weights(cfg, 10, 4.0), make_streams(cfg, 10)
+    run_all_passes(rv, cfg, w, s, TOL_BF16, flags=rv.FLAG_FORCE_SIMT if simt else 0, gating="softmax_all")
+
+
+def test_gating_without_renormalisation_fp32(rv):
+    cfg = CONFIGS["C0"]
+    w, s = scaled_weights(cfg, 11, 5.0), make_streams(cfg, 11)
+    run_all_passes(rv, cfg, w, s, TOL_F32, gating="softmax_all")
