@@ -481,17 +481,19 @@ def run_stack(args, cfg):
     kw = dict(tokens=cfg.tokens, d_model=cfg.d_model, n_experts=cfg.n_experts, top_k=cfg.top_k, d_expert=cfg.d_expert,
               d_shared=cfg.d_shared, weight_dtype=rv.BF16, weights=weights, norm_eps=cfg.norm_eps)
 
-    def timed_variant(caching):
+    def timed_variant(caching, records=False):
         torch.cuda.synchronize()
         base_alloc = torch.cuda.memory_allocated()
         torch.cuda.reset_peak_memory_stats()
-        stk = rv.Stack(caching=caching, **kw)
+        stk = rv.Stack(caching=caching, flags=rv.FLAG_ROUTING_RECORD if records else 0, **kw)
         garr = stk.grads_array([gbuf] * L)
+        # routing records: forward remembers every layer's expert sets and gate values, backward runs no router
+        routing = torch.empty(L * stk.record_bytes, dtype=torch.uint8, device="cuda") if records else None
 
         def step():
             a.copy_(a0); b.copy_(b0); ga.copy_(g0); gb.copy_(g0)
-            stk.forward(a, b)
-            stk.backward(a, b, ga, gb, garr)
+            stk.forward(a, b, routing)
+            stk.backward(a, b, ga, gb, garr, topk_idx=routing)
 
         for _ in range(max(args.warmup, 3)):
             step()
@@ -522,6 +524,7 @@ def run_stack(args, cfg):
         return rec
 
     rev = timed_variant(False)
+    rec = timed_variant(False, records=True)
     cac = timed_variant(True)
 
     # reconstruction drift and routing flips per layer (diagnostic pass, not timed): layer by layer through
@@ -568,7 +571,7 @@ def run_stack(args, cfg):
                                f"each block exists here); weights drawn on the device",
                    "l2": "per-layer working set exceeds the 126 MB L2", "blocks": L},
         "gpu_launches": int(rev["launches"]), "clocks": rev["clocks"],
-        "reversible": rev, "caching": cac,
+        "reversible": rev, "reversible_with_routing_records": rec, "caching": cac,
         "memory": {"weights_bytes": w_bytes,
                    "reversible_activation_bytes": rev["activation_bytes"],
                    "caching_activation_bytes": cac["activation_bytes"],

@@ -87,6 +87,15 @@ enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                
  * gradient (through the softmax denominator), not only the selected ones.  Set the flag on every
  * pass of a block alike. */
 #define REVFFN_FLAG_GATE_SOFTMAX_ALL 8u
+/* Routing records.  With this flag topk_idx_out / topk_idx_in (and the stack's topk_idx, per layer) point
+ * to a routing record of revffn_moe_routing_record_bytes bytes instead of the bare index array: the
+ * [T, k] int32 expert indices, then (each part starting on a 16-byte boundary) the [T, k] fp32 gate
+ * weights and the [T] fp32 shared-expert gate.  forward writes the whole record; inverse and backward,
+ * given one, take routing AND gate values from it and run no router at all: the inverse then subtracts
+ * exactly the branch the forward pass added even when y1 itself is a reconstruction that differs from
+ * the original by rounding (Sec. 3.1 recomputes the router; this remembers 4(2k+1) bytes per token
+ * instead).  Combined with REVFFN_FLAG_GATE_SOFTMAX_ALL only the indices of the record are used. */
+#define REVFFN_FLAG_ROUTING_RECORD 16u
 
 /*
  * Block descriptor.  Shape constraints (else REVFFN_ERR_SHAPE):
@@ -203,7 +212,8 @@ const char* revffn_strerror(int code);
  *                    and intermediates there, backward reads them and runs no inverse.
  *
  * revffn_moe_stack_forward: for l = 0 .. n_blocks-1:  R_l += MLP_l(Norm(P_l))   (Eq. 2).
- *   topk_idx  optional int32 [n_blocks, T, k], the expert sets of every layer.
+ *   topk_idx  optional int32 [n_blocks, T, k], the expert sets of every layer (with
+ *             REVFFN_FLAG_ROUTING_RECORD: n_blocks routing records back to back).
  * revffn_moe_stack_backward: for l = n_blocks-1 .. 0:  R_l -= MLP_l(Norm(P_l)) (the inverse
  *   pass), then dP_l += J_l^T dR_l and layer l's weight gradients; the gradient pass reuses
  *   the branch evaluation of the inverse pass.  On entry stream_a/b hold the stack's
@@ -223,6 +233,9 @@ int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weig
                               float* stream_a, float* stream_b, float* grad_a, float* grad_b,
                               const revffn_moe_grads* grads, const int32_t* topk_idx, void* cache,
                               size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Size of one routing record (REVFFN_FLAG_ROUTING_RECORD), a multiple of 16.  (Planner; no paper counterpart.) */
+int revffn_moe_routing_record_bytes(const revffn_moe_desc* desc, size_t* bytes);
 
 /* Bytes at the start of a workspace that hold what REVFFN_FLAG_SAVE_ACTIVATIONS keeps for
  * the gradient pass (the rest of bwd_bytes is scratch of the gradient pass itself).

@@ -13,7 +13,8 @@ __all__ = ["Block", "Stack", "revffn_moe_saved_size", "revffn_moe_stack_cache_st
            "revffn_moe_inverse", "revffn_moe_status", "revffn_moe_workspace_size", "revffn_strerror",
            "revffn_moe_step_host", "revffn_moe_route_noalloc", "revffn_prof_enable", "revffn_prof_launches",
            "revffn_prof_collect", "RevffnError", "BF16", "F32", "NORM_RMS", "NORM_NONE", "FLAG_FORCE_SIMT",
-           "FLAG_SAVE_ACTIVATIONS", "FLAG_REUSE_ACTIVATIONS", "FLAG_GATE_SOFTMAX_ALL"]
+           "FLAG_SAVE_ACTIVATIONS", "FLAG_REUSE_ACTIVATIONS", "FLAG_GATE_SOFTMAX_ALL", "FLAG_ROUTING_RECORD",
+           "revffn_moe_routing_record_bytes"]
 
 
 def __getattr__(name):

@@ -19,6 +19,7 @@ FLAG_FORCE_SIMT = 1
 FLAG_SAVE_ACTIVATIONS = 2
 FLAG_REUSE_ACTIVATIONS = 4
 FLAG_GATE_SOFTMAX_ALL = 8
+FLAG_ROUTING_RECORD = 16
 
 WEIGHT_NAMES = ("norm_gamma", "w_up", "w_down", "w_router", "b_router", "w_gate", "w_upx", "w_downx",
                 "ws_gate", "ws_up", "ws_down", "ws_sgate")
@@ -77,6 +78,8 @@ def _load() -> C.CDLL:
     lib.revffn_moe_step_host.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.POINTER(Grads), vp, vp, vp, vp, vp, vp,
                                          vp, sz, vp, sz, vp, vp]
     lib.revffn_moe_saved_size.argtypes = [C.POINTER(Desc), C.POINTER(sz)]
+    lib.revffn_moe_routing_record_bytes.argtypes = [C.POINTER(Desc), C.POINTER(sz)]
+    lib.revffn_moe_routing_record_bytes.restype = C.c_int
     lib.revffn_moe_stack_cache_stride.argtypes = [C.POINTER(Desc), C.POINTER(sz)]
     lib.revffn_moe_stack_forward.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp, sz, vp, sz, vp]
     lib.revffn_moe_stack_backward.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp,
@@ -178,6 +181,12 @@ def revffn_moe_route_noalloc(desc: Desc, w: Weights, y1, topk_idx_out, gates_out
 def revffn_moe_saved_size(desc: Desc) -> int:
     n = C.c_size_t(0)
     _check(lib.revffn_moe_saved_size(C.byref(desc), C.byref(n)), "revffn_moe_saved_size")
+    return n.value
+
+
+def revffn_moe_routing_record_bytes(desc: Desc) -> int:
+    n = C.c_size_t(0)
+    _check(lib.revffn_moe_routing_record_bytes(C.byref(desc), C.byref(n)), "revffn_moe_routing_record_bytes")
     return n.value
 
 
@@ -340,6 +349,7 @@ class Stack:
                                                      for w in self.weights])
         self.fwd_bytes, self.bwd_bytes = revffn_moe_workspace_size(self.desc)
         self.saved_bytes = revffn_moe_saved_size(self.desc)
+        self.record_bytes = revffn_moe_routing_record_bytes(self.desc)
         self.cache_stride = revffn_moe_stack_cache_stride(self.desc)
         self.ws = torch.empty(self.bwd_bytes, dtype=torch.uint8, device="cuda")
         self.cache = torch.empty(self.cache_stride * self.n_blocks, dtype=torch.uint8, device="cuda") if caching else None

@@ -172,6 +172,21 @@ static int validate_desc(const revffn_moe_desc* D) {
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Routing record: [T*k] int32 indices | [T*k] float gates | [T] float shared gate, parts 16-byte aligned.
+struct RecordLayout { size_t gates_off, sgate_off, bytes; };
+static RecordLayout record_layout(const revffn_moe_desc& D) {
+  RecordLayout r;
+  const size_t tk = (size_t)D.tokens * D.top_k * 4;
+  r.gates_off = (size_t)round_up((int64_t)tk, 16);
+  r.sgate_off = r.gates_off + (size_t)round_up((int64_t)tk, 16);
+  r.bytes = r.sgate_off + (size_t)round_up((int64_t)D.tokens * 4, 16);
+  return r;
+}
+// Bytes between the index arrays (or routing records) of consecutive layers of a stack.
+static size_t routing_stride(const revffn_moe_desc& D) {
+  return (D.flags & REVFFN_FLAG_ROUTING_RECORD) ? record_layout(D).bytes : (size_t)D.tokens * D.top_k * 4;
+}
+
 static int validate_weights(const revffn_moe_desc& D, const revffn_moe_weights* w) {
   if (!w) return REVFFN_ERR_NULL;
   if (!w->w_up || !w->w_down || !w->w_router || !w->w_gate || !w->w_upx || !w->w_downx) return REVFFN_ERR_NULL;
@@ -262,8 +277,17 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
   }
   CK(cudaGetLastError());
 
-  // Router: fold through P_up, logits, top-k, gates
-  {
+  // Router: fold through P_up, logits, top-k, gates -- or everything from a routing record
+  const bool records = (D.flags & REVFFN_FLAG_ROUTING_RECORD) != 0;
+  const bool gate_all = (D.flags & REVFFN_FLAG_GATE_SOFTMAX_ALL) != 0;
+  const RecordLayout R = record_layout(D);
+  if (idx_in && records && !gate_all) {
+    const char* rec = reinterpret_cast<const char*>(idx_in);
+    const size_t tk = (size_t)Tn * k * 4;
+    CK(cudaMemcpyAsync(c.ws + L.idx.off, rec, tk, cudaMemcpyDeviceToDevice, st));
+    CK(cudaMemcpyAsync(c.ws + L.gates.off, rec + R.gates_off, tk, cudaMemcpyDeviceToDevice, st));
+    CK(cudaMemcpyAsync(c.ws + L.sgate.off, rec + R.sgate_off, (size_t)Tn * 4, cudaMemcpyDeviceToDevice, st));
+  } else {
     { ProfScope ps(TG_FOLD, st);
     CK(launch_fold_router<T>(reinterpret_cast<const T*>(c.W.w_router), reinterpret_cast<const T*>(c.W.ws_sgate), w_up, E,
                              d, h, c.template p<double>(L.w_rc), st));
@@ -272,7 +296,12 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     CK(launch_router_topk(y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, c.template p<double>(L.w_rc),
                           c.W.b_router, Tn, h, E, k, Is > 0 ? 1 : 0, idx_in, c.template p<int32_t>(L.idx),
                           c.template p<float>(L.gates), c.template p<float>(L.sgate), idx_user,
-                          (D.flags & REVFFN_FLAG_GATE_SOFTMAX_ALL) ? c.template p<float>(L.prob) : nullptr, st));
+                          gate_all ? c.template p<float>(L.prob) : nullptr, st));
+    }
+    if (idx_user && records) {      // complete the record the kernel has started with the indices
+      char* rec = reinterpret_cast<char*>(idx_user);
+      CK(cudaMemcpyAsync(rec + R.gates_off, c.ws + L.gates.off, (size_t)Tn * k * 4, cudaMemcpyDeviceToDevice, st));
+      CK(cudaMemcpyAsync(rec + R.sgate_off, c.ws + L.sgate.off, (size_t)Tn * 4, cudaMemcpyDeviceToDevice, st));
     }
   }
 
@@ -636,7 +665,9 @@ static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weight
   if (desc->tokens > 0 && (!y1 || !in2 || !out)) return REVFFN_ERR_NULL;
   if (!aligned16(y1) || !aligned16(in2) || !aligned16(out) || (reinterpret_cast<uintptr_t>(ws) & 255u))
     return REVFFN_ERR_ALIGN;
-  if ((reinterpret_cast<uintptr_t>(idx_in) | reinterpret_cast<uintptr_t>(idx_out)) & 3u) return REVFFN_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(idx_in) | reinterpret_cast<uintptr_t>(idx_out)) &
+      ((desc->flags & REVFFN_FLAG_ROUTING_RECORD) ? 15u : 3u))
+    return REVFFN_ERR_ALIGN;
   if (grads) {
     const float* gs[] = {grads->norm_gamma, grads->w_up, grads->w_down, grads->w_router, grads->b_router,
                          grads->w_gate, grads->w_upx, grads->w_downx, grads->ws_gate, grads->ws_up,
@@ -851,6 +882,14 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
   return REVFFN_OK;
 }
 
+int revffn_moe_routing_record_bytes(const revffn_moe_desc* desc, size_t* bytes) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  if (!bytes) return REVFFN_ERR_NULL;
+  *bytes = record_layout(*desc).bytes;
+  return REVFFN_OK;
+}
+
 int revffn_moe_saved_size(const revffn_moe_desc* desc, size_t* bytes) {
   int r = validate_desc(desc);
   if (r != REVFFN_OK) return r;
@@ -885,7 +924,7 @@ int revffn_moe_stack_forward(const revffn_moe_desc* desc, const revffn_moe_weigh
   if (cache && (cache_bytes < stride * (size_t)n_blocks || (reinterpret_cast<uintptr_t>(cache) & 255u)))
     return REVFFN_ERR_WORKSPACE;
   const size_t slot = stack_stream_slot(*desc);
-  const size_t idx_stride = (size_t)desc->tokens * desc->top_k;
+  const size_t idx_stride = routing_stride(*desc);     // bytes
   const size_t ws_need = plan_workspace(*desc).bwd_bytes;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   revffn_moe_desc d = *desc;
@@ -905,7 +944,7 @@ int revffn_moe_stack_forward(const revffn_moe_desc* desc, const revffn_moe_weigh
       lws = c + slot;
       lws_bytes = ws_need;
     }
-    CKR(revffn_moe_forward(&d, &weights[l], P, R, R, topk_idx ? topk_idx + (size_t)l * idx_stride : nullptr, lws,
+    CKR(revffn_moe_forward(&d, &weights[l], P, R, R, topk_idx ? reinterpret_cast<int32_t*>(reinterpret_cast<char*>(topk_idx) + (size_t)l * idx_stride) : nullptr, lws,
                            lws_bytes, cuda_stream));
   }
   return REVFFN_OK;
@@ -924,7 +963,7 @@ int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weig
   if (cache && (cache_bytes < stride * (size_t)n_blocks || (reinterpret_cast<uintptr_t>(cache) & 255u)))
     return REVFFN_ERR_WORKSPACE;
   const size_t slot = stack_stream_slot(*desc);
-  const size_t idx_stride = (size_t)desc->tokens * desc->top_k;
+  const size_t idx_stride = routing_stride(*desc);     // bytes
   const size_t ws_need = plan_workspace(*desc).bwd_bytes;
   revffn_moe_desc d_inv = *desc, d_bwd = *desc;
   d_inv.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS;
@@ -935,7 +974,8 @@ int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weig
     float* R = (l & 1) ? stream_a : stream_b;
     float* gP = (l & 1) ? grad_b : grad_a;
     float* gR = (l & 1) ? grad_a : grad_b;
-    const int32_t* idx = topk_idx ? topk_idx + (size_t)l * idx_stride : nullptr;
+    const int32_t* idx =
+        topk_idx ? reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(topk_idx) + (size_t)l * idx_stride) : nullptr;
     if (cache) {
       char* c = reinterpret_cast<char*>(cache) + (size_t)l * stride;
       CKR(revffn_moe_backward(&d_bwd, &weights[l], reinterpret_cast<const float*>(c), gR, gP, &grads[l], idx,

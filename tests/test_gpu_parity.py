@@ -307,3 +307,46 @@ def test_gating_without_renormalisation_fp32(rv):
     cfg = CONFIGS["C0"]
     w, s = scaled_weights(cfg, 11, 5.0), make_streams(cfg, 11)
     run_all_passes(rv, cfg, w, s, TOL_F32, gating="softmax_all")
+
+
+def test_routing_record_replaces_the_router(rv):
+    """A routing record written by forward carries indices, gate weights and the shared gate; inverse and
+    backward given the record run no router and use exactly those values, even for a perturbed y1."""
+    cfg = small_cfg(tokens=321, n_experts=8, top_k=3)
+    w, s = scaled_weights(cfg, 12, 4.0), make_streams(cfg, 12)
+    plain = make_block(cfg, w)
+    blk = make_block(cfg, w, flags=rv.FLAG_ROUTING_RECORD)
+    nrec = rv.revffn_moe_routing_record_bytes(blk.desc)
+    T, k = cfg.tokens, cfg.top_k
+    assert nrec % 16 == 0 and nrec >= T * (2 * k + 1) * 4
+    y1, x2, dy2 = dev(s["y1"]), dev(s["x2"]), dev(s["dy2"])
+    rec = torch.zeros(nrec, dtype=torch.uint8, device="cuda")
+    idx = torch.empty(T, k, dtype=torch.int32, device="cuda")
+    y2 = blk.forward(y1, x2, topk_idx_out=rec)
+    assert torch.equal(plain.forward(y1, x2, topk_idx_out=idx), y2)
+    g_off = ((T * k * 4 + 15) // 16) * 16
+    s_off = 2 * g_off
+    assert torch.equal(rec[: T * k * 4].view(torch.int32).view(T, k), idx)
+    gates_fwd = blk.buffer("gates", torch.float32)[: T * k].clone()
+    sgate_fwd = blk.buffer("sgate", torch.float32)[:T].clone()
+    assert torch.equal(rec[g_off: g_off + T * k * 4].view(torch.float32), gates_fwd)
+    assert torch.equal(rec[s_off: s_off + T * 4].view(torch.float32), sgate_fwd)
+    # same y1: the record changes nothing
+    assert torch.equal(blk.inverse(y1, y2, topk_idx_in=rec), plain.inverse(y1, y2))
+    # a y1 that is off by rounding-sized noise: gates still come from the record, bit for bit
+    y1p = y1 + 1e-6 * torch.randn_like(y1)
+    x2p = blk.inverse(y1p, y2, topk_idx_in=rec)
+    assert torch.equal(blk.buffer("gates", torch.float32)[: T * k], gates_fwd)
+    assert torch.equal(blk.buffer("sgate", torch.float32)[:T], sgate_fwd)
+    assert rel_l2(x2p.cpu().numpy(), s["x2"]) <= TOL_RECON
+    x2q = plain.inverse(y1p, y2)          # for comparison: recomputed routing on the perturbed stream
+    assert not torch.equal(plain.buffer("gates", torch.float32)[: T * k], gates_fwd)
+    assert rel_l2(x2q.cpu().numpy(), s["x2"]) <= TOL_RECON
+    # backward through the record equals backward with the remembered indices (same y1: same gates)
+    d_a, d_b = torch.zeros_like(y1), torch.zeros_like(y1)
+    g_a, g_b = grad_buffers(cfg, w), grad_buffers(cfg, w)
+    blk.backward(y1, dy2, d_a, g_a, topk_idx_in=rec)
+    plain.backward(y1, dy2, d_b, g_b, topk_idx_in=idx)
+    assert blk.status() == 0 and torch.equal(d_a, d_b)
+    for n in g_a:
+        assert torch.equal(g_a[n], g_b[n]), n

@@ -135,3 +135,38 @@ def test_empty_stack_and_bad_cache(rv):
     a0 = a.clone()
     rv.revffn_moe_stack_forward(stk.desc, stk.w, 0, a, b, None, None, stk.ws)      # zero layers: nothing happens
     assert torch.equal(a, a0)
+
+
+def test_stack_with_routing_records(rv):
+    """Remembering gate values as well as expert sets: the backward sweep runs no router, reconstructs at
+    least as well as with remembered sets alone, and returns the same gradients to rounding."""
+    L = 5
+    cfg, blocks, s = _setup(L, tokens=300, seed=13)
+    shapes = {n: v.shape for n, v in blocks[0].items()}
+    out = {}
+    for name, flags in (("idx", 0), ("rec", rv.FLAG_ROUTING_RECORD)):
+        stk = rv.Stack(tokens=cfg.tokens, d_model=cfg.d_model, n_experts=cfg.n_experts, top_k=cfg.top_k,
+                       d_expert=cfg.d_expert, d_shared=cfg.d_shared, weight_dtype=rv.BF16,
+                       weights=[to_device_weights(cfg, w) for w in blocks], norm_eps=cfg.norm_eps, flags=flags)
+        per_layer = stk.record_bytes if flags else cfg.tokens * cfg.top_k * 4
+        routing = torch.zeros(L * per_layer, dtype=torch.uint8, device="cuda")
+        a, b = dev(s["y1"]), dev(s["x2"])
+        stk.forward(a, b, routing)
+        ya, yb = a.clone(), b.clone()
+        ga, gb = dev(make_streams(cfg, 99)["dy2"]), dev(make_streams(cfg, 98)["dy2"])
+        gbuf = [{n: torch.zeros(shp, dtype=torch.float32, device="cuda") for n, shp in shapes.items()} for _ in range(L)]
+        launches0 = rv.revffn_prof_launches()
+        stk.backward(a, b, ga, gb, stk.grads_array(gbuf), topk_idx=routing)
+        assert stk.status() == 0
+        out[name] = dict(ya=ya, yb=yb, a=a, b=b, ga=ga, gb=gb, gbuf=gbuf, launches=rv.revffn_prof_launches() - launches0)
+    assert torch.equal(out["idx"]["ya"], out["rec"]["ya"]) and torch.equal(out["idx"]["yb"], out["rec"]["yb"])
+    assert out["rec"]["launches"] == out["idx"]["launches"] - 2 * L          # no router fold, no router: two launches fewer per layer
+    err = {n: max(rel_l2(o["a"].cpu().numpy(), s["y1"]), rel_l2(o["b"].cpu().numpy(), s["x2"])) for n, o in out.items()}
+    assert err["rec"] <= 1.05 * err["idx"] + 1e-7, err
+    for key in ("ga", "gb"):
+        assert rel_l2(out["rec"][key].cpu().numpy(), out["idx"][key].cpu().numpy()) <= 2e-3
+    for l in range(L):
+        for n in shapes:
+            x, y = out["rec"]["gbuf"][l][n].cpu().numpy(), out["idx"]["gbuf"][l][n].cpu().numpy()
+            if np.linalg.norm(y) > 0:
+                assert rel_l2(x, y) <= 5e-3, (l, n)
