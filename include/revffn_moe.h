@@ -348,6 +348,11 @@ typedef struct {
   const int32_t *group_off, *tile_group, *rows_total;
   int64_t b_group_stride, c_group_stride;
   int32_t a_col0, b_col0;
+  /* rows grouped: optional table of (expert, first row, rows, 0) runs of real rows, rows a multiple of
+   * 32 and at most 256, int32 x 4 each, 16-byte aligned; their number at rows_total[1].  With it the
+   * tcgen05 back end works store / gate-scale products with the rows on the MMA N side. */
+  const void* tok_chunks;
+  int32_t no_pair;                 /* tcgen05 back end: one CTA per tile even where CTA pairs apply */
 } revffn_dbg_gemm_args;
 int revffn_dbg_gemm(const revffn_dbg_gemm_args* args, int32_t* status_word_dev, void* cuda_stream);
 

@@ -56,7 +56,7 @@ class DbgGemmArgs(C.Structure):
                 ("dg_part", C.c_void_p), ("dg_ld", C.c_int32), ("group_mode", C.c_int32), ("n_groups", C.c_int32),
                 ("group_off", C.c_void_p), ("tile_group", C.c_void_p), ("rows_total", C.c_void_p),
                 ("b_group_stride", C.c_int64), ("c_group_stride", C.c_int64), ("a_col0", C.c_int32),
-                ("b_col0", C.c_int32)]
+                ("b_col0", C.c_int32), ("tok_chunks", C.c_void_p), ("no_pair", C.c_int32)]
 
 
 def _load() -> C.CDLL:

@@ -18,6 +18,9 @@
 //   GROUP_M: rows of A/C live in the padded expert-major row space; the 128-row
 //            tile i belongs to expert tile_group[i]; B/C1 are offset by
 //            expert * b_group_stride; rows >= *rows_total are not touched.
+//            With tok_chunks the tcgen05 back end may work such a product transposed:
+//            weights on the MMA M side, an expert's real rows (to a multiple of 32) on
+//            the N side, so that padding rows cost no tensor-core time.
 //   GROUP_K: one product per expert e over the rows group_off[e]..group_off[e+1]
 //            as the K range (weight gradients); output offset e * c_group_stride.
 //            With group_cnt the range may stop at the first 64-row boundary past the
@@ -49,6 +52,7 @@ struct GemmProblem {
   float* dg_part; int dg_ld;                   // DSWIGLU: per (row, n-tile) partial of <acc, H>
   int group_mode, n_groups;
   const int32_t* group_off; const int32_t* tile_group; const int32_t* rows_total;
+  const int4* tok_chunks;                      // GROUP_M, optional: (expert, first row, rows, -) runs of real rows; count at rows_total[1]
   const int32_t* group_cnt;                    // GROUP_K, optional: real rows per group (the rest up to the next offset is zero padding)
   int64_t b_group_stride, c_group_stride;
   int a_col0, b_col0;

@@ -30,6 +30,14 @@
 // traffic instead of 48 KB and six stages fit.  The even CTA issues the MMAs; its commits
 // arrive on the barriers of both CTAs, both CTAs' loads complete on its "full" barriers, and
 // both CTAs' epilogue warps release its accumulator barriers.
+//
+// Transposed pair mode (expert-grouped products with bf16 store or gate-scale epilogue): the
+// pair computes C^T.  The MMA M side holds 256 output features (rows of the expert's weight
+// matrix, 128 per CTA), the N side a run of up to 256 of the expert's token rows, real rows
+// only (rounded up to 32), taken from a chunk table built with the permutation.  Padding rows
+// then cost no tensor-core time, and these products get the pair mode's operand savings, which
+// row tiles that must not straddle experts cannot have.  The epilogue transposes each
+// 32-feature x 32-token block on its way through the staging area.
 #pragma once
 
 #include <cuda.h>
@@ -68,6 +76,8 @@ struct TcParams {
   int tiles_m, tiles_n;      // GROUP_M: tiles_m is an upper bound, the device value comes from rows_total
   int tile_n;                // logical output columns per tile
   int k_blocks;              // dense / GROUP_M
+  int tr;                    // transposed pair mode: weights on the MMA M side, an expert's token rows on the N side
+  int tiles_f;               // tr: 256-wide feature tiles per token chunk
   uint32_t idesc;
 };
 
@@ -266,6 +276,18 @@ struct TcTile {
 __device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_dev, int pair_rank = -1) {
   TcTile t;
   const GemmProblem& p = P.p;
+  if (P.tr) {
+    // w = token chunk * tiles_f + feature tile; m0 = first token row, ncols = token rows (the MMA N),
+    // n0 = first feature of this CTA's 128
+    const int ci = w / P.tiles_f, ft = w - ci * P.tiles_f;
+    t.group = 0; t.krow0 = 0; t.k_blocks = P.k_blocks; t.ncols = 0; t.m0 = t.n0 = 0;
+    t.valid = ci < p.rows_total[1];
+    if (!t.valid) return t;
+    const int4 ch = p.tok_chunks[ci];
+    t.group = ch.x; t.m0 = ch.y; t.ncols = ch.z;
+    t.n0 = ft * 2 * TC_BM + pair_rank * TC_BM;
+    return t;
+  }
   if (pair_rank >= 0) tiles_m_dev = (tiles_m_dev + 1) / 2;
   int per_group = tiles_m_dev * P.tiles_n;
   t.group = 0;
@@ -367,6 +389,25 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           if constexpr (PAIR) {
             // both CTAs' loads complete on the even CTA's barrier, which expects the bytes of both
             const uint32_t fbc = mapa_u32(full_bar(stage), 0);
+            if (P.tr) {
+              // M side: 128 rows of the expert's weights; N side: this CTA's half of the chunk's token rows
+              // (a full 128-row box either way; rows past the half are loaded and not used)
+              if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
+              const CUtensorMap* mw = &map_b0;
+              int kw = kb;
+              if (p.concat == CONCAT_K && kb >= k_half) { mw = &map_b1; kw = kb - k_half; }
+              if (!p.b_mn_major) {
+                tma_load_2d_pair(sa, mw, kw * TC_BK, t.group * p.N + t.n0, fbc);
+              } else {
+                const int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
+                const int krow = t.group * kdim + kw * TC_BK;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) tma_load_2d_pair(sa + j * 8192, mw, p.b_col0 + t.n0 + 64 * j, krow, fbc);
+              }
+              tma_load_2d_pair(sb, &map_a, kb * TC_BK, t.m0 + crank * (t.ncols / 2), fbc);
+              if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+              continue;
+            }
             const int nhalf = t.ncols / 2;       // this CTA's share of the tile's columns: 128, or 64 in a ragged last tile
             if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * (TC_A_BYTES + nhalf * TC_BK * 2));
             if (!p.a_mn_major) {
@@ -454,10 +495,12 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           tc_fence_after();
           const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
           const uint32_t sb = sa + TC_A_BYTES;
-          const uint64_t a_desc = p.a_mn_major ? make_smem_desc(sa, 8192, 1024) : make_smem_desc(sa, 16, 1024);
-          const uint64_t b_desc = p.b_mn_major ? make_smem_desc(sb, 8192, 1024) : make_smem_desc(sb, 16, 1024);
-          const uint32_t a_step = p.a_mn_major ? (2048u >> 4) : (32u >> 4);   // 16 k-elements per instruction
-          const uint32_t b_step = p.b_mn_major ? (2048u >> 4) : (32u >> 4);
+          // the M-side slot holds A (or, transposed, the weights B); the N-side slot the other operand
+          const int m_mn = P.tr ? p.b_mn_major : p.a_mn_major, n_mn = P.tr ? p.a_mn_major : p.b_mn_major;
+          const uint64_t a_desc = m_mn ? make_smem_desc(sa, 8192, 1024) : make_smem_desc(sa, 16, 1024);
+          const uint64_t b_desc = n_mn ? make_smem_desc(sb, 8192, 1024) : make_smem_desc(sb, 16, 1024);
+          const uint32_t a_step = m_mn ? (2048u >> 4) : (32u >> 4);   // 16 k-elements per instruction
+          const uint32_t b_step = n_mn ? (2048u >> 4) : (32u >> 4);
 #pragma unroll
           for (int ks = 0; ks < TC_BK / 16; ++ks) {
             if constexpr (PAIR)
@@ -536,7 +579,50 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       uint32_t r0[32];
       float f[32];
 
-      if constexpr (EPI == EPI_STORE || EPI == EPI_ROWSCALE || EPI == EPI_COUPLE || EPI == EPI_WGRAD) {
+      if (PAIR && P.tr) {
+        if constexpr (PAIR && (EPI == EPI_STORE || EPI == EPI_ROWSCALE)) {
+          // Transposed tile: this lane holds output feature t.n0 + 32 q + lane for 32 token rows per block.
+          // Lanes 2i and 2i+1 trade halves so that each ends up with feature PAIRS of single tokens (the even
+          // lane of the even tokens, the odd lane of the odd ones), which it writes as 4-byte pieces into
+          // the [32 tokens][32 features] staging block; a TMA store then writes 32 rows of 64 bytes.
+          const bool odd = lane & 1;
+#pragma unroll 1
+          for (int c = half * 32; c < t.ncols; c += 64) {
+            tmem_ld32(taddr + c, r0);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(r0[i]);
+            if constexpr (EPI == EPI_ROWSCALE) {
+              const float4* g4 = reinterpret_cast<const float4*>(p.rowscale + t.m0 + c);   // the same for every lane
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float4 g = g4[i];
+                f[4 * i] *= g.x; f[4 * i + 1] *= g.y; f[4 * i + 2] *= g.z; f[4 * i + 3] *= g.w;
+              }
+            }
+            const uint32_t off = (n_grp & 1u) * 2048u;
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+            uint8_t* blk = stg + off;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float send = odd ? f[2 * j] : f[2 * j + 1];
+              const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
+              const int tok = 2 * j + (odd ? 1 : 0);
+              const __nv_bfloat162 v = odd ? __floats2bfloat162_rn(recv, f[2 * j + 1]) : __floats2bfloat162_rn(f[2 * j], recv);
+              const int piece = lane >> 3, within = ((lane >> 1) & 3) * 4;
+              *reinterpret_cast<__nv_bfloat162*>(blk + tok * 64 + ((piece ^ ((tok >> 1) & 3)) << 4) + within) = v;
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&map_c, stg_u32 + off, t.n0 + q * 32, t.m0 + c);
+              bulk_commit();
+            }
+            ++n_grp;
+          }
+        }
+      } else if constexpr (EPI == EPI_STORE || EPI == EPI_ROWSCALE || EPI == EPI_COUPLE || EPI == EPI_WGRAD) {
         float rs = 1.f;
         if (EPI == EPI_ROWSCALE && m_ok) rs = p.rowscale[m];
         const bool f32_out = (EPI == EPI_COUPLE) || (EPI == EPI_WGRAD) || (EPI == EPI_STORE && p.out_f32);
@@ -944,10 +1030,20 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   }
   // Pair mode wherever a 256-row tile cannot straddle two experts and every column tile is 256 wide.
   // (a ragged 128-wide last tile splits into 64-column halves, which only the [K, N] storage of B can load)
-  const bool pair = p.group_mode != GROUP_M && (p.N % 256 == 0 || p.b_mn_major) && !p.no_pair;
+  const bool tr = p.group_mode == GROUP_M && p.tok_chunks != nullptr && p.N % 256 == 0 && !p.a_mn_major &&
+                  p.concat != CONCAT_N && !p.no_pair && s.n_sms % 2 == 0 &&
+                  (p.epilogue == EPI_ROWSCALE || (p.epilogue == EPI_STORE && !p.out_f32));
+  const bool pair = tr || (p.group_mode != GROUP_M && (p.N % 256 == 0 || p.b_mn_major) && !p.no_pair);
+  P.tr = tr ? 1 : 0;
+  P.tiles_f = p.N / 256;
   int64_t total = (int64_t)P.tiles_m * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
   int grid = (int)(total < s.n_sms ? total : s.n_sms);
-  if (pair) {
+  if (tr) {
+    // the number of token chunks is only known on the device: a full persistent grid
+    grid = s.n_sms;
+    P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.b_mn_major ? 1 : 0) << 15) |
+              ((uint32_t)(p.a_mn_major ? 1 : 0) << 16) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(2 * TC_BM >> 4) << 24);
+  } else if (pair) {
     total = (int64_t)((P.tiles_m + 1) / 2) * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
     const int64_t pairs = total < s.n_sms / 2 ? total : s.n_sms / 2;
     grid = (int)(2 * pairs);

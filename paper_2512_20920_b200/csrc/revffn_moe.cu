@@ -76,7 +76,8 @@ struct Buf { size_t off = 0, bytes = 0; };
 struct WsLayout {
   // forward / inverse
   Buf status, rows_total, w_rc, n, r, idx, gates, sgate, prob, local_rank, chunk_cnt, chunk_base, expert_cnt,
-      expert_off, tile_group, tok_row, row_tok, row_gate, u, up, hmid, o, hs, s, z;
+      expert_off, tile_group, tok_chunks, tok_row, row_tok, row_gate, u, up, hmid, o, hs, s, z;
+  int max_chunks = 0;
   size_t fwd_bytes = 0;
   size_t saved_bytes = 0;   // fwd region + SwiGLU pre-activations: what a saved evaluation consists of
   // backward only
@@ -120,6 +121,8 @@ static WsLayout plan_workspace(const revffn_moe_desc& D) {
   take(L.expert_cnt, (size_t)E * 4);
   take(L.expert_off, (size_t)(E + 1) * 4);
   take(L.tile_group, (size_t)L.max_tiles * 4);
+  L.max_chunks = (int)(ceil_div(T * k, TOK_CHUNK) + E);
+  take(L.tok_chunks, (size_t)L.max_chunks * 16);
   take(L.tok_row, (size_t)T * k * 4);
   take(L.row_tok, (size_t)Rp * 4);
   take(L.row_gate, (size_t)Rp * 4);
@@ -317,7 +320,7 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
   map_scan_kernel<<<1, 256, (size_t)(E + 1) * 4, st>>>(
       c.template p<int32_t>(L.chunk_cnt), L.n_chunks, E, c.template p<int32_t>(L.chunk_base),
       c.template p<int32_t>(L.expert_cnt), c.template p<int32_t>(L.expert_off), c.template p<int32_t>(L.tile_group),
-      c.template p<int32_t>(L.rows_total), L.max_tiles);
+      c.template p<int32_t>(L.rows_total), L.max_tiles, c.template p<int4>(L.tok_chunks), L.max_chunks);
   }
   CK(cudaGetLastError());
   { ProfScope ps(TG_MAP, st);
@@ -367,6 +370,7 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)d * I;
     p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
     p.rows_total = c.template p<int32_t>(L.rows_total);
+    p.tok_chunks = c.template p<int4>(L.tok_chunks);
     p.epilogue = EPI_ROWSCALE; p.rowscale = c.template p<float>(L.row_gate);
     p.C = c.template p<T>(L.o); p.ldc = d;
     CKR(run_gemm(c, p, TG_EXP_DOWN));
@@ -531,6 +535,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)I * d;
     p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
     p.rows_total = c.template p<int32_t>(L.rows_total);
+    p.tok_chunks = c.template p<int4>(L.tok_chunks);
     p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dup); p.ldc = d;
     CKR(run_gemm(c, p, TG_EXP_DU));
   }
@@ -1060,6 +1065,7 @@ int revffn_dbg_gemm(const revffn_dbg_gemm_args* a, int32_t* status_word_dev, voi
   p.group_off = a->group_off; p.tile_group = a->tile_group; p.rows_total = a->rows_total;
   p.b_group_stride = a->b_group_stride; p.c_group_stride = a->c_group_stride;
   p.a_col0 = a->a_col0; p.b_col0 = a->b_col0;
+  p.tok_chunks = reinterpret_cast<const int4*>(a->tok_chunks); p.no_pair = a->no_pair;
   p.status = status_word_dev;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (a->use_simt) return launch_gemm_simt<bf16>(p, st) == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;

@@ -432,10 +432,13 @@ __global__ void map_rank_kernel(const int32_t* __restrict__ idx, int tokens, int
   }
 }
 
+constexpr int TOK_CHUNK = 256;   // most token rows of one expert in one N-side tile
+
 __global__ void map_scan_kernel(const int32_t* __restrict__ chunk_cnt, int n_chunks, int E,
                                 int32_t* __restrict__ chunk_base, int32_t* __restrict__ expert_cnt,
                                 int32_t* __restrict__ expert_off, int32_t* __restrict__ tile_group,
-                                int32_t* __restrict__ rows_total, int max_tiles) {
+                                int32_t* __restrict__ rows_total, int max_tiles, int4* __restrict__ tok_chunks,
+                                int max_chunks) {
   extern __shared__ int32_t sm_i[];          // [E+1] padded offsets
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
     int run = 0;
@@ -453,7 +456,17 @@ __global__ void map_scan_kernel(const int32_t* __restrict__ chunk_cnt, int n_chu
       off += (int)round_up(expert_cnt[e], ROW_PAD);
     }
     sm_i[E] = off;
-    *rows_total = off;
+    rows_total[0] = off;
+    // Token chunks for the products that put tokens on the MMA N side: per expert, runs of up to
+    // TOK_CHUNK rows covering its real rows rounded up to 32 (the rounding stays inside the expert's
+    // zero padding).  Entry = (expert, first row, rows, 0); the count goes to rows_total[1].
+    int nc = 0;
+    for (int e = 0; e < E; ++e) {
+      const int n = (int)round_up(expert_cnt[e], 32);
+      for (int r = 0; r < n && nc < max_chunks; r += TOK_CHUNK)
+        tok_chunks[nc++] = make_int4(e, sm_i[e] + r, min(TOK_CHUNK, n - r), 0);
+    }
+    rows_total[1] = nc;
   }
   __syncthreads();
   for (int e = threadIdx.x; e <= E; e += blockDim.x) expert_off[e] = sm_i[e];

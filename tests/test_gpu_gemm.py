@@ -204,3 +204,68 @@ def test_grouped_rows_and_grouped_k(rv, simt):
             assert (dW[e] == 0).all()
         else:
             _close(dW[e], ref, 1e-5)
+
+
+def _chunks(counts, off):
+    out = []
+    for e, c in enumerate(counts):
+        n = ((c + 31) // 32) * 32
+        for r in range(0, n, 256):
+            out.append([e, off[e] + r, min(256, n - r), 0])
+    return out
+
+
+@pytest.mark.parametrize("counts", [[130, 0, 5, 256, 1], [700, 33, 0, 257, 64, 1000], [0, 0, 3]])
+def test_grouped_rows_with_tokens_on_the_mma_n_side(rv, counts):
+    """The transposed pair mode of the tcgen05 back end (weights on M, an expert's real rows on N) against the
+    plain evaluation and against the row-tiled mode of the same kernel: store, gate scale, K concatenation
+    with [K, N] weights."""
+    E = len(counts)
+    off, tile_group = _groups(counts)
+    rows = off[-1]
+    rows_cap = rows + 256
+    N, K = 512, 192
+    A = torch.zeros(rows_cap, K, device="cuda", dtype=torch.bfloat16)
+    for e, c in enumerate(counts):
+        A[off[e]: off[e] + c] = _bf((c, K), 20 + e)
+    W = _bf((E, N, K), 30)
+    ch = _chunks(counts, off)
+    g_off = torch.tensor(off, dtype=torch.int32, device="cuda")
+    g_tile = torch.tensor(tile_group + [0] * 8, dtype=torch.int32, device="cuda")
+    g_total = torch.tensor([rows, len(ch)], dtype=torch.int32, device="cuda")
+    g_ch = torch.tensor(ch + [[0, 0, 0, 0]], dtype=torch.int32, device="cuda")
+    scale = torch.zeros(rows_cap, device="cuda")
+    for e, c in enumerate(counts):
+        scale[off[e]: off[e] + c] = torch.rand(c, device="cuda") + 0.5
+    common = dict(M=rows_cap, N=N, K=K, A=A, B0=W, lda=K, ldb=K, ldc=N, group_mode=1, n_groups=E, group_off=g_off,
+                  tile_group=g_tile, rows_total=g_total, b_group_stride=N * K)
+    for epi in ("store", "rowscale"):
+        Ct = torch.full((rows_cap, N), 7.0, device="cuda", dtype=torch.bfloat16)
+        Cr = torch.full((rows_cap, N), 7.0, device="cuda", dtype=torch.bfloat16)
+        _call(rv, False, C=Ct, epilogue=EPI[epi], rowscale=scale, tok_chunks=g_ch, **common)
+        _call(rv, False, C=Cr, epilogue=EPI[epi], rowscale=scale, **common)
+        for e, c in enumerate(counts):
+            if c:
+                ref = A[off[e]: off[e] + c].float() @ W[e].float().T
+                if epi == "rowscale":
+                    ref = ref * scale[off[e]: off[e] + c, None]
+                _close(Ct[off[e]: off[e] + c], ref)
+                assert torch.equal(Ct[off[e]: off[e] + c], Cr[off[e]: off[e] + c])      # same products, same rounding
+            n32 = ((c + 31) // 32) * 32
+            assert (Ct[off[e] + c: off[e] + n32] == 0).all()       # rows up to the next multiple of 32: zeros
+            assert (Ct[off[e] + n32: off[e + 1]] == 7.0).all()     # further padding rows are not touched in this mode
+        assert (Ct[rows:] == 7.0).all()
+    # K concatenation with weights stored [K, N] (the shape of dU = da Wg + db Wu)
+    Kh = 128
+    A2 = torch.zeros(rows_cap, 2 * Kh, device="cuda", dtype=torch.bfloat16)
+    for e, c in enumerate(counts):
+        A2[off[e]: off[e] + c] = _bf((c, 2 * Kh), 50 + e)
+    W0, W1 = _bf((E, Kh, N), 60, 0.3), _bf((E, Kh, N), 61, 0.3)
+    Ct = torch.zeros(rows_cap, N, device="cuda", dtype=torch.bfloat16)
+    _call(rv, False, M=rows_cap, N=N, K=2 * Kh, A=A2, B0=W0, B1=W1, lda=2 * Kh, ldb=N, b_mn_major=1, concat=2, C=Ct, ldc=N,
+          epilogue=EPI["store"], group_mode=1, n_groups=E, group_off=g_off, tile_group=g_tile, rows_total=g_total,
+          b_group_stride=Kh * N, tok_chunks=g_ch)
+    for e, c in enumerate(counts):
+        if c:
+            a = A2[off[e]: off[e] + c].float()
+            _close(Ct[off[e]: off[e] + c], a[:, :Kh] @ W0[e].float() + a[:, Kh:] @ W1[e].float())
