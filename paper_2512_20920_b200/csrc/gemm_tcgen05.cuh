@@ -836,6 +836,12 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   }
   __syncthreads();
   if constexpr (PAIR) {
+    // After an abandoned wait, loads of this CTA may still be in flight (their completion is counted on the
+    // even CTA's barriers, so the per-stage drain above does not see them): give them a bounded time to land.
+    if (*abort_flag) {
+      const long long t0 = clock64();
+      while (clock64() - t0 < 4000000LL) {}
+    }
     // neither CTA frees tensor memory or leaves while the other may still signal its barriers or
     // have MMAs in flight that write its accumulators
     tc_fence_before();
