@@ -252,9 +252,10 @@ int revffn_moe_saved_size(const revffn_moe_desc* desc, size_t* bytes);
  * requires ld_stream == h.  Asynchronous on the stream like the other entry
  * points: synchronise cuda_stream before reading the host outputs.
  * copy_stream: NULL, or a second stream of the caller's on which the transfers that a
- * pass does not need at once run beside the passes (dy2 in during forward and inverse,
+ * pass does not need at once run beside the passes (the second half of y1 and x2 in while
+ * the forward pass works on the first half of the tokens, dy2 in during forward and inverse,
  * y2 out during the inverse pass, the reconstructed x2 out during backward).  The call
- * orders the two streams with events (five per device, created on its first use); when it
+ * orders the two streams with events (seven per device, created on its first use); when it
  * returns, work queued on cuda_stream afterwards follows everything of this step.
  * (Convenience for end-to-end use; no paper counterpart.)
  */

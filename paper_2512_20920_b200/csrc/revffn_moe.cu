@@ -807,12 +807,12 @@ int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* 
 // Events that order the copy stream against the compute stream in revffn_moe_step_host
 // (created on first use, per device; no timing).
 static cudaEvent_t* step_events(int* err) {
-  static cudaEvent_t ev[64][5];
+  static cudaEvent_t ev[64][7];
   static bool made[64] = {false};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = REVFFN_ERR_CUDA; return nullptr; }
   if (!made[dev]) {
-    for (int i = 0; i < 5; ++i)
+    for (int i = 0; i < 7; ++i)
       if (cudaEventCreateWithFlags(&ev[dev][i], cudaEventDisableTiming) != cudaSuccess) { *err = REVFFN_ERR_CUDA; return nullptr; }
     made[dev] = true;
   }
@@ -852,37 +852,61 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
   revffn_moe_desc d_inv = *desc, d_bwd = *desc;
   d_inv.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS;
   d_bwd.flags |= REVFFN_FLAG_REUSE_ACTIVATIONS;
-  // With a copy stream, what a pass does not need right away travels beside the passes: dy2 comes in
-  // during forward and inverse, y2 goes out during the inverse pass, the reconstructed x2 during backward.
+  // With a copy stream, what a pass does not need right away travels beside the passes: the second half of
+  // the tokens comes in while the forward pass works on the first half (tokens are independent through the
+  // branch, so two half-batch forward calls give the same y2), dy2 comes in during forward and inverse, y2 goes
+  // out during the inverse pass, the reconstructed x2 during backward.
+  const int32_t T0 = (two && desc->tokens >= 2048) ? (desc->tokens / 2 / 8) * 8 : desc->tokens;   // first part
+  const size_t n0 = (size_t)T0 * h * sizeof(float);
   if (two) {
     CK(cudaEventRecord(ev[0], st));            // everything queued on the compute stream so far (earlier steps
     CK(cudaStreamWaitEvent(cs, ev[0], 0));     // may still use the staging buffers)
   }
   if (n > 0) {
-    CK(cudaMemcpyAsync(y1, y1_host, n, cudaMemcpyHostToDevice, st));
-    CK(cudaMemcpyAsync(x2, x2_host, n, cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(y1, y1_host, n0, cudaMemcpyHostToDevice, cs));
+    CK(cudaMemcpyAsync(x2, x2_host, n0, cudaMemcpyHostToDevice, cs));
+    if (two) CK(cudaEventRecord(ev[1], cs));   // first part of y1, x2 on the device
+    if (n > n0) {
+      CK(cudaMemcpyAsync(reinterpret_cast<char*>(y1) + n0, reinterpret_cast<const char*>(y1_host) + n0, n - n0,
+                         cudaMemcpyHostToDevice, cs));
+      CK(cudaMemcpyAsync(reinterpret_cast<char*>(x2) + n0, reinterpret_cast<const char*>(x2_host) + n0, n - n0,
+                         cudaMemcpyHostToDevice, cs));
+    }
+    if (two) CK(cudaEventRecord(ev[2], cs));   // all of y1, x2 on the device
     CK(cudaMemcpyAsync(dy2, dy2_host, n, cudaMemcpyHostToDevice, cs));
     CK(cudaMemsetAsync(dy1, 0, n, st));
   }
-  if (two) CK(cudaEventRecord(ev[1], cs));     // dy2 is on the device
-  CKR(revffn_moe_forward(desc, w, y1, x2, y2, nullptr, ws, ws_bytes, cuda_stream));
+  if (two) CK(cudaEventRecord(ev[3], cs));     // dy2 is on the device
+  if (two && T0 < desc->tokens) {
+    revffn_moe_desc d_a = *desc, d_b = *desc;
+    d_a.tokens = T0;
+    d_b.tokens = desc->tokens - T0;
+    CK(cudaStreamWaitEvent(st, ev[1], 0));
+    CKR(revffn_moe_forward(&d_a, w, y1, x2, y2, nullptr, ws, ws_bytes, cuda_stream));
+    CK(cudaStreamWaitEvent(st, ev[2], 0));
+    CKR(revffn_moe_forward(&d_b, w, y1 + (size_t)T0 * h, x2 + (size_t)T0 * h, y2 + (size_t)T0 * h, nullptr, ws, ws_bytes,
+                           cuda_stream));
+  } else {
+    if (two) CK(cudaStreamWaitEvent(st, ev[2], 0));
+    CKR(revffn_moe_forward(desc, w, y1, x2, y2, nullptr, ws, ws_bytes, cuda_stream));
+  }
   if (two) {
-    CK(cudaEventRecord(ev[2], st));
-    CK(cudaStreamWaitEvent(cs, ev[2], 0));
+    CK(cudaEventRecord(ev[4], st));
+    CK(cudaStreamWaitEvent(cs, ev[4], 0));
   }
   if (n > 0) CK(cudaMemcpyAsync(y2_host, y2, n, cudaMemcpyDeviceToHost, cs));
   CKR(revffn_moe_inverse(&d_inv, w, y1, y2, x2r, nullptr, ws, ws_bytes, cuda_stream));
   if (two) {
-    CK(cudaEventRecord(ev[3], st));
-    CK(cudaStreamWaitEvent(cs, ev[3], 0));
+    CK(cudaEventRecord(ev[5], st));
+    CK(cudaStreamWaitEvent(cs, ev[5], 0));
   }
   if (n > 0) CK(cudaMemcpyAsync(x2_rec_host, x2r, n, cudaMemcpyDeviceToHost, cs));
-  if (two) CK(cudaStreamWaitEvent(st, ev[1], 0));
+  if (two) CK(cudaStreamWaitEvent(st, ev[3], 0));
   CKR(revffn_moe_backward(&d_bwd, w, y1, dy2, dy1, grads, nullptr, ws, ws_bytes, cuda_stream));
   if (n > 0) CK(cudaMemcpyAsync(dy1_host, dy1, n, cudaMemcpyDeviceToHost, st));
   if (two) {
-    CK(cudaEventRecord(ev[4], cs));            // the compute stream's completion covers the copy stream's work
-    CK(cudaStreamWaitEvent(st, ev[4], 0));
+    CK(cudaEventRecord(ev[6], cs));            // the compute stream's completion covers the copy stream's work
+    CK(cudaStreamWaitEvent(st, ev[6], 0));
   }
   return REVFFN_OK;
 }

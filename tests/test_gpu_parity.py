@@ -254,11 +254,11 @@ def test_backward_reuses_a_saved_evaluation(rv, simt):
         blk.forward(y1, x2, save=True, ws=small)
 
 
-@pytest.mark.parametrize("two_streams", [False, True])
-def test_host_step_matches_the_device_entry_points(rv, two_streams):
+@pytest.mark.parametrize("two_streams,tokens", [(False, 500), (True, 500), (True, 2100)])
+def test_host_step_matches_the_device_entry_points(rv, two_streams, tokens):
     """The host-buffer step (copies in, three passes, copies out; optionally with a second stream for the
     transfers) returns exactly what the three device entry points return."""
-    cfg = small_cfg(tokens=500)
+    cfg = small_cfg(tokens=tokens)      # from 2048 tokens on, the two-stream form runs the forward pass in two halves
     w, s = scaled_weights(cfg, 8, 4.0), make_streams(cfg, 8)
     blk = make_block(cfg, w)
     y1, x2, dy2 = dev(s["y1"]), dev(s["x2"]), dev(s["dy2"])
