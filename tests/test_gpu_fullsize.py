@@ -1,6 +1,7 @@
 """Full-size parity in the launch configuration the benchmark times: the
-Qwen1.5-MoE-A2.7B-shaped block at 8192 tokens (near-uniform routing) and at
-16384 tokens under Zipf(1.2) routing with two empty experts.
+Qwen1.5-MoE-A2.7B-shaped block at 8192 tokens (near-uniform routing), at
+16384 tokens under Zipf(1.2) routing with two empty experts, and at the two
+ends of the token sweep (512 and 65536 tokens).
 
 The oracle cannot afford the whole batch, so:
   * routing is checked for EVERY token (logits are cheap);
@@ -30,7 +31,7 @@ MARGIN = 1e-6
 N_SAMPLE = 384
 
 
-@pytest.mark.parametrize("name", ["C1", "C2"])
+@pytest.mark.parametrize("name", ["C1", "C2", "C4-512", "C4-65536"])
 def test_full_size_block(name):
     cfg = CONFIGS[name]
     T, k, E = cfg.tokens, cfg.top_k, cfg.n_experts
