@@ -7,15 +7,16 @@
 //   warp 1      MMA issuer: owns the TMEM allocation (two accumulators, so the
 //               epilogue of tile i overlaps the main loop of tile i+1); one
 //               elected lane issues tcgen05.mma kind::f16 (bf16 x bf16 -> fp32),
-//               M = 128, N = 128 or 256, K = 16 per instruction; tcgen05.commit
+//               M = 128 (256 across a CTA pair), N up to 256, K = 16 per instruction; tcgen05.commit
 //               releases stages and publishes finished accumulators.
 //   warps 2..9  epilogue (two warps per TMEM lane quadrant, alternating 32-column blocks):
-//               tcgen05.ld the accumulator (lane = tile row), apply the
-//               fused epilogue (SwiGLU, gate scale, coupling add/sub, SwiGLU
-//               backward, fp32 weight-gradient store), stage 32 x 32 output blocks in
-//               swizzled shared memory and hand them to TMA bulk tensor stores
-//               (reduce-add when a gradient is accumulated), so that global
-//               writes are whole lines whatever the row stride.
+//               tcgen05.ld the accumulator (lane = tile row), apply the fused epilogue
+//               (SwiGLU, gate scale, coupling add/sub, SwiGLU backward, fp32 weight
+//               gradient) and pass each 32 x 32 output block through a per-warp staging
+//               area in shared memory: bf16 blocks leave by TMA bulk tensor stores
+//               (64-byte swizzle), fp32 blocks are transposed there and written with plain
+//               16-byte stores, four 128-byte rows per instruction.  Global writes are whole
+//               lines whatever the row stride.
 // Tile = 128 rows x 256 columns (the last column tile of a row may be 128 wide: N only has
 // to be a multiple of 128), K step 64 (one 128-byte swizzle atom of bf16).
 // Both operands may be K-major or MN-major; MN-major tiles are fetched as
@@ -132,11 +133,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 // Shared -> global bulk tensor store of one box (the box and the swizzle come from the map).
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(src) : "memory");
-}
-// Same box added element-wise (fp32) to what global memory holds.
-__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
-  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(src) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
