@@ -75,7 +75,7 @@ struct Buf { size_t off = 0, bytes = 0; };
 
 struct WsLayout {
   // forward / inverse
-  Buf status, rows_total, w_rc, n, r, idx, gates, sgate, prob, local_rank, chunk_cnt, chunk_base, expert_cnt,
+  Buf status, rows_total, w_rc, w_rc_part, n, r, idx, gates, sgate, prob, local_rank, chunk_cnt, chunk_base, expert_cnt,
       expert_off, tile_group, tok_chunks, tok_row, row_tok, row_gate, u, up, hmid, o, hs, s, z;
   int max_chunks = 0;
   size_t fwd_bytes = 0;
@@ -109,6 +109,7 @@ static WsLayout plan_workspace(const revffn_moe_desc& D) {
   take(L.status, 256);
   take(L.rows_total, 256);
   take(L.w_rc, (size_t)(E + 1) * h * 8);
+  take(L.w_rc_part, (size_t)FOLD_SLICES * (E + 1) * h * 8);
   take(L.n, (size_t)T * h * ts);
   take(L.r, (size_t)T * 4);
   take(L.idx, (size_t)T * k * 4);
@@ -292,8 +293,14 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     CK(cudaMemcpyAsync(c.ws + L.sgate.off, rec + R.sgate_off, (size_t)Tn * 4, cudaMemcpyDeviceToDevice, st));
   } else {
     { ProfScope ps(TG_FOLD, st);
-    CK(launch_fold_router<T>(reinterpret_cast<const T*>(c.W.w_router), reinterpret_cast<const T*>(c.W.ws_sgate), w_up, E,
-                             d, h, c.template p<double>(L.w_rc), st));
+    if (d <= FOLD_SLICES * fold_slice_rows<T>()) {
+      CK(launch_fold_router_mma<T>(reinterpret_cast<const T*>(c.W.w_router), reinterpret_cast<const T*>(c.W.ws_sgate),
+                                   w_up, E, d, h, c.template p<double>(L.w_rc_part), c.template p<double>(L.w_rc), st));
+      ++g_prof.launches;      // two kernels under one timing scope: the slice products and their sum
+    } else {
+      CK(launch_fold_router<T>(reinterpret_cast<const T*>(c.W.w_router), reinterpret_cast<const T*>(c.W.ws_sgate), w_up,
+                               E, d, h, c.template p<double>(L.w_rc), st));
+    }
     }
     { ProfScope ps(TG_ROUTER, st);
     CK(launch_router_topk(y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, c.template p<double>(L.w_rc),

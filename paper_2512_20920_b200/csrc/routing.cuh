@@ -153,6 +153,111 @@ inline cudaError_t launch_fold_router(const T* w_router, const T* w_sgate, const
 }
 
 // ---------------------------------------------------------------------------
+// The same fold on the fp64 tensor-core path, K split across blocks.
+//   fold_router_mma_kernel: block (x: 64 columns i, y: 64 rows e, z: slice of rows j) computes the slice's
+//     part[z][e][i] = sum_{j in slice z} W_r'[e, j] * W_up[j, i] with mma.sync m8n8k4 (warp = 16 rows x
+//     32 columns as 2 x 4 fragments).
+//   fold_router_reduce_kernel: W_rc[e][i] = sum_z part[z][e][i], z ascending (fixed order).
+// Needs FOLD_SLICES * (E+1) * h doubles of scratch, which the workspace has; the entry point that may
+// not use a workspace keeps the FMA kernel above.
+// ---------------------------------------------------------------------------
+constexpr int FOLD_SLICES = 16;        // upper bound on the K slices
+constexpr int FM_J_BYTES = 256;        // a slice is this many bytes of a W_r' row: 128 rows j in bf16, 64 in fp32
+template <typename T> __host__ __device__ constexpr int fold_slice_rows() { return FM_J_BYTES / (int)sizeof(T); }
+constexpr int FM_PAD = 8;              // elements of padding per staged row (keeps rows 16-byte aligned)
+
+__device__ __forceinline__ void fold_dmma(double& d0, double& d1, double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d0), "+d"(d1) : "d"(a), "d"(b));
+}
+
+// The block's whole operand slices are fetched with 16-byte loads that are all in flight together
+// (one memory round trip), kept in shared memory in their storage type, and widened to fp64 as the
+// fragments are read.
+template <typename T>
+__global__ void __launch_bounds__(256)
+fold_router_mma_kernel(const T* __restrict__ w_router, const T* __restrict__ w_sgate, const T* __restrict__ w_up,
+                       int E, int d, int h, double* __restrict__ part) {
+  constexpr int PER16 = 16 / (int)sizeof(T);
+  constexpr int FM_J = fold_slice_rows<T>();
+  constexpr int LDA = FM_J + FM_PAD, LDB = 64 + FM_PAD;
+  __shared__ __align__(16) T as[64 * LDA];       // W_r' slice  [e][j]
+  __shared__ __align__(16) T bs[FM_J * LDB];     // W_up slice  [j][i]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int i0 = blockIdx.x * 64, e0 = blockIdx.y * 64, jb = blockIdx.z * FM_J;
+  const int EP = E + 1;
+  const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+  // d and h are multiples of 8, so a 16-byte piece never straddles the end of a row
+  for (int piece = tid; piece < 64 * (FM_J / PER16); piece += 256) {
+    const int ee = piece / (FM_J / PER16), jj = (piece % (FM_J / PER16)) * PER16;
+    const int e = e0 + ee, j = jb + jj;
+    const T* src = (e < E) ? (w_router + (int64_t)e * d) : (e == E ? w_sgate : nullptr);
+    *reinterpret_cast<uint4*>(&as[ee * LDA + jj]) =
+        (src != nullptr && j < d) ? *reinterpret_cast<const uint4*>(src + j) : zero4;
+  }
+  for (int piece = tid; piece < FM_J * (64 / PER16); piece += 256) {
+    const int jj = piece / (64 / PER16), ii = (piece % (64 / PER16)) * PER16;
+    const int j = jb + jj, i = i0 + ii;
+    *reinterpret_cast<uint4*>(&bs[jj * LDB + ii]) =
+        (j < d && i < h) ? *reinterpret_cast<const uint4*>(w_up + (int64_t)j * h + i) : zero4;
+  }
+  __syncthreads();
+  const int wm = warp >> 1, wn = warp & 1, fr = lane >> 2, fc = lane & 3;
+  double acc[2][4][2];
+#pragma unroll
+  for (int a = 0; a < 2; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) { acc[a][b][0] = 0.0; acc[a][b][1] = 0.0; }
+#pragma unroll 4
+  for (int kk = 0; kk < FM_J; kk += 4) {
+    double af[2], bf[4];
+#pragma unroll
+    for (int a = 0; a < 2; ++a) af[a] = (double)to_f32(as[(wm * 16 + a * 8 + fr) * LDA + kk + fc]);
+#pragma unroll
+    for (int b = 0; b < 4; ++b) bf[b] = (double)to_f32(bs[(kk + fc) * LDB + wn * 32 + b * 8 + fr]);
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) fold_dmma(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+  }
+  double* out = part + (int64_t)blockIdx.z * EP * h;
+#pragma unroll
+  for (int a = 0; a < 2; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const int e = e0 + wm * 16 + a * 8 + fr;
+        const int i = i0 + wn * 32 + b * 8 + 2 * fc + c;
+        if (e < EP && i < h) out[(int64_t)e * h + i] = acc[a][b][c];
+      }
+}
+
+__global__ void fold_router_reduce_kernel(const double* __restrict__ part, int n_slices, int64_t n,
+                                          double* __restrict__ w_rc) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  double v = part[i];
+  for (int z = 1; z < n_slices; ++z) v += part[(int64_t)z * n + i];
+  w_rc[i] = v;
+}
+
+// Returns cudaErrorInvalidValue when d needs more slices than the scratch holds (the caller then uses the FMA kernel).
+template <typename T>
+inline cudaError_t launch_fold_router_mma(const T* w_router, const T* w_sgate, const T* w_up, int E, int d, int h,
+                                          double* part, double* w_rc, cudaStream_t st) {
+  const int n_slices = (int)ceil_div(d, fold_slice_rows<T>());
+  if (n_slices > FOLD_SLICES) return cudaErrorInvalidValue;
+  dim3 grid((unsigned)ceil_div(h, 64), (unsigned)ceil_div(E + 1, 64), (unsigned)n_slices);
+  fold_router_mma_kernel<T><<<grid, 256, 0, st>>>(w_router, w_sgate, w_up, E, d, h, part);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int64_t n = (int64_t)(E + 1) * h;
+  fold_router_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n_slices, n, w_rc);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
 // Router: logits in fp64 from the fp32 stream, top-k by warp shuffles, gates.
 //   block = 256 threads, RT_TOK tokens per block.
 //   phase 1: L[t, e] = r_t <W_rc[e], y_t * gamma> (+ b_r[e]) for e < E; row E is the
