@@ -1,7 +1,8 @@
-"""B200 (sm_100a) library for the MoE coupling branch of a RevFFN block:
-forward Y2 = X2 + MLP(Norm(Y1)), its inverse, and its backward by
-recomputation.  All arithmetic runs in the CUDA library behind the C ABI in
-include/revffn_moe.h; this package only marshals arguments.
+"""B200 (sm_100a) library for the coupling branches of a RevFFN block: the MoE branch
+Y2 = X2 + MLP(Norm(Y1)) and the attention branch Y1 = X1 + Attn(Norm(X1), Norm(X2), Norm(X2)),
+each with its inverse and its backward by recomputation.  All arithmetic runs in the CUDA
+library behind the C ABI in include/revffn_moe.h and include/revffn_attn.h; this package only
+marshals arguments.
 
 Names are resolved from `binding` on first use, so that `build` can be imported
 before the shared library exists.  There is no fallback: using anything here
@@ -14,7 +15,9 @@ __all__ = ["Block", "Stack", "revffn_moe_saved_size", "revffn_moe_stack_cache_st
            "revffn_moe_step_host", "revffn_moe_route_noalloc", "revffn_prof_enable", "revffn_prof_launches",
            "revffn_prof_collect", "RevffnError", "BF16", "F32", "NORM_RMS", "NORM_NONE", "FLAG_FORCE_SIMT",
            "FLAG_SAVE_ACTIVATIONS", "FLAG_REUSE_ACTIVATIONS", "FLAG_GATE_SOFTMAX_ALL", "FLAG_ROUTING_RECORD",
-           "revffn_moe_routing_record_bytes"]
+           "revffn_moe_routing_record_bytes", "AttnBranch", "AttnDesc", "AttnWeights", "AttnGrads",
+           "revffn_attn_workspace_size", "revffn_attn_forward", "revffn_attn_inverse", "revffn_attn_backward",
+           "revffn_attn_status"]
 
 
 def __getattr__(name):

@@ -1,5 +1,5 @@
 """ctypes binding of librevffn_moe.so: the same entry points as
-include/revffn_moe.h, taking torch tensors for device memory and the current
+include/revffn_moe.h and include/revffn_attn.h, taking torch tensors for device memory and the current
 torch CUDA stream.  Argument marshalling only; no arithmetic happens here, and
 there is no fallback: a missing library is an ImportError."""
 from __future__ import annotations
@@ -46,6 +46,24 @@ class Grads(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES] + [("accumulate", C.c_int32)]
 
 
+ATTN_WEIGHT_NAMES = ("norm_gamma", "w_up", "w_down", "w_q", "w_k", "w_v", "w_o", "b_q", "b_k", "b_v")
+_ATTN_F32_ALWAYS = ("norm_gamma", "b_q", "b_k", "b_v")
+
+
+class AttnDesc(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("seq_len", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("weight_dtype", C.c_int32), ("norm_eps", C.c_float),
+                ("rope_theta", C.c_float), ("ld_stream", C.c_int64), ("flags", C.c_uint32)]
+
+
+class AttnWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ATTN_WEIGHT_NAMES]
+
+
+class AttnGrads(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ATTN_WEIGHT_NAMES] + [("accumulate", C.c_int32)]
+
+
 class DbgGemmArgs(C.Structure):
     _fields_ = [("M", C.c_int32), ("N", C.c_int32), ("K", C.c_int32), ("a_mn_major", C.c_int32),
                 ("b_mn_major", C.c_int32), ("concat", C.c_int32), ("epilogue", C.c_int32), ("out_f32", C.c_int32),
@@ -89,6 +107,15 @@ def _load() -> C.CDLL:
         getattr(lib, f).restype = C.c_int
     lib.revffn_moe_route_noalloc.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, vp, vp]
     lib.revffn_moe_route_noalloc.restype = C.c_int
+    lib.revffn_attn_workspace_size.argtypes = [C.POINTER(AttnDesc), C.POINTER(sz), C.POINTER(sz)]
+    lib.revffn_attn_forward.argtypes = [C.POINTER(AttnDesc), C.POINTER(AttnWeights), vp, vp, vp, vp, sz, vp]
+    lib.revffn_attn_inverse.argtypes = [C.POINTER(AttnDesc), C.POINTER(AttnWeights), vp, vp, vp, C.c_int32, vp, sz, vp]
+    lib.revffn_attn_backward.argtypes = [C.POINTER(AttnDesc), C.POINTER(AttnWeights), vp, vp, vp, vp, vp,
+                                         C.POINTER(AttnGrads), vp, sz, vp]
+    lib.revffn_attn_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
+    for f in ("revffn_attn_workspace_size", "revffn_attn_forward", "revffn_attn_inverse", "revffn_attn_backward",
+              "revffn_attn_status"):
+        getattr(lib, f).restype = C.c_int
     lib.revffn_prof_enable.argtypes = [C.c_int]
     lib.revffn_prof_launches.argtypes = []
     lib.revffn_prof_launches.restype = C.c_longlong
@@ -319,6 +346,91 @@ class Block:
         """A named intermediate inside the workspace (tests only)."""
         off, nbytes = ws_lookup(self.desc, name)
         return self.ws[off:off + nbytes].view(dtype)
+
+
+def _nb(t) -> int:
+    return t.numel() * t.element_size()
+
+
+def revffn_attn_workspace_size(desc: AttnDesc):
+    f, b = C.c_size_t(0), C.c_size_t(0)
+    _check(lib.revffn_attn_workspace_size(C.byref(desc), C.byref(f), C.byref(b)), "revffn_attn_workspace_size")
+    return f.value, b.value
+
+
+def revffn_attn_forward(desc: AttnDesc, w: AttnWeights, x1, x2, y1, ws, stream: Optional[int] = None):
+    _check(lib.revffn_attn_forward(C.byref(desc), C.byref(w), _ptr(x1), _ptr(x2), _ptr(y1), _ptr(ws), _nb(ws),
+                                   stream if stream is not None else _stream()), "revffn_attn_forward")
+
+
+def revffn_attn_inverse(desc: AttnDesc, w: AttnWeights, y1, x2, x1, n_iter: int, ws, stream: Optional[int] = None):
+    _check(lib.revffn_attn_inverse(C.byref(desc), C.byref(w), _ptr(y1), _ptr(x2), _ptr(x1), int(n_iter), _ptr(ws),
+                                   _nb(ws), stream if stream is not None else _stream()), "revffn_attn_inverse")
+
+
+def revffn_attn_backward(desc: AttnDesc, w: AttnWeights, x1, x2, dy1, dx1, dx2_inout, grads: AttnGrads, ws,
+                         stream: Optional[int] = None):
+    _check(lib.revffn_attn_backward(C.byref(desc), C.byref(w), _ptr(x1), _ptr(x2), _ptr(dy1), _ptr(dx1),
+                                    _ptr(dx2_inout), C.byref(grads), _ptr(ws), _nb(ws),
+                                    stream if stream is not None else _stream()), "revffn_attn_backward")
+
+
+def revffn_attn_status(ws, stream: Optional[int] = None) -> int:
+    out = C.c_int32(0)
+    _check(lib.revffn_attn_status(_ptr(ws), stream if stream is not None else _stream(), C.byref(out)),
+           "revffn_attn_status")
+    return out.value
+
+
+class AttnBranch:
+    """Descriptor, device weights and workspace of one attention coupling branch, with the three
+    passes as methods.  Pure marshalling around the C entry points."""
+
+    def __init__(self, *, batch: int, seq_len: int, d_model: int, n_heads: int, n_kv_heads: int, weight_dtype: int,
+                 weights: Dict[str, torch.Tensor], norm_eps: float = 1e-6, rope_theta: float = 1e6,
+                 ld_stream: Optional[int] = None, flags: int = 0, backward: bool = True):
+        self.desc = AttnDesc(batch, seq_len, d_model, n_heads, n_kv_heads, weight_dtype, norm_eps, rope_theta,
+                             ld_stream if ld_stream is not None else d_model // 2, flags)
+        wdt = torch.bfloat16 if weight_dtype == BF16 else torch.float32
+        self.weights = {}
+        for name in ATTN_WEIGHT_NAMES:
+            t = weights.get(name)
+            if t is None:
+                continue
+            want = torch.float32 if name in _ATTN_F32_ALWAYS else wdt
+            if t.dtype != want or not t.is_cuda or not t.is_contiguous():
+                raise ValueError(f"weight {name}: need a contiguous CUDA tensor of {want}")
+            self.weights[name] = t
+        self.w = AttnWeights(**{n: _ptr(self.weights.get(n)) for n in ATTN_WEIGHT_NAMES})
+        self.fwd_bytes, self.bwd_bytes = revffn_attn_workspace_size(self.desc)
+        self.ws = torch.empty(self.bwd_bytes if backward else self.fwd_bytes, dtype=torch.uint8, device="cuda")
+
+    def forward(self, x1, x2, y1=None):
+        if y1 is None:
+            y1 = torch.empty_like(x1)
+        revffn_attn_forward(self.desc, self.w, x1, x2, y1, self.ws)
+        return y1
+
+    def inverse(self, y1, x2, x1=None, n_iter: int = 1):
+        if x1 is None:
+            x1 = torch.empty_like(y1)
+        revffn_attn_inverse(self.desc, self.w, y1, x2, x1, n_iter, self.ws)
+        return x1
+
+    def backward(self, x1, x2, dy1, dx2_inout, dx1=None, grads: Optional[Dict[str, torch.Tensor]] = None,
+                 accumulate: bool = False):
+        grads = grads or {}
+        for n, t in grads.items():
+            if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+                raise ValueError(f"gradient {n}: need a contiguous fp32 CUDA tensor")
+        if dx1 is None:
+            dx1 = torch.empty_like(dy1)
+        g = AttnGrads(**{n: _ptr(grads.get(n)) for n in ATTN_WEIGHT_NAMES}, accumulate=1 if accumulate else 0)
+        revffn_attn_backward(self.desc, self.w, x1, x2, dy1, dx1, dx2_inout, g, self.ws)
+        return dx1
+
+    def status(self) -> int:
+        return revffn_attn_status(self.ws)
 
 
 class Stack:

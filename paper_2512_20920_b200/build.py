@@ -21,7 +21,8 @@ def _nvcc() -> str:
 def sources():
     d = os.path.join(HERE, "csrc")
     out = [os.path.join(d, f) for f in sorted(os.listdir(d)) if f.endswith((".cu", ".cuh"))]
-    out.append(os.path.join(os.path.dirname(HERE), "include", "revffn_moe.h"))
+    inc = os.path.join(os.path.dirname(HERE), "include")
+    out += [os.path.join(inc, f) for f in sorted(os.listdir(inc)) if f.endswith(".h")]
     return out
 
 

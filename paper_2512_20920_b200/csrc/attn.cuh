@@ -1,0 +1,144 @@
+// Attention coupling branch (Eq. 1): the steps of Attn_pt that are not plain matrix products.
+//
+//   rope_table        (cos, sin)(s * theta^(-2i/hd)) for every position and rotated pair, from fp64
+//   to_heads          token-major [T, n*hd] (+ bias, + rotation) -> head-major [B, n, S_pad, hd]
+//   from_heads        head-major -> token-major, optionally with the opposite rotation (backward)
+//   softmax_causal    P = softmax(scale * scores) over keys 0..s of query position s
+//   dsoftmax_causal   dS = scale * P * (dP - <P, dP>)
+//   attn_tables       row-block -> key/value group table and group offsets for the grouped products
+//
+// Head-major buffers pad every (sequence, head) to S_pad = round_up(S, ROW_PAD) rows, so that a
+// 128-row tile of a grouped product never spans two heads; the padding rows are kept at zero.
+#pragma once
+
+#include "common.cuh"
+
+namespace revffn {
+
+__global__ void rope_table_kernel(int S, int hd, double theta, float2* __restrict__ cs) {
+  const int half = hd / 2;
+  int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= S * half) return;
+  int s = idx / half, i = idx % half;
+  double ang = (double)s * pow(theta, -2.0 * (double)i / (double)hd);
+  double sn, c;
+  sincos(ang, &sn, &c);
+  cs[idx] = make_float2((float)c, (float)sn);
+}
+
+// One block per token.  in: [T, ld_in] with n heads of hd columns; out: [B, n, S_pad, hd].
+template <typename TIn, typename T>
+__global__ void to_heads_kernel(const TIn* __restrict__ in, int64_t ld_in, const float* __restrict__ bias,
+                                const float2* __restrict__ cs, int S, int Sp, int n, int hd, T* __restrict__ out) {
+  const int t = blockIdx.x, b = t / S, s = t % S, half = hd / 2;
+  const TIn* row = in + (int64_t)t * ld_in;
+  for (int p = threadIdx.x; p < n * half; p += blockDim.x) {
+    const int head = p / half, i = p % half;
+    const int c0 = head * hd + i, c1 = c0 + half;
+    float x0 = to_f32(row[c0]), x1 = to_f32(row[c1]);
+    if (bias) { x0 += bias[c0]; x1 += bias[c1]; }
+    float y0 = x0, y1 = x1;
+    if (cs) {
+      const float2 r = cs[s * half + i];
+      y0 = x0 * r.x - x1 * r.y;
+      y1 = x1 * r.x + x0 * r.y;
+    }
+    T* o = out + (((int64_t)b * n + head) * Sp + s) * hd;
+    o[i] = from_f32<T>(y0);
+    o[i + half] = from_f32<T>(y1);
+  }
+}
+
+// One block per token.  in: [B, n, S_pad, hd]; out: [T, ld_out] at column col0.  sign = -1 undoes the
+// rotation of to_heads (the transpose of a rotation), cs == NULL copies.
+template <typename TIn, typename T>
+__global__ void from_heads_kernel(const TIn* __restrict__ in, const float2* __restrict__ cs, float sign, int S, int Sp,
+                                  int n, int hd, T* __restrict__ out, int64_t ld_out, int col0) {
+  const int t = blockIdx.x, b = t / S, s = t % S, half = hd / 2;
+  T* row = out + (int64_t)t * ld_out + col0;
+  for (int p = threadIdx.x; p < n * half; p += blockDim.x) {
+    const int head = p / half, i = p % half;
+    const TIn* src = in + (((int64_t)b * n + head) * Sp + s) * hd;
+    float x0 = to_f32(src[i]), x1 = to_f32(src[i + half]);
+    float y0 = x0, y1 = x1;
+    if (cs) {
+      const float2 r = cs[s * half + i];
+      const float sn = sign * r.y;
+      y0 = x0 * r.x - x1 * sn;
+      y1 = x1 * r.x + x0 * sn;
+    }
+    row[head * hd + i] = from_f32<T>(y0);
+    row[head * hd + i + half] = from_f32<T>(y1);
+  }
+}
+
+// One warp per row of the score matrix; row = (sequence, head, s) with s < S_pad.  Keys j <= s take part;
+// the rest of the row, and every padding row, is written as zero (later products read whole rows).
+template <typename T>
+__global__ void softmax_causal_kernel(const float* __restrict__ sc, int S, int Sp, float scale_log2e, int64_t rows,
+                                      T* __restrict__ P) {
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const int s = (int)(row % Sp);
+  const float* x = sc + row * Sp;
+  T* p = P + row * Sp;
+  if (s >= S) {
+    for (int j = lane; j < Sp; j += 32) p[j] = from_f32<T>(0.f);
+    return;
+  }
+  const int n = s + 1;
+  float m = -INFINITY;
+  for (int j = lane; j < n; j += 32) m = fmaxf(m, x[j]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  float sum = 0.f;
+  for (int j = lane; j < n; j += 32) sum += exp2f((x[j] - m) * scale_log2e);
+  sum = warp_sum(sum);
+  const float inv = 1.f / sum;
+  for (int j = lane; j < Sp; j += 32) p[j] = from_f32<T>(j < n ? exp2f((x[j] - m) * scale_log2e) * inv : 0.f);
+}
+
+// Softmax backward for one row: dS = scale * P * (dP - sum_j P_j dP_j), zero beyond the causal range.
+template <typename T>
+__global__ void dsoftmax_causal_kernel(const T* __restrict__ P, const float* __restrict__ dP, int S, int Sp, float scale,
+                                       int64_t rows, T* __restrict__ dS) {
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const int s = (int)(row % Sp);
+  const T* p = P + row * Sp;
+  const float* g = dP + row * Sp;
+  T* o = dS + row * Sp;
+  if (s >= S) {
+    for (int j = lane; j < Sp; j += 32) o[j] = from_f32<T>(0.f);
+    return;
+  }
+  const int n = s + 1;
+  float dot = 0.f;
+  for (int j = lane; j < n; j += 32) dot += to_f32(p[j]) * g[j];
+  dot = warp_sum(dot);
+  for (int j = lane; j < Sp; j += 32) o[j] = from_f32<T>(j < n ? scale * to_f32(p[j]) * (g[j] - dot) : 0.f);
+}
+
+// tile_group[i] = key/value group (sequence * n_kv_heads + kv head) of the i-th 128-row block of the
+// head-major query rows; group_off[g] = first query row of group g; rows_total[0] = all rows.
+__global__ void attn_tables_kernel(int n_tiles, int tiles_per_head, int rep, int n_groups, int rows_per_group,
+                                   int32_t* __restrict__ tile_group, int32_t* __restrict__ group_off,
+                                   int32_t* __restrict__ rows_total) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_tiles) tile_group[i] = (i / tiles_per_head) / rep;
+  if (i <= n_groups) group_off[i] = i * rows_per_group;
+  if (i == 0) { rows_total[0] = n_tiles * ROW_PAD; rows_total[1] = 0; }
+}
+
+// out[t, :] = in[t, :] for fp32 streams with row strides (dx1 starts as dy1).
+__global__ void copy_stream_kernel(const float* __restrict__ in, int64_t ld_in, int tokens, int h, float* __restrict__ out,
+                                   int64_t ld_out) {
+  int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= (int64_t)tokens * h) return;
+  int t = (int)(i / h), c = (int)(i % h);
+  *reinterpret_cast<float4*>(out + (int64_t)t * ld_out + c) = *reinterpret_cast<const float4*>(in + (int64_t)t * ld_in + c);
+}
+
+}  // namespace revffn

@@ -24,7 +24,10 @@ enum Tag {
   TG_NORM, TG_FOLD, TG_ROUTER, TG_MAP, TG_PUP, TG_GATHER, TG_EXP_GATEUP, TG_EXP_DOWN, TG_SH_GATEUP, TG_SH_DOWN,
   TG_COMBINE, TG_PDOWN, TG_CAST, TG_DZ, TG_WG_PDOWN, TG_SHGATE_BWD, TG_SH_DH, TG_WG_SH_DOWN, TG_SH_DU,
   TG_WG_SH_GATE, TG_WG_SH_UP, TG_WG_SGATE, TG_GATHER_DZ, TG_EXP_DH, TG_EXP_DU, TG_WG_EXP_DOWN, TG_WG_EXP_GATE,
-  TG_WG_EXP_UP, TG_ROUTER_BWD, TG_WG_ROUTER, TG_DU_REDUCE, TG_DN, TG_WG_PUP, TG_NORM_BWD, TG_DGAMMA, TG_COUNT
+  TG_WG_EXP_UP, TG_ROUTER_BWD, TG_WG_ROUTER, TG_DU_REDUCE, TG_DN, TG_WG_PUP, TG_NORM_BWD, TG_DGAMMA,
+  // attention coupling branch
+  TG_A_TABLES, TG_A_QKV, TG_A_HEADS, TG_A_SCORES, TG_A_SOFTMAX, TG_A_PV, TG_A_WO, TG_A_WGRAD, TG_A_DGRAD, TG_A_BIAS,
+  TG_A_DP, TG_A_DKV, TG_A_DQ, TG_COUNT
 };
 static const char* kTagNames[TG_COUNT] = {
     "rmsnorm_fwd", "fold_router", "router_topk", "permute_maps", "gemm_p_up", "gather_u", "gemm_expert_gate_up_swiglu",
@@ -32,8 +35,11 @@ static const char* kTagNames[TG_COUNT] = {
     "cast_dy2", "gemm_dz", "wgrad_p_down", "shared_gate_bwd", "gemm_shared_dh_dswiglu", "wgrad_shared_down",
     "gemm_shared_du", "wgrad_shared_gate", "wgrad_shared_up", "wgrad_shared_sgate", "gather_dz",
     "gemm_expert_dh_dswiglu", "gemm_expert_du", "wgrad_expert_down", "wgrad_expert_gate", "wgrad_expert_up",
-    "router_bwd", "wgrad_router", "du_reduce", "gemm_dn", "wgrad_p_up", "rmsnorm_bwd", "dgamma"};
-static const char* kPassNames[3] = {"fwd", "inv", "bwd"};
+    "router_bwd", "wgrad_router", "du_reduce", "gemm_dn", "wgrad_p_up", "rmsnorm_bwd", "dgamma",
+    "attn_tables", "gemm_qkv", "attn_heads", "gemm_scores", "attn_softmax", "gemm_pv", "gemm_w_o", "attn_wgrad",
+    "attn_dgrad", "attn_bias_grad", "gemm_dp", "gemm_dk_dv", "gemm_dq"};
+constexpr int N_PASSES = 6;
+static const char* kPassNames[N_PASSES] = {"fwd", "inv", "bwd", "attn_fwd", "attn_inv", "attn_bwd"};
 
 struct Profiler {
   bool on = false;
@@ -1056,11 +1062,11 @@ int revffn_prof_enable(int on) {
 
 long long revffn_prof_launches(void) { return g_prof.launches; }
 
-int revffn_prof_num_slots(void) { return 3 * TG_COUNT; }
+int revffn_prof_num_slots(void) { return N_PASSES * TG_COUNT; }
 
 const char* revffn_prof_slot_name(int slot) {
-  static char buf[3 * TG_COUNT][64];
-  if (slot < 0 || slot >= 3 * TG_COUNT) return "";
+  static char buf[N_PASSES * TG_COUNT][64];
+  if (slot < 0 || slot >= N_PASSES * TG_COUNT) return "";
   snprintf(buf[slot], sizeof(buf[slot]), "%s/%s", kPassNames[slot / TG_COUNT], kTagNames[slot % TG_COUNT]);
   return buf[slot];
 }
@@ -1106,3 +1112,5 @@ int revffn_dbg_gemm(const revffn_dbg_gemm_args* a, int32_t* status_word_dev, voi
 }
 
 }  // extern "C"
+
+#include "revffn_attn.cuh"

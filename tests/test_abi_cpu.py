@@ -19,15 +19,22 @@ def rv():
 
 
 def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "revffn_moe.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(revffn_\w+)\s*\(", text)))
+    inc = os.path.join(ROOT, "include")
+    names = set()
+    for f in sorted(os.listdir(inc)):
+        if not f.endswith(".h"):
+            continue
+        text = open(os.path.join(inc, f)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(revffn_\w+)\s*\(", text))
+    return sorted(names)
 
 
 def test_header_symbols_are_exported(rv):
     names = _declared_functions()
     assert {"revffn_moe_forward", "revffn_moe_inverse", "revffn_moe_backward", "revffn_moe_workspace_size",
-            "revffn_moe_status", "revffn_strerror"} <= set(names)
+            "revffn_moe_status", "revffn_strerror", "revffn_attn_forward", "revffn_attn_inverse",
+            "revffn_attn_backward", "revffn_attn_workspace_size", "revffn_attn_status"} <= set(names)
     for n in names:
         assert hasattr(rv.lib, n), n
 
@@ -95,3 +102,27 @@ def test_ws_lookup(rv):
     assert n_u == 8192 * 2048 * 2 and off_u % 256 == 0
     with pytest.raises(rv.RevffnError):
         binding.ws_lookup(d, "no_such_buffer")
+
+
+def _attn_desc(rv, **kw):
+    base = dict(batch=4, seq_len=2048, d_model=2048, n_heads=16, n_kv_heads=16, weight_dtype=rv.BF16, norm_eps=1e-6,
+                rope_theta=1e6, ld_stream=1024, flags=0)
+    base.update(kw)
+    return rv.AttnDesc(**base)
+
+
+def test_attention_workspace_size_and_bad_descriptors(rv):
+    fwd, bwd = rv.revffn_attn_workspace_size(_attn_desc(rv))
+    rows = 4 * 16 * 2048
+    assert fwd > rows * 2048 * (4 + 2)          # the score matrix in fp32 and P in bf16
+    assert fwd < bwd < 8 * 2**30
+    f2, _ = rv.revffn_attn_workspace_size(_attn_desc(rv, seq_len=2000))     # rows padded to 128 per head
+    assert f2 > rv.revffn_attn_workspace_size(_attn_desc(rv, seq_len=1920))[0]
+    for kw in (dict(d_model=2047), dict(n_heads=15), dict(n_kv_heads=3), dict(seq_len=0), dict(batch=-1),
+               dict(n_heads=32), dict(weight_dtype=5), dict(rope_theta=0.0)):
+        with pytest.raises(rv.RevffnError) as e:
+            rv.revffn_attn_workspace_size(_attn_desc(rv, **kw))
+        assert e.value.code == -2, kw
+    with pytest.raises(rv.RevffnError) as e:
+        rv.revffn_attn_workspace_size(_attn_desc(rv, flags=rv.FLAG_SAVE_ACTIVATIONS))
+    assert e.value.code == -8

@@ -170,3 +170,70 @@ def make_weights_device(cfg: BlockConfig, seed: int = 0, block: int = 0, device:
             t[i:i + m] = v.to(t.dtype)
         out[name] = t.view(shape)
     return out
+
+
+# --------------------------------------------------------------------------- #
+# Attention coupling branch (Sec. 3.1 Eq. 1): shapes of the same base model's attention layer
+# --------------------------------------------------------------------------- #
+@dataclass(frozen=True)
+class AttnConfig:
+    name: str
+    batch: int           # sequences
+    seq_len: int         # positions per sequence; T = batch * seq_len tokens
+    d_model: int
+    n_heads: int
+    n_kv_heads: int
+    weight_dtype: str    # "f32" | "bf16"
+    norm_eps: float = 1e-6
+    rope_theta: float = 1e6
+
+    @property
+    def h(self) -> int:
+        return self.d_model // 2
+
+    @property
+    def tokens(self) -> int:
+        return self.batch * self.seq_len
+
+    @property
+    def head_dim(self) -> int:
+        return self.d_model // self.n_heads
+
+
+ATTN_CONFIGS: Dict[str, AttnConfig] = {
+    # tiny fp32 branch with grouped key/value heads and a ragged sequence length
+    "A0": AttnConfig("A0", batch=2, seq_len=40, d_model=64, n_heads=4, n_kv_heads=2, weight_dtype="f32"),
+    # Qwen1.5-MoE-A2.7B-shaped attention layer, batch 4 x seq 2048 (the token batch of C1)
+    "A1": AttnConfig("A1", batch=4, seq_len=2048, d_model=2048, n_heads=16, n_kv_heads=16, weight_dtype="bf16"),
+}
+
+_ATTN_IDS = {"norm_gamma": 41, "w_up": 42, "w_down": 43, "w_q": 44, "w_k": 45, "w_v": 46, "w_o": 47,
+             "b_q": 48, "b_k": 49, "b_v": 50, "x1": 55, "x2": 56, "dy1": 57, "dx2": 58}
+_TENSOR_IDS.update({"attn." + k: v for k, v in _ATTN_IDS.items()})
+
+
+def attn_weight_shapes(cfg: AttnConfig) -> Dict[str, tuple]:
+    d, h, dkv = cfg.d_model, cfg.h, cfg.n_kv_heads * cfg.head_dim
+    return {"norm_gamma": (h,), "w_up": (d, h), "w_down": (h, d), "w_q": (d, d), "w_k": (dkv, d), "w_v": (dkv, d),
+            "w_o": (d, d), "b_q": (d,), "b_k": (dkv,), "b_v": (dkv,)}
+
+
+def make_attn_weights(cfg: AttnConfig, seed: int = 0, std: float = 0.02, bias_std: float = 0.02) -> Dict[str, np.ndarray]:
+    """Weights of one attention branch as fp32 arrays, row-major [out, in]; with weight_dtype "bf16"
+    every matrix value is exactly representable in bf16 (norm scale and biases stay fp32)."""
+    bf = cfg.weight_dtype == "bf16"
+    w = {}
+    for name, shape in attn_weight_shapes(cfg).items():
+        if name == "norm_gamma":
+            w[name] = _normal(shape, 0.02, 1.0, seed, 0, "attn." + name, False)
+        elif name.startswith("b_"):
+            w[name] = _normal(shape, bias_std, 0.0, seed, 0, "attn." + name, False)
+        else:
+            w[name] = _normal(shape, std, 0.0, seed, 0, "attn." + name, bf)
+    return w
+
+
+def make_attn_streams(cfg: AttnConfig, seed: int = 0) -> Dict[str, np.ndarray]:
+    """Input streams X1, X2, the upstream gradient dY1 and a starting value for dX2, each [T, h] fp32 ~ N(0,1)."""
+    return {name: _normal((cfg.tokens, cfg.h), 1.0, 0.0, seed, 0, "attn." + name, False)
+            for name in ("x1", "x2", "dy1", "dx2")}
