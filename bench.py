@@ -11,6 +11,7 @@ of one Qwen1.5-MoE-A2.7B-shaped block over one batch of synthetic tokens
     python bench.py --config C3             (24-block reversible stack: tokens/s, peak memory against the
                                              activation-caching variant, reconstruction drift per layer)
     python bench.py --config C4             (token-count sweep 512 .. 65536 on the same block shape)
+    python bench.py --config A1             (the attention coupling branch, Eq. 1, of the same block shape)
 """
 from __future__ import annotations
 
@@ -584,6 +585,158 @@ def run_stack(args, cfg):
     finish()
 
 
+def attn_flops(cfg):
+    """Algorithmic flops per launch of the attention branch's matrix products, by profiler slot name.
+    Causal attention needs half of the score and value products; the whole rectangle is counted
+    where the kernel computes it, so 'useful' is stated beside it."""
+    T, d, h, hd = cfg.tokens, cfg.d_model, cfg.h, cfg.head_dim
+    dkv = cfg.n_kv_heads * hd
+    S, rows = cfg.seq_len, cfg.batch * cfg.n_heads * cfg.seq_len
+    core = 2 * rows * S * hd            # one full (rows x S x hd) product
+    return {"gemm_p_up": 2 * T * h * d, "gemm_qkv": 2 * T * d * (d + 2 * dkv) / 3, "gemm_scores": core, "gemm_pv": core,
+            "gemm_w_o": 2 * T * d * d, "gemm_p_down_couple": 2 * T * d * h, "gemm_dp": core, "gemm_dk_dv": core,
+            "gemm_dq": core, "gemm_dn": 2 * (2 * T) * d * h}
+
+
+def run_attn(args, cfg):
+    """The attention coupling branch (Eq. 1) at cfg's shape: step = forward + inverse (one fixed-point
+    iteration, Sec. 3.1) + backward by recomputation.  Prints one JSON line (rank 0)."""
+    import torch
+    import paper_2512_20920_b200 as rv
+    from workloads.generate import make_attn_streams, make_attn_weights
+
+    rank, world, local, barrier = dist_setup()
+    w_host = make_attn_weights(cfg, args.seed)
+    f32 = ("norm_gamma", "b_q", "b_k", "b_v")
+    wdt = torch.bfloat16 if cfg.weight_dtype == "bf16" else torch.float32
+    w_dev = {n: torch.from_numpy(v).cuda().to(torch.float32 if n in f32 else wdt).contiguous() for n, v in w_host.items()}
+    s_host = make_attn_streams(cfg, replica_seed(args.seed, rank))
+    br = rv.AttnBranch(batch=cfg.batch, seq_len=cfg.seq_len, d_model=cfg.d_model, n_heads=cfg.n_heads,
+                       n_kv_heads=cfg.n_kv_heads, weight_dtype=rv.BF16 if cfg.weight_dtype == "bf16" else rv.F32,
+                       weights=w_dev, norm_eps=cfg.norm_eps, rope_theta=cfg.rope_theta)
+    x1, x2, dy1 = (torch.from_numpy(s_host[n]).cuda() for n in ("x1", "x2", "dy1"))
+    y1, x1r, dx1, dx2 = torch.empty_like(x1), torch.empty_like(x1), torch.empty_like(x1), torch.zeros_like(x2)
+    grads = {n: torch.empty(v.shape, dtype=torch.float32, device="cuda") for n, v in w_dev.items()}
+
+    def step():
+        br.forward(x1, x2, y1)
+        br.inverse(y1, x2, x1r, n_iter=1)
+        br.backward(x1r, x2, dy1, dx2, dx1=dx1, grads=grads)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    assert br.status() == 0
+
+    def timed(fn, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = rv.revffn_prof_launches()
+    barrier()
+    if sampler:
+        sampler.start()
+    ms_total = timed(step, args.steps)
+    clocks = sampler.stop() if sampler else None
+    launches = rv.revffn_prof_launches() - launches0
+    assert br.status() == 0
+    rv.revffn_prof_enable(True)
+    barrier()
+    ms_prof_total = timed(step, args.steps)
+    prof = rv.revffn_prof_collect()
+    rv.revffn_prof_enable(False)
+    ms_total = max_over_ranks([ms_total], world)[0]
+    ms_step = ms_total / args.steps
+
+    # reconstruction error of the fixed-point inverse against the number of iterations (Sec. 3.1)
+    recon = {}
+    br.forward(x1, x2, y1)
+    for n in (1, 2, 3, 4):
+        xh = br.inverse(y1, x2, torch.empty_like(x1), n_iter=n)
+        recon[str(n)] = float(((xh - x1).double().norm() / x1.double().norm()).item())
+    recon["0"] = float(((y1 - x1).double().norm() / x1.double().norm()).item())
+
+    # end to end: host-resident streams in, results out, copies inside the timed region
+    pin = lambda a: torch.from_numpy(a).pin_memory()
+    hx1, hx2, hdy1 = pin(s_host["x1"]), pin(s_host["x2"]), pin(s_host["dy1"])
+    hy1, hx1r, hdx1 = (torch.empty_like(hx1).pin_memory() for _ in range(3))
+
+    def host_step():
+        x1.copy_(hx1, non_blocking=True); x2.copy_(hx2, non_blocking=True); dy1.copy_(hdy1, non_blocking=True)
+        step()
+        hy1.copy_(y1, non_blocking=True); hx1r.copy_(x1r, non_blocking=True); hdx1.copy_(dx1, non_blocking=True)
+        torch.cuda.synchronize()
+    host_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        host_step()
+    dt = max_over_ranks([time.perf_counter() - t0], world)[0]
+    if rank != 0:
+        return finish()
+
+    peaks, peak_kind = load_peaks()
+    peak_t = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
+    flops = attn_flops(cfg)
+    kernels = sorted(((ms, cnt, name, name.split("/")[1]) for name, (ms, cnt) in prof.items()), reverse=True)
+    passes = {}
+    for ms, cnt, name, kn in kernels:
+        passes[name.split("/")[0]] = passes.get(name.split("/")[0], 0.0) + ms / args.steps
+    top = [{"kernel": name, "ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps,
+            "tflops": (flops[kn] * cnt / (ms * 1e-3) / 1e12) if kn in flops and ms > 0 else None}
+           for ms, cnt, name, kn in kernels]
+    dom = next((k for k in kernels if k[3] in flops), None)
+    roofline = None
+    if dom:
+        ms, cnt, name, kn = dom
+        achieved = flops[kn] / (ms / cnt * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": name, "achieved": achieved, "peak": peak_t, "unit": "TFLOP/s",
+                    "frac": achieved / peak_t, "peak_source": f"{peak_kind} (sustained bf16 cuBLAS figure)",
+                    "traffic": None, "launch_ms": ms / cnt}
+    cpu_rec = None
+    if world == 1 and not args.no_cpu_baseline:
+        from dataclasses import replace
+        from oracle import revffn_attn_oracle as orc
+        n_seq, S = 1, min(cfg.seq_len, 256)
+        sub = {k: v.reshape(cfg.batch, cfg.seq_len, -1)[:n_seq, :S].reshape(n_seq * S, -1) for k, v in s_host.items()}
+        kw = dict(S=S, n_heads=cfg.n_heads, n_kv_heads=cfg.n_kv_heads, eps=cfg.norm_eps, theta=cfg.rope_theta)
+        t0 = time.perf_counter()
+        Y = orc.forward(w_host, sub["x1"], sub["x2"], **kw)
+        orc.inverse(w_host, Y, sub["x2"], n_iter=1, **kw)
+        orc.backward(w_host, sub["x1"], sub["x2"], sub["dy1"], **kw)
+        cdt = time.perf_counter() - t0
+        cpu_rec = {"value": n_seq * S / cdt, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+                   "sample": f"fwd+inverse+bwd over the first {S} positions of {n_seq} sequence, full weights, "
+                             f"fp64 numpy, {cdt:.1f} s"}
+    out = {
+        "metric": "RevFFN attention branch fwd+inverse+bwd tokens/s", "value": job_tokens_per_s(world, cfg.tokens, args.steps, ms_total),
+        "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: attention coupling branch of one Qwen1.5-MoE-A2.7B-shaped block, "
+                               f"{cfg.batch} sequences x {cfg.seq_len} positions per GPU, d={cfg.d_model}, "
+                               f"{cfg.n_heads} heads ({cfg.n_kv_heads} key/value heads) of {cfg.head_dim}; step = forward + "
+                               f"inverse (one fixed-point iteration) + backward by recomputation, all weight gradients in fp32",
+                   "l2": "per-step working set (score matrices alone 1 GB) exceeds the 126 MB L2",
+                   "parallelism": "independent replicas" if world > 1 else "single GPU"},
+        "passes_ms": passes, "kernels": top, "roofline": roofline, "cpu_baseline": cpu_rec,
+        "reconstruction_rel_l2_by_iterations": recon,
+        "e2e": {"value": job_tokens_per_s(world, cfg.tokens, args.steps, dt * 1e3), "unit": "tokens/s",
+                "h2d_bytes_per_step": 3 * hx1.numel() * 4, "d2h_bytes_per_step": 3 * hx1.numel() * 4,
+                "ms_per_step": 1e3 * dt / args.steps},
+        "gpu_launches": int(launches), "clocks": clocks, "peak_device_bytes": int(torch.cuda.max_memory_allocated()),
+        "workspace_bytes": {"fwd": br.fwd_bytes, "bwd": br.bwd_bytes},
+        "profiled_ms_per_step": ms_prof_total / args.steps,
+    }
+    print(json.dumps(out))
+    finish()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -601,6 +754,9 @@ def main():
                          "definition) or taken from the softmax over all experts")
     args = ap.parse_args()
     from workloads import CONFIGS
+    from workloads.generate import ATTN_CONFIGS
+    if args.config in ATTN_CONFIGS and args.impl == "ours":
+        return run_attn(args, ATTN_CONFIGS[args.config])
     if args.config == "C4":
         if args.impl == "reference":
             args.config = "C1"
