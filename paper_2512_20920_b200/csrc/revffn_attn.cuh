@@ -2,20 +2,21 @@
 // See include/revffn_attn.h for the contract of every entry point.  Included at the end of
 // revffn_moe.cu: it uses that file's launch accounting, error macros and GEMM back ends.
 //
-// Attention core as built here: per (sequence, head) the score matrix is materialised
-// (scores = Q K^T as one grouped product over all heads, fp32), a row kernel turns it into
-// the causal softmax P (operand type), and O = P V is a second grouped product.  The backward
-// pass uses the same pieces: dP = dO V^T, the row kernel for dS, then dV = P^T dO and
-// dK = dS^T Q as grouped weight-gradient-style products and dQ = dS K.
+// Attention core: forward and inverse run it as one tcgen05 kernel (flash_attn.cuh) that never
+// writes the score matrix.  The backward pass, and the CUDA-core cross-check path, materialise it:
+// scores = Q K^T as one grouped product over all heads (fp32), a row kernel turns it into the
+// causal softmax P (operand type), O = P V is a second grouped product; then dP = dO V^T, the row
+// kernel for dS, dV = P^T dO and dK = dS^T Q as grouped weight-gradient-style products, dQ = dS K.
 #pragma once
 
 #include "../../include/revffn_attn.h"
 #include "attn.cuh"
+#include "flash_attn.cuh"
 
 namespace revffn {
 
 struct AttnLayout {
-  Buf status, rows_total, tile_group, group_off, cs, n12, r12, u12, raw, qh, kh, vh, sc, p, oh, o, a;
+  Buf status, rows_total, tile_group, group_off, cs, n12, r12, u12, raw, qh, kh, vh, lse, sc, p, oh, o, a;
   size_t fwd_bytes = 0;
   Buf dyb, da, dob, doh, ds, dqh, dkh, dvh, dq, dkv, du12, dn12, part;
   size_t bwd_bytes = 0;
@@ -50,6 +51,7 @@ static AttnLayout plan_attn(const revffn_attn_desc& D) {
   take(L.qh, (size_t)L.rows * hd * ts);
   take(L.kh, (size_t)L.kv_rows * hd * ts);
   take(L.vh, (size_t)L.kv_rows * hd * ts);
+  take(L.lse, (size_t)L.rows * 4);
   take(L.sc, (size_t)L.rows * Sp * 4);
   take(L.p, (size_t)L.rows * Sp * ts);
   take(L.oh, (size_t)L.rows * hd * ts);
@@ -204,11 +206,20 @@ static GemmProblem a_grouped_rows(const ACtx<T>& c) {
   return p;
 }
 
-// scores, P and O from the head-major q, k, v; O back to token-major.
+// O (token-major) from the head-major q, k, v.  need_p: the backward pass reads P afterwards, so the score
+// matrix is materialised; otherwise the tcgen05 back end runs the attention core as one kernel.
 template <typename T>
-static int a_core(const ACtx<T>& c) {
+static int a_core(const ACtx<T>& c, bool need_p) {
   const revffn_attn_desc& D = c.D;
   const AttnLayout& L = c.L;
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (c.tc && !need_p && L.hd == FA_HD) {
+      ProfScope ps(TG_A_FLASH, c.st);
+      return launch_flash_fwd(c.template p<bf16>(L.qh), c.template p<bf16>(L.kh), c.template p<bf16>(L.vh), D.batch,
+                              D.n_heads, D.n_kv_heads, D.seq_len, L.Sp, c.template p<bf16>(L.o), D.d_model,
+                              c.template p<float>(L.lse), c.template p<int>(L.status), c.st);
+    }
+  }
   {
     GemmProblem p = a_grouped_rows(c);   // scores = Q K^T
     p.N = L.Sp; p.K = L.hd;
@@ -271,10 +282,10 @@ static int a_kv_side(const ACtx<T>& c, const float* x2) {
 }
 
 template <typename T>
-static int a_query_side(const ACtx<T>& c, const float* x1) {
+static int a_query_side(const ACtx<T>& c, const float* x1, bool need_p) {
   CKR(a_norm_up(c, x1, 0));
   CKR(a_project(c, 0, c.W.w_q, c.W.b_q, c.D.n_heads, true, c.template p<T>(c.L.qh)));
-  CKR(a_core(c));
+  CKR(a_core(c, need_p));
   return a_wo(c);
 }
 
@@ -282,7 +293,7 @@ template <typename T>
 static int a_forward(const ACtx<T>& c, const float* x1, const float* x2, float* y1) {
   CKR(a_setup(c, false));
   CKR(a_kv_side(c, x2));
-  CKR(a_query_side(c, x1));
+  CKR(a_query_side(c, x1, false));
   return a_couple(c, x1, 1.f, y1);
 }
 
@@ -302,7 +313,7 @@ static int a_inverse(const ACtx<T>& c, const float* y1, const float* x2, float* 
   CKR(a_kv_side(c, x2));
   const float* cur = y1;
   for (int it = 0; it < n_iter; ++it) {
-    CKR(a_query_side(c, cur));
+    CKR(a_query_side(c, cur, false));
     CKR(a_couple(c, y1, -1.f, x1));
     cur = x1;
   }
@@ -321,7 +332,7 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
   // recompute the branch's intermediates (Sec. 3.1: nothing was cached)
   CKR(a_setup(c, true));
   CKR(a_kv_side(c, x2));
-  CKR(a_query_side(c, x1));
+  CKR(a_query_side(c, x1, true));
 
   auto wgrad = [&](float* out, int M, int N, const void* A, int64_t lda, int a_col0, const void* B, int64_t ldb,
                    int K, int accumulate) -> int {

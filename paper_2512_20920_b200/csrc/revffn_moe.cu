@@ -27,7 +27,7 @@ enum Tag {
   TG_WG_EXP_UP, TG_ROUTER_BWD, TG_WG_ROUTER, TG_DU_REDUCE, TG_DN, TG_WG_PUP, TG_NORM_BWD, TG_DGAMMA,
   // attention coupling branch
   TG_A_TABLES, TG_A_QKV, TG_A_HEADS, TG_A_SCORES, TG_A_SOFTMAX, TG_A_PV, TG_A_WO, TG_A_WGRAD, TG_A_DGRAD, TG_A_BIAS,
-  TG_A_DP, TG_A_DKV, TG_A_DQ, TG_COUNT
+  TG_A_DP, TG_A_DKV, TG_A_DQ, TG_A_FLASH, TG_COUNT
 };
 static const char* kTagNames[TG_COUNT] = {
     "rmsnorm_fwd", "fold_router", "router_topk", "permute_maps", "gemm_p_up", "gather_u", "gemm_expert_gate_up_swiglu",
@@ -37,7 +37,7 @@ static const char* kTagNames[TG_COUNT] = {
     "gemm_expert_dh_dswiglu", "gemm_expert_du", "wgrad_expert_down", "wgrad_expert_gate", "wgrad_expert_up",
     "router_bwd", "wgrad_router", "du_reduce", "gemm_dn", "wgrad_p_up", "rmsnorm_bwd", "dgamma",
     "attn_tables", "gemm_qkv", "attn_heads", "gemm_scores", "attn_softmax", "gemm_pv", "gemm_w_o", "attn_wgrad",
-    "attn_dgrad", "attn_bias_grad", "gemm_dp", "gemm_dk_dv", "gemm_dq"};
+    "attn_dgrad", "attn_bias_grad", "gemm_dp", "gemm_dk_dv", "gemm_dq", "flash_attention"};
 constexpr int N_PASSES = 6;
 static const char* kPassNames[N_PASSES] = {"fwd", "inv", "bwd", "attn_fwd", "attn_inv", "attn_bwd"};
 
