@@ -45,6 +45,40 @@ __device__ __forceinline__ float fa_exp2(float x) {
   return y;
 }
 
+// Row maximum over this thread's 64 scores.  DIAG: the diagonal block, where key c of the block is masked
+// for query row `row` when c > row (col0 = first key of this thread's half).
+template <bool DIAG>
+__device__ __forceinline__ float fa_row_max(const uint32_t (&r0)[32], const uint32_t (&r1)[32], int col0, int row) {
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    if (!DIAG || col0 + i <= row) mx = fmaxf(mx, __uint_as_float(r0[i]));
+    if (!DIAG || col0 + 32 + i <= row) mx = fmaxf(mx, __uint_as_float(r1[i]));
+  }
+  return mx;
+}
+
+// p = exp2(s * cl - mc) for this thread's 64 scores, packed to bf16 (eight 16-byte pieces); returns their sum.
+template <bool DIAG>
+__device__ __forceinline__ float fa_probs(const uint32_t (&r0)[32], const uint32_t (&r1)[32], float cl, float mc, int col0,
+                                          int row, uint4 (&pk)[8]) {
+  float sum = 0.f;
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    float pv[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int kk = 8 * g + i;
+      float p = fa_exp2(__uint_as_float(kk < 32 ? r0[kk] : r1[kk - 32]) * cl - mc);
+      if (DIAG && col0 + kk > row) p = 0.f;
+      pv[i] = p;
+      sum += p;
+    }
+    pk[g] = pack8(pv);
+  }
+  return sum;
+}
+
 struct FlashParams {
   int S, Sp, n_heads, rep;        // rep = query heads per key/value head
   bf16* o; int64_t ld_o;          // [T, ld_o]
@@ -230,11 +264,7 @@ flash_fwd_kernel(const FlashParams P, const __grid_constant__ CUtensorMap map_q,
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(B_SEMPTY + b));
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          if (!diag || 64 * half + i <= row) mx = fmaxf(mx, __uint_as_float(r0[i]));
-          if (!diag || 64 * half + 32 + i <= row) mx = fmaxf(mx, __uint_as_float(r1[i]));
-        }
+        mx = diag ? fa_row_max<true>(r0, r1, 64 * half, row) : fa_row_max<false>(r0, r1, 64 * half, row);
         xmax[(b * 2 + half) * FA_BLK + row] = mx;
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -242,21 +272,9 @@ flash_fwd_kernel(const FlashParams P, const __grid_constant__ CUtensorMap map_q,
         const float m_new = fmaxf(m, fmaxf(mx, xmax[(b * 2 + (half ^ 1)) * FA_BLK + row]));
         const float alpha = fa_exp2((m - m_new) * cl);        // first block: exp2(-inf) = 0
         const float mc = m_new * cl;
-        float sum = 0.f;
         uint4 pk[8];                             // this thread's 64 probabilities as bf16
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          float pv[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int kk = 8 * g + i;
-            float p = fa_exp2(__uint_as_float(kk < 32 ? r0[kk] : r1[kk - 32]) * cl - mc);
-            if (diag && 64 * half + kk > row) p = 0.f;
-            pv[i] = p;
-            sum += p;
-          }
-          pk[g] = pack8(pv);
-        }
+        const float sum = diag ? fa_probs<true>(r0, r1, cl, mc, 64 * half, row, pk)
+                               : fa_probs<false>(r0, r1, cl, mc, 64 * half, row, pk);
         l = l * alpha + sum;
         m = m_new;
         // P has one buffer: the previous block's P V product must have read it
