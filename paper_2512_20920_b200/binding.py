@@ -1,5 +1,5 @@
 """ctypes binding of librevffn_moe.so: the same entry points as
-include/revffn_moe.h and include/revffn_attn.h, taking torch tensors for device memory and the current
+include/revffn_moe.h, include/revffn_attn.h and include/revffn_block.h, taking torch tensors for device memory and the current
 torch CUDA stream.  Argument marshalling only; no arithmetic happens here, and
 there is no fallback: a missing library is an ImportError."""
 from __future__ import annotations
@@ -64,6 +64,10 @@ class AttnGrads(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ATTN_WEIGHT_NAMES] + [("accumulate", C.c_int32)]
 
 
+class BlockDesc(C.Structure):
+    _fields_ = [("attn", AttnDesc), ("moe", Desc), ("inverse_iters", C.c_int32)]
+
+
 class DbgGemmArgs(C.Structure):
     _fields_ = [("M", C.c_int32), ("N", C.c_int32), ("K", C.c_int32), ("a_mn_major", C.c_int32),
                 ("b_mn_major", C.c_int32), ("concat", C.c_int32), ("epilogue", C.c_int32), ("out_f32", C.c_int32),
@@ -115,6 +119,17 @@ def _load() -> C.CDLL:
     lib.revffn_attn_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
     for f in ("revffn_attn_workspace_size", "revffn_attn_forward", "revffn_attn_inverse", "revffn_attn_backward",
               "revffn_attn_status"):
+        getattr(lib, f).restype = C.c_int
+    bd, aw, mw, ag, mg = (C.POINTER(t) for t in (BlockDesc, AttnWeights, Weights, AttnGrads, Grads))
+    lib.revffn_block_workspace_size.argtypes = [bd, C.POINTER(sz), C.POINTER(sz)]
+    lib.revffn_block_forward.argtypes = [bd, aw, mw, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.revffn_block_inverse.argtypes = [bd, aw, mw, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.revffn_block_backward.argtypes = [bd, aw, mw, vp, vp, vp, vp, ag, mg, vp, vp, sz, vp]
+    lib.revffn_block_stack_forward.argtypes = [bd, aw, mw, C.c_int32, vp, vp, vp, vp, sz, vp]
+    lib.revffn_block_stack_backward.argtypes = [bd, aw, mw, C.c_int32, vp, vp, vp, vp, ag, mg, vp, vp, sz, vp]
+    lib.revffn_block_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
+    for f in ("revffn_block_workspace_size", "revffn_block_forward", "revffn_block_inverse", "revffn_block_backward",
+              "revffn_block_stack_forward", "revffn_block_stack_backward", "revffn_block_status"):
         getattr(lib, f).restype = C.c_int
     lib.revffn_prof_enable.argtypes = [C.c_int]
     lib.revffn_prof_launches.argtypes = []
@@ -431,6 +446,104 @@ class AttnBranch:
 
     def status(self) -> int:
         return revffn_attn_status(self.ws)
+
+
+def _st(stream):
+    return stream if stream is not None else _stream()
+
+
+def revffn_block_workspace_size(desc: BlockDesc):
+    f, b = C.c_size_t(0), C.c_size_t(0)
+    _check(lib.revffn_block_workspace_size(C.byref(desc), C.byref(f), C.byref(b)), "revffn_block_workspace_size")
+    return f.value, b.value
+
+
+def revffn_block_forward(desc, wa, wm, x1, x2, y1, y2, topk_idx_out, ws, stream=None):
+    _check(lib.revffn_block_forward(C.byref(desc), C.byref(wa), C.byref(wm), _ptr(x1), _ptr(x2), _ptr(y1), _ptr(y2),
+                                    _ptr(topk_idx_out), _ptr(ws), _nb(ws), _st(stream)), "revffn_block_forward")
+
+
+def revffn_block_inverse(desc, wa, wm, y1, y2, x1, x2, topk_idx_in, ws, stream=None):
+    _check(lib.revffn_block_inverse(C.byref(desc), C.byref(wa), C.byref(wm), _ptr(y1), _ptr(y2), _ptr(x1), _ptr(x2),
+                                    _ptr(topk_idx_in), _ptr(ws), _nb(ws), _st(stream)), "revffn_block_inverse")
+
+
+def revffn_block_backward(desc, wa, wm, s1, s2, g1, g2, ga, gm, topk_idx_in, ws, stream=None):
+    _check(lib.revffn_block_backward(C.byref(desc), C.byref(wa), C.byref(wm), _ptr(s1), _ptr(s2), _ptr(g1), _ptr(g2),
+                                     C.byref(ga), C.byref(gm), _ptr(topk_idx_in), _ptr(ws), _nb(ws), _st(stream)),
+           "revffn_block_backward")
+
+
+def revffn_block_stack_forward(desc, wa_array, wm_array, n_blocks, s1, s2, topk_idx, ws, stream=None):
+    _check(lib.revffn_block_stack_forward(C.byref(desc), wa_array, wm_array, int(n_blocks), _ptr(s1), _ptr(s2),
+                                          _ptr(topk_idx), _ptr(ws), _nb(ws), _st(stream)), "revffn_block_stack_forward")
+
+
+def revffn_block_stack_backward(desc, wa_array, wm_array, n_blocks, s1, s2, g1, g2, ga_array, gm_array, topk_idx, ws,
+                                stream=None):
+    _check(lib.revffn_block_stack_backward(C.byref(desc), wa_array, wm_array, int(n_blocks), _ptr(s1), _ptr(s2), _ptr(g1),
+                                           _ptr(g2), ga_array, gm_array, _ptr(topk_idx), _ptr(ws), _nb(ws), _st(stream)),
+           "revffn_block_stack_backward")
+
+
+def revffn_block_status(ws, stream=None) -> int:
+    out = C.c_int32(0)
+    _check(lib.revffn_block_status(_ptr(ws), _st(stream), C.byref(out)), "revffn_block_status")
+    return out.value
+
+
+class RevStack:
+    """n_blocks whole RevFFN blocks (attention branch then MoE branch per block): descriptors, per-layer device
+    weights and one workspace.  Pure marshalling around revffn_block_stack_forward / _backward; a single block is
+    the case n_blocks = 1."""
+
+    def __init__(self, *, batch: int, seq_len: int, d_model: int, n_heads: int, n_kv_heads: int, n_experts: int,
+                 top_k: int, d_expert: int, d_shared: int, weight_dtype: int, attn_weights, moe_weights,
+                 inverse_iters: int = 1, norm_eps: float = 1e-6, rope_theta: float = 1e6, flags: int = 0,
+                 moe_flags: int = 0, backward: bool = True):
+        h = d_model // 2
+        self.n_blocks = len(attn_weights)
+        if len(moe_weights) != self.n_blocks:
+            raise ValueError("one attention and one MoE weight set per block")
+        self.desc = BlockDesc(AttnDesc(batch, seq_len, d_model, n_heads, n_kv_heads, weight_dtype, norm_eps, rope_theta, h,
+                                       flags),
+                              Desc(batch * seq_len, d_model, n_experts, top_k, d_expert, d_shared, weight_dtype, NORM_RMS,
+                                   norm_eps, h, flags | moe_flags), inverse_iters)
+        self._keep = (attn_weights, moe_weights)            # the structs hold raw pointers into these tensors
+        self.wa = (AttnWeights * self.n_blocks)(*[AttnWeights(**{n: _ptr(w.get(n)) for n in ATTN_WEIGHT_NAMES})
+                                                  for w in attn_weights])
+        self.wm = (Weights * self.n_blocks)(*[Weights(**{n: _ptr(w.get(n)) for n in WEIGHT_NAMES}) for w in moe_weights])
+        self.fwd_bytes, self.bwd_bytes = revffn_block_workspace_size(self.desc)
+        self.ws = torch.empty(self.bwd_bytes if backward else self.fwd_bytes, dtype=torch.uint8, device="cuda")
+
+    def with_iters(self, n: int) -> BlockDesc:
+        d = BlockDesc()
+        C.memmove(C.byref(d), C.byref(self.desc), C.sizeof(BlockDesc))
+        d.inverse_iters = n
+        return d
+
+    def grads_arrays(self, attn_grads, moe_grads, accumulate: bool = False):
+        """attn_grads / moe_grads: one dict of fp32 gradient tensors per block (blocks may share tensors)."""
+        acc = 1 if accumulate else 0
+        ga = (AttnGrads * self.n_blocks)(*[AttnGrads(**{n: _ptr(g.get(n)) for n in ATTN_WEIGHT_NAMES}, accumulate=acc)
+                                           for g in attn_grads])
+        gm = (Grads * self.n_blocks)(*[Grads(**{n: _ptr(g.get(n)) for n in WEIGHT_NAMES}, accumulate=acc)
+                                       for g in moe_grads])
+        return ga, gm
+
+    def forward(self, s1, s2, topk_idx=None):
+        revffn_block_stack_forward(self.desc, self.wa, self.wm, self.n_blocks, s1, s2, topk_idx, self.ws)
+
+    def backward(self, s1, s2, g1, g2, ga, gm, topk_idx=None, inverse_iters: Optional[int] = None):
+        d = self.desc if inverse_iters is None else self.with_iters(inverse_iters)
+        revffn_block_stack_backward(d, self.wa, self.wm, self.n_blocks, s1, s2, g1, g2, ga, gm, topk_idx, self.ws)
+
+    def inverse_block(self, l: int, y1, y2, x1, x2, topk_idx_in=None, inverse_iters: Optional[int] = None):
+        d = self.desc if inverse_iters is None else self.with_iters(inverse_iters)
+        revffn_block_inverse(d, self.wa[l], self.wm[l], y1, y2, x1, x2, topk_idx_in, self.ws)
+
+    def status(self) -> int:
+        return revffn_block_status(self.ws)
 
 
 class Stack:

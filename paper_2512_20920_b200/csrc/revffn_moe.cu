@@ -1114,3 +1114,4 @@ int revffn_dbg_gemm(const revffn_dbg_gemm_args* a, int32_t* status_word_dev, voi
 }  // extern "C"
 
 #include "revffn_attn.cuh"
+#include "revffn_block.cuh"
