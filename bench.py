@@ -12,6 +12,8 @@ of one Qwen1.5-MoE-A2.7B-shaped block over one batch of synthetic tokens
                                              activation-caching variant, reconstruction drift per layer)
     python bench.py --config C4             (token-count sweep 512 .. 65536 on the same block shape)
     python bench.py --config A1             (the attention coupling branch, Eq. 1, of the same block shape)
+    python bench.py --config B3             (24 whole RevFFN blocks, both branches: reversible training step,
+                                             memory, reconstruction error against fixed-point iterations; B1: one block)
 """
 from __future__ import annotations
 
@@ -585,6 +587,140 @@ def run_stack(args, cfg):
     finish()
 
 
+def run_block_stack(args, acfg, mcfg, layers):
+    """B3 / B1: a stack of whole RevFFN blocks (Eq. 1 then Eq. 2 per block); step = forward through all layers +
+    reversible back-propagation (every layer's inputs rebuilt from its outputs, nothing cached)."""
+    import torch
+    import paper_2512_20920_b200 as rv
+    from workloads import make_weights_device, weight_shapes
+    from workloads.generate import attn_weight_shapes, make_attn_streams, make_attn_weights_device
+    rank, world, local, barrier = dist_setup()
+    L = args.blocks or layers
+    wm = [make_weights_device(mcfg, args.seed, block=l) for l in range(L)]
+    wa = [make_attn_weights_device(acfg, args.seed, block=l) for l in range(L)]
+    w_bytes = sum(t.numel() * t.element_size() for ws in (wm, wa) for w in ws for t in w.values())
+    s_host = make_attn_streams(acfg, replica_seed(args.seed, rank))
+    x1, x2, d1, d2 = (torch.from_numpy(s_host[n]).cuda() for n in ("x1", "x2", "dy1", "dx2"))
+    # one fp32 gradient buffer per tensor, reused by every layer; the router stays frozen (Sec. 3.3)
+    gm_buf = {n: torch.empty(shp, dtype=torch.float32, device="cuda") for n, shp in weight_shapes(mcfg).items()
+              if n not in ("w_router", "b_router")}
+    ga_buf = {n: torch.empty(shp, dtype=torch.float32, device="cuda") for n, shp in attn_weight_shapes(acfg).items()}
+    torch.cuda.synchronize()
+    base_alloc = torch.cuda.memory_allocated()
+    torch.cuda.reset_peak_memory_stats()
+    stk = rv.RevStack(batch=acfg.batch, seq_len=acfg.seq_len, d_model=acfg.d_model, n_heads=acfg.n_heads,
+                      n_kv_heads=acfg.n_kv_heads, n_experts=mcfg.n_experts, top_k=mcfg.top_k, d_expert=mcfg.d_expert,
+                      d_shared=mcfg.d_shared, weight_dtype=rv.BF16, attn_weights=wa, moe_weights=wm, inverse_iters=1,
+                      norm_eps=mcfg.norm_eps, rope_theta=acfg.rope_theta)
+    ga, gm = stk.grads_arrays([ga_buf] * L, [gm_buf] * L)
+    a, b, g1, g2 = (torch.empty_like(x1) for _ in range(4))
+    idx = torch.empty(L, acfg.tokens, mcfg.top_k, dtype=torch.int32, device="cuda")
+
+    def step(iters=None, remember=False):
+        a.copy_(x1); b.copy_(x2); g1.copy_(d1); g2.copy_(d2)
+        stk.forward(a, b, idx if remember else None)
+        stk.backward(a, b, g1, g2, ga, gm, topk_idx=idx if remember else None, inverse_iters=iters)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    assert stk.status() == 0
+    l0 = rv.revffn_prof_launches()
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    if sampler:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms = max_over_ranks([e0.elapsed_time(e1)], world)[0] / args.steps
+    launches = rv.revffn_prof_launches() - l0
+    assert stk.status() == 0
+    act_bytes = int(torch.cuda.max_memory_allocated() - base_alloc)
+
+    # per-pass split (one step with an event pair around each sweep)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    a.copy_(x1); b.copy_(x2); g1.copy_(d1); g2.copy_(d2)
+    ev[0].record(); stk.forward(a, b, None); ev[1].record(); stk.backward(a, b, g1, g2, ga, gm); ev[2].record()
+    torch.cuda.synchronize()
+    split = {"forward_ms": ev[0].elapsed_time(ev[1]), "backward_ms": ev[1].elapsed_time(ev[2])}
+
+    # reconstruction error of the stack's inputs after the backward sweep, against the number of fixed-point
+    # iterations of the attention inverse (Sec. 3.1 uses one), with recomputed and with remembered expert sets
+    rel = lambda u, v: float(((u - v).double().norm() / v.double().norm()).item())
+    recon = {}
+    for remember in (False, True):
+        for n in (1, 2, 3):
+            step(iters=n, remember=remember)
+            recon[f"iters={n},{'remembered' if remember else 'recomputed'}_routing"] = [rel(a, x1), rel(b, x2)]
+    assert stk.status() == 0
+
+    # end to end: streams and upstream gradients from pinned host memory, results back
+    pin = lambda t: t.cpu().pin_memory()
+    hx1, hx2, hd1, hd2 = pin(x1), pin(x2), pin(d1), pin(d2)
+    ho = [torch.empty_like(hx1).pin_memory() for _ in range(4)]
+
+    def host_step():
+        a.copy_(hx1, non_blocking=True); b.copy_(hx2, non_blocking=True)
+        g1.copy_(hd1, non_blocking=True); g2.copy_(hd2, non_blocking=True)
+        stk.forward(a, b, None)
+        stk.backward(a, b, g1, g2, ga, gm)
+        for h, t in zip(ho, (a, b, g1, g2)):
+            h.copy_(t, non_blocking=True)
+        torch.cuda.synchronize()
+    host_step()
+    barrier()
+    n_e2e = max(1, min(args.steps, 5))
+    t0 = time.perf_counter()
+    for _ in range(n_e2e):
+        host_step()
+    dt = max_over_ranks([time.perf_counter() - t0], world)[0] / n_e2e
+    if rank != 0:
+        return finish()
+
+    cpu_rec = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import revffn_block_oracle as orc
+        n_seq, S = 1, min(acfg.seq_len, 128)
+        cut = lambda t: t.cpu().numpy().reshape(acfg.batch, acfg.seq_len, -1)[:n_seq, :S].reshape(n_seq * S, -1)
+        pa = {n: t.float().cpu().numpy() for n, t in wa[0].items()}
+        pm = {n: t.float().cpu().numpy() for n, t in wm[0].items()}
+        cfg_o = dict(seq_len=S, n_heads=acfg.n_heads, n_kv_heads=acfg.n_kv_heads, top_k=mcfg.top_k, eps=mcfg.norm_eps,
+                     theta=acfg.rope_theta)
+        t0 = time.perf_counter()
+        Y1, Y2, _ = orc.forward(pa, pm, cut(x1), cut(x2), cfg_o)
+        orc.backward(pa, pm, Y1, Y2, cut(d1), cut(d2), cfg_o, n_iter=1)
+        cdt = time.perf_counter() - t0
+        cpu_rec = {"value": n_seq * S / cdt, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+                   "sample": f"one block (of {L}), forward + reversible backward over the first {S} positions of "
+                             f"{n_seq} sequence, full weights, fp64 numpy, {cdt:.1f} s"}
+    print(json.dumps({
+        "metric": "RevFFN block stack fwd+reversible bwd tokens/s", "value": world * acfg.tokens / (ms * 1e-3),
+        "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{L} whole RevFFN blocks (attention branch Eq. 1 + MoE branch Eq. 2) of the "
+                               f"Qwen1.5-MoE-A2.7B shape, {acfg.batch} x {acfg.seq_len} tokens per GPU; step = forward "
+                               f"through all layers + reversible back-propagation (inverse pass with one fixed-point "
+                               f"iteration, gradients at the rebuilt inputs, no cached activations); weights drawn "
+                               f"on the device", "l2": "per-layer working set exceeds the 126 MB L2", "blocks": L,
+                   "parallelism": "independent replicas" if world > 1 else "single GPU"},
+        "ms_per_block": ms / L, "passes_ms": split, "gpu_launches": int(launches), "clocks": clocks,
+        "memory": {"weights_bytes": w_bytes, "activation_bytes": act_bytes, "workspace_bytes": stk.bwd_bytes,
+                   "peak_device_bytes": int(torch.cuda.max_memory_allocated()),
+                   "note": "activation bytes = peak allocation above weights, input copies and the shared gradient "
+                           "buffers while the stack ran: one workspace, two streams, two stream gradients, whatever "
+                           "the number of layers"},
+        "reconstruction_rel_l2_[x1,x2]": recon, "cpu_baseline": cpu_rec,
+        "roofline": None,
+        "e2e": {"value": world * acfg.tokens / dt, "unit": "tokens/s", "h2d_bytes_per_step": 4 * hx1.numel() * 4,
+                "d2h_bytes_per_step": 4 * hx1.numel() * 4, "ms_per_step": dt * 1e3}}))
+    finish()
+
+
 def attn_flops(cfg):
     """Algorithmic flops per launch of the attention branch's matrix products, by profiler slot name.
     Causal attention needs half of the score and value products; the whole rectangle is counted
@@ -755,6 +891,8 @@ def main():
     args = ap.parse_args()
     from workloads import CONFIGS
     from workloads.generate import ATTN_CONFIGS
+    if args.config in ("B1", "B3") and args.impl == "ours":
+        return run_block_stack(args, ATTN_CONFIGS["A1"], CONFIGS["C1"], 24 if args.config == "B3" else 1)
     if args.config in ATTN_CONFIGS and args.impl == "ours":
         return run_attn(args, ATTN_CONFIGS[args.config])
     if args.config == "C4":

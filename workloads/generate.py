@@ -237,3 +237,18 @@ def make_attn_streams(cfg: AttnConfig, seed: int = 0) -> Dict[str, np.ndarray]:
     """Input streams X1, X2, the upstream gradient dY1 and a starting value for dX2, each [T, h] fp32 ~ N(0,1)."""
     return {name: _normal((cfg.tokens, cfg.h), 1.0, 0.0, seed, 0, "attn." + name, False)
             for name in ("x1", "x2", "dy1", "dx2")}
+
+
+def make_attn_weights_device(cfg: AttnConfig, seed: int = 0, block: int = 0, device: str = "cuda") -> Dict[str, torch.Tensor]:
+    """Attention-branch weights of one block drawn on `device` in their final dtypes: same shapes and
+    distributions as `make_attn_weights`, its own seeded streams (for stacks too large to draw on the host)."""
+    wdt = torch.bfloat16 if cfg.weight_dtype == "bf16" else torch.float32
+    out = {}
+    for name, shape in attn_weight_shapes(cfg).items():
+        g = torch.Generator(device=device)
+        g.manual_seed((int(seed) * 1_000_003 + int(block) * 7919) * 64 + _ATTN_IDS[name] + (1 << 41))
+        v = torch.randn(shape, generator=g, device=device, dtype=torch.float32) * 0.02
+        if name == "norm_gamma":
+            v = v + 1.0
+        out[name] = v.to(torch.float32 if name == "norm_gamma" or name.startswith("b_") else wdt).contiguous()
+    return out
