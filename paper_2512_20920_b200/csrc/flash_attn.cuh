@@ -83,6 +83,7 @@ struct FlashParams {
   int S, Sp, n_heads, rep;        // rep = query heads per key/value head
   bf16* o; int64_t ld_o;          // [T, ld_o]
   float* lse;                     // [B * n_heads * Sp] or NULL
+  float* o32;                     // [B * n_heads * Sp, 128] or NULL: the output before rounding, head-major
   float scale_log2e, scale;
   int* status;
 };
@@ -311,6 +312,13 @@ flash_fwd_kernel(const FlashParams P, const __grid_constant__ CUtensorMap map_q,
         *reinterpret_cast<uint4*>(dst + 8 * g) = pack8(f);
       }
       if (P.lse && half == 0) P.lse[(int64_t)bh * P.Sp + s_pos] = m * P.scale + logf(l);
+      if (P.o32) {
+        float* d32 = P.o32 + ((int64_t)bh * P.Sp + s_pos) * FA_HD + 64 * half;
+#pragma unroll
+        for (int g = 0; g < 16; ++g)
+          *reinterpret_cast<float4*>(d32 + 4 * g) =
+              make_float4(acc[4 * g] * inv, acc[4 * g + 1] * inv, acc[4 * g + 2] * inv, acc[4 * g + 3] * inv);
+      }
     }
   }
 
@@ -335,7 +343,7 @@ flash_fwd_kernel(const FlashParams P, const __grid_constant__ CUtensorMap map_q,
 
 // q: [B * n_heads * Sp, 128], k, v: [B * n_kv_heads * Sp, 128] bf16 head-major; o: [B * S, ld_o] bf16.
 inline int launch_flash_fwd(const bf16* q, const bf16* k, const bf16* v, int batch, int n_heads, int n_kv_heads, int S, int Sp,
-                            bf16* o, int64_t ld_o, float* lse, int* status, cudaStream_t st) {
+                            bf16* o, int64_t ld_o, float* lse, float* o32, int* status, cudaStream_t st) {
   TcState& s = tc_state();
   if (!s.ready) return REVFFN_ERR_CUDA;
   if (batch <= 0) return REVFFN_OK;
@@ -356,12 +364,356 @@ inline int launch_flash_fwd(const bf16* q, const bf16* k, const bf16* v, int bat
   if (r) return r;
   FlashParams P;
   P.S = S; P.Sp = Sp; P.n_heads = n_heads; P.rep = n_heads / n_kv_heads;
-  P.o = o; P.ld_o = ld_o; P.lse = lse;
+  P.o = o; P.ld_o = ld_o; P.lse = lse; P.o32 = o32;
   P.scale = 1.f / sqrtf((float)FA_HD);
   P.scale_log2e = P.scale * 1.4426950408889634f;
   P.status = status;
   const int grid = batch * n_heads * (Sp / FA_BLK);
   flash_fwd_kernel<<<grid, FA_THREADS, FA_SMEM_BYTES, st>>>(P, mq, mk, mv);
+  return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------
+// Backward of the attention core, also without a score matrix in HBM.  P is rebuilt from the row
+// log-sum-exp the forward kernel stored:  P = exp(scale * S - lse),  dS = scale * P * (dP - D) with
+// D = <dO_row, O_row>.  Two launches of one kernel template, neither uses atomics:
+//   DKV = true   a CTA owns 128 keys of one key/value head and walks the 64-row query tiles at or
+//                below them (of every query head of the group):  dV += P^T dO,  dK += dS^T Q
+//   DKV = false  a CTA owns 128 query rows of one head and walks the 64-key tiles up to its diagonal:
+//                dQ += dS K
+// Per step the "own" side is the MMA M side and the walked tile the N side, so both cases compute
+//   S' = X0 Y0^T,  dP' = X1 Y1^T   (128 x 64, K = hd; X = own operands, Y = the walked tiles)
+// into TMEM (double-buffered), eight warps (two threads per own row, 32 columns each) turn them into P' and
+// dS' as bf16 K-major operand tiles in shared memory, and the accumulators (fresh TMEM columns, summed over
+// all steps by the tensor core itself) take  acc0 += P' Y1  (DKV only)  and  acc1 += dS' Y0,  where the same
+// shared-memory bytes of a Y tile that served as a K-major operand are read again as an MN-major one.
+// No cross-thread reduction is needed: the row statistics come from memory.
+// ---------------------------------------------------------------------------
+constexpr int FB_X_OFF = 0;                        // X0, X1: 2 tiles of 16 KB each
+constexpr int FB_Y_OFF = 4 * FA_TILE;              // 2 stages x [Y0 2 x 8 KB | Y1 2 x 8 KB]
+constexpr int FB_P_OFF = FB_Y_OFF + 4 * FA_TILE;   // P' tile, 16 KB
+constexpr int FB_DS_OFF = FB_P_OFF + FA_TILE;      // dS' tile, 16 KB
+constexpr int FB_BAR_OFF = FB_DS_OFF + FA_TILE;
+constexpr int FB_SMEM_BYTES = FB_BAR_OFF + 256 + 1024;
+
+struct FlashBwdParams {
+  int S, Sp, n_heads, rep;
+  const float2* lse_d;            // per query row (head-major index): (lse * log2 e, D)
+  float* out0;                    // DKV: dV [kv rows, 128] fp32
+  float* out1;                    // DKV: dK [kv rows, 128];  else dQ [q rows, 128]
+  float scale_log2e, scale;
+  int* status;
+};
+
+// One element: P' and dS' from a score and a dP value.  MASK: this step's tile touches the causal diagonal or the
+// end of the sequence, `valid` decides; otherwise every element takes part.
+template <bool MASK>
+__device__ __forceinline__ void fb_elem(float s, float dp, float l2, float dv, float cl, float scale, bool valid, float& p,
+                                        float& ds) {
+  p = fa_exp2(s * cl - l2);
+  ds = p * (dp - dv) * scale;
+  if (MASK && !valid) { p = 0.f; ds = 0.f; }
+}
+
+template <bool DKV>
+__global__ void __launch_bounds__(FA_THREADS, 1)
+flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map_x0, const __grid_constant__ CUtensorMap map_x1,
+                 const __grid_constant__ CUtensorMap map_y0, const __grid_constant__ CUtensorMap map_y1) {
+  extern __shared__ uint8_t fa_smem_raw[];
+  const uint32_t raw = smem_u32(fa_smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen_base = fa_smem_raw + (base - raw);
+  const uint32_t bars = base + FB_BAR_OFF;
+  auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
+  enum { B_XFULL = 0, B_YFULL = 1, B_YEMPTY = 3, B_SDFULL = 5, B_SDEMPTY = 7, B_PDFULL = 9, B_PDEMPTY = 10, B_ACCFULL = 11,
+         B_COUNT = 12 };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + FB_BAR_OFF + 8 * B_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + FB_BAR_OFF + 8 * B_COUNT + 8);
+  int* issued = reinterpret_cast<int*>(gen_base + FB_BAR_OFF + 8 * B_COUNT + 16);   // [3]: x, y0, y1 -> phase + 1
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_blk = P.Sp / FA_BLK;                  // 128-row blocks per head
+  const int n_t64 = P.Sp / 64;                      // 64-row tiles per head
+  // heavy work first: DKV: low key blocks see the most query tiles; else: high query blocks see the most key tiles
+  const int per = (int)gridDim.x / n_blk;
+  const int ord = (int)blockIdx.x / per;
+  const int blk = DKV ? ord : n_blk - 1 - ord;      // own 128-row block within the head
+  const int grp = (int)blockIdx.x % per;            // DKV: sequence * n_kv_heads + kv head; else sequence * n_heads + head
+  const int own_row0 = grp * P.Sp + blk * FA_BLK;
+  const int t_begin = DKV ? 2 * blk : 0;
+  const int n_inner = DKV ? n_t64 - 2 * blk : 2 * blk + 2;
+  const int n_steps = (DKV ? P.rep : 1) * n_inner;
+  // first row of the walked operands: DKV: query head grp * rep (+ ho); else: the key/value head of this query head
+  const int y_base = DKV ? grp * P.rep * P.Sp : (grp / P.rep) * P.Sp;
+  auto y_row_of = [&](int s) -> int { return y_base + (s / n_inner) * P.Sp + 64 * (t_begin + s % n_inner); };
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(B_XFULL), 1);
+    mbar_init(bar(B_PDFULL), 8);
+    mbar_init(bar(B_PDEMPTY), 1);
+    mbar_init(bar(B_ACCFULL), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(B_YFULL + s), 1); mbar_init(bar(B_YEMPTY + s), 1);
+      mbar_init(bar(B_SDFULL + s), 1); mbar_init(bar(B_SDEMPTY + s), 8);
+    }
+    for (int i = 0; i < 3; ++i) issued[i] = 0;
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // TMEM columns: step buffer b: S' at 128 b, dP' at 128 b + 64; acc0 at 256, acc1 at 384
+  const uint32_t idesc_sd = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(FA_BLK >> 4) << 24);
+  const uint32_t idesc_acc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(FA_HD >> 3) << 17) |
+                             ((uint32_t)(FA_BLK >> 4) << 24);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      mbar_expect_tx(bar(B_XFULL), 4 * FA_TILE);
+      issued[0] = 1;
+      for (int kb = 0; kb < 2; ++kb) {
+        tma_load_2d(base + FB_X_OFF + kb * FA_TILE, &map_x0, 64 * kb, own_row0, bar(B_XFULL));
+        tma_load_2d(base + FB_X_OFF + (2 + kb) * FA_TILE, &map_x1, 64 * kb, own_row0, bar(B_XFULL));
+      }
+      for (int s = 0; s < n_steps; ++s) {
+        const int b = s & 1;
+        const uint32_t ph = (uint32_t)(s >> 1) & 1u;
+        if (!mbar_wait(bar(B_YEMPTY + b), ph ^ 1u, abort_flag, P.status)) break;
+        mbar_expect_tx(bar(B_YFULL + b), 2 * FA_TILE);
+        issued[1 + b] = (int)ph + 1;
+        const int yr = y_row_of(s);
+        const uint32_t ys = base + FB_Y_OFF + b * 2 * FA_TILE;
+        for (int kb = 0; kb < 2; ++kb) {
+          tma_load_2d(ys + kb * 8192, &map_y0, 64 * kb, yr, bar(B_YFULL + b));
+          tma_load_2d(ys + FA_TILE + kb * 8192, &map_y1, 64 * kb, yr, bar(B_YFULL + b));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = mbar_wait(bar(B_XFULL), 0u, abort_flag, P.status);
+      tc_fence_after();
+      auto issue_sd = [&](int s) -> bool {
+        const int b = s & 1;
+        const uint32_t ph = (uint32_t)(s >> 1) & 1u;
+        if (!mbar_wait(bar(B_YFULL + b), ph, abort_flag, P.status)) return false;
+        if (!mbar_wait(bar(B_SDEMPTY + b), ph ^ 1u, abort_flag, P.status)) return false;
+        tc_fence_after();
+        const uint32_t ys = base + FB_Y_OFF + b * 2 * FA_TILE;
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {            // w = 0: S' = X0 Y0^T, w = 1: dP' = X1 Y1^T
+          const uint32_t d = tmem_base + (uint32_t)(b * 128 + w * 64);
+#pragma unroll
+          for (int kb = 0; kb < 2; ++kb) {
+            const uint64_t a_desc = make_smem_desc(base + FB_X_OFF + (2 * w + kb) * FA_TILE, 16, 1024);
+            const uint64_t b_desc = make_smem_desc(ys + w * FA_TILE + kb * 8192, 16, 1024);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              tc_mma(d, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(2 * ks), idesc_sd, (kb | ks) != 0 ? 1u : 0u);
+          }
+        }
+        tc_commit(bar(B_SDFULL + b));
+        return true;
+      };
+      if (ok) ok = issue_sd(0);
+      for (int s = 0; ok && s < n_steps; ++s) {
+        if (s + 1 < n_steps && !issue_sd(s + 1)) { ok = false; break; }
+        const int b = s & 1;
+        if (!mbar_wait(bar(B_PDFULL), (uint32_t)s & 1u, abort_flag, P.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t ys = base + FB_Y_OFF + b * 2 * FA_TILE;
+        // the walked tiles again, now as [64 rows (K), 128 columns (N)] operands: the two 64-column halves are 8 KB apart
+        if (DKV) {
+          const uint64_t a_desc = make_smem_desc(base + FB_P_OFF, 16, 1024);
+          const uint64_t b_desc = make_smem_desc(ys + FA_TILE, 8192, 1024);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            tc_mma(tmem_base + 256u, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(128 * ks), idesc_acc, (s | ks) != 0 ? 1u : 0u);
+        }
+        {
+          const uint64_t a_desc = make_smem_desc(base + FB_DS_OFF, 16, 1024);
+          const uint64_t b_desc = make_smem_desc(ys, 8192, 1024);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            tc_mma(tmem_base + 384u, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(128 * ks), idesc_acc, (s | ks) != 0 ? 1u : 0u);
+        }
+        tc_commit(bar(B_YEMPTY + b));
+        tc_commit(bar(B_PDEMPTY));
+      }
+      if (ok) tc_commit(bar(B_ACCFULL));
+    }
+  } else {
+    // ------------------------------------------------------------------ P' / dS' (warps 2..9)
+    const int q = warp & 3;                      // TMEM lane quadrant this warp may access
+    const int hh = (warp - 2) >> 2;              // which 32 of the step's 64 columns
+    const int row = q * 32 + lane;               // own row within the block
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+    const float cl = P.scale_log2e, scale = P.scale;
+    const int own_pos = blk * FA_BLK + row;      // position in the sequence of this thread's own row
+    float2 own_ld = make_float2(0.f, 0.f);
+    if (!DKV && own_pos < P.S) own_ld = P.lse_d[own_row0 + row];
+    bool ok = true;
+    for (int s = 0; s < n_steps; ++s) {
+      const int b = s & 1;
+      const uint32_t ph = (uint32_t)(s >> 1) & 1u;
+      if (!mbar_wait(bar(B_SDFULL + b), ph, abort_flag, P.status)) { ok = false; break; }
+      tc_fence_after();
+      uint32_t rs[32], rd[32];
+      tmem_ld32(lane_addr + (uint32_t)(b * 128 + 32 * hh), rs);
+      tmem_ld32(lane_addr + (uint32_t)(b * 128 + 64 + 32 * hh), rd);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_SDEMPTY + b));
+      const int t = t_begin + s % n_inner;
+      const int col0 = 64 * t + 32 * hh;         // position in the sequence of this thread's first column
+      const float2* ld_cols = P.lse_d + y_row_of(s) + 32 * hh;
+      // tiles that touch the diagonal or the end of the sequence need the element-wise test
+      const bool mask = DKV ? (t < 2 * blk + 2 || 64 * t + 63 >= P.S) : (t >= 2 * blk || blk * FA_BLK + FA_BLK - 1 >= P.S);
+      uint4 pp[4], pd[4];
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        float pv[8], dv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int c = 8 * g + i;
+          const float sv = __uint_as_float(rs[c]), dpv = __uint_as_float(rd[c]);
+          if (DKV) {
+            // own row = key, column = query: needs query >= key and query inside the sequence
+            const bool valid = !mask || (col0 + c >= own_pos && col0 + c < P.S);
+            float2 ld = make_float2(0.f, 0.f);
+            if (valid) ld = __ldg(ld_cols + c);
+            if (mask) fb_elem<true>(sv, dpv, ld.x, ld.y, cl, scale, valid, pv[i], dv[i]);
+            else fb_elem<false>(sv, dpv, ld.x, ld.y, cl, scale, true, pv[i], dv[i]);
+          } else {
+            // own row = query, column = key
+            const bool valid = !mask || (col0 + c <= own_pos && own_pos < P.S);
+            if (mask) fb_elem<true>(sv, dpv, own_ld.x, own_ld.y, cl, scale, valid, pv[i], dv[i]);
+            else fb_elem<false>(sv, dpv, own_ld.x, own_ld.y, cl, scale, true, pv[i], dv[i]);
+          }
+        }
+        pp[g] = pack8(pv);
+        pd[g] = pack8(dv);
+      }
+      // the operand tiles have one buffer: the previous step's accumulating products must have read them
+      if (!mbar_wait(bar(B_PDEMPTY), ((uint32_t)s & 1u) ^ 1u, abort_flag, P.status)) { ok = false; break; }
+      uint8_t* prow = gen_base + FB_P_OFF + row * 128;
+      uint8_t* drow = gen_base + FB_DS_OFF + row * 128;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const int piece = ((4 * hh + g) ^ (row & 7)) << 4;
+        if (DKV) *reinterpret_cast<uint4*>(prow + piece) = pp[g];
+        *reinterpret_cast<uint4*>(drow + piece) = pd[g];
+      }
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_PDFULL));
+    }
+    if (ok && !mbar_wait(bar(B_ACCFULL), 0u, abort_flag, P.status)) ok = false;
+    if (ok) {
+      tc_fence_after();
+#pragma unroll
+      for (int a = DKV ? 0 : 1; a < 2; ++a) {
+        float* dst = (a == 0 ? P.out0 : P.out1) + (int64_t)(own_row0 + row) * FA_HD + 64 * (warp >= 6 ? 1 : 0);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t r[32];
+          tmem_ld32(lane_addr + (uint32_t)(256 + 128 * a + 64 * (warp >= 6 ? 1 : 0) + 32 * c), r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<float4*>(dst + 32 * c + 4 * i) =
+                make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),
+                            __uint_as_float(r[4 * i + 3]));
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) {
+    const int bidx[3] = {B_XFULL, B_YFULL, B_YFULL + 1};
+    for (int i = 0; i < 3; ++i) {
+      if (issued[i] == 0) continue;
+      long long t0 = clock64();
+      while (!mbar_try_wait(bar(bidx[i]), (uint32_t)(issued[i] - 1)) && clock64() - t0 < TC_WAIT_CYCLES) {}
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// (lse * log2 e, <dO_row, O_row>) per query row; one warp per head-major row.  O is taken before its rounding to
+// bf16: D stands for sum_j P_j dP_j, and with a peaked row dP - D cancels, so an error in D would show in dS.
+__global__ void attn_rowdot_kernel(const float* __restrict__ o32, const bf16* __restrict__ d_o, const float* __restrict__ lse,
+                                   int S, int Sp, int64_t rows, float2* __restrict__ lse_d) {
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (row >= rows || (int)(row % Sp) >= S) return;
+  const float4 a = *reinterpret_cast<const float4*>(o32 + row * FA_HD + 4 * lane);
+  const uint2 b = *reinterpret_cast<const uint2*>(d_o + row * FA_HD + 4 * lane);
+  const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b);
+  const float2 y0 = __bfloat1622float2(bh[0]), y1 = __bfloat1622float2(bh[1]);
+  float dot = a.x * y0.x + a.y * y0.y + a.z * y1.x + a.w * y1.y;
+  dot = warp_sum(dot);
+  if (lane == 0) lse_d[row] = make_float2(lse[row] * 1.4426950408889634f, dot);
+}
+
+// q, d_o: [B * n_heads * Sp, 128]; k, v: [B * n_kv_heads * Sp, 128] bf16 head-major (rows past the sequence zero).
+// dq: [B * n_heads * Sp, 128], dk, dv: [B * n_kv_heads * Sp, 128] fp32, every row written.
+inline int launch_flash_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* d_o, const float2* lse_d, int batch,
+                            int n_heads, int n_kv_heads, int S, int Sp, float* dq, float* dk, float* dv, int* status,
+                            cudaStream_t st) {
+  TcState& s = tc_state();
+  if (!s.ready) return REVFFN_ERR_CUDA;
+  if (batch <= 0) return REVFFN_OK;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return REVFFN_ERR_CUDA;
+  if (!attr_set[dev]) {
+    if (cudaFuncSetAttribute(flash_bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FB_SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(flash_bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FB_SMEM_BYTES) != cudaSuccess)
+      return REVFFN_ERR_CUDA;
+    attr_set[dev] = true;
+  }
+  const uint64_t q_rows = (uint64_t)batch * n_heads * Sp, kv_rows = (uint64_t)batch * n_kv_heads * Sp;
+  CUtensorMap q128, do128, k128, v128, q64, do64, k64, v64;
+  int r = 0;
+  if (!r) r = tc_make_map(&q128, q, FA_HD, q_rows, FA_HD, 64, 128);
+  if (!r) r = tc_make_map(&do128, d_o, FA_HD, q_rows, FA_HD, 64, 128);
+  if (!r) r = tc_make_map(&k128, k, FA_HD, kv_rows, FA_HD, 64, 128);
+  if (!r) r = tc_make_map(&v128, v, FA_HD, kv_rows, FA_HD, 64, 128);
+  if (!r) r = tc_make_map(&q64, q, FA_HD, q_rows, FA_HD, 64, 64);
+  if (!r) r = tc_make_map(&do64, d_o, FA_HD, q_rows, FA_HD, 64, 64);
+  if (!r) r = tc_make_map(&k64, k, FA_HD, kv_rows, FA_HD, 64, 64);
+  if (!r) r = tc_make_map(&v64, v, FA_HD, kv_rows, FA_HD, 64, 64);
+  if (r) return r;
+  FlashBwdParams P;
+  P.S = S; P.Sp = Sp; P.n_heads = n_heads; P.rep = n_heads / n_kv_heads;
+  P.lse_d = lse_d;
+  P.scale = 1.f / sqrtf((float)FA_HD);
+  P.scale_log2e = P.scale * 1.4426950408889634f;
+  P.status = status;
+  P.out0 = dv; P.out1 = dk;
+  flash_bwd_kernel<true><<<batch * n_kv_heads * (Sp / FA_BLK), FA_THREADS, FB_SMEM_BYTES, st>>>(P, k128, v128, q64, do64);
+  if (cudaGetLastError() != cudaSuccess) return REVFFN_ERR_CUDA;
+  P.out0 = nullptr; P.out1 = dq;
+  flash_bwd_kernel<false><<<batch * n_heads * (Sp / FA_BLK), FA_THREADS, FB_SMEM_BYTES, st>>>(P, q128, do128, k64, v64);
   return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
 

@@ -18,7 +18,7 @@ namespace revffn {
 struct AttnLayout {
   Buf status, rows_total, tile_group, group_off, cs, n12, r12, u12, raw, qh, kh, vh, lse, sc, p, oh, o, a;
   size_t fwd_bytes = 0;
-  Buf dyb, da, dob, doh, ds, dqh, dkh, dvh, dq, dkv, du12, dn12, part;
+  Buf dyb, da, dob, doh, ds, dqh, dkh, dvh, dq, dkv, du12, dn12, part, lse_d;
   size_t bwd_bytes = 0;
   int T = 0, h = 0, hd = 0, d_kv = 0, Sp = 0, n_tiles = 0, groups = 0, strips = 0;
   int64_t rows = 0, kv_rows = 0;
@@ -71,6 +71,7 @@ static AttnLayout plan_attn(const revffn_attn_desc& D) {
   take(L.du12, (size_t)2 * T * d * ts);
   take(L.dn12, (size_t)2 * T * h * 4);
   take(L.part, (size_t)L.strips * d * 4);
+  take(L.lse_d, (size_t)L.rows * 8);
   L.bwd_bytes = off;
   return L;
 }
@@ -209,7 +210,7 @@ static GemmProblem a_grouped_rows(const ACtx<T>& c) {
 // O (token-major) from the head-major q, k, v.  need_p: the backward pass reads P afterwards, so the score
 // matrix is materialised; otherwise the tcgen05 back end runs the attention core as one kernel.
 template <typename T>
-static int a_core(const ACtx<T>& c, bool need_p) {
+static int a_core(const ACtx<T>& c, bool need_p, bool keep_o32 = false) {
   const revffn_attn_desc& D = c.D;
   const AttnLayout& L = c.L;
   if constexpr (std::is_same<T, bf16>::value) {
@@ -217,7 +218,8 @@ static int a_core(const ACtx<T>& c, bool need_p) {
       ProfScope ps(TG_A_FLASH, c.st);
       return launch_flash_fwd(c.template p<bf16>(L.qh), c.template p<bf16>(L.kh), c.template p<bf16>(L.vh), D.batch,
                               D.n_heads, D.n_kv_heads, D.seq_len, L.Sp, c.template p<bf16>(L.o), D.d_model,
-                              c.template p<float>(L.lse), c.template p<int>(L.status), c.st);
+                              c.template p<float>(L.lse), keep_o32 ? c.template p<float>(L.sc) : nullptr,
+                              c.template p<int>(L.status), c.st);
     }
   }
   {
@@ -282,10 +284,10 @@ static int a_kv_side(const ACtx<T>& c, const float* x2) {
 }
 
 template <typename T>
-static int a_query_side(const ACtx<T>& c, const float* x1, bool need_p) {
+static int a_query_side(const ACtx<T>& c, const float* x1, bool need_p, bool keep_o32 = false) {
   CKR(a_norm_up(c, x1, 0));
   CKR(a_project(c, 0, c.W.w_q, c.W.b_q, c.D.n_heads, true, c.template p<T>(c.L.qh)));
-  CKR(a_core(c, need_p));
+  CKR(a_core(c, need_p, keep_o32));
   return a_wo(c);
 }
 
@@ -331,8 +333,12 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
 
   // recompute the branch's intermediates (Sec. 3.1: nothing was cached)
   CKR(a_setup(c, true));
+  // tcgen05 back end: the attention core runs fused in both directions and P is never written;
+  // otherwise the score matrix is materialised and the gradient pass reads P from memory
+  bool fused = false;
+  if constexpr (std::is_same<T, bf16>::value) fused = c.tc && hd == FA_HD;
   CKR(a_kv_side(c, x2));
-  CKR(a_query_side(c, x1, true));
+  CKR(a_query_side(c, x1, !fused, fused));      // fused: the score buffer holds the unrounded output instead
 
   auto wgrad = [&](float* out, int M, int N, const void* A, int64_t lda, int a_col0, const void* B, int64_t ldb,
                    int K, int accumulate) -> int {
@@ -385,39 +391,57 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
   CK(cudaGetLastError());
 
   // attention core backward
-  {
-    GemmProblem p = a_grouped_rows(c);   // dP = dO V^T
-    p.N = Sp; p.K = hd;
-    p.A = c.template p<T>(L.doh); p.lda = hd;
-    p.B0 = c.template p<T>(L.vh); p.ldb = hd;
-    p.epilogue = EPI_STORE; p.out_f32 = 1; p.C = c.template p<float>(L.sc); p.ldc = Sp;
-    CKR(a_gemm(c, p, TG_A_DP));
-  }
-  { ProfScope ps(TG_A_SOFTMAX, st);
-  dsoftmax_causal_kernel<T><<<(unsigned)ceil_div(L.rows * 32, 256), 256, 0, st>>>(
-      c.template p<T>(L.p), c.template p<float>(L.sc), D.seq_len, Sp, 1.f / sqrtf((float)hd), L.rows, c.template p<T>(L.ds));
-  }
-  CK(cudaGetLastError());
-  auto kv_grad = [&](const T* A, const T* Bm, float* out) -> int {
-    GemmProblem p = blank_problem();   // out[g] = A_g^T B_g over the query rows of key/value group g
-    p.M = Sp; p.N = hd; p.K = (int)L.rows;
-    p.a_mn_major = 1; p.b_mn_major = 1;
-    p.A = A; p.lda = Sp;
-    p.B0 = Bm; p.ldb = hd;
-    p.epilogue = EPI_WGRAD; p.accumulate = 0;
-    p.C = out; p.ldc = hd; p.c_group_stride = (int64_t)Sp * hd;
-    p.group_mode = GROUP_K; p.n_groups = L.groups; p.group_off = c.template p<int32_t>(L.group_off);
-    return a_gemm(c, p, TG_A_DKV);
-  };
-  CKR(kv_grad(c.template p<T>(L.p), c.template p<T>(L.doh), c.template p<float>(L.dvh)));    // dV = P^T dO
-  CKR(kv_grad(c.template p<T>(L.ds), c.template p<T>(L.qh), c.template p<float>(L.dkh)));    // dK = dS^T Q
-  {
-    GemmProblem p = a_grouped_rows(c);   // dQ = dS K
-    p.N = hd; p.K = Sp;
-    p.A = c.template p<T>(L.ds); p.lda = Sp;
-    p.B0 = c.template p<T>(L.kh); p.ldb = hd; p.b_mn_major = 1;
-    p.epilogue = EPI_STORE; p.out_f32 = 1; p.C = c.template p<float>(L.dqh); p.ldc = hd;
-    CKR(a_gemm(c, p, TG_A_DQ));
+  if (fused) {
+    if constexpr (std::is_same<T, bf16>::value) {
+      { ProfScope ps(TG_A_SOFTMAX, st);
+      attn_rowdot_kernel<<<(unsigned)ceil_div(L.rows * 32, 256), 256, 0, st>>>(
+          c.template p<float>(L.sc), c.template p<bf16>(L.doh), c.template p<float>(L.lse), D.seq_len, Sp, L.rows,
+          c.template p<float2>(L.lse_d));
+      }
+      CK(cudaGetLastError());
+      { ProfScope ps(TG_A_FLASH, st);
+      CKR(launch_flash_bwd(c.template p<bf16>(L.qh), c.template p<bf16>(L.kh), c.template p<bf16>(L.vh),
+                           c.template p<bf16>(L.doh), c.template p<float2>(L.lse_d), D.batch, D.n_heads, D.n_kv_heads,
+                           D.seq_len, Sp, c.template p<float>(L.dqh), c.template p<float>(L.dkh), c.template p<float>(L.dvh),
+                           c.template p<int>(L.status), st));
+      ++g_prof.launches;
+      }
+    }
+  } else {
+    {
+      GemmProblem p = a_grouped_rows(c);   // dP = dO V^T
+      p.N = Sp; p.K = hd;
+      p.A = c.template p<T>(L.doh); p.lda = hd;
+      p.B0 = c.template p<T>(L.vh); p.ldb = hd;
+      p.epilogue = EPI_STORE; p.out_f32 = 1; p.C = c.template p<float>(L.sc); p.ldc = Sp;
+      CKR(a_gemm(c, p, TG_A_DP));
+    }
+    { ProfScope ps(TG_A_SOFTMAX, st);
+    dsoftmax_causal_kernel<T><<<(unsigned)ceil_div(L.rows * 32, 256), 256, 0, st>>>(
+        c.template p<T>(L.p), c.template p<float>(L.sc), D.seq_len, Sp, 1.f / sqrtf((float)hd), L.rows, c.template p<T>(L.ds));
+    }
+    CK(cudaGetLastError());
+    auto kv_grad = [&](const T* A, const T* Bm, float* out) -> int {
+      GemmProblem p = blank_problem();   // out[g] = A_g^T B_g over the query rows of key/value group g
+      p.M = Sp; p.N = hd; p.K = (int)L.rows;
+      p.a_mn_major = 1; p.b_mn_major = 1;
+      p.A = A; p.lda = Sp;
+      p.B0 = Bm; p.ldb = hd;
+      p.epilogue = EPI_WGRAD; p.accumulate = 0;
+      p.C = out; p.ldc = hd; p.c_group_stride = (int64_t)Sp * hd;
+      p.group_mode = GROUP_K; p.n_groups = L.groups; p.group_off = c.template p<int32_t>(L.group_off);
+      return a_gemm(c, p, TG_A_DKV);
+    };
+    CKR(kv_grad(c.template p<T>(L.p), c.template p<T>(L.doh), c.template p<float>(L.dvh)));    // dV = P^T dO
+    CKR(kv_grad(c.template p<T>(L.ds), c.template p<T>(L.qh), c.template p<float>(L.dkh)));    // dK = dS^T Q
+    {
+      GemmProblem p = a_grouped_rows(c);   // dQ = dS K
+      p.N = hd; p.K = Sp;
+      p.A = c.template p<T>(L.ds); p.lda = Sp;
+      p.B0 = c.template p<T>(L.kh); p.ldb = hd; p.b_mn_major = 1;
+      p.epilogue = EPI_STORE; p.out_f32 = 1; p.C = c.template p<float>(L.dqh); p.ldc = hd;
+      CKR(a_gemm(c, p, TG_A_DQ));
+    }
   }
   // back to token-major; the rotation is undone by its transpose
   { ProfScope ps(TG_A_HEADS, st);
