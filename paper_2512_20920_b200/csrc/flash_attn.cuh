@@ -394,25 +394,56 @@ constexpr int FB_Y_OFF = 4 * FA_TILE;              // 2 stages x [Y0 2 x 8 KB | 
 constexpr int FB_P_OFF = FB_Y_OFF + 4 * FA_TILE;   // P' tile, 16 KB
 constexpr int FB_DS_OFF = FB_P_OFF + FA_TILE;      // dS' tile, 16 KB
 constexpr int FB_BAR_OFF = FB_DS_OFF + FA_TILE;
-constexpr int FB_SMEM_BYTES = FB_BAR_OFF + 256 + 1024;
+constexpr int FB_LD_OFF = FB_BAR_OFF + 256;        // DKV: (lse * log2 e, D * scale) of the step's 64 query rows, 2 stages x 512 B
+constexpr int FB_SMEM_BYTES = FB_LD_OFF + 1024 + 1024;
 
 struct FlashBwdParams {
   int S, Sp, n_heads, rep;
-  const float2* lse_d;            // per query row (head-major index): (lse * log2 e, D)
+  const float2* lse_d;            // per query row (head-major index): (lse * log2 e, D * scale)
   float* out0;                    // DKV: dV [kv rows, 128] fp32
   float* out1;                    // DKV: dK [kv rows, 128];  else dQ [q rows, 128]
   float scale_log2e, scale;
   int* status;
 };
 
-// One element: P' and dS' from a score and a dP value.  MASK: this step's tile touches the causal diagonal or the
-// end of the sequence, `valid` decides; otherwise every element takes part.
-template <bool MASK>
-__device__ __forceinline__ void fb_elem(float s, float dp, float l2, float dv, float cl, float scale, bool valid, float& p,
-                                        float& ds) {
-  p = fa_exp2(s * cl - l2);
-  ds = p * (dp - dv) * scale;
-  if (MASK && !valid) { p = 0.f; ds = 0.f; }
+// Untiled bulk copy global -> shared (both addresses 16-byte aligned, size a multiple of 16), completing on an mbarrier.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+}
+
+// This thread's 32 elements of a step: P' = exp2(s * cl - lse2), dS' = P' * (dP * scale - D * scale), packed to bf16.
+// The row statistics belong to the query: the column's (DKV, read from shared memory) or this thread's own row's.
+// MASK: the tile touches the causal diagonal or the end of the sequence and every element is tested.
+template <bool DKV, bool MASK>
+__device__ __forceinline__ void fb_tile(const uint32_t (&rs)[32], const uint32_t (&rd)[32], const float4* __restrict__ ld_cols,
+                                        float2 own_ld, float cl, float scale, int col0, int own_pos, int S, uint4 (&pp)[4],
+                                        uint4 (&pd)[4]) {
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    float pv[8], dv[8];
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+      float4 ld = make_float4(own_ld.x, own_ld.y, own_ld.x, own_ld.y);
+      if (DKV) ld = ld_cols[(8 * g + i) >> 1];          // two columns' (lse2, D * scale)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int c = 8 * g + i + e;
+        const float l2 = e ? ld.z : ld.x, dsc = e ? ld.w : ld.y;
+        float p = fa_exp2(__uint_as_float(rs[c]) * cl - l2);
+        float ds = p * fmaf(__uint_as_float(rd[c]), scale, -dsc);
+        if (MASK) {
+          // DKV: own row = key, column = query (needs query >= key, query inside the sequence); else the roles swap
+          const bool valid = DKV ? (col0 + c >= own_pos && col0 + c < S) : (col0 + c <= own_pos && own_pos < S);
+          if (!valid) { p = 0.f; ds = 0.f; }
+        }
+        pv[i + e] = p;
+        dv[i + e] = ds;
+      }
+    }
+    if (DKV) pp[g] = pack8(pv);
+    pd[g] = pack8(dv);
+  }
 }
 
 template <bool DKV>
@@ -488,9 +519,10 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
         const int b = s & 1;
         const uint32_t ph = (uint32_t)(s >> 1) & 1u;
         if (!mbar_wait(bar(B_YEMPTY + b), ph ^ 1u, abort_flag, P.status)) break;
-        mbar_expect_tx(bar(B_YFULL + b), 2 * FA_TILE);
+        mbar_expect_tx(bar(B_YFULL + b), 2 * FA_TILE + (DKV ? 512 : 0));
         issued[1 + b] = (int)ph + 1;
         const int yr = y_row_of(s);
+        if (DKV) bulk_load_1d(base + FB_LD_OFF + b * 512, P.lse_d + yr, 512, bar(B_YFULL + b));
         const uint32_t ys = base + FB_Y_OFF + b * 2 * FA_TILE;
         for (int kb = 0; kb < 2; ++kb) {
           tma_load_2d(ys + kb * 8192, &map_y0, 64 * kb, yr, bar(B_YFULL + b));
@@ -567,6 +599,8 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       const int b = s & 1;
       const uint32_t ph = (uint32_t)(s >> 1) & 1u;
       if (!mbar_wait(bar(B_SDFULL + b), ph, abort_flag, P.status)) { ok = false; break; }
+      // DKV: this thread reads the stage's row statistics itself, so it observes the stage's barrier itself
+      if (DKV && !mbar_wait(bar(B_YFULL + b), ph, abort_flag, P.status)) { ok = false; break; }
       tc_fence_after();
       uint32_t rs[32], rd[32];
       tmem_ld32(lane_addr + (uint32_t)(b * 128 + 32 * hh), rs);
@@ -577,34 +611,13 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       if (lane == 0) mbar_arrive(bar(B_SDEMPTY + b));
       const int t = t_begin + s % n_inner;
       const int col0 = 64 * t + 32 * hh;         // position in the sequence of this thread's first column
-      const float2* ld_cols = P.lse_d + y_row_of(s) + 32 * hh;
       // tiles that touch the diagonal or the end of the sequence need the element-wise test
       const bool mask = DKV ? (t < 2 * blk + 2 || 64 * t + 63 >= P.S) : (t >= 2 * blk || blk * FA_BLK + FA_BLK - 1 >= P.S);
+      // DKV: the step's row statistics came with the walked tiles (S' complete implies that stage has landed)
+      const float4* ld_cols = reinterpret_cast<const float4*>(gen_base + FB_LD_OFF + b * 512) + 16 * hh;
       uint4 pp[4], pd[4];
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        float pv[8], dv[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int c = 8 * g + i;
-          const float sv = __uint_as_float(rs[c]), dpv = __uint_as_float(rd[c]);
-          if (DKV) {
-            // own row = key, column = query: needs query >= key and query inside the sequence
-            const bool valid = !mask || (col0 + c >= own_pos && col0 + c < P.S);
-            float2 ld = make_float2(0.f, 0.f);
-            if (valid) ld = __ldg(ld_cols + c);
-            if (mask) fb_elem<true>(sv, dpv, ld.x, ld.y, cl, scale, valid, pv[i], dv[i]);
-            else fb_elem<false>(sv, dpv, ld.x, ld.y, cl, scale, true, pv[i], dv[i]);
-          } else {
-            // own row = query, column = key
-            const bool valid = !mask || (col0 + c <= own_pos && own_pos < P.S);
-            if (mask) fb_elem<true>(sv, dpv, own_ld.x, own_ld.y, cl, scale, valid, pv[i], dv[i]);
-            else fb_elem<false>(sv, dpv, own_ld.x, own_ld.y, cl, scale, true, pv[i], dv[i]);
-          }
-        }
-        pp[g] = pack8(pv);
-        pd[g] = pack8(dv);
-      }
+      if (mask) fb_tile<DKV, true>(rs, rd, ld_cols, own_ld, cl, scale, col0, own_pos, P.S, pp, pd);
+      else fb_tile<DKV, false>(rs, rd, ld_cols, own_ld, cl, scale, col0, own_pos, P.S, pp, pd);
       // the operand tiles have one buffer: the previous step's accumulating products must have read them
       if (!mbar_wait(bar(B_PDEMPTY), ((uint32_t)s & 1u) ^ 1u, abort_flag, P.status)) { ok = false; break; }
       uint8_t* prow = gen_base + FB_P_OFF + row * 128;
@@ -658,10 +671,10 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   }
 }
 
-// (lse * log2 e, <dO_row, O_row>) per query row; one warp per head-major row.  O is taken before its rounding to
+// (lse * log2 e, scale * <dO_row, O_row>) per query row; one warp per head-major row.  O is taken before its rounding to
 // bf16: D stands for sum_j P_j dP_j, and with a peaked row dP - D cancels, so an error in D would show in dS.
 __global__ void attn_rowdot_kernel(const float* __restrict__ o32, const bf16* __restrict__ d_o, const float* __restrict__ lse,
-                                   int S, int Sp, int64_t rows, float2* __restrict__ lse_d) {
+                                   int S, int Sp, int64_t rows, float scale, float2* __restrict__ lse_d) {
   const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (row >= rows || (int)(row % Sp) >= S) return;
@@ -671,7 +684,7 @@ __global__ void attn_rowdot_kernel(const float* __restrict__ o32, const bf16* __
   const float2 y0 = __bfloat1622float2(bh[0]), y1 = __bfloat1622float2(bh[1]);
   float dot = a.x * y0.x + a.y * y0.y + a.z * y1.x + a.w * y1.y;
   dot = warp_sum(dot);
-  if (lane == 0) lse_d[row] = make_float2(lse[row] * 1.4426950408889634f, dot);
+  if (lane == 0) lse_d[row] = make_float2(lse[row] * 1.4426950408889634f, dot * scale);
 }
 
 // q, d_o: [B * n_heads * Sp, 128]; k, v: [B * n_kv_heads * Sp, 128] bf16 head-major (rows past the sequence zero).

@@ -396,7 +396,7 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
       { ProfScope ps(TG_A_SOFTMAX, st);
       attn_rowdot_kernel<<<(unsigned)ceil_div(L.rows * 32, 256), 256, 0, st>>>(
           c.template p<float>(L.sc), c.template p<bf16>(L.doh), c.template p<float>(L.lse), D.seq_len, Sp, L.rows,
-          c.template p<float2>(L.lse_d));
+          1.f / sqrtf((float)hd), c.template p<float2>(L.lse_d));
       }
       CK(cudaGetLastError());
       { ProfScope ps(TG_A_FLASH, st);
