@@ -384,16 +384,17 @@ inline int launch_flash_fwd(const bf16* q, const bf16* k, const bf16* v, int bat
 // Per step the "own" side is the MMA M side and the walked tile the N side, so both cases compute
 //   S' = X0 Y0^T,  dP' = X1 Y1^T   (128 x 64, K = hd; X = own operands, Y = the walked tiles)
 // into TMEM (double-buffered), eight warps (two threads per own row, 32 columns each) turn them into P' and
-// dS' as bf16 K-major operand tiles in shared memory, and the accumulators (fresh TMEM columns, summed over
+// dS' as bf16 K-major operand tiles in shared memory (double-buffered too, so that neither side waits for the other's
+// current step), and the accumulators (fresh TMEM columns, summed over
 // all steps by the tensor core itself) take  acc0 += P' Y1  (DKV only)  and  acc1 += dS' Y0,  where the same
 // shared-memory bytes of a Y tile that served as a K-major operand are read again as an MN-major one.
 // No cross-thread reduction is needed: the row statistics come from memory.
 // ---------------------------------------------------------------------------
 constexpr int FB_X_OFF = 0;                        // X0, X1: 2 tiles of 16 KB each
 constexpr int FB_Y_OFF = 4 * FA_TILE;              // 2 stages x [Y0 2 x 8 KB | Y1 2 x 8 KB]
-constexpr int FB_P_OFF = FB_Y_OFF + 4 * FA_TILE;   // P' tile, 16 KB
-constexpr int FB_DS_OFF = FB_P_OFF + FA_TILE;      // dS' tile, 16 KB
-constexpr int FB_BAR_OFF = FB_DS_OFF + FA_TILE;
+constexpr int FB_P_OFF = FB_Y_OFF + 4 * FA_TILE;   // P' tiles, 2 x 16 KB
+constexpr int FB_DS_OFF = FB_P_OFF + 2 * FA_TILE;  // dS' tiles, 2 x 16 KB
+constexpr int FB_BAR_OFF = FB_DS_OFF + 2 * FA_TILE;
 constexpr int FB_LD_OFF = FB_BAR_OFF + 256;        // DKV: (lse * log2 e, D * scale) of the step's 64 query rows, 2 stages x 512 B
 constexpr int FB_SMEM_BYTES = FB_LD_OFF + 1024 + 1024;
 
@@ -456,8 +457,8 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   uint8_t* gen_base = fa_smem_raw + (base - raw);
   const uint32_t bars = base + FB_BAR_OFF;
   auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
-  enum { B_XFULL = 0, B_YFULL = 1, B_YEMPTY = 3, B_SDFULL = 5, B_SDEMPTY = 7, B_PDFULL = 9, B_PDEMPTY = 10, B_ACCFULL = 11,
-         B_COUNT = 12 };
+  enum { B_XFULL = 0, B_YFULL = 1, B_YEMPTY = 3, B_SDFULL = 5, B_SDEMPTY = 7, B_PDFULL = 9, B_PDEMPTY = 11, B_ACCFULL = 13,
+         B_COUNT = 14 };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + FB_BAR_OFF + 8 * B_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + FB_BAR_OFF + 8 * B_COUNT + 8);
   int* issued = reinterpret_cast<int*>(gen_base + FB_BAR_OFF + 8 * B_COUNT + 16);   // [3]: x, y0, y1 -> phase + 1
@@ -480,12 +481,11 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
 
   if (threadIdx.x == 0) {
     mbar_init(bar(B_XFULL), 1);
-    mbar_init(bar(B_PDFULL), 8);
-    mbar_init(bar(B_PDEMPTY), 1);
     mbar_init(bar(B_ACCFULL), 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(B_YFULL + s), 1); mbar_init(bar(B_YEMPTY + s), 1);
       mbar_init(bar(B_SDFULL + s), 1); mbar_init(bar(B_SDEMPTY + s), 8);
+      mbar_init(bar(B_PDFULL + s), 8); mbar_init(bar(B_PDEMPTY + s), 1);
     }
     for (int i = 0; i < 3; ++i) issued[i] = 0;
     *abort_flag = 0;
@@ -561,26 +561,26 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       for (int s = 0; ok && s < n_steps; ++s) {
         if (s + 1 < n_steps && !issue_sd(s + 1)) { ok = false; break; }
         const int b = s & 1;
-        if (!mbar_wait(bar(B_PDFULL), (uint32_t)s & 1u, abort_flag, P.status)) { ok = false; break; }
+        if (!mbar_wait(bar(B_PDFULL + b), (uint32_t)(s >> 1) & 1u, abort_flag, P.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t ys = base + FB_Y_OFF + b * 2 * FA_TILE;
         // the walked tiles again, now as [64 rows (K), 128 columns (N)] operands: the two 64-column halves are 8 KB apart
         if (DKV) {
-          const uint64_t a_desc = make_smem_desc(base + FB_P_OFF, 16, 1024);
+          const uint64_t a_desc = make_smem_desc(base + FB_P_OFF + b * FA_TILE, 16, 1024);
           const uint64_t b_desc = make_smem_desc(ys + FA_TILE, 8192, 1024);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
             tc_mma(tmem_base + 256u, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(128 * ks), idesc_acc, (s | ks) != 0 ? 1u : 0u);
         }
         {
-          const uint64_t a_desc = make_smem_desc(base + FB_DS_OFF, 16, 1024);
+          const uint64_t a_desc = make_smem_desc(base + FB_DS_OFF + b * FA_TILE, 16, 1024);
           const uint64_t b_desc = make_smem_desc(ys, 8192, 1024);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
             tc_mma(tmem_base + 384u, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(128 * ks), idesc_acc, (s | ks) != 0 ? 1u : 0u);
         }
         tc_commit(bar(B_YEMPTY + b));
-        tc_commit(bar(B_PDEMPTY));
+        tc_commit(bar(B_PDEMPTY + b));
       }
       if (ok) tc_commit(bar(B_ACCFULL));
     }
@@ -618,10 +618,10 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       uint4 pp[4], pd[4];
       if (mask) fb_tile<DKV, true>(rs, rd, ld_cols, own_ld, cl, scale, col0, own_pos, P.S, pp, pd);
       else fb_tile<DKV, false>(rs, rd, ld_cols, own_ld, cl, scale, col0, own_pos, P.S, pp, pd);
-      // the operand tiles have one buffer: the previous step's accumulating products must have read them
-      if (!mbar_wait(bar(B_PDEMPTY), ((uint32_t)s & 1u) ^ 1u, abort_flag, P.status)) { ok = false; break; }
-      uint8_t* prow = gen_base + FB_P_OFF + row * 128;
-      uint8_t* drow = gen_base + FB_DS_OFF + row * 128;
+      // two buffers of operand tiles: the accumulating products of the step before last must have read this one
+      if (!mbar_wait(bar(B_PDEMPTY + b), ph ^ 1u, abort_flag, P.status)) { ok = false; break; }
+      uint8_t* prow = gen_base + FB_P_OFF + b * FA_TILE + row * 128;
+      uint8_t* drow = gen_base + FB_DS_OFF + b * FA_TILE + row * 128;
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         const int piece = ((4 * hh + g) ^ (row & 7)) << 4;
@@ -630,7 +630,7 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       }
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_PDFULL));
+      if (lane == 0) mbar_arrive(bar(B_PDFULL + b));
     }
     if (ok && !mbar_wait(bar(B_ACCFULL), 0u, abort_flag, P.status)) ok = false;
     if (ok) {
