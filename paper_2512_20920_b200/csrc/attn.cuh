@@ -72,6 +72,96 @@ __global__ void from_heads_kernel(const TIn* __restrict__ in, const float2* __re
   }
 }
 
+// The same two layout changes with 16-byte accesses, for head widths whose half is a multiple of 8: a thread takes 8
+// consecutive columns i .. i+7 of a head's first half and their partners i + hd/2 ..; a block covers
+// blockDim.x / (n * hd / 16) tokens.
+template <typename TIn, typename T>
+__global__ void to_heads_vec_kernel(const TIn* __restrict__ in, int64_t ld_in, const float* __restrict__ bias,
+                                    const float2* __restrict__ cs, int tokens, int S, int Sp, int n, int hd, T* __restrict__ out) {
+  const int half = hd / 2, units = n * half / 8;
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int t = (int)(gid / units), u = (int)(gid % units);
+  if (t >= tokens) return;
+  const int head = u / (half / 8), i = (u % (half / 8)) * 8;
+  const int b = t / S, s = t % S, c0 = head * hd + i, c1 = c0 + half;
+  Vec8<TIn> v0, v1;
+  v0.load(in + (int64_t)t * ld_in + c0);
+  v1.load(in + (int64_t)t * ld_in + c1);
+  float x0[8], x1[8], y0[8], y1[8];
+  v0.get(x0); v1.get(x1);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    if (bias) { x0[e] += bias[c0 + e]; x1[e] += bias[c1 + e]; }
+    y0[e] = x0[e]; y1[e] = x1[e];
+    if (cs) {
+      const float2 r = cs[s * half + i + e];
+      y0[e] = x0[e] * r.x - x1[e] * r.y;
+      y1[e] = x1[e] * r.x + x0[e] * r.y;
+    }
+  }
+  T* o = out + (((int64_t)b * n + head) * Sp + s) * hd + i;
+  Vec8<T> w0, w1;
+  w0.set(y0); w1.set(y1);
+  w0.store(o); w1.store(o + half);
+}
+
+template <typename TIn, typename T>
+__global__ void from_heads_vec_kernel(const TIn* __restrict__ in, const float2* __restrict__ cs, float sign, int tokens, int S,
+                                      int Sp, int n, int hd, T* __restrict__ out, int64_t ld_out, int col0) {
+  const int half = hd / 2, units = n * half / 8;
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int t = (int)(gid / units), u = (int)(gid % units);
+  if (t >= tokens) return;
+  const int head = u / (half / 8), i = (u % (half / 8)) * 8;
+  const int b = t / S, s = t % S;
+  const TIn* src = in + (((int64_t)b * n + head) * Sp + s) * hd + i;
+  Vec8<TIn> v0, v1;
+  v0.load(src); v1.load(src + half);
+  float x0[8], x1[8], y0[8], y1[8];
+  v0.get(x0); v1.get(x1);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    y0[e] = x0[e]; y1[e] = x1[e];
+    if (cs) {
+      const float2 r = cs[s * half + i + e];
+      const float sn = sign * r.y;
+      y0[e] = x0[e] * r.x - x1[e] * sn;
+      y1[e] = x1[e] * r.x + x0[e] * sn;
+    }
+  }
+  T* o = out + (int64_t)t * ld_out + col0 + head * hd + i;
+  Vec8<T> w0, w1;
+  w0.set(y0); w1.set(y1);
+  w0.store(o); w1.store(o + half);
+}
+
+template <typename TIn, typename T>
+inline cudaError_t launch_to_heads(const TIn* in, int64_t ld_in, const float* bias, const float2* cs, int tokens, int S, int Sp,
+                                   int n, int hd, T* out, cudaStream_t st) {
+  if (tokens <= 0) return cudaSuccess;
+  if ((hd / 2) % 8 == 0 && ld_in % 8 == 0) {
+    const int64_t threads = (int64_t)tokens * (n * (hd / 2) / 8);
+    to_heads_vec_kernel<TIn, T><<<(unsigned)ceil_div(threads, 256), 256, 0, st>>>(in, ld_in, bias, cs, tokens, S, Sp, n, hd, out);
+  } else {
+    to_heads_kernel<TIn, T><<<tokens, 256, 0, st>>>(in, ld_in, bias, cs, S, Sp, n, hd, out);
+  }
+  return cudaGetLastError();
+}
+
+template <typename TIn, typename T>
+inline cudaError_t launch_from_heads(const TIn* in, const float2* cs, float sign, int tokens, int S, int Sp, int n, int hd, T* out,
+                                     int64_t ld_out, int col0, cudaStream_t st) {
+  if (tokens <= 0) return cudaSuccess;
+  if ((hd / 2) % 8 == 0 && ld_out % 8 == 0 && col0 % 8 == 0) {
+    const int64_t threads = (int64_t)tokens * (n * (hd / 2) / 8);
+    from_heads_vec_kernel<TIn, T><<<(unsigned)ceil_div(threads, 256), 256, 0, st>>>(in, cs, sign, tokens, S, Sp, n, hd, out,
+                                                                                    ld_out, col0);
+  } else {
+    from_heads_kernel<TIn, T><<<tokens, 256, 0, st>>>(in, cs, sign, S, Sp, n, hd, out, ld_out, col0);
+  }
+  return cudaGetLastError();
+}
+
 // One warp per row of the score matrix; row = (sequence, head, s) with s < S_pad.  Keys j <= s take part;
 // the rest of the row, and every padding row, is written as zero (later products read whole rows).
 template <typename T>

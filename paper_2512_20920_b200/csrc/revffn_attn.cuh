@@ -188,11 +188,9 @@ static int a_project(const ACtx<T>& c, int side, const void* W, const float* bia
   p.epilogue = EPI_STORE; p.out_f32 = 1; p.C = c.template p<float>(L.raw); p.ldc = n * L.hd;
   CKR(a_gemm(c, p, TG_A_QKV));
   { ProfScope ps(TG_A_HEADS, c.st);
-  to_heads_kernel<float, T><<<Tn, 256, 0, c.st>>>(c.template p<float>(L.raw), (int64_t)n * L.hd, bias,
-                                                   rotate ? c.template p<float2>(L.cs) : nullptr, D.seq_len, L.Sp, n,
-                                                   L.hd, heads);
+  CK((launch_to_heads<float, T>(c.template p<float>(L.raw), (int64_t)n * L.hd, bias,
+                                rotate ? c.template p<float2>(L.cs) : nullptr, Tn, D.seq_len, L.Sp, n, L.hd, heads, c.st)));
   }
-  CK(cudaGetLastError());
   return REVFFN_OK;
 }
 
@@ -244,10 +242,9 @@ static int a_core(const ACtx<T>& c, bool need_p, bool keep_o32 = false) {
     CKR(a_gemm(c, p, TG_A_PV));
   }
   { ProfScope ps(TG_A_HEADS, c.st);
-  from_heads_kernel<T, T><<<L.T, 256, 0, c.st>>>(c.template p<T>(L.oh), nullptr, 1.f, D.seq_len, L.Sp, D.n_heads, L.hd,
-                                                 c.template p<T>(L.o), D.d_model, 0);
+  CK((launch_from_heads<T, T>(c.template p<T>(L.oh), nullptr, 1.f, L.T, D.seq_len, L.Sp, D.n_heads, L.hd,
+                              c.template p<T>(L.o), D.d_model, 0, c.st)));
   }
-  CK(cudaGetLastError());
   return REVFFN_OK;
 }
 
@@ -360,11 +357,12 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
     p.epilogue = EPI_STORE; p.out_f32 = f32 ? 1 : 0; p.C = C; p.ldc = N;
     return a_gemm(c, p, tag);
   };
+  const int strip = STRIP;      // rows per partial sum of the two-pass column reductions
   auto colsum = [&](const T* X, int64_t ldx, int cols, float* out) -> int {
-    const int strips = (int)ceil_div(Tn, STRIP);
+    const int strips = (int)ceil_div(Tn, strip);
     dim3 grid((unsigned)ceil_div(cols, 256), (unsigned)strips);
     { ProfScope ps(TG_A_BIAS, st);
-    colsum_partial_kernel<T><<<grid, 256, 0, st>>>(X, ldx, nullptr, Tn, cols, STRIP, c.template p<float>(L.part));
+    colsum_partial_kernel<T><<<grid, 256, 0, st>>>(X, ldx, nullptr, Tn, cols, strip, c.template p<float>(L.part));
     }
     CK(cudaGetLastError());
     { ProfScope ps(TG_A_BIAS, st);
@@ -385,10 +383,9 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
   if (G.w_o) CKR(wgrad(G.w_o, d, d, c.template p<T>(L.da), d, 0, c.template p<T>(L.o), d, Tn, acc));
   CKR(dgrad(TG_A_DGRAD, Tn, d, d, c.template p<T>(L.da), d, c.W.w_o, d, c.template p<T>(L.dob), false));
   { ProfScope ps(TG_A_HEADS, st);
-  to_heads_kernel<T, T><<<Tn, 256, 0, st>>>(c.template p<T>(L.dob), d, nullptr, nullptr, D.seq_len, Sp, D.n_heads, hd,
-                                            c.template p<T>(L.doh));
+  CK((launch_to_heads<T, T>(c.template p<T>(L.dob), d, nullptr, nullptr, Tn, D.seq_len, Sp, D.n_heads, hd,
+                            c.template p<T>(L.doh), st)));
   }
-  CK(cudaGetLastError());
 
   // attention core backward
   if (fused) {
@@ -445,20 +442,17 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
   }
   // back to token-major; the rotation is undone by its transpose
   { ProfScope ps(TG_A_HEADS, st);
-  from_heads_kernel<float, T><<<Tn, 256, 0, st>>>(c.template p<float>(L.dqh), c.template p<float2>(L.cs), -1.f, D.seq_len,
-                                                  Sp, D.n_heads, hd, c.template p<T>(L.dq), d, 0);
+  CK((launch_from_heads<float, T>(c.template p<float>(L.dqh), c.template p<float2>(L.cs), -1.f, Tn, D.seq_len, Sp,
+                                  D.n_heads, hd, c.template p<T>(L.dq), d, 0, st)));
   }
-  CK(cudaGetLastError());
   { ProfScope ps(TG_A_HEADS, st);
-  from_heads_kernel<float, T><<<Tn, 256, 0, st>>>(c.template p<float>(L.dkh), c.template p<float2>(L.cs), -1.f, D.seq_len,
-                                                  Sp, D.n_kv_heads, hd, c.template p<T>(L.dkv), 2 * (int64_t)dkv, 0);
+  CK((launch_from_heads<float, T>(c.template p<float>(L.dkh), c.template p<float2>(L.cs), -1.f, Tn, D.seq_len, Sp,
+                                  D.n_kv_heads, hd, c.template p<T>(L.dkv), 2 * (int64_t)dkv, 0, st)));
   }
-  CK(cudaGetLastError());
   { ProfScope ps(TG_A_HEADS, st);
-  from_heads_kernel<float, T><<<Tn, 256, 0, st>>>(c.template p<float>(L.dvh), nullptr, 1.f, D.seq_len, Sp, D.n_kv_heads,
-                                                  hd, c.template p<T>(L.dkv), 2 * (int64_t)dkv, dkv);
+  CK((launch_from_heads<float, T>(c.template p<float>(L.dvh), nullptr, 1.f, Tn, D.seq_len, Sp, D.n_kv_heads, hd,
+                                  c.template p<T>(L.dkv), 2 * (int64_t)dkv, dkv, st)));
   }
-  CK(cudaGetLastError());
 
   // q/k/v projections backward
   const T* u1 = c.template p<T>(L.u12);
@@ -505,11 +499,11 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
   }
   CK(cudaGetLastError());
   if (G.norm_gamma) {
-    const int strips = (int)ceil_div(Tn, STRIP);
+    const int strips = (int)ceil_div(Tn, strip);
     dim3 grid((unsigned)ceil_div(h, 256), (unsigned)strips);
     for (int side = 0; side < 2; ++side) {
       { ProfScope ps(TG_DGAMMA, st);
-      dgamma_partial_kernel<<<grid, 256, 0, st>>>(side ? dn2 : dn1, side ? x2 : x1, D.ld_stream, side ? r2 : r1, Tn, h, STRIP,
+      dgamma_partial_kernel<<<grid, 256, 0, st>>>(side ? dn2 : dn1, side ? x2 : x1, D.ld_stream, side ? r2 : r1, Tn, h, strip,
                                                   c.template p<float>(L.part));
       }
       CK(cudaGetLastError());
