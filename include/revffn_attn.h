@@ -47,7 +47,7 @@ extern "C" {
  *   divides n_heads; head_dim = d_model / n_heads is even.
  *   weight_dtype REVFFN_F32 : h, d and head_dim multiples of 8.
  *   weight_dtype REVFFN_BF16: h and d multiples of 128, head_dim 128 (TMA / tcgen05 tiles).
- * flags: REVFFN_FLAG_FORCE_SIMT only.
+ * flags: REVFFN_FLAG_FORCE_SIMT; REVFFN_FLAG_REUSE_ACTIVATIONS on a backward call (below).
  */
 typedef struct {
   int32_t batch, seq_len;       /* T = batch * seq_len tokens                              */
@@ -108,6 +108,10 @@ int revffn_attn_inverse(const revffn_attn_desc* desc, const revffn_attn_weights*
  *   dx2_inout[t] += J2^T dy1               (the gradient that reaches x2 through keys and values)
  *   grads->X (+)= dL/dX                    for every non-NULL member.
  * ws must hold at least bwd_bytes.
+ * With REVFFN_FLAG_REUSE_ACTIVATIONS the call takes the key/value side (which depends on x2 and the
+ * weights only) from the workspace, where a revffn_attn_inverse call with n_iter >= 1, the same x2,
+ * weights and descriptor has left it, and evaluates only the query side again: in reversible
+ * back-propagation the inverse pass of a block runs right before its gradient pass.
  */
 int revffn_attn_backward(const revffn_attn_desc* desc, const revffn_attn_weights* w,
                          const float* x1, const float* x2, const float* dy1,

@@ -90,7 +90,7 @@ static int validate_attn_desc(const revffn_attn_desc* D) {
     return REVFFN_ERR_SHAPE;
   }
   if (!(D->rope_theta > 0.f)) return REVFFN_ERR_SHAPE;
-  if (D->flags & ~REVFFN_FLAG_FORCE_SIMT) return REVFFN_ERR_UNSUPPORTED;
+  if (D->flags & ~(REVFFN_FLAG_FORCE_SIMT | REVFFN_FLAG_REUSE_ACTIVATIONS)) return REVFFN_ERR_UNSUPPORTED;
   if (D->ld_stream < h || (D->ld_stream % 4)) return REVFFN_ERR_ALIGN;
   const int64_t Sp = round_up(D->seq_len, ROW_PAD);
   if ((int64_t)D->batch * D->n_heads * Sp > (int64_t)1 << 30 || (int64_t)D->batch * D->seq_len > (int64_t)1 << 28)
@@ -329,12 +329,16 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
   cudaStream_t st = c.st;
 
   // recompute the branch's intermediates (Sec. 3.1: nothing was cached)
-  CKR(a_setup(c, true));
+  // REUSE: an inverse call (at least one iteration) on this workspace with the same x2 and weights has left the
+  // tables and the key/value side (n2, u2, k, v head-major) behind; only the query side is evaluated again
+  const bool reuse_kv = (D.flags & REVFFN_FLAG_REUSE_ACTIVATIONS) != 0;
+  if (!reuse_kv) CKR(a_setup(c, true));
+  else if (L.Sp != D.seq_len) CK(cudaMemsetAsync(c.ws + L.doh.off, 0, L.doh.bytes, st));
   // tcgen05 back end: the attention core runs fused in both directions and P is never written;
   // otherwise the score matrix is materialised and the gradient pass reads P from memory
   bool fused = false;
   if constexpr (std::is_same<T, bf16>::value) fused = c.tc && hd == FA_HD;
-  CKR(a_kv_side(c, x2));
+  if (!reuse_kv) CKR(a_kv_side(c, x2));
   CKR(a_query_side(c, x1, !fused, fused));      // fused: the score buffer holds the unrounded output instead
 
   auto wgrad = [&](float* out, int M, int N, const void* A, int64_t lda, int a_col0, const void* B, int64_t ldb,

@@ -78,7 +78,10 @@ static int block_backward_one(const revffn_block_desc& D, const revffn_attn_weig
   // Eq. 1 backwards: X1 by fixed-point iteration, then both stream gradients through the attention branch
   CKR(revffn_attn_inverse(&D.attn, wa, s1, s2, b.tmp, D.inverse_iters, b.ws, b.sub, stream));
   CKR(block_merge(b, st));
-  CKR(revffn_attn_backward(&D.attn, wa, b.tmp, s2, g1, g1, g2, ga, b.ws, b.sub, stream));
+  // the inverse pass has just evaluated the key/value side from the same X2 in this workspace
+  revffn_attn_desc d_ab = D.attn;
+  if (D.inverse_iters >= 1) d_ab.flags |= REVFFN_FLAG_REUSE_ACTIVATIONS;
+  CKR(revffn_attn_backward(&d_ab, wa, b.tmp, s2, g1, g1, g2, ga, b.ws, b.sub, stream));
   CKR(block_merge(b, st));
   if (D.moe.tokens > 0)
     CK(cudaMemcpy2DAsync(s1, (size_t)D.moe.ld_stream * 4, b.tmp, (size_t)D.moe.ld_stream * 4,
