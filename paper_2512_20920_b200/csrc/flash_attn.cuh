@@ -8,13 +8,14 @@
 //   warp 1      MMA issuer and TMEM owner.  TMEM (512 columns): two score accumulators S0/S1 and two
 //               output accumulators O0/O1 of 128 fp32 columns each.
 //               S_j = Q K_j^T is issued one block ahead of O_j = P_j V_j, so the tensor pipe computes
-//               the next scores while the softmax warps work on the current ones.
+//               the next scores while the softmax warps work on the current ones.  P_j is the A operand
+//               of the second product straight from tensor memory.
 //   warps 2..9  softmax: two threads per query row (= TMEM lane), 64 keys each.  Per block: the scores
 //               into registers, row maximum (the halves exchange theirs through shared memory),
-//               p = exp2((s - m) * scale * log2 e), P as bf16 into shared memory in the K-major
-//               128-byte-swizzled operand layout (one buffer: written once the previous block's
-//               P V product has read it), then the PREVIOUS block's O_j (this thread's 64 columns) is
-//               added into a register accumulator,
+//               p = exp2((s - m) * scale * log2 e), P as bf16 pairs over the first 64 columns of the
+//               score accumulator it came from (tcgen05.st; no shared-memory round trip, and the
+//               tensor core reads 4 KB less per instruction), then the PREVIOUS block's O_j (this
+//               thread's 64 columns) is added into a register accumulator,
 //               acc = acc * exp2((m_old - m_new) ...) + O_j.  Every O_j is a fresh TMEM accumulator, so
 //               no rescaling pass over TMEM is needed and P_j V_j never waits for a correction.
 // Operands: q, k, v head-major [.., S_pad, hd] bf16 with hd = 128 (rows past the sequence are zero);
@@ -33,8 +34,7 @@ constexpr int FA_TILE = FA_BLK * 64 * 2;          // one 64-wide K block of an o
 constexpr int FA_Q_OFF = 0;                       // Q: 2 tiles
 constexpr int FA_K_OFF = 2 * FA_TILE;             // K: 2 stages x 2 tiles
 constexpr int FA_V_OFF = FA_K_OFF + 4 * FA_TILE;  // V: 2 stages x 2 k-blocks (each 2 chunks of 8 KB)
-constexpr int FA_P_OFF = FA_V_OFF + 4 * FA_TILE;  // P: 2 tiles
-constexpr int FA_BAR_OFF = FA_P_OFF + 2 * FA_TILE;
+constexpr int FA_BAR_OFF = FA_V_OFF + 4 * FA_TILE;
 constexpr int FA_XMAX_OFF = FA_BAR_OFF + 256;             // row maxima exchanged between the two halves: [2][2][128] floats
 constexpr int FA_XSUM_OFF = FA_XMAX_OFF + 2048;           // row sums exchanged at the end: [2][128] floats
 constexpr int FA_SMEM_BYTES = FA_XSUM_OFF + 1024 + 1024;  // + alignment slack
@@ -79,6 +79,27 @@ __device__ __forceinline__ float fa_probs(const uint32_t (&r0)[32], const uint32
   return sum;
 }
 
+// 32 consecutive 32-bit columns of this thread's TMEM lane, written from registers.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
+        "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
+        "r"(r[30]), "r"(r[31]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// D += A B with A in tensor memory (rows = lanes, two 16-bit K elements per 32-bit column), B from shared memory.
+__device__ __forceinline__ void tc_mma_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+
 struct FlashParams {
   int S, Sp, n_heads, rep;        // rep = query heads per key/value head
   bf16* o; int64_t ld_o;          // [T, ld_o]
@@ -99,7 +120,7 @@ flash_fwd_kernel(const FlashParams P, const __grid_constant__ CUtensorMap map_q,
   // barrier slots (8 bytes each)
   auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
   enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_SEMPTY = 11, B_PFULL = 13,
-         B_OFULL = 14, B_OEMPTY = 16, B_COUNT = 18 };
+         B_OFULL = 15, B_OEMPTY = 17, B_COUNT = 19 };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + FA_BAR_OFF + 8 * B_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + FA_BAR_OFF + 8 * B_COUNT + 8);
   int* issued = reinterpret_cast<int*>(gen_base + FA_BAR_OFF + 8 * B_COUNT + 16);   // [5]: q, k0, k1, v0, v1 -> phase + 1
@@ -118,11 +139,10 @@ flash_fwd_kernel(const FlashParams P, const __grid_constant__ CUtensorMap map_q,
 
   if (threadIdx.x == 0) {
     mbar_init(bar(B_QFULL), 1);
-    mbar_init(bar(B_PFULL), 8);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(B_KFULL + s), 1); mbar_init(bar(B_KEMPTY + s), 1);
       mbar_init(bar(B_VFULL + s), 1); mbar_init(bar(B_VEMPTY + s), 1);
-      mbar_init(bar(B_SFULL + s), 1); mbar_init(bar(B_SEMPTY + s), 8);
+      mbar_init(bar(B_SFULL + s), 1); mbar_init(bar(B_SEMPTY + s), 1); mbar_init(bar(B_PFULL + s), 8);
       mbar_init(bar(B_OFULL + s), 1); mbar_init(bar(B_OEMPTY + s), 8);
     }
     for (int i = 0; i < 5; ++i) issued[i] = 0;
@@ -197,19 +217,20 @@ flash_fwd_kernel(const FlashParams P, const __grid_constant__ CUtensorMap map_q,
         const uint32_t ph = (uint32_t)(j >> 1) & 1u;
         if (!mbar_wait(bar(B_VFULL + b), ph, abort_flag, P.status)) { ok = false; break; }
         if (!mbar_wait(bar(B_OEMPTY + b), ph ^ 1u, abort_flag, P.status)) { ok = false; break; }
-        if (!mbar_wait(bar(B_PFULL), (uint32_t)j & 1u, abort_flag, P.status)) { ok = false; break; }
+        if (!mbar_wait(bar(B_PFULL + b), ph, abort_flag, P.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d = tmem_base + (uint32_t)(2 * FA_BLK + b * FA_BLK);
+        const uint32_t a_tmem = tmem_base + (uint32_t)(b * FA_BLK);      // P over the first 64 columns of S
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
-          const uint64_t a_desc = make_smem_desc(base + FA_P_OFF + kb * FA_TILE, 16, 1024);
           const uint64_t b_desc = make_smem_desc(base + FA_V_OFF + (2 * b + kb) * FA_TILE, 8192, 1024);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
-            tc_mma(d, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(128 * ks), idesc_pv, (kb | ks) != 0 ? 1u : 0u);
+            tc_mma_ta(d, a_tmem + (uint32_t)(8 * (4 * kb + ks)), b_desc + (uint64_t)(128 * ks), idesc_pv, (kb | ks) != 0 ? 1u : 0u);
         }
         tc_commit(bar(B_VEMPTY + b));
         tc_commit(bar(B_OFULL + b));
+        tc_commit(bar(B_SEMPTY + b));      // the scores' columns (now holding P) are free again
       }
     }
   } else {
@@ -261,10 +282,6 @@ flash_fwd_kernel(const FlashParams P, const __grid_constant__ CUtensorMap map_q,
         tmem_ld32(lane_addr + (uint32_t)(b * FA_BLK), r0);
         tmem_ld32(lane_addr + (uint32_t)(b * FA_BLK + 32), r1);
         tmem_ld_wait();
-        // scores are in registers: the accumulator may be overwritten by the block after next
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(B_SEMPTY + b));
         mx = diag ? fa_row_max<true>(r0, r1, 64 * half, row) : fa_row_max<false>(r0, r1, 64 * half, row);
         xmax[(b * 2 + half) * FA_BLK + row] = mx;
       }
@@ -278,16 +295,20 @@ flash_fwd_kernel(const FlashParams P, const __grid_constant__ CUtensorMap map_q,
                                : fa_probs<false>(r0, r1, cl, mc, 64 * half, row, pk);
         l = l * alpha + sum;
         m = m_new;
-        // P has one buffer: the previous block's P V product must have read it
-        if (j >= 1 && !wait_o(j - 1)) ok = false;
-        if (ok) {
-          // this thread's 64 keys are exactly tile `half` of P (64 keys per tile): eight 16-byte pieces of its row
-          uint8_t* tile_row = gen_base + FA_P_OFF + half * FA_TILE + row * 128;
+        {
+          // P over the scores in tensor memory: this thread's 64 keys are 32 columns of packed pairs.  Both halves
+          // of the row have their scores in registers (they met at the barrier above).
+          uint32_t pw[32];
 #pragma unroll
-          for (int g = 0; g < 8; ++g) *reinterpret_cast<uint4*>(tile_row + ((g ^ (row & 7)) << 4)) = pk[g];
-          fence_async_smem();                    // P visible to the tensor core's reads
+          for (int g = 0; g < 8; ++g) { pw[4 * g] = pk[g].x; pw[4 * g + 1] = pk[g].y; pw[4 * g + 2] = pk[g].z; pw[4 * g + 3] = pk[g].w; }
+          tmem_st32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * FA_BLK + 32 * half), pw);
+          tmem_st_wait();
+          tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar(B_PFULL));
+          if (lane == 0) mbar_arrive(bar(B_PFULL + b));
+          if (j >= 1 && !wait_o(j - 1)) ok = false;
+        }
+        if (ok) {
           if (j >= 1) add_block(j - 1, alpha_pending);
           alpha_pending = alpha;
         }
@@ -388,6 +409,8 @@ inline int launch_flash_fwd(const bf16* q, const bf16* k, const bf16* v, int bat
 // current step), and the accumulators (fresh TMEM columns, summed over
 // all steps by the tensor core itself) take  acc0 += P' Y1  (DKV only)  and  acc1 += dS' Y0,  where the same
 // shared-memory bytes of a Y tile that served as a K-major operand are read again as an MN-major one.
+// The dQ launch has TMEM columns to spare and keeps its owned operands there (A operand from tensor memory),
+// which takes two thirds of the shared-memory reads out of its steps.
 // No cross-thread reduction is needed: the row statistics come from memory.
 // ---------------------------------------------------------------------------
 constexpr int FB_X_OFF = 0;                        // X0, X1: 2 tiles of 16 KB each
@@ -401,6 +424,7 @@ constexpr int FB_SMEM_BYTES = FB_LD_OFF + 1024 + 1024;
 struct FlashBwdParams {
   int S, Sp, n_heads, rep;
   const float2* lse_d;            // per query row (head-major index): (lse * log2 e, D * scale)
+  const bf16* x0; const bf16* x1; // !DKV: the owned operands (q, d_o head-major), read by the CTA's threads themselves
   float* out0;                    // DKV: dV [kv rows, 128] fp32
   float* out1;                    // DKV: dK [kv rows, 128];  else dQ [q rows, 128]
   float scale_log2e, scale;
@@ -480,7 +504,7 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   auto y_row_of = [&](int s) -> int { return y_base + (s / n_inner) * P.Sp + 64 * (t_begin + s % n_inner); };
 
   if (threadIdx.x == 0) {
-    mbar_init(bar(B_XFULL), 1);
+    mbar_init(bar(B_XFULL), DKV ? 1 : 8);
     mbar_init(bar(B_ACCFULL), 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(B_YFULL + s), 1); mbar_init(bar(B_YEMPTY + s), 1);
@@ -509,11 +533,13 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
-      mbar_expect_tx(bar(B_XFULL), 4 * FA_TILE);
-      issued[0] = 1;
-      for (int kb = 0; kb < 2; ++kb) {
-        tma_load_2d(base + FB_X_OFF + kb * FA_TILE, &map_x0, 64 * kb, own_row0, bar(B_XFULL));
-        tma_load_2d(base + FB_X_OFF + (2 + kb) * FA_TILE, &map_x1, 64 * kb, own_row0, bar(B_XFULL));
+      if (DKV) {
+        mbar_expect_tx(bar(B_XFULL), 4 * FA_TILE);
+        issued[0] = 1;
+        for (int kb = 0; kb < 2; ++kb) {
+          tma_load_2d(base + FB_X_OFF + kb * FA_TILE, &map_x0, 64 * kb, own_row0, bar(B_XFULL));
+          tma_load_2d(base + FB_X_OFF + (2 + kb) * FA_TILE, &map_x1, 64 * kb, own_row0, bar(B_XFULL));
+        }
       }
       for (int s = 0; s < n_steps; ++s) {
         const int b = s & 1;
@@ -550,8 +576,13 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
             const uint64_t a_desc = make_smem_desc(base + FB_X_OFF + (2 * w + kb) * FA_TILE, 16, 1024);
             const uint64_t b_desc = make_smem_desc(ys + w * FA_TILE + kb * 8192, 16, 1024);
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              tc_mma(d, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(2 * ks), idesc_sd, (kb | ks) != 0 ? 1u : 0u);
+            for (int ks = 0; ks < 4; ++ks) {
+              if (DKV)
+                tc_mma(d, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(2 * ks), idesc_sd, (kb | ks) != 0 ? 1u : 0u);
+              else   // the owned operand sits in tensor memory: 8 columns of packed pairs per 16 k
+                tc_mma_ta(d, tmem_base + (uint32_t)(256 + 64 * w + 8 * (4 * kb + ks)), b_desc + (uint64_t)(2 * ks), idesc_sd,
+                          (kb | ks) != 0 ? 1u : 0u);
+            }
           }
         }
         tc_commit(bar(B_SDFULL + b));
@@ -594,6 +625,25 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
     const int own_pos = blk * FA_BLK + row;      // position in the sequence of this thread's own row
     float2 own_ld = make_float2(0.f, 0.f);
     if (!DKV && own_pos < P.S) own_ld = P.lse_d[own_row0 + row];
+    if (!DKV) {
+      // The owned operands never change: each thread puts its row's 64 columns of both into tensor memory
+      // (TMEM columns 256.. for X0, 320.. for X1), where every step's products read them as the A operand.
+#pragma unroll
+      for (int w = 0; w < 2; ++w) {
+        const uint4* src = reinterpret_cast<const uint4*>((w ? P.x1 : P.x0) + (int64_t)(own_row0 + row) * FA_HD + 64 * hh);
+        uint32_t xw[32];
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint4 v = __ldg(src + g);
+          xw[4 * g] = v.x; xw[4 * g + 1] = v.y; xw[4 * g + 2] = v.z; xw[4 * g + 3] = v.w;
+        }
+        tmem_st32(lane_addr + (uint32_t)(256 + 64 * w + 32 * hh), xw);
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_XFULL));
+    }
     bool ok = true;
     for (int s = 0; s < n_steps; ++s) {
       const int b = s & 1;
@@ -723,9 +773,11 @@ inline int launch_flash_bwd(const bf16* q, const bf16* k, const bf16* v, const b
   P.scale_log2e = P.scale * 1.4426950408889634f;
   P.status = status;
   P.out0 = dv; P.out1 = dk;
+  P.x0 = nullptr; P.x1 = nullptr;
   flash_bwd_kernel<true><<<batch * n_kv_heads * (Sp / FA_BLK), FA_THREADS, FB_SMEM_BYTES, st>>>(P, k128, v128, q64, do64);
   if (cudaGetLastError() != cudaSuccess) return REVFFN_ERR_CUDA;
   P.out0 = nullptr; P.out1 = dq;
+  P.x0 = q; P.x1 = d_o;
   flash_bwd_kernel<false><<<batch * n_heads * (Sp / FA_BLK), FA_THREADS, FB_SMEM_BYTES, st>>>(P, q128, do128, k64, v64);
   return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
