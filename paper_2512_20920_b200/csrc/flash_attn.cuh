@@ -405,21 +405,29 @@ inline int launch_flash_fwd(const bf16* q, const bf16* k, const bf16* v, int bat
 // Per step the "own" side is the MMA M side and the walked tile the N side, so both cases compute
 //   S' = X0 Y0^T,  dP' = X1 Y1^T   (128 x 64, K = hd; X = own operands, Y = the walked tiles)
 // into TMEM (double-buffered), eight warps (two threads per own row, 32 columns each) turn them into P' and
-// dS' as bf16 K-major operand tiles in shared memory (double-buffered too, so that neither side waits for the other's
-// current step), and the accumulators (fresh TMEM columns, summed over
+// dS' as bf16 K-major operand tiles in shared memory, and the accumulators (fresh TMEM columns, summed over
 // all steps by the tensor core itself) take  acc0 += P' Y1  (DKV only)  and  acc1 += dS' Y0,  where the same
 // shared-memory bytes of a Y tile that served as a K-major operand are read again as an MN-major one.
 // The dQ launch has TMEM columns to spare and keeps its owned operands there (A operand from tensor memory),
 // which takes two thirds of the shared-memory reads out of its steps.
 // No cross-thread reduction is needed: the row statistics come from memory.
 // ---------------------------------------------------------------------------
-constexpr int FB_X_OFF = 0;                        // X0, X1: 2 tiles of 16 KB each
-constexpr int FB_Y_OFF = 4 * FA_TILE;              // 2 stages x [Y0 2 x 8 KB | Y1 2 x 8 KB]
-constexpr int FB_P_OFF = FB_Y_OFF + 4 * FA_TILE;   // P' tiles, 2 x 16 KB
-constexpr int FB_DS_OFF = FB_P_OFF + 2 * FA_TILE;  // dS' tiles, 2 x 16 KB
-constexpr int FB_BAR_OFF = FB_DS_OFF + 2 * FA_TILE;
-constexpr int FB_LD_OFF = FB_BAR_OFF + 256;        // DKV: (lse * log2 e, D * scale) of the step's 64 query rows, 2 stages x 512 B
-constexpr int FB_SMEM_BYTES = FB_LD_OFF + 1024 + 1024;
+// Shared memory.  DKV: [X0, X1 64 KB | 3 stages of walked tiles 96 KB]; else (owned operands in tensor memory):
+// [5 stages 160 KB]; then in both: P' tile 16 KB, dS' tile 16 KB, barriers, row statistics of the stages.
+// A stage: [Y0 2 x 8 KB | Y1 2 x 8 KB].  The walked tiles come from L2 with a latency of more than one step,
+// hence the deep ring.
+constexpr int FB_X_OFF = 0;
+constexpr int FB_STAGE = 2 * FA_TILE;
+template <bool DKV> struct FbCfg {
+  static constexpr int NS = DKV ? 3 : 5;
+  static constexpr int Y_OFF = DKV ? 4 * FA_TILE : 0;
+};
+constexpr int FB_P_OFF = 10 * FA_TILE;
+constexpr int FB_DS_OFF = FB_P_OFF + FA_TILE;
+constexpr int FB_BAR_OFF = FB_DS_OFF + FA_TILE;
+constexpr int FB_LD_OFF = FB_BAR_OFF + 256;        // DKV: (lse * log2 e, D * scale) of a stage's 64 query rows, 512 B per stage
+constexpr int FB_SMEM_BYTES = FB_LD_OFF + 2048 + 1024;
+constexpr int FB_MAX_NS = 5;
 
 struct FlashBwdParams {
   int S, Sp, n_heads, rep;
@@ -481,11 +489,13 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   uint8_t* gen_base = fa_smem_raw + (base - raw);
   const uint32_t bars = base + FB_BAR_OFF;
   auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
-  enum { B_XFULL = 0, B_YFULL = 1, B_YEMPTY = 3, B_SDFULL = 5, B_SDEMPTY = 7, B_PDFULL = 9, B_PDEMPTY = 11, B_ACCFULL = 13,
-         B_COUNT = 14 };
+  constexpr int NS = FbCfg<DKV>::NS;
+  constexpr int Y_OFF = FbCfg<DKV>::Y_OFF;
+  enum { B_XFULL = 0, B_YFULL = 1, B_YEMPTY = 1 + FB_MAX_NS, B_SDFULL = 1 + 2 * FB_MAX_NS, B_SDEMPTY = B_SDFULL + 2,
+         B_PDFULL = B_SDEMPTY + 2, B_PDEMPTY = B_PDFULL + 1, B_ACCFULL = B_PDEMPTY + 1, B_COUNT = B_ACCFULL + 1 };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + FB_BAR_OFF + 8 * B_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + FB_BAR_OFF + 8 * B_COUNT + 8);
-  int* issued = reinterpret_cast<int*>(gen_base + FB_BAR_OFF + 8 * B_COUNT + 16);   // [3]: x, y0, y1 -> phase + 1
+  int* issued = reinterpret_cast<int*>(gen_base + FB_BAR_OFF + 8 * B_COUNT + 16);   // [1 + NS]: x, y stages -> phase + 1
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_blk = P.Sp / FA_BLK;                  // 128-row blocks per head
@@ -506,12 +516,11 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   if (threadIdx.x == 0) {
     mbar_init(bar(B_XFULL), DKV ? 1 : 8);
     mbar_init(bar(B_ACCFULL), 1);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(bar(B_YFULL + s), 1); mbar_init(bar(B_YEMPTY + s), 1);
-      mbar_init(bar(B_SDFULL + s), 1); mbar_init(bar(B_SDEMPTY + s), 8);
-      mbar_init(bar(B_PDFULL + s), 8); mbar_init(bar(B_PDEMPTY + s), 1);
-    }
-    for (int i = 0; i < 3; ++i) issued[i] = 0;
+    mbar_init(bar(B_PDFULL), 8);
+    mbar_init(bar(B_PDEMPTY), 1);
+    for (int s = 0; s < NS; ++s) { mbar_init(bar(B_YFULL + s), 1); mbar_init(bar(B_YEMPTY + s), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(bar(B_SDFULL + s), 1); mbar_init(bar(B_SDEMPTY + s), 8); }
+    for (int i = 0; i < 1 + NS; ++i) issued[i] = 0;
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -542,17 +551,17 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
         }
       }
       for (int s = 0; s < n_steps; ++s) {
-        const int b = s & 1;
-        const uint32_t ph = (uint32_t)(s >> 1) & 1u;
-        if (!mbar_wait(bar(B_YEMPTY + b), ph ^ 1u, abort_flag, P.status)) break;
-        mbar_expect_tx(bar(B_YFULL + b), 2 * FA_TILE + (DKV ? 512 : 0));
-        issued[1 + b] = (int)ph + 1;
+        const int st = s % NS;
+        const uint32_t ph = (uint32_t)(s / NS) & 1u;
+        if (!mbar_wait(bar(B_YEMPTY + st), ph ^ 1u, abort_flag, P.status)) break;
+        mbar_expect_tx(bar(B_YFULL + st), FB_STAGE + (DKV ? 512 : 0));
+        issued[1 + st] = (int)ph + 1;
         const int yr = y_row_of(s);
-        if (DKV) bulk_load_1d(base + FB_LD_OFF + b * 512, P.lse_d + yr, 512, bar(B_YFULL + b));
-        const uint32_t ys = base + FB_Y_OFF + b * 2 * FA_TILE;
+        if (DKV) bulk_load_1d(base + FB_LD_OFF + st * 512, P.lse_d + yr, 512, bar(B_YFULL + st));
+        const uint32_t ys = base + Y_OFF + st * FB_STAGE;
         for (int kb = 0; kb < 2; ++kb) {
-          tma_load_2d(ys + kb * 8192, &map_y0, 64 * kb, yr, bar(B_YFULL + b));
-          tma_load_2d(ys + FA_TILE + kb * 8192, &map_y1, 64 * kb, yr, bar(B_YFULL + b));
+          tma_load_2d(ys + kb * 8192, &map_y0, 64 * kb, yr, bar(B_YFULL + st));
+          tma_load_2d(ys + FA_TILE + kb * 8192, &map_y1, 64 * kb, yr, bar(B_YFULL + st));
         }
       }
     }
@@ -562,12 +571,12 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       bool ok = mbar_wait(bar(B_XFULL), 0u, abort_flag, P.status);
       tc_fence_after();
       auto issue_sd = [&](int s) -> bool {
-        const int b = s & 1;
+        const int b = s & 1, st = s % NS;
         const uint32_t ph = (uint32_t)(s >> 1) & 1u;
-        if (!mbar_wait(bar(B_YFULL + b), ph, abort_flag, P.status)) return false;
+        if (!mbar_wait(bar(B_YFULL + st), (uint32_t)(s / NS) & 1u, abort_flag, P.status)) return false;
         if (!mbar_wait(bar(B_SDEMPTY + b), ph ^ 1u, abort_flag, P.status)) return false;
         tc_fence_after();
-        const uint32_t ys = base + FB_Y_OFF + b * 2 * FA_TILE;
+        const uint32_t ys = base + Y_OFF + st * FB_STAGE;
 #pragma unroll
         for (int w = 0; w < 2; ++w) {            // w = 0: S' = X0 Y0^T, w = 1: dP' = X1 Y1^T
           const uint32_t d = tmem_base + (uint32_t)(b * 128 + w * 64);
@@ -591,27 +600,27 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       if (ok) ok = issue_sd(0);
       for (int s = 0; ok && s < n_steps; ++s) {
         if (s + 1 < n_steps && !issue_sd(s + 1)) { ok = false; break; }
-        const int b = s & 1;
-        if (!mbar_wait(bar(B_PDFULL + b), (uint32_t)(s >> 1) & 1u, abort_flag, P.status)) { ok = false; break; }
+        const int st = s % NS;
+        if (!mbar_wait(bar(B_PDFULL), (uint32_t)s & 1u, abort_flag, P.status)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t ys = base + FB_Y_OFF + b * 2 * FA_TILE;
+        const uint32_t ys = base + Y_OFF + st * FB_STAGE;
         // the walked tiles again, now as [64 rows (K), 128 columns (N)] operands: the two 64-column halves are 8 KB apart
         if (DKV) {
-          const uint64_t a_desc = make_smem_desc(base + FB_P_OFF + b * FA_TILE, 16, 1024);
+          const uint64_t a_desc = make_smem_desc(base + FB_P_OFF, 16, 1024);
           const uint64_t b_desc = make_smem_desc(ys + FA_TILE, 8192, 1024);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
             tc_mma(tmem_base + 256u, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(128 * ks), idesc_acc, (s | ks) != 0 ? 1u : 0u);
         }
         {
-          const uint64_t a_desc = make_smem_desc(base + FB_DS_OFF + b * FA_TILE, 16, 1024);
+          const uint64_t a_desc = make_smem_desc(base + FB_DS_OFF, 16, 1024);
           const uint64_t b_desc = make_smem_desc(ys, 8192, 1024);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
             tc_mma(tmem_base + 384u, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(128 * ks), idesc_acc, (s | ks) != 0 ? 1u : 0u);
         }
-        tc_commit(bar(B_YEMPTY + b));
-        tc_commit(bar(B_PDEMPTY + b));
+        tc_commit(bar(B_YEMPTY + st));
+        tc_commit(bar(B_PDEMPTY));
       }
       if (ok) tc_commit(bar(B_ACCFULL));
     }
@@ -650,7 +659,7 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       const uint32_t ph = (uint32_t)(s >> 1) & 1u;
       if (!mbar_wait(bar(B_SDFULL + b), ph, abort_flag, P.status)) { ok = false; break; }
       // DKV: this thread reads the stage's row statistics itself, so it observes the stage's barrier itself
-      if (DKV && !mbar_wait(bar(B_YFULL + b), ph, abort_flag, P.status)) { ok = false; break; }
+      if (DKV && !mbar_wait(bar(B_YFULL + s % NS), (uint32_t)(s / NS) & 1u, abort_flag, P.status)) { ok = false; break; }
       tc_fence_after();
       uint32_t rs[32], rd[32];
       tmem_ld32(lane_addr + (uint32_t)(b * 128 + 32 * hh), rs);
@@ -664,14 +673,14 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       // tiles that touch the diagonal or the end of the sequence need the element-wise test
       const bool mask = DKV ? (t < 2 * blk + 2 || 64 * t + 63 >= P.S) : (t >= 2 * blk || blk * FA_BLK + FA_BLK - 1 >= P.S);
       // DKV: the step's row statistics came with the walked tiles (S' complete implies that stage has landed)
-      const float4* ld_cols = reinterpret_cast<const float4*>(gen_base + FB_LD_OFF + b * 512) + 16 * hh;
+      const float4* ld_cols = reinterpret_cast<const float4*>(gen_base + FB_LD_OFF + (s % NS) * 512) + 16 * hh;
       uint4 pp[4], pd[4];
       if (mask) fb_tile<DKV, true>(rs, rd, ld_cols, own_ld, cl, scale, col0, own_pos, P.S, pp, pd);
       else fb_tile<DKV, false>(rs, rd, ld_cols, own_ld, cl, scale, col0, own_pos, P.S, pp, pd);
-      // two buffers of operand tiles: the accumulating products of the step before last must have read this one
-      if (!mbar_wait(bar(B_PDEMPTY + b), ph ^ 1u, abort_flag, P.status)) { ok = false; break; }
-      uint8_t* prow = gen_base + FB_P_OFF + b * FA_TILE + row * 128;
-      uint8_t* drow = gen_base + FB_DS_OFF + b * FA_TILE + row * 128;
+      // the operand tiles have one buffer: the previous step's accumulating products must have read them
+      if (!mbar_wait(bar(B_PDEMPTY), ((uint32_t)s & 1u) ^ 1u, abort_flag, P.status)) { ok = false; break; }
+      uint8_t* prow = gen_base + FB_P_OFF + row * 128;
+      uint8_t* drow = gen_base + FB_DS_OFF + row * 128;
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         const int piece = ((4 * hh + g) ^ (row & 7)) << 4;
@@ -680,7 +689,7 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       }
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_PDFULL + b));
+      if (lane == 0) mbar_arrive(bar(B_PDFULL));
     }
     if (ok && !mbar_wait(bar(B_ACCFULL), 0u, abort_flag, P.status)) ok = false;
     if (ok) {
@@ -707,11 +716,10 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   tc_fence_before();
   __syncthreads();
   if (*abort_flag && threadIdx.x == 0) {
-    const int bidx[3] = {B_XFULL, B_YFULL, B_YFULL + 1};
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < 1 + NS; ++i) {      // slot 0: the owned operands, slot 1 + st: stage st of the walked tiles
       if (issued[i] == 0) continue;
       long long t0 = clock64();
-      while (!mbar_try_wait(bar(bidx[i]), (uint32_t)(issued[i] - 1)) && clock64() - t0 < TC_WAIT_CYCLES) {}
+      while (!mbar_try_wait(bar(i == 0 ? B_XFULL : B_YFULL + i - 1), (uint32_t)(issued[i] - 1)) && clock64() - t0 < TC_WAIT_CYCLES) {}
     }
   }
   __syncthreads();
