@@ -143,13 +143,25 @@ __global__ void colsum_partial_kernel(const T* __restrict__ X, int64_t ldx, cons
   part[(int64_t)b * cols + c] = acc;
 }
 
-__global__ void colsum_final_kernel(const float* __restrict__ part, int n_strips, int cols, int accumulate,
-                                    float* __restrict__ out) {
-  int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= cols) return;
+// Launch with COLSUM_FINAL_COLS columns per block of 256 threads: 8 threads share a column, each adds every 8th
+// strip in ascending order, and the 8 sums are added in a fixed order.
+constexpr int COLSUM_FINAL_COLS = 32;
+__global__ void __launch_bounds__(256)
+colsum_final_kernel(const float* __restrict__ part, int n_strips, int cols, int accumulate, float* __restrict__ out) {
+  __shared__ float red[8][COLSUM_FINAL_COLS];
+  const int cl = threadIdx.x % COLSUM_FINAL_COLS, g = threadIdx.x / COLSUM_FINAL_COLS;
+  const int c = blockIdx.x * COLSUM_FINAL_COLS + cl;
   float acc = 0.f;
-  for (int b = 0; b < n_strips; ++b) acc += part[(int64_t)b * cols + c];
-  out[c] = (accumulate ? out[c] : 0.f) + acc;
+  if (c < cols)
+    for (int b = g; b < n_strips; b += 8) acc += part[(int64_t)b * cols + c];
+  red[g][cl] = acc;
+  __syncthreads();
+  if (g == 0 && c < cols) {
+    float v = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v += red[i][cl];
+    out[c] = (accumulate ? out[c] : 0.f) + v;
+  }
 }
 
 // dU[t, :] = sum_s dUp[tok_row[t,s], :] + dUsh[t, :] + sum_s tok_dl[t,s] * W_r[idx[t,s], :]

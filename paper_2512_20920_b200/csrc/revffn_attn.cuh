@@ -370,7 +370,7 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
     }
     CK(cudaGetLastError());
     { ProfScope ps(TG_A_BIAS, st);
-    colsum_final_kernel<<<(unsigned)ceil_div(cols, 256), 256, 0, st>>>(c.template p<float>(L.part), strips, cols, acc, out);
+    colsum_final_kernel<<<(unsigned)ceil_div(cols, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), strips, cols, acc, out);
     }
     CK(cudaGetLastError());
     return REVFFN_OK;
@@ -512,7 +512,7 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
       }
       CK(cudaGetLastError());
       { ProfScope ps(TG_DGAMMA, st);
-      colsum_final_kernel<<<(unsigned)ceil_div(h, 256), 256, 0, st>>>(c.template p<float>(L.part), strips, h,
+      colsum_final_kernel<<<(unsigned)ceil_div(h, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), strips, h,
                                                                       side ? 1 : acc, G.norm_gamma);
       }
       CK(cudaGetLastError());

@@ -512,7 +512,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       }
       CK(cudaGetLastError());
       { ProfScope ps(TG_WG_SGATE, st);
-      colsum_final_kernel<<<(unsigned)ceil_div(d, 256), 256, 0, st>>>(c.template p<float>(L.part), L.strips, d, acc,
+      colsum_final_kernel<<<(unsigned)ceil_div(d, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), L.strips, d, acc,
                                                                       G.ws_sgate);
       }
       CK(cudaGetLastError());
@@ -600,7 +600,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       }
       CK(cudaGetLastError());
       { ProfScope ps(TG_WG_ROUTER, st);
-      colsum_final_kernel<<<(unsigned)ceil_div(E, 256), 256, 0, st>>>(c.template p<float>(L.part), L.strips, E, acc,
+      colsum_final_kernel<<<(unsigned)ceil_div(E, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), L.strips, E, acc,
                                                                       G.b_router);
       }
       CK(cudaGetLastError());
@@ -643,7 +643,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       }
       CK(cudaGetLastError());
       { ProfScope ps(TG_DGAMMA, st);
-      colsum_final_kernel<<<(unsigned)ceil_div(h, 256), 256, 0, st>>>(c.template p<float>(L.part), L.strips, h, acc,
+      colsum_final_kernel<<<(unsigned)ceil_div(h, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), L.strips, h, acc,
                                                                       G.norm_gamma);
       }
       CK(cudaGetLastError());
