@@ -130,17 +130,49 @@ __global__ void router_wgrad_kernel(const T* __restrict__ Up, const float* __res
 //   part[b, c] = sum_{t in strip b} w[t] * X[t, c]      (colsum_partial)
 //   out[c] (+)= sum_b part[b, c]                        (colsum_final)
 // Used for d w_sgate = sum_t dl[t] u_t (and, with w == NULL meaning all ones, for plain column sums).
-template <typename T>
+// V = 4: a thread takes four consecutive columns with one 8- or 16-byte load per row (cols and ldx multiples of 4,
+// X 16-byte aligned); V = 1: any shape.
+template <typename T, int V>
 __global__ void colsum_partial_kernel(const T* __restrict__ X, int64_t ldx, const float* __restrict__ w,
                                       int rows, int cols, int strip, float* __restrict__ part) {
-  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  int c = (blockIdx.x * blockDim.x + threadIdx.x) * V;
   int b = blockIdx.y;
   if (c >= cols) return;
   int t0 = b * strip, t1 = min(rows, t0 + strip);
-  float acc = 0.f;
+  float acc[V];
+#pragma unroll
+  for (int v = 0; v < V; ++v) acc[v] = 0.f;
 #pragma unroll 8
-  for (int t = t0; t < t1; ++t) acc += (w ? w[t] : 1.f) * to_f32(X[(int64_t)t * ldx + c]);
-  part[(int64_t)b * cols + c] = acc;
+  for (int t = t0; t < t1; ++t) {
+    const float wt = w ? w[t] : 1.f;
+    const T* px = X + (int64_t)t * ldx + c;
+    if constexpr (V == 4 && sizeof(T) == 2) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(px);
+      const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&raw);
+      const float2 a = __bfloat1622float2(hp[0]), b2 = __bfloat1622float2(hp[1]);
+      acc[0] += wt * a.x; acc[1] += wt * a.y; acc[2] += wt * b2.x; acc[3] += wt * b2.y;
+    } else if constexpr (V == 4) {
+      const float4 a = *reinterpret_cast<const float4*>(px);
+      acc[0] += wt * a.x; acc[1] += wt * a.y; acc[2] += wt * a.z; acc[3] += wt * a.w;
+    } else {
+      acc[0] += wt * to_f32(px[0]);
+    }
+  }
+#pragma unroll
+  for (int v = 0; v < V; ++v) part[(int64_t)b * cols + c + v] = acc[v];
+}
+
+template <typename T>
+inline cudaError_t launch_colsum_partial(const T* X, int64_t ldx, const float* w, int rows, int cols, int strip, int n_strips,
+                                         float* part, cudaStream_t st) {
+  if (cols % 4 == 0 && ldx % 4 == 0 && (reinterpret_cast<uintptr_t>(X) & 15u) == 0) {
+    dim3 grid((unsigned)ceil_div(cols, 4 * 128), (unsigned)n_strips);
+    colsum_partial_kernel<T, 4><<<grid, 128, 0, st>>>(X, ldx, w, rows, cols, strip, part);
+  } else {
+    dim3 grid((unsigned)ceil_div(cols, 256), (unsigned)n_strips);
+    colsum_partial_kernel<T, 1><<<grid, 256, 0, st>>>(X, ldx, w, rows, cols, strip, part);
+  }
+  return cudaGetLastError();
 }
 
 // Launch with COLSUM_FINAL_COLS columns per block of 256 threads: 8 threads share a column, each adds every 8th
@@ -242,18 +274,30 @@ __global__ void rmsnorm_bwd_rows_kernel(const float* __restrict__ dn, const floa
   }
 }
 
-// dgamma partials: part[b, c] = sum_{t in strip b} dn[t, c] * y[t, c] * r[t]
+// dgamma partials: part[b, c] = sum_{t in strip b} dn[t, c] * y[t, c] * r[t]; four columns per thread (h and ld are
+// multiples of 4, both arrays 16-byte aligned)
 __global__ void dgamma_partial_kernel(const float* __restrict__ dn, const float* __restrict__ y, int64_t ld,
                                       const float* __restrict__ r, int tokens, int h, int strip,
                                       float* __restrict__ part) {
-  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  int c = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   int b = blockIdx.y;
   if (c >= h) return;
   int t0 = b * strip, t1 = min(tokens, t0 + strip);
-  float acc = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 8
-  for (int t = t0; t < t1; ++t) acc += dn[(int64_t)t * h + c] * y[(int64_t)t * ld + c] * r[t];
-  part[(int64_t)b * h + c] = acc;
+  for (int t = t0; t < t1; ++t) {
+    const float4 a = *reinterpret_cast<const float4*>(dn + (int64_t)t * h + c);
+    const float4 v = *reinterpret_cast<const float4*>(y + (int64_t)t * ld + c);
+    const float rt = r[t];
+    acc.x += a.x * v.x * rt; acc.y += a.y * v.y * rt; acc.z += a.z * v.z * rt; acc.w += a.w * v.w * rt;
+  }
+  *reinterpret_cast<float4*>(part + (int64_t)b * h + c) = acc;
+}
+inline cudaError_t launch_dgamma_partial(const float* dn, const float* y, int64_t ld, const float* r, int tokens, int h, int strip,
+                                         int n_strips, float* part, cudaStream_t st) {
+  dim3 grid((unsigned)ceil_div(h, 4 * 128), (unsigned)n_strips);
+  dgamma_partial_kernel<<<grid, 128, 0, st>>>(dn, y, ld, r, tokens, h, strip, part);
+  return cudaGetLastError();
 }
 
 }  // namespace revffn

@@ -364,11 +364,9 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
   const int strip = STRIP;      // rows per partial sum of the two-pass column reductions
   auto colsum = [&](const T* X, int64_t ldx, int cols, float* out) -> int {
     const int strips = (int)ceil_div(Tn, strip);
-    dim3 grid((unsigned)ceil_div(cols, 256), (unsigned)strips);
     { ProfScope ps(TG_A_BIAS, st);
-    colsum_partial_kernel<T><<<grid, 256, 0, st>>>(X, ldx, nullptr, Tn, cols, strip, c.template p<float>(L.part));
+    CK(launch_colsum_partial<T>(X, ldx, nullptr, Tn, cols, strip, strips, c.template p<float>(L.part), st));
     }
-    CK(cudaGetLastError());
     { ProfScope ps(TG_A_BIAS, st);
     colsum_final_kernel<<<(unsigned)ceil_div(cols, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), strips, cols, acc, out);
     }
@@ -504,13 +502,11 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
   CK(cudaGetLastError());
   if (G.norm_gamma) {
     const int strips = (int)ceil_div(Tn, strip);
-    dim3 grid((unsigned)ceil_div(h, 256), (unsigned)strips);
     for (int side = 0; side < 2; ++side) {
       { ProfScope ps(TG_DGAMMA, st);
-      dgamma_partial_kernel<<<grid, 256, 0, st>>>(side ? dn2 : dn1, side ? x2 : x1, D.ld_stream, side ? r2 : r1, Tn, h, strip,
-                                                  c.template p<float>(L.part));
+      CK(launch_dgamma_partial(side ? dn2 : dn1, side ? x2 : x1, D.ld_stream, side ? r2 : r1, Tn, h, strip, strips,
+                               c.template p<float>(L.part), st));
       }
-      CK(cudaGetLastError());
       { ProfScope ps(TG_DGAMMA, st);
       colsum_final_kernel<<<(unsigned)ceil_div(h, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), strips, h,
                                                                       side ? 1 : acc, G.norm_gamma);

@@ -505,12 +505,10 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     if (G.ws_gate) CKR(wgrad(TG_WG_SH_GATE, G.ws_gate, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, 0, c.template p<T>(L.u), d, false, 0));
     if (G.ws_up) CKR(wgrad(TG_WG_SH_UP, G.ws_up, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, Is, c.template p<T>(L.u), d, false, 0));
     if (G.ws_sgate) {
-      dim3 grid((unsigned)ceil_div(d, 256), (unsigned)L.strips);
       { ProfScope ps(TG_WG_SGATE, st);
-      colsum_partial_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.u), d, c.template p<float>(L.dl), Tn, d, STRIP,
-                                                     c.template p<float>(L.part));
+      CK(launch_colsum_partial<T>(c.template p<T>(L.u), d, c.template p<float>(L.dl), Tn, d, STRIP, L.strips,
+                                  c.template p<float>(L.part), st));
       }
-      CK(cudaGetLastError());
       { ProfScope ps(TG_WG_SGATE, st);
       colsum_final_kernel<<<(unsigned)ceil_div(d, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), L.strips, d, acc,
                                                                       G.ws_sgate);
@@ -593,12 +591,10 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     if (G.w_router)
       CKR(wgrad(TG_WG_ROUTER, G.w_router, E, d, c.template p<T>(L.dlf), L.ld_dlf, 0, c.template p<T>(L.u), d, false, 0));
     if (G.b_router) {
-      dim3 grid((unsigned)ceil_div(E, 256), (unsigned)L.strips);
       { ProfScope ps(TG_WG_ROUTER, st);
-      colsum_partial_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.dlf), L.ld_dlf, nullptr, Tn, E, STRIP,
-                                                     c.template p<float>(L.part));
+      CK(launch_colsum_partial<T>(c.template p<T>(L.dlf), L.ld_dlf, nullptr, Tn, E, STRIP, L.strips,
+                                  c.template p<float>(L.part), st));
       }
-      CK(cudaGetLastError());
       { ProfScope ps(TG_WG_ROUTER, st);
       colsum_final_kernel<<<(unsigned)ceil_div(E, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), L.strips, E, acc,
                                                                       G.b_router);
@@ -636,12 +632,10 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     if (norm_none) {
       if (!acc) CK(cudaMemsetAsync(G.norm_gamma, 0, (size_t)h * 4, st));
     } else {
-      dim3 grid((unsigned)ceil_div(h, 256), (unsigned)L.strips);
       { ProfScope ps(TG_DGAMMA, st);
-      dgamma_partial_kernel<<<grid, 256, 0, st>>>(c.template p<float>(L.dn), y1, D.ld_stream, c.template p<float>(L.r),
-                                                  Tn, h, STRIP, c.template p<float>(L.part));
+      CK(launch_dgamma_partial(c.template p<float>(L.dn), y1, D.ld_stream, c.template p<float>(L.r), Tn, h, STRIP, L.strips,
+                               c.template p<float>(L.part), st));
       }
-      CK(cudaGetLastError());
       { ProfScope ps(TG_DGAMMA, st);
       colsum_final_kernel<<<(unsigned)ceil_div(h, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), L.strips, h, acc,
                                                                       G.norm_gamma);
