@@ -269,9 +269,8 @@ inline cudaError_t launch_fold_router_mma(const T* w_router, const T* w_sgate, c
 //            spent its time on shared-memory operand reads: 8 values per 16 FMAs.)
 //            The staging threads also sum y^2 (fp64), which gives
 //            r_t = (mean(y_t^2)+eps)^-1/2; the scale is applied to the finished sums.
-//   phase 2: per token the k largest logits (ties -> lowest index): up to 64 experts by rank counting on
-//            order-preserving integer keys, beyond that k rounds of warp arg-max by shuffles; then the softmax
-//            over the k selected logits and the sigmoid of the shared-gate logit.
+//   phase 2: per token, k rounds of warp arg-max (ties -> lowest index), softmax
+//            over the k selected logits, sigmoid of the shared-gate logit.
 // idx_in != NULL: expert sets are taken from it (gates are still recomputed).
 // prob_out != NULL: gates are the selected entries of the softmax over ALL experts (not
 // renormalised), and that softmax is written to prob_out[T, E].
@@ -301,10 +300,6 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
   double* ws = ns + RT_TOK * RT_LD;           // [RT_EC][RT_LD]   W_rc chunk, one row per expert
   double* rs = ws + RT_EC * RT_LD;            // [RT_TOK]
   double* Ls = rs + RT_TOK;                   // [RT_TOK][EP]
-  // per-warp scratch of the rank selection: keys [8][64], selected values [8][8] and indices [8][8]
-  unsigned long long* keys_all = reinterpret_cast<unsigned long long*>(Ls + (size_t)RT_TOK * (E + 1));
-  double* selv_all = reinterpret_cast<double*>(keys_all + 8 * 64);
-  int* selx_all = reinterpret_cast<int*>(selv_all + 8 * 8);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t0 = blockIdx.x * RT_TOK;
 
@@ -418,42 +413,6 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
 #pragma unroll
       for (int s = 0; s < 8; ++s)
         if (s < k) { seli[s] = idx_in[(int64_t)t * k + s]; sel[s] = L[seli[s]]; }
-    } else if (E <= 64) {
-      // Rank selection: every logit becomes a 64-bit key whose unsigned order is the logits' order (a total order,
-      // so the ranks are a permutation whatever the values), a lane counts for its one or two candidates the
-      // logits that beat them (larger, or equal with a lower index), and rank r < k is slot r.  No dependent
-      // chain of shuffles: the E comparisons of a candidate are independent.
-      unsigned long long* keys = keys_all + warp * 64;
-      double* selv = selv_all + warp * 8;
-      int* selx = selx_all + warp * 8;
-      unsigned long long kc[2];
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        const int e = lane + 32 * c;
-        kc[c] = 0ull;
-        if (e < E) {
-          const long long u = __double_as_longlong(L[e] + 0.0);     // + 0.0: -0 and +0 get one key
-          kc[c] = u < 0 ? ~(unsigned long long)u : ((unsigned long long)u | 0x8000000000000000ull);
-          keys[e] = kc[c];
-        }
-      }
-      __syncwarp();
-      int rank[2] = {0, 0};
-      for (int j = 0; j < E; ++j) {
-        const unsigned long long kj = keys[j];
-#pragma unroll
-        for (int c = 0; c < 2; ++c) rank[c] += (kj > kc[c] || (kj == kc[c] && j < lane + 32 * c)) ? 1 : 0;
-      }
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        const int e = lane + 32 * c;
-        if (e < E && rank[c] < k) { selv[rank[c]] = L[e]; selx[rank[c]] = e; }
-      }
-      __syncwarp();
-#pragma unroll
-      for (int s = 0; s < 8; ++s)
-        if (s < k) { sel[s] = selv[s]; seli[s] = selx[s]; }
-      __syncwarp();                             // the next token of this warp reuses the scratch
     } else {
       // candidates of this lane: e = lane + 32 j
       unsigned taken = 0u;                    // bit j set: candidate j already selected
@@ -526,7 +485,7 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
 }
 
 inline size_t router_smem_bytes(int E) {
-  return sizeof(double) * ((size_t)(RT_TOK + RT_EC) * RT_LD + RT_TOK + (size_t)RT_TOK * (E + 1)) + 8 * 64 * 8 + 8 * 8 * 8 + 8 * 8 * 4;
+  return sizeof(double) * ((size_t)(RT_TOK + RT_EC) * RT_LD + RT_TOK + (size_t)RT_TOK * (E + 1));
 }
 
 // Raises the kernel's dynamic shared-memory limit when the logits of a block do not
