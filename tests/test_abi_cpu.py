@@ -126,3 +126,21 @@ def test_attention_workspace_size_and_bad_descriptors(rv):
     with pytest.raises(rv.RevffnError) as e:
         rv.revffn_attn_workspace_size(_attn_desc(rv, flags=rv.FLAG_SAVE_ACTIVATIONS))
     assert e.value.code == -8
+
+
+def test_block_workspace_is_the_larger_branch_plus_one_stream(rv):
+    a = _attn_desc(rv)
+    m = _desc(rv)
+    d = rv.BlockDesc(a, m, 1)
+    fwd, bwd = rv.revffn_block_workspace_size(d)
+    af, ab = rv.revffn_attn_workspace_size(a)
+    mf, mb = rv.revffn_moe_workspace_size(m)
+    stream = 8192 * 1024 * 4
+    assert max(af, mf) + stream <= fwd <= max(af, mf) + stream + 4096
+    assert max(ab, mb) + stream <= bwd <= max(ab, mb) + stream + 4096
+    # the two halves of a block must describe the same tokens
+    for bad in (rv.BlockDesc(_attn_desc(rv, seq_len=1024), m, 1), rv.BlockDesc(_attn_desc(rv, d_model=1024, n_heads=8, n_kv_heads=8, ld_stream=512), m, 1),
+                rv.BlockDesc(a, _desc(rv, ld_stream=2048), 1), rv.BlockDesc(a, m, -1)):
+        with pytest.raises(rv.RevffnError) as e:
+            rv.revffn_block_workspace_size(bad)
+        assert e.value.code == -2
