@@ -731,7 +731,13 @@ def attn_flops(cfg):
     core = 2 * rows * S * hd            # one full (rows x S x hd) product
     return {"gemm_p_up": 2 * T * h * d, "gemm_qkv": 2 * T * d * (d + 2 * dkv) / 3, "gemm_scores": core, "gemm_pv": core,
             "gemm_w_o": 2 * T * d * d, "gemm_p_down_couple": 2 * T * d * h, "gemm_dp": core, "gemm_dk_dv": core,
-            "gemm_dq": core, "gemm_dn": 2 * (2 * T) * d * h}
+            "gemm_dq": core, "gemm_dn": 2 * (2 * T) * d * h,
+            # scopes that cover several launches: average per scope
+            "attn_wgrad": 2 * T * (h * d + 2 * d * d + 2 * dkv * d + 2 * d * h) / 6,
+            "attn_dgrad": 2 * T * (d * h + 2 * d * d + 2 * dkv * d) / 4,
+            # fused attention core, the causal half only: forward 2 products; gradient pass 7 (dK/dV 4, dQ 3)
+            "flash_attention": core,
+            "attn_bwd/flash_attention": (core + 3.5 * core) / 2}
 
 
 def run_attn(args, cfg):
@@ -757,7 +763,9 @@ def run_attn(args, cfg):
     def step():
         br.forward(x1, x2, y1)
         br.inverse(y1, x2, x1r, n_iter=1)
-        br.backward(x1r, x2, dy1, dx2, dx1=dx1, grads=grads)
+        # the gradient pass takes keys and values from the inverse pass before it (same x2), as a block's
+        # reversible back-propagation does
+        br.backward(x1r, x2, dy1, dx2, dx1=dx1, grads=grads, reuse_kv=True)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -824,14 +832,15 @@ def run_attn(args, cfg):
     passes = {}
     for ms, cnt, name, kn in kernels:
         passes[name.split("/")[0]] = passes.get(name.split("/")[0], 0.0) + ms / args.steps
+    fl = lambda name, kn: flops.get(name, flops.get(kn))
     top = [{"kernel": name, "ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps,
-            "tflops": (flops[kn] * cnt / (ms * 1e-3) / 1e12) if kn in flops and ms > 0 else None}
+            "tflops": (fl(name, kn) * cnt / (ms * 1e-3) / 1e12) if fl(name, kn) and ms > 0 else None}
            for ms, cnt, name, kn in kernels]
-    dom = next((k for k in kernels if k[3] in flops), None)
+    dom = next((k for k in kernels if fl(k[2], k[3])), None)
     roofline = None
     if dom:
         ms, cnt, name, kn = dom
-        achieved = flops[kn] / (ms / cnt * 1e-3) / 1e12
+        achieved = fl(name, kn) / (ms / cnt * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": name, "achieved": achieved, "peak": peak_t, "unit": "TFLOP/s",
                     "frac": achieved / peak_t, "peak_source": f"{peak_kind} (sustained bf16 cuBLAS figure)",
                     "traffic": None, "launch_ms": ms / cnt}
@@ -857,7 +866,7 @@ def run_attn(args, cfg):
         "config": {"workload": f"{cfg.name}: attention coupling branch of one Qwen1.5-MoE-A2.7B-shaped block, "
                                f"{cfg.batch} sequences x {cfg.seq_len} positions per GPU, d={cfg.d_model}, "
                                f"{cfg.n_heads} heads ({cfg.n_kv_heads} key/value heads) of {cfg.head_dim}; step = forward + "
-                               f"inverse (one fixed-point iteration) + backward by recomputation, all weight gradients in fp32",
+                               f"inverse (one fixed-point iteration) + backward by recomputation (keys and values shared with the inverse pass), all weight gradients in fp32",
                    "l2": "per-step working set (score matrices alone 1 GB) exceeds the 126 MB L2",
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},
         "passes_ms": passes, "kernels": top, "roofline": roofline, "cpu_baseline": cpu_rec,

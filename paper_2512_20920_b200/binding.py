@@ -433,7 +433,8 @@ class AttnBranch:
         return x1
 
     def backward(self, x1, x2, dy1, dx2_inout, dx1=None, grads: Optional[Dict[str, torch.Tensor]] = None,
-                 accumulate: bool = False):
+                 accumulate: bool = False, reuse_kv: bool = False):
+        """reuse_kv=True: the workspace still holds the key/value side that inverse(n_iter >= 1) left for this x2."""
         grads = grads or {}
         for n, t in grads.items():
             if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
@@ -441,7 +442,12 @@ class AttnBranch:
         if dx1 is None:
             dx1 = torch.empty_like(dy1)
         g = AttnGrads(**{n: _ptr(grads.get(n)) for n in ATTN_WEIGHT_NAMES}, accumulate=1 if accumulate else 0)
-        revffn_attn_backward(self.desc, self.w, x1, x2, dy1, dx1, dx2_inout, g, self.ws)
+        d = self.desc
+        if reuse_kv:
+            d = AttnDesc()
+            C.memmove(C.byref(d), C.byref(self.desc), C.sizeof(AttnDesc))
+            d.flags |= FLAG_REUSE_ACTIVATIONS
+        revffn_attn_backward(d, self.w, x1, x2, dy1, dx1, dx2_inout, g, self.ws)
         return dx1
 
     def status(self) -> int:

@@ -142,8 +142,6 @@ def test_strided_streams_and_bad_arguments():
 def test_backward_reuses_the_key_value_side_of_the_inverse_pass():
     """Reversible back-propagation runs a block's inverse pass right before its gradient pass; with the
     reuse flag the gradient pass takes keys and values from the workspace.  Same arithmetic, same bits."""
-    import ctypes as C
-    import paper_2512_20920_b200 as rv
     cfg = AttnConfig("r", batch=2, seq_len=200, d_model=256, n_heads=2, n_kv_heads=1, weight_dtype="bf16")
     w = make_attn_weights(cfg, 4, std=0.05, bias_std=0.05)
     s = make_attn_streams(cfg, 4)
@@ -157,12 +155,7 @@ def test_backward_reuses_the_key_value_side_of_the_inverse_pass():
     dx1_a = br.backward(x1, x2, dy1, dx2_a, grads=g_a)
     # inverse pass (leaves keys and values behind), then the gradient pass at the same x1 with the flag
     br.inverse(y1, x2, n_iter=1)
-    d = rv.AttnDesc()
-    C.memmove(C.byref(d), C.byref(br.desc), C.sizeof(rv.AttnDesc))
-    d.flags |= rv.FLAG_REUSE_ACTIVATIONS
-    ga = rv.AttnGrads(**{n: (g_b[n].data_ptr() if n in g_b else None) for n in rv.binding.ATTN_WEIGHT_NAMES}, accumulate=0)
-    dx1_b = torch.empty_like(dy1)
-    rv.revffn_attn_backward(d, br.w, x1, x2, dy1, dx1_b, dx2_b, ga, br.ws)
+    dx1_b = br.backward(x1, x2, dy1, dx2_b, grads=g_b, reuse_kv=True)
     assert br.status() == 0
     assert torch.equal(dx1_a, dx1_b) and torch.equal(dx2_a, dx2_b)
     for n in names:
