@@ -31,7 +31,7 @@
 
 namespace revffn {
 
-enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_ROWSCALE = 2, EPI_COUPLE = 3, EPI_DSWIGLU = 4, EPI_WGRAD = 5 };
+enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_ROWSCALE = 2, EPI_COUPLE = 3, EPI_DSWIGLU = 4, EPI_WGRAD = 5, EPI_HEADS = 6 };
 enum { CONCAT_NONE = 0, CONCAT_N = 1, CONCAT_K = 2 };
 enum { GROUP_NONE = 0, GROUP_M = 1, GROUP_K = 2 };
 
@@ -57,6 +57,10 @@ struct GemmProblem {
   int64_t b_group_stride, c_group_stride;
   int a_col0, b_col0;
   int no_pair;        // tcgen05 back end: never pair CTAs for this product
+  // EPI_HEADS (tcgen05 back end, dense products only): the N columns are heads of 128; C receives, head-major
+  // [sequence, head, hm_Sp, 128], the product plus hm_bias, with the pairs (i, i + 64) of a head turned by the
+  // angle of hm_cs[position, i] (cos, sin) when hm_cs is given.  Row m is position m % hm_S of sequence m / hm_S.
+  const float* hm_bias; const float2* hm_cs; int hm_S, hm_Sp;
   int* status;
 };
 

@@ -694,6 +694,49 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             ++n_grp;
           }
         }
+      } else if constexpr (EPI == EPI_HEADS) {
+        // Columns are heads of 128: the tile holds two (or, ragged, one).  This warp's 32-column blocks c and c + 64
+        // are the two halves of a rotated pair range: bias, rotation by the position's angles, bf16, and out as
+        // 64-byte pieces of the row's place in the head-major tensor.
+        uint32_t r1[32];
+        const int seq = m_ok ? m / p.hm_S : 0, pos = m_ok ? m % p.hm_S : 0;
+        const int n_heads = p.N / 128;
+#pragma unroll 1
+        for (int c = half * 32; c < t.ncols; c += 128) {
+          if (!slab_ok) continue;      // warp-uniform
+          const int n = t.n0 + c;      // first column of the lower half-range; n + 64 is its partner
+          tmem_ld32(taddr + c, r0);
+          tmem_ld32(taddr + c + 64, r1);
+          tmem_ld_wait();
+          if (!m_ok) continue;
+          const int head = n / 128, i0 = n % 128;            // i0 is 0 or 32
+          bf16* dst = reinterpret_cast<bf16*>(p.C) + (((int64_t)seq * n_heads + head) * p.hm_Sp + pos) * 128 + i0;
+          float y0[32], y1[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) { y0[i] = __uint_as_float(r0[i]); y1[i] = __uint_as_float(r1[i]); }
+          if (p.hm_bias) {
+            const float4* b0 = reinterpret_cast<const float4*>(p.hm_bias + n);        // the same for every lane
+            const float4* b1 = reinterpret_cast<const float4*>(p.hm_bias + n + 64);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float4 u = b0[i], v = b1[i];
+              y0[4 * i] += u.x; y0[4 * i + 1] += u.y; y0[4 * i + 2] += u.z; y0[4 * i + 3] += u.w;
+              y1[4 * i] += v.x; y1[4 * i + 1] += v.y; y1[4 * i + 2] += v.z; y1[4 * i + 3] += v.w;
+            }
+          }
+          if (p.hm_cs) {
+            const float4* cs2 = reinterpret_cast<const float4*>(p.hm_cs + pos * 64 + i0);   // two (cos, sin) pairs per load
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float4 cs = cs2[i];
+              const float a0 = y0[2 * i], b0v = y1[2 * i], a1 = y0[2 * i + 1], b1v = y1[2 * i + 1];
+              y0[2 * i] = a0 * cs.x - b0v * cs.y;         y1[2 * i] = b0v * cs.x + a0 * cs.y;
+              y0[2 * i + 1] = a1 * cs.z - b1v * cs.w;     y1[2 * i + 1] = b1v * cs.z + a1 * cs.w;
+            }
+          }
+          store32_bf16(dst, y0);
+          store32_bf16(dst + 64, y1);
+        }
       } else if constexpr (EPI == EPI_SWIGLU) {
         // columns [0, MMA_N/2) hold the gate projection, [MMA_N/2, MMA_N) the up projection.
         // H goes out through two alternating 2 KB staging buffers; when the a|b copy is wanted too,
@@ -896,6 +939,7 @@ inline int tc_prepare() {
   if (e == cudaSuccess) e = tc_set_attr<256, EPI_COUPLE>();
   if (e == cudaSuccess) e = tc_set_attr<256, EPI_DSWIGLU>();
   if (e == cudaSuccess) e = tc_set_attr<256, EPI_WGRAD>();
+  if (e == cudaSuccess) e = tc_set_attr<256, EPI_HEADS>();
   if (e != cudaSuccess) return REVFFN_ERR_CUDA;
   s.ready = true;
   return REVFFN_OK;
@@ -1003,7 +1047,11 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   CUtensorMap mc, mc1;
   memset(&mc, 0, sizeof(mc));
   memset(&mc1, 0, sizeof(mc1));
-  if (p.epilogue == EPI_DSWIGLU) {
+  if (p.epilogue == EPI_HEADS) {
+    // plain stores into the head-major tensor, no output map
+    if (p.group_mode != 0 || p.N % 128 != 0 || p.hm_S <= 0 || p.hm_Sp < p.hm_S || (reinterpret_cast<uintptr_t>(p.C) & 15u))
+      return REVFFN_ERR_SHAPE;
+  } else if (p.epilogue == EPI_DSWIGLU) {
     // a|b are loaded and written back in place through one map; g*H (optional) through the other
     if ((reinterpret_cast<uintptr_t>(p.ab) & 15u) || (p.ld_ab * 2) % 16 != 0) return REVFFN_ERR_ALIGN;
     int r = tc_make_out_map(&mc, p.ab, false, (uint64_t)2 * p.N, (uint64_t)p.M, (uint64_t)p.ld_ab);
@@ -1056,7 +1104,7 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
 #define TC_CASE(N_, E_) \
   if (mma_n == N_ && p.epilogue == E_) return tc_launch<N_, E_>(P, ma, mb0, mb1, mc, mc1, grid, pair, st);
   TC_CASE(256, EPI_STORE) TC_CASE(256, EPI_SWIGLU) TC_CASE(256, EPI_ROWSCALE) TC_CASE(256, EPI_COUPLE)
-  TC_CASE(256, EPI_DSWIGLU) TC_CASE(256, EPI_WGRAD)
+  TC_CASE(256, EPI_DSWIGLU) TC_CASE(256, EPI_WGRAD) TC_CASE(256, EPI_HEADS)
 #undef TC_CASE
   return REVFFN_ERR_UNSUPPORTED;
 }

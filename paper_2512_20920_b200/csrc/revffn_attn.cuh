@@ -185,6 +185,14 @@ static int a_project(const ACtx<T>& c, int side, const void* W, const float* bia
   p.M = Tn; p.N = n * L.hd; p.K = d;
   p.A = c.template p<T>(L.u12) + (int64_t)side * Tn * d; p.lda = d;
   p.B0 = W; p.ldb = d;
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (c.tc && L.hd == 128) {
+      // bias, rotation and the head-major layout happen in the product's epilogue: no fp32 round trip
+      p.epilogue = EPI_HEADS; p.C = heads;
+      p.hm_bias = bias; p.hm_cs = rotate ? c.template p<float2>(L.cs) : nullptr; p.hm_S = D.seq_len; p.hm_Sp = L.Sp;
+      return a_gemm(c, p, TG_A_QKV);
+    }
+  }
   p.epilogue = EPI_STORE; p.out_f32 = 1; p.C = c.template p<float>(L.raw); p.ldc = n * L.hd;
   CKR(a_gemm(c, p, TG_A_QKV));
   { ProfScope ps(TG_A_HEADS, c.st);
