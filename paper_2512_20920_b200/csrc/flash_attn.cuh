@@ -433,8 +433,13 @@ struct FlashBwdParams {
   int S, Sp, n_heads, rep;
   const float2* lse_d;            // per query row (head-major index): (lse * log2 e, D * scale)
   const bf16* x0; const bf16* x1; // !DKV: the owned operands (q, d_o head-major), read by the CTA's threads themselves
-  float* out0;                    // DKV: dV [kv rows, 128] fp32
-  float* out1;                    // DKV: dK [kv rows, 128];  else dQ [q rows, 128]
+  // Outputs, token-major bf16 [T, ld_out]: a row's head lands at column col + head * 128.  out0: dV (DKV only, as it
+  // is); out1: dK (DKV) or dQ, with the rotation of the forward pass undone (its transpose), pairs (i, i + 64).
+  bf16* out0; bf16* out1;
+  int64_t ld_out0, ld_out1;
+  int col0, col1;
+  int heads_own;                  // heads per sequence on the owned side (key/value heads for DKV, query heads else)
+  const float2* cs;               // [S, 64] (cos, sin)
   float scale_log2e, scale;
   int* status;
 };
@@ -634,6 +639,7 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
     const int own_pos = blk * FA_BLK + row;      // position in the sequence of this thread's own row
     float2 own_ld = make_float2(0.f, 0.f);
     if (!DKV && own_pos < P.S) own_ld = P.lse_d[own_row0 + row];
+    __syncwarp();
     if (!DKV) {
       // The owned operands never change: each thread puts its row's 64 columns of both into tensor memory
       // (TMEM columns 256.. for X0, 320.. for X1), where every step's products read them as the A operand.
@@ -694,19 +700,37 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
     if (ok && !mbar_wait(bar(B_ACCFULL), 0u, abort_flag, P.status)) ok = false;
     if (ok) {
       tc_fence_after();
+      // This thread takes columns [32 hh, +32) and their rotation partners [64 + 32 hh, +32) of its row.  The
+      // tensor-memory loads are warp-wide instructions: every lane executes them, rows past the sequence only
+      // skip the stores.
+      const bool row_ok = own_pos < P.S;
+      const int seq = grp / P.heads_own, head = grp % P.heads_own;
+      const int64_t tok = (int64_t)seq * P.S + (row_ok ? own_pos : 0);
+      {
 #pragma unroll
-      for (int a = DKV ? 0 : 1; a < 2; ++a) {
-        float* dst = (a == 0 ? P.out0 : P.out1) + (int64_t)(own_row0 + row) * FA_HD + 64 * (warp >= 6 ? 1 : 0);
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t r[32];
-          tmem_ld32(lane_addr + (uint32_t)(256 + 128 * a + 64 * (warp >= 6 ? 1 : 0) + 32 * c), r);
+        for (int a = DKV ? 0 : 1; a < 2; ++a) {
+          uint32_t rl[32], rh[32];
+          __syncwarp();               // lanes that skipped the previous output rejoin before the warp-wide loads
+          tmem_ld32(lane_addr + (uint32_t)(256 + 128 * a + 32 * hh), rl);
+          tmem_ld32(lane_addr + (uint32_t)(256 + 128 * a + 64 + 32 * hh), rh);
           tmem_ld_wait();
+          if (!row_ok) continue;
+          float y0[32], y1[32];
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            *reinterpret_cast<float4*>(dst + 32 * c + 4 * i) =
-                make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),
-                            __uint_as_float(r[4 * i + 3]));
+          for (int i = 0; i < 32; ++i) { y0[i] = __uint_as_float(rl[i]); y1[i] = __uint_as_float(rh[i]); }
+          if (a == 1) {
+            const float4* cs2 = reinterpret_cast<const float4*>(P.cs + own_pos * 64 + 32 * hh);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float4 cs = cs2[i];
+              const float a0 = y0[2 * i], b0 = y1[2 * i], a1 = y0[2 * i + 1], b1 = y1[2 * i + 1];
+              y0[2 * i] = a0 * cs.x + b0 * cs.y;         y1[2 * i] = b0 * cs.x - a0 * cs.y;
+              y0[2 * i + 1] = a1 * cs.z + b1 * cs.w;     y1[2 * i + 1] = b1 * cs.z - a1 * cs.w;
+            }
+          }
+          bf16* dst = (a == 0 ? P.out0 + tok * P.ld_out0 + P.col0 : P.out1 + tok * P.ld_out1 + P.col1) + head * FA_HD + 32 * hh;
+          store32_bf16(dst, y0);
+          store32_bf16(dst + 64, y1);
         }
       }
     }
@@ -746,10 +770,10 @@ __global__ void attn_rowdot_kernel(const float* __restrict__ o32, const bf16* __
 }
 
 // q, d_o: [B * n_heads * Sp, 128]; k, v: [B * n_kv_heads * Sp, 128] bf16 head-major (rows past the sequence zero).
-// dq: [B * n_heads * Sp, 128], dk, dv: [B * n_kv_heads * Sp, 128] fp32, every row written.
-inline int launch_flash_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* d_o, const float2* lse_d, int batch,
-                            int n_heads, int n_kv_heads, int S, int Sp, float* dq, float* dk, float* dv, int* status,
-                            cudaStream_t st) {
+// Outputs token-major bf16, rotation undone: dq [T, ld_dq]; dk at column 0 and dv at column dv_col of dkv [T, ld_dkv].
+inline int launch_flash_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* d_o, const float2* lse_d, const float2* cs,
+                            int batch, int n_heads, int n_kv_heads, int S, int Sp, bf16* dq, int64_t ld_dq, bf16* dkv,
+                            int64_t ld_dkv, int dv_col, int* status, cudaStream_t st) {
   TcState& s = tc_state();
   if (!s.ready) return REVFFN_ERR_CUDA;
   if (batch <= 0) return REVFFN_OK;
@@ -780,11 +804,16 @@ inline int launch_flash_bwd(const bf16* q, const bf16* k, const bf16* v, const b
   P.scale = 1.f / sqrtf((float)FA_HD);
   P.scale_log2e = P.scale * 1.4426950408889634f;
   P.status = status;
-  P.out0 = dv; P.out1 = dk;
+  P.cs = cs;
+  P.out0 = dkv; P.ld_out0 = ld_dkv; P.col0 = dv_col;
+  P.out1 = dkv; P.ld_out1 = ld_dkv; P.col1 = 0;
+  P.heads_own = n_kv_heads;
   P.x0 = nullptr; P.x1 = nullptr;
   flash_bwd_kernel<true><<<batch * n_kv_heads * (Sp / FA_BLK), FA_THREADS, FB_SMEM_BYTES, st>>>(P, k128, v128, q64, do64);
   if (cudaGetLastError() != cudaSuccess) return REVFFN_ERR_CUDA;
-  P.out0 = nullptr; P.out1 = dq;
+  P.out0 = nullptr; P.ld_out0 = 0; P.col0 = 0;
+  P.out1 = dq; P.ld_out1 = ld_dq; P.col1 = 0;
+  P.heads_own = n_heads;
   P.x0 = q; P.x1 = d_o;
   flash_bwd_kernel<false><<<batch * n_heads * (Sp / FA_BLK), FA_THREADS, FB_SMEM_BYTES, st>>>(P, q128, do128, k64, v64);
   return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;

@@ -705,6 +705,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         for (int c = half * 32; c < t.ncols; c += 128) {
           if (!slab_ok) continue;      // warp-uniform
           const int n = t.n0 + c;      // first column of the lower half-range; n + 64 is its partner
+          __syncwarp();                // lanes past the last row skipped the previous block's stores: rejoin before the warp-wide loads
           tmem_ld32(taddr + c, r0);
           tmem_ld32(taddr + c + 64, r1);
           tmem_ld_wait();

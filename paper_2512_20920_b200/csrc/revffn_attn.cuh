@@ -391,10 +391,19 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
   if (G.w_down) CKR(wgrad(G.w_down, h, d, c.template p<T>(L.dyb), h, 0, c.template p<T>(L.a), d, Tn, acc));
   CKR(dgrad(TG_A_DGRAD, Tn, d, h, c.template p<T>(L.dyb), h, c.W.w_down, d, c.template p<T>(L.da), false));
   if (G.w_o) CKR(wgrad(G.w_o, d, d, c.template p<T>(L.da), d, 0, c.template p<T>(L.o), d, Tn, acc));
-  CKR(dgrad(TG_A_DGRAD, Tn, d, d, c.template p<T>(L.da), d, c.W.w_o, d, c.template p<T>(L.dob), false));
-  { ProfScope ps(TG_A_HEADS, st);
-  CK((launch_to_heads<T, T>(c.template p<T>(L.dob), d, nullptr, nullptr, Tn, D.seq_len, Sp, D.n_heads, hd,
-                            c.template p<T>(L.doh), st)));
+  if (fused) {
+    GemmProblem p = blank_problem();   // dO = da W_o, written head-major by the product's epilogue
+    p.M = Tn; p.N = d; p.K = d;
+    p.A = c.template p<T>(L.da); p.lda = d;
+    p.B0 = c.W.w_o; p.ldb = d; p.b_mn_major = 1;
+    p.epilogue = EPI_HEADS; p.C = c.template p<T>(L.doh); p.hm_S = D.seq_len; p.hm_Sp = Sp;
+    CKR(a_gemm(c, p, TG_A_DGRAD));
+  } else {
+    CKR(dgrad(TG_A_DGRAD, Tn, d, d, c.template p<T>(L.da), d, c.W.w_o, d, c.template p<T>(L.dob), false));
+    { ProfScope ps(TG_A_HEADS, st);
+    CK((launch_to_heads<T, T>(c.template p<T>(L.dob), d, nullptr, nullptr, Tn, D.seq_len, Sp, D.n_heads, hd,
+                              c.template p<T>(L.doh), st)));
+    }
   }
 
   // attention core backward
@@ -407,10 +416,11 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
       }
       CK(cudaGetLastError());
       { ProfScope ps(TG_A_FLASH, st);
+      // the two launches also undo the rotation and write dq and dk|dv token-major in the operand type
       CKR(launch_flash_bwd(c.template p<bf16>(L.qh), c.template p<bf16>(L.kh), c.template p<bf16>(L.vh),
-                           c.template p<bf16>(L.doh), c.template p<float2>(L.lse_d), D.batch, D.n_heads, D.n_kv_heads,
-                           D.seq_len, Sp, c.template p<float>(L.dqh), c.template p<float>(L.dkh), c.template p<float>(L.dvh),
-                           c.template p<int>(L.status), st));
+                           c.template p<bf16>(L.doh), c.template p<float2>(L.lse_d), c.template p<float2>(L.cs), D.batch,
+                           D.n_heads, D.n_kv_heads, D.seq_len, Sp, c.template p<bf16>(L.dq), d, c.template p<bf16>(L.dkv),
+                           2 * (int64_t)dkv, dkv, c.template p<int>(L.status), st));
       ++g_prof.launches;
       }
     }
@@ -450,18 +460,20 @@ static int a_backward(const ACtx<T>& c, const float* x1, const float* x2, const 
       CKR(a_gemm(c, p, TG_A_DQ));
     }
   }
-  // back to token-major; the rotation is undone by its transpose
-  { ProfScope ps(TG_A_HEADS, st);
-  CK((launch_from_heads<float, T>(c.template p<float>(L.dqh), c.template p<float2>(L.cs), -1.f, Tn, D.seq_len, Sp,
-                                  D.n_heads, hd, c.template p<T>(L.dq), d, 0, st)));
-  }
-  { ProfScope ps(TG_A_HEADS, st);
-  CK((launch_from_heads<float, T>(c.template p<float>(L.dkh), c.template p<float2>(L.cs), -1.f, Tn, D.seq_len, Sp,
-                                  D.n_kv_heads, hd, c.template p<T>(L.dkv), 2 * (int64_t)dkv, 0, st)));
-  }
-  { ProfScope ps(TG_A_HEADS, st);
-  CK((launch_from_heads<float, T>(c.template p<float>(L.dvh), nullptr, 1.f, Tn, D.seq_len, Sp, D.n_kv_heads, hd,
-                                  c.template p<T>(L.dkv), 2 * (int64_t)dkv, dkv, st)));
+  if (!fused) {
+    // back to token-major; the rotation is undone by its transpose
+    { ProfScope ps(TG_A_HEADS, st);
+    CK((launch_from_heads<float, T>(c.template p<float>(L.dqh), c.template p<float2>(L.cs), -1.f, Tn, D.seq_len, Sp,
+                                    D.n_heads, hd, c.template p<T>(L.dq), d, 0, st)));
+    }
+    { ProfScope ps(TG_A_HEADS, st);
+    CK((launch_from_heads<float, T>(c.template p<float>(L.dkh), c.template p<float2>(L.cs), -1.f, Tn, D.seq_len, Sp,
+                                    D.n_kv_heads, hd, c.template p<T>(L.dkv), 2 * (int64_t)dkv, 0, st)));
+    }
+    { ProfScope ps(TG_A_HEADS, st);
+    CK((launch_from_heads<float, T>(c.template p<float>(L.dvh), nullptr, 1.f, Tn, D.seq_len, Sp, D.n_kv_heads, hd,
+                                    c.template p<T>(L.dkv), 2 * (int64_t)dkv, dkv, st)));
+    }
   }
 
   // q/k/v projections backward
