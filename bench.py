@@ -904,6 +904,8 @@ def main():
         return run_block_stack(args, ATTN_CONFIGS["A1"], CONFIGS["C1"], 24 if args.config == "B3" else 1)
     if args.config in ATTN_CONFIGS and args.impl == "ours":
         return run_attn(args, ATTN_CONFIGS[args.config])
+    if args.impl == "reference" and args.config not in CONFIGS:
+        args.config = "C1"          # the reference arm times the oracle of the headline path only
     if args.config == "C4":
         if args.impl == "reference":
             args.config = "C1"
