@@ -26,6 +26,36 @@ __global__ void rope_table_kernel(int S, int hd, double theta, float2* __restric
   cs[idx] = make_float2((float)c, (float)sn);
 }
 
+// RMSNorm of both streams in one launch: warp w < tokens normalises row w of x1, the others row w - tokens of x2;
+// output rows in that order (the layout the shared P_up product reads).  Same arithmetic as rmsnorm_fwd_kernel.
+template <typename T>
+__global__ void rmsnorm2_fwd_kernel(const float* __restrict__ x1, const float* __restrict__ x2, int64_t ld,
+                                    const float* __restrict__ gamma, float eps, int tokens, int h, T* __restrict__ n_out,
+                                    float* __restrict__ r_out) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (warp >= 2 * tokens) return;
+  const float* row = warp < tokens ? x1 + (int64_t)warp * ld : x2 + (int64_t)(warp - tokens) * ld;
+  float ss = 0.f;
+  for (int i = lane * 4; i < h; i += 128) {
+    float4 v = *reinterpret_cast<const float4*>(row + i);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = warp_sum(ss);
+  const float r = rsqrtf(ss / (float)h + eps);
+  if (lane == 0) r_out[warp] = r;
+  T* out = n_out + (int64_t)warp * h;
+  for (int i = lane * 4; i < h; i += 128) {
+    float4 v = *reinterpret_cast<const float4*>(row + i);
+    float4 g = make_float4(1.f, 1.f, 1.f, 1.f);
+    if (gamma) g = *reinterpret_cast<const float4*>(gamma + i);
+    out[i + 0] = from_f32<T>(v.x * r * g.x);
+    out[i + 1] = from_f32<T>(v.y * r * g.y);
+    out[i + 2] = from_f32<T>(v.z * r * g.z);
+    out[i + 3] = from_f32<T>(v.w * r * g.w);
+  }
+}
+
 // One block per token.  in: [T, ld_in] with n heads of hd columns; out: [B, n, S_pad, hd].
 template <typename TIn, typename T>
 __global__ void to_heads_kernel(const TIn* __restrict__ in, int64_t ld_in, const float* __restrict__ bias,

@@ -296,11 +296,30 @@ static int a_query_side(const ACtx<T>& c, const float* x1, bool need_p, bool kee
   return a_wo(c);
 }
 
+// Forward pass: both streams are known at once, so the norm and P_up run over the 2T rows together.
 template <typename T>
 static int a_forward(const ACtx<T>& c, const float* x1, const float* x2, float* y1) {
+  const revffn_attn_desc& D = c.D;
+  const AttnLayout& L = c.L;
   CKR(a_setup(c, false));
-  CKR(a_kv_side(c, x2));
-  CKR(a_query_side(c, x1, false));
+  { ProfScope ps(TG_NORM, c.st);
+  rmsnorm2_fwd_kernel<T><<<(unsigned)ceil_div((int64_t)2 * L.T * 32, 128), 128, 0, c.st>>>(
+      x1, x2, D.ld_stream, c.W.norm_gamma, D.norm_eps, L.T, L.h, c.template p<T>(L.n12), c.template p<float>(L.r12));
+  }
+  CK(cudaGetLastError());
+  {
+    GemmProblem p = blank_problem();
+    p.M = 2 * L.T; p.N = D.d_model; p.K = L.h;
+    p.A = c.template p<T>(L.n12); p.lda = L.h;
+    p.B0 = c.W.w_up; p.ldb = L.h;
+    p.epilogue = EPI_STORE; p.C = c.template p<T>(L.u12); p.ldc = D.d_model;
+    CKR(a_gemm(c, p, TG_PUP));
+  }
+  CKR(a_project(c, 1, c.W.w_k, c.W.b_k, D.n_kv_heads, true, c.template p<T>(L.kh)));
+  CKR(a_project(c, 1, c.W.w_v, c.W.b_v, D.n_kv_heads, false, c.template p<T>(L.vh)));
+  CKR(a_project(c, 0, c.W.w_q, c.W.b_q, D.n_heads, true, c.template p<T>(L.qh)));
+  CKR(a_core(c, false));
+  CKR(a_wo(c));
   return a_couple(c, x1, 1.f, y1);
 }
 
