@@ -395,50 +395,45 @@ inline int launch_flash_fwd(const bf16* q, const bf16* k, const bf16* v, int bat
 }
 
 // ---------------------------------------------------------------------------
+// ---------------------------------------------------------------------------
 // Backward of the attention core, also without a score matrix in HBM.  P is rebuilt from the row
 // log-sum-exp the forward kernel stored:  P = exp(scale * S - lse),  dS = scale * P * (dP - D) with
-// D = <dO_row, O_row>.  Two launches of one kernel template, neither uses atomics:
-//   DKV = true   a CTA owns 128 keys of one key/value head and walks the 64-row query tiles at or
-//                below them (of every query head of the group):  dV += P^T dO,  dK += dS^T Q
-//   DKV = false  a CTA owns 128 query rows of one head and walks the 64-key tiles up to its diagonal:
-//                dQ += dS K
-// Per step the "own" side is the MMA M side and the walked tile the N side, so both cases compute
-//   S' = X0 Y0^T,  dP' = X1 Y1^T   (128 x 64, K = hd; X = own operands, Y = the walked tiles)
-// into TMEM (double-buffered), eight warps (two threads per own row, 32 columns each) turn them into P' and
+// D = <dO_row, O_row>.  Two kernels, neither uses atomics:
+//   flash_bwd_dkv_kernel  a CTA owns 128 keys of one key/value head and walks the 64-row query tiles at or
+//                         below them (of every query head of the group):  dV += P^T dO,  dK += dS^T Q
+//   flash_bwd_dq_kernel   a CTA owns 128 query rows of one head and walks the 128-key tiles up to its diagonal:
+//                         dQ += dS K
+// In both the "own" side is the MMA M side and the walked tile the N side.  dK/dV, per step:
+//   S' = K_j Q_t^T,  dP' = V_j dO_t^T   (128 x 64, K = hd)
+// into TMEM (double-buffered), eight warps (two threads per key row, 32 query columns each) turn them into P' and
 // dS' as bf16 K-major operand tiles in shared memory, and the accumulators (fresh TMEM columns, summed over
-// all steps by the tensor core itself) take  acc0 += P' Y1  (DKV only)  and  acc1 += dS' Y0,  where the same
-// shared-memory bytes of a Y tile that served as a K-major operand are read again as an MN-major one.
-// The dQ launch has TMEM columns to spare and keeps its owned operands there (A operand from tensor memory),
-// which takes two thirds of the shared-memory reads out of its steps.
+// all steps by the tensor core itself) take  dV += P' dO_t  and  dK += dS' Q_t,  where the same shared-memory
+// bytes of a walked tile that served as a K-major operand are read again as an MN-major one.
 // No cross-thread reduction is needed: the row statistics come from memory.
 // ---------------------------------------------------------------------------
-// Shared memory.  DKV: [X0, X1 64 KB | 3 stages of walked tiles 96 KB]; else (owned operands in tensor memory):
-// [5 stages 160 KB]; then in both: P' tile 16 KB, dS' tile 16 KB, barriers, row statistics of the stages.
-// A stage: [Y0 2 x 8 KB | Y1 2 x 8 KB].  The walked tiles come from L2 with a latency of more than one step,
-// hence the deep ring.
+// Shared memory of the dK/dV kernel: [K_j, V_j 64 KB | 3 stages of walked tiles 96 KB | P' tile 16 KB | dS' tile
+// 16 KB | barriers | row statistics of the stages].  A stage: [Q_t 2 x 8 KB | dO_t 2 x 8 KB].  The walked tiles
+// come from L2 with a latency of more than one step, hence the ring of three.
 constexpr int FB_X_OFF = 0;
 constexpr int FB_STAGE = 2 * FA_TILE;
-template <bool DKV> struct FbCfg {
-  static constexpr int NS = DKV ? 3 : 5;
-  static constexpr int Y_OFF = DKV ? 4 * FA_TILE : 0;
-};
-constexpr int FB_P_OFF = 10 * FA_TILE;
+constexpr int FB_NS = 3;
+constexpr int FB_Y_OFF = 4 * FA_TILE;
+constexpr int FB_P_OFF = FB_Y_OFF + FB_NS * FB_STAGE;
 constexpr int FB_DS_OFF = FB_P_OFF + FA_TILE;
 constexpr int FB_BAR_OFF = FB_DS_OFF + FA_TILE;
-constexpr int FB_LD_OFF = FB_BAR_OFF + 256;        // DKV: (lse * log2 e, D * scale) of a stage's 64 query rows, 512 B per stage
+constexpr int FB_LD_OFF = FB_BAR_OFF + 256;        // (lse * log2 e, D * scale) of a stage's 64 query rows, 512 B per stage
 constexpr int FB_SMEM_BYTES = FB_LD_OFF + 2048 + 1024;
-constexpr int FB_MAX_NS = 5;
 
 struct FlashBwdParams {
   int S, Sp, n_heads, rep;
   const float2* lse_d;            // per query row (head-major index): (lse * log2 e, D * scale)
-  const bf16* x0; const bf16* x1; // !DKV: the owned operands (q, d_o head-major), read by the CTA's threads themselves
-  // Outputs, token-major bf16 [T, ld_out]: a row's head lands at column col + head * 128.  out0: dV (DKV only, as it
-  // is); out1: dK (DKV) or dQ, with the rotation of the forward pass undone (its transpose), pairs (i, i + 64).
+  const bf16* x0; const bf16* x1; // dQ kernel: its owned operands (q, d_o head-major), read by the CTA's threads themselves
+  // Outputs, token-major bf16 [T, ld_out]: a row's head lands at column col + head * 128.  out0: dV (dK/dV kernel, as
+  // it is); out1: dK or dQ, with the rotation of the forward pass undone (its transpose), pairs (i, i + 64).
   bf16* out0; bf16* out1;
   int64_t ld_out0, ld_out1;
   int col0, col1;
-  int heads_own;                  // heads per sequence on the owned side (key/value heads for DKV, query heads else)
+  int heads_own;                  // heads per sequence on the owned side (key/value heads for dK/dV, query heads for dQ)
   const float2* cs;               // [S, 64] (cos, sin)
   float scale_log2e, scale;
   int* status;
@@ -484,9 +479,8 @@ __device__ __forceinline__ void fb_tile(const uint32_t (&rs)[32], const uint32_t
   }
 }
 
-template <bool DKV>
 __global__ void __launch_bounds__(FA_THREADS, 1)
-flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map_x0, const __grid_constant__ CUtensorMap map_x1,
+flash_bwd_dkv_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map_x0, const __grid_constant__ CUtensorMap map_x1,
                  const __grid_constant__ CUtensorMap map_y0, const __grid_constant__ CUtensorMap map_y1) {
   extern __shared__ uint8_t fa_smem_raw[];
   const uint32_t raw = smem_u32(fa_smem_raw);
@@ -494,9 +488,10 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   uint8_t* gen_base = fa_smem_raw + (base - raw);
   const uint32_t bars = base + FB_BAR_OFF;
   auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
-  constexpr int NS = FbCfg<DKV>::NS;
-  constexpr int Y_OFF = FbCfg<DKV>::Y_OFF;
-  enum { B_XFULL = 0, B_YFULL = 1, B_YEMPTY = 1 + FB_MAX_NS, B_SDFULL = 1 + 2 * FB_MAX_NS, B_SDEMPTY = B_SDFULL + 2,
+  constexpr int NS = FB_NS;
+  constexpr int Y_OFF = FB_Y_OFF;
+  constexpr bool DKV = true;      // the element routine is shared with the dQ kernel and takes the role as a parameter
+  enum { B_XFULL = 0, B_YFULL = 1, B_YEMPTY = 1 + FB_NS, B_SDFULL = 1 + 2 * FB_NS, B_SDEMPTY = B_SDFULL + 2,
          B_PDFULL = B_SDEMPTY + 2, B_PDEMPTY = B_PDFULL + 1, B_ACCFULL = B_PDEMPTY + 1, B_COUNT = B_ACCFULL + 1 };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + FB_BAR_OFF + 8 * B_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + FB_BAR_OFF + 8 * B_COUNT + 8);
@@ -505,21 +500,19 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_blk = P.Sp / FA_BLK;                  // 128-row blocks per head
   const int n_t64 = P.Sp / 64;                      // 64-row tiles per head
-  // heavy work first: DKV: low key blocks see the most query tiles; else: high query blocks see the most key tiles
+  // heavy work first: low key blocks see the most query tiles
   const int per = (int)gridDim.x / n_blk;
-  const int ord = (int)blockIdx.x / per;
-  const int blk = DKV ? ord : n_blk - 1 - ord;      // own 128-row block within the head
-  const int grp = (int)blockIdx.x % per;            // DKV: sequence * n_kv_heads + kv head; else sequence * n_heads + head
+  const int blk = (int)blockIdx.x / per;            // own 128-key block within the head
+  const int grp = (int)blockIdx.x % per;            // sequence * n_kv_heads + kv head
   const int own_row0 = grp * P.Sp + blk * FA_BLK;
-  const int t_begin = DKV ? 2 * blk : 0;
-  const int n_inner = DKV ? n_t64 - 2 * blk : 2 * blk + 2;
-  const int n_steps = (DKV ? P.rep : 1) * n_inner;
-  // first row of the walked operands: DKV: query head grp * rep (+ ho); else: the key/value head of this query head
-  const int y_base = DKV ? grp * P.rep * P.Sp : (grp / P.rep) * P.Sp;
+  const int t_begin = 2 * blk;
+  const int n_inner = n_t64 - 2 * blk;
+  const int n_steps = P.rep * n_inner;              // every query head of the group in turn
+  const int y_base = grp * P.rep * P.Sp;            // first row of the group's first query head
   auto y_row_of = [&](int s) -> int { return y_base + (s / n_inner) * P.Sp + 64 * (t_begin + s % n_inner); };
 
   if (threadIdx.x == 0) {
-    mbar_init(bar(B_XFULL), DKV ? 1 : 8);
+    mbar_init(bar(B_XFULL), 1);
     mbar_init(bar(B_ACCFULL), 1);
     mbar_init(bar(B_PDFULL), 8);
     mbar_init(bar(B_PDEMPTY), 1);
@@ -547,22 +540,20 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
-      if (DKV) {
-        mbar_expect_tx(bar(B_XFULL), 4 * FA_TILE);
-        issued[0] = 1;
-        for (int kb = 0; kb < 2; ++kb) {
-          tma_load_2d(base + FB_X_OFF + kb * FA_TILE, &map_x0, 64 * kb, own_row0, bar(B_XFULL));
-          tma_load_2d(base + FB_X_OFF + (2 + kb) * FA_TILE, &map_x1, 64 * kb, own_row0, bar(B_XFULL));
-        }
+      mbar_expect_tx(bar(B_XFULL), 4 * FA_TILE);
+      issued[0] = 1;
+      for (int kb = 0; kb < 2; ++kb) {
+        tma_load_2d(base + FB_X_OFF + kb * FA_TILE, &map_x0, 64 * kb, own_row0, bar(B_XFULL));
+        tma_load_2d(base + FB_X_OFF + (2 + kb) * FA_TILE, &map_x1, 64 * kb, own_row0, bar(B_XFULL));
       }
       for (int s = 0; s < n_steps; ++s) {
         const int st = s % NS;
         const uint32_t ph = (uint32_t)(s / NS) & 1u;
         if (!mbar_wait(bar(B_YEMPTY + st), ph ^ 1u, abort_flag, P.status)) break;
-        mbar_expect_tx(bar(B_YFULL + st), FB_STAGE + (DKV ? 512 : 0));
+        mbar_expect_tx(bar(B_YFULL + st), FB_STAGE + 512);
         issued[1 + st] = (int)ph + 1;
         const int yr = y_row_of(s);
-        if (DKV) bulk_load_1d(base + FB_LD_OFF + st * 512, P.lse_d + yr, 512, bar(B_YFULL + st));
+        bulk_load_1d(base + FB_LD_OFF + st * 512, P.lse_d + yr, 512, bar(B_YFULL + st));
         const uint32_t ys = base + Y_OFF + st * FB_STAGE;
         for (int kb = 0; kb < 2; ++kb) {
           tma_load_2d(ys + kb * 8192, &map_y0, 64 * kb, yr, bar(B_YFULL + st));
@@ -590,13 +581,8 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
             const uint64_t a_desc = make_smem_desc(base + FB_X_OFF + (2 * w + kb) * FA_TILE, 16, 1024);
             const uint64_t b_desc = make_smem_desc(ys + w * FA_TILE + kb * 8192, 16, 1024);
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-              if (DKV)
-                tc_mma(d, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(2 * ks), idesc_sd, (kb | ks) != 0 ? 1u : 0u);
-              else   // the owned operand sits in tensor memory: 8 columns of packed pairs per 16 k
-                tc_mma_ta(d, tmem_base + (uint32_t)(256 + 64 * w + 8 * (4 * kb + ks)), b_desc + (uint64_t)(2 * ks), idesc_sd,
-                          (kb | ks) != 0 ? 1u : 0u);
-            }
+            for (int ks = 0; ks < 4; ++ks)
+              tc_mma(d, a_desc + (uint64_t)(2 * ks), b_desc + (uint64_t)(2 * ks), idesc_sd, (kb | ks) != 0 ? 1u : 0u);
           }
         }
         tc_commit(bar(B_SDFULL + b));
@@ -610,7 +596,7 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
         tc_fence_after();
         const uint32_t ys = base + Y_OFF + st * FB_STAGE;
         // the walked tiles again, now as [64 rows (K), 128 columns (N)] operands: the two 64-column halves are 8 KB apart
-        if (DKV) {
+        {
           const uint64_t a_desc = make_smem_desc(base + FB_P_OFF, 16, 1024);
           const uint64_t b_desc = make_smem_desc(ys + FA_TILE, 8192, 1024);
 #pragma unroll
@@ -637,35 +623,14 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     const float cl = P.scale_log2e, scale = P.scale;
     const int own_pos = blk * FA_BLK + row;      // position in the sequence of this thread's own row
-    float2 own_ld = make_float2(0.f, 0.f);
-    if (!DKV && own_pos < P.S) own_ld = P.lse_d[own_row0 + row];
-    __syncwarp();
-    if (!DKV) {
-      // The owned operands never change: each thread puts its row's 64 columns of both into tensor memory
-      // (TMEM columns 256.. for X0, 320.. for X1), where every step's products read them as the A operand.
-#pragma unroll
-      for (int w = 0; w < 2; ++w) {
-        const uint4* src = reinterpret_cast<const uint4*>((w ? P.x1 : P.x0) + (int64_t)(own_row0 + row) * FA_HD + 64 * hh);
-        uint32_t xw[32];
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          const uint4 v = __ldg(src + g);
-          xw[4 * g] = v.x; xw[4 * g + 1] = v.y; xw[4 * g + 2] = v.z; xw[4 * g + 3] = v.w;
-        }
-        tmem_st32(lane_addr + (uint32_t)(256 + 64 * w + 32 * hh), xw);
-      }
-      tmem_st_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_XFULL));
-    }
+    const float2 own_ld = make_float2(0.f, 0.f);      // unused by the key-row role
     bool ok = true;
     for (int s = 0; s < n_steps; ++s) {
       const int b = s & 1;
       const uint32_t ph = (uint32_t)(s >> 1) & 1u;
       if (!mbar_wait(bar(B_SDFULL + b), ph, abort_flag, P.status)) { ok = false; break; }
-      // DKV: this thread reads the stage's row statistics itself, so it observes the stage's barrier itself
-      if (DKV && !mbar_wait(bar(B_YFULL + s % NS), (uint32_t)(s / NS) & 1u, abort_flag, P.status)) { ok = false; break; }
+      // this thread reads the stage's row statistics itself, so it observes the stage's barrier itself
+      if (!mbar_wait(bar(B_YFULL + s % NS), (uint32_t)(s / NS) & 1u, abort_flag, P.status)) { ok = false; break; }
       tc_fence_after();
       uint32_t rs[32], rd[32];
       tmem_ld32(lane_addr + (uint32_t)(b * 128 + 32 * hh), rs);
@@ -677,8 +642,8 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       const int t = t_begin + s % n_inner;
       const int col0 = 64 * t + 32 * hh;         // position in the sequence of this thread's first column
       // tiles that touch the diagonal or the end of the sequence need the element-wise test
-      const bool mask = DKV ? (t < 2 * blk + 2 || 64 * t + 63 >= P.S) : (t >= 2 * blk || blk * FA_BLK + FA_BLK - 1 >= P.S);
-      // DKV: the step's row statistics came with the walked tiles (S' complete implies that stage has landed)
+      const bool mask = t < 2 * blk + 2 || 64 * t + 63 >= P.S;
+      // the step's row statistics came with the walked tiles
       const float4* ld_cols = reinterpret_cast<const float4*>(gen_base + FB_LD_OFF + (s % NS) * 512) + 16 * hh;
       uint4 pp[4], pd[4];
       if (mask) fb_tile<DKV, true>(rs, rd, ld_cols, own_ld, cl, scale, col0, own_pos, P.S, pp, pd);
@@ -690,7 +655,7 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         const int piece = ((4 * hh + g) ^ (row & 7)) << 4;
-        if (DKV) *reinterpret_cast<uint4*>(prow + piece) = pp[g];
+        *reinterpret_cast<uint4*>(prow + piece) = pp[g];
         *reinterpret_cast<uint4*>(drow + piece) = pd[g];
       }
       fence_async_smem();
@@ -708,7 +673,7 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
       const int64_t tok = (int64_t)seq * P.S + (row_ok ? own_pos : 0);
       {
 #pragma unroll
-        for (int a = DKV ? 0 : 1; a < 2; ++a) {
+        for (int a = 0; a < 2; ++a) {          // a = 0: dV as it is, a = 1: dK with the rotation undone
           uint32_t rl[32], rh[32];
           __syncwarp();               // lanes that skipped the previous output rejoin before the warp-wide loads
           tmem_ld32(lane_addr + (uint32_t)(256 + 128 * a + 32 * hh), rl);
@@ -753,6 +718,235 @@ flash_bwd_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map
   }
 }
 
+// ---------------------------------------------------------------------------
+// dQ with 128-key walked tiles.  The 128 x 64 x 16 instructions of the kernel above run at 55 clk against 32 at
+// full rate; the dQ launch has the tensor memory for the 128-wide shape: its owned operands (Q_i, dO_i) sit in
+// tensor memory as A operands (128 columns), S' and dP' take 128 columns each (one buffer: the softmax warps free
+// it once the scores are in registers) and dQ the last 128.  Shared memory: three 64 KB stages of [K_t | V_t] and
+// the dS' operand tile.
+// ---------------------------------------------------------------------------
+constexpr int FQ_NS = 3;
+constexpr int FQ_STAGE = 4 * FA_TILE;
+constexpr int FQ_DS_OFF = FQ_NS * FQ_STAGE;
+constexpr int FQ_BAR_OFF = FQ_DS_OFF + 2 * FA_TILE;
+constexpr int FQ_SMEM_BYTES = FQ_BAR_OFF + 256 + 1024;
+
+__global__ void __launch_bounds__(FA_THREADS, 1)
+flash_bwd_dq_kernel(const FlashBwdParams P, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
+  extern __shared__ uint8_t fa_smem_raw[];
+  const uint32_t raw = smem_u32(fa_smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen_base = fa_smem_raw + (base - raw);
+  const uint32_t bars = base + FQ_BAR_OFF;
+  auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
+  enum { B_XFULL = 0, B_YFULL = 1, B_YEMPTY = 1 + FQ_NS, B_SDFULL = 1 + 2 * FQ_NS, B_SDEMPTY, B_PDFULL, B_PDEMPTY, B_ACCFULL, B_COUNT };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + FQ_BAR_OFF + 8 * B_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + FQ_BAR_OFF + 8 * B_COUNT + 8);
+  int* issued = reinterpret_cast<int*>(gen_base + FQ_BAR_OFF + 8 * B_COUNT + 16);   // [FQ_NS]: stage -> phase + 1
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_blk = P.Sp / FA_BLK;
+  const int per = (int)gridDim.x / n_blk;
+  const int blk = n_blk - 1 - (int)blockIdx.x / per;     // heavy work first: high query blocks see the most key tiles
+  const int grp = (int)blockIdx.x % per;                 // sequence * n_heads + head
+  const int own_row0 = grp * P.Sp + blk * FA_BLK;
+  const int n_steps = blk + 1;                           // key tiles 0 .. the diagonal one
+  const int kv_row0 = (grp / P.rep) * P.Sp;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(B_XFULL), 8);
+    mbar_init(bar(B_SDFULL), 1); mbar_init(bar(B_SDEMPTY), 8);
+    mbar_init(bar(B_PDFULL), 8); mbar_init(bar(B_PDEMPTY), 1);
+    mbar_init(bar(B_ACCFULL), 1);
+    for (int s = 0; s < FQ_NS; ++s) { mbar_init(bar(B_YFULL + s), 1); mbar_init(bar(B_YEMPTY + s), 1); issued[s] = 0; }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // TMEM columns: S' 0..127, dP' 128..255, Q_i 256..319, dO_i 320..383 (packed pairs), dQ 384..511
+  const uint32_t idesc_sd = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(FA_BLK >> 3) << 17) | ((uint32_t)(FA_BLK >> 4) << 24);
+  const uint32_t idesc_acc = idesc_sd | (1u << 16);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      for (int s = 0; s < n_steps; ++s) {
+        const int st = s % FQ_NS;
+        const uint32_t ph = (uint32_t)(s / FQ_NS) & 1u;
+        if (!mbar_wait(bar(B_YEMPTY + st), ph ^ 1u, abort_flag, P.status)) break;
+        mbar_expect_tx(bar(B_YFULL + st), FQ_STAGE);
+        issued[st] = (int)ph + 1;
+        const int yr = kv_row0 + s * FA_BLK;
+        const uint32_t ys = base + st * FQ_STAGE;
+        for (int kb = 0; kb < 2; ++kb) {
+          tma_load_2d(ys + kb * FA_TILE, &map_k, 64 * kb, yr, bar(B_YFULL + st));
+          tma_load_2d(ys + (2 + kb) * FA_TILE, &map_v, 64 * kb, yr, bar(B_YFULL + st));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = mbar_wait(bar(B_XFULL), 0u, abort_flag, P.status);
+      tc_fence_after();
+      auto issue_sd = [&](int s) -> bool {
+        const int st = s % FQ_NS;
+        if (!mbar_wait(bar(B_YFULL + st), (uint32_t)(s / FQ_NS) & 1u, abort_flag, P.status)) return false;
+        if (!mbar_wait(bar(B_SDEMPTY), ((uint32_t)s & 1u) ^ 1u, abort_flag, P.status)) return false;
+        tc_fence_after();
+        const uint32_t ys = base + st * FQ_STAGE;
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {            // w = 0: S' = Q_i K_t^T, w = 1: dP' = dO_i V_t^T
+#pragma unroll
+          for (int kb = 0; kb < 2; ++kb) {
+            const uint64_t b_desc = make_smem_desc(ys + (2 * w + kb) * FA_TILE, 16, 1024);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              tc_mma_ta(tmem_base + (uint32_t)(128 * w), tmem_base + (uint32_t)(256 + 64 * w + 8 * (4 * kb + ks)),
+                        b_desc + (uint64_t)(2 * ks), idesc_sd, (kb | ks) != 0 ? 1u : 0u);
+          }
+        }
+        tc_commit(bar(B_SDFULL));
+        return true;
+      };
+      if (ok) ok = issue_sd(0);
+      for (int s = 0; ok && s < n_steps; ++s) {
+        if (s + 1 < n_steps && !issue_sd(s + 1)) { ok = false; break; }
+        const int st = s % FQ_NS;
+        if (!mbar_wait(bar(B_PDFULL), (uint32_t)s & 1u, abort_flag, P.status)) { ok = false; break; }
+        tc_fence_after();
+        // dQ += dS' K_t: K_t's two 64-column tiles read as one [128 keys, 128 columns] operand, halves 16 KB apart
+        const uint64_t b_desc = make_smem_desc(base + st * FQ_STAGE, 2 * 8192, 1024);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t a_desc = make_smem_desc(base + FQ_DS_OFF + (kk >> 2) * FA_TILE, 16, 1024);
+          tc_mma(tmem_base + 384u, a_desc + (uint64_t)(2 * (kk & 3)), b_desc + (uint64_t)(128 * kk), idesc_acc, (s | kk) != 0 ? 1u : 0u);
+        }
+        tc_commit(bar(B_YEMPTY + st));
+        tc_commit(bar(B_PDEMPTY));
+      }
+      if (ok) tc_commit(bar(B_ACCFULL));
+    }
+  } else {
+    // ------------------------------------------------------------------ dS' (warps 2..9)
+    const int q = warp & 3;
+    const int hh = (warp - 2) >> 2;              // which 64 of the tile's 128 keys
+    const int row = q * 32 + lane;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+    const float cl = P.scale_log2e, scale = P.scale;
+    const int own_pos = blk * FA_BLK + row;
+    float2 own_ld = make_float2(0.f, 0.f);
+    if (own_pos < P.S) own_ld = P.lse_d[own_row0 + row];
+    __syncwarp();
+    // the owned operands into tensor memory: this thread's 64 columns of its row of Q_i and of dO_i
+#pragma unroll
+    for (int w = 0; w < 2; ++w) {
+      const uint4* src = reinterpret_cast<const uint4*>((w ? P.x1 : P.x0) + (int64_t)(own_row0 + row) * FA_HD + 64 * hh);
+      uint32_t xw[32];
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        const uint4 v = __ldg(src + g);
+        xw[4 * g] = v.x; xw[4 * g + 1] = v.y; xw[4 * g + 2] = v.z; xw[4 * g + 3] = v.w;
+      }
+      tmem_st32(lane_addr + (uint32_t)(256 + 64 * w + 32 * hh), xw);
+    }
+    tmem_st_wait();
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(B_XFULL));
+    bool ok = true;
+    const bool edge = blk * FA_BLK + FA_BLK - 1 >= P.S;
+    for (int s = 0; s < n_steps; ++s) {
+      if (!mbar_wait(bar(B_SDFULL), (uint32_t)s & 1u, abort_flag, P.status)) { ok = false; break; }
+      __syncwarp();
+      tc_fence_after();
+      const bool mask = s == blk || edge;
+      const int col0 = FA_BLK * s + 64 * hh;     // position in the sequence of this thread's first key
+      uint32_t rs[32], rd[32];
+      uint4 pp[4], pa[4], pb[4];
+      tmem_ld32(lane_addr + (uint32_t)(64 * hh), rs);
+      tmem_ld32(lane_addr + (uint32_t)(128 + 64 * hh), rd);
+      tmem_ld_wait();
+      if (mask) fb_tile<false, true>(rs, rd, nullptr, own_ld, cl, scale, col0, own_pos, P.S, pp, pa);
+      else fb_tile<false, false>(rs, rd, nullptr, own_ld, cl, scale, col0, own_pos, P.S, pp, pa);
+      __syncwarp();
+      tmem_ld32(lane_addr + (uint32_t)(64 * hh + 32), rs);
+      tmem_ld32(lane_addr + (uint32_t)(128 + 64 * hh + 32), rd);
+      tmem_ld_wait();
+      // every score of the step is in registers: the buffer may take the next tile's
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_SDEMPTY));
+      if (mask) fb_tile<false, true>(rs, rd, nullptr, own_ld, cl, scale, col0 + 32, own_pos, P.S, pp, pb);
+      else fb_tile<false, false>(rs, rd, nullptr, own_ld, cl, scale, col0 + 32, own_pos, P.S, pp, pb);
+      // the operand tile has one buffer: the previous step's accumulating product must have read it
+      if (!mbar_wait(bar(B_PDEMPTY), ((uint32_t)s & 1u) ^ 1u, abort_flag, P.status)) { ok = false; break; }
+      uint8_t* drow = gen_base + FQ_DS_OFF + hh * FA_TILE + row * 128;      // this thread's 64 keys are tile hh
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        *reinterpret_cast<uint4*>(drow + ((g ^ (row & 7)) << 4)) = pa[g];
+        *reinterpret_cast<uint4*>(drow + (((4 + g) ^ (row & 7)) << 4)) = pb[g];
+      }
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_PDFULL));
+    }
+    if (ok && !mbar_wait(bar(B_ACCFULL), 0u, abort_flag, P.status)) ok = false;
+    if (ok) {
+      tc_fence_after();
+      // columns [32 hh, +32) and their rotation partners [64 + 32 hh, +32); every lane executes the warp-wide loads
+      const bool row_ok = own_pos < P.S;
+      const int seq = grp / P.heads_own, head = grp % P.heads_own;
+      const int64_t tok = (int64_t)seq * P.S + (row_ok ? own_pos : 0);
+      uint32_t rl[32], rh[32];
+      __syncwarp();
+      tmem_ld32(lane_addr + (uint32_t)(384 + 32 * hh), rl);
+      tmem_ld32(lane_addr + (uint32_t)(384 + 64 + 32 * hh), rh);
+      tmem_ld_wait();
+      if (row_ok) {
+        float y0[32], y1[32];
+        const float4* cs2 = reinterpret_cast<const float4*>(P.cs + own_pos * 64 + 32 * hh);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float4 cs = cs2[i];
+          const float a0 = __uint_as_float(rl[2 * i]), b0 = __uint_as_float(rh[2 * i]);
+          const float a1 = __uint_as_float(rl[2 * i + 1]), b1 = __uint_as_float(rh[2 * i + 1]);
+          y0[2 * i] = a0 * cs.x + b0 * cs.y;         y1[2 * i] = b0 * cs.x - a0 * cs.y;
+          y0[2 * i + 1] = a1 * cs.z + b1 * cs.w;     y1[2 * i + 1] = b1 * cs.z - a1 * cs.w;
+        }
+        bf16* dst = P.out1 + tok * P.ld_out1 + P.col1 + head * FA_HD + 32 * hh;
+        store32_bf16(dst, y0);
+        store32_bf16(dst + 64, y1);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) {
+    for (int i = 0; i < FQ_NS; ++i) {
+      if (issued[i] == 0) continue;
+      long long t0 = clock64();
+      while (!mbar_try_wait(bar(B_YFULL + i), (uint32_t)(issued[i] - 1)) && clock64() - t0 < TC_WAIT_CYCLES) {}
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // (lse * log2 e, scale * <dO_row, O_row>) per query row; one warp per head-major row.  O is taken before its rounding to
 // bf16: D stands for sum_j P_j dP_j, and with a peaked row dP - D cancels, so an error in D would show in dS.
 __global__ void attn_rowdot_kernel(const float* __restrict__ o32, const bf16* __restrict__ d_o, const float* __restrict__ lse,
@@ -781,8 +975,8 @@ inline int launch_flash_bwd(const bf16* q, const bf16* k, const bf16* v, const b
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return REVFFN_ERR_CUDA;
   if (!attr_set[dev]) {
-    if (cudaFuncSetAttribute(flash_bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FB_SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(flash_bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FB_SMEM_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(flash_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FB_SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(flash_bwd_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FQ_SMEM_BYTES) != cudaSuccess)
       return REVFFN_ERR_CUDA;
     attr_set[dev] = true;
   }
@@ -809,13 +1003,13 @@ inline int launch_flash_bwd(const bf16* q, const bf16* k, const bf16* v, const b
   P.out1 = dkv; P.ld_out1 = ld_dkv; P.col1 = 0;
   P.heads_own = n_kv_heads;
   P.x0 = nullptr; P.x1 = nullptr;
-  flash_bwd_kernel<true><<<batch * n_kv_heads * (Sp / FA_BLK), FA_THREADS, FB_SMEM_BYTES, st>>>(P, k128, v128, q64, do64);
+  flash_bwd_dkv_kernel<<<batch * n_kv_heads * (Sp / FA_BLK), FA_THREADS, FB_SMEM_BYTES, st>>>(P, k128, v128, q64, do64);
   if (cudaGetLastError() != cudaSuccess) return REVFFN_ERR_CUDA;
   P.out0 = nullptr; P.ld_out0 = 0; P.col0 = 0;
   P.out1 = dq; P.ld_out1 = ld_dq; P.col1 = 0;
   P.heads_own = n_heads;
   P.x0 = q; P.x1 = d_o;
-  flash_bwd_kernel<false><<<batch * n_heads * (Sp / FA_BLK), FA_THREADS, FB_SMEM_BYTES, st>>>(P, q128, do128, k64, v64);
+  flash_bwd_dq_kernel<<<batch * n_heads * (Sp / FA_BLK), FA_THREADS, FQ_SMEM_BYTES, st>>>(P, k128, v128);
   return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
 
