@@ -19,7 +19,7 @@ __all__ = ["Block", "Stack", "revffn_moe_saved_size", "revffn_moe_stack_cache_st
            "revffn_attn_workspace_size", "revffn_attn_forward", "revffn_attn_inverse", "revffn_attn_backward",
            "revffn_attn_status", "BlockDesc", "RevStack", "revffn_block_workspace_size", "revffn_block_forward",
            "revffn_block_inverse", "revffn_block_backward", "revffn_block_stack_forward", "revffn_block_stack_backward",
-           "revffn_block_status"]
+           "revffn_block_status", "trainable_names"]
 
 
 def __getattr__(name):

@@ -498,6 +498,17 @@ def revffn_block_status(ws, stream=None) -> int:
     return out.value
 
 
+def trainable_names(stage: int):
+    """Which weights receive gradients in the two stages of the paper's schedule (Sec. 3.3): stage 1 trains only
+    the projection adapters of both branches, stage 2 everything except the MoE router, which stays frozen.
+    Returns (attention names, MoE names); gradients of the other weights are passed as NULL and skipped."""
+    if stage == 1:
+        return ("w_up", "w_down"), ("w_up", "w_down")
+    if stage == 2:
+        return tuple(ATTN_WEIGHT_NAMES), tuple(n for n in WEIGHT_NAMES if n not in ("w_router", "b_router"))
+    raise ValueError("stage must be 1 or 2")
+
+
 class RevStack:
     """n_blocks whole RevFFN blocks (attention branch then MoE branch per block): descriptors, per-layer device
     weights and one workspace.  Pure marshalling around revffn_block_stack_forward / _backward; a single block is
@@ -528,13 +539,15 @@ class RevStack:
         d.inverse_iters = n
         return d
 
-    def grads_arrays(self, attn_grads, moe_grads, accumulate: bool = False):
-        """attn_grads / moe_grads: one dict of fp32 gradient tensors per block (blocks may share tensors)."""
+    def grads_arrays(self, attn_grads, moe_grads, accumulate: bool = False, stage: Optional[int] = None):
+        """attn_grads / moe_grads: one dict of fp32 gradient tensors per block (blocks may share tensors).
+        stage: 1 or 2 keeps only the gradients that stage of the schedule trains (Sec. 3.3)."""
         acc = 1 if accumulate else 0
-        ga = (AttnGrads * self.n_blocks)(*[AttnGrads(**{n: _ptr(g.get(n)) for n in ATTN_WEIGHT_NAMES}, accumulate=acc)
-                                           for g in attn_grads])
-        gm = (Grads * self.n_blocks)(*[Grads(**{n: _ptr(g.get(n)) for n in WEIGHT_NAMES}, accumulate=acc)
-                                       for g in moe_grads])
+        keep_a, keep_m = (ATTN_WEIGHT_NAMES, WEIGHT_NAMES) if stage is None else trainable_names(stage)
+        ga = (AttnGrads * self.n_blocks)(*[AttnGrads(**{n: (_ptr(g.get(n)) if n in keep_a else None)
+                                                        for n in ATTN_WEIGHT_NAMES}, accumulate=acc) for g in attn_grads])
+        gm = (Grads * self.n_blocks)(*[Grads(**{n: (_ptr(g.get(n)) if n in keep_m else None) for n in WEIGHT_NAMES},
+                                             accumulate=acc) for g in moe_grads])
         return ga, gm
 
     def forward(self, s1, s2, topk_idx=None):

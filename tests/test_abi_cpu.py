@@ -144,3 +144,13 @@ def test_block_workspace_is_the_larger_branch_plus_one_stream(rv):
         with pytest.raises(rv.RevffnError) as e:
             rv.revffn_block_workspace_size(bad)
         assert e.value.code == -2
+
+
+def test_schedule_stages_select_the_trainable_weights(rv):
+    a1, m1 = rv.trainable_names(1)
+    assert set(a1) == {"w_up", "w_down"} and set(m1) == {"w_up", "w_down"}          # adapters only
+    a2, m2 = rv.trainable_names(2)
+    assert "w_q" in a2 and "norm_gamma" in a2 and "w_gate" in m2 and "ws_down" in m2
+    assert "w_router" not in m2 and "b_router" not in m2                            # the router stays frozen
+    with pytest.raises(ValueError):
+        rv.trainable_names(3)

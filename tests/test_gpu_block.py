@@ -124,3 +124,33 @@ def test_mismatched_descriptors_are_rejected():
     with pytest.raises(rv.RevffnError) as e:
         rv.revffn_block_workspace_size(d)
     assert e.value.code == -2
+
+
+def test_stage_one_trains_only_the_adapters():
+    """Sec. 3.3, stage 1: every pre-trained weight is frozen; only the adapters' gradients are written, and they
+    equal the ones of a backward pass that computes everything."""
+    acfg = AttnConfig("a", batch=1, seq_len=24, d_model=64, n_heads=2, n_kv_heads=2, weight_dtype="f32", rope_theta=1e4)
+    mcfg = BlockConfig("m", tokens=24, d_model=64, n_experts=4, top_k=2, d_expert=32, d_shared=0, weight_dtype="f32")
+    st, host, cfg, dev_a, dev_m = _make(acfg, mcfg, 2, 0.1)
+    s = make_attn_streams(acfg, 11)
+
+    def run(stage):
+        a, b, g1, g2 = dev(s["x1"]), dev(s["x2"]), dev(s["dy1"]), dev(s["dx2"])
+        st.forward(a, b)
+        ga_t = [{n: torch.full(v.shape, float("nan"), dtype=torch.float32, device="cuda") for n, v in w.items()} for w in dev_a]
+        gm_t = [{n: torch.full(v.shape, float("nan"), dtype=torch.float32, device="cuda") for n, v in w.items()} for w in dev_m]
+        ga, gm = st.grads_arrays(ga_t, gm_t, stage=stage)
+        st.backward(a, b, g1, g2, ga, gm)
+        assert st.status() == 0
+        return ga_t, gm_t, g1, g2
+
+    full_a, full_m, f1, f2 = run(None)
+    s1_a, s1_m, h1, h2 = run(1)
+    assert torch.equal(f1, h1) and torch.equal(f2, h2)            # the stream gradients do not depend on the mask
+    for l in range(2):
+        for grads, full in ((s1_a[l], full_a[l]), (s1_m[l], full_m[l])):
+            for n, t in grads.items():
+                if n in ("w_up", "w_down"):
+                    assert torch.equal(t, full[n]), (l, n)
+                else:
+                    assert torch.isnan(t).all(), (l, n)           # never touched
