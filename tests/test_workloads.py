@@ -42,3 +42,24 @@ def test_zipf_bias_skews_load_with_slope_and_two_empty_experts():
     slope = np.polyfit(np.log(ranks[sel]), np.log(cnt[sel]), 1)[0]
     assert abs(slope + cfg.zipf_s) < 0.1
     assert cnt[0] > 20 * cnt[50]
+
+
+def test_attention_inputs_have_the_stated_shapes_and_distributions():
+    from workloads.generate import ATTN_CONFIGS, attn_weight_shapes, make_attn_streams, make_attn_weights
+    a0, a1 = ATTN_CONFIGS["A0"], ATTN_CONFIGS["A1"]
+    assert (a1.batch, a1.seq_len, a1.d_model, a1.n_heads, a1.n_kv_heads, a1.head_dim) == (4, 2048, 2048, 16, 16, 128)
+    assert a1.tokens == CONFIGS["C1"].tokens and a1.d_model == CONFIGS["C1"].d_model     # the same token batch as C1
+    w, s = make_attn_weights(a0, 0), make_attn_streams(a0, 0)
+    assert {n: v.shape for n, v in w.items()} == attn_weight_shapes(a0)
+    assert w["w_k"].shape == (a0.n_kv_heads * a0.head_dim, a0.d_model) and w["b_k"].shape == (a0.n_kv_heads * a0.head_dim,)
+    assert s["x1"].shape == (a0.tokens, a0.h) and s["x1"].dtype == np.float32
+    assert set(s) == {"x1", "x2", "dy1", "dx2"} and not np.array_equal(s["x1"], s["x2"])
+    assert abs(s["x2"].std() - 1.0) < 0.05 and abs(w["norm_gamma"].mean() - 1.0) < 0.02
+    w2 = make_attn_weights(a0, 0)
+    assert all(np.array_equal(w[n], w2[n]) for n in w)                 # seeded
+    assert not np.array_equal(make_attn_weights(a0, 1)["w_q"], w["w_q"])
+    # bf16 configurations: matrices exactly representable in bf16, biases and the norm scale stay fp32
+    from dataclasses import replace
+    wb = make_attn_weights(replace(a0, weight_dtype="bf16"), 0)
+    assert (wb["w_q"].view(np.uint32) & 0xFFFF == 0).all() and (wb["w_up"].view(np.uint32) & 0xFFFF == 0).all()
+    assert (wb["b_q"].view(np.uint32) & 0xFFFF != 0).any()
