@@ -894,6 +894,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--blocks", type=int, default=0, help="C3: number of layers (default: the configuration's 24)")
     ap.add_argument("--no-drift", action="store_true", help="C3: skip the per-layer drift pass")
+    ap.add_argument("--seq-len", type=int, default=0, help="A1: sequence length at the same token count (default 2048)")
     ap.add_argument("--gating", default="renorm", choices=["renorm", "softmax_all"],
                     help="single-block runs: gate weights renormalised over the top-k (default, the benchmark's "
                          "definition) or taken from the softmax over all experts")
@@ -903,7 +904,12 @@ def main():
     if args.config in ("B1", "B3") and args.impl == "ours":
         return run_block_stack(args, ATTN_CONFIGS["A1"], CONFIGS["C1"], 24 if args.config == "B3" else 1)
     if args.config in ATTN_CONFIGS and args.impl == "ours":
-        return run_attn(args, ATTN_CONFIGS[args.config])
+        acfg = ATTN_CONFIGS[args.config]
+        if args.seq_len:        # same number of tokens in fewer, longer (or more, shorter) sequences
+            from dataclasses import replace
+            acfg = replace(acfg, seq_len=args.seq_len, batch=max(1, acfg.tokens // args.seq_len),
+                           name=f"{acfg.name}@seq{args.seq_len}")
+        return run_attn(args, acfg)
     if args.impl == "reference" and args.config not in CONFIGS:
         args.config = "C1"          # the reference arm times the oracle of the headline path only
     if args.config == "C4":
