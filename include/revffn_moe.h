@@ -34,9 +34,19 @@
  *     as void*).  Calls that share a workspace must be ordered on one stream.
  *   - Return value: REVFFN_OK (0) or a negative revffn_error.  On an error
  *     return nothing has been launched.  Device-side problems (a bounded wait
- *     that expired) set a status word in the workspace, first error wins; each
- *     forward/inverse/backward call clears it when it starts, so
- *     revffn_moe_status reports the most recent call.
+ *     that expired, an expert index out of range) set a status word in the
+ *     workspace, first error wins; each forward/inverse/backward call clears it
+ *     when it starts unless REVFFN_FLAG_KEEP_STATUS is set, so revffn_moe_status
+ *     reports the most recent call.  The entry points that chain several passes
+ *     on one workspace (the stack, the host step) clear it once and report the
+ *     first error of the whole chain.
+ *   - Expert indices handed in by the caller (topk_idx_in, routing records, the
+ *     stack's topk_idx) must lie in [0, E).  An entry outside that range is not
+ *     used: its (token, slot) pair contributes nothing, the status word becomes
+ *     REVFFN_ERR_INDEX, and no access leaves the buffers.
+ *   - One device per process at a time is the tested configuration.  Per-device
+ *     set-up (kernel attributes, the SM count) is done on the first call on each
+ *     device under a lock; the profiler of revffn_debug.h is not thread-safe.
  */
 #ifndef REVFFN_MOE_H_
 #define REVFFN_MOE_H_
@@ -58,7 +68,10 @@ typedef enum {
   REVFFN_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed                */
   REVFFN_ERR_DEVICE_WAIT = -7,  /* status word: a bounded device-side wait expired  */
   REVFFN_ERR_UNSUPPORTED = -8,  /* valid request that this build does not implement */
-  REVFFN_ERR_NOALLOC_LIMIT = -9 /* revffn_moe_route_noalloc: problem exceeds its fixed scratch */
+  REVFFN_ERR_NOALLOC_LIMIT = -9, /* revffn_moe_route_noalloc: problem exceeds its fixed scratch */
+  REVFFN_ERR_INDEX = -10,       /* status word: a caller-supplied expert index is outside [0, E)   */
+  REVFFN_ERR_CANARY = -11,      /* status word (DEBUG_CHECKS): a guard word between workspace buffers was overwritten */
+  REVFFN_ERR_NONFINITE = -12    /* status word (DEBUG_CHECKS): a router logit is NaN or infinite    */
 } revffn_error;
 
 enum { REVFFN_F32 = 0, REVFFN_BF16 = 1 };          /* weight_dtype                    */
@@ -96,6 +109,26 @@ enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                
  * the original by rounding (Sec. 3.1 recomputes the router; this remembers 4(2k+1) bytes per token
  * instead).  Combined with REVFFN_FLAG_GATE_SOFTMAX_ALL only the indices of the record are used. */
 #define REVFFN_FLAG_ROUTING_RECORD 16u
+/* Keep the status word: the call does not clear the workspace's status word when it starts, so
+ * that several calls chained on one workspace report the FIRST device-side error of the chain
+ * (clear the word once, with a call that does not carry the flag or with a memset of the first
+ * 4 bytes of the workspace, then read it after the last call).  The stack and host-step entry
+ * points use it for their inner calls. */
+#define REVFFN_FLAG_KEEP_STATUS 32u
+/* Debug checks (the stand-in for a memory checker): every sub-buffer of the workspace is followed
+ * by a 256-byte guard zone that the call fills with a pattern when it starts and verifies when it
+ * ends (REVFFN_ERR_CANARY in the status word names an overrun), and the router raises
+ * REVFFN_ERR_NONFINITE for a NaN or infinite logit.  The workspace is larger with the flag set
+ * (ask revffn_moe_workspace_size with the same flags) and every pass runs two more small kernels.
+ * Range checks of caller-supplied expert indices are always on (REVFFN_ERR_INDEX). */
+#define REVFFN_FLAG_DEBUG_CHECKS 64u
+/* The router folded through P_up (an (E+1) x h fp64 matrix that forward / inverse / backward derive
+ * from w_router, ws_sgate and w_up at the start of each call) is still in this workspace from an
+ * earlier call with the same weights: skip that step.  The paper freezes the router (Sec. 3.3) and the
+ * adapters change once per optimiser step, so within a training step every pass after the first may
+ * set the flag.  The caller vouches that the three tensors are unchanged since that call and that no
+ * call with another descriptor has used the workspace in between. */
+#define REVFFN_FLAG_ROUTER_FOLDED 128u
 
 /*
  * Block descriptor.  Shape constraints (else REVFFN_ERR_SHAPE):
@@ -276,19 +309,31 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
  *   topk_idx_out [T, k] int32   selected experts per token, descending logit
  *   gates_out    [T, k] fp32    softmax over the selected logits
  *   sgate_out    [T]    fp32    shared-expert sigmoid gate (0 without one)
- * from y1 ([T, h] fp32, stride ld_stream) exactly as revffn_moe_forward does,
- * but keeps its one piece of scratch -- the router folded through P_up,
- * (E + 1) * h doubles -- in a fixed array inside the library's device image
- * rather than in a workspace.  It calls no cudaMalloc, cudaFree or other
- * allocating routine.
+ * from y1 ([T, h] fp32, stride ld_stream) with the selection rule of
+ * revffn_moe_forward (fp64 logits from the folded router, ties to the lower
+ * index, softmax over the k selected logits), but keeps its one piece of
+ * scratch -- the router folded through P_up, (E + 1) * h doubles -- in a fixed
+ * array inside the library's device image rather than in a workspace.  The fold
+ * is summed in a different order than in revffn_moe_forward (which splits it
+ * over partial sums that need scratch of their own), so the folded matrix
+ * agrees to fp64 rounding, not bit for bit; the selected experts differ only
+ * for tokens whose k-th and (k+1)-th logits tie to about 1e-13.  It calls no
+ * cudaMalloc, cudaFree or other allocating routine.
  *
  * Limits and sharing
  *   - (E + 1) * h <= REVFFN_ROUTE_NOALLOC_MAX_ELEMS (512 KB of scratch, held by
- *     every device that loads the library until the process exits) and
- *     n_experts small enough for 48 KB of shared memory (E <= 100 or so);
- *     otherwise REVFFN_ERR_NOALLOC_LIMIT and nothing is launched.
- *   - The first call on a device looks up the array's device address; make that
- *     first call outside any stream capture.
+ *     every device that loads the library until the process exits); otherwise
+ *     REVFFN_ERR_NOALLOC_LIMIT and nothing is launched.  The router kernel keeps
+ *     a 64-token tile of logits in shared memory, 8 * 64 * (E + 1) bytes plus
+ *     37 KB of operand staging: above 48 KB in total (E >= 23) the first call on
+ *     a device raises the kernel's dynamic shared-memory limit, which is a
+ *     function attribute, not an allocation; E = 256 needs 166 KB.
+ *   - REVFFN_FLAG_GATE_SOFTMAX_ALL is not supported here (its gates need the
+ *     softmax over all E logits, which this entry point does not form):
+ *     REVFFN_ERR_UNSUPPORTED, nothing is launched.  Other flags are ignored.
+ *   - The first call on a device looks up the array's device address (and may
+ *     raise the shared-memory limit, above); make that first call outside any
+ *     stream capture.
  *   - All calls on a device share the one array.  Each call rewrites the part
  *     it uses before reading it, so nothing has to be cleared, but two calls
  *     that overlap on the GPU (different streams) race: order them.
@@ -296,66 +341,6 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
 #define REVFFN_ROUTE_NOALLOC_MAX_ELEMS 65536
 int revffn_moe_route_noalloc(const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1,
                              int32_t* topk_idx_out, float* gates_out, float* sgate_out, void* cuda_stream);
-
-/*
- * Launch accounting and optional per-kernel timing.  (No paper counterpart.)
- * revffn_prof_enable(1) makes every later kernel launch of this library record
- * a CUDA event before and after itself on the caller's stream;
- * revffn_prof_collect waits for those events and returns, per slot, the summed
- * device milliseconds and the number of launches (host arrays of
- * revffn_prof_num_slots() entries), then forgets them.  Slots are named
- * "<pass>/<kernel>", pass in {fwd, inv, bwd}.  revffn_prof_launches counts
- * every kernel this library has launched since it was loaded, enabled or not.
- * Not thread-safe.
- */
-int revffn_prof_enable(int on);
-long long revffn_prof_launches(void);
-int revffn_prof_num_slots(void);
-const char* revffn_prof_slot_name(int slot);
-int revffn_prof_collect(float* ms, int32_t* count, int n_slots);
-
-/*
- * Introspection for tests: byte offset and size inside the backward workspace
- * layout of a named intermediate ("n", "u", "gates", "sgate", "tok_row",
- * "row_tok", "expert_off", "up", "hmid", "o", "hs", "s", "z", "ab", ...).
- * The forward layout is a prefix of the backward layout.  Returns
- * REVFFN_ERR_UNSUPPORTED for unknown names.  (No paper counterpart.)
- */
-int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* offset, size_t* bytes);
-
-/*
- * One C = A * B^T problem on either GEMM backend; used by the tests to check
- * the tcgen05 kernels against the CUDA-core kernels.  See revffn_gemm_problem
- * in the library source for field meanings.  (No paper counterpart.)
- */
-typedef struct {
-  int32_t M, N, K;
-  int32_t a_mn_major, b_mn_major;  /* 0: [rows, K] K contiguous; 1: [K, rows] rows contiguous */
-  int32_t concat;                  /* 0 none, 1 N-concat (SwiGLU pair), 2 K-concat            */
-  int32_t epilogue;                /* 0 store, 1 swiglu, 2 rowscale, 3 couple, 4 dswiglu, 5 wgrad */
-  int32_t out_f32;                 /* store epilogue: fp32 instead of bf16 output             */
-  int32_t accumulate;
-  int32_t use_simt;
-  const void *A, *B0, *B1;         /* bf16                                                    */
-  int64_t lda, ldb;
-  void *C, *C1;
-  int64_t ldc, ldc1;
-  const float* rowscale;
-  const float* resid; int64_t ld_resid; float resid_sign;
-  void* ab; int64_t ld_ab;         /* dswiglu: [M, 2N] bf16 a|b in, da|db out                  */
-  float* dg_part; int32_t dg_ld;
-  /* grouping: 0 none, 1 rows grouped (group_off, tile_group, rows_total), 2 K grouped */
-  int32_t group_mode, n_groups;
-  const int32_t *group_off, *tile_group, *rows_total;
-  int64_t b_group_stride, c_group_stride;
-  int32_t a_col0, b_col0;
-  /* rows grouped: optional table of (expert, first row, rows, 0) runs of real rows, rows a multiple of
-   * 32 and at most 256, int32 x 4 each, 16-byte aligned; their number at rows_total[1].  With it the
-   * tcgen05 back end works store / gate-scale products with the rows on the MMA N side. */
-  const void* tok_chunks;
-  int32_t no_pair;                 /* tcgen05 back end: one CTA per tile even where CTA pairs apply */
-} revffn_dbg_gemm_args;
-int revffn_dbg_gemm(const revffn_dbg_gemm_args* args, int32_t* status_word_dev, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -20,6 +20,11 @@ FLAG_SAVE_ACTIVATIONS = 2
 FLAG_REUSE_ACTIVATIONS = 4
 FLAG_GATE_SOFTMAX_ALL = 8
 FLAG_ROUTING_RECORD = 16
+FLAG_KEEP_STATUS = 32
+FLAG_DEBUG_CHECKS = 64
+FLAG_ROUTER_FOLDED = 128
+
+ERR_DEVICE_WAIT, ERR_UNSUPPORTED, ERR_NOALLOC_LIMIT, ERR_INDEX, ERR_CANARY, ERR_NONFINITE = -7, -8, -9, -10, -11, -12
 
 WEIGHT_NAMES = ("norm_gamma", "w_up", "w_down", "w_router", "b_router", "w_gate", "w_upx", "w_downx",
                 "ws_gate", "ws_up", "ws_down", "ws_sgate")
@@ -78,7 +83,8 @@ class DbgGemmArgs(C.Structure):
                 ("dg_part", C.c_void_p), ("dg_ld", C.c_int32), ("group_mode", C.c_int32), ("n_groups", C.c_int32),
                 ("group_off", C.c_void_p), ("tile_group", C.c_void_p), ("rows_total", C.c_void_p),
                 ("b_group_stride", C.c_int64), ("c_group_stride", C.c_int64), ("a_col0", C.c_int32),
-                ("b_col0", C.c_int32), ("tok_chunks", C.c_void_p), ("no_pair", C.c_int32)]
+                ("b_col0", C.c_int32), ("tok_chunks", C.c_void_p), ("no_pair", C.c_int32),
+                ("wait_cycles", C.c_int64), ("starve_operands", C.c_int32)]
 
 
 def _load() -> C.CDLL:
@@ -97,6 +103,8 @@ def _load() -> C.CDLL:
     lib.revffn_strerror.restype = C.c_char_p
     lib.revffn_moe_ws_lookup.argtypes = [C.POINTER(Desc), C.c_char_p, C.POINTER(sz), C.POINTER(sz)]
     lib.revffn_dbg_gemm.argtypes = [C.POINTER(DbgGemmArgs), vp, vp]
+    lib.revffn_dbg_check_guards.argtypes = [C.POINTER(Desc), vp, sz, vp]
+    lib.revffn_dbg_check_guards.restype = C.c_int
     lib.revffn_moe_step_host.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.POINTER(Grads), vp, vp, vp, vp, vp, vp,
                                          vp, sz, vp, sz, vp, vp]
     lib.revffn_moe_saved_size.argtypes = [C.POINTER(Desc), C.POINTER(sz)]
@@ -276,6 +284,12 @@ def revffn_prof_collect() -> Dict[str, tuple]:
     return {lib.revffn_prof_slot_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i] > 0}
 
 
+def revffn_dbg_check_guards(desc: Desc, ws, stream: Optional[int] = None) -> None:
+    """Verify the workspace's guard zones now (desc must carry FLAG_DEBUG_CHECKS); the result is in the status word."""
+    _check(lib.revffn_dbg_check_guards(C.byref(desc), _ptr(ws), ws.numel() * ws.element_size(),
+                                       stream if stream is not None else _stream()), "revffn_dbg_check_guards")
+
+
 def ws_lookup(desc: Desc, name: str):
     off, nbytes = C.c_size_t(0), C.c_size_t(0)
     _check(lib.revffn_moe_ws_lookup(C.byref(desc), name.encode(), C.byref(off), C.byref(nbytes)), "revffn_moe_ws_lookup")
@@ -323,30 +337,31 @@ class Block:
         d.flags = self.desc.flags | extra_flags
         return d
 
-    def forward(self, y1, x2, y2=None, topk_idx_out=None, save: bool = False, ws=None):
-        """save=True keeps the branch's intermediates for a later backward(reuse=True)."""
+    def forward(self, y1, x2, y2=None, topk_idx_out=None, save: bool = False, ws=None, flags: int = 0):
+        """save=True keeps the branch's intermediates for a later backward(reuse=True); flags: more REVFFN_FLAG_* bits
+        for this call (e.g. FLAG_ROUTER_FOLDED, FLAG_KEEP_STATUS)."""
         if y2 is None:
             y2 = torch.empty_like(x2)
-        revffn_moe_forward(self._desc(FLAG_SAVE_ACTIVATIONS if save else 0), self.w, y1, x2, y2, topk_idx_out,
+        revffn_moe_forward(self._desc((FLAG_SAVE_ACTIVATIONS if save else 0) | flags), self.w, y1, x2, y2, topk_idx_out,
                            self.ws if ws is None else ws)
         return y2
 
-    def inverse(self, y1, y2, x2=None, topk_idx_in=None, save: bool = False, ws=None):
+    def inverse(self, y1, y2, x2=None, topk_idx_in=None, save: bool = False, ws=None, flags: int = 0):
         if x2 is None:
             x2 = torch.empty_like(y2)
-        revffn_moe_inverse(self._desc(FLAG_SAVE_ACTIVATIONS if save else 0), self.w, y1, y2, x2, topk_idx_in,
+        revffn_moe_inverse(self._desc((FLAG_SAVE_ACTIVATIONS if save else 0) | flags), self.w, y1, y2, x2, topk_idx_in,
                            self.ws if ws is None else ws)
         return x2
 
     def backward(self, y1, dy2, dy1_inout, grads: Optional[Dict[str, torch.Tensor]] = None, accumulate: bool = False,
-                 topk_idx_in=None, reuse: bool = False, ws=None):
+                 topk_idx_in=None, reuse: bool = False, ws=None, flags: int = 0):
         """reuse=True: the workspace still holds what forward/inverse(save=True) left for this y1."""
         grads = grads or {}
         for n, t in grads.items():
             if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
                 raise ValueError(f"gradient {n}: need a contiguous fp32 CUDA tensor")
         g = Grads(**{n: _ptr(grads.get(n)) for n in WEIGHT_NAMES}, accumulate=1 if accumulate else 0)
-        revffn_moe_backward(self._desc(FLAG_REUSE_ACTIVATIONS if reuse else 0), self.w, y1, dy2, dy1_inout, g,
+        revffn_moe_backward(self._desc((FLAG_REUSE_ACTIVATIONS if reuse else 0) | flags), self.w, y1, dy2, dy1_inout, g,
                             topk_idx_in, self.ws if ws is None else ws)
         return dy1_inout
 

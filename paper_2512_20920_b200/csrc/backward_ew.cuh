@@ -54,17 +54,19 @@ __global__ void router_bwd_kernel(const float* __restrict__ dg_part, int dg_ld, 
   if (t >= tokens) return;
   float dg[8], g[8], mix = 0.f;
   for (int s = 0; s < k; ++s) {
-    int row = tok_row[(int64_t)t * k + s];
+    int row = tok_row[(int64_t)t * k + s];      // -1: entry with an out-of-range expert index, contributes nothing
     float acc = 0.f;
-    for (int j = 0; j < n_part; ++j) acc += dg_part[(int64_t)row * dg_ld + j];
+    if (row >= 0)
+      for (int j = 0; j < n_part; ++j) acc += dg_part[(int64_t)row * dg_ld + j];
     dg[s] = acc;
-    g[s] = gate[(int64_t)t * k + s];
+    g[s] = row >= 0 ? gate[(int64_t)t * k + s] : 0.f;
     mix += g[s] * acc;
   }
   for (int s = 0; s < k; ++s) {
     float v = g[s] * (dg[s] - mix);
     tok_dl[(int64_t)t * k + s] = v;
-    row_dl[tok_row[(int64_t)t * k + s]] = v;
+    const int row = tok_row[(int64_t)t * k + s];
+    if (row >= 0) row_dl[row] = v;
   }
 }
 
@@ -83,12 +85,13 @@ __global__ void router_bwd_dense_kernel(const float* __restrict__ dg_part, int d
   const float* p = prob + (int64_t)t * E;
   float c = 0.f;
   for (int s = 0; s < k; ++s) {
-    int row = tok_row[(int64_t)t * k + s];
+    int row = tok_row[(int64_t)t * k + s];      // -1: entry with an out-of-range expert index, contributes nothing
     float acc = 0.f;
-    for (int j = 0; j < n_part; ++j) acc += dg_part[(int64_t)row * dg_ld + j];
+    if (row >= 0)
+      for (int j = 0; j < n_part; ++j) acc += dg_part[(int64_t)row * dg_ld + j];
     dg[s] = acc;
-    ex[s] = idx[(int64_t)t * k + s];
-    c += p[ex[s]] * acc;
+    ex[s] = row >= 0 ? idx[(int64_t)t * k + s] : -1;
+    if (row >= 0) c += p[ex[s]] * acc;
   }
   T* o = dl_out + (int64_t)t * ld_dl;
   for (int j = 0; j < ld_dl; ++j) {
@@ -209,7 +212,7 @@ __global__ void du_reduce_kernel(const T* __restrict__ dUp, const int32_t* __res
   int rows[8], ex[8];
   float dls[8];
   for (int s = 0; s < k; ++s) {
-    rows[s] = tok_row[(int64_t)t * k + s];
+    rows[s] = tok_row[(int64_t)t * k + s];      // -1: entry with an out-of-range expert index, skipped below
     ex[s] = idx[(int64_t)t * k + s];
     dls[s] = dUr ? 0.f : tok_dl[(int64_t)t * k + s];
   }
@@ -220,6 +223,7 @@ __global__ void du_reduce_kernel(const T* __restrict__ dUp, const int32_t* __res
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
     Vec8<T> v;
     for (int s = 0; s < k; ++s) {
+      if (rows[s] < 0) continue;
       v.load(dUp + (int64_t)rows[s] * width + c); v.get(f);
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[i] += f[i];
@@ -238,6 +242,7 @@ __global__ void du_reduce_kernel(const T* __restrict__ dUp, const int32_t* __res
       for (int i = 0; i < 8; ++i) acc[i] += f[i];
     } else {
       for (int s = 0; s < k; ++s) {
+        if (rows[s] < 0) continue;
         v.load(w_router + (int64_t)ex[s] * width + c); v.get(f);
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] += dls[s] * f[i];

@@ -57,6 +57,8 @@ struct GemmProblem {
   int64_t b_group_stride, c_group_stride;
   int a_col0, b_col0;
   int no_pair;        // tcgen05 back end: never pair CTAs for this product
+  long long dbg_wait_cycles;   // tcgen05 back end, tests: bound on every device-side wait (0 = default)
+  int dbg_starve;              // tcgen05 back end, tests (needs no_pair): no operand loads are issued
   // EPI_HEADS (tcgen05 back end, dense products only): the N columns are heads of 128; C receives, head-major
   // [sequence, head, hm_Sp, 128], the product plus hm_bias, with the pairs (i, i + 64) of a head turned by the
   // angle of hm_cs[position, i] (cos, sin) when hm_cs is given.  Row m is position m % hm_S of sequence m / hm_S.

@@ -3,7 +3,8 @@
 // One persistent, warp-specialised kernel (1 CTA per SM, 320 threads):
 //   warp 0      TMA producer: cp.async.bulk.tensor 2D loads (128-byte swizzle) of
 //               A and B tiles into a ring of shared-memory stages, completion on
-//               mbarriers (no cluster multicast anywhere).
+//               mbarriers (no multicast LOADS anywhere: every CTA fetches its own operands; the only
+//               cluster-wide instruction is the pair mode's tcgen05.commit, a barrier arrive).
 //   warp 1      MMA issuer: owns the TMEM allocation (two accumulators, so the
 //               epilogue of tile i overlaps the main loop of tile i+1); one
 //               elected lane issues tcgen05.mma kind::f16 (bf16 x bf16 -> fp32),
@@ -43,6 +44,7 @@
 
 #include <cuda.h>
 #include <cstring>
+#include <mutex>
 #include <type_traits>
 
 #include "common.cuh"
@@ -80,6 +82,8 @@ struct TcParams {
   int tr;                    // transposed pair mode: weights on the MMA M side, an expert's token rows on the N side
   int tiles_f;               // tr: 256-wide feature tiles per token chunk
   uint32_t idesc;
+  long long wait_cycles;     // bound on every wait of the kernel (clock cycles)
+  int starve;                // failure-path test: the load warp issues nothing, so the first wait for operands runs out
 };
 
 // ---------------------------------------------------------------------------
@@ -107,7 +111,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the wait was abandoned (this or another
 // role ran out of time); the caller then leaves its loop.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long limit = TC_WAIT_CYCLES) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = clock64();
   int spins = 0;
@@ -115,7 +120,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if (((++spins) & 63) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > TC_WAIT_CYCLES) {
+      if (clock64() - t0 > limit) {
         *abort_flag = 1;
         set_status(status, REVFFN_ERR_DEVICE_WAIT);
         return false;
@@ -330,6 +335,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + 2 + a); };
   auto epi_bar = [&](int ew, int s) { return bars + 128u + 8u * (ew * 2 + s); };   // SwiGLU backward: operand loads
+  const uint32_t drain_bar = bars + 320u;      // abort path of the MMA thread: "every product issued so far is done"
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + Cfg::BAR_OFF + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* issued = reinterpret_cast<int*>(tmem_slot + 2);   // [STAGES] parity+1 of the last load issued per stage
@@ -344,6 +350,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
     for (int s = 0; s < Cfg::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); issued[s] = 0; }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), PAIR ? 2 * TC_EPI_WARPS : TC_EPI_WARPS); }
     for (int a = 0; a < 2 * TC_EPI_WARPS; ++a) mbar_init(epi_bar(a / 2, a % 2), 1);
+    mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -370,7 +377,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
-    if (lane == 0) {
+    if (lane == 0 && !P.starve) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -379,7 +386,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         if (!t.valid) break;
         const int k_half = t.k_blocks / 2;
         for (int kb = 0; kb < t.k_blocks; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, P.wait_cycles)) { ok = false; break; }
           const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
           const uint32_t sb = sa + TC_A_BYTES;
           if constexpr (PAIR) {
@@ -482,12 +489,12 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         if (!t.valid) break;
         const int acc = it & 1;
         const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, P.wait_cycles)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MMA_N);
         const uint32_t idesc = (P.idesc & ~(0x3Fu << 17)) | ((uint32_t)(t.ncols >> 3) << 17);   // N of this tile
         for (int kb = 0; kb < t.k_blocks; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, P.wait_cycles)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
           const uint32_t sb = sa + TC_A_BYTES;
@@ -512,6 +519,15 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         }
         if (!ok) break;
         if constexpr (PAIR) tc_commit_pair(tfull_bar(acc)); else tc_commit(tfull_bar(acc));   // accumulator complete
+      }
+      if (!ok && !PAIR) {
+        // A wait was abandoned.  Products issued before it may still be running: they read the stage ring and
+        // write tensor memory, so they must have finished before the teardown below releases either.  A commit
+        // on a barrier of its own completes once every product issued so far is done (products wait for
+        // nothing themselves, so this ends; the wait is bounded all the same).
+        tc_commit(drain_bar);
+        const long long t0 = clock64();
+        while (!mbar_try_wait(drain_bar, 0u) && clock64() - t0 < P.wait_cycles) {}
       }
     }
   } else {
@@ -562,7 +578,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       if (!t.valid) break;
       const int acc = it & 1;
       const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, P.wait_cycles)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * MMA_N);
       const int m = t.m0 + row_in_tile;
@@ -800,7 +816,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           const int c = (half + 2 * ci) * 32;
           const int n = t.n0 + c;
           tmem_ld32(taddr + c, r0);
-          if (!mbar_wait(epi_bar(ew, s2), par, abort_flag, p.status)) { ok = false; tmem_ld_wait(); break; }
+          if (!mbar_wait(epi_bar(ew, s2), par, abort_flag, p.status, P.wait_cycles)) { ok = false; tmem_ld_wait(); break; }
           tmem_ld_wait();
           uint8_t* set = stg + s2 * DS_SET;
           uint8_t* row_a = set + lane * 64;
@@ -856,7 +872,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       if (lane == 0) {
         for (uint32_t g = ds_g; g < ds_pf_g; ++g) {
           long long t0 = clock64();
-          while (!mbar_try_wait(epi_bar(ew, (int)(g & 1u)), (g >> 1) & 1u) && clock64() - t0 < TC_WAIT_CYCLES) {}
+          while (!mbar_try_wait(epi_bar(ew, (int)(g & 1u)), (g >> 1) & 1u) && clock64() - t0 < P.wait_cycles) {}
         }
       }
     }
@@ -871,7 +887,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
     for (int s = 0; s < Cfg::STAGES; ++s) {
       if (issued[s] == 0) continue;
       long long t0 = clock64();
-      while (!mbar_try_wait(full_bar(s), (uint32_t)(issued[s] - 1)) && clock64() - t0 < TC_WAIT_CYCLES) {}
+      while (!mbar_try_wait(full_bar(s), (uint32_t)(issued[s] - 1)) && clock64() - t0 < P.wait_cycles) {}
     }
   }
   __syncthreads();
@@ -905,12 +921,20 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Per-device set-up state (kernel attributes and the SM count belong to a device, not to the process).
 struct TcState {
   EncodeTiledFn encode = nullptr;
   int n_sms = 0;
   bool ready = false;
 };
-inline TcState& tc_state() { static TcState s; return s; }
+constexpr int TC_MAX_DEVICES = 64;
+// State of the current device; devices beyond the table share the last slot and are refused by tc_prepare.
+inline TcState& tc_state() {
+  static TcState s[TC_MAX_DEVICES + 1];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= TC_MAX_DEVICES) dev = TC_MAX_DEVICES;
+  return s[dev];
+}
 
 template <int MMA_N, int EPI>
 inline cudaError_t tc_set_attr() {
@@ -921,10 +945,18 @@ inline cudaError_t tc_set_attr() {
                               TcCfg<MMA_N, EPI, true>::SMEM_BYTES);
 }
 
-// Once per process: driver entry point for tensor-map encoding, SM count, shared-memory opt-in.
+// Once per device (under a lock: two host threads may arrive together): driver entry point for tensor-map
+// encoding, SM count, shared-memory opt-in of every kernel instance.
 inline int tc_prepare() {
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
   TcState& s = tc_state();
   if (s.ready) return REVFFN_OK;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return REVFFN_ERR_CUDA;
+    if (dev < 0 || dev >= TC_MAX_DEVICES) return REVFFN_ERR_UNSUPPORTED;
+  }
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
@@ -1010,6 +1042,9 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   P.tiles_m = (int)ceil_div(p.M, TC_BM);
   P.tiles_n = (int)ceil_div(p.N, P.tile_n);
   P.k_blocks = (int)ceil_div(p.K, TC_BK);
+  P.wait_cycles = p.dbg_wait_cycles > 0 ? p.dbg_wait_cycles : TC_WAIT_CYCLES;
+  P.starve = p.dbg_starve;
+  if (p.dbg_starve && !p.no_pair) return REVFFN_ERR_UNSUPPORTED;      // the starved-wait test runs one CTA per tile
   if (p.N % 128 != 0) return REVFFN_ERR_SHAPE;
   // K need not be a multiple of the 64-wide K step: the tensor maps end at K, so the rest of the last
   // step is loaded as zeros (K-major rows must still start on 16-byte boundaries: lda, ldb)

@@ -2,12 +2,15 @@
 // See include/revffn_moe.h for the contract of every entry point.
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <type_traits>
 #include <string>
 #include <vector>
 
 #include "common.cuh"
+#include "../../include/revffn_debug.h"
 #include "routing.cuh"
 #include "backward_ew.cuh"
 #include "gemm.cuh"
@@ -78,6 +81,8 @@ struct ProfScope {
 // Workspace layout
 // ---------------------------------------------------------------------------
 struct Buf { size_t off = 0, bytes = 0; };
+constexpr int MAX_GUARDS = 80;
+constexpr int GUARD_BYTES = 256;
 
 struct WsLayout {
   // forward / inverse
@@ -92,6 +97,9 @@ struct WsLayout {
   size_t bwd_bytes = 0;
   int64_t rows_pad = 0;   // upper bound on padded rows
   int n_chunks = 0, max_tiles = 0, dg_ld = 0, strips = 0;
+  // REVFFN_FLAG_DEBUG_CHECKS: a guard zone of GUARD_BYTES follows every buffer
+  int n_guards = 0;
+  size_t guard_off[MAX_GUARDS];
 };
 
 constexpr int STRIP = 32;    // tokens per strip in two-pass column reductions
@@ -108,9 +116,14 @@ static WsLayout plan_workspace(const revffn_moe_desc& D) {
   L.strips = (int)ceil_div(T > 0 ? T : 1, STRIP);
   const int64_t Rp = L.rows_pad;
   size_t off = 0;
+  const bool guards = (D.flags & REVFFN_FLAG_DEBUG_CHECKS) != 0;
   auto take = [&](Buf& b, size_t bytes) {
     b.off = off; b.bytes = bytes;
     off += (size_t)round_up((int64_t)(bytes > 0 ? bytes : 1), 256);
+    if (guards && L.n_guards < MAX_GUARDS) {
+      L.guard_off[L.n_guards++] = off;
+      off += GUARD_BYTES;
+    }
   };
   take(L.status, 256);
   take(L.rows_total, 256);
@@ -228,6 +241,45 @@ static int check_device() {
   } while (0)
 
 // ---------------------------------------------------------------------------
+// Guard zones between the workspace's buffers (REVFFN_FLAG_DEBUG_CHECKS): filled with a
+// position-dependent pattern when a pass starts, verified when it ends.  A kernel that
+// writes past the end of its buffer lands in one of them.
+// ---------------------------------------------------------------------------
+struct GuardTable { int n; unsigned long long off[MAX_GUARDS]; };
+
+__device__ __forceinline__ uint32_t guard_word(int zone, int i) { return 0xC0DE0000u ^ (uint32_t)(zone * 64 + i) * 2654435761u; }
+
+__global__ void guard_fill_kernel(char* __restrict__ ws, const GuardTable g) {
+  const int z = blockIdx.x, i = threadIdx.x;
+  reinterpret_cast<uint32_t*>(ws + g.off[z])[i] = guard_word(z, i);
+}
+__global__ void guard_check_kernel(const char* __restrict__ ws, const GuardTable g, int* __restrict__ status) {
+  const int z = blockIdx.x, i = threadIdx.x;
+  if (reinterpret_cast<const uint32_t*>(ws + g.off[z])[i] != guard_word(z, i)) set_status(status, REVFFN_ERR_CANARY);
+}
+
+// Guards that lie inside the first `limit` bytes of the workspace (a forward pass may own only fwd_bytes).
+static GuardTable guard_table(const WsLayout& L, size_t limit) {
+  GuardTable g;
+  g.n = 0;
+  for (int i = 0; i < L.n_guards; ++i)
+    if (L.guard_off[i] + GUARD_BYTES <= limit) g.off[g.n++] = L.guard_off[i];
+  return g;
+}
+static int guards_fill(const WsLayout& L, size_t limit, char* ws, cudaStream_t st) {
+  const GuardTable g = guard_table(L, limit);
+  if (g.n == 0) return REVFFN_OK;
+  guard_fill_kernel<<<g.n, GUARD_BYTES / 4, 0, st>>>(ws, g);
+  return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
+}
+static int guards_check(const WsLayout& L, size_t limit, char* ws, cudaStream_t st) {
+  const GuardTable g = guard_table(L, limit);
+  if (g.n == 0) return REVFFN_OK;
+  guard_check_kernel<<<g.n, GUARD_BYTES / 4, 0, st>>>(ws, g, reinterpret_cast<int*>(ws + L.status.off));
+  return cudaGetLastError() == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------
 // Launch context
 // ---------------------------------------------------------------------------
 template <typename T>
@@ -298,7 +350,8 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     CK(cudaMemcpyAsync(c.ws + L.gates.off, rec + R.gates_off, tk, cudaMemcpyDeviceToDevice, st));
     CK(cudaMemcpyAsync(c.ws + L.sgate.off, rec + R.sgate_off, (size_t)Tn * 4, cudaMemcpyDeviceToDevice, st));
   } else {
-    { ProfScope ps(TG_FOLD, st);
+    if (!(D.flags & REVFFN_FLAG_ROUTER_FOLDED)) {     // else the folded router of an earlier call is still in the workspace
+    ProfScope ps(TG_FOLD, st);
     if (d <= FOLD_SLICES * fold_slice_rows<T>()) {
       CK(launch_fold_router_mma<T>(reinterpret_cast<const T*>(c.W.w_router), reinterpret_cast<const T*>(c.W.ws_sgate),
                                    w_up, E, d, h, c.template p<double>(L.w_rc_part), c.template p<double>(L.w_rc), st));
@@ -312,7 +365,8 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     CK(launch_router_topk(y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, c.template p<double>(L.w_rc),
                           c.W.b_router, Tn, h, E, k, Is > 0 ? 1 : 0, idx_in, c.template p<int32_t>(L.idx),
                           c.template p<float>(L.gates), c.template p<float>(L.sgate), idx_user,
-                          gate_all ? c.template p<float>(L.prob) : nullptr, st));
+                          gate_all ? c.template p<float>(L.prob) : nullptr, c.template p<int>(L.status),
+                          (D.flags & REVFFN_FLAG_DEBUG_CHECKS) ? 1 : 0, st));
     }
     if (idx_user && records) {      // complete the record the kernel has started with the indices
       char* rec = reinterpret_cast<char*>(idx_user);
@@ -326,7 +380,8 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
   CK(cudaMemsetAsync(c.ws + L.row_gate.off, 0, L.row_gate.bytes, st));
   { ProfScope ps(TG_MAP, st);
   map_rank_kernel<<<L.n_chunks, 256, (size_t)MAP_CHUNK * k * 4, st>>>(
-      c.template p<int32_t>(L.idx), Tn, k, E, c.template p<int32_t>(L.local_rank), c.template p<int32_t>(L.chunk_cnt));
+      c.template p<int32_t>(L.idx), Tn, k, E, c.template p<int32_t>(L.local_rank), c.template p<int32_t>(L.chunk_cnt),
+      c.template p<int>(L.status));
   }
   CK(cudaGetLastError());
   { ProfScope ps(TG_MAP, st);
@@ -660,11 +715,19 @@ static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weight
   g_prof.pass = (int)pass;
   c.tc = std::is_same<T, bf16>::value && !(D.flags & REVFFN_FLAG_FORCE_SIMT);
   if (c.tc) CKR(tc_prepare());
-  CK(cudaMemsetAsync(c.ws + L.status.off, 0, L.status.bytes, st));
+  if (!(D.flags & REVFFN_FLAG_KEEP_STATUS)) CK(cudaMemsetAsync(c.ws + L.status.off, 0, L.status.bytes, st));
   if (D.tokens == 0) return REVFFN_OK;   // empty batch: nothing to compute, gradients untouched
-  if (pass == PASS_BWD) return run_backward(c, y1, in2, out, *G, idx_in);
-  CKR(run_branch(c, y1, idx_in, idx_out, (D.flags & REVFFN_FLAG_SAVE_ACTIVATIONS) != 0));
-  return run_couple(c, in2, pass == PASS_FWD ? 1.f : -1.f, out);
+  const bool big_ws = pass == PASS_BWD || (D.flags & REVFFN_FLAG_SAVE_ACTIVATIONS);
+  const size_t ws_limit = big_ws ? L.bwd_bytes : L.fwd_bytes;
+  if (L.n_guards) CKR(guards_fill(L, ws_limit, c.ws, st));
+  if (pass == PASS_BWD) {
+    CKR(run_backward(c, y1, in2, out, *G, idx_in));
+  } else {
+    CKR(run_branch(c, y1, idx_in, idx_out, (D.flags & REVFFN_FLAG_SAVE_ACTIVATIONS) != 0));
+    CKR(run_couple(c, in2, pass == PASS_FWD ? 1.f : -1.f, out));
+  }
+  if (L.n_guards) CKR(guards_check(L, ws_limit, c.ws, st));
+  return REVFFN_OK;
 }
 
 static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1,
@@ -708,6 +771,8 @@ static __device__ __align__(256) double g_route_scratch[REVFFN_ROUTE_NOALLOC_MAX
 // symbol itself is only a handle, not something a kernel may dereference.
 static double* route_scratch_ptr(int* err) {
   static double* ptr[64] = {nullptr};
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = REVFFN_ERR_CUDA; return nullptr; }
   if (!ptr[dev]) {
@@ -727,7 +792,7 @@ static int route_noalloc_launch(const revffn_moe_desc& D, const revffn_moe_weigh
   CK(launch_fold_router<T>(reinterpret_cast<const T*>(W.w_router), reinterpret_cast<const T*>(W.ws_sgate),
                            reinterpret_cast<const T*>(W.w_up), E, d, h, w_rc, st));
   CK(launch_router_topk(y1, D.ld_stream, W.norm_gamma, D.norm_eps, norm_none, w_rc, W.b_router, D.tokens, h, E,
-                        D.top_k, D.d_shared > 0 ? 1 : 0, nullptr, idx, gates, sgate, nullptr, nullptr, st));
+                        D.top_k, D.d_shared > 0 ? 1 : 0, nullptr, idx, gates, sgate, nullptr, nullptr, nullptr, 0, st));
   g_prof.launches += 2;
   return REVFFN_OK;
 }
@@ -784,6 +849,9 @@ const char* revffn_strerror(int code) {
     case REVFFN_ERR_DEVICE_WAIT: return "a bounded device-side wait expired";
     case REVFFN_ERR_UNSUPPORTED: return "not supported";
     case REVFFN_ERR_NOALLOC_LIMIT: return "problem exceeds the fixed scratch of the no-allocation entry point";
+    case REVFFN_ERR_INDEX: return "an expert index supplied by the caller is out of range";
+    case REVFFN_ERR_CANARY: return "a guard zone between workspace buffers was overwritten";
+    case REVFFN_ERR_NONFINITE: return "a router logit is not finite";
     default: return "unknown error";
   }
 }
@@ -808,6 +876,14 @@ int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* 
       if (bytes) *bytes = t.b->bytes;
       return REVFFN_OK;
     }
+  if (strncmp(name, "guard", 5) == 0 && name[5] >= '0' && name[5] <= '9') {
+    const int i = atoi(name + 5);
+    if (i < L.n_guards) {
+      if (offset) *offset = L.guard_off[i];
+      if (bytes) *bytes = GUARD_BYTES;
+      return REVFFN_OK;
+    }
+  }
   return REVFFN_ERR_UNSUPPORTED;
 }
 
@@ -816,6 +892,8 @@ int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* 
 static cudaEvent_t* step_events(int* err) {
   static cudaEvent_t ev[64][7];
   static bool made[64] = {false};
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = REVFFN_ERR_CUDA; return nullptr; }
   if (!made[dev]) {
@@ -856,9 +934,11 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
   float* x2r = reinterpret_cast<float*>(sp + 4 * slot);
   float* dy1 = reinterpret_cast<float*>(sp + 5 * slot);
   // the inverse and the gradient pass share one evaluation of the branch
+  // the status word is cleared once (by the first forward call); every later pass keeps it, so that
+  // revffn_moe_status reports the first device-side error of the whole step
   revffn_moe_desc d_inv = *desc, d_bwd = *desc;
-  d_inv.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS;
-  d_bwd.flags |= REVFFN_FLAG_REUSE_ACTIVATIONS;
+  d_inv.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS | REVFFN_FLAG_KEEP_STATUS | REVFFN_FLAG_ROUTER_FOLDED;
+  d_bwd.flags |= REVFFN_FLAG_REUSE_ACTIVATIONS | REVFFN_FLAG_KEEP_STATUS;
   // With a copy stream, what a pass does not need right away travels beside the passes: the second half of
   // the tokens comes in while the forward pass works on the first half (tokens are independent through the
   // branch, so two half-batch forward calls give the same y2), dy2 comes in during forward and inverse, y2 goes
@@ -888,6 +968,7 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
     revffn_moe_desc d_a = *desc, d_b = *desc;
     d_a.tokens = T0;
     d_b.tokens = desc->tokens - T0;
+    d_b.flags |= REVFFN_FLAG_KEEP_STATUS | REVFFN_FLAG_ROUTER_FOLDED;
     CK(cudaStreamWaitEvent(st, ev[1], 0));
     CKR(revffn_moe_forward(&d_a, w, y1, x2, y2, nullptr, ws, ws_bytes, cuda_stream));
     CK(cudaStreamWaitEvent(st, ev[2], 0));
@@ -965,8 +1046,11 @@ int revffn_moe_stack_forward(const revffn_moe_desc* desc, const revffn_moe_weigh
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   revffn_moe_desc d = *desc;
   if (cache) d.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS;
-  // with a cache every layer runs in its own slot: the shared workspace still reports "no error"
-  if (cache && ws && ws_bytes >= 256) CK(cudaMemsetAsync(ws, 0, 256, st));
+  // Without a cache all layers share `ws`: its status word is cleared here, once, and every layer keeps it, so
+  // that it reports the first device-side error of the whole sweep (a later layer would otherwise erase it).
+  // With a cache every layer runs in, and reports through, its own slot; the shared workspace reads "no error".
+  if (ws && ws_bytes >= 256) CK(cudaMemsetAsync(ws, 0, 256, st));
+  if (!cache) d.flags |= REVFFN_FLAG_KEEP_STATUS;
   for (int l = 0; l < n_blocks; ++l) {
     float* P = (l & 1) ? stream_b : stream_a;
     float* R = (l & 1) ? stream_a : stream_b;
@@ -1002,9 +1086,10 @@ int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weig
   const size_t idx_stride = routing_stride(*desc);     // bytes
   const size_t ws_need = plan_workspace(*desc).bwd_bytes;
   revffn_moe_desc d_inv = *desc, d_bwd = *desc;
-  d_inv.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS;
-  d_bwd.flags |= REVFFN_FLAG_REUSE_ACTIVATIONS;
-  if (cache && ws && ws_bytes >= 256) CK(cudaMemsetAsync(ws, 0, 256, reinterpret_cast<cudaStream_t>(cuda_stream)));
+  d_inv.flags |= REVFFN_FLAG_SAVE_ACTIVATIONS | REVFFN_FLAG_KEEP_STATUS;
+  // with a cache the slot's word still holds what the layer's forward pass reported: keep it as well
+  d_bwd.flags |= REVFFN_FLAG_REUSE_ACTIVATIONS | REVFFN_FLAG_KEEP_STATUS;
+  if (ws && ws_bytes >= 256) CK(cudaMemsetAsync(ws, 0, 256, reinterpret_cast<cudaStream_t>(cuda_stream)));
   for (int l = n_blocks - 1; l >= 0; --l) {
     float* P = (l & 1) ? stream_b : stream_a;
     float* R = (l & 1) ? stream_a : stream_b;
@@ -1032,9 +1117,9 @@ int revffn_moe_route_noalloc(const revffn_moe_desc* desc, const revffn_moe_weigh
   if (r != REVFFN_OK) return r;
   if (desc->tokens > 0 && (!y1 || !topk_idx_out || !gates_out || !sgate_out)) return REVFFN_ERR_NULL;
   if (!aligned16(y1) || !aligned16(topk_idx_out)) return REVFFN_ERR_ALIGN;
+  if (desc->flags & REVFFN_FLAG_GATE_SOFTMAX_ALL) return REVFFN_ERR_UNSUPPORTED;   // needs the softmax over all E logits
   const int64_t need = (int64_t)(desc->n_experts + 1) * (desc->d_model / 2);
-  if (need > REVFFN_ROUTE_NOALLOC_MAX_ELEMS || router_smem_bytes(desc->n_experts) > 200 * 1024)
-    return REVFFN_ERR_NOALLOC_LIMIT;
+  if (need > REVFFN_ROUTE_NOALLOC_MAX_ELEMS) return REVFFN_ERR_NOALLOC_LIMIT;
   r = check_device();
   if (r != REVFFN_OK) return r;
   if (desc->tokens == 0) return REVFFN_OK;
@@ -1044,6 +1129,17 @@ int revffn_moe_route_noalloc(const revffn_moe_desc* desc, const revffn_moe_weigh
   if (desc->weight_dtype == REVFFN_BF16)
     return route_noalloc_launch<bf16>(*desc, *w, y1, scratch, topk_idx_out, gates_out, sgate_out, st);
   return route_noalloc_launch<float>(*desc, *w, y1, scratch, topk_idx_out, gates_out, sgate_out, st);
+}
+
+int revffn_dbg_check_guards(const revffn_moe_desc* desc, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  if (!ws) return REVFFN_ERR_NULL;
+  if (!(desc->flags & REVFFN_FLAG_DEBUG_CHECKS)) return REVFFN_ERR_UNSUPPORTED;
+  WsLayout L = plan_workspace(*desc);
+  if (ws_bytes < L.fwd_bytes) return REVFFN_ERR_WORKSPACE;
+  return guards_check(L, ws_bytes < L.bwd_bytes ? L.fwd_bytes : L.bwd_bytes, reinterpret_cast<char*>(ws),
+                      reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
 int revffn_prof_enable(int on) {
@@ -1097,6 +1193,7 @@ int revffn_dbg_gemm(const revffn_dbg_gemm_args* a, int32_t* status_word_dev, voi
   p.b_group_stride = a->b_group_stride; p.c_group_stride = a->c_group_stride;
   p.a_col0 = a->a_col0; p.b_col0 = a->b_col0;
   p.tok_chunks = reinterpret_cast<const int4*>(a->tok_chunks); p.no_pair = a->no_pair;
+  p.dbg_wait_cycles = a->wait_cycles; p.dbg_starve = a->starve_operands;
   p.status = status_word_dev;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (a->use_simt) return launch_gemm_simt<bf16>(p, st) == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;

@@ -9,6 +9,8 @@
 //   combine_rows       Z[t] = sum_s O[row(t,s)] + sgate_t * S[t]
 #pragma once
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace revffn {
@@ -293,7 +295,8 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
                    int norm_none, const double* __restrict__ w_rc, const float* __restrict__ b_router,
                    int tokens, int h, int E, int k, int has_shared, const int32_t* __restrict__ idx_in,
                    int32_t* __restrict__ idx_out, float* __restrict__ gate_out, float* __restrict__ sgate_out,
-                   int32_t* __restrict__ idx_user, float* __restrict__ prob_out) {
+                   int32_t* __restrict__ idx_user, float* __restrict__ prob_out, int* __restrict__ status,
+                   int check_finite) {
   extern __shared__ __align__(16) double smem_d[];
   const int EP = E + 1;                       // logits per token incl. the shared-gate row
   double* ns = smem_d;                        // [RT_TOK][RT_LD]  stream chunk, one row per token
@@ -409,10 +412,24 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
     const double* L = Ls + tt * EP;
     double sel[8];
     int seli[8];
+    if (check_finite) {
+      // a NaN or infinite logit (non-finite input or weight) makes the selection meaningless: report it
+      bool bad = false;
+      for (int e = lane; e < EP; e += 32) bad |= !isfinite(L[e]);
+      if (__any_sync(0xffffffffu, bad) && lane == 0) set_status(status, REVFFN_ERR_NONFINITE);
+    }
     if (idx_in) {
+      // Expert sets from the caller.  An index outside [0, E) is reported and kept as -1: the
+      // permutation maps skip such an entry, and its gate weight is zero.
 #pragma unroll
       for (int s = 0; s < 8; ++s)
-        if (s < k) { seli[s] = idx_in[(int64_t)t * k + s]; sel[s] = L[seli[s]]; }
+        if (s < k) {
+          const int e = idx_in[(int64_t)t * k + s];
+          const bool in_range = (unsigned)e < (unsigned)E;
+          if (!in_range && lane == 0) set_status(status, REVFFN_ERR_INDEX);
+          seli[s] = in_range ? e : -1;
+          sel[s] = in_range ? L[e] : __longlong_as_double(0xfff0000000000000LL);
+        }
     } else {
       // candidates of this lane: e = lane + 32 j
       unsigned taken = 0u;                    // bit j set: candidate j already selected
@@ -493,14 +510,17 @@ inline size_t router_smem_bytes(int E) {
 inline cudaError_t launch_router_topk(const float* y, int64_t ld, const float* gamma, float eps, int norm_none,
                                       const double* w_rc, const float* b_router, int tokens, int h, int E, int k,
                                       int has_shared, const int32_t* idx_in, int32_t* idx_out, float* gate_out,
-                                      float* sgate_out, int32_t* idx_user, float* prob_out, cudaStream_t st) {
+                                      float* sgate_out, int32_t* idx_user, float* prob_out, int* status,
+                                      int check_finite, cudaStream_t st) {
   static size_t raised[64] = {0};
+  static std::mutex mu;
   const size_t smem = router_smem_bytes(E);
   if (smem > 48 * 1024) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
     if (raised[dev] < smem) {
       e = cudaFuncSetAttribute(router_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
@@ -509,7 +529,7 @@ inline cudaError_t launch_router_topk(const float* y, int64_t ld, const float* g
   }
   router_topk_kernel<<<(unsigned)ceil_div(tokens, RT_TOK), 256, smem, st>>>(
       y, ld, gamma, eps, norm_none, w_rc, b_router, tokens, h, E, k, has_shared, idx_in, idx_out, gate_out,
-      sgate_out, idx_user, prob_out);
+      sgate_out, idx_user, prob_out, status, check_finite);
   return cudaGetLastError();
 }
 
@@ -521,13 +541,20 @@ inline cudaError_t launch_router_topk(const float* y, int64_t ld, const float* g
 //   map_scan:   per expert totals, padded offsets, per-chunk bases, tile->expert
 //   map_assign: row of each entry; row -> token; row -> gate weight
 // ---------------------------------------------------------------------------
+// An entry outside [0, E) (possible only in expert sets handed in by the caller) matches no expert: it gets
+// no rank and no row, map_assign marks it with row -1, and every later step skips it.  It is reported once here.
 __global__ void map_rank_kernel(const int32_t* __restrict__ idx, int tokens, int k, int E,
-                                int32_t* __restrict__ local_rank, int32_t* __restrict__ chunk_cnt) {
+                                int32_t* __restrict__ local_rank, int32_t* __restrict__ chunk_cnt,
+                                int* __restrict__ status) {
   extern __shared__ int32_t sm_i[];
   int chunk = blockIdx.x;
   int64_t e0 = (int64_t)chunk * MAP_CHUNK * k;
   int n = (int)min((int64_t)MAP_CHUNK * k, (int64_t)tokens * k - e0);
-  for (int i = threadIdx.x; i < n; i += blockDim.x) sm_i[i] = idx[e0 + i];
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int e = idx[e0 + i];
+    sm_i[i] = e;
+    if ((unsigned)e >= (unsigned)E) set_status(status, REVFFN_ERR_INDEX);
+  }
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
     int c = 0;
@@ -589,6 +616,7 @@ __global__ void map_assign_kernel(const int32_t* __restrict__ idx, const float* 
   if (i >= (int64_t)tokens * k) return;
   int t = (int)(i / k);
   int e = idx[i];
+  if ((unsigned)e >= (unsigned)E) { tok_row[i] = -1; return; }      // reported by map_rank
   int chunk = t / MAP_CHUNK;
   int row = expert_off[e] + chunk_base[(int64_t)chunk * E + e] + local_rank[i];
   tok_row[i] = row;
@@ -634,6 +662,7 @@ __global__ void combine_rows_kernel(const T* __restrict__ O, const int32_t* __re
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
     Vec8<T> v;
     for (int s = 0; s < k; ++s) {
+      if (rows[s] < 0) continue;      // entry with an out-of-range expert index
       v.load(O + (int64_t)rows[s] * width + c);
       v.get(f);
 #pragma unroll

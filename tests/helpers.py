@@ -14,6 +14,21 @@ def rel_l2(a, b) -> float:
     return float(np.linalg.norm(a - b) / (den if den > 0 else 1.0))
 
 
+def max_block_rel_l2(a, b, axis: int = 0):
+    """Largest relative L2 error over the slices along `axis` (one expert of a stacked weight gradient,
+    one token row of a stream), skipping slices whose reference is all zero (those must be all zero in `a`
+    too).  A per-tensor norm cannot see one wrong slice inside a large tensor; this can."""
+    a = np.moveaxis(np.asarray(a, dtype=np.float64), axis, 0)
+    b = np.moveaxis(np.asarray(b, dtype=np.float64), axis, 0)
+    a = a.reshape(a.shape[0], -1)
+    b = b.reshape(b.shape[0], -1)
+    den = np.linalg.norm(b, axis=1)
+    num = np.linalg.norm(a - b, axis=1)
+    zero = den == 0
+    assert (num[zero] == 0).all(), "non-zero values where the reference slice is exactly zero"
+    return float((num[~zero] / den[~zero]).max()) if (~zero).any() else 0.0
+
+
 def to_device_weights(cfg: BlockConfig, w: dict) -> dict:
     wdt = torch.bfloat16 if cfg.weight_dtype == "bf16" else torch.float32
     out = {}
