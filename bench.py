@@ -87,6 +87,7 @@ def gemm_flops(cfg, routed_rows):
         "gemm_shared_du": 2 * T * 2 * Is * d, "wgrad_shared_gate": 2 * T * Is * d, "wgrad_shared_up": 2 * T * Is * d,
         "gemm_expert_dh_dswiglu": 2 * R * d * I, "gemm_expert_du": 2 * R * 2 * I * d,
         "wgrad_expert_down": 2 * R * d * I, "wgrad_expert_gate": 2 * R * I * d, "wgrad_expert_up": 2 * R * I * d,
+        "wgrad_expert_gate_up": 2 * R * 2 * I * d,
         "gemm_dn": 2 * T * d * h, "wgrad_p_up": 2 * T * d * h,
     }
 

@@ -219,6 +219,48 @@ int revffn_moe_backward(const revffn_moe_desc* desc, const revffn_moe_weights* w
                         const revffn_moe_grads* grads, const int32_t* topk_idx_in,
                         void* ws, size_t ws_bytes, void* cuda_stream);
 
+/*
+ * Backward pass with the optimiser step fused into the weight-gradient products (Sec. 3.3: the schedule trains
+ * the adapters in stage 1 and adapters plus experts in stage 2; the paper's optimiser is not this one -- plain
+ * SGD is what can be applied tile by tile without optimiser state, and it is enough to show the mechanism).
+ * For every matrix named in sgd->mask the product that would have produced its fp32 gradient applies
+ *     W <- W - lr * dL/dW
+ * to the weight itself, tile by tile, in its epilogue, and the gradient is never written: at the benchmark
+ * block shape that saves the 2.1 GB of fp32 expert gradients.  Without a master copy the step is taken on the
+ * stored weight (bf16 weights: read, updated in fp32, rounded to nearest even; steps much smaller than the
+ * weight's last bit are lost, as in any pure-bf16 update).  With a master copy (sgd->m_X, fp32, same shape) the
+ * step is taken there and W receives the rounded master value.
+ *   - `w` is modified: the matrices named in the mask are written through their (const) pointers.  Every product
+ *     of this call that reads such a matrix runs before the product that updates it.
+ *   - grads: as in revffn_moe_backward for everything NOT in the mask (the vectors norm_gamma, ws_sgate, w_router,
+ *     b_router are never fused); a matrix may not be both in the mask and have a gradient pointer
+ *     (REVFFN_ERR_UNSUPPORTED).  grads->accumulate applies to the written gradients only.
+ *   - Stage masks: stage 1 = REVFFN_UPD_W_UP | REVFFN_UPD_W_DOWN, stage 2 = REVFFN_UPD_ALL.
+ *   - A workspace that caches the folded router (REVFFN_FLAG_ROUTER_FOLDED) is stale once w_up has been updated.
+ * revffn_moe_stack_backward_sgd: the reversible sweep of revffn_moe_stack_backward with one revffn_moe_sgd per
+ * layer (HOST array of n_blocks structs, or NULL for none): layer l's weights are updated right after the last
+ * use of layer l in the sweep, so the sweep is one training step of the whole stack with no gradient buffers
+ * for the matrices in the masks.
+ */
+#define REVFFN_UPD_W_UP 1u
+#define REVFFN_UPD_W_DOWN 2u
+#define REVFFN_UPD_W_GATE 4u
+#define REVFFN_UPD_W_UPX 8u
+#define REVFFN_UPD_W_DOWNX 16u
+#define REVFFN_UPD_WS_GATE 32u
+#define REVFFN_UPD_WS_UP 64u
+#define REVFFN_UPD_WS_DOWN 128u
+#define REVFFN_UPD_ALL 255u
+typedef struct {
+  float lr;
+  uint32_t mask;          /* REVFFN_UPD_* bits                                              */
+  float *m_w_up, *m_w_down, *m_w_gate, *m_w_upx, *m_w_downx, *m_ws_gate, *m_ws_up, *m_ws_down;   /* fp32 master copies or NULL */
+} revffn_moe_sgd;
+int revffn_moe_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weights* w,
+                            const float* y1, const float* dy2, float* dy1_inout,
+                            const revffn_moe_grads* grads, const revffn_moe_sgd* sgd, const int32_t* topk_idx_in,
+                            void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Synchronise the stream and copy the workspace's device status word to
  * *device_status (host pointer): 0 or a negative revffn_error.  (No paper counterpart.) */
 int revffn_moe_status(const void* ws, void* cuda_stream, int32_t* device_status);
@@ -266,6 +308,11 @@ int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weig
                               float* stream_a, float* stream_b, float* grad_a, float* grad_b,
                               const revffn_moe_grads* grads, const int32_t* topk_idx, void* cache,
                               size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream);
+
+int revffn_moe_stack_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                                  float* stream_a, float* stream_b, float* grad_a, float* grad_b,
+                                  const revffn_moe_grads* grads, const revffn_moe_sgd* sgd, const int32_t* topk_idx,
+                                  void* cache, size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Size of one routing record (REVFFN_FLAG_ROUTING_RECORD), a multiple of 16.  (Planner; no paper counterpart.) */
 int revffn_moe_routing_record_bytes(const revffn_moe_desc* desc, size_t* bytes);
@@ -324,10 +371,10 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
  *   - (E + 1) * h <= REVFFN_ROUTE_NOALLOC_MAX_ELEMS (512 KB of scratch, held by
  *     every device that loads the library until the process exits); otherwise
  *     REVFFN_ERR_NOALLOC_LIMIT and nothing is launched.  The router kernel keeps
- *     a 64-token tile of logits in shared memory, 8 * 64 * (E + 1) bytes plus
- *     37 KB of operand staging: above 48 KB in total (E >= 23) the first call on
+ *     a 32-token tile of logits in shared memory, 8 * 32 * (E + 1) bytes plus
+ *     27.3 KB of operand staging: above 48 KB in total (E >= 83) the first call on
  *     a device raises the kernel's dynamic shared-memory limit, which is a
- *     function attribute, not an allocation; E = 256 needs 166 KB.
+ *     function attribute, not an allocation; E = 256 needs 92 KB.
  *   - REVFFN_FLAG_GATE_SOFTMAX_ALL is not supported here (its gates need the
  *     softmax over all E logits, which this entry point does not form):
  *     REVFFN_ERR_UNSUPPORTED, nothing is launched.  Other flags are ignored.

@@ -303,6 +303,18 @@ def backward(p, Y1, dY2, k: int, eps: float = 1e-6, norm: str = "rms", route_ove
 
 
 # --------------------------------------------------------------------------- #
+# One optimiser step on the gradients above (Sec. 3.3 trains the adapters, then adapters
+# and experts, with a first-order optimiser; plain SGD is the step written out here).
+# --------------------------------------------------------------------------- #
+def sgd_step(p, grads, lr: float, names):
+    """W <- W - lr * dL/dW for the named weights (fp64); the others are returned as they are."""
+    out = dict(p)
+    for n in names:
+        out[n] = _w(p, n) - lr * np.asarray(grads[n], dtype=F64)
+    return out
+
+
+# --------------------------------------------------------------------------- #
 # A stack of coupling branches (Sec. 3.1: the two output streams of a layer are
 # the input of the next one; Sec. 2: inputs are rebuilt layer by layer from the
 # outputs during back-propagation, nothing is cached).

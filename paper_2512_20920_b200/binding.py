@@ -51,6 +51,28 @@ class Grads(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES] + [("accumulate", C.c_int32)]
 
 
+UPD_NAMES = ("w_up", "w_down", "w_gate", "w_upx", "w_downx", "ws_gate", "ws_up", "ws_down")     # bit i of the mask
+UPD_ALL = 255
+
+
+class Sgd(C.Structure):
+    """revffn_moe_sgd: learning rate, mask of the matrices updated in place, optional fp32 master copies."""
+    _fields_ = [("lr", C.c_float), ("mask", C.c_uint32)] + [("m_" + n, C.c_void_p) for n in UPD_NAMES]
+
+
+def upd_mask(names) -> int:
+    """REVFFN_UPD_* mask of the named matrices."""
+    return sum(1 << UPD_NAMES.index(n) for n in names)
+
+
+def make_sgd(lr: float, names, masters: Optional[Dict[str, torch.Tensor]] = None) -> Sgd:
+    masters = masters or {}
+    for n, t in masters.items():
+        if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+            raise ValueError(f"master copy {n}: need a contiguous fp32 CUDA tensor")
+    return Sgd(lr=lr, mask=upd_mask(names), **{"m_" + n: _ptr(masters.get(n)) for n in UPD_NAMES})
+
+
 ATTN_WEIGHT_NAMES = ("norm_gamma", "w_up", "w_down", "w_q", "w_k", "w_v", "w_o", "b_q", "b_k", "b_v")
 _ATTN_F32_ALWAYS = ("norm_gamma", "b_q", "b_k", "b_v")
 
@@ -98,6 +120,12 @@ def _load() -> C.CDLL:
     lib.revffn_moe_inverse.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, vp, vp, sz, vp]
     lib.revffn_moe_backward.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, C.POINTER(Grads), vp, vp,
                                         sz, vp]
+    lib.revffn_moe_backward_sgd.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, C.POINTER(Grads), C.POINTER(Sgd),
+                                            vp, vp, sz, vp]
+    lib.revffn_moe_backward_sgd.restype = C.c_int
+    lib.revffn_moe_stack_backward_sgd.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp,
+                                                  C.POINTER(Grads), C.POINTER(Sgd), vp, vp, sz, vp, sz, vp]
+    lib.revffn_moe_stack_backward_sgd.restype = C.c_int
     lib.revffn_moe_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
     lib.revffn_strerror.argtypes = [C.c_int]
     lib.revffn_strerror.restype = C.c_char_p
@@ -200,6 +228,14 @@ def revffn_moe_backward(desc: Desc, w: Weights, y1, dy2, dy1_inout, grads: Grads
            "revffn_moe_backward")
 
 
+def revffn_moe_backward_sgd(desc: Desc, w: Weights, y1, dy2, dy1_inout, grads: Grads, sgd: Sgd, topk_idx_in, ws,
+                            stream: Optional[int] = None):
+    _check(lib.revffn_moe_backward_sgd(C.byref(desc), C.byref(w), _ptr(y1), _ptr(dy2), _ptr(dy1_inout), C.byref(grads),
+                                       C.byref(sgd), _ptr(topk_idx_in), _ptr(ws), ws.numel() * ws.element_size(),
+                                       stream if stream is not None else _stream()),
+           "revffn_moe_backward_sgd")
+
+
 def revffn_moe_status(ws, stream: Optional[int] = None) -> int:
     out = C.c_int32(0)
     _check(lib.revffn_moe_status(_ptr(ws), stream if stream is not None else _stream(), C.byref(out)),
@@ -265,6 +301,15 @@ def revffn_moe_stack_backward(desc: Desc, weights, n_blocks: int, stream_a, stre
                                          _ptr(grad_a), _ptr(grad_b), grads, _ptr(topk_idx), _ptr(cache),
                                          _nbytes(cache), _ptr(ws), _nbytes(ws),
                                          stream if stream is not None else _stream()), "revffn_moe_stack_backward")
+
+
+def revffn_moe_stack_backward_sgd(desc: Desc, weights, n_blocks: int, stream_a, stream_b, grad_a, grad_b, grads, sgd,
+                                  topk_idx, cache, ws, stream: Optional[int] = None):
+    """`sgd`: ctypes array of n_blocks Sgd structs (or None)."""
+    _check(lib.revffn_moe_stack_backward_sgd(C.byref(desc), weights, n_blocks, _ptr(stream_a), _ptr(stream_b),
+                                             _ptr(grad_a), _ptr(grad_b), grads, sgd, _ptr(topk_idx), _ptr(cache),
+                                             _nbytes(cache), _ptr(ws), _nbytes(ws),
+                                             stream if stream is not None else _stream()), "revffn_moe_stack_backward_sgd")
 
 
 def revffn_prof_enable(on: bool) -> bool:
@@ -354,15 +399,20 @@ class Block:
         return x2
 
     def backward(self, y1, dy2, dy1_inout, grads: Optional[Dict[str, torch.Tensor]] = None, accumulate: bool = False,
-                 topk_idx_in=None, reuse: bool = False, ws=None, flags: int = 0):
-        """reuse=True: the workspace still holds what forward/inverse(save=True) left for this y1."""
+                 topk_idx_in=None, reuse: bool = False, ws=None, flags: int = 0, sgd: Optional[Sgd] = None):
+        """reuse=True: the workspace still holds what forward/inverse(save=True) left for this y1.
+        sgd: a Sgd struct (make_sgd) -- the matrices in its mask are updated in place instead of having their
+        gradients written (revffn_moe_backward_sgd)."""
         grads = grads or {}
         for n, t in grads.items():
             if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
                 raise ValueError(f"gradient {n}: need a contiguous fp32 CUDA tensor")
         g = Grads(**{n: _ptr(grads.get(n)) for n in WEIGHT_NAMES}, accumulate=1 if accumulate else 0)
-        revffn_moe_backward(self._desc((FLAG_REUSE_ACTIVATIONS if reuse else 0) | flags), self.w, y1, dy2, dy1_inout, g,
-                            topk_idx_in, self.ws if ws is None else ws)
+        d = self._desc((FLAG_REUSE_ACTIVATIONS if reuse else 0) | flags)
+        if sgd is not None:
+            revffn_moe_backward_sgd(d, self.w, y1, dy2, dy1_inout, g, sgd, topk_idx_in, self.ws if ws is None else ws)
+        else:
+            revffn_moe_backward(d, self.w, y1, dy2, dy1_inout, g, topk_idx_in, self.ws if ws is None else ws)
         return dy1_inout
 
     def grads_struct(self, grads: Optional[Dict[str, torch.Tensor]] = None, accumulate: bool = False) -> Grads:
@@ -513,6 +563,12 @@ def revffn_block_status(ws, stream=None) -> int:
     return out.value
 
 
+def stage_update_mask(stage: int) -> int:
+    """REVFFN_UPD_* mask of the MoE branch's matrices that a stage of the schedule trains (Sec. 3.3): stage 1 the
+    projection adapters, stage 2 adapters and experts (the vectors and the frozen router are never fused)."""
+    return upd_mask([n for n in trainable_names(stage)[1] if n in UPD_NAMES])
+
+
 def trainable_names(stage: int):
     """Which weights receive gradients in the two stages of the paper's schedule (Sec. 3.3): stage 1 trains only
     the projection adapters of both branches, stage 2 everything except the MoE router, which stays frozen.
@@ -628,7 +684,15 @@ class Stack:
     def forward(self, stream_a, stream_b, topk_idx=None):
         revffn_moe_stack_forward(self.desc, self.w, self.n_blocks, stream_a, stream_b, topk_idx, self.cache, self.ws)
 
-    def backward(self, stream_a, stream_b, grad_a, grad_b, grads_array, topk_idx=None):
+    def backward(self, stream_a, stream_b, grad_a, grad_b, grads_array, topk_idx=None, sgd=None):
+        """sgd: list of n_blocks Sgd structs -- one reversible sweep then is one SGD step of the whole stack."""
+        if sgd is not None:
+            if len(sgd) != self.n_blocks:
+                raise ValueError("one Sgd struct per layer")
+            arr = (Sgd * max(self.n_blocks, 1))(*sgd)
+            revffn_moe_stack_backward_sgd(self.desc, self.w, self.n_blocks, stream_a, stream_b, grad_a, grad_b,
+                                          grads_array, arr, topk_idx, self.cache, self.ws)
+            return
         revffn_moe_stack_backward(self.desc, self.w, self.n_blocks, stream_a, stream_b, grad_a, grad_b, grads_array,
                                   topk_idx, self.cache, self.ws)
 

@@ -44,9 +44,9 @@ struct GemmProblem {
   int accumulate;     // EPI_WGRAD: add to C
   const void* A; const void* B0; const void* B1;
   int64_t lda, ldb;
-  void* C; void* C1;  // C1: SWIGLU -> optional [M, 2N] pre-activations a|b; DSWIGLU -> optional g*H
+  void* C; void* C1;  // C1: SWIGLU -> optional [M, 2N] pre-activations a|b
   int64_t ldc, ldc1;
-  const float* rowscale;                       // ROWSCALE / DSWIGLU (NULL = 1)
+  const float* rowscale;                       // ROWSCALE / SWIGLU (scales H) / DSWIGLU (scales dH) (NULL = 1)
   const float* resid; int64_t ld_resid; float resid_sign;   // COUPLE: C = resid + sign * acc (fp32)
   void* ab; int64_t ld_ab;                     // DSWIGLU: [M, 2N] a|b in, da|db out (in place)
   float* dg_part; int dg_ld;                   // DSWIGLU: per (row, n-tile) partial of <acc, H>
@@ -56,6 +56,14 @@ struct GemmProblem {
   const int32_t* group_cnt;                    // GROUP_K, optional: real rows per group (the rest up to the next offset is zero padding)
   int64_t b_group_stride, c_group_stride;
   int a_col0, b_col0;
+  // EPI_WGRAD, two outputs from one product: rows >= split_m of (every group's) M belong to C2, which is laid out
+  // like C with M replaced by split_m (M must be 2 * split_m); 0 = one output.  Used for dW_gate | dW_up, whose
+  // A operand is the one [rows, 2I] buffer da|db.
+  void* C2; int split_m;
+  // EPI_WGRAD, fused SGD step: instead of writing the gradient g to C, update the weight it belongs to in place,
+  // W <- W - upd_lr * g (W of the operand type, same layout as C; upd_w2 goes with C2's rows).  With a master
+  // copy (fp32, same layout) the step is taken there and W receives the rounded result.  C / C2 may then be NULL.
+  void* upd_w; void* upd_w2; float* upd_m; float* upd_m2; float upd_lr;
   int no_pair;        // tcgen05 back end: never pair CTAs for this product
   long long dbg_wait_cycles;   // tcgen05 back end, tests: bound on every device-side wait (0 = default)
   int dbg_starve;              // tcgen05 back end, tests (needs no_pair): no operand loads are issued
@@ -197,7 +205,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmProblem p) {
           break;
         case EPI_SWIGLU: {
           float w = acc1[i][j];
-          reinterpret_cast<T*>(p.C)[(int64_t)m * p.ldc + n] = from_f32<T>(swiglu_f(v, w));
+          reinterpret_cast<T*>(p.C)[(int64_t)m * p.ldc + n] = from_f32<T>(rs * swiglu_f(v, w));
           if (p.C1) {
             T* ab = reinterpret_cast<T*>(p.C1) + (int64_t)m * p.ldc1;
             ab[n] = from_f32<T>(v);
@@ -218,12 +226,22 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmProblem p) {
           float H = dswiglu_f(a, b, rs * v, da, db);
           ab[n] = from_f32<T>(da);
           ab[p.N + n] = from_f32<T>(db);
-          if (p.C1) reinterpret_cast<T*>(p.C1)[(int64_t)m * p.ldc1 + n] = from_f32<T>(rs * H);
           dg_local[i] += v * H;
         } break;
         case EPI_WGRAD: {
-          float* o = reinterpret_cast<float*>(p.C) + (int64_t)group * p.c_group_stride + (int64_t)m * p.ldc + n;
-          *o = (p.accumulate ? *o : 0.f) + v;
+          // element index inside the output this row belongs to (first or second, see split_m)
+          const bool second = p.split_m > 0 && m >= p.split_m;
+          const int64_t at = (int64_t)group * p.c_group_stride + (int64_t)(second ? m - p.split_m : m) * p.ldc + n;
+          T* W = reinterpret_cast<T*>(second ? p.upd_w2 : p.upd_w);
+          if (W) {
+            float* master = second ? p.upd_m2 : p.upd_m;
+            const float w_new = (master ? master[at] : to_f32(W[at])) - p.upd_lr * v;
+            if (master) master[at] = w_new;
+            W[at] = from_f32<T>(w_new);
+          } else {
+            float* o = reinterpret_cast<float*>(second ? p.C2 : p.C) + at;
+            *o = (p.accumulate ? *o : 0.f) + v;
+          }
         } break;
       }
     }

@@ -62,10 +62,8 @@ constexpr long long TC_WAIT_CYCLES = 4000000000LL;       // ~2 s: bound on any s
 template <int MMA_N, int EPI, bool PAIR> struct TcCfg {
   static constexpr int B_BYTES = (PAIR ? MMA_N / 2 : MMA_N) * TC_BK * 2;
   static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
-  // The SwiGLU-backward epilogue streams its a|b operands through shared memory as well
-  // and gets a larger staging area at the price of pipeline stages.
-  static constexpr int STAGES = PAIR ? ((EPI == EPI_DSWIGLU) ? 4 : 6) : ((EPI == EPI_DSWIGLU) ? 3 : 4);
-  static constexpr int EPI_WARP_BYTES = (EPI == EPI_DSWIGLU) ? 10240 : 4096;   // staging per epilogue warp
+  static constexpr int STAGES = PAIR ? 6 : 4;
+  static constexpr int EPI_WARP_BYTES = 4096;           // staging per epilogue warp: two 32 x 32 bf16 blocks or one fp32 block
   static constexpr int TMEM_COLS = 2 * MMA_N;           // two accumulators; a power of two >= 32
   // stage ring | epilogue staging | barriers; the ring starts 1024-byte aligned and
   // every stage is a multiple of 1024 bytes, so the staging area is aligned too
@@ -187,6 +185,29 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, ui
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
 }
 
+// One product with the descriptors given as (low, high) words: the high words never change inside a kernel, and
+// the low words move by small additions, so the issuing thread carries 32-bit values only.
+template <bool PAIR>
+__device__ __forceinline__ void tc_mma_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                            uint32_t idesc, uint32_t acc) {
+  if constexpr (PAIR)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -265,6 +286,44 @@ __device__ __forceinline__ void stage32_bf16(uint8_t* buf, int r, const float* f
   for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(row + ((j ^ ((r >> 1) & 3)) << 4)) = pack8(f + 8 * j);
 }
 
+// A warp's 32-row x 32-column bf16 block (rows of 64 bytes, row stride ld elements) between global memory and
+// the staging layout above, in "distributed" form: instruction i of four moves rows 8i .. 8i+7, lane l the
+// 16-byte piece l & 3 of row 8i + (l >> 2).  Eight lanes cover four whole 64-byte row segments, so every
+// 32-byte sector a request touches is used in full, and the 512 contiguous staging bytes an instruction
+// touches spread over all banks.  rows_ok: rows of the block that exist (the rest read as zeros / are not stored).
+__device__ __forceinline__ void blk_load_dist(const bf16* g, int64_t ld, int rows_ok, int lane, uint4 (&raw)[4]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = 8 * i + (lane >> 2);
+    raw[i] = (r < rows_ok) ? __ldcg(reinterpret_cast<const uint4*>(g + (int64_t)r * ld + (lane & 3) * 8))
+                           : make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+__device__ __forceinline__ void blk_dist_to_stage(uint8_t* buf, int lane, const uint4 (&raw)[4]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = 8 * i + (lane >> 2);
+    *reinterpret_cast<uint4*>(buf + r * 64 + (((lane & 3) ^ ((r >> 1) & 3)) << 4)) = raw[i];
+  }
+}
+__device__ __forceinline__ void blk_stage_to_global(const uint8_t* buf, int lane, bf16* g, int64_t ld, int rows_ok) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = 8 * i + (lane >> 2);
+    const uint4 v = *reinterpret_cast<const uint4*>(buf + r * 64 + (((lane & 3) ^ ((r >> 1) & 3)) << 4));
+    if (r < rows_ok) *reinterpret_cast<uint4*>(g + (int64_t)r * ld + (lane & 3) * 8) = v;
+  }
+}
+
+// Logistic function from one ex2.approx and one rcp.approx (relative error about 2^-21, far inside what the
+// bf16 results around it can show).
+__device__ __forceinline__ float sigmoid_approx(float x) {
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * -1.4426950408889634f));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.f + e));
+  return r;
+}
+
 // Tile coordinates shared by the three roles.
 struct TcTile {
   int m0, n0, group, k_blocks, krow0;
@@ -334,7 +393,6 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   auto empty_bar = [&](int s) { return bars + 8u * (Cfg::STAGES + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * Cfg::STAGES + 2 + a); };
-  auto epi_bar = [&](int ew, int s) { return bars + 128u + 8u * (ew * 2 + s); };   // SwiGLU backward: operand loads
   const uint32_t drain_bar = bars + 320u;      // abort path of the MMA thread: "every product issued so far is done"
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + Cfg::BAR_OFF + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -349,7 +407,6 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   if (threadIdx.x == 0) {
     for (int s = 0; s < Cfg::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); issued[s] = 0; }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), PAIR ? 2 * TC_EPI_WARPS : TC_EPI_WARPS); }
-    for (int a = 0; a < 2 * TC_EPI_WARPS; ++a) mbar_init(epi_bar(a / 2, a % 2), 1);
     mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -377,6 +434,9 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
+    // (A version of this loop that kept per-tile "load slots" -- tensor-map pointer, destination, coordinates --
+    // in registers and issued one load per slot measured 15-40 % slower: a load whose tensor map is named through
+    // a pointer chosen at run time, rather than as the kernel parameter itself, is slow to issue.)
     if (lane == 0 && !P.starve) {
       int stage = 0;
       uint32_t phase = 0;
@@ -479,11 +539,26 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
+    // One thread issues every product of the CTA (pair), so the cycles this loop spends per K step bound the
+    // kernel as surely as the tensor pipe does: four products take about 300 clocks to issue and the commit
+    // 60, against 512 clocks of tensor work in a 128 x 256 x 64 step.  Everything that does not change inside a
+    // tile (descriptor high words, layout steps, barrier addresses) is therefore set up outside the loop, and a
+    // K step costs the wait, two additions, the four products and the commit.
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       int it = 0;
+      // the M-side slot holds A (or, transposed, the weights B); the N-side slot the other operand
+      const int m_mn = P.tr ? p.b_mn_major : p.a_mn_major, n_mn = P.tr ? p.a_mn_major : p.b_mn_major;
+      const uint64_t a_desc0 = m_mn ? make_smem_desc(base, 8192, 1024) : make_smem_desc(base, 16, 1024);
+      const uint64_t b_desc0 = n_mn ? make_smem_desc(base + TC_A_BYTES, 8192, 1024) : make_smem_desc(base + TC_A_BYTES, 16, 1024);
+      const uint32_t a_hi = (uint32_t)(a_desc0 >> 32), b_hi = (uint32_t)(b_desc0 >> 32);
+      const uint32_t a_lo0 = (uint32_t)a_desc0, b_lo0 = (uint32_t)b_desc0;    // address field (bits 0..13, 16-byte units) + leading offset
+      const uint32_t a_step = m_mn ? (2048u >> 4) : (32u >> 4);   // 16 k-elements per instruction
+      const uint32_t b_step = n_mn ? (2048u >> 4) : (32u >> 4);
+      constexpr uint32_t SB16 = (uint32_t)Cfg::STAGE_BYTES >> 4;  // the whole ring stays below 256 KB: no carry out of the field
+      uint32_t a_lo = a_lo0, b_lo = b_lo0, fbar = full_bar(0), ebar = empty_bar(0);
       for (int w = w0; ok && crank == 0; w += wstride, ++it) {
         TcTile t = tc_tile(P, w, tiles_m_dev, prank);
         if (!t.valid) break;
@@ -493,29 +568,18 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MMA_N);
         const uint32_t idesc = (P.idesc & ~(0x3Fu << 17)) | ((uint32_t)(t.ncols >> 3) << 17);   // N of this tile
-        for (int kb = 0; kb < t.k_blocks; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, P.wait_cycles)) { ok = false; break; }
+        const int nk = t.k_blocks;
+        for (int kb = 0; kb < nk; ++kb) {
+          if (!mbar_wait(fbar, phase, abort_flag, p.status, P.wait_cycles)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + stage * Cfg::STAGE_BYTES;
-          const uint32_t sb = sa + TC_A_BYTES;
-          // the M-side slot holds A (or, transposed, the weights B); the N-side slot the other operand
-          const int m_mn = P.tr ? p.b_mn_major : p.a_mn_major, n_mn = P.tr ? p.a_mn_major : p.b_mn_major;
-          const uint64_t a_desc = m_mn ? make_smem_desc(sa, 8192, 1024) : make_smem_desc(sa, 16, 1024);
-          const uint64_t b_desc = n_mn ? make_smem_desc(sb, 8192, 1024) : make_smem_desc(sb, 16, 1024);
-          const uint32_t a_step = m_mn ? (2048u >> 4) : (32u >> 4);   // 16 k-elements per instruction
-          const uint32_t b_step = n_mn ? (2048u >> 4) : (32u >> 4);
-#pragma unroll
-          for (int ks = 0; ks < TC_BK / 16; ++ks) {
-            if constexpr (PAIR)
-              tc_mma_pair(d_tmem, a_desc + (uint64_t)(a_step * ks), b_desc + (uint64_t)(b_step * ks), idesc,
-                          (kb | ks) != 0 ? 1u : 0u);
-            else
-              tc_mma(d_tmem, a_desc + (uint64_t)(a_step * ks), b_desc + (uint64_t)(b_step * ks), idesc,
-                     (kb | ks) != 0 ? 1u : 0u);
-          }
+          tc_mma_lohi<PAIR>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, kb != 0 ? 1u : 0u);
+          tc_mma_lohi<PAIR>(d_tmem, a_lo + a_step, a_hi, b_lo + b_step, b_hi, idesc, 1u);
+          tc_mma_lohi<PAIR>(d_tmem, a_lo + 2 * a_step, a_hi, b_lo + 2 * b_step, b_hi, idesc, 1u);
+          tc_mma_lohi<PAIR>(d_tmem, a_lo + 3 * a_step, a_hi, b_lo + 3 * b_step, b_hi, idesc, 1u);
           // stage reusable once these MMAs have read it (in both CTAs of a pair)
-          if constexpr (PAIR) tc_commit_pair(empty_bar(stage)); else tc_commit(empty_bar(stage));
-          if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+          if constexpr (PAIR) tc_commit_pair(ebar); else tc_commit(ebar);
+          a_lo += SB16; b_lo += SB16; fbar += 8u; ebar += 8u;
+          if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; a_lo = a_lo0; b_lo = b_lo0; fbar = full_bar(0); ebar = empty_bar(0); }
         }
         if (!ok) break;
         if constexpr (PAIR) tc_commit_pair(tfull_bar(acc)); else tc_commit(tfull_bar(acc));   // accumulator complete
@@ -541,50 +605,30 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
     bool ok = true;
     int it = 0;
     uint32_t n_grp = 0;                          // bulk groups committed so far (same in every lane)
-    // SwiGLU backward: a|b blocks arrive by TMA in one of two 4 KB sets [a 2 KB | b 2 KB]; the
-    // prefetch cursor runs one block ahead of the consumer, across tile boundaries.
-    constexpr int DS_SET = 4096;
-    auto ds_chunks = [&](const TcTile& t) -> int {   // blocks of this warp in tile t
-      if (!t.valid) return 0;
-      const int lim = (p.group_mode == GROUP_M) ? tiles_m_dev * TC_BM : p.M;
-      return (t.m0 + q * 32 < lim) ? (t.ncols / 32 - half + 1) / 2 : 0;
-    };
-    uint32_t ds_g = 0, ds_pf_g = 0;              // blocks consumed / loads issued
-    int ds_pf_w = w0, ds_pf_c = 0;
-    TcTile ds_pf_t;
-    ds_pf_t.valid = false;
-    auto ds_prefetch = [&]() {
-      while (ds_pf_t.valid && ds_pf_c >= ds_chunks(ds_pf_t)) {
-        ds_pf_w += wstride; ds_pf_c = 0;
-        ds_pf_t = tc_tile(P, ds_pf_w, tiles_m_dev, prank);
-      }
-      if (!ds_pf_t.valid) return;
-      const int s2 = (int)(ds_pf_g & 1u);
-      if (lane == 0) {
-        const int n = ds_pf_t.n0 + (half + 2 * ds_pf_c) * 32, y = ds_pf_t.m0 + q * 32;
-        const uint32_t dst = stg_u32 + s2 * DS_SET, bar = epi_bar(ew, s2);
-        mbar_expect_tx(bar, 4096);
-        tma_load_2d(dst, &map_c, n, y, bar);
-        tma_load_2d(dst + 2048, &map_c, p.N + n, y, bar);
-      }
-      ++ds_pf_c; ++ds_pf_g;
-    };
-    if constexpr (EPI == EPI_DSWIGLU) {
-      ds_pf_t = tc_tile(P, ds_pf_w, tiles_m_dev, prank);
-      ds_prefetch();
-    }
     for (int w = w0; ok; w += wstride, ++it) {
       TcTile t = tc_tile(P, w, tiles_m_dev, prank);
       if (!t.valid) break;
       const int acc = it & 1;
       const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, P.wait_cycles)) { ok = false; break; }
-      tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * MMA_N);
       const int m = t.m0 + row_in_tile;
       const int m_lim = (p.group_mode == GROUP_M) ? tiles_m_dev * TC_BM : p.M;
       const bool m_ok = m < m_lim;
       const bool slab_ok = t.m0 + q * 32 < m_lim;             // this warp's 32 rows hold at least one real row
+      const int rows_ok = min(32, m_lim - (t.m0 + q * 32));   // real rows among them (<= 0: none)
+      // SwiGLU backward: the a|b operands of the warp's first block do not depend on the accumulator, so
+      // their loads go out before the wait for it (ds_a / ds_b: one block in distributed form)
+      uint4 ds_a[4], ds_b[4];
+      bf16* ds_blk = nullptr;
+      if constexpr (EPI == EPI_DSWIGLU) {
+        ds_blk = reinterpret_cast<bf16*>(p.ab) + (int64_t)(t.m0 + q * 32) * p.ld_ab + t.n0;
+        if (slab_ok && half * 32 < t.ncols) {
+          blk_load_dist(ds_blk + half * 32, p.ld_ab, rows_ok, lane, ds_a);
+          blk_load_dist(ds_blk + p.N + half * 32, p.ld_ab, rows_ok, lane, ds_b);
+        }
+      }
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, P.wait_cycles)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * MMA_N);
       // row coordinate of the slab in the output tensor map (rows past its extent are clipped by the store)
       const int y0 = (p.group_mode == GROUP_K ? t.group * p.M : 0) + t.m0 + q * 32;
       const bool have_acc = t.k_blocks > 0;      // an empty K range leaves the accumulator undefined: use zeros
@@ -678,20 +722,56 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             }
             __syncwarp();
             const int piece = lane & 7;
-            const int64_t y_lim = (p.group_mode == GROUP_K) ? (int64_t)(t.group + 1) * p.M
-                                                            : (p.group_mode == GROUP_M ? (int64_t)m_lim : (int64_t)p.M);
-            float* cbase = reinterpret_cast<float*>(p.C) + n + piece * 4;
+            int64_t y_lim = (p.group_mode == GROUP_K) ? (int64_t)(t.group + 1) * p.M
+                                                      : (p.group_mode == GROUP_M ? (int64_t)m_lim : (int64_t)p.M);
+            int64_t yb = y0;                                   // first output row of this warp's slab
+            float* cptr = reinterpret_cast<float*>(p.C);
+            bf16* wptr = reinterpret_cast<bf16*>(p.upd_w);
+            float* mptr = p.upd_m;
+            if (EPI == EPI_WGRAD && p.split_m > 0) {
+              // two outputs: the slab lies wholly in the first or in the second (split_m is a multiple of 128)
+              int local = t.m0 + q * 32;
+              if (local >= p.split_m) {
+                local -= p.split_m;
+                cptr = reinterpret_cast<float*>(p.C2); wptr = reinterpret_cast<bf16*>(p.upd_w2); mptr = p.upd_m2;
+              }
+              yb = (int64_t)t.group * p.split_m + local;
+              y_lim = (int64_t)(t.group + 1) * p.split_m;
+            }
+            const int64_t col = n + piece * 4;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               const int r = i * 4 + (lane >> 3);
               const float4 v = *reinterpret_cast<const float4*>(stg + r * 128 + ((piece ^ (r & 7)) << 4));
-              if ((int64_t)y0 + r < y_lim) {
-                float4* o = reinterpret_cast<float4*>(cbase + ((int64_t)y0 + r) * p.ldc);
-                if (EPI == EPI_WGRAD && p.accumulate) {
-                  float4 old = *o;
-                  *o = make_float4(old.x + v.x, old.y + v.y, old.z + v.z, old.w + v.w);
+              if (yb + r < y_lim) {
+                const int64_t at = (yb + r) * p.ldc + col;
+                if (EPI == EPI_WGRAD && wptr) {
+                  // fused SGD step on the weight tile this gradient tile belongs to; the gradient is not stored
+                  float4 wv;
+                  if (mptr) {
+                    wv = *reinterpret_cast<const float4*>(mptr + at);
+                  } else {
+                    const uint2 raw = *reinterpret_cast<const uint2*>(wptr + at);
+                    const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+                    const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+                    wv = make_float4(lo.x, lo.y, hi.x, hi.y);
+                  }
+                  wv.x -= p.upd_lr * v.x; wv.y -= p.upd_lr * v.y; wv.z -= p.upd_lr * v.z; wv.w -= p.upd_lr * v.w;
+                  if (mptr) *reinterpret_cast<float4*>(mptr + at) = wv;
+                  uint2 out;
+                  __nv_bfloat162 h2 = __floats2bfloat162_rn(wv.x, wv.y);
+                  out.x = *reinterpret_cast<uint32_t*>(&h2);
+                  h2 = __floats2bfloat162_rn(wv.z, wv.w);
+                  out.y = *reinterpret_cast<uint32_t*>(&h2);
+                  *reinterpret_cast<uint2*>(wptr + at) = out;
                 } else {
-                  *o = v;
+                  float4* o = reinterpret_cast<float4*>(cptr + at);
+                  if (EPI == EPI_WGRAD && p.accumulate) {
+                    float4 old = *o;
+                    *o = make_float4(old.x + v.x, old.y + v.y, old.z + v.z, old.w + v.w);
+                  } else {
+                    *o = v;
+                  }
                 }
               }
             }
@@ -756,10 +836,12 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         }
       } else if constexpr (EPI == EPI_SWIGLU) {
         // columns [0, MMA_N/2) hold the gate projection, [MMA_N/2, MMA_N) the up projection.
-        // H goes out through two alternating 2 KB staging buffers; when the a|b copy is wanted too,
-        // a|b and H take turns in the staging area.
+        // H (times the row's scale, when one is given: the routed experts' gate weight) goes out through two
+        // alternating 2 KB staging buffers and TMA stores; when the a|b copy is wanted too, a|b and H take turns
+        // in the staging area.  (Plain line-wide stores for the a|b copy measured 0.01 ms slower per launch.)
         uint32_t r1[32];
         float g[32];
+        const float rs = (p.rowscale && m_ok) ? p.rowscale[m] : 1.f;
 #pragma unroll 1
         for (int c = half * 32; c < MMA_N / 2; c += 64) {
           const int n = t.n0 + c;
@@ -787,7 +869,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             }
           }
 #pragma unroll
-          for (int i = 0; i < 32; ++i) f[i] = swiglu_f(f[i], g[i]);
+          for (int i = 0; i < 32; ++i) f[i] = rs * (f[i] * sigmoid_approx(f[i]) * g[i]);
           const uint32_t off = p.C1 ? 0u : (n_grp & 1u) * 2048u;
           if (lane == 0) { if (p.C1) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
           __syncwarp();
@@ -801,61 +883,50 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           ++n_grp;
         }
       } else {   // EPI_DSWIGLU
-        // Per 32-column block: a|b arrive by TMA in a set [a 2 KB | b 2 KB] of this warp's staging
-        // area, da|db are written over them, g*H into a buffer of its own, and three TMA stores
-        // take them back to global memory.  Two sets alternate; the load of the warp's next block
-        // is issued as soon as the stores of its previous block have read their set.
-        float rs = (p.rowscale && m_ok) ? p.rowscale[m] : 1.f;
+        // Per 32-column block: a|b arrive in distributed form by plain 16-byte loads (the next block's are in
+        // flight during this block's arithmetic), pass through the staging area into row-per-lane form, da|db are
+        // written over them there and leave by plain line-wide stores.  Nothing in this path queues behind the
+        // load warp's operand traffic in the copy engine or waits for a bulk store to drain, which is what
+        // bounded the first version of this epilogue (a|b by TMA, two sets, three bulk stores per block).
+        const float rs = (p.rowscale && m_ok) ? p.rowscale[m] : 1.f;
         float dg = 0.f;
-        float a[32], b[32];
-        const int nch = ds_chunks(t);
 #pragma unroll 1
-        for (int ci = 0; ci < nch && ok; ++ci, ++ds_g) {
-          const int s2 = (int)(ds_g & 1u);
-          const uint32_t par = (ds_g >> 1) & 1u;
-          const int c = (half + 2 * ci) * 32;
-          const int n = t.n0 + c;
+        for (int c = half * 32; c < t.ncols; c += 64) {
+          if (!slab_ok) continue;      // warp-uniform
+          blk_dist_to_stage(stg, lane, ds_a);
+          blk_dist_to_stage(stg + 2048, lane, ds_b);
+          __syncwarp();
+          if (c + 64 < t.ncols) {
+            blk_load_dist(ds_blk + c + 64, p.ld_ab, rows_ok, lane, ds_a);
+            blk_load_dist(ds_blk + p.N + c + 64, p.ld_ab, rows_ok, lane, ds_b);
+          }
           tmem_ld32(taddr + c, r0);
-          if (!mbar_wait(epi_bar(ew, s2), par, abort_flag, p.status, P.wait_cycles)) { ok = false; tmem_ld_wait(); break; }
           tmem_ld_wait();
-          uint8_t* set = stg + s2 * DS_SET;
-          uint8_t* row_a = set + lane * 64;
-          uint8_t* row_b = set + 2048 + lane * 64;
-          uint8_t* row_h = stg + 2 * DS_SET + lane * 64;
+          uint8_t* row_a = stg + lane * 64;
+          uint8_t* row_b = stg + 2048 + lane * 64;
           const int sw = (lane >> 1) & 3;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            unpack8(*reinterpret_cast<const uint4*>(row_a + ((j ^ sw) << 4)), a + 8 * j);
-            unpack8(*reinterpret_cast<const uint4*>(row_b + ((j ^ sw) << 4)), b + 8 * j);
-          }
-          // the previous block's stores have read their sources: its set is free for the next load,
-          // and the single g*H buffer may be rewritten
-          if (lane == 0) bulk_wait_read<0>();
-          __syncwarp();
-          ds_prefetch();
+            float a[8], b[8];
+            unpack8(*reinterpret_cast<const uint4*>(row_a + ((j ^ sw) << 4)), a);
+            unpack8(*reinterpret_cast<const uint4*>(row_b + ((j ^ sw) << 4)), b);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            float v = __uint_as_float(r0[i]);
-            float da, db;
-            float H = dswiglu_f(a[i], b[i], rs * v, da, db);
-            if (m_ok) dg += v * H;
-            a[i] = da; b[i] = db; f[i] = rs * H;
+            for (int i = 0; i < 8; ++i) {
+              const float v = __uint_as_float(r0[8 * j + i]);
+              const float sg = sigmoid_approx(a[i]);
+              const float si = a[i] * sg;                 // silu(a)
+              const float dh = rs * v;                    // dL/dH of this row
+              dg = fmaf(v, si * b[i], dg);                // <dH', H>: gradient of the row's gate weight
+              a[i] = dh * b[i] * (sg * (1.f + a[i] - si));   // da = dh b silu'(a), silu'(a) = s (1 + a (1 - s))
+              b[i] = dh * si;                             // db = dh silu(a)
+            }
+            *reinterpret_cast<uint4*>(row_a + ((j ^ sw) << 4)) = pack8(a);
+            *reinterpret_cast<uint4*>(row_b + ((j ^ sw) << 4)) = pack8(b);
           }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            *reinterpret_cast<uint4*>(row_a + ((j ^ sw) << 4)) = pack8(a + 8 * j);
-            *reinterpret_cast<uint4*>(row_b + ((j ^ sw) << 4)) = pack8(b + 8 * j);
-            *reinterpret_cast<uint4*>(row_h + ((j ^ sw) << 4)) = pack8(f + 8 * j);
-          }
-          fence_async_smem();
           __syncwarp();
-          if (lane == 0) {
-            const uint32_t src = stg_u32 + s2 * DS_SET;
-            tma_store_2d(&map_c, src, n, y0);
-            tma_store_2d(&map_c, src + 2048, p.N + n, y0);
-            if (p.C1) tma_store_2d(&map_c1, stg_u32 + 2 * DS_SET, n, y0);
-            bulk_commit();
-          }
+          blk_stage_to_global(stg, lane, ds_blk + c, p.ld_ab, rows_ok);
+          blk_stage_to_global(stg + 2048, lane, ds_blk + p.N + c, p.ld_ab, rows_ok);
+          __syncwarp();
         }
         if (p.dg_part && m_ok) p.dg_part[(int64_t)m * p.dg_ld + 2 * (t.n0 / P.tile_n) + half] = dg;
       }
@@ -865,15 +936,6 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
       if (lane == 0) {
         if constexpr (PAIR) mbar_arrive_cluster(mapa_u32(tempty_bar(acc), 0));   // the even CTA's MMA warp waits for both
         else mbar_arrive(tempty_bar(acc));
-      }
-    }
-    if constexpr (EPI == EPI_DSWIGLU) {
-      // operand loads issued but not consumed (only after an abandoned wait) must land before the CTA exits
-      if (lane == 0) {
-        for (uint32_t g = ds_g; g < ds_pf_g; ++g) {
-          long long t0 = clock64();
-          while (!mbar_try_wait(epi_bar(ew, (int)(g & 1u)), (g >> 1) & 1u) && clock64() - t0 < P.wait_cycles) {}
-        }
       }
     }
     // this lane's stores must be complete (shared memory read, global memory written) before the CTA exits
@@ -1088,26 +1150,35 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
     if (p.group_mode != 0 || p.N % 128 != 0 || p.hm_S <= 0 || p.hm_Sp < p.hm_S || (reinterpret_cast<uintptr_t>(p.C) & 15u))
       return REVFFN_ERR_SHAPE;
   } else if (p.epilogue == EPI_DSWIGLU) {
-    // a|b are loaded and written back in place through one map; g*H (optional) through the other
+    // a|b are read and rewritten in place with plain 16-byte accesses, no tensor map
     if ((reinterpret_cast<uintptr_t>(p.ab) & 15u) || (p.ld_ab * 2) % 16 != 0) return REVFFN_ERR_ALIGN;
-    int r = tc_make_out_map(&mc, p.ab, false, (uint64_t)2 * p.N, (uint64_t)p.M, (uint64_t)p.ld_ab);
-    if (r) return r;
-    if (p.C1) {
-      if ((reinterpret_cast<uintptr_t>(p.C1) & 15u) || (p.ldc1 * 2) % 16 != 0) return REVFFN_ERR_ALIGN;
-      r = tc_make_out_map(&mc1, p.C1, false, (uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.ldc1);
-      if (r) return r;
-    }
+    if (p.C1) return REVFFN_ERR_UNSUPPORTED;
   } else {
     const bool f32_out = p.epilogue == EPI_COUPLE || p.epilogue == EPI_WGRAD || (p.epilogue == EPI_STORE && p.out_f32);
     uint64_t rows = (uint64_t)p.M;
     if (p.group_mode == GROUP_K) {
-      // group g's block must start g * M rows further down one 2D tensor
-      if (p.M % TC_BM != 0 || p.c_group_stride != (int64_t)p.M * p.ldc) return REVFFN_ERR_SHAPE;
+      // group g's block must start g * M rows further down one 2D tensor (g * split_m rows with two outputs)
+      const int64_t m_out = p.split_m > 0 ? p.split_m : p.M;
+      if (p.M % TC_BM != 0 || p.c_group_stride != m_out * p.ldc) return REVFFN_ERR_SHAPE;
       rows = (uint64_t)groups * p.M;
     }
-    if ((reinterpret_cast<uintptr_t>(p.C) & 15u) || (p.ldc * (f32_out ? 4 : 2)) % 16 != 0) return REVFFN_ERR_ALIGN;
-    int r = tc_make_out_map(&mc, p.C, f32_out, (uint64_t)p.N, rows, (uint64_t)p.ldc);
-    if (r) return r;
+    if (p.split_m > 0 && (p.epilogue != EPI_WGRAD || p.M != 2 * p.split_m || p.split_m % TC_BM != 0)) return REVFFN_ERR_SHAPE;
+    if (p.epilogue == EPI_WGRAD && p.upd_w) {
+      // fused update: the weights (and master copies) are read and rewritten 8 / 16 bytes at a time
+      if ((reinterpret_cast<uintptr_t>(p.upd_w) & 15u) || (reinterpret_cast<uintptr_t>(p.upd_w2) & 15u) ||
+          (reinterpret_cast<uintptr_t>(p.upd_m) & 15u) || (reinterpret_cast<uintptr_t>(p.upd_m2) & 15u) || p.ldc % 4 != 0)
+        return REVFFN_ERR_ALIGN;
+      if (p.split_m > 0 && !p.upd_w2) return REVFFN_ERR_NULL;
+    } else {
+      if (!p.C || (p.split_m > 0 && !p.C2)) return REVFFN_ERR_NULL;
+      if ((reinterpret_cast<uintptr_t>(p.C) & 15u) || (reinterpret_cast<uintptr_t>(p.C2) & 15u) || (p.ldc * (f32_out ? 4 : 2)) % 16 != 0)
+        return REVFFN_ERR_ALIGN;
+    }
+    if (!f32_out) {      // fp32 outputs leave through plain stores and need no map
+      int r = tc_make_out_map(&mc, p.C, false, (uint64_t)p.N, rows, (uint64_t)p.ldc);
+      if (r) return r;
+    }
+    int r = 0;
     if (p.epilogue == EPI_SWIGLU && p.C1) {
       if ((reinterpret_cast<uintptr_t>(p.C1) & 15u) || (p.ldc1 * 2) % 16 != 0) return REVFFN_ERR_ALIGN;
       r = tc_make_out_map(&mc1, p.C1, false, (uint64_t)2 * p.N, (uint64_t)p.M, (uint64_t)p.ldc1);

@@ -27,7 +27,7 @@ enum Tag {
   TG_NORM, TG_FOLD, TG_ROUTER, TG_MAP, TG_PUP, TG_GATHER, TG_EXP_GATEUP, TG_EXP_DOWN, TG_SH_GATEUP, TG_SH_DOWN,
   TG_COMBINE, TG_PDOWN, TG_CAST, TG_DZ, TG_WG_PDOWN, TG_SHGATE_BWD, TG_SH_DH, TG_WG_SH_DOWN, TG_SH_DU,
   TG_WG_SH_GATE, TG_WG_SH_UP, TG_WG_SGATE, TG_GATHER_DZ, TG_EXP_DH, TG_EXP_DU, TG_WG_EXP_DOWN, TG_WG_EXP_GATE,
-  TG_WG_EXP_UP, TG_ROUTER_BWD, TG_WG_ROUTER, TG_DU_REDUCE, TG_DN, TG_WG_PUP, TG_NORM_BWD, TG_DGAMMA,
+  TG_WG_EXP_UP, TG_WG_EXP_GATEUP, TG_ROUTER_BWD, TG_WG_ROUTER, TG_DU_REDUCE, TG_DN, TG_WG_PUP, TG_NORM_BWD, TG_DGAMMA,
   // attention coupling branch
   TG_A_TABLES, TG_A_QKV, TG_A_HEADS, TG_A_SCORES, TG_A_SOFTMAX, TG_A_PV, TG_A_WO, TG_A_WGRAD, TG_A_DGRAD, TG_A_BIAS,
   TG_A_DP, TG_A_DKV, TG_A_DQ, TG_A_FLASH, TG_COUNT
@@ -37,7 +37,7 @@ static const char* kTagNames[TG_COUNT] = {
     "gemm_expert_down_scale", "gemm_shared_gate_up_swiglu", "gemm_shared_down", "combine", "gemm_p_down_couple",
     "cast_dy2", "gemm_dz", "wgrad_p_down", "shared_gate_bwd", "gemm_shared_dh_dswiglu", "wgrad_shared_down",
     "gemm_shared_du", "wgrad_shared_gate", "wgrad_shared_up", "wgrad_shared_sgate", "gather_dz",
-    "gemm_expert_dh_dswiglu", "gemm_expert_du", "wgrad_expert_down", "wgrad_expert_gate", "wgrad_expert_up",
+    "gemm_expert_dh_dswiglu", "gemm_expert_du", "wgrad_expert_down", "wgrad_expert_gate", "wgrad_expert_up", "wgrad_expert_gate_up",
     "router_bwd", "wgrad_router", "du_reduce", "gemm_dn", "wgrad_p_up", "rmsnorm_bwd", "dgamma",
     "attn_tables", "gemm_qkv", "attn_heads", "gemm_scores", "attn_softmax", "gemm_pv", "gemm_w_o", "attn_wgrad",
     "attn_dgrad", "attn_bias_grad", "gemm_dp", "gemm_dk_dv", "gemm_dq", "flash_attention"};
@@ -417,7 +417,9 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
   }
   CK(cudaGetLastError());
 
-  // Routed experts: H = silu(Up Wg^T) * (Up Wu^T);  O = g * (H Wd^T)
+  // Routed experts: H' = g * silu(Up Wg^T) * (Up Wu^T);  O = H' Wd^T.  The row's gate weight g goes onto H in
+  // the first product's epilogue: the second then needs no scaling, and the backward pass finds in H' exactly the
+  // operand its down-projection weight gradient takes (dW_d = dO^T (g H)).
   {
     GemmProblem p = blank_problem();
     p.M = (int)L.rows_pad; p.N = I; p.K = d;
@@ -427,6 +429,7 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
     p.rows_total = c.template p<int32_t>(L.rows_total);
     p.epilogue = EPI_SWIGLU; p.C = c.template p<T>(L.hmid); p.ldc = I;
+    p.rowscale = c.template p<float>(L.row_gate);
     if (save_ab) { p.C1 = c.template p<T>(L.ab); p.ldc1 = 2 * (int64_t)I; }
     CKR(run_gemm(c, p, TG_EXP_GATEUP));
   }
@@ -439,7 +442,7 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
     p.rows_total = c.template p<int32_t>(L.rows_total);
     p.tok_chunks = c.template p<int4>(L.tok_chunks);
-    p.epilogue = EPI_ROWSCALE; p.rowscale = c.template p<float>(L.row_gate);
+    p.epilogue = EPI_STORE;
     p.C = c.template p<T>(L.o); p.ldc = d;
     CKR(run_gemm(c, p, TG_EXP_DOWN));
   }
@@ -488,7 +491,7 @@ static int run_couple(const Ctx<T>& c, const float* resid, float sign, float* ou
 
 template <typename T>
 static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, float* dy1, const revffn_moe_grads& G,
-                        const int32_t* idx_in) {
+                        const revffn_moe_sgd* sgd, const int32_t* idx_in) {
   const revffn_moe_desc& D = c.D;
   const WsLayout& L = c.L;
   const int Tn = D.tokens, d = D.d_model, h = d / 2, E = D.n_experts, k = D.top_k, I = D.d_expert, Is = D.d_shared;
@@ -499,15 +502,29 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
 
   if (!(D.flags & REVFFN_FLAG_REUSE_ACTIVATIONS)) CKR(run_branch(c, y1, idx_in, nullptr, true));
 
-  auto wgrad = [&](int tag, float* out, int M, int N, const void* A, int64_t lda, int a_col0, const void* B, int64_t ldb,
-                   bool grouped, int64_t cstride) -> int {
+  // One weight gradient: `out` receives it (fp32), or, when the fused SGD step covers this weight (its bit in
+  // sgd->mask), the weight W itself is updated tile by tile in the product's epilogue and no gradient is stored.
+  // out2 / W2 / master2: second output of a product whose M is two stacked weights (gate | up of the experts).
+  const uint32_t upd_mask = sgd ? sgd->mask : 0u;
+  auto wgrad = [&](int tag, uint32_t bit, float* out, const void* W, float* master, int M, int N, const void* A, int64_t lda,
+                   int a_col0, const void* B, int64_t ldb, bool grouped, int64_t cstride, float* out2 = nullptr,
+                   const void* W2 = nullptr, float* master2 = nullptr) -> int {
+    const bool upd = (upd_mask & bit) != 0;
+    if (!upd && !out) return REVFFN_OK;      // frozen: neither gradient nor update wanted
     GemmProblem p = blank_problem();
     p.M = M; p.N = N; p.K = grouped ? Rp : Tn;   // grouped: bound on rows, the range comes from group_off
     p.a_mn_major = 1; p.b_mn_major = 1;
     p.A = A; p.lda = lda; p.a_col0 = a_col0;
     p.B0 = B; p.ldb = ldb;
     p.epilogue = EPI_WGRAD; p.accumulate = acc;
-    p.C = out; p.ldc = N; p.c_group_stride = cstride;
+    p.ldc = N; p.c_group_stride = cstride;
+    if (upd) {
+      p.upd_w = const_cast<void*>(W); p.upd_m = master; p.upd_lr = sgd->lr;
+      p.upd_w2 = const_cast<void*>(W2); p.upd_m2 = master2;
+    } else {
+      p.C = out; p.C2 = out2;
+    }
+    if (out2 || W2) p.split_m = M / 2;
     if (grouped) {
       p.group_mode = GROUP_K; p.n_groups = E;
       p.group_off = c.template p<int32_t>(L.expert_off);
@@ -515,6 +532,8 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     }
     return run_gemm(c, p, tag);
   };
+  const revffn_moe_sgd no_sgd = {};
+  const revffn_moe_sgd& S = sgd ? *sgd : no_sgd;
 
   // P_down backward: dZ = G W_down;  dW_down = G^T Z
   { ProfScope ps(TG_CAST, st);
@@ -530,7 +549,8 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dz); p.ldc = d;
     CKR(run_gemm(c, p, TG_DZ));
   }
-  if (G.w_down) CKR(wgrad(TG_WG_PDOWN, G.w_down, h, d, c.template p<T>(L.gb), h, 0, c.template p<T>(L.z), d, false, 0));
+  CKR(wgrad(TG_WG_PDOWN, REVFFN_UPD_W_DOWN, G.w_down, c.W.w_down, S.m_w_down, h, d, c.template p<T>(L.gb), h, 0,
+            c.template p<T>(L.z), d, false, 0));
 
   // Shared expert backward
   if (Is > 0) {
@@ -548,7 +568,8 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       p.epilogue = EPI_DSWIGLU; p.ab = c.template p<T>(L.abs); p.ld_ab = 2 * (int64_t)Is;
       CKR(run_gemm(c, p, TG_SH_DH));
     }
-    if (G.ws_down) CKR(wgrad(TG_WG_SH_DOWN, G.ws_down, d, Is, c.template p<T>(L.ds), d, 0, c.template p<T>(L.hs), Is, false, 0));
+    CKR(wgrad(TG_WG_SH_DOWN, REVFFN_UPD_WS_DOWN, G.ws_down, c.W.ws_down, S.m_ws_down, d, Is, c.template p<T>(L.ds), d, 0,
+              c.template p<T>(L.hs), Is, false, 0));
     {
       GemmProblem p = blank_problem();   // dU_sh = da Ws_g + db Ws_u
       p.M = Tn; p.N = d; p.K = 2 * Is;
@@ -557,8 +578,10 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dush); p.ldc = d;
       CKR(run_gemm(c, p, TG_SH_DU));
     }
-    if (G.ws_gate) CKR(wgrad(TG_WG_SH_GATE, G.ws_gate, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, 0, c.template p<T>(L.u), d, false, 0));
-    if (G.ws_up) CKR(wgrad(TG_WG_SH_UP, G.ws_up, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, Is, c.template p<T>(L.u), d, false, 0));
+    CKR(wgrad(TG_WG_SH_GATE, REVFFN_UPD_WS_GATE, G.ws_gate, c.W.ws_gate, S.m_ws_gate, Is, d, c.template p<T>(L.abs),
+              2 * (int64_t)Is, 0, c.template p<T>(L.u), d, false, 0));
+    CKR(wgrad(TG_WG_SH_UP, REVFFN_UPD_WS_UP, G.ws_up, c.W.ws_up, S.m_ws_up, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, Is,
+              c.template p<T>(L.u), d, false, 0));
     if (G.ws_sgate) {
       { ProfScope ps(TG_WG_SGATE, st);
       CK(launch_colsum_partial<T>(c.template p<T>(L.u), d, c.template p<float>(L.dl), Tn, d, STRIP, L.strips,
@@ -580,7 +603,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
   CK(cudaGetLastError());
   const int n_part = dg_parts(c, I);
   {
-    GemmProblem p = blank_problem();   // dH' = dO Wd; SwiGLU backward; dg partials; hmid <- g * H
+    GemmProblem p = blank_problem();   // dH' = dO Wd; SwiGLU backward in place on a|b; dg partials
     p.M = Rp; p.N = I; p.K = d;
     p.A = c.template p<T>(L.dop); p.lda = d;
     p.B0 = c.W.w_downx; p.ldb = I; p.b_mn_major = 1;
@@ -589,7 +612,6 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.rows_total = c.template p<int32_t>(L.rows_total);
     p.epilogue = EPI_DSWIGLU; p.ab = c.template p<T>(L.ab); p.ld_ab = 2 * (int64_t)I;
     p.rowscale = c.template p<float>(L.row_gate);
-    p.C1 = c.template p<T>(L.hmid); p.ldc1 = I;
     p.dg_part = c.template p<float>(L.dg_part); p.dg_ld = L.dg_ld;
     CKR(run_gemm(c, p, TG_EXP_DH));
   }
@@ -605,9 +627,22 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dup); p.ldc = d;
     CKR(run_gemm(c, p, TG_EXP_DU));
   }
-  if (G.w_downx) CKR(wgrad(TG_WG_EXP_DOWN, G.w_downx, d, I, c.template p<T>(L.dop), d, 0, c.template p<T>(L.hmid), I, true, (int64_t)d * I));
-  if (G.w_gate) CKR(wgrad(TG_WG_EXP_GATE, G.w_gate, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, 0, c.template p<T>(L.up), d, true, (int64_t)I * d));
-  if (G.w_upx) CKR(wgrad(TG_WG_EXP_UP, G.w_upx, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, I, c.template p<T>(L.up), d, true, (int64_t)I * d));
+  CKR(wgrad(TG_WG_EXP_DOWN, REVFFN_UPD_W_DOWNX, G.w_downx, c.W.w_downx, S.m_w_downx, d, I, c.template p<T>(L.dop), d, 0,
+            c.template p<T>(L.hmid), I, true, (int64_t)d * I));
+  {
+    // dW_gate and dW_up share their B operand (the permuted u rows) and their A operand is one buffer da|db:
+    // when both are wanted in the same form they are one product with M = 2I and two outputs.
+    const bool ug = (upd_mask & REVFFN_UPD_W_GATE) != 0, uu = (upd_mask & REVFFN_UPD_W_UPX) != 0;
+    if ((ug && uu) || (!ug && !uu && G.w_gate && G.w_upx)) {
+      CKR(wgrad(TG_WG_EXP_GATEUP, REVFFN_UPD_W_GATE, G.w_gate, c.W.w_gate, S.m_w_gate, 2 * I, d, c.template p<T>(L.ab),
+                2 * (int64_t)I, 0, c.template p<T>(L.up), d, true, (int64_t)I * d, G.w_upx, c.W.w_upx, S.m_w_upx));
+    } else {
+      CKR(wgrad(TG_WG_EXP_GATE, REVFFN_UPD_W_GATE, G.w_gate, c.W.w_gate, S.m_w_gate, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, 0,
+                c.template p<T>(L.up), d, true, (int64_t)I * d));
+      CKR(wgrad(TG_WG_EXP_UP, REVFFN_UPD_W_UPX, G.w_upx, c.W.w_upx, S.m_w_upx, I, d, c.template p<T>(L.ab), 2 * (int64_t)I, I,
+                c.template p<T>(L.up), d, true, (int64_t)I * d));
+    }
+  }
 
   // Gate / router backward
   const bool dense_gate = (D.flags & REVFFN_FLAG_GATE_SOFTMAX_ALL) != 0;
@@ -644,7 +679,8 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       CKR(run_gemm(c, p, TG_ROUTER_BWD));
     }
     if (G.w_router)
-      CKR(wgrad(TG_WG_ROUTER, G.w_router, E, d, c.template p<T>(L.dlf), L.ld_dlf, 0, c.template p<T>(L.u), d, false, 0));
+      CKR(wgrad(TG_WG_ROUTER, 0u, G.w_router, nullptr, nullptr, E, d, c.template p<T>(L.dlf), L.ld_dlf, 0, c.template p<T>(L.u), d,
+                false, 0));
     if (G.b_router) {
       { ProfScope ps(TG_WG_ROUTER, st);
       CK(launch_colsum_partial<T>(c.template p<T>(L.dlf), L.ld_dlf, nullptr, Tn, E, STRIP, L.strips,
@@ -676,7 +712,8 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.epilogue = EPI_STORE; p.out_f32 = 1; p.C = c.template p<float>(L.dn); p.ldc = h;
     CKR(run_gemm(c, p, TG_DN));
   }
-  if (G.w_up) CKR(wgrad(TG_WG_PUP, G.w_up, d, h, c.template p<T>(L.du), d, 0, c.template p<T>(L.n), h, false, 0));
+  CKR(wgrad(TG_WG_PUP, REVFFN_UPD_W_UP, G.w_up, c.W.w_up, S.m_w_up, d, h, c.template p<T>(L.du), d, 0, c.template p<T>(L.n), h,
+            false, 0));
   { ProfScope ps(TG_NORM_BWD, st);
   rmsnorm_bwd_rows_kernel<<<(unsigned)ceil_div((int64_t)Tn * 32, 128), 128, 0, st>>>(
       c.template p<float>(L.dn), y1, D.ld_stream, c.W.norm_gamma, c.template p<float>(L.r), norm_none, Tn, h, dy1,
@@ -709,7 +746,7 @@ enum Pass { PASS_FWD, PASS_INV, PASS_BWD };
 template <typename T>
 static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weights& W, const WsLayout& L, void* ws,
                     cudaStream_t st, const float* y1, const float* in2, float* out, const revffn_moe_grads* G,
-                    const int32_t* idx_in, int32_t* idx_out) {
+                    const revffn_moe_sgd* sgd, const int32_t* idx_in, int32_t* idx_out) {
   Ctx<T> c;
   c.D = D; c.W = W; c.L = L; c.ws = reinterpret_cast<char*>(ws); c.st = st;
   g_prof.pass = (int)pass;
@@ -721,7 +758,7 @@ static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weight
   const size_t ws_limit = big_ws ? L.bwd_bytes : L.fwd_bytes;
   if (L.n_guards) CKR(guards_fill(L, ws_limit, c.ws, st));
   if (pass == PASS_BWD) {
-    CKR(run_backward(c, y1, in2, out, *G, idx_in));
+    CKR(run_backward(c, y1, in2, out, *G, sgd, idx_in));
   } else {
     CKR(run_branch(c, y1, idx_in, idx_out, (D.flags & REVFFN_FLAG_SAVE_ACTIVATIONS) != 0));
     CKR(run_couple(c, in2, pass == PASS_FWD ? 1.f : -1.f, out));
@@ -732,7 +769,7 @@ static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weight
 
 static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1,
                  const float* in2, float* out, const revffn_moe_grads* grads, const int32_t* idx_in,
-                 int32_t* idx_out, void* ws, size_t ws_bytes, void* cuda_stream) {
+                 int32_t* idx_out, void* ws, size_t ws_bytes, void* cuda_stream, const revffn_moe_sgd* sgd = nullptr) {
   CKR(validate_desc(desc));
   CKR(validate_weights(*desc, w));
   if (!ws) return REVFFN_ERR_NULL;
@@ -743,6 +780,19 @@ static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weight
   if ((reinterpret_cast<uintptr_t>(idx_in) | reinterpret_cast<uintptr_t>(idx_out)) &
       ((desc->flags & REVFFN_FLAG_ROUTING_RECORD) ? 15u : 3u))
     return REVFFN_ERR_ALIGN;
+  if (sgd) {
+    if (sgd->mask & ~REVFFN_UPD_ALL) return REVFFN_ERR_SHAPE;
+    if (desc->d_shared == 0 && (sgd->mask & (REVFFN_UPD_WS_GATE | REVFFN_UPD_WS_UP | REVFFN_UPD_WS_DOWN))) return REVFFN_ERR_NULL;
+    const float* ms[] = {sgd->m_w_up, sgd->m_w_down, sgd->m_w_gate, sgd->m_w_upx, sgd->m_w_downx, sgd->m_ws_gate,
+                         sgd->m_ws_up, sgd->m_ws_down};
+    for (const float* m : ms)
+      if (m && !aligned16(m)) return REVFFN_ERR_ALIGN;
+    // a weight is either updated in place or has its gradient written, not both
+    const float* gs8[] = {grads->w_up, grads->w_down, grads->w_gate, grads->w_upx, grads->w_downx, grads->ws_gate,
+                          grads->ws_up, grads->ws_down};
+    for (int i = 0; i < 8; ++i)
+      if ((sgd->mask & (1u << i)) && gs8[i]) return REVFFN_ERR_UNSUPPORTED;
+  }
   if (grads) {
     const float* gs[] = {grads->norm_gamma, grads->w_up, grads->w_down, grads->w_router, grads->b_router,
                          grads->w_gate, grads->w_upx, grads->w_downx, grads->ws_gate, grads->ws_up,
@@ -756,8 +806,8 @@ static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weight
   CKR(check_device());
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (desc->weight_dtype == REVFFN_BF16)
-    return dispatch<bf16>(pass, *desc, *w, L, ws, st, y1, in2, out, grads, idx_in, idx_out);
-  return dispatch<float>(pass, *desc, *w, L, ws, st, y1, in2, out, grads, idx_in, idx_out);
+    return dispatch<bf16>(pass, *desc, *w, L, ws, st, y1, in2, out, grads, sgd, idx_in, idx_out);
+  return dispatch<float>(pass, *desc, *w, L, ws, st, y1, in2, out, grads, sgd, idx_in, idx_out);
 }
 
 // ---------------------------------------------------------------------------
@@ -826,6 +876,13 @@ int revffn_moe_backward(const revffn_moe_desc* desc, const revffn_moe_weights* w
                         float* dy1_inout, const revffn_moe_grads* grads, const int32_t* topk_idx_in, void* ws,
                         size_t ws_bytes, void* cuda_stream) {
   return entry(PASS_BWD, desc, w, y1, dy2, dy1_inout, grads, topk_idx_in, nullptr, ws, ws_bytes, cuda_stream);
+}
+
+int revffn_moe_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1, const float* dy2,
+                            float* dy1_inout, const revffn_moe_grads* grads, const revffn_moe_sgd* sgd,
+                            const int32_t* topk_idx_in, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!sgd) return REVFFN_ERR_NULL;
+  return entry(PASS_BWD, desc, w, y1, dy2, dy1_inout, grads, topk_idx_in, nullptr, ws, ws_bytes, cuda_stream, sgd);
 }
 
 int revffn_moe_status(const void* ws, void* cuda_stream, int32_t* device_status) {
@@ -1074,6 +1131,14 @@ int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weig
                               float* stream_a, float* stream_b, float* grad_a, float* grad_b,
                               const revffn_moe_grads* grads, const int32_t* topk_idx, void* cache,
                               size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return revffn_moe_stack_backward_sgd(desc, weights, n_blocks, stream_a, stream_b, grad_a, grad_b, grads, nullptr, topk_idx,
+                                       cache, cache_bytes, ws, ws_bytes, cuda_stream);
+}
+
+int revffn_moe_stack_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                                  float* stream_a, float* stream_b, float* grad_a, float* grad_b,
+                                  const revffn_moe_grads* grads, const revffn_moe_sgd* sgd, const int32_t* topk_idx,
+                                  void* cache, size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream) {
   int r = validate_desc(desc);
   if (r != REVFFN_OK) return r;
   if (n_blocks < 0) return REVFFN_ERR_SHAPE;
@@ -1099,11 +1164,15 @@ int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weig
         topk_idx ? reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(topk_idx) + (size_t)l * idx_stride) : nullptr;
     if (cache) {
       char* c = reinterpret_cast<char*>(cache) + (size_t)l * stride;
-      CKR(revffn_moe_backward(&d_bwd, &weights[l], reinterpret_cast<const float*>(c), gR, gP, &grads[l], idx,
-                              c + slot, ws_need, cuda_stream));
+      CKR(entry(PASS_BWD, &d_bwd, &weights[l], reinterpret_cast<const float*>(c), gR, gP, &grads[l], idx, nullptr, c + slot,
+                ws_need, cuda_stream, sgd ? &sgd[l] : nullptr));
     } else {
+      // the layer's weights are read for the last time in this step by these two calls (inverse, then the
+      // gradient pass, whose weight-gradient products come after every product that reads the same weight),
+      // so a fused update of layer l cannot disturb any other layer's reconstruction
       CKR(revffn_moe_inverse(&d_inv, &weights[l], P, R, R, idx, ws, ws_bytes, cuda_stream));
-      CKR(revffn_moe_backward(&d_bwd, &weights[l], P, gR, gP, &grads[l], idx, ws, ws_bytes, cuda_stream));
+      CKR(entry(PASS_BWD, &d_bwd, &weights[l], P, gR, gP, &grads[l], idx, nullptr, ws, ws_bytes, cuda_stream,
+                sgd ? &sgd[l] : nullptr));
     }
   }
   return REVFFN_OK;

@@ -265,9 +265,12 @@ inline cudaError_t launch_fold_router_mma(const T* w_router, const T* w_sgate, c
 //   phase 1: L[t, e] = r_t <W_rc[e], y_t * gamma> (+ b_r[e]) for e < E; row E is the
 //            shared gate.  The product runs on the fp64 tensor-core path
 //            (mma.sync m8n8k4): y*gamma (fp64, [token][i]) and W_rc ([expert][i]) are
-//            staged chunk-wise in shared memory, each warp owns a 16-token x 32-expert
-//            block of the 64 x 64 tile as 2 x 4 fragments, and reads 6 operand values
-//            per 8 instructions.  (A register-tiled DFMA version of the same product
+//            staged chunk-wise in shared memory, each warp owns a 16-token x 16-expert
+//            block of the 32 x 64 tile as 2 x 2 fragments.  (Blocks of 64 tokens with 16 x 32
+//            per warp read fewer operand values per instruction, but a batch of 8192 tokens
+//            then fills the GPU with one block of 8 warps per SM, which cannot hide the
+//            latency of its own loads: 32-token blocks, two or three to an SM, took the kernel
+//            from 0.106 to the time recorded in the design notes.)  (A register-tiled DFMA version of the same product
 //            spent its time on shared-memory operand reads: 8 values per 16 FMAs.)
 //            The staging threads also sum y^2 (fp64), which gives
 //            r_t = (mean(y_t^2)+eps)^-1/2; the scale is applied to the finished sums.
@@ -277,7 +280,7 @@ inline cudaError_t launch_fold_router_mma(const T* w_router, const T* w_sgate, c
 // prob_out != NULL: gates are the selected entries of the softmax over ALL experts (not
 // renormalised), and that softmax is written to prob_out[T, E].
 // ---------------------------------------------------------------------------
-constexpr int RT_TOK = 64;   // tokens per block
+constexpr int RT_TOK = 32;   // tokens per block
 constexpr int RT_KC = 32;    // k-chunk
 constexpr int RT_EC = 64;    // experts per pass
 constexpr int RT_LD = RT_KC + 4;    // row stride (doubles) of both staged chunks: rows 4 doubles apart modulo 16 banks,
@@ -306,24 +309,28 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t0 = blockIdx.x * RT_TOK;
 
-  // phase 1: logits.  Warp (wm, wn) owns tokens 16 wm .. +15 and experts e0 + 32 wn .. +31.
-  const int wm = warp >> 1, wn = warp & 1;
+  // phase 1: logits.  Warp (wm, wn) owns tokens 16 wm .. +15 and experts e0 + 16 wn .. +15.
+  const int wm = warp >> 2, wn = warp & 3;
+  constexpr int NY = RT_TOK * RT_KC / 4 / 256;      // float4 pieces of the stream chunk per thread
+  static_assert(NY >= 1 && RT_TOK * RT_KC / 4 % 256 == 0, "stream chunk must split evenly over the block");
   const int fr = lane >> 2, fc = lane & 3;          // fragment row / column of this lane
   for (int e0 = 0; e0 < EP; e0 += RT_EC) {
-    double acc[2][4][2];
+    double acc[2][2][2];
 #pragma unroll
     for (int a = 0; a < 2; ++a)
 #pragma unroll
-      for (int b = 0; b < 4; ++b) { acc[a][b][0] = 0.0; acc[a][b][1] = 0.0; }
+      for (int b = 0; b < 2; ++b) { acc[a][b][0] = 0.0; acc[a][b][1] = 0.0; }
     // Register prefetch: the global loads of chunk c+1 are in flight while chunk c is summed.
-    //   y:    RT_TOK x RT_KC floats  = 2 float4 per thread  (token tt, 4 consecutive i)
+    //   y:    RT_TOK x RT_KC floats  = NY float4 per thread (token tt, 4 consecutive i)
     //   W_rc: RT_EC x RT_KC doubles  = 4 double2 per thread (expert ee, 2 consecutive i)
-    float4 py[2];
+    float4 py[NY];
     double2 pw[4];
-    double ss[2] = {0.0, 0.0};      // sum of y^2 over this thread's 4-column strip of its two tokens
+    double ss[NY];                  // sum of y^2 over this thread's 4-column strip of its token(s)
+#pragma unroll
+    for (int q = 0; q < NY; ++q) ss[q] = 0.0;
     auto prefetch = [&](int k0) {
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
+      for (int q = 0; q < NY; ++q) {
         int idx = tid + q * 256;
         int tt = idx / (RT_KC / 4), kq = (idx % (RT_KC / 4)) * 4;
         int t = t0 + tt, i = k0 + kq;
@@ -342,7 +349,7 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
     prefetch(0);
     for (int k0 = 0; k0 < h; k0 += RT_KC) {
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
+      for (int q = 0; q < NY; ++q) {
         int idx = tid + q * 256;
         int tt = idx / (RT_KC / 4), kq = (idx % (RT_KC / 4)) * 4;
         int i = k0 + kq;
@@ -363,24 +370,24 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
       __syncthreads();
       if (k0 + RT_KC < h) prefetch(k0 + RT_KC);
       const double* ap = ns + (wm * 16 + fr) * RT_LD + fc;
-      const double* bp = ws + (wn * 32 + fr) * RT_LD + fc;
+      const double* bp = ws + (wn * 16 + fr) * RT_LD + fc;
 #pragma unroll
       for (int kk = 0; kk < RT_KC; kk += 4) {
-        double af[2], bf[4];
+        double af[2], bf[2];
 #pragma unroll
         for (int a = 0; a < 2; ++a) af[a] = ap[a * 8 * RT_LD + kk];
 #pragma unroll
-        for (int b = 0; b < 4; ++b) bf[b] = bp[b * 8 * RT_LD + kk];
+        for (int b = 0; b < 2; ++b) bf[b] = bp[b * 8 * RT_LD + kk];
 #pragma unroll
         for (int a = 0; a < 2; ++a)
 #pragma unroll
-          for (int b = 0; b < 4; ++b) dmma_8x8x4(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+          for (int b = 0; b < 2; ++b) dmma_8x8x4(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
       }
       __syncthreads();
     }
     // r per token: the 8 threads that staged one token hold its strips (lanes 8m .. 8m+7)
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
+    for (int q = 0; q < NY; ++q) {
       double v = ss[q];
       v += __shfl_xor_sync(0xffffffffu, v, 1);
       v += __shfl_xor_sync(0xffffffffu, v, 2);
@@ -391,11 +398,11 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
 #pragma unroll
     for (int a = 0; a < 2; ++a)
 #pragma unroll
-      for (int b = 0; b < 4; ++b)
+      for (int b = 0; b < 2; ++b)
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           const int tt = wm * 16 + a * 8 + fr;
-          const int e = e0 + wn * 32 + b * 8 + 2 * fc + c;
+          const int e = e0 + wn * 16 + b * 8 + 2 * fc + c;
           if (e < EP) {
             double v = acc[a][b][c] * rs[tt];
             if (e < E && b_router) v += (double)b_router[e];
@@ -441,6 +448,8 @@ router_topk_kernel(const float* __restrict__ y, int64_t ld, const float* __restr
         for (int j = 0; lane + 32 * j < E; ++j) {
           if (taken & (1u << j)) continue;
           double v = L[lane + 32 * j];
+          if (v != v) v = __longlong_as_double(0xfff0000000000000LL);   // NaN orders as -inf: the comparisons below stay a
+                                                                        // total order and every lane names the same winner
           int e = lane + 32 * j;
           if (v > best || (v == best && e < besti) || besti == 0x7fffffff) { best = v; besti = e; }
         }
@@ -592,6 +601,7 @@ __global__ void map_scan_kernel(const int32_t* __restrict__ chunk_cnt, int n_chu
     // Token chunks for the products that put tokens on the MMA N side: per expert, runs of up to
     // TOK_CHUNK rows covering its real rows rounded up to 32 (the rounding stays inside the expert's
     // zero padding).  Entry = (expert, first row, rows, 0); the count goes to rows_total[1].
+    // (Runs of equal length, 3 x 192 instead of 256 + 256 + 64 for 546 rows, measured 1-2 % slower.)
     int nc = 0;
     for (int e = 0; e < E; ++e) {
       const int n = (int)round_up(expert_cnt[e], 32);

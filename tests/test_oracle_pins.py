@@ -404,3 +404,34 @@ def test_softmax_all_backward_matches_central_differences(seed):
     never = np.setdiff1d(np.arange(cfg.n_experts), np.unique(info["idx"]))
     if never.size:
         assert np.abs(g["w_router"][never]).max() > 0
+
+
+# ------------------------------------------------------------------ optimiser step
+def test_sgd_step_descends_by_lr_times_the_squared_gradient_norm():
+    """Pins sign and scale of the update against the forward map alone: for L(W) = <dY2, Y2(W)> a step
+    W' = W - lr * g changes L by -lr * |g|^2 to first order, so (L(W') - L(W)) / lr -> -|g|^2 as lr -> 0,
+    with an error that shrinks in proportion to lr.  Only the named weights may move."""
+    cfg, p, s = _tiny(seed=4, top_k=5)          # k = E: smooth everywhere, no routing jumps
+    G = np.random.default_rng(2).standard_normal(s["x2"].shape)
+
+    def loss(q):
+        y2, _ = orc.forward(q, s["y1"], s["x2"], cfg.top_k, cfg.norm_eps)
+        return float(np.sum(G * y2))
+
+    g = orc.backward(p, s["y1"], G, cfg.top_k, cfg.norm_eps)
+    names = ("w_up", "w_gate", "w_downx", "ws_up")
+    sq = sum(float(np.sum(g[n] ** 2)) for n in names)
+    L0 = loss(p)
+    errs = []
+    for lr in (1e-4, 1e-5):
+        q = orc.sgd_step(p, g, lr, names)
+        for n in p:
+            if n in names:
+                assert np.allclose(q[n], np.asarray(p[n], np.float64) - lr * g[n], rtol=0, atol=0)
+            else:
+                assert q[n] is p[n]
+        errs.append(abs((loss(q) - L0) / lr + sq) / sq)
+    assert errs[0] < 2e-2 and errs[1] < errs[0] / 5          # first-order term exact, remainder O(lr)
+    # an ascent step does the opposite
+    up = orc.sgd_step(p, g, -1e-5, names)
+    assert loss(up) > L0 > loss(orc.sgd_step(p, g, 1e-5, names))

@@ -6,9 +6,9 @@ plug-ins that only see their inputs and outputs).  Its scratch is a fixed array
 inside the library, shared by every call on the device, so the test makes two
 calls in a row on different inputs and checks each against what
 revffn_moe_forward selects and weighs for the same tokens, and against the
-oracle's routing.  Further cases: the Qwen-shaped router (60 experts, more
-shared memory than the default limit, (E+1)*h just under the scratch limit) and
-the flag the entry point does not support.  Collected last on purpose: a run
+oracle's routing.  Further cases: the Qwen-shaped router (60 experts,
+(E+1)*h just under the scratch limit) and the flag the entry point does not
+support.  Collected last on purpose: a run
 that stops at the first failure has by then run everything else.
 """
 import numpy as np
@@ -83,8 +83,8 @@ def test_route_noalloc_matches_forward_on_two_calls_in_a_row():
 
 
 def test_route_noalloc_at_the_benchmark_router_shape():
-    """60 experts over 1024-wide streams: (E+1)*h = 62464 of the 65536 scratch elements, and a logit tile
-    that needs the shared-memory limit raised (68.6 KB).  Two calls in a row, against the oracle and forward."""
+    """60 experts over 1024-wide streams: (E+1)*h = 62464 of the 65536 scratch elements.  Two calls in a row,
+    against the oracle and forward."""
     import paper_2512_20920_b200 as rv
     base = CONFIGS["C1"]
     for seed, tokens in ((0, 1000), (1, 777)):
