@@ -236,7 +236,8 @@ def dist_setup():
 
 
 def run_ours(args, cfg):
-    out = measure_block(args, cfg, e2e=True, cpu=not args.no_cpu_baseline)
+    out = measure_block(args, cfg, e2e=not args.steps_only, cpu=not (args.no_cpu_baseline or args.steps_only),
+                        steps_only=args.steps_only)
     if out is not None:
         print(json.dumps(out))
     finish()
@@ -248,7 +249,7 @@ def finish():
         dist.destroy_process_group()
 
 
-def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
+def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_only=False):
     """One block at cfg.tokens tokens per GPU; returns the JSON record (rank 0) or None."""
     import torch
     import torch.distributed as dist
@@ -314,6 +315,14 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None):
     clocks = sampler.stop() if sampler else None
     launches = rv.revffn_prof_launches() - launches0
     assert blk.status() == 0, "device status word set during the timed region"
+    if steps_only:
+        ms_total = max_over_ranks([ms_total], world)[0]
+        if rank != 0:
+            return None
+        return {"metric": METRIC, "value": job_tokens_per_s(world, cfg.tokens, args.steps, ms_total), "unit": "tokens/s",
+                "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": f"{cfg.name}: steps only"}, "gpu_launches": int(launches), "clocks": clocks}
     # the same K steps again with an event pair around every launch: per-kernel durations
     rv.revffn_prof_enable(True)
     barrier()
@@ -954,6 +963,9 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-sample-tokens", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--steps-only", action="store_true",
+                    help="single-block runs: warm-up and the timed steps only (no per-kernel pass, no unshared variant, no "
+                         "end-to-end or CPU leg) -- the short command the profiler captures are taken from")
     ap.add_argument("--blocks", type=int, default=0, help="C3: number of layers (default: the configuration's 24)")
     ap.add_argument("--no-drift", action="store_true", help="C3: skip the per-layer drift pass")
     ap.add_argument("--seq-len", type=int, default=0, help="A1: sequence length at the same token count (default 2048)")

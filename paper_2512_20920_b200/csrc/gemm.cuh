@@ -25,6 +25,9 @@
 //            as the K range (weight gradients); output offset e * c_group_stride.
 //            With group_cnt the range may stop at the first 64-row boundary past the
 //            expert's real rows: what follows is zero padding.
+//            Without group_off the n_groups ranges are equal slices of K (a multiple of 64 rows
+//            each, the last one ends at K): a dense weight gradient split over K, whose n_groups
+//            partial results are added by splitk_reduce_kernel.
 #pragma once
 
 #include "common.cuh"
@@ -94,6 +97,39 @@ __device__ __forceinline__ float dswiglu_f(float a, float b, float dh, float& da
 // --------------------------------------------------------------------------
 constexpr int SIMT_BM = 64, SIMT_BN = 64, SIMT_BK = 16;
 
+// Rows of K per slice when a dense product is split into n equal K ranges (whole 64-row K steps).
+__host__ __device__ inline int64_t split_k_rows(int64_t K, int n) { return round_up(ceil_div(K, n), 64); }
+
+// Sum of the n partial results of a K-split weight gradient, slices in ascending order (fixed order), then what
+// the product's own epilogue would have done with the sum: write it, add it to the gradient buffer, or take the
+// fused SGD step on the weight (and its master copy).
+template <typename T>
+__global__ void splitk_reduce_kernel(const float* __restrict__ part, int n, int64_t count, float* __restrict__ out,
+                                     int accumulate, T* __restrict__ W, float* __restrict__ master, float lr) {
+  const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= count) return;
+  float4 v = *reinterpret_cast<const float4*>(part + i);
+  for (int s = 1; s < n; ++s) {
+    const float4 u = *reinterpret_cast<const float4*>(part + (int64_t)s * count + i);
+    v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
+  }
+  if (W) {
+    float w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) w[j] = master ? master[i + j] : to_f32(W[i + j]);
+    w[0] -= lr * v.x; w[1] -= lr * v.y; w[2] -= lr * v.z; w[3] -= lr * v.w;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (master) master[i + j] = w[j];
+      W[i + j] = from_f32<T>(w[j]);
+    }
+  } else {
+    float4* o = reinterpret_cast<float4*>(out + i);
+    if (accumulate) { const float4 old = *o; v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w; }
+    *o = v;
+  }
+}
+
 template <typename T>
 __device__ __forceinline__ float simt_load_a(const GemmProblem& p, int m, int64_t k, int m_lim, int64_t k_lim) {
   if (m >= m_lim || k >= k_lim) return 0.f;
@@ -128,8 +164,15 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmProblem p) {
     m_lim = total;
   } else if (p.group_mode == GROUP_K) {
     group = blockIdx.z;
-    k_begin = p.group_off[group];
-    k_end = p.group_off[group + 1];
+    if (p.group_off) {
+      k_begin = p.group_off[group];
+      k_end = p.group_off[group + 1];
+    } else {
+      const int64_t slice = split_k_rows(p.K, p.n_groups);
+      k_begin = group * slice;
+      k_end = k_begin + slice < p.K ? k_begin + slice : p.K;
+      if (k_begin > k_end) k_begin = k_end;
+    }
   }
   const T* B0 = reinterpret_cast<const T*>(p.B0);
   const T* B1 = reinterpret_cast<const T*>(p.B1);

@@ -324,6 +324,17 @@ __device__ __forceinline__ float sigmoid_approx(float x) {
   return r;
 }
 
+__device__ __forceinline__ float2 sigmoid_approx2(float2 x) {
+  const float2 t = __fmul2_rn(x, make_float2(-1.4426950408889634f, -1.4426950408889634f));
+  float e0, e1, r0, r1;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(t.x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(t.y));
+  const float2 den = __fadd2_rn(make_float2(e0, e1), make_float2(1.f, 1.f));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(den.x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(den.y));
+  return make_float2(r0, r1);
+}
+
 // Tile coordinates shared by the three roles.
 struct TcTile {
   int m0, n0, group, k_blocks, krow0;
@@ -361,10 +372,18 @@ __device__ __forceinline__ TcTile tc_tile(const TcParams& P, int w, int tiles_m_
   if (p.group_mode == GROUP_K) {
     t.group = w / per_group;
     r = w - t.group * per_group;
-    int k0 = p.group_off[t.group], k1 = p.group_off[t.group + 1];
-    t.krow0 = k0;
-    t.k_blocks = (k1 - k0) / TC_BK;
-    if (p.group_cnt) t.k_blocks = min(t.k_blocks, (p.group_cnt[t.group] + TC_BK - 1) / TC_BK);   // skip all-zero K blocks
+    if (p.group_off) {
+      int k0 = p.group_off[t.group], k1 = p.group_off[t.group + 1];
+      t.krow0 = k0;
+      t.k_blocks = (k1 - k0) / TC_BK;
+      if (p.group_cnt) t.k_blocks = min(t.k_blocks, (p.group_cnt[t.group] + TC_BK - 1) / TC_BK);   // skip all-zero K blocks
+    } else {
+      // equal slices of a dense K (split-K): rows past K in the last K step load as zeros
+      const int slice = (int)split_k_rows(p.K, p.n_groups);
+      const int k0 = min(t.group * slice, p.K), k1 = min(k0 + slice, p.K);
+      t.krow0 = k0;
+      t.k_blocks = (k1 - k0 + TC_BK - 1) / TC_BK;
+    }
   }
   int tm = r / P.tiles_n, tn = r - tm * P.tiles_n;
   t.m0 = (pair_rank >= 0) ? tm * 2 * TC_BM + pair_rank * TC_BM : tm * TC_BM;
@@ -869,7 +888,11 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             }
           }
 #pragma unroll
-          for (int i = 0; i < 32; ++i) f[i] = rs * (f[i] * sigmoid_approx(f[i]) * g[i]);
+          for (int i = 0; i < 32; i += 2) {
+            const float2 A = make_float2(f[i], f[i + 1]);
+            const float2 Hh = __fmul2_rn(__fmul2_rn(__fmul2_rn(A, sigmoid_approx2(A)), make_float2(g[i], g[i + 1])), make_float2(rs, rs));
+            f[i] = Hh.x; f[i + 1] = Hh.y;
+          }
           const uint32_t off = p.C1 ? 0u : (n_grp & 1u) * 2048u;
           if (lane == 0) { if (p.C1) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
           __syncwarp();
@@ -889,7 +912,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         // load warp's operand traffic in the copy engine or waits for a bulk store to drain, which is what
         // bounded the first version of this epilogue (a|b by TMA, two sets, three bulk stores per block).
         const float rs = (p.rowscale && m_ok) ? p.rowscale[m] : 1.f;
-        float dg = 0.f;
+        float2 dg2 = make_float2(0.f, 0.f);
 #pragma unroll 1
         for (int c = half * 32; c < t.ncols; c += 64) {
           if (!slab_ok) continue;      // warp-uniform
@@ -910,15 +933,20 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             float a[8], b[8];
             unpack8(*reinterpret_cast<const uint4*>(row_a + ((j ^ sw) << 4)), a);
             unpack8(*reinterpret_cast<const uint4*>(row_b + ((j ^ sw) << 4)), b);
+            // two elements at a time on the packed fp32 pipe (half the instructions of the scalar form)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const float v = __uint_as_float(r0[8 * j + i]);
-              const float sg = sigmoid_approx(a[i]);
-              const float si = a[i] * sg;                 // silu(a)
-              const float dh = rs * v;                    // dL/dH of this row
-              dg = fmaf(v, si * b[i], dg);                // <dH', H>: gradient of the row's gate weight
-              a[i] = dh * b[i] * (sg * (1.f + a[i] - si));   // da = dh b silu'(a), silu'(a) = s (1 + a (1 - s))
-              b[i] = dh * si;                             // db = dh silu(a)
+            for (int i = 0; i < 8; i += 2) {
+              const float2 A = make_float2(a[i], a[i + 1]), B = make_float2(b[i], b[i + 1]);
+              const float2 V = make_float2(__uint_as_float(r0[8 * j + i]), __uint_as_float(r0[8 * j + i + 1]));
+              const float2 S = sigmoid_approx2(A);
+              const float2 SI = __fmul2_rn(A, S);                         // silu(a)
+              const float2 DH = __fmul2_rn(make_float2(rs, rs), V);       // dL/dH of this row
+              dg2 = __ffma2_rn(V, __fmul2_rn(SI, B), dg2);                // <dH', H>: gradient of the row's gate weight
+              // da = dh b silu'(a), silu'(a) = s (1 + a (1 - s)) = s (1 + a - silu(a));  db = dh silu(a)
+              const float2 T1 = __fadd2_rn(__fadd2_rn(A, make_float2(1.f, 1.f)), make_float2(-SI.x, -SI.y));
+              const float2 DA = __fmul2_rn(__fmul2_rn(DH, B), __fmul2_rn(S, T1));
+              const float2 DB = __fmul2_rn(DH, SI);
+              a[i] = DA.x; a[i + 1] = DA.y; b[i] = DB.x; b[i + 1] = DB.y;
             }
             *reinterpret_cast<uint4*>(row_a + ((j ^ sw) << 4)) = pack8(a);
             *reinterpret_cast<uint4*>(row_b + ((j ^ sw) << 4)) = pack8(b);
@@ -928,7 +956,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           blk_stage_to_global(stg + 2048, lane, ds_blk + p.N + c, p.ld_ab, rows_ok);
           __syncwarp();
         }
-        if (p.dg_part && m_ok) p.dg_part[(int64_t)m * p.dg_ld + 2 * (t.n0 / P.tile_n) + half] = dg;
+        if (p.dg_part && m_ok) p.dg_part[(int64_t)m * p.dg_ld + 2 * (t.n0 / P.tile_n) + half] = dg2.x + dg2.y;
       }
       // accumulator may be overwritten by the MMA warp
       tc_fence_before();

@@ -1,6 +1,7 @@
 // C ABI, workspace planner and launch sequences of the RevFFN MoE coupling branch.
 // See include/revffn_moe.h for the contract of every entry point.
 
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -92,7 +93,7 @@ struct WsLayout {
   size_t fwd_bytes = 0;
   size_t saved_bytes = 0;   // fwd region + SwiGLU pre-activations: what a saved evaluation consists of
   // backward only
-  Buf ab, abs, gb, dz, ds, dl, dop, dg_part, tok_dl, row_dl, dlf, dur, dup, dush, du, dn, part;
+  Buf ab, abs, gb, dz, ds, dl, dop, dg_part, tok_dl, row_dl, dlf, dur, dup, dush, du, dn, part, ksplit;
   int ld_dlf = 0;
   size_t bwd_bytes = 0;
   int64_t rows_pad = 0;   // upper bound on padded rows
@@ -103,6 +104,7 @@ struct WsLayout {
 };
 
 constexpr int STRIP = 32;    // tokens per strip in two-pass column reductions
+constexpr int SPLIT_K_MAX = 4;   // most K slices of a dense weight gradient
 
 static WsLayout plan_workspace(const revffn_moe_desc& D) {
   WsLayout L;
@@ -174,6 +176,7 @@ static WsLayout plan_workspace(const revffn_moe_desc& D) {
   take(L.du, (size_t)T * d * ts);
   take(L.dn, (size_t)T * h * 4);
   take(L.part, (size_t)L.strips * d * 4);
+  take(L.ksplit, (size_t)SPLIT_K_MAX * d * h * 4);      // partial sums of the adapters' K-split weight gradients
   L.bwd_bytes = off;
   return L;
 }
@@ -530,7 +533,33 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       p.group_off = c.template p<int32_t>(L.expert_off);
       p.group_cnt = c.template p<int32_t>(L.expert_cnt);
     }
-    return run_gemm(c, p, tag);
+    // A dense weight gradient with few output tiles (the adapters': 32 tiles of 256 x 256) leaves most of the GPU
+    // idle while every tile walks all T tokens.  Split K over the tokens into as many slices as fill the GPU, write
+    // the partial results to the workspace and add them in a second, fixed-order pass, which also does what the
+    // epilogue would have done (store, accumulate or the fused update).
+    int n_split = 1;
+    if constexpr (std::is_same<T, bf16>::value) {
+      if (c.tc && !grouped && !p.split_m) {
+        const int64_t tiles = ceil_div(M, 2 * TC_BM) * ceil_div(N, 256);
+        const int pairs = tc_state().n_sms / 2;
+        n_split = (int)std::min<int64_t>(SPLIT_K_MAX, pairs / (tiles > 0 ? tiles : 1));
+        if ((size_t)n_split * M * N * 4 > L.ksplit.bytes || Tn < 64 * 8 * n_split || (M * (int64_t)N) % 4 != 0 || M % TC_BM != 0) n_split = 1;
+      }
+    }
+    if (n_split <= 1) return run_gemm(c, p, tag);
+    p.group_mode = GROUP_K; p.n_groups = n_split; p.group_off = nullptr;
+    p.C = c.template p<float>(L.ksplit); p.C2 = nullptr; p.c_group_stride = (int64_t)M * N; p.accumulate = 0;
+    p.upd_w = nullptr; p.upd_m = nullptr;
+    CKR(run_gemm(c, p, tag));
+    {
+      ProfScope ps(tag, st);
+      const int64_t count = (int64_t)M * N;
+      splitk_reduce_kernel<T><<<(unsigned)ceil_div(count, 4 * 256), 256, 0, st>>>(
+          c.template p<float>(L.ksplit), n_split, count, out, acc, upd ? reinterpret_cast<T*>(const_cast<void*>(W)) : nullptr,
+          upd ? master : nullptr, upd ? sgd->lr : 0.f);
+    }
+    CK(cudaGetLastError());
+    return REVFFN_OK;
   };
   const revffn_moe_sgd no_sgd = {};
   const revffn_moe_sgd& S = sgd ? *sgd : no_sgd;

@@ -581,13 +581,25 @@ __global__ void map_scan_kernel(const int32_t* __restrict__ chunk_cnt, int n_chu
                                 int32_t* __restrict__ rows_total, int max_tiles, int4* __restrict__ tok_chunks,
                                 int max_chunks) {
   extern __shared__ int32_t sm_i[];          // [E+1] padded offsets
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+  // Per expert, the exclusive prefix sum of its chunk counts: a warp per expert, 32 chunks per round, so the
+  // dependent loads of a round are one round trip (a thread per expert walking its chunks one by one spent a
+  // memory latency per chunk).
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  for (int e = warp; e < E; e += n_warps) {
     int run = 0;
-    for (int c = 0; c < n_chunks; ++c) {
-      chunk_base[(int64_t)c * E + e] = run;
-      run += chunk_cnt[(int64_t)c * E + e];
+    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+      const int c = c0 + lane;
+      const int v = c < n_chunks ? chunk_cnt[(int64_t)c * E + e] : 0;
+      int incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += u;
+      }
+      if (c < n_chunks) chunk_base[(int64_t)c * E + e] = run + incl - v;
+      run += __shfl_sync(0xffffffffu, incl, 31);
     }
-    expert_cnt[e] = run;
+    if (lane == 0) expert_cnt[e] = run;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
