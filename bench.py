@@ -35,16 +35,16 @@ METRIC = "RevFFN MoE block fwd+inverse+bwd tokens/s; % of B200 bf16 tensor peak"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # DRAM traffic per launch (bytes) at C1 from one single-pass ncu capture at full size
-# (dram__bytes_read.sum + dram__bytes_write.sum; profiles/traffic_gemm_expert_gate_up_C1.md).
+# (dram__bytes_read.sum + dram__bytes_write.sum; profiles/tensor_pipe_gemms_C1.md).
 # Keyed by pass/kernel; anything else, or any other workload, reports null.
 NCU_TRAFFIC_BYTES = {
-    "fwd/gemm_expert_gate_up_swiglu": 937_895_936, "inv/gemm_expert_gate_up_swiglu": 1_126_080_512,
-    "fwd/gemm_shared_gate_up_swiglu": 189_896_960, "inv/gemm_shared_gate_up_swiglu": 414_986_240,
+    "fwd/gemm_expert_gate_up_swiglu": 935_900_000, "inv/gemm_expert_gate_up_swiglu": 1_131_000_000,
+    "fwd/gemm_shared_gate_up_swiglu": 178_500_000, "inv/gemm_shared_gate_up_swiglu": 420_900_000,
 }
 
 
 NCU_TRAFFIC_SOURCE = ("stored figure, not measured in this run: dram__bytes_read.sum + dram__bytes_write.sum of one "
-                      "single-pass ncu capture at this size, profiles/traffic_gemm_expert_gate_up_C1.md")
+                      "ncu capture of this kernel at this size, profiles/tensor_pipe_gemms_C1.md")
 GROUPED_EXPERT_KERNELS = ("gemm_expert_gate_up_swiglu", "gemm_expert_down_scale", "gemm_expert_dh_dswiglu",
                           "gemm_expert_du", "wgrad_expert_down", "wgrad_expert_gate", "wgrad_expert_up",
                           "wgrad_expert_gate_up")
