@@ -40,6 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES = {
     "fwd/gemm_expert_gate_up_swiglu": 935_900_000, "inv/gemm_expert_gate_up_swiglu": 1_131_000_000,
     "fwd/gemm_shared_gate_up_swiglu": 178_500_000, "inv/gemm_shared_gate_up_swiglu": 420_900_000,
+    "bwd/wgrad_expert_gate_up": 1_663_200_000, "bwd/wgrad_expert_down": 874_900_000,
 }
 
 
@@ -90,6 +91,18 @@ def gemm_flops(cfg, routed_rows):
         "wgrad_expert_gate_up": 2 * R * 2 * I * d,
         "gemm_dn": 2 * T * d * h, "wgrad_p_up": 2 * T * d * h,
     }
+
+
+def gemm_bytes(cfg, routed_rows):
+    """Algorithmic DRAM bytes per launch of the products whose output is large against their flops (the weight
+    gradients of the experts: fp32 [E, I, d]-shaped results from about 546 rows of K each): every operand read
+    once, every result written once.  A launch is held against the HBM roofline when these bytes at the measured
+    copy bandwidth take longer than its flops at the measured tensor peak."""
+    d, I, E = cfg.d_model, cfg.d_expert, cfg.n_experts
+    R = routed_rows
+    out = E * I * d * 4
+    return {"wgrad_expert_down": out + R * d * 2 + R * I * 2, "wgrad_expert_gate": out + R * I * 2 + R * d * 2,
+            "wgrad_expert_up": out + R * I * 2 + R * d * 2, "wgrad_expert_gate_up": 2 * out + R * 2 * I * 2 + R * d * 2}
 
 
 class ClockSampler:
@@ -421,6 +434,23 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
                     "share_of_step": ms / (ms_prof_step * args.steps),
                     "timed_over": f"a second pass of the same {args.steps} steps with a CUDA-event pair around "
                                   f"every launch ({ms_prof_step:.3f} ms per step against {ms_step:.3f} without)"}
+        nbytes = gemm_bytes(cfg, routed_rows).get(kn)
+        if nbytes and nbytes / (peaks["hbm_gbs"] * 1e9) > flops[kn] / (peak * 1e12):
+            # this launch moves more bytes than it can compute on: HBM is its roofline
+            gbs = nbytes / (ms / cnt * 1e-3) / 1e9
+            roofline.update(bound="hbm", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s", frac=gbs / peaks["hbm_gbs"],
+                            peak_source=f"{peak_kind}: hbm_gbs of MEASURED_PEAKS.json (copy bandwidth)",
+                            algorithmic_bytes=nbytes, traffic=NCU_TRAFFIC_BYTES.get(name) if cfg.name == "C1" else None,
+                            traffic_source=NCU_TRAFFIC_SOURCE if (cfg.name == "C1" and name in NCU_TRAFFIC_BYTES) else None,
+                            why=f"{nbytes / 1e6:.0f} MB of operands and fp32 results at the copy bandwidth take "
+                                f"{nbytes / (peaks['hbm_gbs'] * 1e9) * 1e3:.3f} ms, its {flops[kn] / 1e12:.3f} TFLOP at the tensor peak "
+                                f"{flops[kn] / (peak * 1e12) * 1e3:.3f} ms; the tensor view of the same launch is under 'dominant'")
+        # the largest launch that the tensor pipe bounds, for comparison with earlier records
+        dom_t = next(((m_, c_, n_, k_) for m_, c_, n_, k_ in kernels if k_ in flops and k_ not in gemm_bytes(cfg, routed_rows)), None)
+        if dom_t:
+            roofline["largest_tensor_bound_launch"] = dict(tensor_fractions(flops[dom_t[3]] / (dom_t[0] / dom_t[1] * 1e-3) / 1e12),
+                                                           kernel=dom_t[2], launch_ms=dom_t[0] / dom_t[1],
+                                                           traffic=NCU_TRAFFIC_BYTES.get(dom_t[2]) if cfg.name == "C1" else None)
         if g_ms > 0:
             # the quantity the target is stated on: every expert-grouped product of the step together
             roofline["grouped"] = dict(tensor_fractions(g_fl / (g_ms * 1e-3) / 1e12), ms_per_step=g_ms / args.steps,
