@@ -270,7 +270,7 @@ inline cudaError_t launch_fold_router_mma(const T* w_router, const T* w_sgate, c
 //            per warp read fewer operand values per instruction, but a batch of 8192 tokens
 //            then fills the GPU with one block of 8 warps per SM, which cannot hide the
 //            latency of its own loads: 32-token blocks, two or three to an SM, took the kernel
-//            from 0.106 to the time recorded in the design notes.)  (A register-tiled DFMA version of the same product
+//            from 0.106 to 0.083 ms.)  (A register-tiled DFMA version of the same product
 //            spent its time on shared-memory operand reads: 8 values per 16 FMAs.)
 //            The staging threads also sum y^2 (fp64), which gives
 //            r_t = (mean(y_t^2)+eps)^-1/2; the scale is applied to the finished sums.
