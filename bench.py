@@ -390,10 +390,15 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
     # per-pass and per-kernel accounting
     passes = {"fwd": 0.0, "inv": 0.0, "bwd": 0.0}
     kernels = []
-    for name, (ms, cnt) in prof.items():
+    # A profiler slot is one product (or kernel) of one pass; some products run as several launches (row pairs +
+    # odd tiles of the experts, K slices + their sum): the slot's time is the sum, its flops are counted once per
+    # step.  `cnt` below is therefore the number of times the PRODUCT ran (= steps), `launches` the kernel launches.
+    slot_launches = {}
+    for name, (ms, launches_) in prof.items():
         ps, kn = name.split("/")
         passes[ps] += ms / args.steps
-        kernels.append((ms, cnt, name, kn))
+        slot_launches[name] = launches_
+        kernels.append((ms, args.steps, name, kn))
     kernels.sort(reverse=True)
     step_flops = {"fwd": 0.0, "inv": 0.0, "bwd": 0.0}
     for ms, cnt, name, kn in kernels:
@@ -454,11 +459,11 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
         if g_ms > 0:
             # the quantity the target is stated on: every expert-grouped product of the step together
             roofline["grouped"] = dict(tensor_fractions(g_fl / (g_ms * 1e-3) / 1e12), ms_per_step=g_ms / args.steps,
-                                       launches_per_step=sum(k[1] for k in grouped) / args.steps,
+                                       launches_per_step=sum(slot_launches[k[2]] for k in grouped) / args.steps,
                                        share_of_step=g_ms / (ms_prof_step * args.steps),
                                        kernels=sorted({k[3] for k in grouped}))
         roofline["whole_step"] = tensor_fractions(total_flops / (ms_step * 1e-3) / 1e12)
-    top = [{"kernel": name, "ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps,
+    top = [{"kernel": name, "ms_per_step": ms / args.steps, "launches_per_step": slot_launches[name] / args.steps,
             "tflops": (flops[kn] * cnt / (ms * 1e-3) / 1e12) if kn in flops and ms > 0 else None}
            for ms, cnt, name, kn in kernels]
 

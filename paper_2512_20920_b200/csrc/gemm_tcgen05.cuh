@@ -505,8 +505,15 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             if (!p.b_mn_major) {
               // this CTA's 128 of the 256 accumulator columns: gate rows (rank 0) or up rows (rank 1) of a
               // SwiGLU pair, else rows n0 + 128 rank .. + 127 of B
-              if (p.concat == CONCAT_N) tma_load_2d_pair(sb, crank == 0 ? &map_b0 : &map_b1, kbp * TC_BK, t.n0, fbc);
-              else tma_load_2d_pair(sb, mbp, kbp * TC_BK, t.n0 + 128 * crank, fbc);
+              // (the tensor map is named directly in each call: a map chosen through a pointer is slow to issue)
+              if (p.concat == CONCAT_N) {
+                if (crank == 0) tma_load_2d_pair(sb, &map_b0, kbp * TC_BK, t.n0, fbc);
+                else tma_load_2d_pair(sb, &map_b1, kbp * TC_BK, t.n0, fbc);
+              } else if (p.concat == CONCAT_K && kb >= k_half) {
+                tma_load_2d_pair(sb, &map_b1, kbp * TC_BK, t.n0 + 128 * crank, fbc);
+              } else {
+                tma_load_2d_pair(sb, &map_b0, kbp * TC_BK, t.n0 + 128 * crank, fbc);
+              }
             } else {
               const int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
               (void)kdim;
