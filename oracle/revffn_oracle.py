@@ -120,6 +120,53 @@ def gate_weights(L: np.ndarray, idx: np.ndarray, gating: str = "renorm") -> np.n
 
 
 # --------------------------------------------------------------------------- #
+# FP8 variant of the routed experts (not in the paper: a variant of MLP_pt's arithmetic in
+# which the routed experts' three products take e4m3 operands, each row of an operand scaled
+# by its own power-free fp32 factor).  The quantisation DECIDES integer codes, so it is
+# written in the precision the kernels use: operands are first rounded to bf16 (what the
+# kernels hold), the scale and the scaled value are fp32, the code is e4m3 by round to
+# nearest even with saturation to the largest finite value.
+# --------------------------------------------------------------------------- #
+E4M3_MAX = 448.0
+
+
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """fp32 values rounded to the nearest bf16 value (ties to even), returned as fp32."""
+    u = np.asarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32)
+
+
+def e4m3_round(v: np.ndarray) -> np.ndarray:
+    """Nearest e4m3 value (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities; ties to the
+    even mantissa; magnitudes beyond 448 saturate to 448), returned as fp32."""
+    v = np.asarray(v, dtype=np.float32)
+    a = np.abs(v).astype(np.float64)
+    _, e = np.frexp(a)                       # a = m * 2^e with m in [0.5, 1)
+    e = np.maximum(e - 1, -6)                # exponent of the leading bit; subnormals share the exponent -6
+    step = np.ldexp(1.0, e - 3)              # spacing of e4m3 values in that binade
+    q = np.rint(a / step) * step             # np.rint rounds halves to even
+    q = np.minimum(q, E4M3_MAX)
+    return (np.sign(v) * q).astype(np.float32)
+
+
+def quantize_rows_e4m3(x: np.ndarray):
+    """Per row: scale = max|x| / 448 (1 for an all-zero row), codes = e4m3_round(x / scale), all in fp32.
+    Returns (dequantised codes as fp32 [rows, cols] -- the values the product sums --, scale [rows])."""
+    x = np.asarray(x, dtype=np.float32)
+    amax = np.max(np.abs(x), axis=-1)
+    scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    q = e4m3_round((x / scale[..., None]).astype(np.float32))
+    return q, scale
+
+
+def fp8_matmul(xq, xs, wq, ws):
+    """(x W^T) with both operands quantised per row: the exact sum of products of the codes, then the two scales."""
+    acc = xq.astype(F64) @ wq.astype(F64).T
+    return acc * xs.astype(F64)[:, None] * ws.astype(F64)[None, :]
+
+
+# --------------------------------------------------------------------------- #
 # One token, written out step by step (the definition)
 # --------------------------------------------------------------------------- #
 def branch_token(p, y: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
@@ -151,10 +198,13 @@ def branch_token(p, y: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
 # All tokens (same arithmetic, tokens grouped per expert so matmul can be used)
 # --------------------------------------------------------------------------- #
 def branch(p, Y1: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
-           route_override: Optional[np.ndarray] = None, keep: bool = False, gating: str = "renorm"):
+           route_override: Optional[np.ndarray] = None, keep: bool = False, gating: str = "renorm",
+           fp8_experts: bool = False):
     """F[T,h] = MLP(Norm(Y1)) for all tokens.  Returns (F, info); info holds the
     routing (idx, gates, margin, logits) and, with keep=True, the intermediates
-    the backward pass needs."""
+    the backward pass needs.  fp8_experts: the routed experts' products take e4m3 operands
+    (see quantize_rows_e4m3): u and g*H are rounded to bf16 and quantised per token row, the
+    expert weights per output row; everything else is unchanged."""
     Y1 = np.asarray(Y1, dtype=F64)
     T = Y1.shape[0]
     n, r = norm_fwd(Y1, p.get("norm_gamma"), eps, norm)
@@ -171,6 +221,15 @@ def branch(p, Y1: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
         if toks.size == 0:
             continue
         ue = u[toks]
+        if fp8_experts:
+            uq, us = quantize_rows_e4m3(round_bf16(ue.astype(np.float32)))
+            a = fp8_matmul(uq, us, *quantize_rows_e4m3(np.asarray(p["w_gate"][e], np.float32)))
+            b = fp8_matmul(uq, us, *quantize_rows_e4m3(np.asarray(p["w_upx"][e], np.float32)))
+            # the gate weight goes onto H before it is rounded and quantised (as the kernels do)
+            hg = round_bf16((g[toks, slots][:, None] * (silu(a) * b)).astype(np.float32))
+            hq, hs = quantize_rows_e4m3(hg)
+            z[toks] += fp8_matmul(hq, hs, *quantize_rows_e4m3(np.asarray(p["w_downx"][e], np.float32)))
+            continue
         a = ue @ _w(p, "w_gate", e).T
         b = ue @ _w(p, "w_upx", e).T
         hm = silu(a) * b
@@ -195,16 +254,18 @@ def branch(p, Y1: np.ndarray, k: int, eps: float = 1e-6, norm: str = "rms",
     return F, info
 
 
-def forward(p, Y1, X2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None, gating: str = "renorm"):
+def forward(p, Y1, X2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None, gating: str = "renorm",
+            fp8_experts: bool = False):
     """Eq. 2: Y2 = X2 + MLP(Norm(Y1)).  Returns (Y2, info)."""
-    F, info = branch(p, Y1, k, eps, norm, route_override, gating=gating)
+    F, info = branch(p, Y1, k, eps, norm, route_override, gating=gating, fp8_experts=fp8_experts)
     info["F"] = F
     return np.asarray(X2, dtype=F64) + F, info
 
 
-def inverse(p, Y1, Y2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None, gating: str = "renorm"):
+def inverse(p, Y1, Y2, k: int, eps: float = 1e-6, norm: str = "rms", route_override=None, gating: str = "renorm",
+            fp8_experts: bool = False):
     """Inverse pass of Sec. 3.1: X2 = Y2 - MLP(Norm(Y1)).  Returns (X2, info)."""
-    F, info = branch(p, Y1, k, eps, norm, route_override, gating=gating)
+    F, info = branch(p, Y1, k, eps, norm, route_override, gating=gating, fp8_experts=fp8_experts)
     info["F"] = F
     return np.asarray(Y2, dtype=F64) - F, info
 

@@ -435,3 +435,93 @@ def test_sgd_step_descends_by_lr_times_the_squared_gradient_norm():
     # an ascent step does the opposite
     up = orc.sgd_step(p, g, -1e-5, names)
     assert loss(up) > L0 > loss(orc.sgd_step(p, g, 1e-5, names))
+
+
+# ------------------------------------------------------------------ FP8 variant of the routed experts
+def _e4m3_table():
+    """Every finite e4m3 value from the format's definition: 1 sign bit, 4 exponent bits (bias 7), 3 mantissa bits,
+    exponent field 0 = subnormal, the code S.1111.111 is NaN, no infinities."""
+    vals = []
+    for ebits in range(16):
+        for m in range(8):
+            if ebits == 15 and m == 7:
+                continue
+            vals.append(m / 8 * 2.0 ** -6 if ebits == 0 else (1 + m / 8) * 2.0 ** (ebits - 7))
+    return np.array(sorted(set(vals)))
+
+
+def test_e4m3_rounding_against_the_value_table_and_the_library_cast():
+    tab = _e4m3_table()
+    assert tab.max() == 448.0 and tab[1] == 2.0 ** -9 and len(tab) == 127
+    assert np.array_equal(orc.e4m3_round(tab.astype(np.float32)), tab.astype(np.float32))          # representable values stay
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.standard_normal(20000) * 100, rng.standard_normal(20000) * 0.01, rng.uniform(-448, 448, 20000),
+                        (tab[:-1] + tab[1:]) / 2, -(tab[:-1] + tab[1:]) / 2]).astype(np.float32)      # incl. every tie
+    got = orc.e4m3_round(x)
+    # brute force: nearest table value, ties to the even mantissa (= even position in the table), saturation
+    a = np.minimum(np.abs(x.astype(np.float64)), 448.0)
+    j = np.searchsorted(tab, a)
+    lo, hi = tab[np.maximum(j - 1, 0)], tab[np.minimum(j, len(tab) - 1)]
+    pick_hi = (hi - a < a - lo) | ((hi - a == a - lo) & (np.minimum(j, len(tab) - 1) % 2 == 0))
+    want = np.sign(x) * np.where(pick_hi, hi, lo)
+    assert np.array_equal(got.astype(np.float64), want)
+    # the installed library's cast (no saturation there: stay inside the finite range)
+    inside = np.abs(x) <= 448
+    lib = torch.from_numpy(x[inside]).to(torch.float8_e4m3fn).to(torch.float32).numpy()
+    assert np.array_equal(got[inside], lib)
+    assert np.array_equal(orc.e4m3_round(np.array([449, 1e6, -500], np.float32)), np.array([448, 448, -448], np.float32))
+    # bf16 rounding against the library's cast
+    y = (rng.standard_normal(50000) * 3).astype(np.float32)
+    assert np.array_equal(orc.round_bf16(y), torch.from_numpy(y).to(torch.bfloat16).to(torch.float32).numpy())
+
+
+def test_row_quantisation_scales_and_error_bound():
+    rng = np.random.default_rng(1)
+    x = (rng.standard_normal((37, 96)) * rng.uniform(0.01, 30, (37, 1))).astype(np.float32)
+    x[5] = 0
+    q, s = orc.quantize_rows_e4m3(x)
+    assert s[5] == 1 and (q[5] == 0).all()
+    assert np.allclose(np.abs(q).max(axis=1)[np.arange(37) != 5], 448.0)          # the row maximum maps onto the largest code
+    back = q * s[:, None]
+    # relative error of a normal e4m3 value is at most 2^-4; tiny entries sit on the subnormal grid 2^-9 * scale
+    assert (np.abs(back - x) <= np.maximum(np.abs(x) * 2.0 ** -4, s[:, None] * 2.0 ** -10) * (1 + 1e-6)).all()
+    # a product of quantised operands is the product of the dequantised ones
+    w = (rng.standard_normal((11, 96)) * 0.05).astype(np.float32)
+    wq, ws_ = orc.quantize_rows_e4m3(w)
+    f64 = np.float64
+    assert np.allclose(orc.fp8_matmul(q, s, wq, ws_), (q.astype(f64) * s.astype(f64)[:, None]) @ (wq.astype(f64) * ws_.astype(f64)[:, None]).T, rtol=1e-12)
+
+
+def test_fp8_experts_is_the_branch_with_quantised_expert_operands():
+    """Written a second time with the library's casts: the FP8 branch equals the plain branch evaluated on
+    dequantised operands at the three expert products; and it stays within the format's error of the exact one."""
+    cfg, p, s = _tiny(seed=6, d_model=64, d_expert=32, d_shared=32, tokens=19)
+    F8, info = orc.branch(p, s["y1"], cfg.top_k, cfg.norm_eps, fp8_experts=True)
+    F, info0 = orc.branch(p, s["y1"], cfg.top_k, cfg.norm_eps)
+    assert np.array_equal(info["idx"], info0["idx"]) and np.allclose(info["gates"], info0["gates"])     # routing is untouched
+
+    def q8(t):      # per-row e4m3 through torch, dequantised
+        amax = t.abs().amax(dim=-1, keepdim=True)
+        sc = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
+        return (t / sc).to(torch.float8_e4m3fn).to(torch.float32).double() * sc.double()
+
+    n, _ = orc.norm_fwd(s["y1"], p["norm_gamma"], cfg.norm_eps)
+    u = n @ p["w_up"].astype(np.float64).T
+    z = np.zeros_like(u)
+    for t in range(cfg.tokens):
+        ub = q8(torch.from_numpy(u[t:t + 1].astype(np.float32)).to(torch.bfloat16).float())
+        for slot, e in enumerate(info["idx"][t]):
+            a = ub @ q8(torch.from_numpy(p["w_gate"][e])).T
+            b = ub @ q8(torch.from_numpy(p["w_upx"][e])).T
+            hg = (info["gates"][t, slot] * torch.nn.functional.silu(a) * b).float().to(torch.bfloat16).float()
+            z[t] += (q8(hg) @ q8(torch.from_numpy(p["w_downx"][e])).T).numpy()[0]
+    a_s = u @ p["ws_gate"].astype(np.float64).T
+    S = (orc.silu(a_s) * (u @ p["ws_up"].astype(np.float64).T)) @ p["ws_down"].astype(np.float64).T
+    z += info["sgate"][:, None] * S
+    assert np.allclose(F8, z @ p["w_down"].astype(np.float64).T, rtol=1e-9, atol=1e-12)
+    err = np.linalg.norm(F8 - F) / np.linalg.norm(F)
+    assert 1e-3 < err < 1e-1          # the quantisation is visible, and of the size three bits of mantissa give
+    # forward then inverse with the same arithmetic reconstructs exactly
+    y2, _ = orc.forward(p, s["y1"], s["x2"], cfg.top_k, cfg.norm_eps, fp8_experts=True)
+    x2, _ = orc.inverse(p, s["y1"], y2, cfg.top_k, cfg.norm_eps, fp8_experts=True)
+    assert np.max(np.abs(x2 - s["x2"])) < 1e-10
