@@ -129,6 +129,15 @@ enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                
  * set the flag.  The caller vouches that the three tensors are unchanged since that call and that no
  * call with another descriptor has used the workspace in between. */
 #define REVFFN_FLAG_ROUTER_FOLDED 128u
+/* FP8 routed experts (forward and inverse passes; bf16 weights only; no paper counterpart: a variant of the
+ * arithmetic of MLP_pt's routed experts).  The three products of the routed experts take e4m3 operands with fp32
+ * accumulation: each token row of u and of g*H is scaled by max|row| / 448 and rounded to e4m3 on the fly, and the
+ * expert weights come quantised per output row from revffn_moe_quantize_experts (the q_* / s_* members of
+ * revffn_moe_weights; the bf16 weights stay the master copy).  Three bits of mantissa put the branch output about
+ * 4 % (relative L2) away from the bf16 evaluation; forward and inverse still add and subtract bit-identical
+ * branches.  Not with REVFFN_FLAG_FORCE_SIMT, SAVE/REUSE_ACTIVATIONS or in revffn_moe_backward
+ * (REVFFN_ERR_UNSUPPORTED): gradients are taken on the bf16 path. */
+#define REVFFN_FLAG_FP8_EXPERTS 256u
 
 /*
  * Block descriptor.  Shape constraints (else REVFFN_ERR_SHAPE):
@@ -164,6 +173,14 @@ typedef struct {
   const void* ws_up;       /* [I_s, d]                                                   */
   const void* ws_down;     /* [d, I_s]                                                   */
   const void* ws_sgate;    /* [d]      shared-expert sigmoid gate                        */
+  /* REVFFN_FLAG_FP8_EXPERTS only (NULL otherwise): e4m3 codes and fp32 per-output-row scales of the expert
+   * weights, written by revffn_moe_quantize_experts from the bf16 weights above. */
+  const void* q_gate;      /* [E, I, d] e4m3                                             */
+  const void* q_upx;       /* [E, I, d] e4m3                                             */
+  const void* q_downx;     /* [E, d, I] e4m3                                             */
+  const float* s_gate;     /* [E, I] fp32                                                */
+  const float* s_upx;      /* [E, I] fp32                                                */
+  const float* s_downx;    /* [E, d] fp32                                                */
 } revffn_moe_weights;
 
 /*
@@ -260,6 +277,15 @@ int revffn_moe_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weight
                             const float* y1, const float* dy2, float* dy1_inout,
                             const revffn_moe_grads* grads, const revffn_moe_sgd* sgd, const int32_t* topk_idx_in,
                             void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Quantise the bf16 expert weights for REVFFN_FLAG_FP8_EXPERTS: per output row r of w_gate / w_upx ([E*I] rows of
+ * d) and of w_downx ([E*d] rows of I), scale[r] = max|row| / 448 (1 for an all-zero row) and
+ * code = e4m3(w / scale[r]), round to nearest even, saturating.  Writes the six q_* / s_* buffers named in `w`
+ * (caller-owned device memory of the sizes given at revffn_moe_weights, 16-byte aligned); call again whenever
+ * the bf16 weights change.  Needs d and I to be multiples of 128 and at most 2048.  Enqueued on the stream.
+ */
+int revffn_moe_quantize_experts(const revffn_moe_desc* desc, const revffn_moe_weights* w, void* cuda_stream);
 
 /* Synchronise the stream and copy the workspace's device status word to
  * *device_status (host pointer): 0 or a negative revffn_error.  (No paper counterpart.) */

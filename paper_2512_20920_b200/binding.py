@@ -23,6 +23,7 @@ FLAG_ROUTING_RECORD = 16
 FLAG_KEEP_STATUS = 32
 FLAG_DEBUG_CHECKS = 64
 FLAG_ROUTER_FOLDED = 128
+FLAG_FP8_EXPERTS = 256
 
 ERR_DEVICE_WAIT, ERR_UNSUPPORTED, ERR_NOALLOC_LIMIT, ERR_INDEX, ERR_CANARY, ERR_NONFINITE = -7, -8, -9, -10, -11, -12
 
@@ -43,8 +44,11 @@ class Desc(C.Structure):
                 ("norm_kind", C.c_int32), ("norm_eps", C.c_float), ("ld_stream", C.c_int64), ("flags", C.c_uint32)]
 
 
+FP8_NAMES = ("q_gate", "q_upx", "q_downx", "s_gate", "s_upx", "s_downx")      # e4m3 codes and fp32 row scales of the experts
+
+
 class Weights(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES + FP8_NAMES]
 
 
 class Grads(C.Structure):
@@ -126,6 +130,8 @@ def _load() -> C.CDLL:
     lib.revffn_moe_stack_backward_sgd.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp,
                                                   C.POINTER(Grads), C.POINTER(Sgd), vp, vp, sz, vp, sz, vp]
     lib.revffn_moe_stack_backward_sgd.restype = C.c_int
+    lib.revffn_moe_quantize_experts.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp]
+    lib.revffn_moe_quantize_experts.restype = C.c_int
     lib.revffn_moe_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
     lib.revffn_strerror.argtypes = [C.c_int]
     lib.revffn_strerror.restype = C.c_char_p
@@ -373,6 +379,22 @@ class Block:
     @property
     def tokens(self) -> int:
         return self.desc.tokens
+
+    def quantize_experts(self) -> Dict[str, torch.Tensor]:
+        """Buffers for the e4m3 copies of the expert weights and their row scales, filled by
+        revffn_moe_quantize_experts and entered into this block's weight struct (needed with FLAG_FP8_EXPERTS)."""
+        E, I, d = self.desc.n_experts, self.desc.d_expert, self.desc.d_model
+        q = {"q_gate": torch.empty(E, I, d, dtype=torch.uint8, device="cuda"),
+             "q_upx": torch.empty(E, I, d, dtype=torch.uint8, device="cuda"),
+             "q_downx": torch.empty(E, d, I, dtype=torch.uint8, device="cuda"),
+             "s_gate": torch.empty(E, I, dtype=torch.float32, device="cuda"),
+             "s_upx": torch.empty(E, I, dtype=torch.float32, device="cuda"),
+             "s_downx": torch.empty(E, d, dtype=torch.float32, device="cuda")}
+        for n, t in q.items():
+            setattr(self.w, n, _ptr(t))
+        self.fp8 = q
+        _check(lib.revffn_moe_quantize_experts(C.byref(self.desc), C.byref(self.w), _stream()), "revffn_moe_quantize_experts")
+        return q
 
     def _desc(self, extra_flags: int) -> Desc:
         if not extra_flags:

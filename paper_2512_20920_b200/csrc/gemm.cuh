@@ -67,6 +67,10 @@ struct GemmProblem {
   // W <- W - upd_lr * g (W of the operand type, same layout as C; upd_w2 goes with C2's rows).  With a master
   // copy (fp32, same layout) the step is taken there and W receives the rounded result.  C / C2 may then be NULL.
   void* upd_w; void* upd_w2; float* upd_m; float* upd_m2; float upd_lr;
+  // tcgen05 back end, fp8 operands (both K-major): A and B hold e4m3 codes, one byte per element; the accumulator
+  // is multiplied by a_scale[row] * b_scale[(group * N +) column] before the epilogue's own arithmetic
+  // (b_scale1: the second matrix of an N-concatenated pair).  lda / ldb / K count elements (= bytes).
+  int fp8; const float* a_scale; const float* b_scale0; const float* b_scale1;
   int no_pair;        // tcgen05 back end: never pair CTAs for this product
   long long dbg_wait_cycles;   // tcgen05 back end, tests: bound on every device-side wait (0 = default)
   int dbg_starve;              // tcgen05 back end, tests (needs no_pair): no operand loads are issued

@@ -82,6 +82,7 @@ struct TcParams {
   uint32_t idesc;
   long long wait_cycles;     // bound on every wait of the kernel (clock cycles)
   int starve;                // failure-path test: the load warp issues nothing, so the first wait for operands runs out
+  int bk;                    // operand elements per K step: 64 (bf16) or 128 (e4m3); a K step is 128 bytes of a row either way
 };
 
 // ---------------------------------------------------------------------------
@@ -187,6 +188,28 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, ui
 
 // One product with the descriptors given as (low, high) words: the high words never change inside a kernel, and
 // the low words move by small additions, so the issuing thread carries 32-bit values only.
+// The same for e4m3 operands (kind::f8f6f4: 32 one-byte elements of K per instruction, the same 32 bytes).
+template <bool PAIR>
+__device__ __forceinline__ void tc_mma_lohi_f8(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                               uint32_t idesc, uint32_t acc) {
+  if constexpr (PAIR)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");
+}
+
 template <bool PAIR>
 __device__ __forceinline__ void tc_mma_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
                                             uint32_t idesc, uint32_t acc) {
@@ -479,14 +502,14 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
               int kw = kb;
               if (p.concat == CONCAT_K && kb >= k_half) { mw = &map_b1; kw = kb - k_half; }
               if (!p.b_mn_major) {
-                tma_load_2d_pair(sa, mw, kw * TC_BK, t.group * p.N + t.n0, fbc);
+                tma_load_2d_pair(sa, mw, kw * P.bk, t.group * p.N + t.n0, fbc);
               } else {
                 const int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
                 const int krow = t.group * kdim + kw * TC_BK;
 #pragma unroll
                 for (int j = 0; j < 2; ++j) tma_load_2d_pair(sa + j * 8192, mw, p.b_col0 + t.n0 + 64 * j, krow, fbc);
               }
-              tma_load_2d_pair(sb, &map_a, kb * TC_BK, t.m0 + crank * (t.ncols / 2), fbc);
+              tma_load_2d_pair(sb, &map_a, kb * P.bk, t.m0 + crank * (t.ncols / 2), fbc);
               if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
               continue;
             }
@@ -530,7 +553,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
           issued[stage] = (int)phase + 1;
           // A tile
           if (!p.a_mn_major) {
-            tma_load_2d(sa, &map_a, kb * TC_BK, t.m0, fb);
+            tma_load_2d(sa, &map_a, kb * P.bk, t.m0, fb);
           } else {
             int krow = t.krow0 + kb * TC_BK;
 #pragma unroll
@@ -544,12 +567,12 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             // rows of the flattened [groups * N, K] weight tensor
             int row0 = (p.group_mode == GROUP_M ? t.group * p.N : 0) + t.n0;
             if (p.concat == CONCAT_N) {
-              tma_load_2d(sb, &map_b0, kb_b * TC_BK, row0, fb);
-              tma_load_2d(sb + 16384, &map_b1, kb_b * TC_BK, row0, fb);
+              tma_load_2d(sb, &map_b0, kb_b * P.bk, row0, fb);
+              tma_load_2d(sb + 16384, &map_b1, kb_b * P.bk, row0, fb);
             } else {
 #pragma unroll
               for (int j = 0; j < MMA_N / 128; ++j)
-                if (128 * j < t.ncols) tma_load_2d(sb + j * 16384, mb, kb_b * TC_BK, row0 + 128 * j, fb);
+                if (128 * j < t.ncols) tma_load_2d(sb + j * 16384, mb, kb_b * P.bk, row0 + 128 * j, fb);
             }
           } else {
             // rows of the flattened [groups * Kdim, N] weight tensor, or token rows (GROUP_K / dense wgrad)
@@ -598,10 +621,17 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         for (int kb = 0; kb < nk; ++kb) {
           if (!mbar_wait(fbar, phase, abort_flag, p.status, P.wait_cycles)) { ok = false; break; }
           tc_fence_after();
-          tc_mma_lohi<PAIR>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, kb != 0 ? 1u : 0u);
-          tc_mma_lohi<PAIR>(d_tmem, a_lo + a_step, a_hi, b_lo + b_step, b_hi, idesc, 1u);
-          tc_mma_lohi<PAIR>(d_tmem, a_lo + 2 * a_step, a_hi, b_lo + 2 * b_step, b_hi, idesc, 1u);
-          tc_mma_lohi<PAIR>(d_tmem, a_lo + 3 * a_step, a_hi, b_lo + 3 * b_step, b_hi, idesc, 1u);
+          if (p.fp8) {
+            tc_mma_lohi_f8<PAIR>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, kb != 0 ? 1u : 0u);
+            tc_mma_lohi_f8<PAIR>(d_tmem, a_lo + a_step, a_hi, b_lo + b_step, b_hi, idesc, 1u);
+            tc_mma_lohi_f8<PAIR>(d_tmem, a_lo + 2 * a_step, a_hi, b_lo + 2 * b_step, b_hi, idesc, 1u);
+            tc_mma_lohi_f8<PAIR>(d_tmem, a_lo + 3 * a_step, a_hi, b_lo + 3 * b_step, b_hi, idesc, 1u);
+          } else {
+            tc_mma_lohi<PAIR>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, kb != 0 ? 1u : 0u);
+            tc_mma_lohi<PAIR>(d_tmem, a_lo + a_step, a_hi, b_lo + b_step, b_hi, idesc, 1u);
+            tc_mma_lohi<PAIR>(d_tmem, a_lo + 2 * a_step, a_hi, b_lo + 2 * b_step, b_hi, idesc, 1u);
+            tc_mma_lohi<PAIR>(d_tmem, a_lo + 3 * a_step, a_hi, b_lo + 3 * b_step, b_hi, idesc, 1u);
+          }
           // stage reusable once these MMAs have read it (in both CTAs of a pair)
           if constexpr (PAIR) tc_commit_pair(ebar); else tc_commit(ebar);
           a_lo += SB16; b_lo += SB16; fbar += 8u; ebar += 8u;
@@ -674,6 +704,16 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(r0[i]);
+            if (p.fp8) {
+              // e4m3 operands: this lane's feature scale times the 32 tokens' row scales
+              const float sw = p.b_scale0[(int64_t)t.group * p.N + t.n0 + q * 32 + lane];
+              const float4* a4 = reinterpret_cast<const float4*>(p.a_scale + t.m0 + c);    // the same for every lane
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float4 a = a4[i];
+                f[4 * i] *= sw * a.x; f[4 * i + 1] *= sw * a.y; f[4 * i + 2] *= sw * a.z; f[4 * i + 3] *= sw * a.w;
+              }
+            }
             if constexpr (EPI == EPI_ROWSCALE) {
               const float4* g4 = reinterpret_cast<const float4*>(p.rowscale + t.m0 + c);   // the same for every lane
 #pragma unroll
@@ -880,6 +920,19 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             f[i] = __uint_as_float(r0[i]);
             g[i] = __uint_as_float(r1[i]);
           }
+          if (p.fp8) {
+            // e4m3 operands: the sums of code products times the row's and the columns' scales
+            const float sa = m_ok ? p.a_scale[m] : 0.f;
+            const int64_t col0 = (p.group_mode == GROUP_M ? (int64_t)t.group * p.N : 0) + n;
+            const float4* s0 = reinterpret_cast<const float4*>(p.b_scale0 + col0);      // the same for every lane
+            const float4* s1 = reinterpret_cast<const float4*>(p.b_scale1 + col0);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float4 u0 = s0[i], u1 = s1[i];
+              f[4 * i] *= sa * u0.x; f[4 * i + 1] *= sa * u0.y; f[4 * i + 2] *= sa * u0.z; f[4 * i + 3] *= sa * u0.w;
+              g[4 * i] *= sa * u1.x; g[4 * i + 1] *= sa * u1.y; g[4 * i + 2] *= sa * u1.z; g[4 * i + 3] *= sa * u1.w;
+            }
+          }
           if (p.C1) {
             // the a|b copy goes first, through the whole staging area; H follows once that store has read it
             if (lane == 0) bulk_wait_read<0>();
@@ -1076,13 +1129,14 @@ inline int tc_prepare() {
 }
 
 // 2D bf16 tensor map: `inner` contiguous elements per row, `outer` rows of stride ld elements.
+// u8 = true: one-byte elements (e4m3 codes), box_inner counts bytes.
 inline int tc_make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer, uint64_t ld,
-                       uint32_t box_inner, uint32_t box_outer) {
+                       uint32_t box_inner, uint32_t box_outer, bool u8 = false) {
   cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {ld * 2};
+  cuuint64_t strides[1] = {ld * (u8 ? 1u : 2u)};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = tc_state().encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
+  CUresult r = tc_state().encode(map, u8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? REVFFN_OK : REVFFN_ERR_CUDA;
@@ -1138,7 +1192,18 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   P.tile_n = (p.concat == CONCAT_N) ? mma_n / 2 : mma_n;
   P.tiles_m = (int)ceil_div(p.M, TC_BM);
   P.tiles_n = (int)ceil_div(p.N, P.tile_n);
-  P.k_blocks = (int)ceil_div(p.K, TC_BK);
+  const bool f8 = p.fp8 != 0;
+  P.bk = f8 ? 2 * TC_BK : TC_BK;
+  P.k_blocks = (int)ceil_div(p.K, P.bk);
+  if (f8) {
+    // e4m3 operands: K-major on both sides, the SwiGLU pair (one CTA per tile) or the transposed store
+    if (p.a_mn_major || p.b_mn_major || p.concat == CONCAT_K || !p.a_scale || !p.b_scale0 ||
+        (p.concat == CONCAT_N && !p.b_scale1) || p.lda % 16 != 0 || p.ldb % 16 != 0 || p.K % 16 != 0)
+      return REVFFN_ERR_UNSUPPORTED;
+    if (!((p.epilogue == EPI_SWIGLU && p.group_mode == GROUP_M && !p.C1) ||
+          (p.epilogue == EPI_STORE && !p.out_f32 && p.group_mode == GROUP_M && p.tok_chunks)))
+      return REVFFN_ERR_UNSUPPORTED;
+  }
   P.wait_cycles = p.dbg_wait_cycles > 0 ? p.dbg_wait_cycles : TC_WAIT_CYCLES;
   P.starve = p.dbg_starve;
   if (p.dbg_starve && !p.no_pair) return REVFFN_ERR_UNSUPPORTED;      // the starved-wait test runs one CTA per tile
@@ -1146,7 +1211,9 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   // K need not be a multiple of the 64-wide K step: the tensor maps end at K, so the rest of the last
   // step is loaded as zeros (K-major rows must still start on 16-byte boundaries: lda, ldb)
   if (p.concat == CONCAT_K && (P.k_blocks & 1)) return REVFFN_ERR_SHAPE;
-  P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.a_mn_major ? 1 : 0) << 15) |
+  // fp32 accumulator; operand formats bf16 (1) for kind::f16, e4m3 (0) for kind::f8f6f4
+  const uint32_t fmt = f8 ? 0u : ((1u << 7) | (1u << 10));
+  P.idesc = (1u << 4) | fmt | ((uint32_t)(p.a_mn_major ? 1 : 0) << 15) |
             ((uint32_t)(p.b_mn_major ? 1 : 0) << 16) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 
   const int groups = p.n_groups > 0 ? p.n_groups : 1;
@@ -1154,7 +1221,7 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   // A
   if (!p.a_mn_major) {
     // [rows, K]: dense M rows, or the padded row space for GROUP_M
-    int r = tc_make_map(&ma, p.A, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.lda, 64, 128);
+    int r = tc_make_map(&ma, p.A, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.lda, f8 ? 128 : 64, 128, f8);
     if (r) return r;
   } else {
     // [K rows, lda columns]; K rows = tokens (dense) or the bound on padded rows (GROUP_K)
@@ -1165,9 +1232,9 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   const int k_half = (p.concat == CONCAT_K) ? p.K / 2 : p.K;
   if (!p.b_mn_major) {
     uint64_t rows = (p.group_mode == GROUP_M) ? (uint64_t)groups * p.N : (uint64_t)p.N;
-    int r = tc_make_map(&mb0, p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, 64, 128);
+    int r = tc_make_map(&mb0, p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, f8 ? 128 : 64, 128, f8);
     if (r) return r;
-    r = tc_make_map(&mb1, p.B1 ? p.B1 : p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, 64, 128);
+    r = tc_make_map(&mb1, p.B1 ? p.B1 : p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, f8 ? 128 : 64, 128, f8);
     if (r) return r;
   } else {
     uint64_t rows = (p.group_mode == GROUP_M) ? (uint64_t)groups * k_half : (uint64_t)p.K;
@@ -1226,6 +1293,7 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
                   p.concat != CONCAT_N && !p.no_pair && s.n_sms % 2 == 0 &&
                   (p.epilogue == EPI_ROWSCALE || (p.epilogue == EPI_STORE && !p.out_f32));
   const bool pair = tr || (p.group_mode != GROUP_M && (p.N % 256 == 0 || p.b_mn_major) && !p.no_pair);
+  if (f8 && p.epilogue == EPI_STORE && !tr) return REVFFN_ERR_UNSUPPORTED;      // only the transposed store scales its accumulator
   P.tr = tr ? 1 : 0;
   P.tiles_f = p.N / 256;
   int64_t total = (int64_t)P.tiles_m * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);
@@ -1233,7 +1301,7 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   if (tr) {
     // the number of token chunks is only known on the device: a full persistent grid
     grid = s.n_sms;
-    P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.b_mn_major ? 1 : 0) << 15) |
+    P.idesc = (1u << 4) | fmt | ((uint32_t)(p.b_mn_major ? 1 : 0) << 15) |
               ((uint32_t)(p.a_mn_major ? 1 : 0) << 16) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(2 * TC_BM >> 4) << 24);
   } else if (pair) {
     total = (int64_t)((P.tiles_m + 1) / 2) * P.tiles_n * (p.group_mode == GROUP_K ? groups : 1);

@@ -16,6 +16,7 @@
 #include "backward_ew.cuh"
 #include "gemm.cuh"
 #include "gemm_tcgen05.cuh"
+#include "fp8.cuh"
 
 namespace revffn {
 
@@ -88,7 +89,7 @@ constexpr int GUARD_BYTES = 256;
 struct WsLayout {
   // forward / inverse
   Buf status, rows_total, w_rc, w_rc_part, n, r, idx, gates, sgate, prob, local_rank, chunk_cnt, chunk_base, expert_cnt,
-      expert_off, tile_group, tok_chunks, tok_row, row_tok, row_gate, u, up, hmid, o, hs, s, z;
+      expert_off, tile_group, tok_chunks, tok_row, row_tok, row_gate, u, up, hmid, o, hs, s, z, upq, up_scale, hq, h_scale;
   int max_chunks = 0;
   size_t fwd_bytes = 0;
   size_t saved_bytes = 0;   // fwd region + SwiGLU pre-activations: what a saved evaluation consists of
@@ -155,6 +156,12 @@ static WsLayout plan_workspace(const revffn_moe_desc& D) {
   take(L.hs, (size_t)T * Is * ts);
   take(L.s, (size_t)T * d * ts);
   take(L.z, (size_t)T * d * ts);
+  // REVFFN_FLAG_FP8_EXPERTS: e4m3 copies of the permuted u rows and of g*H with their row scales
+  const bool fp8 = (D.flags & REVFFN_FLAG_FP8_EXPERTS) != 0;
+  take(L.upq, fp8 ? (size_t)Rp * d : 0);
+  take(L.up_scale, fp8 ? (size_t)Rp * 4 : 0);
+  take(L.hq, fp8 ? (size_t)Rp * I : 0);
+  take(L.h_scale, fp8 ? (size_t)Rp * 4 : 0);
   L.fwd_bytes = off;
   take(L.ab, (size_t)Rp * 2 * I * ts);
   take(L.abs, (size_t)T * 2 * Is * ts);
@@ -193,6 +200,11 @@ static int validate_desc(const revffn_moe_desc* D) {
   if (h % mult || D->d_model % mult || D->d_expert % mult || D->d_shared % mult) return REVFFN_ERR_SHAPE;
   if (D->ld_stream < h || (D->ld_stream % 4)) return REVFFN_ERR_ALIGN;
   if ((int64_t)D->tokens * D->top_k > (int64_t)1 << 28) return REVFFN_ERR_SHAPE;
+  if (D->flags & REVFFN_FLAG_FP8_EXPERTS) {
+    if (D->weight_dtype != REVFFN_BF16 || (D->flags & (REVFFN_FLAG_FORCE_SIMT | REVFFN_FLAG_SAVE_ACTIVATIONS | REVFFN_FLAG_REUSE_ACTIVATIONS)) ||
+        D->d_model > 2048 || D->d_expert > 2048 || D->d_model % 256 != 0)
+      return REVFFN_ERR_UNSUPPORTED;
+  }
   return REVFFN_OK;
 }
 
@@ -217,6 +229,13 @@ static int validate_weights(const revffn_moe_desc& D, const revffn_moe_weights* 
   if (!w) return REVFFN_ERR_NULL;
   if (!w->w_up || !w->w_down || !w->w_router || !w->w_gate || !w->w_upx || !w->w_downx) return REVFFN_ERR_NULL;
   if (D.d_shared > 0 && (!w->ws_gate || !w->ws_up || !w->ws_down || !w->ws_sgate)) return REVFFN_ERR_NULL;
+  if ((D.flags & REVFFN_FLAG_FP8_EXPERTS) && (!w->q_gate || !w->q_upx || !w->q_downx || !w->s_gate || !w->s_upx || !w->s_downx))
+    return REVFFN_ERR_NULL;
+  {
+    const void* qs[] = {w->q_gate, w->q_upx, w->q_downx, w->s_gate, w->s_upx, w->s_downx};
+    for (const void* q : qs)
+      if (q && !aligned16(q)) return REVFFN_ERR_ALIGN;
+  }
   const void* ps[] = {w->norm_gamma, w->w_up, w->w_down, w->w_router, w->b_router, w->w_gate, w->w_upx,
                       w->w_downx, w->ws_gate, w->ws_up, w->ws_down, w->ws_sgate};
   for (const void* p : ps)
@@ -412,43 +431,88 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     CKR(run_gemm(c, p, TG_PUP));
   }
 
-  // Permute: Up[row] = U[token(row)]
-  { ProfScope ps(TG_GATHER, st);
-  gather_rows_kernel<T><<<(unsigned)L.rows_pad, 256, 0, st>>>(c.template p<T>(L.u), d, c.template p<int32_t>(L.row_tok),
-                                                              c.template p<int32_t>(L.rows_total), d,
-                                                              c.template p<T>(L.up));
+  const bool fp8 = (D.flags & REVFFN_FLAG_FP8_EXPERTS) != 0;
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (fp8) {
+      // Routed experts on e4m3 operands: the permutation quantises the u rows as it gathers them, the first
+      // product's epilogue applies the scales before the SwiGLU, g*H is quantised row by row, and the down
+      // projection (tokens on the MMA N side) applies its scales before it stores.
+      { ProfScope ps(TG_GATHER, st);
+      CK(launch_quantize_rows(c.template p<bf16>(L.u), d, c.template p<int32_t>(L.row_tok), c.template p<int32_t>(L.rows_total),
+                              L.rows_pad, d, c.template p<uint8_t>(L.upq), c.template p<float>(L.up_scale), st));
+      }
+      {
+        GemmProblem p = blank_problem();
+        p.M = (int)L.rows_pad; p.N = I; p.K = d;
+        p.fp8 = 1; p.A = c.template p<uint8_t>(L.upq); p.lda = d; p.a_scale = c.template p<float>(L.up_scale);
+        p.B0 = c.W.q_gate; p.B1 = c.W.q_upx; p.ldb = d; p.concat = CONCAT_N;
+        p.b_scale0 = c.W.s_gate; p.b_scale1 = c.W.s_upx;
+        p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)I * d;
+        p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
+        p.rows_total = c.template p<int32_t>(L.rows_total);
+        p.epilogue = EPI_SWIGLU; p.C = c.template p<T>(L.hmid); p.ldc = I;
+        p.rowscale = c.template p<float>(L.row_gate);
+        CKR(run_gemm(c, p, TG_EXP_GATEUP));
+      }
+      { ProfScope ps(TG_GATHER, st);
+      CK(launch_quantize_rows(c.template p<bf16>(L.hmid), I, nullptr, c.template p<int32_t>(L.rows_total), L.rows_pad, I,
+                              c.template p<uint8_t>(L.hq), c.template p<float>(L.h_scale), st));
+      }
+      {
+        GemmProblem p = blank_problem();
+        p.M = (int)L.rows_pad; p.N = d; p.K = I;
+        p.fp8 = 1; p.A = c.template p<uint8_t>(L.hq); p.lda = I; p.a_scale = c.template p<float>(L.h_scale);
+        p.B0 = c.W.q_downx; p.ldb = I; p.b_scale0 = c.W.s_downx;
+        p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)d * I;
+        p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
+        p.rows_total = c.template p<int32_t>(L.rows_total);
+        p.tok_chunks = c.template p<int4>(L.tok_chunks);
+        p.epilogue = EPI_STORE;
+        p.C = c.template p<T>(L.o); p.ldc = d;
+        CKR(run_gemm(c, p, TG_EXP_DOWN));
+      }
+    }
   }
-  CK(cudaGetLastError());
-
-  // Routed experts: H' = g * silu(Up Wg^T) * (Up Wu^T);  O = H' Wd^T.  The row's gate weight g goes onto H in
-  // the first product's epilogue: the second then needs no scaling, and the backward pass finds in H' exactly the
-  // operand its down-projection weight gradient takes (dW_d = dO^T (g H)).
-  {
-    GemmProblem p = blank_problem();
-    p.M = (int)L.rows_pad; p.N = I; p.K = d;
-    p.A = c.template p<T>(L.up); p.lda = d;
-    p.B0 = c.W.w_gate; p.B1 = c.W.w_upx; p.ldb = d; p.concat = CONCAT_N;
-    p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)I * d;
-    p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
-    p.rows_total = c.template p<int32_t>(L.rows_total);
-    p.epilogue = EPI_SWIGLU; p.C = c.template p<T>(L.hmid); p.ldc = I;
-    p.rowscale = c.template p<float>(L.row_gate);
-    if (save_ab) { p.C1 = c.template p<T>(L.ab); p.ldc1 = 2 * (int64_t)I; }
-    CKR(run_gemm(c, p, TG_EXP_GATEUP));
-  }
-  {
-    GemmProblem p = blank_problem();
-    p.M = (int)L.rows_pad; p.N = d; p.K = I;
-    p.A = c.template p<T>(L.hmid); p.lda = I;
-    p.B0 = c.W.w_downx; p.ldb = I;
-    p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)d * I;
-    p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
-    p.rows_total = c.template p<int32_t>(L.rows_total);
-    p.tok_chunks = c.template p<int4>(L.tok_chunks);
-    p.epilogue = EPI_STORE;
-    p.C = c.template p<T>(L.o); p.ldc = d;
-    CKR(run_gemm(c, p, TG_EXP_DOWN));
-  }
+  if (!fp8) {
+    // Permute: Up[row] = U[token(row)]
+    { ProfScope ps(TG_GATHER, st);
+    gather_rows_kernel<T><<<(unsigned)L.rows_pad, 256, 0, st>>>(c.template p<T>(L.u), d, c.template p<int32_t>(L.row_tok),
+                                                                c.template p<int32_t>(L.rows_total), d,
+                                                                c.template p<T>(L.up));
+    }
+    CK(cudaGetLastError());
+  
+    // Routed experts: H' = g * silu(Up Wg^T) * (Up Wu^T);  O = H' Wd^T.  The row's gate weight g goes onto H in
+    // the first product's epilogue: the second then needs no scaling, and the backward pass finds in H' exactly the
+    // operand its down-projection weight gradient takes (dW_d = dO^T (g H)).
+    {
+      GemmProblem p = blank_problem();
+      p.M = (int)L.rows_pad; p.N = I; p.K = d;
+      p.A = c.template p<T>(L.up); p.lda = d;
+      p.B0 = c.W.w_gate; p.B1 = c.W.w_upx; p.ldb = d; p.concat = CONCAT_N;
+      p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)I * d;
+      p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
+      p.rows_total = c.template p<int32_t>(L.rows_total);
+      p.epilogue = EPI_SWIGLU; p.C = c.template p<T>(L.hmid); p.ldc = I;
+      p.rowscale = c.template p<float>(L.row_gate);
+      if (save_ab) { p.C1 = c.template p<T>(L.ab); p.ldc1 = 2 * (int64_t)I; }
+      CKR(run_gemm(c, p, TG_EXP_GATEUP));
+    }
+    {
+      GemmProblem p = blank_problem();
+      p.M = (int)L.rows_pad; p.N = d; p.K = I;
+      p.A = c.template p<T>(L.hmid); p.lda = I;
+      p.B0 = c.W.w_downx; p.ldb = I;
+      p.group_mode = GROUP_M; p.n_groups = E; p.b_group_stride = (int64_t)d * I;
+      p.group_off = c.template p<int32_t>(L.expert_off); p.tile_group = c.template p<int32_t>(L.tile_group);
+      p.rows_total = c.template p<int32_t>(L.rows_total);
+      p.tok_chunks = c.template p<int4>(L.tok_chunks);
+      p.epilogue = EPI_STORE;
+      p.C = c.template p<T>(L.o); p.ldc = d;
+      CKR(run_gemm(c, p, TG_EXP_DOWN));
+    }
+  
+}
 
   // Shared expert: S = (silu(U Wsg^T) * (U Wsu^T)) Wsd^T
   if (Is > 0) {
@@ -803,6 +867,7 @@ static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weight
   CKR(validate_weights(*desc, w));
   if (!ws) return REVFFN_ERR_NULL;
   if (pass == PASS_BWD && !grads) return REVFFN_ERR_NULL;
+  if (pass == PASS_BWD && (desc->flags & REVFFN_FLAG_FP8_EXPERTS)) return REVFFN_ERR_UNSUPPORTED;      // gradients are taken on the bf16 path
   if (desc->tokens > 0 && (!y1 || !in2 || !out)) return REVFFN_ERR_NULL;
   if (!aligned16(y1) || !aligned16(in2) || !aligned16(out) || (reinterpret_cast<uintptr_t>(ws) & 255u))
     return REVFFN_ERR_ALIGN;
@@ -912,6 +977,30 @@ int revffn_moe_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weight
                             const int32_t* topk_idx_in, void* ws, size_t ws_bytes, void* cuda_stream) {
   if (!sgd) return REVFFN_ERR_NULL;
   return entry(PASS_BWD, desc, w, y1, dy2, dy1_inout, grads, topk_idx_in, nullptr, ws, ws_bytes, cuda_stream, sgd);
+}
+
+int revffn_moe_quantize_experts(const revffn_moe_desc* desc, const revffn_moe_weights* w, void* cuda_stream) {
+  int r = validate_desc(desc);
+  if (r != REVFFN_OK) return r;
+  if (!w || !w->w_gate || !w->w_upx || !w->w_downx || !w->q_gate || !w->q_upx || !w->q_downx || !w->s_gate || !w->s_upx || !w->s_downx)
+    return REVFFN_ERR_NULL;
+  if (desc->weight_dtype != REVFFN_BF16 || desc->d_model > 2048 || desc->d_expert > 2048) return REVFFN_ERR_UNSUPPORTED;
+  const void* ps[] = {w->w_gate, w->w_upx, w->w_downx, w->q_gate, w->q_upx, w->q_downx, w->s_gate, w->s_upx, w->s_downx};
+  for (const void* p : ps)
+    if (!aligned16(p)) return REVFFN_ERR_ALIGN;
+  r = check_device();
+  if (r != REVFFN_OK) return r;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const int64_t E = desc->n_experts, I = desc->d_expert, d = desc->d_model;
+  auto q = [&](const void* in, int64_t rows, int width, const void* out, const float* scale) {
+    return launch_quantize_rows(reinterpret_cast<const bf16*>(in), width, nullptr, nullptr, rows, width,
+                                reinterpret_cast<uint8_t*>(const_cast<void*>(out)), const_cast<float*>(scale), st);
+  };
+  CK(q(w->w_gate, E * I, (int)d, w->q_gate, w->s_gate));
+  CK(q(w->w_upx, E * I, (int)d, w->q_upx, w->s_upx));
+  CK(q(w->w_downx, E * d, (int)I, w->q_downx, w->s_downx));
+  g_prof.launches += 3;
+  return REVFFN_OK;
 }
 
 int revffn_moe_status(const void* ws, void* cuda_stream, int32_t* device_status) {
