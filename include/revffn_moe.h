@@ -281,7 +281,8 @@ int revffn_moe_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weight
 /*
  * Quantise the bf16 expert weights for REVFFN_FLAG_FP8_EXPERTS: per output row r of w_gate / w_upx ([E*I] rows of
  * d) and of w_downx ([E*d] rows of I), scale[r] = max|row| / 448 (1 for an all-zero row) and
- * code = e4m3(w / scale[r]), round to nearest even, saturating.  Writes the six q_* / s_* buffers named in `w`
+ * code = e4m3(w * (1 / scale[r])), every step a correctly rounded fp32 operation, round to nearest even,
+ * saturating.  Writes the six q_* / s_* buffers named in `w`
  * (caller-owned device memory of the sizes given at revffn_moe_weights, 16-byte aligned); call again whenever
  * the bf16 weights change.  Needs d and I to be multiples of 128 and at most 2048.  Enqueued on the stream.
  */

@@ -151,12 +151,14 @@ def e4m3_round(v: np.ndarray) -> np.ndarray:
 
 
 def quantize_rows_e4m3(x: np.ndarray):
-    """Per row: scale = max|x| / 448 (1 for an all-zero row), codes = e4m3_round(x / scale), all in fp32.
-    Returns (dequantised codes as fp32 [rows, cols] -- the values the product sums --, scale [rows])."""
+    """Per row: scale = max|x| / 448 (1 for an all-zero row), codes = e4m3_round(x * (1 / scale)), every
+    operation a correctly rounded fp32 one (the kernels multiply by the row's reciprocal).
+    Returns (the codes' values as fp32 [rows, cols] -- what the product sums --, scale [rows])."""
     x = np.asarray(x, dtype=np.float32)
     amax = np.max(np.abs(x), axis=-1)
     scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
-    q = e4m3_round((x / scale[..., None]).astype(np.float32))
+    inv = (np.float32(1.0) / scale).astype(np.float32)
+    q = e4m3_round((x * inv[..., None]).astype(np.float32))
     return q, scale
 
 

@@ -503,7 +503,7 @@ def test_fp8_experts_is_the_branch_with_quantised_expert_operands():
     def q8(t):      # per-row e4m3 through torch, dequantised
         amax = t.abs().amax(dim=-1, keepdim=True)
         sc = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
-        return (t / sc).to(torch.float8_e4m3fn).to(torch.float32).double() * sc.double()
+        return (t * (1.0 / sc)).to(torch.float8_e4m3fn).to(torch.float32).double() * sc.double()
 
     n, _ = orc.norm_fwd(s["y1"], p["norm_gamma"], cfg.norm_eps)
     u = n @ p["w_up"].astype(np.float64).T
