@@ -1,6 +1,6 @@
 """FP8 (e4m3) routed experts, forward and inverse, against the oracle evaluated with the same quantisation.
 
-Both sides round the same fp32 quotient to e4m3 (the decision is taken in the kernels' precision), and for the
+Both sides round the same fp32 value x * (1 / scale) to e4m3 (the decision is taken in the kernels' precision), and for the
 weights, whose bytes are identical on both sides, codes and scales must equal the oracle's quantiser bit for bit.
 The activations are not identical on both sides: the kernels' u comes from a bf16-rounded n and an fp32
 accumulation, the oracle's from fp64, so about 2^-9 of relative difference reaches the quantiser, and a value
