@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <algorithm>
 #include <cuda_bf16.h>
 #include <stdint.h>
 
@@ -67,6 +68,18 @@ __device__ __forceinline__ void set_status(int* status, int code) {
 }
 
 // 8 elements of T as one vector: loads/stores of 16 bytes for bf16, 2x16 for float.
+// Blocks of `kernel` that are resident on the current device at once (one wave) for this block size and dynamic
+// shared memory: the grid size of the grid-stride kernels.
+template <typename Kernel>
+inline cudaError_t resident_blocks(Kernel kernel, int threads, size_t smem, int* blocks) {
+  int dev = 0, sms = 0, per_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
+  *blocks = (e == cudaSuccess) ? std::max(1, sms * per_sm) : 0;
+  return e;
+}
+
 template <typename T> struct Vec8;
 template <> struct Vec8<bf16> {
   uint4 raw;

@@ -534,9 +534,9 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
   // Combine: Z[t] = sum_s O[row(t,s)] + sgate_t S[t]
   if (Tn > 0) {
     { ProfScope ps(TG_COMBINE, st);
-    combine_rows_kernel<T><<<Tn, 256, 0, st>>>(c.template p<T>(L.o), c.template p<int32_t>(L.tok_row), k,
-                                               Is > 0 ? c.template p<T>(L.s) : nullptr, c.template p<float>(L.sgate),
-                                               d, c.template p<T>(L.z));
+    CK(launch_combine_rows<T>(c.template p<T>(L.o), c.template p<int32_t>(L.tok_row), k,
+                              Is > 0 ? c.template p<T>(L.s) : nullptr, c.template p<float>(L.sgate), d, Tn,
+                              c.template p<T>(L.z), st));
     }
     CK(cudaGetLastError());
   }
@@ -789,12 +789,11 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
 
   // dU, then P_up backward and the norm
   { ProfScope ps(TG_DU_REDUCE, st);
-  du_reduce_kernel<T><<<Tn, 256, 0, st>>>(c.template p<T>(L.dup), c.template p<int32_t>(L.tok_row),
-                                          c.template p<int32_t>(L.idx), c.template p<float>(L.tok_dl), k,
-                                          Is > 0 ? c.template p<T>(L.dush) : nullptr,
-                                          reinterpret_cast<const T*>(c.W.w_router), c.template p<float>(L.dl),
-                                          reinterpret_cast<const T*>(c.W.ws_sgate),
-                                          dense_gate ? c.template p<T>(L.dur) : nullptr, d, c.template p<T>(L.du));
+  CK(launch_du_reduce<T>(c.template p<T>(L.dup), c.template p<int32_t>(L.tok_row), c.template p<int32_t>(L.idx),
+                         c.template p<float>(L.tok_dl), k, Is > 0 ? c.template p<T>(L.dush) : nullptr,
+                         reinterpret_cast<const T*>(c.W.w_router), E, c.template p<float>(L.dl),
+                         reinterpret_cast<const T*>(c.W.ws_sgate), dense_gate ? c.template p<T>(L.dur) : nullptr, d,
+                         Tn, c.template p<T>(L.du), st));
   }
   CK(cudaGetLastError());
   {

@@ -668,37 +668,68 @@ __global__ void gather_rows_kernel(const T* __restrict__ src, int64_t ld_src, co
 // ---------------------------------------------------------------------------
 // Combine: Z[t, :] = sum_{s<k} O[tok_row[t,s], :] + sgate[t] * S[t, :]
 // fp32 sums in slot order (fixed, so forward and inverse agree bit for bit).
-// `extra` (optional) adds more per-token terms: used by the backward pass.
+// One warp per token, eight tokens per block; each lane walks the row in 256-element strides with all k + 1
+// row pieces of a stride requested before the first is used (K = k at compile time; K = 0 takes k <= 8 at run
+// time and pays for eight slots).  Many short blocks: a one-wave grid striding over the tokens measured 12 %
+// slower.
 // ---------------------------------------------------------------------------
-template <typename T>
-__global__ void combine_rows_kernel(const T* __restrict__ O, const int32_t* __restrict__ tok_row, int k,
-                                    const T* __restrict__ S, const float* __restrict__ sgate, int width,
-                                    T* __restrict__ Z) {
-  int t = blockIdx.x;
-  int rows[8];
-  for (int s = 0; s < k; ++s) rows[s] = tok_row[(int64_t)t * k + s];
-  float sg = S ? sgate[t] : 0.f;
-  for (int c = threadIdx.x * 8; c < width; c += blockDim.x * 8) {
+constexpr int COMBINE_TOKENS = 8;      // tokens (warps) per block
+
+template <typename T, int K>
+__global__ void __launch_bounds__(32 * COMBINE_TOKENS)
+combine_rows_kernel(const T* __restrict__ O, const int32_t* __restrict__ tok_row, int k_rt,
+                    const T* __restrict__ S, const float* __restrict__ sgate, int width, int tokens,
+                    T* __restrict__ Z) {
+  constexpr int KS = K ? K : 8;
+  const int k = K ? K : k_rt;
+  const int lane = threadIdx.x & 31;
+  const int64_t t = (int64_t)blockIdx.x * COMBINE_TOKENS + (threadIdx.x >> 5);
+  if (t >= tokens) return;
+  const T* rows[KS];
+#pragma unroll
+  for (int s = 0; s < KS; ++s) {
+    const int r = s < k ? tok_row[t * k + s] : -1;      // -1: entry with an out-of-range expert index
+    rows[s] = r >= 0 ? O + (int64_t)r * width : nullptr;
+  }
+  const float sg = S ? sgate[t] : 0.f;
+  const T* srow = S ? S + t * width : nullptr;
+  T* zrow = Z + t * width;
+  for (int c = lane * 8; c < width; c += 256) {
+    Vec8<T> v[KS], vs;
+#pragma unroll
+    for (int s = 0; s < KS; ++s) {
+      if (rows[s]) v[s].load(rows[s] + c); else v[s].zero();
+    }
+    if (srow) vs.load(srow + c); else vs.zero();
     float acc[8], f[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-    Vec8<T> v;
-    for (int s = 0; s < k; ++s) {
-      if (rows[s] < 0) continue;      // entry with an out-of-range expert index
-      v.load(O + (int64_t)rows[s] * width + c);
-      v.get(f);
+#pragma unroll
+    for (int s = 0; s < KS; ++s) {
+      v[s].get(f);
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[i] += f[i];
     }
-    if (S) {
-      v.load(S + (int64_t)t * width + c);
-      v.get(f);
+    vs.get(f);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] += sg * f[i];
-    }
-    v.set(acc);
-    v.store(Z + (int64_t)t * width + c);
+    for (int i = 0; i < 8; ++i) acc[i] += sg * f[i];
+    vs.set(acc);
+    vs.store(zrow + c);
   }
+}
+
+template <typename T>
+inline cudaError_t launch_combine_rows(const T* O, const int32_t* tok_row, int k, const T* S, const float* sgate,
+                                       int width, int tokens, T* Z, cudaStream_t st) {
+  if (tokens <= 0) return cudaSuccess;
+  const int blocks = (int)ceil_div(tokens, COMBINE_TOKENS), th = 32 * COMBINE_TOKENS;
+  switch (k) {
+    case 1: combine_rows_kernel<T, 1><<<blocks, th, 0, st>>>(O, tok_row, k, S, sgate, width, tokens, Z); break;
+    case 2: combine_rows_kernel<T, 2><<<blocks, th, 0, st>>>(O, tok_row, k, S, sgate, width, tokens, Z); break;
+    case 4: combine_rows_kernel<T, 4><<<blocks, th, 0, st>>>(O, tok_row, k, S, sgate, width, tokens, Z); break;
+    default: combine_rows_kernel<T, 0><<<blocks, th, 0, st>>>(O, tok_row, k, S, sgate, width, tokens, Z); break;
+  }
+  return cudaGetLastError();
 }
 
 }  // namespace revffn
