@@ -392,16 +392,17 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
     ms_prof_step = ms_prof_total / args.steps
     value = job_tokens_per_s(world, cfg.tokens, args.steps, ms_total)
 
-    e2e_value, dt, bytes_dir = None, 0.0, 0
+    e2e_value, e2e_sync_value, dt, dt_sync, bytes_dir = None, None, 0.0, 0.0, 0
     if e2e:
         # end to end: host-resident streams, H2D and D2H copies inside the timed region
         pin = lambda a: torch.from_numpy(a).pin_memory()
         hy1, hx2, hdy2 = pin(s_host["y1"]), pin(s_host["x2"]), pin(s_host["dy2"])
         hy2, hx2r, hdy1 = (torch.empty_like(hy1).pin_memory() for _ in range(3))
         slot = ((hy1.numel() * 4 + 255) // 256) * 256
-        staging = torch.empty(6 * slot, dtype=torch.uint8, device="cuda")
+        staging = torch.empty(12 * slot, dtype=torch.uint8, device="cuda")
         g_struct = blk.grads_struct(grads)
         copy_stream = torch.cuda.Stream()
+        # (1) one step at a time: the host waits for a step's results before it starts the next one
         host_step = lambda: rv.revffn_moe_step_host(blk.desc, blk.w, g_struct, hy1, hx2, hdy2, hy2, hx2r, hdy1, staging,
                                                     blk.ws, copy_stream=copy_stream.cuda_stream)
         for _ in range(2):
@@ -411,9 +412,33 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
         for _ in range(args.steps):
             host_step()
             torch.cuda.synchronize()     # the step's results are read on the host
+        dt_sync = time.perf_counter() - t0
+        dt_sync = max_over_ranks([dt_sync], world)[0]
+        # (2) a loop of steps, pipelined: every step still uploads its inputs from pinned host memory and
+        # downloads its results, and the host waits for the results of step i - 1 while step i runs; the
+        # transfers of neighbouring steps run beside the passes (two staging sets, two sets of host outputs)
+        outs = [(hy2, hx2r, hdy1), tuple(torch.empty_like(hy1).pin_memory() for _ in range(3))]
+        def piped(n_steps):
+            prev = None
+            for i in range(n_steps):
+                o = outs[i & 1]
+                rv.revffn_moe_step_host(blk.desc, blk.w, g_struct, hy1, hx2, hdy2, o[0], o[1], o[2], staging, blk.ws,
+                                        copy_stream=copy_stream.cuda_stream, pipelined=True)
+                ev = torch.cuda.Event()
+                ev.record(copy_stream)
+                if prev is not None:
+                    prev.synchronize()   # the previous step's results are on the host
+                prev = ev
+            prev.synchronize()
+            torch.cuda.synchronize()
+        piped(3)
+        barrier()
+        t0 = time.perf_counter()
+        piped(args.steps)
         dt = time.perf_counter() - t0
         dt = max_over_ranks([dt], world)[0]
         e2e_value = job_tokens_per_s(world, cfg.tokens, args.steps, dt * 1e3)
+        e2e_sync_value = job_tokens_per_s(world, cfg.tokens, args.steps, dt_sync * 1e3)
         bytes_dir = 3 * hy1.numel() * 4
 
     if rank != 0:
@@ -541,7 +566,13 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
         "roofline": roofline,
         "cpu_baseline": cpu_rec,
         "e2e": ({"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": bytes_dir,
-                 "d2h_bytes_per_step": bytes_dir, "ms_per_step": 1e3 * dt / args.steps} if e2e else None),
+                 "d2h_bytes_per_step": bytes_dir, "ms_per_step": 1e3 * dt / args.steps,
+                 "mode": "loop of revffn_moe_step_host calls in the pipelined form: each step uploads its three "
+                         "input streams from pinned host memory and downloads its three result streams; the host "
+                         "waits for the results of step i-1 while step i runs",
+                 "one_step_at_a_time": {"value": e2e_sync_value, "ms_per_step": 1e3 * dt_sync / args.steps,
+                                        "note": "host synchronises after every step before starting the next"}}
+                if e2e else None),
         "gpu_launches": int(launches),
         "clocks": clocks,
         "clocks_per_kernel_pass": clocks_prof,

@@ -138,6 +138,9 @@ enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                
  * branches.  Not with REVFFN_FLAG_FORCE_SIMT, SAVE/REUSE_ACTIVATIONS or in revffn_moe_backward
  * (REVFFN_ERR_UNSUPPORTED): gradients are taken on the bf16 path. */
 #define REVFFN_FLAG_FP8_EXPERTS 256u
+/* revffn_moe_step_host only: the pipelined form described there (two staging sets used in turn, results
+ * complete when the copy stream completes).  Other entry points ignore it. */
+#define REVFFN_FLAG_STEP_PIPELINED 512u
 
 /*
  * Block descriptor.  Shape constraints (else REVFFN_ERR_SHAPE):
@@ -364,6 +367,16 @@ int revffn_moe_saved_size(const revffn_moe_desc* desc, size_t* bytes);
  * y2 out during the inverse pass, the reconstructed x2 out during backward).  The call
  * orders the two streams with events (seven per device, created on its first use); when it
  * returns, work queued on cuda_stream afterwards follows everything of this step.
+ *
+ * REVFFN_FLAG_STEP_PIPELINED (needs copy_stream and staging of 12 slots, else REVFFN_ERR_UNSUPPORTED /
+ * REVFFN_ERR_WORKSPACE): for a loop of steps.  Consecutive calls on a device use the two halves of `staging` in
+ * turn; the inputs go up on a stream the library creates on first use, the results come down on copy_stream,
+ * and cuda_stream does NOT wait for the downloads.  The uploads of a call therefore run while the passes of
+ * the previous call are still computing, and its downloads while the next call computes: in a loop the
+ * transfers disappear behind the passes.  The contract changes accordingly: the host outputs of a call are
+ * complete when copy_stream has completed the work this call queued on it (record an event there after the
+ * call); the host inputs may be overwritten from then on too; the results are the same bits as in the plain
+ * form.  The workspace is shared by consecutive calls and is used in stream order.
  * (Convenience for end-to-end use; no paper counterpart.)
  */
 int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* w, const revffn_moe_grads* grads,

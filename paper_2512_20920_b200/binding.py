@@ -24,6 +24,7 @@ FLAG_KEEP_STATUS = 32
 FLAG_DEBUG_CHECKS = 64
 FLAG_ROUTER_FOLDED = 128
 FLAG_FP8_EXPERTS = 256
+FLAG_STEP_PIPELINED = 512
 
 ERR_DEVICE_WAIT, ERR_UNSUPPORTED, ERR_NOALLOC_LIMIT, ERR_INDEX, ERR_CANARY, ERR_NONFINITE = -7, -8, -9, -10, -11, -12
 
@@ -250,9 +251,16 @@ def revffn_moe_status(ws, stream: Optional[int] = None) -> int:
 
 
 def revffn_moe_step_host(desc: Desc, w: Weights, grads: Grads, y1_host, x2_host, dy2_host, y2_host, x2_rec_host,
-                         dy1_host, staging, ws, stream: Optional[int] = None, copy_stream: Optional[int] = None):
+                         dy1_host, staging, ws, stream: Optional[int] = None, copy_stream: Optional[int] = None,
+                         pipelined: bool = False):
     """Host-resident streams (pinned CPU tensors) in and out; see the header.  copy_stream: raw handle of a
-    second CUDA stream for the transfers that can run beside the passes, or None."""
+    second CUDA stream for the transfers that can run beside the passes, or None.  pipelined: the call is made
+    with FLAG_STEP_PIPELINED (12 staging slots, results complete when copy_stream completes)."""
+    if pipelined:
+        d2 = Desc()
+        C.memmove(C.byref(d2), C.byref(desc), C.sizeof(Desc))
+        d2.flags |= FLAG_STEP_PIPELINED
+        desc = d2
     _check(lib.revffn_moe_step_host(C.byref(desc), C.byref(w), C.byref(grads), _ptr(y1_host), _ptr(x2_host),
                                     _ptr(dy2_host), _ptr(y2_host), _ptr(x2_rec_host), _ptr(dy1_host), _ptr(staging),
                                     staging.numel() * staging.element_size(), _ptr(ws),

@@ -1061,22 +1061,86 @@ int revffn_moe_ws_lookup(const revffn_moe_desc* desc, const char* name, size_t* 
   return REVFFN_ERR_UNSUPPORTED;
 }
 
-// Events that order the copy stream against the compute stream in revffn_moe_step_host
-// (created on first use, per device; no timing).
-static cudaEvent_t* step_events(int* err) {
-  static cudaEvent_t ev[64][7];
-  static bool made[64] = {false};
+// Events that order the copy streams against the compute stream in revffn_moe_step_host, the upload stream
+// of the pipelined form and its call counter (created on first use, per device; no timing).
+struct StepState {
+  cudaEvent_t ev[10];            // 0..6 plain form; pipelined form: 0 inputs A, 1 inputs B, 2..4 passes done, 8/9 set free
+  cudaStream_t upload = nullptr; // pipelined form: host -> device copies
+  unsigned calls = 0;            // pipelined form: parity selects the staging set
+  bool made = false;
+};
+
+static StepState* step_state(int* err) {
+  static StepState state[64];
   static std::mutex mu;
   std::lock_guard<std::mutex> lock(mu);
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = REVFFN_ERR_CUDA; return nullptr; }
-  if (!made[dev]) {
-    for (int i = 0; i < 7; ++i)
-      if (cudaEventCreateWithFlags(&ev[dev][i], cudaEventDisableTiming) != cudaSuccess) { *err = REVFFN_ERR_CUDA; return nullptr; }
-    made[dev] = true;
+  StepState& s = state[dev];
+  if (!s.made) {
+    for (int i = 0; i < 10; ++i)
+      if (cudaEventCreateWithFlags(&s.ev[i], cudaEventDisableTiming) != cudaSuccess) { *err = REVFFN_ERR_CUDA; return nullptr; }
+    if (cudaStreamCreateWithFlags(&s.upload, cudaStreamNonBlocking) != cudaSuccess) { *err = REVFFN_ERR_CUDA; return nullptr; }
+    s.made = true;
   }
   *err = REVFFN_OK;
-  return ev[dev];
+  return &s;
+}
+
+// The pipelined form of revffn_moe_step_host (REVFFN_FLAG_STEP_PIPELINED): two sets of staging slots used in
+// turn, uploads on a stream of the library's own, downloads on the caller's copy stream, and no join of the
+// copy stream into the compute stream, so that the uploads of one call run beside the passes of the call before
+// it and its downloads beside the passes of the call after it.
+static int step_host_pipelined(const revffn_moe_desc* desc, const revffn_moe_weights* w, const revffn_moe_grads* grads,
+                               const float* y1_host, const float* x2_host, const float* dy2_host, float* y2_host,
+                               float* x2_rec_host, float* dy1_host, char* staging, size_t slot, size_t n, void* ws,
+                               size_t ws_bytes, cudaStream_t st, cudaStream_t cs) {
+  int r = REVFFN_OK;
+  StepState* S = step_state(&r);
+  if (r != REVFFN_OK) return r;
+  const unsigned set = S->calls++ & 1u;
+  cudaStream_t up = S->upload;
+  cudaEvent_t ev_free = S->ev[8 + set];
+  char* sp = staging + (size_t)set * 6 * slot;
+  float* y1 = reinterpret_cast<float*>(sp);
+  float* x2 = reinterpret_cast<float*>(sp + slot);
+  float* dy2 = reinterpret_cast<float*>(sp + 2 * slot);
+  float* y2 = reinterpret_cast<float*>(sp + 3 * slot);
+  float* x2r = reinterpret_cast<float*>(sp + 4 * slot);
+  float* dy1 = reinterpret_cast<float*>(sp + 5 * slot);
+  revffn_moe_desc d_fwd = *desc, d_inv = *desc, d_bwd = *desc;
+  d_fwd.flags &= ~REVFFN_FLAG_STEP_PIPELINED;
+  d_inv.flags = d_fwd.flags | REVFFN_FLAG_SAVE_ACTIVATIONS | REVFFN_FLAG_KEEP_STATUS | REVFFN_FLAG_ROUTER_FOLDED;
+  d_bwd.flags = d_fwd.flags | REVFFN_FLAG_REUSE_ACTIVATIONS | REVFFN_FLAG_KEEP_STATUS;
+  // this set's slots are free once the call before the previous one has sent its last result to the host
+  CK(cudaStreamWaitEvent(up, ev_free, 0));
+  CK(cudaStreamWaitEvent(st, ev_free, 0));
+  if (n > 0) {
+    CK(cudaMemcpyAsync(y1, y1_host, n, cudaMemcpyHostToDevice, up));
+    CK(cudaMemcpyAsync(x2, x2_host, n, cudaMemcpyHostToDevice, up));
+  }
+  CK(cudaEventRecord(S->ev[0], up));
+  if (n > 0) {
+    CK(cudaMemcpyAsync(dy2, dy2_host, n, cudaMemcpyHostToDevice, up));
+    CK(cudaMemsetAsync(dy1, 0, n, st));
+  }
+  CK(cudaEventRecord(S->ev[1], up));
+  CK(cudaStreamWaitEvent(st, S->ev[0], 0));
+  CKR(revffn_moe_forward(&d_fwd, w, y1, x2, y2, nullptr, ws, ws_bytes, st));
+  CK(cudaEventRecord(S->ev[2], st));
+  CK(cudaStreamWaitEvent(cs, S->ev[2], 0));
+  if (n > 0) CK(cudaMemcpyAsync(y2_host, y2, n, cudaMemcpyDeviceToHost, cs));
+  CKR(revffn_moe_inverse(&d_inv, w, y1, y2, x2r, nullptr, ws, ws_bytes, st));
+  CK(cudaEventRecord(S->ev[3], st));
+  CK(cudaStreamWaitEvent(cs, S->ev[3], 0));
+  if (n > 0) CK(cudaMemcpyAsync(x2_rec_host, x2r, n, cudaMemcpyDeviceToHost, cs));
+  CK(cudaStreamWaitEvent(st, S->ev[1], 0));
+  CKR(revffn_moe_backward(&d_bwd, w, y1, dy2, dy1, grads, nullptr, ws, ws_bytes, st));
+  CK(cudaEventRecord(S->ev[4], st));
+  CK(cudaStreamWaitEvent(cs, S->ev[4], 0));
+  if (n > 0) CK(cudaMemcpyAsync(dy1_host, dy1, n, cudaMemcpyDeviceToHost, cs));
+  CK(cudaEventRecord(ev_free, cs));
+  return REVFFN_OK;
 }
 
 int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* w, const revffn_moe_grads* grads,
@@ -1090,15 +1154,22 @@ int revffn_moe_step_host(const revffn_moe_desc* desc, const revffn_moe_weights* 
   if (desc->ld_stream != h) return REVFFN_ERR_SHAPE;
   const size_t n = (size_t)desc->tokens * h * sizeof(float);
   const size_t slot = (size_t)round_up((int64_t)(n > 0 ? n : 1), 256);
-  if (staging_bytes < 6 * slot || (reinterpret_cast<uintptr_t>(staging) & 255u)) return REVFFN_ERR_WORKSPACE;
+  const bool pipelined = (desc->flags & REVFFN_FLAG_STEP_PIPELINED) != 0;
+  if (staging_bytes < (pipelined ? 12 : 6) * slot || (reinterpret_cast<uintptr_t>(staging) & 255u)) return REVFFN_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(copy_stream);
   const bool two = copy_stream != nullptr && cs != st;
+  if (pipelined) {
+    if (!two) return REVFFN_ERR_UNSUPPORTED;      // the downloads need a stream of their own
+    return step_host_pipelined(desc, w, grads, y1_host, x2_host, dy2_host, y2_host, x2_rec_host, dy1_host,
+                               reinterpret_cast<char*>(staging), slot, n, ws, ws_bytes, st, cs);
+  }
   if (!two) cs = st;
   cudaEvent_t* ev = nullptr;
   if (two) {
-    ev = step_events(&r);
+    StepState* S = step_state(&r);
     if (r != REVFFN_OK) return r;
+    ev = S->ev;
   }
   char* sp = reinterpret_cast<char*>(staging);
   float* y1 = reinterpret_cast<float*>(sp);

@@ -286,6 +286,58 @@ def test_host_step_matches_the_device_entry_points(rv, two_streams, tokens):
         assert torch.equal(g[n], g_ref[n]), n
 
 
+def test_pipelined_host_steps_match_the_device_entry_points(rv):
+    """Five pipelined host steps on alternating inputs (the uploads of a step run beside the step before it,
+    its downloads beside the step after it): every step's host outputs, read once the copy stream has passed the
+    event recorded after its call, equal the device entry points' results bit for bit."""
+    cfg = small_cfg(tokens=700)
+    w = scaled_weights(cfg, 8, 4.0)
+    blk = make_block(cfg, w)
+    pin = lambda a: torch.from_numpy(a).pin_memory()
+    cases = []
+    for seed in (21, 22):
+        s = make_streams(cfg, seed)
+        y1, x2, dy2 = dev(s["y1"]), dev(s["x2"]), dev(s["dy2"])
+        y2 = blk.forward(y1, x2)
+        x2r = blk.inverse(y1, y2)
+        dy1, g_ref = torch.zeros_like(y1), grad_buffers(cfg, w)
+        blk.backward(y1, dy2, dy1, g_ref)
+        host_in = [pin(s[n]) for n in ("y1", "x2", "dy2")]
+        host_out = [torch.empty_like(host_in[0]).pin_memory() for _ in range(3)]
+        cases.append((host_in, host_out, [y2.cpu(), x2r.cpu(), dy1.cpu()], g_ref))
+    slot = ((cases[0][0][0].numel() * 4 + 255) // 256) * 256
+    staging = torch.empty(12 * slot, dtype=torch.uint8, device="cuda")
+    cs = torch.cuda.Stream()
+    g = grad_buffers(cfg, w)
+    with pytest.raises(rv.RevffnError):                                # six slots are not enough for this form
+        rv.revffn_moe_step_host(blk.desc, blk.w, blk.grads_struct(g), *cases[0][0], *cases[0][1], staging[:6 * slot], blk.ws,
+                                copy_stream=cs.cuda_stream, pipelined=True)
+    with pytest.raises(rv.RevffnError) as e:                           # and it needs the copy stream
+        rv.revffn_moe_step_host(blk.desc, blk.w, blk.grads_struct(g), *cases[0][0], *cases[0][1], staging, blk.ws, pipelined=True)
+    assert e.value.code == rv.ERR_UNSUPPORTED
+    events, prev = [], None
+    for i in range(5):
+        host_in, host_out, ref, g_ref = cases[i & 1]
+        rv.revffn_moe_step_host(blk.desc, blk.w, blk.grads_struct(g), *host_in, *host_out, staging, blk.ws,
+                                copy_stream=cs.cuda_stream, pipelined=True)
+        ev = torch.cuda.Event()
+        ev.record(cs)
+        if prev is not None:            # read the previous step's results while this one runs
+            prev[0].synchronize()
+            for got, want in zip(prev[1], prev[2]):
+                assert torch.equal(got, want)
+            for t in prev[1]:
+                t.fill_(float("nan"))
+        prev = (ev, host_out, ref)
+    prev[0].synchronize()
+    for got, want in zip(prev[1], prev[2]):
+        assert torch.equal(got, want)
+    torch.cuda.synchronize()
+    assert blk.status() == 0
+    for n in g:                          # the gradients of the last step (case 0)
+        assert torch.equal(g[n], cases[0][3][n]), n
+
+
 @pytest.mark.parametrize("kw", [dict(n_experts=64, top_k=8, tokens=150), dict(n_experts=130, top_k=3, tokens=97),
                                 dict(n_experts=256, top_k=8, tokens=70, d_shared=0)])
 def test_many_experts(rv, kw):
