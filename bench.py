@@ -86,6 +86,7 @@ def gemm_flops(cfg, routed_rows):
         "gemm_shared_down": 2 * T * Is * d, "gemm_p_down_couple": 2 * T * d * h, "gemm_dz": 2 * T * h * d,
         "wgrad_p_down": 2 * T * h * d, "gemm_shared_dh_dswiglu": 2 * T * d * Is, "wgrad_shared_down": 2 * T * d * Is,
         "gemm_shared_du": 2 * T * 2 * Is * d, "wgrad_shared_gate": 2 * T * Is * d, "wgrad_shared_up": 2 * T * Is * d,
+        "wgrad_shared_gate_up": 2 * T * 2 * Is * d,
         "gemm_expert_dh_dswiglu": 2 * R * d * I, "gemm_expert_du": 2 * R * 2 * I * d,
         "wgrad_expert_down": 2 * R * d * I, "wgrad_expert_gate": 2 * R * I * d, "wgrad_expert_up": 2 * R * I * d,
         "wgrad_expert_gate_up": 2 * R * 2 * I * d,
@@ -297,6 +298,12 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
         blk.inverse(y1, y2, x2r, save=True, flags=rv.FLAG_ROUTER_FOLDED)
         blk.backward(y1, dy2, dy1, grads, reuse=True)
 
+    def step_single():
+        # the same step with every launch on one stream (the library's second stream switched off)
+        blk.forward(y1, x2, y2, flags=rv.FLAG_SINGLE_STREAM)
+        blk.inverse(y1, y2, x2r, save=True, flags=rv.FLAG_ROUTER_FOLDED | rv.FLAG_SINGLE_STREAM)
+        blk.backward(y1, dy2, dy1, grads, reuse=True, flags=rv.FLAG_SINGLE_STREAM)
+
     def step_unshared():
         # every pass recomputes the branch on its own
         blk.forward(y1, x2, y2)
@@ -353,6 +360,9 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
     step_unshared()
     barrier()
     ms_unshared = timed(step_unshared, n_un) / n_un
+    step_single()
+    barrier()
+    ms_single = timed(step_single, n_un) / n_un
     # the FP8 variant of the routed experts (forward and inverse passes only): same block, e4m3 expert operands
     fp8_rec = None
     if cfg.weight_dtype == "bf16" and cfg.d_model <= 2048 and cfg.d_model % 256 == 0 and args.gating == "renorm":
@@ -387,7 +397,7 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
                    "note": "routed experts' three products on e4m3 operands with per-row scales (REVFFN_FLAG_FP8_EXPERTS); "
                            "branch output about 4-5 % (relative L2) from the bf16 evaluation; not part of the headline"}
         del blk8
-    ms_total, ms_unshared = max_over_ranks([ms_total, ms_unshared], world)
+    ms_total, ms_unshared, ms_single = max_over_ranks([ms_total, ms_unshared, ms_single], world)
     ms_step = ms_total / args.steps
     ms_prof_step = ms_prof_total / args.steps
     value = job_tokens_per_s(world, cfg.tokens, args.steps, ms_total)
@@ -556,6 +566,10 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
         "step_tflops": total_flops / (ms_step * 1e-3) / 1e12,
         "unshared": {"ms_per_step": ms_unshared, "value": world * cfg.tokens / (ms_unshared * 1e-3),
                      "note": "forward, inverse and backward each recompute the branch (3 evaluations, not 2)"},
+        "single_stream": {"ms_per_step": ms_single, "value": world * cfg.tokens / (ms_single * 1e-3),
+                          "note": "REVFFN_FLAG_SINGLE_STREAM: the shared expert and the weight gradients queue behind "
+                                  "the other launches instead of running beside them on the library's second stream; "
+                                  "the per-kernel figures (profiler on) are taken in this form"},
         "passes_ms": passes,
         "passes_tokens_per_s": {k: (cfg.tokens / (v * 1e-3) if v > 0 else None) for k, v in passes.items()},
         "grouped_expert_gemms": {"tflops": g_fl / (g_ms * 1e-3) / 1e12 if g_ms > 0 else None,

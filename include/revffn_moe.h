@@ -141,6 +141,12 @@ enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                
 /* revffn_moe_step_host only: the pipelined form described there (two staging sets used in turn, results
  * complete when the copy stream completes).  Other entry points ignore it. */
 #define REVFFN_FLAG_STEP_PIPELINED 512u
+/* Keep every launch of the call on cuda_stream.  Without it, calls of 1024 tokens or more on the tcgen05 back end
+ * put launches that nothing later in the pass depends on (the shared expert beside the routed experts, the weight
+ * gradients beside the input gradients) on a second stream that the library creates per device on first use,
+ * ordered against cuda_stream by events; cuda_stream still ends after everything of the call, and the results
+ * are the same bits either way. */
+#define REVFFN_FLAG_SINGLE_STREAM 1024u
 
 /*
  * Block descriptor.  Shape constraints (else REVFFN_ERR_SHAPE):

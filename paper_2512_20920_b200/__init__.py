@@ -15,7 +15,7 @@ __all__ = ["Block", "Stack", "revffn_moe_saved_size", "revffn_moe_stack_cache_st
            "revffn_moe_step_host", "revffn_moe_route_noalloc", "revffn_prof_enable", "revffn_prof_launches",
            "revffn_prof_collect", "RevffnError", "BF16", "F32", "NORM_RMS", "NORM_NONE", "FLAG_FORCE_SIMT",
            "FLAG_SAVE_ACTIVATIONS", "FLAG_REUSE_ACTIVATIONS", "FLAG_GATE_SOFTMAX_ALL", "FLAG_ROUTING_RECORD",
-           "FLAG_KEEP_STATUS", "FLAG_FP8_EXPERTS", "FLAG_STEP_PIPELINED", "FLAG_DEBUG_CHECKS", "FLAG_ROUTER_FOLDED", "ERR_DEVICE_WAIT", "ERR_UNSUPPORTED",
+           "FLAG_KEEP_STATUS", "FLAG_FP8_EXPERTS", "FLAG_STEP_PIPELINED", "FLAG_SINGLE_STREAM", "FLAG_DEBUG_CHECKS", "FLAG_ROUTER_FOLDED", "ERR_DEVICE_WAIT", "ERR_UNSUPPORTED",
            "ERR_NOALLOC_LIMIT", "ERR_INDEX", "Sgd", "make_sgd", "upd_mask", "UPD_NAMES", "UPD_ALL", "stage_update_mask",
            "revffn_moe_backward_sgd", "revffn_moe_stack_backward_sgd", "ERR_CANARY", "ERR_NONFINITE", "revffn_dbg_check_guards", "ws_lookup",
            "revffn_moe_routing_record_bytes", "AttnBranch", "AttnDesc", "AttnWeights", "AttnGrads",

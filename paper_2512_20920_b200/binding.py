@@ -25,6 +25,7 @@ FLAG_DEBUG_CHECKS = 64
 FLAG_ROUTER_FOLDED = 128
 FLAG_FP8_EXPERTS = 256
 FLAG_STEP_PIPELINED = 512
+FLAG_SINGLE_STREAM = 1024
 
 ERR_DEVICE_WAIT, ERR_UNSUPPORTED, ERR_NOALLOC_LIMIT, ERR_INDEX, ERR_CANARY, ERR_NONFINITE = -7, -8, -9, -10, -11, -12
 

@@ -2,6 +2,7 @@
 // See include/revffn_moe.h for the contract of every entry point.
 
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -28,7 +29,7 @@ namespace revffn {
 enum Tag {
   TG_NORM, TG_FOLD, TG_ROUTER, TG_MAP, TG_PUP, TG_GATHER, TG_EXP_GATEUP, TG_EXP_DOWN, TG_SH_GATEUP, TG_SH_DOWN,
   TG_COMBINE, TG_PDOWN, TG_CAST, TG_DZ, TG_WG_PDOWN, TG_SHGATE_BWD, TG_SH_DH, TG_WG_SH_DOWN, TG_SH_DU,
-  TG_WG_SH_GATE, TG_WG_SH_UP, TG_WG_SGATE, TG_GATHER_DZ, TG_EXP_DH, TG_EXP_DU, TG_WG_EXP_DOWN, TG_WG_EXP_GATE,
+  TG_WG_SH_GATE, TG_WG_SH_UP, TG_WG_SH_GATEUP, TG_WG_SGATE, TG_GATHER_DZ, TG_EXP_DH, TG_EXP_DU, TG_WG_EXP_DOWN, TG_WG_EXP_GATE,
   TG_WG_EXP_UP, TG_WG_EXP_GATEUP, TG_ROUTER_BWD, TG_WG_ROUTER, TG_DU_REDUCE, TG_DN, TG_WG_PUP, TG_NORM_BWD, TG_DGAMMA,
   // attention coupling branch
   TG_A_TABLES, TG_A_QKV, TG_A_HEADS, TG_A_SCORES, TG_A_SOFTMAX, TG_A_PV, TG_A_WO, TG_A_WGRAD, TG_A_DGRAD, TG_A_BIAS,
@@ -38,7 +39,7 @@ static const char* kTagNames[TG_COUNT] = {
     "rmsnorm_fwd", "fold_router", "router_topk", "permute_maps", "gemm_p_up", "gather_u", "gemm_expert_gate_up_swiglu",
     "gemm_expert_down_scale", "gemm_shared_gate_up_swiglu", "gemm_shared_down", "combine", "gemm_p_down_couple",
     "cast_dy2", "gemm_dz", "wgrad_p_down", "shared_gate_bwd", "gemm_shared_dh_dswiglu", "wgrad_shared_down",
-    "gemm_shared_du", "wgrad_shared_gate", "wgrad_shared_up", "wgrad_shared_sgate", "gather_dz",
+    "gemm_shared_du", "wgrad_shared_gate", "wgrad_shared_up", "wgrad_shared_gate_up", "wgrad_shared_sgate", "gather_dz",
     "gemm_expert_dh_dswiglu", "gemm_expert_du", "wgrad_expert_down", "wgrad_expert_gate", "wgrad_expert_up", "wgrad_expert_gate_up",
     "router_bwd", "wgrad_router", "du_reduce", "gemm_dn", "wgrad_p_up", "rmsnorm_bwd", "dgamma",
     "attn_tables", "gemm_qkv", "attn_heads", "gemm_scores", "attn_softmax", "gemm_pv", "gemm_w_o", "attn_wgrad",
@@ -304,6 +305,40 @@ static int guards_check(const WsLayout& L, size_t limit, char* ws, cudaStream_t 
 // ---------------------------------------------------------------------------
 // Launch context
 // ---------------------------------------------------------------------------
+// A second stream per device for launches that do not depend on what the caller's stream is doing at that point
+// (the shared expert beside the routed experts, the weight gradients beside the chain of input gradients).  The
+// matrix products are persistent kernels of one CTA per SM and equal tiles, so most of them end with a partly
+// empty last round of tiles; a kernel from the other stream starts on the SMs that fall idle there.  Ordering is by
+// events from a small ring (a wait refers to the record that preceded it, so an event can be recorded again while
+// an older wait is still pending).  Created on first use.
+struct Overlap {
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev[64];
+  std::atomic<unsigned> next{0};
+  bool made = false;
+  cudaEvent_t mark(cudaStream_t s, cudaError_t* e) {       // an event that follows everything queued on s so far
+    cudaEvent_t x = ev[next.fetch_add(1) & 63u];
+    *e = cudaEventRecord(x, s);
+    return x;
+  }
+};
+
+static Overlap* overlap_state() {
+  static Overlap state[64];
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  Overlap& o = state[dev];
+  if (!o.made) {
+    for (auto& x : o.ev)
+      if (cudaEventCreateWithFlags(&x, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithFlags(&o.side, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    o.made = true;
+  }
+  return &o;
+}
+
 template <typename T>
 struct Ctx {
   revffn_moe_desc D;
@@ -311,6 +346,16 @@ struct Ctx {
   WsLayout L;
   char* ws;
   cudaStream_t st;
+  Overlap* ov = nullptr;   // non-null: the second stream is in use for this call
+  // what is queued on `to` from now on follows everything queued on `from` so far (no-op without the second stream)
+  int order(cudaStream_t from, cudaStream_t to) const {
+    if (!ov || from == to) return REVFFN_OK;
+    cudaError_t e;
+    cudaEvent_t x = ov->mark(from, &e);
+    if (e != cudaSuccess || cudaStreamWaitEvent(to, x, 0) != cudaSuccess) return REVFFN_ERR_CUDA;
+    return REVFFN_OK;
+  }
+  cudaStream_t side() const { return ov ? ov->side : st; }
   bool tc;   // tcgen05 back end for the matrix products
   template <typename U> U* p(const Buf& b) const { return reinterpret_cast<U*>(ws + b.off); }
   int T_() const { return D.tokens; }
@@ -352,7 +397,9 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
   const int Tn = D.tokens, d = D.d_model, h = d / 2, E = D.n_experts, k = D.top_k, I = D.d_expert, Is = D.d_shared;
   const int norm_none = D.norm_kind == REVFFN_NORM_NONE;
   cudaStream_t st = c.st;
+  cudaStream_t rt = c.side();      // router and permutation maps (the caller's stream without the second stream)
   const T* w_up = reinterpret_cast<const T*>(c.W.w_up);
+  CKR(c.order(st, rt));
 
   // Norm
   { ProfScope ps(TG_NORM, st);
@@ -361,60 +408,62 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
   }
   CK(cudaGetLastError());
 
-  // Router: fold through P_up, logits, top-k, gates -- or everything from a routing record
+  // Router: fold through P_up, logits, top-k, gates -- or everything from a routing record.  The router reads y1
+  // and the permutation maps read the router's result: neither needs the norm or P_up, so with the second stream
+  // they run beside those two.
   const bool records = (D.flags & REVFFN_FLAG_ROUTING_RECORD) != 0;
   const bool gate_all = (D.flags & REVFFN_FLAG_GATE_SOFTMAX_ALL) != 0;
   const RecordLayout R = record_layout(D);
   if (idx_in && records && !gate_all) {
     const char* rec = reinterpret_cast<const char*>(idx_in);
     const size_t tk = (size_t)Tn * k * 4;
-    CK(cudaMemcpyAsync(c.ws + L.idx.off, rec, tk, cudaMemcpyDeviceToDevice, st));
-    CK(cudaMemcpyAsync(c.ws + L.gates.off, rec + R.gates_off, tk, cudaMemcpyDeviceToDevice, st));
-    CK(cudaMemcpyAsync(c.ws + L.sgate.off, rec + R.sgate_off, (size_t)Tn * 4, cudaMemcpyDeviceToDevice, st));
+    CK(cudaMemcpyAsync(c.ws + L.idx.off, rec, tk, cudaMemcpyDeviceToDevice, rt));
+    CK(cudaMemcpyAsync(c.ws + L.gates.off, rec + R.gates_off, tk, cudaMemcpyDeviceToDevice, rt));
+    CK(cudaMemcpyAsync(c.ws + L.sgate.off, rec + R.sgate_off, (size_t)Tn * 4, cudaMemcpyDeviceToDevice, rt));
   } else {
     if (!(D.flags & REVFFN_FLAG_ROUTER_FOLDED)) {     // else the folded router of an earlier call is still in the workspace
-    ProfScope ps(TG_FOLD, st);
+    ProfScope ps(TG_FOLD, rt);
     if (d <= FOLD_SLICES * fold_slice_rows<T>()) {
       CK(launch_fold_router_mma<T>(reinterpret_cast<const T*>(c.W.w_router), reinterpret_cast<const T*>(c.W.ws_sgate),
-                                   w_up, E, d, h, c.template p<double>(L.w_rc_part), c.template p<double>(L.w_rc), st));
+                                   w_up, E, d, h, c.template p<double>(L.w_rc_part), c.template p<double>(L.w_rc), rt));
       ++g_prof.launches;      // two kernels under one timing scope: the slice products and their sum
     } else {
       CK(launch_fold_router<T>(reinterpret_cast<const T*>(c.W.w_router), reinterpret_cast<const T*>(c.W.ws_sgate), w_up,
-                               E, d, h, c.template p<double>(L.w_rc), st));
+                               E, d, h, c.template p<double>(L.w_rc), rt));
     }
     }
-    { ProfScope ps(TG_ROUTER, st);
+    { ProfScope ps(TG_ROUTER, rt);
     CK(launch_router_topk(y1, D.ld_stream, c.W.norm_gamma, D.norm_eps, norm_none, c.template p<double>(L.w_rc),
                           c.W.b_router, Tn, h, E, k, Is > 0 ? 1 : 0, idx_in, c.template p<int32_t>(L.idx),
                           c.template p<float>(L.gates), c.template p<float>(L.sgate), idx_user,
                           gate_all ? c.template p<float>(L.prob) : nullptr, c.template p<int>(L.status),
-                          (D.flags & REVFFN_FLAG_DEBUG_CHECKS) ? 1 : 0, st));
+                          (D.flags & REVFFN_FLAG_DEBUG_CHECKS) ? 1 : 0, rt));
     }
     if (idx_user && records) {      // complete the record the kernel has started with the indices
       char* rec = reinterpret_cast<char*>(idx_user);
-      CK(cudaMemcpyAsync(rec + R.gates_off, c.ws + L.gates.off, (size_t)Tn * k * 4, cudaMemcpyDeviceToDevice, st));
-      CK(cudaMemcpyAsync(rec + R.sgate_off, c.ws + L.sgate.off, (size_t)Tn * 4, cudaMemcpyDeviceToDevice, st));
+      CK(cudaMemcpyAsync(rec + R.gates_off, c.ws + L.gates.off, (size_t)Tn * k * 4, cudaMemcpyDeviceToDevice, rt));
+      CK(cudaMemcpyAsync(rec + R.sgate_off, c.ws + L.sgate.off, (size_t)Tn * 4, cudaMemcpyDeviceToDevice, rt));
     }
   }
 
   // Permutation maps
-  CK(cudaMemsetAsync(c.ws + L.row_tok.off, 0xFF, L.row_tok.bytes, st));
-  CK(cudaMemsetAsync(c.ws + L.row_gate.off, 0, L.row_gate.bytes, st));
-  { ProfScope ps(TG_MAP, st);
-  map_rank_kernel<<<L.n_chunks, 256, (size_t)MAP_CHUNK * k * 4, st>>>(
+  CK(cudaMemsetAsync(c.ws + L.row_tok.off, 0xFF, L.row_tok.bytes, rt));
+  CK(cudaMemsetAsync(c.ws + L.row_gate.off, 0, L.row_gate.bytes, rt));
+  { ProfScope ps(TG_MAP, rt);
+  map_rank_kernel<<<L.n_chunks, 256, (size_t)MAP_CHUNK * k * 4, rt>>>(
       c.template p<int32_t>(L.idx), Tn, k, E, c.template p<int32_t>(L.local_rank), c.template p<int32_t>(L.chunk_cnt),
       c.template p<int>(L.status));
   }
   CK(cudaGetLastError());
-  { ProfScope ps(TG_MAP, st);
-  map_scan_kernel<<<1, 256, (size_t)(E + 1) * 4, st>>>(
+  { ProfScope ps(TG_MAP, rt);
+  map_scan_kernel<<<1, 256, (size_t)(E + 1) * 4, rt>>>(
       c.template p<int32_t>(L.chunk_cnt), L.n_chunks, E, c.template p<int32_t>(L.chunk_base),
       c.template p<int32_t>(L.expert_cnt), c.template p<int32_t>(L.expert_off), c.template p<int32_t>(L.tile_group),
       c.template p<int32_t>(L.rows_total), L.max_tiles, c.template p<int4>(L.tok_chunks), L.max_chunks);
   }
   CK(cudaGetLastError());
-  { ProfScope ps(TG_MAP, st);
-  map_assign_kernel<<<(unsigned)ceil_div((int64_t)Tn * k, 256), 256, 0, st>>>(
+  { ProfScope ps(TG_MAP, rt);
+  map_assign_kernel<<<(unsigned)ceil_div((int64_t)Tn * k, 256), 256, 0, rt>>>(
       c.template p<int32_t>(L.idx), c.template p<float>(L.gates), c.template p<int32_t>(L.local_rank),
       c.template p<int32_t>(L.chunk_base), c.template p<int32_t>(L.expert_off), Tn, k, E,
       c.template p<int32_t>(L.tok_row), c.template p<int32_t>(L.row_tok), c.template p<float>(L.row_gate));
@@ -430,6 +479,11 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     p.epilogue = EPI_STORE; p.C = c.template p<T>(L.u); p.ldc = d;
     CKR(run_gemm(c, p, TG_PUP));
   }
+  CKR(c.order(rt, st));            // the permutation needs the maps
+  // The shared expert needs u and nothing else of this pass: on the second stream it runs beside the routed experts.
+  Ctx<T> cs = c;
+  cs.st = c.side();
+  if (Is > 0) CKR(c.order(st, cs.st));
 
   const bool fp8 = (D.flags & REVFFN_FLAG_FP8_EXPERTS) != 0;
   if constexpr (std::is_same<T, bf16>::value) {
@@ -511,8 +565,7 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
       p.C = c.template p<T>(L.o); p.ldc = d;
       CKR(run_gemm(c, p, TG_EXP_DOWN));
     }
-  
-}
+  }
 
   // Shared expert: S = (silu(U Wsg^T) * (U Wsu^T)) Wsd^T
   if (Is > 0) {
@@ -522,13 +575,14 @@ static int run_branch(const Ctx<T>& c, const float* y1, const int32_t* idx_in, i
     p.B0 = c.W.ws_gate; p.B1 = c.W.ws_up; p.ldb = d; p.concat = CONCAT_N;
     p.epilogue = EPI_SWIGLU; p.C = c.template p<T>(L.hs); p.ldc = Is;
     if (save_ab) { p.C1 = c.template p<T>(L.abs); p.ldc1 = 2 * (int64_t)Is; }
-    CKR(run_gemm(c, p, TG_SH_GATEUP));
+    CKR(run_gemm(cs, p, TG_SH_GATEUP));
     GemmProblem q = blank_problem();
     q.M = Tn; q.N = d; q.K = Is;
     q.A = c.template p<T>(L.hs); q.lda = Is;
     q.B0 = c.W.ws_down; q.ldb = Is;
     q.epilogue = EPI_STORE; q.C = c.template p<T>(L.s); q.ldc = d;
-    CKR(run_gemm(c, q, TG_SH_DOWN));
+    CKR(run_gemm(cs, q, TG_SH_DOWN));
+    CKR(c.order(cs.st, st));
   }
 
   // Combine: Z[t] = sum_s O[row(t,s)] + sgate_t S[t]
@@ -573,11 +627,16 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
   // sgd->mask), the weight W itself is updated tile by tile in the product's epilogue and no gradient is stored.
   // out2 / W2 / master2: second output of a product whose M is two stacked weights (gate | up of the experts).
   const uint32_t upd_mask = sgd ? sgd->mask : 0u;
+  Ctx<T> cw = c;
+  cw.st = c.side();
   auto wgrad = [&](int tag, uint32_t bit, float* out, const void* W, float* master, int M, int N, const void* A, int64_t lda,
                    int a_col0, const void* B, int64_t ldb, bool grouped, int64_t cstride, float* out2 = nullptr,
                    const void* W2 = nullptr, float* master2 = nullptr) -> int {
     const bool upd = (upd_mask & bit) != 0;
     if (!upd && !out) return REVFFN_OK;      // frozen: neither gradient nor update wanted
+    // Nothing later in this pass reads a weight gradient (or an updated weight): the product goes to the second
+    // stream, after everything queued so far (its operands, and every product that reads the weight it may update).
+    CKR(c.order(st, cw.st));
     GemmProblem p = blank_problem();
     p.M = M; p.N = N; p.K = grouped ? Rp : Tn;   // grouped: bound on rows, the range comes from group_off
     p.a_mn_major = 1; p.b_mn_major = 1;
@@ -610,15 +669,15 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
         if ((size_t)n_split * M * N * 4 > L.ksplit.bytes || Tn < 64 * 8 * n_split || (M * (int64_t)N) % 4 != 0 || M % TC_BM != 0) n_split = 1;
       }
     }
-    if (n_split <= 1) return run_gemm(c, p, tag);
+    if (n_split <= 1) return run_gemm(cw, p, tag);
     p.group_mode = GROUP_K; p.n_groups = n_split; p.group_off = nullptr;
     p.C = c.template p<float>(L.ksplit); p.C2 = nullptr; p.c_group_stride = (int64_t)M * N; p.accumulate = 0;
     p.upd_w = nullptr; p.upd_m = nullptr;
-    CKR(run_gemm(c, p, tag));
+    CKR(run_gemm(cw, p, tag));
     {
-      ProfScope ps(tag, st);
+      ProfScope ps(tag, cw.st);
       const int64_t count = (int64_t)M * N;
-      splitk_reduce_kernel<T><<<(unsigned)ceil_div(count, 4 * 256), 256, 0, st>>>(
+      splitk_reduce_kernel<T><<<(unsigned)ceil_div(count, 4 * 256), 256, 0, cw.st>>>(
           c.template p<float>(L.ksplit), n_split, count, out, acc, upd ? reinterpret_cast<T*>(const_cast<void*>(W)) : nullptr,
           upd ? master : nullptr, upd ? sgd->lr : 0.f);
     }
@@ -671,10 +730,21 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       p.epilogue = EPI_STORE; p.C = c.template p<T>(L.dush); p.ldc = d;
       CKR(run_gemm(c, p, TG_SH_DU));
     }
-    CKR(wgrad(TG_WG_SH_GATE, REVFFN_UPD_WS_GATE, G.ws_gate, c.W.ws_gate, S.m_ws_gate, Is, d, c.template p<T>(L.abs),
-              2 * (int64_t)Is, 0, c.template p<T>(L.u), d, false, 0));
-    CKR(wgrad(TG_WG_SH_UP, REVFFN_UPD_WS_UP, G.ws_up, c.W.ws_up, S.m_ws_up, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, Is,
-              c.template p<T>(L.u), d, false, 0));
+    {
+      // as for the routed experts below: da|db is one buffer and both gradients read u, so when both are wanted in
+      // the same form they are one product with M = 2 I_s and two outputs (352 instead of 2 x 176 output tiles of
+      // 256 x 256 at the benchmark shape: 4.8 instead of 2 x 2.4 waves of 74 CTA pairs)
+      const bool ug = (upd_mask & REVFFN_UPD_WS_GATE) != 0, uu = (upd_mask & REVFFN_UPD_WS_UP) != 0;
+      if ((ug && uu) || (!ug && !uu && G.ws_gate && G.ws_up)) {
+        CKR(wgrad(TG_WG_SH_GATEUP, REVFFN_UPD_WS_GATE, G.ws_gate, c.W.ws_gate, S.m_ws_gate, 2 * Is, d, c.template p<T>(L.abs),
+                  2 * (int64_t)Is, 0, c.template p<T>(L.u), d, false, 0, G.ws_up, c.W.ws_up, S.m_ws_up));
+      } else {
+        CKR(wgrad(TG_WG_SH_GATE, REVFFN_UPD_WS_GATE, G.ws_gate, c.W.ws_gate, S.m_ws_gate, Is, d, c.template p<T>(L.abs),
+                  2 * (int64_t)Is, 0, c.template p<T>(L.u), d, false, 0));
+        CKR(wgrad(TG_WG_SH_UP, REVFFN_UPD_WS_UP, G.ws_up, c.W.ws_up, S.m_ws_up, Is, d, c.template p<T>(L.abs), 2 * (int64_t)Is, Is,
+                  c.template p<T>(L.u), d, false, 0));
+      }
+    }
     if (G.ws_sgate) {
       { ProfScope ps(TG_WG_SGATE, st);
       CK(launch_colsum_partial<T>(c.template p<T>(L.u), d, c.template p<float>(L.dl), Tn, d, STRIP, L.strips,
@@ -827,6 +897,7 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       CK(cudaGetLastError());
     }
   }
+  CKR(c.order(cw.st, st));      // the caller's stream ends after the weight gradients too
   return REVFFN_OK;
 }
 
@@ -843,6 +914,12 @@ static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weight
   c.D = D; c.W = W; c.L = L; c.ws = reinterpret_cast<char*>(ws); c.st = st;
   g_prof.pass = (int)pass;
   c.tc = std::is_same<T, bf16>::value && !(D.flags & REVFFN_FLAG_FORCE_SIMT);
+  // second stream: only where the launches are long enough for their last rounds to matter, and never while the
+  // per-launch profiler is on (its events bracket launches on one stream)
+  if (c.tc && !g_prof.on && !(D.flags & REVFFN_FLAG_SINGLE_STREAM) && D.tokens >= 1024) {
+    c.ov = overlap_state();
+    if (!c.ov) return REVFFN_ERR_CUDA;
+  }
   if (c.tc) CKR(tc_prepare());
   if (!(D.flags & REVFFN_FLAG_KEEP_STATUS)) CK(cudaMemsetAsync(c.ws + L.status.off, 0, L.status.bytes, st));
   if (D.tokens == 0) return REVFFN_OK;   // empty batch: nothing to compute, gradients untouched
