@@ -89,6 +89,8 @@ typedef struct {
    * context must stay usable.  Nothing is in flight when that wait expires. */
   int64_t wait_cycles;
   int32_t starve_operands;
+  /* measurements: operand loads issued by two threads (1) or by one (2); 0 = the library's choice per epilogue */
+  int32_t split_loads;
 } revffn_dbg_gemm_args;
 int revffn_dbg_gemm(const revffn_dbg_gemm_args* args, int32_t* status_word_dev, void* cuda_stream);
 

@@ -1,10 +1,13 @@
 // tcgen05 / TMEM / TMA back end for every bf16 matrix product on the path.
 //
-// One persistent, warp-specialised kernel (1 CTA per SM, 320 threads):
-//   warp 0      TMA producer: cp.async.bulk.tensor 2D loads (128-byte swizzle) of
+// One persistent, warp-specialised kernel (1 CTA per SM, 352 threads):
+//   warps 0, 10 TMA producers: cp.async.bulk.tensor 2D loads (128-byte swizzle) of
 //               A and B tiles into a ring of shared-memory stages, completion on
 //               mbarriers (no multicast LOADS anywhere: every CTA fetches its own operands; the only
-//               cluster-wide instruction is the pair mode's tcgen05.commit, a barrier arrive).
+//               cluster-wide instruction is the pair mode's tcgen05.commit, a barrier arrive).  One thread
+//               of warp 0 announces a stage's bytes and loads the first operand's share, one thread of
+//               warp 10 loads the second operand's: a single thread cannot issue a stage's loads as fast
+//               as the tensor core consumes them.
 //   warp 1      MMA issuer: owns the TMEM allocation (two accumulators, so the
 //               epilogue of tile i overlaps the main loop of tile i+1); one
 //               elected lane issues tcgen05.mma kind::f16 (bf16 x bf16 -> fp32),
@@ -54,7 +57,8 @@ namespace revffn {
 
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;
-constexpr int TC_THREADS = 320;
+constexpr int TC_THREADS = 352;      // warp 0, 10: operand loads; warp 1: products; warps 2..9: epilogue
+constexpr int TC_LOAD_WARP_B = 10;   // the second load warp
 constexpr int TC_EPI_WARPS = 8;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;            // 16 KB
 constexpr long long TC_WAIT_CYCLES = 4000000000LL;       // ~2 s: bound on any single wait
@@ -83,6 +87,7 @@ struct TcParams {
   long long wait_cycles;     // bound on every wait of the kernel (clock cycles)
   int starve;                // failure-path test: the load warp issues nothing, so the first wait for operands runs out
   int bk;                    // operand elements per K step: 64 (bf16) or 128 (e4m3); a K step is 128 bytes of a row either way
+  int split_loads;           // 1: the second load warp issues the second operand's loads; 0: one thread issues all of them
 };
 
 // ---------------------------------------------------------------------------
@@ -439,6 +444,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + Cfg::BAR_OFF + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* issued = reinterpret_cast<int*>(tmem_slot + 2);   // [STAGES] parity+1 of the last load issued per stage
+  int* issued_b = issued + Cfg::STAGES;                  // the same for the second load warp: nonzero once it has issued
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int crank = PAIR ? (int)cluster_ctarank() : 0;     // rank in the pair; rank 0 issues the MMAs
@@ -447,7 +453,7 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   const int wstride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < Cfg::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); issued[s] = 0; }
+    for (int s = 0; s < Cfg::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); issued[s] = 0; issued_b[s] = 0; }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), PAIR ? 2 * TC_EPI_WARPS : TC_EPI_WARPS); }
     mbar_init(drain_bar, 1);
     *abort_flag = 0;
@@ -474,12 +480,22 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   int tiles_m_dev = P.tiles_m;
   if (p.group_mode == GROUP_M) tiles_m_dev = min(P.tiles_m, *p.rows_total / TC_BM);
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ producer
+  if (warp == 0 || warp == TC_LOAD_WARP_B) {
+    // ------------------------------------------------------------------ operand loads
+    // Two threads, one in each load warp, walk the same tiles and stages.  A tensor load takes the issuing thread
+    // 150-250 clocks (more in the pair form, whose completion is signalled in the partner CTA), and a stage needs
+    // two to six of them: issued by one thread they took 500-850 clocks per stage, more than the 512 clocks of
+    // tensor work in a stage, and the MMA thread waited for operands in every product.  Thread A announces the
+    // stage's bytes and loads the first operand's share of the stage, thread B loads the second operand's; the
+    // bytes may arrive before they are announced (the barrier's phase cannot complete before the announcing
+    // arrival).
     // (A version of this loop that kept per-tile "load slots" -- tensor-map pointer, destination, coordinates --
     // in registers and issued one load per slot measured 15-40 % slower: a load whose tensor map is named through
     // a pointer chosen at run time, rather than as the kernel parameter itself, is slow to issue.)
-    if (lane == 0 && !P.starve) {
+    // la: this thread loads the first operand's share (and announces the stage); lb: the second operand's.
+    // Without split_loads the first warp's thread does both and the second warp has nothing to do.
+    const bool la = warp == 0, lb = P.split_loads ? warp != 0 : warp == 0;
+    if (lane == 0 && !P.starve && (la || lb)) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -497,90 +513,110 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             if (P.tr) {
               // M side: 128 rows of the expert's weights; N side: this CTA's half of the chunk's token rows
               // (a full 128-row box either way; rows past the half are loaded and not used)
-              if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
-              const CUtensorMap* mw = &map_b0;
-              int kw = kb;
-              if (p.concat == CONCAT_K && kb >= k_half) { mw = &map_b1; kw = kb - k_half; }
-              if (!p.b_mn_major) {
-                tma_load_2d_pair(sa, mw, kw * P.bk, t.group * p.N + t.n0, fbc);
-              } else {
-                const int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
-                const int krow = t.group * kdim + kw * TC_BK;
+              if (la) {
+                if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
+                int kw = kb;
+                const bool second = p.concat == CONCAT_K && kb >= k_half;
+                if (second) kw = kb - k_half;
+                if (!p.b_mn_major) {
+                  if (second) tma_load_2d_pair(sa, &map_b1, kw * P.bk, t.group * p.N + t.n0, fbc);
+                  else tma_load_2d_pair(sa, &map_b0, kw * P.bk, t.group * p.N + t.n0, fbc);
+                } else {
+                  const int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
+                  const int krow = t.group * kdim + kw * TC_BK;
 #pragma unroll
-                for (int j = 0; j < 2; ++j) tma_load_2d_pair(sa + j * 8192, mw, p.b_col0 + t.n0 + 64 * j, krow, fbc);
+                  for (int j = 0; j < 2; ++j) {
+                    if (second) tma_load_2d_pair(sa + j * 8192, &map_b1, p.b_col0 + t.n0 + 64 * j, krow, fbc);
+                    else tma_load_2d_pair(sa + j * 8192, &map_b0, p.b_col0 + t.n0 + 64 * j, krow, fbc);
+                  }
+                }
               }
-              tma_load_2d_pair(sb, &map_a, kb * P.bk, t.m0 + crank * (t.ncols / 2), fbc);
+              if (lb) tma_load_2d_pair(sb, &map_a, kb * P.bk, t.m0 + crank * (t.ncols / 2), fbc);
               if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
               continue;
             }
             const int nhalf = t.ncols / 2;       // this CTA's share of the tile's columns: 128, or 64 in a ragged last tile
-            if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * (TC_A_BYTES + nhalf * TC_BK * 2));
-            if (!p.a_mn_major) {
-              tma_load_2d_pair(sa, &map_a, kb * TC_BK, t.m0, fbc);
-            } else {
-              const int krow = t.krow0 + kb * TC_BK;
-#pragma unroll
-              for (int j = 0; j < 2; ++j) tma_load_2d_pair(sa + j * 8192, &map_a, p.a_col0 + t.m0 + 64 * j, krow, fbc);
-            }
-            const CUtensorMap* mbp = &map_b0;
-            int kbp = kb;
-            if (p.concat == CONCAT_K && kb >= k_half) { mbp = &map_b1; kbp = kb - k_half; }
-            if (!p.b_mn_major) {
-              // this CTA's 128 of the 256 accumulator columns: gate rows (rank 0) or up rows (rank 1) of a
-              // SwiGLU pair, else rows n0 + 128 rank .. + 127 of B
-              // (the tensor map is named directly in each call: a map chosen through a pointer is slow to issue)
-              if (p.concat == CONCAT_N) {
-                if (crank == 0) tma_load_2d_pair(sb, &map_b0, kbp * TC_BK, t.n0, fbc);
-                else tma_load_2d_pair(sb, &map_b1, kbp * TC_BK, t.n0, fbc);
-              } else if (p.concat == CONCAT_K && kb >= k_half) {
-                tma_load_2d_pair(sb, &map_b1, kbp * TC_BK, t.n0 + 128 * crank, fbc);
+            if (la) {
+              if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * (TC_A_BYTES + nhalf * TC_BK * 2));
+              if (!p.a_mn_major) {
+                tma_load_2d_pair(sa, &map_a, kb * TC_BK, t.m0, fbc);
               } else {
-                tma_load_2d_pair(sb, &map_b0, kbp * TC_BK, t.n0 + 128 * crank, fbc);
-              }
-            } else {
-              const int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
-              (void)kdim;
-              const int krow = t.krow0 + kbp * TC_BK;
+                const int krow = t.krow0 + kb * TC_BK;
 #pragma unroll
-              for (int j = 0; j < 2; ++j)
-                if (64 * j < nhalf) tma_load_2d_pair(sb + j * 8192, mbp, p.b_col0 + t.n0 + nhalf * crank + 64 * j, krow, fbc);
+                for (int j = 0; j < 2; ++j) tma_load_2d_pair(sa + j * 8192, &map_a, p.a_col0 + t.m0 + 64 * j, krow, fbc);
+              }
+            }
+            if (lb) {
+              const bool second = p.concat == CONCAT_K && kb >= k_half;
+              const int kbp = second ? kb - k_half : kb;
+              if (!p.b_mn_major) {
+                // this CTA's 128 of the 256 accumulator columns: gate rows (rank 0) or up rows (rank 1) of a
+                // SwiGLU pair, else rows n0 + 128 rank .. + 127 of B
+                // (the tensor map is named directly in each call: a map chosen through a pointer is slow to issue)
+                if (p.concat == CONCAT_N) {
+                  if (crank == 0) tma_load_2d_pair(sb, &map_b0, kbp * TC_BK, t.n0, fbc);
+                  else tma_load_2d_pair(sb, &map_b1, kbp * TC_BK, t.n0, fbc);
+                } else if (second) {
+                  tma_load_2d_pair(sb, &map_b1, kbp * TC_BK, t.n0 + 128 * crank, fbc);
+                } else {
+                  tma_load_2d_pair(sb, &map_b0, kbp * TC_BK, t.n0 + 128 * crank, fbc);
+                }
+              } else {
+                const int krow = t.krow0 + kbp * TC_BK;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                  if (64 * j >= nhalf) continue;
+                  if (second) tma_load_2d_pair(sb + j * 8192, &map_b1, p.b_col0 + t.n0 + nhalf * crank + 64 * j, krow, fbc);
+                  else tma_load_2d_pair(sb + j * 8192, &map_b0, p.b_col0 + t.n0 + nhalf * crank + 64 * j, krow, fbc);
+                }
+              }
             }
             if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
             continue;
           }
           const uint32_t fb = full_bar(stage);
-          mbar_expect_tx(fb, TC_A_BYTES + t.ncols * TC_BK * 2);
-          issued[stage] = (int)phase + 1;
-          // A tile
-          if (!p.a_mn_major) {
-            tma_load_2d(sa, &map_a, kb * P.bk, t.m0, fb);
-          } else {
-            int krow = t.krow0 + kb * TC_BK;
-#pragma unroll
-            for (int j = 0; j < 2; ++j) tma_load_2d(sa + j * 8192, &map_a, p.a_col0 + t.m0 + 64 * j, krow, fb);
-          }
-          // B tile
-          const CUtensorMap* mb = &map_b0;
-          int kb_b = kb;
-          if (p.concat == CONCAT_K && kb >= k_half) { mb = &map_b1; kb_b = kb - k_half; }
-          if (!p.b_mn_major) {
-            // rows of the flattened [groups * N, K] weight tensor
-            int row0 = (p.group_mode == GROUP_M ? t.group * p.N : 0) + t.n0;
-            if (p.concat == CONCAT_N) {
-              tma_load_2d(sb, &map_b0, kb_b * P.bk, row0, fb);
-              tma_load_2d(sb + 16384, &map_b1, kb_b * P.bk, row0, fb);
+          if (la) {
+            mbar_expect_tx(fb, TC_A_BYTES + t.ncols * TC_BK * 2);
+            issued[stage] = (int)phase + 1;
+            // A tile
+            if (!p.a_mn_major) {
+              tma_load_2d(sa, &map_a, kb * P.bk, t.m0, fb);
             } else {
+              int krow = t.krow0 + kb * TC_BK;
 #pragma unroll
-              for (int j = 0; j < MMA_N / 128; ++j)
-                if (128 * j < t.ncols) tma_load_2d(sb + j * 16384, mb, kb_b * P.bk, row0 + 128 * j, fb);
+              for (int j = 0; j < 2; ++j) tma_load_2d(sa + j * 8192, &map_a, p.a_col0 + t.m0 + 64 * j, krow, fb);
             }
-          } else {
-            // rows of the flattened [groups * Kdim, N] weight tensor, or token rows (GROUP_K / dense wgrad)
-            int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
-            int krow = (p.group_mode == GROUP_M ? t.group * kdim : t.krow0) + kb_b * TC_BK;
+          }
+          if (lb) {
+            issued_b[stage] = (int)phase + 1;
+            // B tile
+            const bool second = p.concat == CONCAT_K && kb >= k_half;
+            const int kb_b = second ? kb - k_half : kb;
+            if (!p.b_mn_major) {
+              // rows of the flattened [groups * N, K] weight tensor
+              int row0 = (p.group_mode == GROUP_M ? t.group * p.N : 0) + t.n0;
+              if (p.concat == CONCAT_N) {
+                tma_load_2d(sb, &map_b0, kb_b * P.bk, row0, fb);
+                tma_load_2d(sb + 16384, &map_b1, kb_b * P.bk, row0, fb);
+              } else {
 #pragma unroll
-            for (int j = 0; j < MMA_N / 64; ++j)
-              if (64 * j < t.ncols) tma_load_2d(sb + j * 8192, mb, p.b_col0 + t.n0 + 64 * j, krow, fb);
+                for (int j = 0; j < MMA_N / 128; ++j) {
+                  if (128 * j >= t.ncols) continue;
+                  if (second) tma_load_2d(sb + j * 16384, &map_b1, kb_b * P.bk, row0 + 128 * j, fb);
+                  else tma_load_2d(sb + j * 16384, &map_b0, kb_b * P.bk, row0 + 128 * j, fb);
+                }
+              }
+            } else {
+              // rows of the flattened [groups * Kdim, N] weight tensor, or token rows (GROUP_K / dense wgrad)
+              int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
+              int krow = (p.group_mode == GROUP_M ? t.group * kdim : t.krow0) + kb_b * TC_BK;
+#pragma unroll
+              for (int j = 0; j < MMA_N / 64; ++j) {
+                if (64 * j >= t.ncols) continue;
+                if (second) tma_load_2d(sb + j * 8192, &map_b1, p.b_col0 + t.n0 + 64 * j, krow, fb);
+                else tma_load_2d(sb + j * 8192, &map_b0, p.b_col0 + t.n0 + 64 * j, krow, fb);
+              }
+            }
           }
           if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -1034,10 +1070,16 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
   __syncthreads();
   if (*abort_flag && threadIdx.x == 0) {
     // loads already issued into this CTA's shared memory must land before the CTA exits
+    bool unannounced = false;     // the second load warp issued into a stage whose bytes the first never announced
     for (int s = 0; s < Cfg::STAGES; ++s) {
+      if (issued_b[s] != 0 && issued_b[s] != issued[s]) unannounced = true;
       if (issued[s] == 0) continue;
       long long t0 = clock64();
       while (!mbar_try_wait(full_bar(s), (uint32_t)(issued[s] - 1)) && clock64() - t0 < P.wait_cycles) {}
+    }
+    if (unannounced) {            // that stage's barrier cannot complete: give its loads a bounded time to land
+      const long long t0 = clock64();
+      while (clock64() - t0 < 4000000LL) {}
     }
   }
   __syncthreads();
@@ -1206,6 +1248,9 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   }
   P.wait_cycles = p.dbg_wait_cycles > 0 ? p.dbg_wait_cycles : TC_WAIT_CYCLES;
   P.starve = p.dbg_starve;
+  // Two load threads in every mode: measured against one thread in the same process, alternating, the whole step
+  // is 4-5 % faster and no product is slower (the one-thread form stays selectable for such measurements).
+  P.split_loads = p.dbg_split_loads != 2;
   if (p.dbg_starve && !p.no_pair) return REVFFN_ERR_UNSUPPORTED;      // the starved-wait test runs one CTA per tile
   if (p.N % 128 != 0) return REVFFN_ERR_SHAPE;
   // K need not be a multiple of the 64-wide K step: the tensor maps end at K, so the rest of the last
