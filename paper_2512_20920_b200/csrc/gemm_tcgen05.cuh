@@ -87,6 +87,7 @@ struct TcParams {
   long long wait_cycles;     // bound on every wait of the kernel (clock cycles)
   int starve;                // failure-path test: the load warp issues nothing, so the first wait for operands runs out
   int bk;                    // operand elements per K step: 64 (bf16) or 128 (e4m3); a K step is 128 bytes of a row either way
+  int mn3d;                  // MN-major operands are loaded 128 columns at a time through 3-D tensor maps
   int split_loads;           // 1: the second load warp issues the second operand's loads; 0: one thread issues all of them
 };
 
@@ -158,6 +159,32 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_cluster) : "memory");
+}
+// 128 columns x 64 K rows of an MN-major operand ([K rows, ld columns] in memory) into two consecutive 8 KB
+// blocks of 64 columns each, the layout the MMA descriptors expect.  mn3d: one load through a 3-D view of the
+// matrix {64 columns, K rows, ld / 64 column groups} with a box of two groups; else two 2-D loads of 64 x 64.
+// A tensor load costs its issuing thread a couple of hundred clocks whatever its size, so halving their number
+// matters as much as spreading them over two threads.
+__device__ __forceinline__ void tma_load_mn128(bool mn3d, uint32_t dst, const CUtensorMap* map, int col, int krow, uint32_t bar) {
+  if (mn3d) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(krow), "r"(col >> 6), "r"(bar) : "memory");
+  } else {
+    tma_load_2d(dst, map, col, krow, bar);
+    tma_load_2d(dst + 8192, map, col + 64, krow, bar);
+  }
+}
+__device__ __forceinline__ void tma_load_mn128_pair(bool mn3d, uint32_t dst, const CUtensorMap* map, int col, int krow,
+                                                    uint32_t bar_cluster, bool second_block = true) {
+  if (mn3d) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(krow), "r"(col >> 6), "r"(bar_cluster) : "memory");
+  } else {
+    tma_load_2d_pair(dst, map, col, krow, bar_cluster);
+    if (second_block) tma_load_2d_pair(dst + 8192, map, col + 64, krow, bar_cluster);
+  }
 }
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -524,11 +551,8 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
                 } else {
                   const int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
                   const int krow = t.group * kdim + kw * TC_BK;
-#pragma unroll
-                  for (int j = 0; j < 2; ++j) {
-                    if (second) tma_load_2d_pair(sa + j * 8192, &map_b1, p.b_col0 + t.n0 + 64 * j, krow, fbc);
-                    else tma_load_2d_pair(sa + j * 8192, &map_b0, p.b_col0 + t.n0 + 64 * j, krow, fbc);
-                  }
+                  if (second) tma_load_mn128_pair(P.mn3d, sa, &map_b1, p.b_col0 + t.n0, krow, fbc);
+                  else tma_load_mn128_pair(P.mn3d, sa, &map_b0, p.b_col0 + t.n0, krow, fbc);
                 }
               }
               if (lb) tma_load_2d_pair(sb, &map_a, kb * P.bk, t.m0 + crank * (t.ncols / 2), fbc);
@@ -537,13 +561,13 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             }
             const int nhalf = t.ncols / 2;       // this CTA's share of the tile's columns: 128, or 64 in a ragged last tile
             if (la) {
-              if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * (TC_A_BYTES + nhalf * TC_BK * 2));
+              // (a 3-D load of an MN-major B always brings 128 columns, also where this CTA's share is 64)
+              const int b_cols = (p.b_mn_major && P.mn3d) ? 128 : nhalf;
+              if (crank == 0) mbar_expect_tx(full_bar(stage), 2 * (TC_A_BYTES + b_cols * TC_BK * 2));
               if (!p.a_mn_major) {
                 tma_load_2d_pair(sa, &map_a, kb * TC_BK, t.m0, fbc);
               } else {
-                const int krow = t.krow0 + kb * TC_BK;
-#pragma unroll
-                for (int j = 0; j < 2; ++j) tma_load_2d_pair(sa + j * 8192, &map_a, p.a_col0 + t.m0 + 64 * j, krow, fbc);
+                tma_load_mn128_pair(P.mn3d, sa, &map_a, p.a_col0 + t.m0, t.krow0 + kb * TC_BK, fbc);
               }
             }
             if (lb) {
@@ -563,18 +587,19 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
                 }
               } else {
                 const int krow = t.krow0 + kbp * TC_BK;
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                  if (64 * j >= nhalf) continue;
-                  if (second) tma_load_2d_pair(sb + j * 8192, &map_b1, p.b_col0 + t.n0 + nhalf * crank + 64 * j, krow, fbc);
-                  else tma_load_2d_pair(sb + j * 8192, &map_b0, p.b_col0 + t.n0 + nhalf * crank + 64 * j, krow, fbc);
-                }
+                if (second) tma_load_mn128_pair(P.mn3d, sb, &map_b1, p.b_col0 + t.n0 + nhalf * crank, krow, fbc, nhalf > 64);
+                else tma_load_mn128_pair(P.mn3d, sb, &map_b0, p.b_col0 + t.n0 + nhalf * crank, krow, fbc, nhalf > 64);
               }
             }
             if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
             continue;
           }
           const uint32_t fb = full_bar(stage);
+          const bool second = p.concat == CONCAT_K && kb >= k_half;
+          const int kb_b = second ? kb - k_half : kb;
+          // An MN-major B tile is four 64 x 64 boxes against one or two loads for A: with two load threads the
+          // first takes B's last boxes too (3 + 2 loads, or 3 + 3 when A is MN-major as well).
+          const int b_mn_split = !p.b_mn_major ? 0 : (!P.split_loads ? 0 : ((p.a_mn_major && !P.mn3d) ? 3 : 2));
           if (la) {
             mbar_expect_tx(fb, TC_A_BYTES + t.ncols * TC_BK * 2);
             issued[stage] = (int)phase + 1;
@@ -582,16 +607,29 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             if (!p.a_mn_major) {
               tma_load_2d(sa, &map_a, kb * P.bk, t.m0, fb);
             } else {
-              int krow = t.krow0 + kb * TC_BK;
+              tma_load_mn128(P.mn3d, sa, &map_a, p.a_col0 + t.m0, t.krow0 + kb * TC_BK, fb);
+            }
+            if (b_mn_split) {
+              int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
+              int krow = (p.group_mode == GROUP_M ? t.group * kdim : t.krow0) + kb_b * TC_BK;
+              if (P.mn3d) {          // the second 128 columns
+                if (t.ncols > 128) {
+                  if (second) tma_load_mn128(true, sb + 16384, &map_b1, p.b_col0 + t.n0 + 128, krow, fb);
+                  else tma_load_mn128(true, sb + 16384, &map_b0, p.b_col0 + t.n0 + 128, krow, fb);
+                }
+              } else {
 #pragma unroll
-              for (int j = 0; j < 2; ++j) tma_load_2d(sa + j * 8192, &map_a, p.a_col0 + t.m0 + 64 * j, krow, fb);
+                for (int j = 2; j < MMA_N / 64; ++j) {
+                  if (j < b_mn_split || 64 * j >= t.ncols) continue;
+                  if (second) tma_load_2d(sb + j * 8192, &map_b1, p.b_col0 + t.n0 + 64 * j, krow, fb);
+                  else tma_load_2d(sb + j * 8192, &map_b0, p.b_col0 + t.n0 + 64 * j, krow, fb);
+                }
+              }
             }
           }
           if (lb) {
             issued_b[stage] = (int)phase + 1;
             // B tile
-            const bool second = p.concat == CONCAT_K && kb >= k_half;
-            const int kb_b = second ? kb - k_half : kb;
             if (!p.b_mn_major) {
               // rows of the flattened [groups * N, K] weight tensor
               int row0 = (p.group_mode == GROUP_M ? t.group * p.N : 0) + t.n0;
@@ -610,11 +648,20 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
               // rows of the flattened [groups * Kdim, N] weight tensor, or token rows (GROUP_K / dense wgrad)
               int kdim = (p.concat == CONCAT_K) ? k_half * TC_BK : t.k_blocks * TC_BK;
               int krow = (p.group_mode == GROUP_M ? t.group * kdim : t.krow0) + kb_b * TC_BK;
+              if (P.mn3d) {
+                if (second) tma_load_mn128(true, sb, &map_b1, p.b_col0 + t.n0, krow, fb);
+                else tma_load_mn128(true, sb, &map_b0, p.b_col0 + t.n0, krow, fb);
+                if (!b_mn_split && t.ncols > 128) {
+                  if (second) tma_load_mn128(true, sb + 16384, &map_b1, p.b_col0 + t.n0 + 128, krow, fb);
+                  else tma_load_mn128(true, sb + 16384, &map_b0, p.b_col0 + t.n0 + 128, krow, fb);
+                }
+              } else {
 #pragma unroll
-              for (int j = 0; j < MMA_N / 64; ++j) {
-                if (64 * j >= t.ncols) continue;
-                if (second) tma_load_2d(sb + j * 8192, &map_b1, p.b_col0 + t.n0 + 64 * j, krow, fb);
-                else tma_load_2d(sb + j * 8192, &map_b0, p.b_col0 + t.n0 + 64 * j, krow, fb);
+                for (int j = 0; j < MMA_N / 64; ++j) {
+                  if ((b_mn_split && j >= b_mn_split) || 64 * j >= t.ncols) continue;
+                  if (second) tma_load_2d(sb + j * 8192, &map_b1, p.b_col0 + t.n0 + 64 * j, krow, fb);
+                  else tma_load_2d(sb + j * 8192, &map_b0, p.b_col0 + t.n0 + 64 * j, krow, fb);
+                }
               }
             }
           }
@@ -1184,6 +1231,19 @@ inline int tc_make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64
   return r == CUDA_SUCCESS ? REVFFN_OK : REVFFN_ERR_CUDA;
 }
 
+// Tensor map of an MN-major bf16 operand ([rows, ld] in memory, rows = K) seen as {64 columns, rows, ld / 64
+// column groups}: a box of 64 x 64 x 2 is 128 columns of 64 K rows, delivered as two 8 KB blocks of 64 columns.
+inline int tc_make_map_mn3d(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t ld) {
+  cuuint64_t dims[3] = {64, rows, ld / 64};
+  cuuint64_t strides[2] = {ld * 2u, 128u};
+  cuuint32_t box[3] = {64, 64, 2};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = tc_state().encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? REVFFN_OK : REVFFN_ERR_CUDA;
+}
+
 // Tensor map of an epilogue output: boxes of 32 rows x 64 bytes (32 bf16 or 16 fp32 columns),
 // 64-byte swizzle.
 inline int tc_make_out_map(CUtensorMap* map, const void* ptr, bool f32, uint64_t inner, uint64_t outer, uint64_t ld) {
@@ -1261,31 +1321,46 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
   P.idesc = (1u << 4) | fmt | ((uint32_t)(p.a_mn_major ? 1 : 0) << 15) |
             ((uint32_t)(p.b_mn_major ? 1 : 0) << 16) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 
+  // 3-D views of the MN-major operands need whole 64-column groups everywhere
+  P.mn3d = (!p.a_mn_major || (p.lda % 64 == 0 && p.a_col0 % 64 == 0)) && (!p.b_mn_major || (p.ldb % 64 == 0 && p.b_col0 % 64 == 0));
   const int groups = p.n_groups > 0 ? p.n_groups : 1;
   CUtensorMap ma, mb0, mb1;
-  // A
-  if (!p.a_mn_major) {
-    // [rows, K]: dense M rows, or the padded row space for GROUP_M
-    int r = tc_make_map(&ma, p.A, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.lda, f8 ? 128 : 64, 128, f8);
-    if (r) return r;
-  } else {
-    // [K rows, lda columns]; K rows = tokens (dense) or the bound on padded rows (GROUP_K)
-    int r = tc_make_map(&ma, p.A, (uint64_t)p.lda, (uint64_t)p.K, (uint64_t)p.lda, 64, 64);
-    if (r) return r;
-  }
-  // B
   const int k_half = (p.concat == CONCAT_K) ? p.K / 2 : p.K;
-  if (!p.b_mn_major) {
-    uint64_t rows = (p.group_mode == GROUP_M) ? (uint64_t)groups * p.N : (uint64_t)p.N;
-    int r = tc_make_map(&mb0, p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, f8 ? 128 : 64, 128, f8);
-    if (r) return r;
-    r = tc_make_map(&mb1, p.B1 ? p.B1 : p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, f8 ? 128 : 64, 128, f8);
-    if (r) return r;
-  } else {
-    uint64_t rows = (p.group_mode == GROUP_M) ? (uint64_t)groups * k_half : (uint64_t)p.K;
-    int r = tc_make_map(&mb0, p.B0, (uint64_t)p.ldb, rows, (uint64_t)p.ldb, 64, 64);
-    if (r) return r;
-    r = tc_make_map(&mb1, p.B1 ? p.B1 : p.B0, (uint64_t)p.ldb, rows, (uint64_t)p.ldb, 64, 64);
+  auto operand_maps = [&](bool mn3d) -> int {
+    // A
+    if (!p.a_mn_major) {
+      // [rows, K]: dense M rows, or the padded row space for GROUP_M
+      int r = tc_make_map(&ma, p.A, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.lda, f8 ? 128 : 64, 128, f8);
+      if (r) return r;
+    } else {
+      // [K rows, lda columns]; K rows = tokens (dense) or the bound on padded rows (GROUP_K)
+      int r = mn3d ? tc_make_map_mn3d(&ma, p.A, (uint64_t)p.K, (uint64_t)p.lda)
+                   : tc_make_map(&ma, p.A, (uint64_t)p.lda, (uint64_t)p.K, (uint64_t)p.lda, 64, 64);
+      if (r) return r;
+    }
+    // B
+    if (!p.b_mn_major) {
+      uint64_t rows = (p.group_mode == GROUP_M) ? (uint64_t)groups * p.N : (uint64_t)p.N;
+      int r = tc_make_map(&mb0, p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, f8 ? 128 : 64, 128, f8);
+      if (r) return r;
+      r = tc_make_map(&mb1, p.B1 ? p.B1 : p.B0, (uint64_t)k_half, rows, (uint64_t)p.ldb, f8 ? 128 : 64, 128, f8);
+      if (r) return r;
+    } else {
+      uint64_t rows = (p.group_mode == GROUP_M) ? (uint64_t)groups * k_half : (uint64_t)p.K;
+      int r = mn3d ? tc_make_map_mn3d(&mb0, p.B0, rows, (uint64_t)p.ldb)
+                   : tc_make_map(&mb0, p.B0, (uint64_t)p.ldb, rows, (uint64_t)p.ldb, 64, 64);
+      if (r) return r;
+      r = mn3d ? tc_make_map_mn3d(&mb1, p.B1 ? p.B1 : p.B0, rows, (uint64_t)p.ldb)
+               : tc_make_map(&mb1, p.B1 ? p.B1 : p.B0, (uint64_t)p.ldb, rows, (uint64_t)p.ldb, 64, 64);
+      if (r) return r;
+    }
+    return REVFFN_OK;
+  };
+  // should the driver not take the 3-D view (its column-group stride is smaller than its row stride), the 64 x 64
+  // boxes of the plain 2-D maps do the same work with twice the loads
+  if (P.mn3d && operand_maps(true) != REVFFN_OK) P.mn3d = 0;
+  if (!P.mn3d) {
+    int r = operand_maps(false);
     if (r) return r;
   }
   // epilogue outputs written through TMA stores
