@@ -257,6 +257,58 @@ def test_backward_reuses_a_saved_evaluation(rv, simt):
         blk.forward(y1, x2, save=True, ws=small)
 
 
+@pytest.mark.parametrize("gating", ["renorm", "softmax_all"])
+def test_all_passes_with_the_second_stream(rv, gating):
+    """From 1024 tokens on, the tensor-core back end puts the router, the shared expert and the weight gradients on
+    a second stream of the library's own: the same parity as everywhere else, at a size the oracle does in full."""
+    cfg = small_cfg(tokens=1300, n_experts=7, top_k=3)
+    w, s = scaled_weights(cfg, 12, 4.0), make_streams(cfg, 12)
+    run_all_passes(rv, cfg, w, s, TOL_BF16, gating=gating)
+
+
+@pytest.mark.parametrize("sgd", [False, True])
+def test_the_second_stream_changes_no_bit(rv, sgd):
+    """Every output of the three passes (recomputing and shared evaluation, gradients or the fused update) with the
+    second stream equals, bit for bit, the output with every launch on the caller's stream; repeated, because a
+    missing ordering between the two streams would show only now and then."""
+    cfg = small_cfg(tokens=2304, n_experts=8, top_k=2, d_model=512, d_expert=256, d_shared=512)
+    w, s = scaled_weights(cfg, 13, 4.0), make_streams(cfg, 13)
+    y1, x2, dy2 = dev(s["y1"]), dev(s["x2"]), dev(s["dy2"])
+
+    def one_round(extra):
+        blk = make_block(cfg, w)              # fresh weights: the fused update changes them
+        out = {}
+        out["y2"] = blk.forward(y1, x2, flags=extra)
+        out["x2r"] = blk.inverse(y1, out["y2"], save=True, flags=rv.FLAG_ROUTER_FOLDED | extra)
+        names = [n for n in rv.UPD_NAMES if n in blk.weights] if sgd else []
+        g = {n: t for n, t in grad_buffers(cfg, w).items() if n not in names}
+        dy1 = torch.zeros_like(y1)
+        if sgd:
+            blk.backward(y1, dy2, dy1, g, reuse=True, flags=extra, sgd=rv.make_sgd(1e-3, names))
+            for n in names:
+                out["W_" + n] = blk.weights[n].clone()
+        else:
+            blk.backward(y1, dy2, dy1, g, reuse=True, flags=extra)
+            dy1b, g2 = torch.zeros_like(y1), grad_buffers(cfg, w)
+            blk.backward(y1, dy2, dy1b, g2, flags=extra)          # recomputing form
+            out["dy1_recomputed"] = dy1b
+            for n, t in g2.items():
+                out["g2_" + n] = t
+        out["dy1"] = dy1
+        for n, t in g.items():
+            out["g_" + n] = t
+        torch.cuda.synchronize()
+        assert blk.status() == 0
+        return out
+
+    ref = one_round(rv.FLAG_SINGLE_STREAM)
+    for _ in range(4):
+        got = one_round(0)
+        assert got.keys() == ref.keys()
+        for n in ref:
+            assert torch.equal(got[n], ref[n]), n
+
+
 @pytest.mark.parametrize("two_streams,tokens", [(False, 500), (True, 500), (True, 2100)])
 def test_host_step_matches_the_device_entry_points(rv, two_streams, tokens):
     """The host-buffer step (copies in, three passes, copies out; optionally with a second stream for the
