@@ -28,10 +28,19 @@
  *     (y1, x2, y2, dy2, dy1) are fp32 [T, h] with row stride ld_stream elements
  *     (h for packed streams, d for views into an interleaved [X1, X2] tensor).
  *   - The caller owns every buffer including the workspace.  The library
- *     allocates no device memory, creates no streams and never synchronises,
- *     except revffn_moe_status, which synchronises the given stream.
- *   - All kernels are enqueued on the caller's CUDA stream (cudaStream_t passed
- *     as void*).  Calls that share a workspace must be ordered on one stream.
+ *     allocates no device memory and never synchronises, except
+ *     revffn_moe_status, which synchronises the given stream.
+ *   - Work is enqueued on the caller's CUDA stream (cudaStream_t passed as
+ *     void*), and the call is asynchronous on it: what the caller queues on that
+ *     stream afterwards follows everything of the call.  Inside a call of 1024
+ *     tokens or more on the tcgen05 back end, launches that nothing later in the
+ *     pass depends on run on a second stream that the library creates per device
+ *     on its first such call (with a ring of events that order it against the
+ *     caller's stream); REVFFN_FLAG_SINGLE_STREAM keeps every launch on the
+ *     caller's stream.  The results are the same bits either way.  The pipelined
+ *     host step (REVFFN_FLAG_STEP_PIPELINED) owns one more stream, for uploads.
+ *     Calls that share a workspace must be ordered on one stream, and calls on
+ *     one device must not be made from two host threads at once.
  *   - Return value: REVFFN_OK (0) or a negative revffn_error.  On an error
  *     return nothing has been launched.  Device-side problems (a bounded wait
  *     that expired, an expert index out of range) set a status word in the
