@@ -91,6 +91,9 @@ typedef struct {
   int32_t starve_operands;
   /* measurements: operand loads issued by two threads (1) or by one (2); 0 = the library's choice per epilogue */
   int32_t split_loads;
+  /* tests: 1 = load MN-major operands as 64 x 64 boxes of 2-D tensor maps, the form the library falls back to when a
+   * leading dimension or column offset is not a multiple of 64 (0 = 3-D maps, 128 columns per load, where possible) */
+  int32_t mn_boxes;
 } revffn_dbg_gemm_args;
 int revffn_dbg_gemm(const revffn_dbg_gemm_args* args, int32_t* status_word_dev, void* cuda_stream);
 

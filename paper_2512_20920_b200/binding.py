@@ -112,7 +112,7 @@ class DbgGemmArgs(C.Structure):
                 ("group_off", C.c_void_p), ("tile_group", C.c_void_p), ("rows_total", C.c_void_p),
                 ("b_group_stride", C.c_int64), ("c_group_stride", C.c_int64), ("a_col0", C.c_int32),
                 ("b_col0", C.c_int32), ("tok_chunks", C.c_void_p), ("no_pair", C.c_int32),
-                ("wait_cycles", C.c_int64), ("starve_operands", C.c_int32), ("split_loads", C.c_int32)]
+                ("wait_cycles", C.c_int64), ("starve_operands", C.c_int32), ("split_loads", C.c_int32), ("mn_boxes", C.c_int32)]
 
 
 def _load() -> C.CDLL:

@@ -75,6 +75,7 @@ struct GemmProblem {
   long long dbg_wait_cycles;   // tcgen05 back end, tests: bound on every device-side wait (0 = default)
   int dbg_starve;              // tcgen05 back end, tests (needs no_pair): no operand loads are issued
   int dbg_split_loads;         // tcgen05 back end, measurements: 0 the kernel's own choice, 1 two load threads, 2 one
+  int dbg_mn_boxes;            // tcgen05 back end, tests: MN-major operands through 64 x 64 boxes of 2-D maps (the fallback form)
   // EPI_HEADS (tcgen05 back end, dense products only): the N columns are heads of 128; C receives, head-major
   // [sequence, head, hm_Sp, 128], the product plus hm_bias, with the pairs (i, i + 64) of a head turned by the
   // angle of hm_cs[position, i] (cos, sin) when hm_cs is given.  Row m is position m % hm_S of sequence m / hm_S.

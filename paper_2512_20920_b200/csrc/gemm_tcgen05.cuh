@@ -1322,7 +1322,7 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
             ((uint32_t)(p.b_mn_major ? 1 : 0) << 16) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 
   // 3-D views of the MN-major operands need whole 64-column groups everywhere
-  P.mn3d = (!p.a_mn_major || (p.lda % 64 == 0 && p.a_col0 % 64 == 0)) && (!p.b_mn_major || (p.ldb % 64 == 0 && p.b_col0 % 64 == 0));
+  P.mn3d = !p.dbg_mn_boxes && (!p.a_mn_major || (p.lda % 64 == 0 && p.a_col0 % 64 == 0)) && (!p.b_mn_major || (p.ldb % 64 == 0 && p.b_col0 % 64 == 0));
   const int groups = p.n_groups > 0 ? p.n_groups : 1;
   CUtensorMap ma, mb0, mb1;
   const int k_half = (p.concat == CONCAT_K) ? p.K / 2 : p.K;

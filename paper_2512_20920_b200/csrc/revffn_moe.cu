@@ -1527,7 +1527,7 @@ int revffn_dbg_gemm(const revffn_dbg_gemm_args* a, int32_t* status_word_dev, voi
   p.b_group_stride = a->b_group_stride; p.c_group_stride = a->c_group_stride;
   p.a_col0 = a->a_col0; p.b_col0 = a->b_col0;
   p.tok_chunks = reinterpret_cast<const int4*>(a->tok_chunks); p.no_pair = a->no_pair;
-  p.dbg_wait_cycles = a->wait_cycles; p.dbg_starve = a->starve_operands; p.dbg_split_loads = a->split_loads;
+  p.dbg_wait_cycles = a->wait_cycles; p.dbg_starve = a->starve_operands; p.dbg_split_loads = a->split_loads; p.dbg_mn_boxes = a->mn_boxes;
   p.status = status_word_dev;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (a->use_simt) return launch_gemm_simt<bf16>(p, st) == cudaSuccess ? REVFFN_OK : REVFFN_ERR_CUDA;

@@ -277,3 +277,66 @@ def test_grouped_rows_with_tokens_on_the_mma_n_side(rv, counts):
         if c:
             a = A2[off[e]: off[e] + c].float()
             _close(Ct[off[e]: off[e] + c], a[:, :Kh] @ W0[e].float() + a[:, Kh:] @ W1[e].float())
+
+
+def test_load_forms_give_the_same_bits(rv):
+    """The operand loads have two switches that must not change a result: one or two load threads, and MN-major
+    operands through 3-D tensor maps (128 columns per load) or through 64 x 64 boxes of 2-D maps (the form the
+    library falls back to when a leading dimension is not a multiple of 64).  Every product shape with an
+    MN-major operand, in all four combinations, against the default."""
+    counts = [130, 0, 5, 300, 64]
+    E = len(counts)
+    off, tile_group = _groups(counts)
+    rows = off[-1]
+    ch = _chunks(counts, off)
+    g_off = torch.tensor(off, dtype=torch.int32, device="cuda")
+    g_tile = torch.tensor(tile_group + [0] * 8, dtype=torch.int32, device="cuda")
+    g_total = torch.tensor([rows, len(ch)], dtype=torch.int32, device="cuda")
+    g_ch = torch.tensor(ch + [[0, 0, 0, 0]], dtype=torch.int32, device="cuda")
+    K, N = 256, 384                                     # N = 384: the last column tile is 128 wide
+    X = torch.zeros(rows, K, device="cuda", dtype=torch.bfloat16)
+    for e, c in enumerate(counts):
+        X[off[e]: off[e] + c] = _bf((c, K), 70 + e)
+    Wkn = _bf((E, K, N), 80, 0.3)                       # weights stored [K, N]
+    G = torch.zeros(rows, N, device="cuda", dtype=torch.bfloat16)
+    for e, c in enumerate(counts):
+        G[off[e]: off[e] + c] = _bf((c, N), 90 + e)
+    Kh = 128
+    W0, W1 = _bf((E, Kh, N), 60, 0.3), _bf((E, Kh, N), 61, 0.3)
+    Ad, Bd = _bf((1000, 256 + 128), 5), _bf((1000, N + 128), 6)
+
+    def products(**dbg):
+        out = {}
+        # row-tiled experts, B [K, N] (the shape of dH = dO W_down)
+        out["rows"] = torch.zeros(rows, N, device="cuda", dtype=torch.bfloat16)
+        _call(rv, False, M=rows, N=N, K=K, A=X, B0=Wkn, lda=K, ldb=N, b_mn_major=1, C=out["rows"], ldc=N, epilogue=EPI["store"],
+              group_mode=1, n_groups=E, group_off=g_off, tile_group=g_tile, rows_total=g_total, b_group_stride=K * N, **dbg)
+        # transposed pair mode, K concatenation of two [K, N] weights (the shape of dU = da W_g + db W_u)
+        out["tr"] = torch.zeros(rows, N, device="cuda", dtype=torch.bfloat16)
+        _call(rv, False, M=rows, N=N, K=2 * Kh, A=X, B0=W0, B1=W1, lda=K, ldb=N, b_mn_major=1, concat=2, C=out["tr"], ldc=N,
+              epilogue=EPI["store"], group_mode=1, n_groups=E, group_off=g_off, tile_group=g_tile, rows_total=g_total,
+              b_group_stride=Kh * N, tok_chunks=g_ch, **dbg)
+        # K-grouped weight gradient, both operands MN-major
+        out["wgrad"] = torch.zeros(E, K, N, device="cuda")
+        _call(rv, False, M=K, N=N, K=rows, A=X, B0=G, lda=K, ldb=N, a_mn_major=1, b_mn_major=1, C=out["wgrad"], ldc=N,
+              epilogue=EPI["wgrad"], group_mode=2, n_groups=E, group_off=g_off, c_group_stride=K * N, **dbg)
+        # dense weight gradient from column windows of wider buffers, ragged K
+        out["dense"] = torch.zeros(256, N, device="cuda")
+        _call(rv, False, M=256, N=N, K=1000, A=Ad, B0=Bd, lda=256 + 128, ldb=N + 128, a_mn_major=1, b_mn_major=1, a_col0=128,
+              b_col0=128, C=out["dense"], ldc=N, epilogue=EPI["wgrad"], **dbg)
+        # dense product with B [K, N]
+        out["store"] = torch.zeros(1000, N, device="cuda", dtype=torch.bfloat16)
+        _call(rv, False, M=1000, N=N, K=256 + 128, A=Ad, B0=Wkn[0].contiguous().repeat(2, 1)[:256 + 128].contiguous(), lda=256 + 128,
+              ldb=N, b_mn_major=1, C=out["store"], ldc=N, epilogue=EPI["store"], **dbg)
+        return out
+
+    ref = products()
+    _close(ref["dense"], Ad[:, 128:].float().T @ Bd[:, 128:].float(), 1e-5)
+    for e, c in enumerate(counts):
+        if c:
+            _close(ref["rows"][off[e]: off[e] + c], X[off[e]: off[e] + c].float() @ Wkn[e].float())
+    for split in (1, 2):
+        for boxes in (0, 1):
+            got = products(split_loads=split, mn_boxes=boxes)
+            for n in ref:
+                assert torch.equal(got[n], ref[n]), (n, split, boxes)
