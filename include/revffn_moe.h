@@ -297,6 +297,34 @@ int revffn_moe_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weight
                             void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The same fusion with Adam (decoupled weight decay) as the rule.  (The paper names no optimiser for its method;
+ * this is the second reading of "the update applied where the gradient is produced", for callers that train
+ * with moment estimates.)  Per element of every matrix in the mask, with g the gradient the product has just
+ * accumulated, all in fp32:
+ *     m <- beta1 m + (1 - beta1) g          v <- beta2 v + (1 - beta2) g^2
+ *     W <- W - lr ( (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps) + weight_decay W )
+ * mom[i] / var[i] (fp32, shape of matrix i, 16-byte aligned, caller-owned, zero before the first step) are read
+ * and rewritten in the same epilogue; master[i] is the optional fp32 copy of the weight as in revffn_moe_sgd.
+ * Index i is the position of the matrix's REVFFN_UPD_* bit (w_up 0, w_down 1, w_gate 2, w_upx 3, w_downx 4,
+ * ws_gate 5, ws_up 6, ws_down 7).  step >= 1 is the caller's step counter.  Everything else (mask rules, which
+ * gradients are still written, ordering of reads and updates) is as for revffn_moe_backward_sgd.  The moments
+ * add 16 bytes of traffic per element to the 4 of the weight: the fused form saves the gradient's 8 (write, then
+ * read by a separate optimiser pass), not the moments'.
+ */
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay;
+  int32_t step;
+  uint32_t mask;          /* REVFFN_UPD_* bits                                              */
+  float* mom[8];          /* first moments, by bit position                                 */
+  float* var[8];          /* second moments                                                 */
+  float* master[8];       /* fp32 master copies or NULL                                     */
+} revffn_moe_adam;
+int revffn_moe_backward_adam(const revffn_moe_desc* desc, const revffn_moe_weights* w,
+                             const float* y1, const float* dy2, float* dy1_inout,
+                             const revffn_moe_grads* grads, const revffn_moe_adam* adam, const int32_t* topk_idx_in,
+                             void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Quantise the bf16 expert weights for REVFFN_FLAG_FP8_EXPERTS: per output row r of w_gate / w_upx ([E*I] rows of
  * d) and of w_downx ([E*d] rows of I), scale[r] = max|row| / 448 (1 for an all-zero row) and
  * code = e4m3(w * (1 / scale[r])), every step a correctly rounded fp32 operation, round to nearest even,

@@ -377,6 +377,26 @@ def sgd_step(p, grads, lr: float, names):
     return out
 
 
+def adam_step(p, grads, mom, var, lr: float, step: int, names, beta1: float = 0.9, beta2: float = 0.999,
+              eps: float = 1e-8, weight_decay: float = 0.0):
+    """One Adam step with decoupled weight decay on the named weights (fp64), written out from the rule's
+    definition: m <- b1 m + (1 - b1) g;  v <- b2 v + (1 - b2) g^2;  m^ = m / (1 - b1^t);  v^ = v / (1 - b2^t);
+    W <- W - lr (m^ / (sqrt(v^) + eps) + weight_decay W).  mom / var: dicts of the moment estimates before the
+    step (missing = zeros).  Returns (weights, mom, var) after it.  (The paper names no optimiser for its method:
+    this is the moment-based reading of the fused update, beside sgd_step.)"""
+    out, m_out, v_out = dict(p), dict(mom), dict(var)
+    for n in names:
+        g = np.asarray(grads[n], dtype=F64)
+        w = _w(p, n)
+        m = beta1 * np.asarray(mom.get(n, 0.0), dtype=F64) + (1.0 - beta1) * g
+        v = beta2 * np.asarray(var.get(n, 0.0), dtype=F64) + (1.0 - beta2) * g * g
+        m_hat = m / (1.0 - beta1 ** step)
+        v_hat = v / (1.0 - beta2 ** step)
+        out[n] = w - lr * (m_hat / (np.sqrt(v_hat) + eps) + weight_decay * w)
+        m_out[n], v_out[n] = m, v
+    return out, m_out, v_out
+
+
 # --------------------------------------------------------------------------- #
 # A stack of coupling branches (Sec. 3.1: the two output streams of a layer are
 # the input of the next one; Sec. 2: inputs are rebuilt layer by layer from the

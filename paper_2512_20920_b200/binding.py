@@ -79,6 +79,28 @@ def make_sgd(lr: float, names, masters: Optional[Dict[str, torch.Tensor]] = None
     return Sgd(lr=lr, mask=upd_mask(names), **{"m_" + n: _ptr(masters.get(n)) for n in UPD_NAMES})
 
 
+class Adam(C.Structure):
+    """revffn_moe_adam: the rule's constants, the caller's step counter, mask, moment buffers and optional fp32
+    master copies (arrays indexed by the position of the matrix in UPD_NAMES)."""
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float), ("step", C.c_int32), ("mask", C.c_uint32), ("mom", C.c_void_p * 8),
+                ("var", C.c_void_p * 8), ("master", C.c_void_p * 8)]
+
+
+def make_adam(lr: float, step: int, names, mom: Dict[str, torch.Tensor], var: Dict[str, torch.Tensor],
+              masters: Optional[Dict[str, torch.Tensor]] = None, beta1: float = 0.9, beta2: float = 0.999,
+              eps: float = 1e-8, weight_decay: float = 0.0) -> Adam:
+    masters = masters or {}
+    for d in (mom, var, masters):
+        for n, t in d.items():
+            if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+                raise ValueError(f"{n}: need a contiguous fp32 CUDA tensor")
+    a = Adam(lr=lr, beta1=beta1, beta2=beta2, eps=eps, weight_decay=weight_decay, step=step, mask=upd_mask(names))
+    for i, n in enumerate(UPD_NAMES):
+        a.mom[i], a.var[i], a.master[i] = _ptr(mom.get(n)), _ptr(var.get(n)), _ptr(masters.get(n))
+    return a
+
+
 ATTN_WEIGHT_NAMES = ("norm_gamma", "w_up", "w_down", "w_q", "w_k", "w_v", "w_o", "b_q", "b_k", "b_v")
 _ATTN_F32_ALWAYS = ("norm_gamma", "b_q", "b_k", "b_v")
 
@@ -129,6 +151,9 @@ def _load() -> C.CDLL:
     lib.revffn_moe_backward_sgd.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, C.POINTER(Grads), C.POINTER(Sgd),
                                             vp, vp, sz, vp]
     lib.revffn_moe_backward_sgd.restype = C.c_int
+    lib.revffn_moe_backward_adam.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp, vp, vp, C.POINTER(Grads), C.POINTER(Adam),
+                                             vp, vp, sz, vp]
+    lib.revffn_moe_backward_adam.restype = C.c_int
     lib.revffn_moe_stack_backward_sgd.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp,
                                                   C.POINTER(Grads), C.POINTER(Sgd), vp, vp, sz, vp, sz, vp]
     lib.revffn_moe_stack_backward_sgd.restype = C.c_int
@@ -242,6 +267,14 @@ def revffn_moe_backward_sgd(desc: Desc, w: Weights, y1, dy2, dy1_inout, grads: G
                                        C.byref(sgd), _ptr(topk_idx_in), _ptr(ws), ws.numel() * ws.element_size(),
                                        stream if stream is not None else _stream()),
            "revffn_moe_backward_sgd")
+
+
+def revffn_moe_backward_adam(desc: Desc, w: Weights, y1, dy2, dy1_inout, grads: Grads, adam: Adam, topk_idx_in, ws,
+                             stream: Optional[int] = None):
+    _check(lib.revffn_moe_backward_adam(C.byref(desc), C.byref(w), _ptr(y1), _ptr(dy2), _ptr(dy1_inout), C.byref(grads),
+                                        C.byref(adam), _ptr(topk_idx_in), _ptr(ws), ws.numel() * ws.element_size(),
+                                        stream if stream is not None else _stream()),
+           "revffn_moe_backward_adam")
 
 
 def revffn_moe_status(ws, stream: Optional[int] = None) -> int:
@@ -432,15 +465,17 @@ class Block:
     def backward(self, y1, dy2, dy1_inout, grads: Optional[Dict[str, torch.Tensor]] = None, accumulate: bool = False,
                  topk_idx_in=None, reuse: bool = False, ws=None, flags: int = 0, sgd: Optional[Sgd] = None):
         """reuse=True: the workspace still holds what forward/inverse(save=True) left for this y1.
-        sgd: a Sgd struct (make_sgd) -- the matrices in its mask are updated in place instead of having their
-        gradients written (revffn_moe_backward_sgd)."""
+        sgd: a Sgd struct (make_sgd) or an Adam struct (make_adam) -- the matrices in its mask are updated in place
+        instead of having their gradients written (revffn_moe_backward_sgd / revffn_moe_backward_adam)."""
         grads = grads or {}
         for n, t in grads.items():
             if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
                 raise ValueError(f"gradient {n}: need a contiguous fp32 CUDA tensor")
         g = Grads(**{n: _ptr(grads.get(n)) for n in WEIGHT_NAMES}, accumulate=1 if accumulate else 0)
         d = self._desc((FLAG_REUSE_ACTIVATIONS if reuse else 0) | flags)
-        if sgd is not None:
+        if isinstance(sgd, Adam):
+            revffn_moe_backward_adam(d, self.w, y1, dy2, dy1_inout, g, sgd, topk_idx_in, self.ws if ws is None else ws)
+        elif sgd is not None:
             revffn_moe_backward_sgd(d, self.w, y1, dy2, dy1_inout, g, sgd, topk_idx_in, self.ws if ws is None else ws)
         else:
             revffn_moe_backward(d, self.w, y1, dy2, dy1_inout, g, topk_idx_in, self.ws if ws is None else ws)

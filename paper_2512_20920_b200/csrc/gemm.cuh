@@ -38,6 +38,21 @@ enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_ROWSCALE = 2, EPI_COUPLE = 3, EPI_DSWI
 enum { CONCAT_NONE = 0, CONCAT_N = 1, CONCAT_K = 2 };
 enum { GROUP_NONE = 0, GROUP_M = 1, GROUP_K = 2 };
 
+// Update rule of a fused optimiser step (EPI_WGRAD with upd_w set).  kind 0: W <- W - lr g.  kind 1: Adam with
+// decoupled weight decay, m <- b1 m + (1 - b1) g, v <- b2 v + (1 - b2) g^2,
+// W <- W - lr (m / c1 / (sqrt(v / c2) + eps) + wd W), c1 = 1 - b1^t, c2 = 1 - b2^t.
+struct UpdRule { int kind; float lr, b1, b2, eps, c1, c2, wd; };
+
+// One element of the step: returns the new weight; for Adam also rewrites the element's two moments.
+__device__ __forceinline__ float upd_step(const UpdRule& r, float w, float g, float* mom, float* var) {
+  if (r.kind == 0) return w - r.lr * g;
+  const float m = r.b1 * *mom + (1.f - r.b1) * g;
+  const float v = r.b2 * *var + (1.f - r.b2) * g * g;
+  *mom = m;
+  *var = v;
+  return w - r.lr * ((m / r.c1) / (sqrtf(v / r.c2) + r.eps) + r.wd * w);
+}
+
 struct GemmProblem {
   int M, N, K;
   int a_mn_major, b_mn_major;
@@ -66,7 +81,10 @@ struct GemmProblem {
   // EPI_WGRAD, fused SGD step: instead of writing the gradient g to C, update the weight it belongs to in place,
   // W <- W - upd_lr * g (W of the operand type, same layout as C; upd_w2 goes with C2's rows).  With a master
   // copy (fp32, same layout) the step is taken there and W receives the rounded result.  C / C2 may then be NULL.
-  void* upd_w; void* upd_w2; float* upd_m; float* upd_m2; float upd_lr;
+  // upd.kind 1 (Adam): upd_mom / upd_var (fp32, same layout, and their second-output twins) hold the moment
+  // estimates, which are updated in place as well.
+  void* upd_w; void* upd_w2; float* upd_m; float* upd_m2; UpdRule upd;
+  float* upd_mom; float* upd_mom2; float* upd_var; float* upd_var2;
   // tcgen05 back end, fp8 operands (both K-major): A and B hold e4m3 codes, one byte per element; the accumulator
   // is multiplied by a_scale[row] * b_scale[(group * N +) column] before the epilogue's own arithmetic
   // (b_scale1: the second matrix of an N-concatenated pair).  lda / ldb / K count elements (= bytes).
@@ -111,7 +129,8 @@ __host__ __device__ inline int64_t split_k_rows(int64_t K, int n) { return round
 // fused SGD step on the weight (and its master copy).
 template <typename T>
 __global__ void splitk_reduce_kernel(const float* __restrict__ part, int n, int64_t count, float* __restrict__ out,
-                                     int accumulate, T* __restrict__ W, float* __restrict__ master, float lr) {
+                                     int accumulate, T* __restrict__ W, float* __restrict__ master, UpdRule rule,
+                                     float* __restrict__ mom, float* __restrict__ var) {
   const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= count) return;
   float4 v = *reinterpret_cast<const float4*>(part + i);
@@ -123,7 +142,9 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int n, int6
     float w[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) w[j] = master ? master[i + j] : to_f32(W[i + j]);
-    w[0] -= lr * v.x; w[1] -= lr * v.y; w[2] -= lr * v.z; w[3] -= lr * v.w;
+    const float g[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) w[j] = upd_step(rule, w[j], g[j], mom ? mom + i + j : nullptr, var ? var + i + j : nullptr);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       if (master) master[i + j] = w[j];
@@ -284,7 +305,10 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmProblem p) {
           T* W = reinterpret_cast<T*>(second ? p.upd_w2 : p.upd_w);
           if (W) {
             float* master = second ? p.upd_m2 : p.upd_m;
-            const float w_new = (master ? master[at] : to_f32(W[at])) - p.upd_lr * v;
+            float* mom = second ? p.upd_mom2 : p.upd_mom;
+            float* var = second ? p.upd_var2 : p.upd_var;
+            const float w_new = upd_step(p.upd, master ? master[at] : to_f32(W[at]), v, mom ? mom + at : nullptr,
+                                         var ? var + at : nullptr);
             if (master) master[at] = w_new;
             W[at] = from_f32<T>(w_new);
           } else {

@@ -877,12 +877,15 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
             float* cptr = reinterpret_cast<float*>(p.C);
             bf16* wptr = reinterpret_cast<bf16*>(p.upd_w);
             float* mptr = p.upd_m;
+            float* momptr = p.upd_mom;
+            float* varptr = p.upd_var;
             if (EPI == EPI_WGRAD && p.split_m > 0) {
               // two outputs: the slab lies wholly in the first or in the second (split_m is a multiple of 128)
               int local = t.m0 + q * 32;
               if (local >= p.split_m) {
                 local -= p.split_m;
                 cptr = reinterpret_cast<float*>(p.C2); wptr = reinterpret_cast<bf16*>(p.upd_w2); mptr = p.upd_m2;
+                momptr = p.upd_mom2; varptr = p.upd_var2;
               }
               yb = (int64_t)t.group * p.split_m + local;
               y_lim = (int64_t)(t.group + 1) * p.split_m;
@@ -905,7 +908,19 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
                     const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
                     wv = make_float4(lo.x, lo.y, hi.x, hi.y);
                   }
-                  wv.x -= p.upd_lr * v.x; wv.y -= p.upd_lr * v.y; wv.z -= p.upd_lr * v.z; wv.w -= p.upd_lr * v.w;
+                  if (p.upd.kind == 0) {
+                    wv.x -= p.upd.lr * v.x; wv.y -= p.upd.lr * v.y; wv.z -= p.upd.lr * v.z; wv.w -= p.upd.lr * v.w;
+                  } else {
+                    // Adam: the element's two moments live beside the weight (fp32, same layout): 16 bytes each per lane
+                    float4 mo = *reinterpret_cast<const float4*>(momptr + at);
+                    float4 va = *reinterpret_cast<const float4*>(varptr + at);
+                    wv.x = upd_step(p.upd, wv.x, v.x, &mo.x, &va.x);
+                    wv.y = upd_step(p.upd, wv.y, v.y, &mo.y, &va.y);
+                    wv.z = upd_step(p.upd, wv.z, v.z, &mo.z, &va.z);
+                    wv.w = upd_step(p.upd, wv.w, v.w, &mo.w, &va.w);
+                    *reinterpret_cast<float4*>(momptr + at) = mo;
+                    *reinterpret_cast<float4*>(varptr + at) = va;
+                  }
                   if (mptr) *reinterpret_cast<float4*>(mptr + at) = wv;
                   uint2 out;
                   __nv_bfloat162 h2 = __floats2bfloat162_rn(wv.x, wv.y);
@@ -1388,9 +1403,12 @@ inline int launch_gemm_tc(const GemmProblem& p, cudaStream_t st) {
     if (p.epilogue == EPI_WGRAD && p.upd_w) {
       // fused update: the weights (and master copies) are read and rewritten 8 / 16 bytes at a time
       if ((reinterpret_cast<uintptr_t>(p.upd_w) & 15u) || (reinterpret_cast<uintptr_t>(p.upd_w2) & 15u) ||
-          (reinterpret_cast<uintptr_t>(p.upd_m) & 15u) || (reinterpret_cast<uintptr_t>(p.upd_m2) & 15u) || p.ldc % 4 != 0)
+          (reinterpret_cast<uintptr_t>(p.upd_m) & 15u) || (reinterpret_cast<uintptr_t>(p.upd_m2) & 15u) ||
+          (reinterpret_cast<uintptr_t>(p.upd_mom) & 15u) || (reinterpret_cast<uintptr_t>(p.upd_mom2) & 15u) ||
+          (reinterpret_cast<uintptr_t>(p.upd_var) & 15u) || (reinterpret_cast<uintptr_t>(p.upd_var2) & 15u) || p.ldc % 4 != 0)
         return REVFFN_ERR_ALIGN;
       if (p.split_m > 0 && !p.upd_w2) return REVFFN_ERR_NULL;
+      if (p.upd.kind == 1 && (!p.upd_mom || !p.upd_var || (p.split_m > 0 && (!p.upd_mom2 || !p.upd_var2)))) return REVFFN_ERR_NULL;
     } else {
       if (!p.C || (p.split_m > 0 && !p.C2)) return REVFFN_ERR_NULL;
       if ((reinterpret_cast<uintptr_t>(p.C) & 15u) || (reinterpret_cast<uintptr_t>(p.C2) & 15u) || (p.ldc * (f32_out ? 4 : 2)) % 16 != 0)

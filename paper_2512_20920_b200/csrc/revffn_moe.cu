@@ -3,6 +3,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -610,9 +611,43 @@ static int run_couple(const Ctx<T>& c, const float* resid, float sign, float* ou
   return run_gemm(c, p, TG_PDOWN);
 }
 
+// A fused optimiser step as the gradient pass sees it: which matrices (REVFFN_UPD_* bits, bit i = entry i of the
+// arrays), the rule, and per matrix the optional fp32 master copy and, for Adam, the two moment buffers.
+struct UpdateSpec {
+  uint32_t mask = 0;
+  UpdRule rule = {};
+  float* master[8] = {};
+  float* mom[8] = {};
+  float* var[8] = {};
+};
+
+static UpdateSpec spec_from_sgd(const revffn_moe_sgd& s) {
+  UpdateSpec u;
+  u.mask = s.mask;
+  u.rule.kind = 0;
+  u.rule.lr = s.lr;
+  float* m[8] = {s.m_w_up, s.m_w_down, s.m_w_gate, s.m_w_upx, s.m_w_downx, s.m_ws_gate, s.m_ws_up, s.m_ws_down};
+  for (int i = 0; i < 8; ++i) u.master[i] = m[i];
+  return u;
+}
+
+static int spec_from_adam(const revffn_moe_adam& a, UpdateSpec* u) {
+  if (a.step < 1 || !(a.beta1 >= 0.f && a.beta1 < 1.f) || !(a.beta2 >= 0.f && a.beta2 < 1.f) || !(a.eps > 0.f)) return REVFFN_ERR_SHAPE;
+  u->mask = a.mask;
+  u->rule.kind = 1;
+  u->rule.lr = a.lr; u->rule.b1 = a.beta1; u->rule.b2 = a.beta2; u->rule.eps = a.eps; u->rule.wd = a.weight_decay;
+  u->rule.c1 = (float)(1.0 - pow((double)a.beta1, (double)a.step));
+  u->rule.c2 = (float)(1.0 - pow((double)a.beta2, (double)a.step));
+  for (int i = 0; i < 8; ++i) {
+    u->master[i] = a.master[i]; u->mom[i] = a.mom[i]; u->var[i] = a.var[i];
+    if ((a.mask & (1u << i)) && (!a.mom[i] || !a.var[i])) return REVFFN_ERR_NULL;
+  }
+  return REVFFN_OK;
+}
+
 template <typename T>
 static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, float* dy1, const revffn_moe_grads& G,
-                        const revffn_moe_sgd* sgd, const int32_t* idx_in) {
+                        const UpdateSpec* sgd, const int32_t* idx_in) {
   const revffn_moe_desc& D = c.D;
   const WsLayout& L = c.L;
   const int Tn = D.tokens, d = D.d_model, h = d / 2, E = D.n_experts, k = D.top_k, I = D.d_expert, Is = D.d_shared;
@@ -634,6 +669,8 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
                    const void* W2 = nullptr, float* master2 = nullptr) -> int {
     const bool upd = (upd_mask & bit) != 0;
     if (!upd && !out) return REVFFN_OK;      // frozen: neither gradient nor update wanted
+    int wi = 0;                              // index of this matrix in the update's arrays
+    while (wi < 7 && !((bit >> wi) & 1u)) ++wi;
     // Nothing later in this pass reads a weight gradient (or an updated weight): the product goes to the second
     // stream, after everything queued so far (its operands, and every product that reads the weight it may update).
     CKR(c.order(st, cw.st));
@@ -645,8 +682,10 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     p.epilogue = EPI_WGRAD; p.accumulate = acc;
     p.ldc = N; p.c_group_stride = cstride;
     if (upd) {
-      p.upd_w = const_cast<void*>(W); p.upd_m = master; p.upd_lr = sgd->lr;
+      p.upd_w = const_cast<void*>(W); p.upd_m = master; p.upd = sgd->rule;
       p.upd_w2 = const_cast<void*>(W2); p.upd_m2 = master2;
+      p.upd_mom = sgd->mom[wi]; p.upd_var = sgd->var[wi];
+      if (W2) { p.upd_mom2 = sgd->mom[wi + 1]; p.upd_var2 = sgd->var[wi + 1]; }    // gate | up: neighbouring bits
     } else {
       p.C = out; p.C2 = out2;
     }
@@ -672,20 +711,22 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     if (n_split <= 1) return run_gemm(cw, p, tag);
     p.group_mode = GROUP_K; p.n_groups = n_split; p.group_off = nullptr;
     p.C = c.template p<float>(L.ksplit); p.C2 = nullptr; p.c_group_stride = (int64_t)M * N; p.accumulate = 0;
-    p.upd_w = nullptr; p.upd_m = nullptr;
+    p.upd_w = nullptr; p.upd_m = nullptr; p.upd_mom = nullptr; p.upd_var = nullptr;
     CKR(run_gemm(cw, p, tag));
     {
       ProfScope ps(tag, cw.st);
       const int64_t count = (int64_t)M * N;
       splitk_reduce_kernel<T><<<(unsigned)ceil_div(count, 4 * 256), 256, 0, cw.st>>>(
           c.template p<float>(L.ksplit), n_split, count, out, acc, upd ? reinterpret_cast<T*>(const_cast<void*>(W)) : nullptr,
-          upd ? master : nullptr, upd ? sgd->lr : 0.f);
+          upd ? master : nullptr, upd ? sgd->rule : UpdRule{}, upd ? sgd->mom[wi] : nullptr, upd ? sgd->var[wi] : nullptr);
     }
     CK(cudaGetLastError());
     return REVFFN_OK;
   };
-  const revffn_moe_sgd no_sgd = {};
-  const revffn_moe_sgd& S = sgd ? *sgd : no_sgd;
+  struct Masters { float *m_w_up, *m_w_down, *m_w_gate, *m_w_upx, *m_w_downx, *m_ws_gate, *m_ws_up, *m_ws_down; };
+  const Masters S = sgd ? Masters{sgd->master[0], sgd->master[1], sgd->master[2], sgd->master[3], sgd->master[4],
+                                  sgd->master[5], sgd->master[6], sgd->master[7]}
+                        : Masters{};
 
   // P_down backward: dZ = G W_down;  dW_down = G^T Z
   { ProfScope ps(TG_CAST, st);
@@ -909,7 +950,7 @@ enum Pass { PASS_FWD, PASS_INV, PASS_BWD };
 template <typename T>
 static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weights& W, const WsLayout& L, void* ws,
                     cudaStream_t st, const float* y1, const float* in2, float* out, const revffn_moe_grads* G,
-                    const revffn_moe_sgd* sgd, const int32_t* idx_in, int32_t* idx_out) {
+                    const UpdateSpec* sgd, const int32_t* idx_in, int32_t* idx_out) {
   Ctx<T> c;
   c.D = D; c.W = W; c.L = L; c.ws = reinterpret_cast<char*>(ws); c.st = st;
   g_prof.pass = (int)pass;
@@ -938,7 +979,7 @@ static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weight
 
 static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1,
                  const float* in2, float* out, const revffn_moe_grads* grads, const int32_t* idx_in,
-                 int32_t* idx_out, void* ws, size_t ws_bytes, void* cuda_stream, const revffn_moe_sgd* sgd = nullptr) {
+                 int32_t* idx_out, void* ws, size_t ws_bytes, void* cuda_stream, const UpdateSpec* sgd = nullptr) {
   CKR(validate_desc(desc));
   CKR(validate_weights(*desc, w));
   if (!ws) return REVFFN_ERR_NULL;
@@ -953,10 +994,8 @@ static int entry(Pass pass, const revffn_moe_desc* desc, const revffn_moe_weight
   if (sgd) {
     if (sgd->mask & ~REVFFN_UPD_ALL) return REVFFN_ERR_SHAPE;
     if (desc->d_shared == 0 && (sgd->mask & (REVFFN_UPD_WS_GATE | REVFFN_UPD_WS_UP | REVFFN_UPD_WS_DOWN))) return REVFFN_ERR_NULL;
-    const float* ms[] = {sgd->m_w_up, sgd->m_w_down, sgd->m_w_gate, sgd->m_w_upx, sgd->m_w_downx, sgd->m_ws_gate,
-                         sgd->m_ws_up, sgd->m_ws_down};
-    for (const float* m : ms)
-      if (m && !aligned16(m)) return REVFFN_ERR_ALIGN;
+    for (int i = 0; i < 8; ++i)
+      if (!aligned16(sgd->master[i]) || !aligned16(sgd->mom[i]) || !aligned16(sgd->var[i])) return REVFFN_ERR_ALIGN;
     // a weight is either updated in place or has its gradient written, not both
     const float* gs8[] = {grads->w_up, grads->w_down, grads->w_gate, grads->w_upx, grads->w_downx, grads->ws_gate,
                           grads->ws_up, grads->ws_down};
@@ -1052,7 +1091,17 @@ int revffn_moe_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weight
                             float* dy1_inout, const revffn_moe_grads* grads, const revffn_moe_sgd* sgd,
                             const int32_t* topk_idx_in, void* ws, size_t ws_bytes, void* cuda_stream) {
   if (!sgd) return REVFFN_ERR_NULL;
-  return entry(PASS_BWD, desc, w, y1, dy2, dy1_inout, grads, topk_idx_in, nullptr, ws, ws_bytes, cuda_stream, sgd);
+  const UpdateSpec u = spec_from_sgd(*sgd);
+  return entry(PASS_BWD, desc, w, y1, dy2, dy1_inout, grads, topk_idx_in, nullptr, ws, ws_bytes, cuda_stream, &u);
+}
+
+int revffn_moe_backward_adam(const revffn_moe_desc* desc, const revffn_moe_weights* w, const float* y1, const float* dy2,
+                             float* dy1_inout, const revffn_moe_grads* grads, const revffn_moe_adam* adam,
+                             const int32_t* topk_idx_in, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!adam) return REVFFN_ERR_NULL;
+  UpdateSpec u;
+  CKR(spec_from_adam(*adam, &u));
+  return entry(PASS_BWD, desc, w, y1, dy2, dy1_inout, grads, topk_idx_in, nullptr, ws, ws_bytes, cuda_stream, &u);
 }
 
 int revffn_moe_quantize_experts(const revffn_moe_desc* desc, const revffn_moe_weights* w, void* cuda_stream) {
@@ -1427,17 +1476,19 @@ int revffn_moe_stack_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_
     float* gR = (l & 1) ? grad_a : grad_b;
     const int32_t* idx =
         topk_idx ? reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(topk_idx) + (size_t)l * idx_stride) : nullptr;
+    UpdateSpec u;
+    if (sgd) u = spec_from_sgd(sgd[l]);
     if (cache) {
       char* c = reinterpret_cast<char*>(cache) + (size_t)l * stride;
       CKR(entry(PASS_BWD, &d_bwd, &weights[l], reinterpret_cast<const float*>(c), gR, gP, &grads[l], idx, nullptr, c + slot,
-                ws_need, cuda_stream, sgd ? &sgd[l] : nullptr));
+                ws_need, cuda_stream, sgd ? &u : nullptr));
     } else {
       // the layer's weights are read for the last time in this step by these two calls (inverse, then the
       // gradient pass, whose weight-gradient products come after every product that reads the same weight),
       // so a fused update of layer l cannot disturb any other layer's reconstruction
       CKR(revffn_moe_inverse(&d_inv, &weights[l], P, R, R, idx, ws, ws_bytes, cuda_stream));
       CKR(entry(PASS_BWD, &d_bwd, &weights[l], P, gR, gP, &grads[l], idx, nullptr, ws, ws_bytes, cuda_stream,
-                sgd ? &sgd[l] : nullptr));
+                sgd ? &u : nullptr));
     }
   }
   return REVFFN_OK;

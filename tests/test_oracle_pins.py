@@ -525,3 +525,28 @@ def test_fp8_experts_is_the_branch_with_quantised_expert_operands():
     y2, _ = orc.forward(p, s["y1"], s["x2"], cfg.top_k, cfg.norm_eps, fp8_experts=True)
     x2, _ = orc.inverse(p, s["y1"], y2, cfg.top_k, cfg.norm_eps, fp8_experts=True)
     assert np.max(np.abs(x2 - s["x2"])) < 1e-10
+
+
+def test_adam_step_is_the_library_optimiser():
+    """adam_step against torch.optim.Adam / AdamW (an independent implementation of the same rule) over three
+    steps with changing gradients, and its first step in closed form: from zero moments the step is
+    -lr * g / (|g| + eps), whatever beta1 and beta2 are."""
+    rng = np.random.default_rng(11)
+    w0 = {"a": rng.standard_normal((5, 7)), "b": rng.standard_normal((3,))}
+    gs = [{n: rng.standard_normal(v.shape) * 10.0 ** rng.integers(-3, 2) for n, v in w0.items()} for _ in range(3)]
+    for wd in (0.0, 0.1):
+        tw = {n: torch.tensor(v.copy(), dtype=torch.float64, requires_grad=True) for n, v in w0.items()}
+        opt = (torch.optim.AdamW if wd else torch.optim.Adam)(list(tw.values()), lr=3e-3, betas=(0.8, 0.95), eps=1e-6,
+                                                              **({"weight_decay": wd} if wd else {}))
+        w, m, v = dict(w0), {}, {}
+        for t, g in enumerate(gs, start=1):
+            for n in tw:
+                tw[n].grad = torch.tensor(g[n], dtype=torch.float64)
+            opt.step()
+            w, m, v = orc.adam_step(w, g, m, v, 3e-3, t, list(w0), beta1=0.8, beta2=0.95, eps=1e-6, weight_decay=wd)
+            for n in w0:
+                assert np.allclose(w[n], tw[n].detach().numpy(), rtol=1e-12, atol=1e-14), (n, t, wd)
+    w1, m1, v1 = orc.adam_step(w0, gs[0], {}, {}, 1e-2, 1, ["a"], beta1=0.3, beta2=0.7, eps=1e-9)
+    g = gs[0]["a"]
+    assert np.allclose(w1["a"] - w0["a"], -1e-2 * g / (np.abs(g) + 1e-9), rtol=1e-9)
+    assert np.allclose(m1["a"], 0.7 * g) and np.allclose(v1["a"], 0.3 * g * g) and w1["b"] is w0["b"]
