@@ -41,16 +41,22 @@ enum { GROUP_NONE = 0, GROUP_M = 1, GROUP_K = 2 };
 // Update rule of a fused optimiser step (EPI_WGRAD with upd_w set).  kind 0: W <- W - lr g.  kind 1: Adam with
 // decoupled weight decay, m <- b1 m + (1 - b1) g, v <- b2 v + (1 - b2) g^2,
 // W <- W - lr (m / c1 / (sqrt(v / c2) + eps) + wd W), c1 = 1 - b1^t, c2 = 1 - b2^t.
-struct UpdRule { int kind; float lr, b1, b2, eps, c1, c2, wd; };
+// The host passes the reciprocals 1 / c1, 1 / c2.
+struct UpdRule { int kind; float lr, b1, b2, eps, inv_c1, inv_c2, wd; };
 
 // One element of the step: returns the new weight; for Adam also rewrites the element's two moments.
+// The square root and the quotient use the hardware approximations (rsqrt, rcp: about 2 ulp, far inside every
+// tolerance of the update): with correctly rounded divisions and square root the element cost about a hundred
+// instructions and the experts' weight-gradient epilogue became arithmetic-bound (4 ms for dW_gate|dW_up).
 __device__ __forceinline__ float upd_step(const UpdRule& r, float w, float g, float* mom, float* var) {
   if (r.kind == 0) return w - r.lr * g;
   const float m = r.b1 * *mom + (1.f - r.b1) * g;
   const float v = r.b2 * *var + (1.f - r.b2) * g * g;
   *mom = m;
   *var = v;
-  return w - r.lr * ((m / r.c1) / (sqrtf(v / r.c2) + r.eps) + r.wd * w);
+  const float vh = v * r.inv_c2;
+  const float root = vh > 0.f ? vh * __frsqrt_rn(vh) : 0.f;
+  return w - r.lr * (__fdividef(m * r.inv_c1, root + r.eps) + r.wd * w);
 }
 
 struct GemmProblem {

@@ -831,10 +831,65 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
         float rs = 1.f;
         if (EPI == EPI_ROWSCALE && m_ok) rs = p.rowscale[m];
         const bool f32_out = (EPI == EPI_COUPLE) || (EPI == EPI_WGRAD) || (EPI == EPI_STORE && p.out_f32);
+        // where this warp's slab of an fp32 result goes
+        const int piece = lane & 7;
+        int64_t y_lim, yb;                                 // row limit and first output row of this warp's slab
+        float* cptr;
+        bf16* wptr;
+        float *mptr, *momptr, *varptr;
+        auto slab_target = [&](const TcTile& tt, int64_t y0_tt) {
+          y_lim = (p.group_mode == GROUP_K) ? (int64_t)(tt.group + 1) * p.M
+                                            : (p.group_mode == GROUP_M ? (int64_t)m_lim : (int64_t)p.M);
+          yb = y0_tt;
+          cptr = reinterpret_cast<float*>(p.C);
+          wptr = reinterpret_cast<bf16*>(p.upd_w);
+          mptr = p.upd_m; momptr = p.upd_mom; varptr = p.upd_var;
+          if (EPI == EPI_WGRAD && p.split_m > 0) {
+            // two outputs: the slab lies wholly in the first or in the second (split_m is a multiple of 128)
+            int local = tt.m0 + q * 32;
+            if (local >= p.split_m) {
+              local -= p.split_m;
+              cptr = reinterpret_cast<float*>(p.C2); wptr = reinterpret_cast<bf16*>(p.upd_w2); mptr = p.upd_m2;
+              momptr = p.upd_mom2; varptr = p.upd_var2;
+            }
+            yb = (int64_t)tt.group * p.split_m + local;
+            y_lim = (int64_t)(tt.group + 1) * p.split_m;
+          }
+        };
+        slab_target(t, y0);
+        // Read-modify-write forms of the weight-gradient epilogue (fused update, accumulation): what the eight
+        // pieces of a block need is requested before the block's accumulator is fetched and staged, and used
+        // after.  Taken piece by piece, each piece's loads waited behind the previous piece's stores (the compiler
+        // cannot tell that they do not overlap) and a 32 x 32 block cost eight memory round trips: the fused SGD
+        // pass measured 2.4 ms slower than writing the gradients.  (Asking the next tile's lines into the L2 a
+        // tile ahead, prefetch.global.L2 per row, changed nothing measurable on top of this.)
+        const bool rmw = EPI == EPI_WGRAD && (wptr != nullptr || p.accumulate);
+        auto as_f4 = [](const uint4& u) {
+          return make_float4(__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w));
+        };
+        auto bf_f4 = [](const uint4& u) {
+          const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.x));
+          const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.y));
+          return make_float4(lo.x, lo.y, hi.x, hi.y);
+        };
 #pragma unroll 1
         for (int c = half * 32; c < t.ncols; c += 64) {
           const int n = t.n0 + c;
           if (!slab_ok) continue;      // warp-uniform
+          const int64_t col = n + piece * 4;
+          uint4 ld[8];          // four floats (stored gradient or master copy), or four bf16 weights in .x, .y
+          if (rmw) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r = i * 4 + (lane >> 3);
+              const int64_t at = (yb + r) * p.ldc + col;
+              if (yb + r < y_lim) {
+                if (!wptr) ld[i] = *reinterpret_cast<const uint4*>(cptr + at);
+                else if (mptr) ld[i] = *reinterpret_cast<const uint4*>(mptr + at);
+                else { const uint2 w2 = *reinterpret_cast<const uint2*>(wptr + at); ld[i].x = w2.x; ld[i].y = w2.y; }
+              }
+            }
+          }
           if (have_acc) { tmem_ld32(taddr + c, r0); tmem_ld_wait(); }
 #pragma unroll
           for (int i = 0; i < 32; ++i) f[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
@@ -870,73 +925,74 @@ gemm_tc_kernel(const __grid_constant__ TcParams P, const __grid_constant__ CUten
                     make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
             }
             __syncwarp();
-            const int piece = lane & 7;
-            int64_t y_lim = (p.group_mode == GROUP_K) ? (int64_t)(t.group + 1) * p.M
-                                                      : (p.group_mode == GROUP_M ? (int64_t)m_lim : (int64_t)p.M);
-            int64_t yb = y0;                                   // first output row of this warp's slab
-            float* cptr = reinterpret_cast<float*>(p.C);
-            bf16* wptr = reinterpret_cast<bf16*>(p.upd_w);
-            float* mptr = p.upd_m;
-            float* momptr = p.upd_mom;
-            float* varptr = p.upd_var;
-            if (EPI == EPI_WGRAD && p.split_m > 0) {
-              // two outputs: the slab lies wholly in the first or in the second (split_m is a multiple of 128)
-              int local = t.m0 + q * 32;
-              if (local >= p.split_m) {
-                local -= p.split_m;
-                cptr = reinterpret_cast<float*>(p.C2); wptr = reinterpret_cast<bf16*>(p.upd_w2); mptr = p.upd_m2;
-                momptr = p.upd_mom2; varptr = p.upd_var2;
-              }
-              yb = (int64_t)t.group * p.split_m + local;
-              y_lim = (int64_t)(t.group + 1) * p.split_m;
-            }
-            const int64_t col = n + piece * 4;
+            if (rmw) {
+              if (wptr && p.upd.kind != 0) {
+                // Adam: the element's two moments live beside the weight (fp32, same layout), 16 bytes each per lane;
+                // two passes of four pieces keep the registers in bounds
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const int r = i * 4 + (lane >> 3);
-              const float4 v = *reinterpret_cast<const float4*>(stg + r * 128 + ((piece ^ (r & 7)) << 4));
-              if (yb + r < y_lim) {
-                const int64_t at = (yb + r) * p.ldc + col;
-                if (EPI == EPI_WGRAD && wptr) {
-                  // fused SGD step on the weight tile this gradient tile belongs to; the gradient is not stored
-                  float4 wv;
-                  if (mptr) {
-                    wv = *reinterpret_cast<const float4*>(mptr + at);
-                  } else {
-                    const uint2 raw = *reinterpret_cast<const uint2*>(wptr + at);
-                    const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-                    const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                    wv = make_float4(lo.x, lo.y, hi.x, hi.y);
+                for (int h4 = 0; h4 < 8; h4 += 4) {
+                  float4 mo[4], va[4];
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    const int r = (h4 + i) * 4 + (lane >> 3);
+                    const int64_t at = (yb + r) * p.ldc + col;
+                    if (yb + r < y_lim) {
+                      mo[i] = *reinterpret_cast<const float4*>(momptr + at);
+                      va[i] = *reinterpret_cast<const float4*>(varptr + at);
+                    }
                   }
-                  if (p.upd.kind == 0) {
-                    wv.x -= p.upd.lr * v.x; wv.y -= p.upd.lr * v.y; wv.z -= p.upd.lr * v.z; wv.w -= p.upd.lr * v.w;
-                  } else {
-                    // Adam: the element's two moments live beside the weight (fp32, same layout): 16 bytes each per lane
-                    float4 mo = *reinterpret_cast<const float4*>(momptr + at);
-                    float4 va = *reinterpret_cast<const float4*>(varptr + at);
-                    wv.x = upd_step(p.upd, wv.x, v.x, &mo.x, &va.x);
-                    wv.y = upd_step(p.upd, wv.y, v.y, &mo.y, &va.y);
-                    wv.z = upd_step(p.upd, wv.z, v.z, &mo.z, &va.z);
-                    wv.w = upd_step(p.upd, wv.w, v.w, &mo.w, &va.w);
-                    *reinterpret_cast<float4*>(momptr + at) = mo;
-                    *reinterpret_cast<float4*>(varptr + at) = va;
-                  }
-                  if (mptr) *reinterpret_cast<float4*>(mptr + at) = wv;
-                  uint2 out;
-                  __nv_bfloat162 h2 = __floats2bfloat162_rn(wv.x, wv.y);
-                  out.x = *reinterpret_cast<uint32_t*>(&h2);
-                  h2 = __floats2bfloat162_rn(wv.z, wv.w);
-                  out.y = *reinterpret_cast<uint32_t*>(&h2);
-                  *reinterpret_cast<uint2*>(wptr + at) = out;
-                } else {
-                  float4* o = reinterpret_cast<float4*>(cptr + at);
-                  if (EPI == EPI_WGRAD && p.accumulate) {
-                    float4 old = *o;
-                    *o = make_float4(old.x + v.x, old.y + v.y, old.z + v.z, old.w + v.w);
-                  } else {
-                    *o = v;
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    const int r = (h4 + i) * 4 + (lane >> 3);
+                    const int64_t at = (yb + r) * p.ldc + col;
+                    if (yb + r >= y_lim) continue;
+                    const float4 v = *reinterpret_cast<const float4*>(stg + r * 128 + ((piece ^ (r & 7)) << 4));
+                    float4 w4 = mptr ? as_f4(ld[h4 + i]) : bf_f4(ld[h4 + i]);
+                    w4.x = upd_step(p.upd, w4.x, v.x, &mo[i].x, &va[i].x);
+                    w4.y = upd_step(p.upd, w4.y, v.y, &mo[i].y, &va[i].y);
+                    w4.z = upd_step(p.upd, w4.z, v.z, &mo[i].z, &va[i].z);
+                    w4.w = upd_step(p.upd, w4.w, v.w, &mo[i].w, &va[i].w);
+                    *reinterpret_cast<float4*>(momptr + at) = mo[i];
+                    *reinterpret_cast<float4*>(varptr + at) = va[i];
+                    if (mptr) *reinterpret_cast<float4*>(mptr + at) = w4;
+                    uint2 out;
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(w4.x, w4.y);
+                    out.x = *reinterpret_cast<uint32_t*>(&h2);
+                    h2 = __floats2bfloat162_rn(w4.z, w4.w);
+                    out.y = *reinterpret_cast<uint32_t*>(&h2);
+                    *reinterpret_cast<uint2*>(wptr + at) = out;
                   }
                 }
+              } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const int r = i * 4 + (lane >> 3);
+                  const int64_t at = (yb + r) * p.ldc + col;
+                  if (yb + r >= y_lim) continue;
+                  const float4 v = *reinterpret_cast<const float4*>(stg + r * 128 + ((piece ^ (r & 7)) << 4));
+                  if (!wptr) {          // accumulate into the stored gradient
+                    const float4 o = as_f4(ld[i]);
+                    *reinterpret_cast<float4*>(cptr + at) = make_float4(o.x + v.x, o.y + v.y, o.z + v.z, o.w + v.w);
+                    continue;
+                  }
+                  // fused SGD step on the weight tile this gradient tile belongs to; the gradient is not stored
+                  float4 w4 = mptr ? as_f4(ld[i]) : bf_f4(ld[i]);
+                  w4.x -= p.upd.lr * v.x; w4.y -= p.upd.lr * v.y; w4.z -= p.upd.lr * v.z; w4.w -= p.upd.lr * v.w;
+                  if (mptr) *reinterpret_cast<float4*>(mptr + at) = w4;
+                  uint2 out;
+                  __nv_bfloat162 h2 = __floats2bfloat162_rn(w4.x, w4.y);
+                  out.x = *reinterpret_cast<uint32_t*>(&h2);
+                  h2 = __floats2bfloat162_rn(w4.z, w4.w);
+                  out.y = *reinterpret_cast<uint32_t*>(&h2);
+                  *reinterpret_cast<uint2*>(wptr + at) = out;
+                }
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int r = i * 4 + (lane >> 3);
+                const float4 v = *reinterpret_cast<const float4*>(stg + r * 128 + ((piece ^ (r & 7)) << 4));
+                if (yb + r < y_lim) *reinterpret_cast<float4*>(cptr + (yb + r) * p.ldc + col) = v;
               }
             }
             __syncwarp();

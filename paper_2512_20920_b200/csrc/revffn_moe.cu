@@ -636,8 +636,8 @@ static int spec_from_adam(const revffn_moe_adam& a, UpdateSpec* u) {
   u->mask = a.mask;
   u->rule.kind = 1;
   u->rule.lr = a.lr; u->rule.b1 = a.beta1; u->rule.b2 = a.beta2; u->rule.eps = a.eps; u->rule.wd = a.weight_decay;
-  u->rule.c1 = (float)(1.0 - pow((double)a.beta1, (double)a.step));
-  u->rule.c2 = (float)(1.0 - pow((double)a.beta2, (double)a.step));
+  u->rule.inv_c1 = (float)(1.0 / (1.0 - pow((double)a.beta1, (double)a.step)));
+  u->rule.inv_c2 = (float)(1.0 / (1.0 - pow((double)a.beta2, (double)a.step)));
   for (int i = 0; i < 8; ++i) {
     u->master[i] = a.master[i]; u->mom[i] = a.mom[i]; u->var[i] = a.var[i];
     if ((a.mask & (1u << i)) && (!a.mom[i] || !a.var[i])) return REVFFN_ERR_NULL;
