@@ -38,10 +38,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # (dram__bytes_read.sum + dram__bytes_write.sum; profiles/tensor_pipe_gemms_C1.md).
 # Keyed by pass/kernel; anything else, or any other workload, reports null.
 NCU_TRAFFIC_BYTES = {
-    "fwd/gemm_expert_gate_up_swiglu": 935_800_000, "inv/gemm_expert_gate_up_swiglu": 1_129_900_000,
-    "fwd/gemm_shared_gate_up_swiglu": 182_800_000, "inv/gemm_shared_gate_up_swiglu": 431_500_000,
-    "bwd/wgrad_expert_gate_up": 1_660_600_000, "bwd/wgrad_expert_down": 878_000_000,
-    "bwd/gemm_expert_du": 1_055_300_000, "bwd/wgrad_shared_gate_up": 427_500_000,
+    "fwd/gemm_expert_gate_up_swiglu": 936_000_000, "inv/gemm_expert_gate_up_swiglu": 1_134_600_000,
+    "fwd/gemm_shared_gate_up_swiglu": 185_100_000, "inv/gemm_shared_gate_up_swiglu": 434_600_000,
+    "bwd/wgrad_expert_gate_up": 1_660_000_000, "bwd/wgrad_expert_down": 871_600_000,
+    "bwd/gemm_expert_du": 1_075_400_000, "bwd/wgrad_shared_gate_up": 425_600_000,
 }
 
 
