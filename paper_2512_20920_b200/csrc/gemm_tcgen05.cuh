@@ -1,7 +1,7 @@
 // tcgen05 / TMEM / TMA back end for every bf16 matrix product on the path.
 //
 // One persistent, warp-specialised kernel (1 CTA per SM, 352 threads):
-//   warps 0, 10 TMA producers: cp.async.bulk.tensor 2D loads (128-byte swizzle) of
+//   warps 0, 10 TMA producers: cp.async.bulk.tensor loads (128-byte swizzle) of
 //               A and B tiles into a ring of shared-memory stages, completion on
 //               mbarriers (no multicast LOADS anywhere: every CTA fetches its own operands; the only
 //               cluster-wide instruction is the pair mode's tcgen05.commit, a barrier arrive).  One thread
@@ -23,8 +23,9 @@
 //               lines whatever the row stride.
 // Tile = 128 rows x 256 columns (the last column tile of a row may be 128 wide: N only has
 // to be a multiple of 128), K step 64 (one 128-byte swizzle atom of bf16).
-// Both operands may be K-major or MN-major; MN-major tiles are fetched as
-// 64x64 boxes and described to the tensor core with leading/stride offsets.
+// Both operands may be K-major or MN-major; MN-major tiles are fetched 128 columns x 64 K rows at a time through a
+// 3-D view of the matrix (64 x 64 boxes of a 2-D map as the fallback) and described to the tensor core with
+// leading/stride offsets.
 // Every wait is bounded; on expiry the kernel sets the status word and leaves.
 //
 // Pair mode (template flag PAIR; dense and K-grouped problems whose N is a multiple of 256, or of 128
