@@ -307,7 +307,8 @@ int revffn_moe_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weight
  * and rewritten in the same epilogue; master[i] is the optional fp32 copy of the weight as in revffn_moe_sgd.
  * Index i is the position of the matrix's REVFFN_UPD_* bit (w_up 0, w_down 1, w_gate 2, w_upx 3, w_downx 4,
  * ws_gate 5, ws_up 6, ws_down 7).  step >= 1 is the caller's step counter.  Everything else (mask rules, which
- * gradients are still written, ordering of reads and updates) is as for revffn_moe_backward_sgd.  The moments
+ * gradients are still written, ordering of reads and updates) is as for revffn_moe_backward_sgd;
+ * revffn_moe_stack_backward_adam is the reversible sweep with one such struct per layer.  The moments
  * add 16 bytes of traffic per element to the 4 of the weight: the fused form saves the gradient's 8 (write, then
  * read by a separate optimiser pass), not the moments'.
  */
@@ -386,6 +387,13 @@ int revffn_moe_stack_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_
                                   float* stream_a, float* stream_b, float* grad_a, float* grad_b,
                                   const revffn_moe_grads* grads, const revffn_moe_sgd* sgd, const int32_t* topk_idx,
                                   void* cache, size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* The reversible sweep with one revffn_moe_adam per layer (HOST array of n_blocks structs): as
+ * revffn_moe_stack_backward_sgd, with the rule of revffn_moe_backward_adam. */
+int revffn_moe_stack_backward_adam(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                                   float* stream_a, float* stream_b, float* grad_a, float* grad_b,
+                                   const revffn_moe_grads* grads, const revffn_moe_adam* adam, const int32_t* topk_idx,
+                                   void* cache, size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Size of one routing record (REVFFN_FLAG_ROUTING_RECORD), a multiple of 16.  (Planner; no paper counterpart.) */
 int revffn_moe_routing_record_bytes(const revffn_moe_desc* desc, size_t* bytes);

@@ -17,7 +17,7 @@ __all__ = ["Block", "Stack", "revffn_moe_saved_size", "revffn_moe_stack_cache_st
            "FLAG_SAVE_ACTIVATIONS", "FLAG_REUSE_ACTIVATIONS", "FLAG_GATE_SOFTMAX_ALL", "FLAG_ROUTING_RECORD",
            "FLAG_KEEP_STATUS", "FLAG_FP8_EXPERTS", "FLAG_STEP_PIPELINED", "FLAG_SINGLE_STREAM", "FLAG_DEBUG_CHECKS", "FLAG_ROUTER_FOLDED", "ERR_DEVICE_WAIT", "ERR_UNSUPPORTED",
            "ERR_NOALLOC_LIMIT", "ERR_INDEX", "Sgd", "make_sgd", "upd_mask", "UPD_NAMES", "UPD_ALL", "stage_update_mask",
-           "revffn_moe_backward_sgd", "revffn_moe_backward_adam", "Adam", "make_adam", "revffn_moe_stack_backward_sgd", "ERR_CANARY", "ERR_NONFINITE", "revffn_dbg_check_guards", "ws_lookup",
+           "revffn_moe_backward_sgd", "revffn_moe_backward_adam", "revffn_moe_stack_backward_adam", "Adam", "make_adam", "revffn_moe_stack_backward_sgd", "ERR_CANARY", "ERR_NONFINITE", "revffn_dbg_check_guards", "ws_lookup",
            "revffn_moe_routing_record_bytes", "AttnBranch", "AttnDesc", "AttnWeights", "AttnGrads",
            "revffn_attn_workspace_size", "revffn_attn_forward", "revffn_attn_inverse", "revffn_attn_backward",
            "revffn_attn_status", "BlockDesc", "RevStack", "revffn_block_workspace_size", "revffn_block_forward",

@@ -157,6 +157,9 @@ def _load() -> C.CDLL:
     lib.revffn_moe_stack_backward_sgd.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp,
                                                   C.POINTER(Grads), C.POINTER(Sgd), vp, vp, sz, vp, sz, vp]
     lib.revffn_moe_stack_backward_sgd.restype = C.c_int
+    lib.revffn_moe_stack_backward_adam.argtypes = [C.POINTER(Desc), C.POINTER(Weights), C.c_int32, vp, vp, vp, vp,
+                                                   C.POINTER(Grads), C.POINTER(Adam), vp, vp, sz, vp, sz, vp]
+    lib.revffn_moe_stack_backward_adam.restype = C.c_int
     lib.revffn_moe_quantize_experts.argtypes = [C.POINTER(Desc), C.POINTER(Weights), vp]
     lib.revffn_moe_quantize_experts.restype = C.c_int
     lib.revffn_moe_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
@@ -358,6 +361,15 @@ def revffn_moe_stack_backward_sgd(desc: Desc, weights, n_blocks: int, stream_a, 
                                              _ptr(grad_a), _ptr(grad_b), grads, sgd, _ptr(topk_idx), _ptr(cache),
                                              _nbytes(cache), _ptr(ws), _nbytes(ws),
                                              stream if stream is not None else _stream()), "revffn_moe_stack_backward_sgd")
+
+
+def revffn_moe_stack_backward_adam(desc: Desc, weights, n_blocks: int, stream_a, stream_b, grad_a, grad_b, grads, adam,
+                                   topk_idx, cache, ws, stream: Optional[int] = None):
+    """`adam`: ctypes array of n_blocks Adam structs."""
+    _check(lib.revffn_moe_stack_backward_adam(C.byref(desc), weights, n_blocks, _ptr(stream_a), _ptr(stream_b),
+                                              _ptr(grad_a), _ptr(grad_b), grads, adam, _ptr(topk_idx), _ptr(cache),
+                                              _nbytes(cache), _ptr(ws), _nbytes(ws),
+                                              stream if stream is not None else _stream()), "revffn_moe_stack_backward_adam")
 
 
 def revffn_prof_enable(on: bool) -> bool:
@@ -751,7 +763,15 @@ class Stack:
         revffn_moe_stack_forward(self.desc, self.w, self.n_blocks, stream_a, stream_b, topk_idx, self.cache, self.ws)
 
     def backward(self, stream_a, stream_b, grad_a, grad_b, grads_array, topk_idx=None, sgd=None):
-        """sgd: list of n_blocks Sgd structs -- one reversible sweep then is one SGD step of the whole stack."""
+        """sgd: list of n_blocks Sgd (or Adam) structs -- one reversible sweep then is one optimiser step of the
+        whole stack."""
+        if sgd is not None and len(sgd) > 0 and isinstance(sgd[0], Adam):
+            if len(sgd) != self.n_blocks:
+                raise ValueError("one Adam struct per layer")
+            arr = (Adam * max(self.n_blocks, 1))(*sgd)
+            revffn_moe_stack_backward_adam(self.desc, self.w, self.n_blocks, stream_a, stream_b, grad_a, grad_b,
+                                           grads_array, arr, topk_idx, self.cache, self.ws)
+            return
         if sgd is not None:
             if len(sgd) != self.n_blocks:
                 raise ValueError("one Sgd struct per layer")

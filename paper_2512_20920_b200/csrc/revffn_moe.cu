@@ -1449,10 +1449,33 @@ int revffn_moe_stack_backward(const revffn_moe_desc* desc, const revffn_moe_weig
                                        cache, cache_bytes, ws, ws_bytes, cuda_stream);
 }
 
+static int stack_backward_impl(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                               float* stream_a, float* stream_b, float* grad_a, float* grad_b,
+                               const revffn_moe_grads* grads, const revffn_moe_sgd* sgd, const revffn_moe_adam* adam,
+                               const int32_t* topk_idx, void* cache, size_t cache_bytes, void* ws, size_t ws_bytes,
+                               void* cuda_stream);
+
 int revffn_moe_stack_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
                                   float* stream_a, float* stream_b, float* grad_a, float* grad_b,
                                   const revffn_moe_grads* grads, const revffn_moe_sgd* sgd, const int32_t* topk_idx,
                                   void* cache, size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return stack_backward_impl(desc, weights, n_blocks, stream_a, stream_b, grad_a, grad_b, grads, sgd, nullptr, topk_idx,
+                             cache, cache_bytes, ws, ws_bytes, cuda_stream);
+}
+
+int revffn_moe_stack_backward_adam(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                                   float* stream_a, float* stream_b, float* grad_a, float* grad_b,
+                                   const revffn_moe_grads* grads, const revffn_moe_adam* adam, const int32_t* topk_idx,
+                                   void* cache, size_t cache_bytes, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return stack_backward_impl(desc, weights, n_blocks, stream_a, stream_b, grad_a, grad_b, grads, nullptr, adam, topk_idx,
+                             cache, cache_bytes, ws, ws_bytes, cuda_stream);
+}
+
+static int stack_backward_impl(const revffn_moe_desc* desc, const revffn_moe_weights* weights, int32_t n_blocks,
+                               float* stream_a, float* stream_b, float* grad_a, float* grad_b,
+                               const revffn_moe_grads* grads, const revffn_moe_sgd* sgd, const revffn_moe_adam* adam,
+                               const int32_t* topk_idx, void* cache, size_t cache_bytes, void* ws, size_t ws_bytes,
+                               void* cuda_stream) {
   int r = validate_desc(desc);
   if (r != REVFFN_OK) return r;
   if (n_blocks < 0) return REVFFN_ERR_SHAPE;
@@ -1478,17 +1501,18 @@ int revffn_moe_stack_backward_sgd(const revffn_moe_desc* desc, const revffn_moe_
         topk_idx ? reinterpret_cast<const int32_t*>(reinterpret_cast<const char*>(topk_idx) + (size_t)l * idx_stride) : nullptr;
     UpdateSpec u;
     if (sgd) u = spec_from_sgd(sgd[l]);
+    if (adam) CKR(spec_from_adam(adam[l], &u));
     if (cache) {
       char* c = reinterpret_cast<char*>(cache) + (size_t)l * stride;
       CKR(entry(PASS_BWD, &d_bwd, &weights[l], reinterpret_cast<const float*>(c), gR, gP, &grads[l], idx, nullptr, c + slot,
-                ws_need, cuda_stream, sgd ? &u : nullptr));
+                ws_need, cuda_stream, (sgd || adam) ? &u : nullptr));
     } else {
       // the layer's weights are read for the last time in this step by these two calls (inverse, then the
       // gradient pass, whose weight-gradient products come after every product that reads the same weight),
       // so a fused update of layer l cannot disturb any other layer's reconstruction
       CKR(revffn_moe_inverse(&d_inv, &weights[l], P, R, R, idx, ws, ws_bytes, cuda_stream));
       CKR(entry(PASS_BWD, &d_bwd, &weights[l], P, gR, gP, &grads[l], idx, nullptr, ws, ws_bytes, cuda_stream,
-                sgd ? &u : nullptr));
+                (sgd || adam) ? &u : nullptr));
     }
   }
   return REVFFN_OK;

@@ -18,7 +18,7 @@ import torch
 from oracle import revffn_oracle as orc
 from workloads import CONFIGS, BlockConfig, make_streams, make_weights, to_bf16_values
 
-from helpers import dev, grad_buffers, make_block, rel_l2
+from helpers import dev, grad_buffers, make_block, rel_l2, to_device_weights
 
 pytestmark = pytest.mark.gpu
 
@@ -136,3 +136,50 @@ def test_fused_adam_argument_checks(rv):
     g_nonzero = m["w_up"].abs() > 1e-6
     assert g_nonzero.float().mean() > 0.9
     assert torch.allclose(moved[g_nonzero], torch.full_like(moved[g_nonzero], 1e-2), rtol=1e-3)
+
+
+def test_reversible_stack_sweep_as_one_adam_step(rv):
+    """Three layers: forward, then the reversible sweep with the fused Adam update per layer.  Every layer's
+    master weights must move as the oracle's adam_step moves them on the gradients of the oracle's reversible
+    back-propagation, and the rebuilt inputs and input gradients must be those of the sweep without updates."""
+    cfg = BlockConfig("U", tokens=210, d_model=256, n_experts=6, top_k=2, d_expert=128, d_shared=256, weight_dtype="bf16")
+    L = 3
+    ws_host = [_weights(cfg, 40 + l) for l in range(L)]
+    weights = [to_device_weights(cfg, w) for w in ws_host]
+    stk = rv.Stack(weights=weights, tokens=cfg.tokens, d_model=cfg.d_model, n_experts=cfg.n_experts, top_k=cfg.top_k,
+                   d_expert=cfg.d_expert, d_shared=cfg.d_shared, weight_dtype=rv.BF16)
+    s = make_streams(cfg, 6)
+    a, b = dev(s["y1"]), dev(s["x2"])
+    idx = torch.empty(L, cfg.tokens, cfg.top_k, dtype=torch.int32, device="cuda")
+    stk.forward(a, b, idx)
+    a_out, b_out = a.clone(), b.clone()
+    g0 = dev(s["dy2"])
+    ga, gb = g0.clone(), g0.clone()
+    stk.backward(a, b, ga, gb, stk.grads_array([{}] * L), topk_idx=idx)                 # the sweep without updates
+    _, _, _, _, grads = orc.stack_backward(ws_host, a_out.cpu().numpy(), b_out.cpu().numpy(), s["dy2"], s["dy2"],
+                                           cfg.top_k, cfg.norm_eps, route_overrides=idx.cpu().numpy())
+    names = list(rv.UPD_NAMES)
+    lr = 0.05 * float(np.sqrt(np.mean(ws_host[0]["w_up"] ** 2)))
+    structs, state = [], []
+    for l in range(L):
+        mom0, var0 = _moments(grads[l], names, 50 + l)
+        mom = {n: dev(mom0[n]) for n in names}
+        var = {n: dev(var0[n]) for n in names}
+        masters = {n: weights[l][n].float().clone() for n in names}
+        w_old = {n: masters[n].cpu().numpy().astype(np.float64) for n in names}
+        structs.append(rv.make_adam(lr, STEP, names, mom, var, masters, beta1=B1, beta2=B2, eps=EPS, weight_decay=WD))
+        state.append((mom0, var0, mom, var, masters, w_old))
+    a2, b2, ga2, gb2 = a_out.clone(), b_out.clone(), g0.clone(), g0.clone()
+    stk.backward(a2, b2, ga2, gb2, stk.grads_array([{}] * L), topk_idx=idx, sgd=structs)
+    assert stk.status() == 0
+    assert torch.equal(a2, a) and torch.equal(b2, b) and torch.equal(ga2, ga) and torch.equal(gb2, gb)
+    for l in range(L):
+        mom0, var0, mom, var, masters, w_old = state[l]
+        new, m_ref, v_ref = orc.adam_step(ws_host[l], grads[l], mom0, var0, lr, STEP, names, beta1=B1, beta2=B2, eps=EPS,
+                                          weight_decay=WD)
+        for n in names:
+            assert rel_l2(mom[n].cpu().numpy(), m_ref[n]) <= TOL_BF16, (l, n)
+            assert rel_l2(var[n].cpu().numpy(), v_ref[n]) <= 2 * TOL_BF16, (l, n)
+            step = masters[n].cpu().numpy().astype(np.float64) - w_old[n]
+            assert rel_l2(step, new[n] - ws_host[l][n]) <= 2 * TOL_BF16, (l, n, rel_l2(step, new[n] - ws_host[l][n]))
+            assert torch.equal(weights[l][n], masters[n].to(torch.bfloat16)), (l, n)
