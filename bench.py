@@ -452,6 +452,40 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
         e2e_sync_value = job_tokens_per_s(world, cfg.tokens, args.steps, dt_sync * 1e3)
         bytes_dir = 3 * hy1.numel() * 4
 
+    # the optimiser step fused into the weight-gradient products (last: it changes the weights, by steps far below
+    # their last bit): inverse + backward with the gradients written, with the fused SGD step, with the fused Adam step
+    fused_rec = None
+    if e2e and cfg.weight_dtype == "bf16" and args.gating == "renorm":
+        names = [n for n in rv.UPD_NAMES if n in blk.weights]
+        rest = {n: t for n, t in grads.items() if n not in names}
+        mom = {n: torch.zeros_like(blk.weights[n], dtype=torch.float32) for n in names}
+        var = {n: torch.zeros_like(blk.weights[n], dtype=torch.float32) for n in names}
+        adam_t = [0]
+
+        def inv_bwd(upd):
+            blk.inverse(y1, y2, x2r, save=True)
+            if upd == "adam":
+                adam_t[0] += 1
+                blk.backward(y1, dy2, dy1, rest, reuse=True, sgd=rv.make_adam(1e-9, adam_t[0], names, mom, var))
+            elif upd == "sgd":
+                blk.backward(y1, dy2, dy1, rest, reuse=True, sgd=rv.make_sgd(1e-9, names))
+            else:
+                blk.backward(y1, dy2, dy1, grads, reuse=True)
+
+        n_f = max(3, min(args.steps, 10))
+        fused_ms = {}
+        for upd in ("none", "sgd", "adam"):
+            inv_bwd(upd)
+            barrier()
+            fused_ms[upd] = timed(lambda: inv_bwd(upd), n_f) / n_f
+        assert blk.status() == 0
+        fused_rec = {"inverse_plus_backward_ms": {"gradients_written": fused_ms["none"], "fused_sgd": fused_ms["sgd"],
+                                                  "fused_adam": fused_ms["adam"]},
+                     "gradient_bytes_not_written": int(sum(blk.weights[n].numel() for n in names) * 4),
+                     "note": "revffn_moe_backward_sgd / revffn_moe_backward_adam with all eight matrices in the mask; "
+                             "not part of the headline step"}
+        del mom, var
+
     if rank != 0:
         return None
 
@@ -578,6 +612,7 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
                                  "peak": peak_name, "ms_per_step": g_ms / args.steps},
         "kernels": top,
         "fp8_experts": fp8_rec,
+        "fused_update": fused_rec,
         "roofline": roofline,
         "cpu_baseline": cpu_rec,
         "e2e": ({"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": bytes_dir,
