@@ -455,6 +455,7 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
     # the optimiser step fused into the weight-gradient products (last: it changes the weights, by steps far below
     # their last bit): inverse + backward with the gradients written, with the fused SGD step, with the fused Adam step
     fused_rec = None
+    peak_device_bytes = int(torch.cuda.max_memory_allocated())      # before the moment buffers of the Adam leg
     if e2e and cfg.weight_dtype == "bf16" and args.gating == "renorm":
         names = [n for n in rv.UPD_NAMES if n in blk.weights]
         rest = {n: t for n, t in grads.items() if n not in names}
@@ -626,7 +627,7 @@ def measure_block(args, cfg, e2e=True, cpu=True, w_dev=None, w_host=None, steps_
         "gpu_launches": int(launches),
         "clocks": clocks,
         "clocks_per_kernel_pass": clocks_prof,
-        "peak_device_bytes": int(torch.cuda.max_memory_allocated()),
+        "peak_device_bytes": peak_device_bytes,
         "workspace_bytes": {"fwd": blk.fwd_bytes, "bwd": blk.bwd_bytes},
     }
     # achieved GB/s of the copy-like kernels (algorithmic bytes: rows read + rows written)
