@@ -32,10 +32,9 @@
  *     revffn_moe_status, which synchronises the given stream.
  *   - Work is enqueued on the caller's CUDA stream (cudaStream_t passed as
  *     void*), and the call is asynchronous on it: what the caller queues on that
- *     stream afterwards follows everything of the call.  Inside a call of 1024
- *     tokens or more on the tcgen05 back end, launches that nothing later in the
- *     pass depends on run on a second stream that the library creates per device
- *     on its first such call (with a ring of events that order it against the
+ *     stream afterwards follows everything of the call.  Inside a call on the
+ *     tcgen05 back end, launches that nothing later in the pass depends on run on a second stream that the library creates per device
+ *     on its first call (with a ring of events that order it against the
  *     caller's stream); REVFFN_FLAG_SINGLE_STREAM keeps every launch on the
  *     caller's stream.  The results are the same bits either way.  The pipelined
  *     host step (REVFFN_FLAG_STEP_PIPELINED) owns one more stream, for uploads.
@@ -150,8 +149,7 @@ enum { REVFFN_NORM_RMS = 0, REVFFN_NORM_NONE = 1 }; /* norm_kind                
 /* revffn_moe_step_host only: the pipelined form described there (two staging sets used in turn, results
  * complete when the copy stream completes).  Other entry points ignore it. */
 #define REVFFN_FLAG_STEP_PIPELINED 512u
-/* Keep every launch of the call on cuda_stream.  Without it, calls of 1024 tokens or more on the tcgen05 back end
- * put launches that nothing later in the pass depends on (the shared expert beside the routed experts, the weight
+/* Keep every launch of the call on cuda_stream.  Without it, calls on the tcgen05 back end put launches that nothing later in the pass depends on (the shared expert beside the routed experts, the weight
  * gradients beside the input gradients) on a second stream that the library creates per device on first use,
  * ordered against cuda_stream by events; cuda_stream still ends after everything of the call, and the results
  * are the same bits either way. */

@@ -955,9 +955,9 @@ static int dispatch(Pass pass, const revffn_moe_desc& D, const revffn_moe_weight
   c.D = D; c.W = W; c.L = L; c.ws = reinterpret_cast<char*>(ws); c.st = st;
   g_prof.pass = (int)pass;
   c.tc = std::is_same<T, bf16>::value && !(D.flags & REVFFN_FLAG_FORCE_SIMT);
-  // second stream: only where the launches are long enough for their last rounds to matter, and never while the
-  // per-launch profiler is on (its events bracket launches on one stream)
-  if (c.tc && !g_prof.on && !(D.flags & REVFFN_FLAG_SINGLE_STREAM) && D.tokens >= 1024) {
+  // second stream: every call on the tcgen05 back end (at 512 tokens, where the launches are short, the step still
+  // gains 13 %), never while the per-launch profiler is on (its events bracket launches on one stream)
+  if (c.tc && !g_prof.on && !(D.flags & REVFFN_FLAG_SINGLE_STREAM)) {
     c.ov = overlap_state();
     if (!c.ov) return REVFFN_ERR_CUDA;
   }

@@ -100,8 +100,8 @@ def test_fused_adam_matches_oracle_gradients_and_step(rv, simt):
 
 
 def test_fused_adam_on_the_second_stream_and_a_partial_mask(rv):
-    """1300 tokens: the weight-gradient products run on the library's second stream; only the experts and one
-    adapter are in the mask, the other gradients are written as usual."""
+    """A larger batch (the weight-gradient products run on the library's second stream, as in every tensor-core
+    case); only the experts and one adapter are in the mask, the other gradients are written as usual."""
     cfg = BlockConfig("U", tokens=1300, d_model=256, n_experts=5, top_k=2, d_expert=128, d_shared=256, weight_dtype="bf16")
     w, s = _weights(cfg, 32), make_streams(cfg, 32)
     _run(rv, cfg, w, s, ["w_up", "w_gate", "w_upx", "w_downx"], TOL_BF16)

@@ -259,8 +259,9 @@ def test_backward_reuses_a_saved_evaluation(rv, simt):
 
 @pytest.mark.parametrize("gating", ["renorm", "softmax_all"])
 def test_all_passes_with_the_second_stream(rv, gating):
-    """From 1024 tokens on, the tensor-core back end puts the router, the shared expert and the weight gradients on
-    a second stream of the library's own: the same parity as everywhere else, at a size the oracle does in full."""
+    """The tensor-core back end puts the router, the shared expert and the weight gradients on a second stream of
+    the library's own (every tensor-core case in this file runs that way): the same parity at the largest size the
+    oracle does in full, with both gate conventions."""
     cfg = small_cfg(tokens=1300, n_experts=7, top_k=3)
     w, s = scaled_weights(cfg, 12, 4.0), make_streams(cfg, 12)
     run_all_passes(rv, cfg, w, s, TOL_BF16, gating=gating)
