@@ -787,12 +787,15 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       }
     }
     if (G.ws_sgate) {
-      { ProfScope ps(TG_WG_SGATE, st);
+      // a leaf like the matrix gradients: second stream (which also owns the column-sum scratch `part`: every
+      // user of it, this one, the router bias and the norm scale, is queued there, in order)
+      CKR(c.order(st, cw.st));
+      { ProfScope ps(TG_WG_SGATE, cw.st);
       CK(launch_colsum_partial<T>(c.template p<T>(L.u), d, c.template p<float>(L.dl), Tn, d, STRIP, L.strips,
-                                  c.template p<float>(L.part), st));
+                                  c.template p<float>(L.part), cw.st));
       }
-      { ProfScope ps(TG_WG_SGATE, st);
-      colsum_final_kernel<<<(unsigned)ceil_div(d, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), L.strips, d, acc,
+      { ProfScope ps(TG_WG_SGATE, cw.st);
+      colsum_final_kernel<<<(unsigned)ceil_div(d, COLSUM_FINAL_COLS), 256, 0, cw.st>>>(c.template p<float>(L.part), L.strips, d, acc,
                                                                       G.ws_sgate);
       }
       CK(cudaGetLastError());
@@ -859,8 +862,9 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     CK(cudaGetLastError());
     if (G.w_router || G.b_router) {
       dim3 grid((unsigned)ceil_div(d, 256), (unsigned)E);
-      { ProfScope ps(TG_WG_ROUTER, st);
-      router_wgrad_kernel<T><<<grid, 256, 0, st>>>(c.template p<T>(L.up), c.template p<float>(L.row_dl),
+      CKR(c.order(st, cw.st));
+      { ProfScope ps(TG_WG_ROUTER, cw.st);
+      router_wgrad_kernel<T><<<grid, 256, 0, cw.st>>>(c.template p<T>(L.up), c.template p<float>(L.row_dl),
                                                    c.template p<int32_t>(L.expert_off), c.template p<int32_t>(L.expert_cnt),
                                                    d, acc, G.w_router, G.b_router);
       }
@@ -886,12 +890,13 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
       CKR(wgrad(TG_WG_ROUTER, 0u, G.w_router, nullptr, nullptr, E, d, c.template p<T>(L.dlf), L.ld_dlf, 0, c.template p<T>(L.u), d,
                 false, 0));
     if (G.b_router) {
-      { ProfScope ps(TG_WG_ROUTER, st);
+      CKR(c.order(st, cw.st));
+      { ProfScope ps(TG_WG_ROUTER, cw.st);
       CK(launch_colsum_partial<T>(c.template p<T>(L.dlf), L.ld_dlf, nullptr, Tn, E, STRIP, L.strips,
-                                  c.template p<float>(L.part), st));
+                                  c.template p<float>(L.part), cw.st));
       }
-      { ProfScope ps(TG_WG_ROUTER, st);
-      colsum_final_kernel<<<(unsigned)ceil_div(E, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), L.strips, E, acc,
+      { ProfScope ps(TG_WG_ROUTER, cw.st);
+      colsum_final_kernel<<<(unsigned)ceil_div(E, COLSUM_FINAL_COLS), 256, 0, cw.st>>>(c.template p<float>(L.part), L.strips, E, acc,
                                                                       G.b_router);
       }
       CK(cudaGetLastError());
@@ -927,12 +932,13 @@ static int run_backward(const Ctx<T>& c, const float* y1, const float* dy2, floa
     if (norm_none) {
       if (!acc) CK(cudaMemsetAsync(G.norm_gamma, 0, (size_t)h * 4, st));
     } else {
-      { ProfScope ps(TG_DGAMMA, st);
+      CKR(c.order(st, cw.st));
+      { ProfScope ps(TG_DGAMMA, cw.st);
       CK(launch_dgamma_partial(c.template p<float>(L.dn), y1, D.ld_stream, c.template p<float>(L.r), Tn, h, STRIP, L.strips,
-                               c.template p<float>(L.part), st));
+                               c.template p<float>(L.part), cw.st));
       }
-      { ProfScope ps(TG_DGAMMA, st);
-      colsum_final_kernel<<<(unsigned)ceil_div(h, COLSUM_FINAL_COLS), 256, 0, st>>>(c.template p<float>(L.part), L.strips, h, acc,
+      { ProfScope ps(TG_DGAMMA, cw.st);
+      colsum_final_kernel<<<(unsigned)ceil_div(h, COLSUM_FINAL_COLS), 256, 0, cw.st>>>(c.template p<float>(L.part), L.strips, h, acc,
                                                                       G.norm_gamma);
       }
       CK(cudaGetLastError());
