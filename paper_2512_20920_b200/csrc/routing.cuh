@@ -613,7 +613,8 @@ __global__ void map_scan_kernel(const int32_t* __restrict__ chunk_cnt, int n_chu
     // Token chunks for the products that put tokens on the MMA N side: per expert, runs of up to
     // TOK_CHUNK rows covering its real rows rounded up to 32 (the rounding stays inside the expert's
     // zero padding).  Entry = (expert, first row, rows, 0); the count goes to rows_total[1].
-    // (Runs of equal length, 3 x 192 instead of 256 + 256 + 64 for 546 rows, measured 1-2 % slower.)
+    // (Runs of equal length, 3 x 192 instead of 256 + 256 + 64 for 546 rows, stay within 2 % either way: the two
+    // products that use the table measured 2 % faster alone and the whole step 1-2 % slower.)
     int nc = 0;
     for (int e = 0; e < E; ++e) {
       const int n = (int)round_up(expert_cnt[e], 32);
